@@ -1,0 +1,205 @@
+"""ctypes front-end of the CPU oracle (oracle/osc_oracle.c).
+
+TEST INFRASTRUCTURE ONLY: imported by tests/, the smoke check and the bench's
+cpu-baseline leg.  The CUDA package never imports this module and this module
+never imports the CUDA package.  All arguments and results are numpy arrays in
+host memory; bf16 tensors are uint16 bit patterns.
+
+Function-to-paper map (details in the C file):
+  quantize_extract / prepare_weights  Algorithm 2 (+ Section 3.3 weight split)
+  gemm_dual / linear                   Eq. 5
+  fp8_quantize / fp8_gemm / fp8_linear Section 3.4 fallback
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "osc_oracle.c")
+_LIB = os.path.join(_HERE, "libosc_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (no fast-math, no FMA contraction)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        subprocess.check_call(["gcc", "-O2", "-ffp-contract=off", "-fopenmp", "-fPIC", "-shared",
+                               "-o", _LIB, _SRC, "-lm"])
+    return _LIB
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(build())
+        _lib.osc_ref_e2m1_decode.restype = C.c_double
+        _lib.osc_ref_e2m1_decode.argtypes = [C.c_int]
+        _lib.osc_ref_e2m1_encode.argtypes = [C.c_double]
+        _lib.osc_ref_e4m3_decode.restype = C.c_double
+        _lib.osc_ref_e4m3_decode.argtypes = [C.c_int]
+        _lib.osc_ref_e4m3_encode.argtypes = [C.c_double]
+        _lib.osc_ref_e8m0_from_amax.argtypes = [C.c_double]
+        _lib.osc_ref_sf_index.restype = C.c_int64
+        _lib.osc_ref_sf_index.argtypes = [C.c_int64, C.c_int64, C.c_int64]
+        _lib.osc_ref_sf_bytes.restype = C.c_int64
+        _lib.osc_ref_sf_bytes.argtypes = [C.c_int64, C.c_int64]
+        _lib.osc_ref_sf_row_base.restype = C.c_int64
+    return _lib
+
+
+def _p(a):
+    return a.ctypes.data_as(C.c_void_p)
+
+
+def num_threads() -> int:
+    return int(lib().osc_ref_num_threads())
+
+
+def e2m1_encode(v: float) -> int:
+    return int(lib().osc_ref_e2m1_encode(float(v)))
+
+
+def e2m1_decode(n: int) -> float:
+    return float(lib().osc_ref_e2m1_decode(int(n)))
+
+
+def e4m3_encode(v: float) -> int:
+    return int(lib().osc_ref_e4m3_encode(float(v)))
+
+
+def e4m3_decode(b: int) -> float:
+    return float(lib().osc_ref_e4m3_decode(int(b)))
+
+
+def e8m0_from_amax(a: float) -> int:
+    return int(lib().osc_ref_e8m0_from_amax(float(a)))
+
+
+def sf_index(r: int, g: int, K: int) -> int:
+    return int(lib().osc_ref_sf_index(r, g, K))
+
+
+def sf_bytes(rows: int, K: int) -> int:
+    return int(lib().osc_ref_sf_bytes(rows, K))
+
+
+def lut_normalize(lut: np.ndarray, K: int):
+    """-> (K_o, K_o_pad, mask u32[Kg], prefix i32[Kg], idx_o i32[K_o]); raises on a bad table."""
+    lut = np.ascontiguousarray(lut, dtype=np.int8)
+    Kg = K // 32
+    if lut.ndim == 1:
+        lut = lut.reshape(Kg, -1)
+    assert lut.shape[0] == Kg
+    mask = np.zeros(Kg, np.uint32)
+    prefix = np.zeros(Kg, np.int32)
+    idx = np.zeros(max(K, 1), np.int32)
+    ko = lib().osc_ref_lut_normalize(_p(lut), Kg, lut.shape[1], _p(mask), _p(prefix), _p(idx))
+    if ko < 0:
+        raise ValueError({-1: "lookup-table entry outside -1..31", -2: "duplicate channel in a group"}[ko])
+    return ko, int(lib().osc_ref_ko_pad(ko)), mask, prefix, idx[:ko].copy()
+
+
+def quantize_extract(X: np.ndarray, lut: np.ndarray):
+    """Algorithm 2 on bf16 rows X [M,K] -> dict(xq [M,K/2] u8, sf u8 (block layout), xo [M,K_o_pad] u16)."""
+    X = np.ascontiguousarray(X, dtype=np.uint16)
+    M, K = X.shape
+    lut = np.ascontiguousarray(lut, dtype=np.int8).reshape(K // 32, -1)
+    ko, kop, mask, prefix, idx = lut_normalize(lut, K)
+    xq = np.zeros((M, K // 2), np.uint8)
+    sf = np.zeros(sf_bytes(M, K), np.uint8)
+    xo = np.zeros((M, kop), np.uint16)
+    rc = lib().osc_ref_quantize_extract(_p(X), C.c_int64(K), M, K, _p(lut), lut.shape[1], _p(xq), _p(sf), _p(xo))
+    assert rc == ko
+    return {"xq": xq, "sf": sf, "xo": xo, "K_o": ko, "K_o_pad": kop, "mask": mask, "prefix": prefix, "idx_o": idx}
+
+
+def prepare_weights(W: np.ndarray, lut: np.ndarray):
+    """Offline weight split (Section 3.3): the same routine on the rows of W [N,K]."""
+    return quantize_extract(W, lut)
+
+
+def sf_row_base(off: np.ndarray):
+    off = np.ascontiguousarray(off, dtype=np.int32)
+    E = off.size - 1
+    base = np.zeros(max(E, 1), np.int64)
+    total = lib().osc_ref_sf_row_base(_p(off), E, _p(base))
+    return base[:E], int(total)
+
+
+def quantize_extract_grouped(X: np.ndarray, off: np.ndarray, lut: np.ndarray):
+    X = np.ascontiguousarray(X, dtype=np.uint16)
+    off = np.ascontiguousarray(off, dtype=np.int32)
+    M, K = X.shape
+    E = off.size - 1
+    lut = np.ascontiguousarray(lut, dtype=np.int8).reshape(K // 32, -1)
+    ko, kop, mask, prefix, idx = lut_normalize(lut, K)
+    base, total = sf_row_base(off)
+    xq = np.zeros((M, K // 2), np.uint8)
+    sf = np.zeros(sf_bytes(total, K), np.uint8)
+    xo = np.zeros((M, kop), np.uint16)
+    rc = lib().osc_ref_quantize_extract_grouped(_p(X), C.c_int64(K), _p(off), E, K, _p(lut), lut.shape[1],
+                                                _p(xq), _p(sf), _p(xo), kop)
+    assert rc >= 0
+    return {"xq": xq, "sf": sf, "xo": xo, "K_o": ko, "K_o_pad": kop, "sf_row_base": base, "sf_rows": total}
+
+
+def gemm_dual(act: dict, wts: dict, rows=None, sf_rows=None):
+    """Eq. 5 for the listed activation rows (all rows if None) -> (Y, T) float64 [nrows, N]."""
+    xq, sfa, xo = act["xq"], act["sf"], act["xo"]
+    wq, sfw, wo = wts["xq"], wts["sf"], wts["xo"]
+    M, K2 = xq.shape
+    K = 2 * K2
+    N = wq.shape[0]
+    kop = xo.shape[1]
+    assert wq.shape[1] == K2 and wo.shape[1] == kop
+    if rows is None:
+        rows = np.arange(M, dtype=np.int32)
+    rows = np.ascontiguousarray(rows, dtype=np.int32)
+    sf_rows = rows if sf_rows is None else np.ascontiguousarray(sf_rows, dtype=np.int32)
+    Y = np.zeros((rows.size, N), np.float64)
+    T = np.zeros((rows.size, N), np.float64)
+    lib().osc_ref_gemm_dual_rows(_p(xq), _p(sfa), _p(xo), _p(rows), _p(sf_rows), rows.size,
+                                 _p(wq), _p(sfw), _p(wo), N, K, kop, _p(Y), _p(T))
+    return Y, T
+
+
+def linear(X: np.ndarray, W: np.ndarray, lut: np.ndarray, rows=None):
+    """The whole OSC linear: Algorithm 2 on X, weight split on W, Eq. 5."""
+    act = quantize_extract(X, lut)
+    wts = prepare_weights(W, lut)
+    Y, T = gemm_dual(act, wts, rows)
+    return Y, T, act, wts
+
+
+def fp8_quantize(X: np.ndarray):
+    X = np.ascontiguousarray(X, dtype=np.uint16)
+    M, K = X.shape
+    x8 = np.zeros((M, K), np.uint8)
+    sx = np.zeros(M, np.float32)
+    lib().osc_ref_fp8_quantize(_p(X), C.c_int64(K), M, K, _p(x8), _p(sx))
+    return x8, sx
+
+
+def fp8_gemm(x8, sx, w8, sw, rows=None):
+    M, K = x8.shape
+    N = w8.shape[0]
+    if rows is None:
+        rows = np.arange(M, dtype=np.int32)
+    rows = np.ascontiguousarray(rows, dtype=np.int32)
+    Y = np.zeros((rows.size, N), np.float64)
+    T = np.zeros((rows.size, N), np.float64)
+    lib().osc_ref_fp8_gemm_rows(_p(np.ascontiguousarray(x8)), _p(np.ascontiguousarray(sx, dtype=np.float32)),
+                                _p(rows), rows.size, _p(np.ascontiguousarray(w8)),
+                                _p(np.ascontiguousarray(sw, dtype=np.float32)), N, K, _p(Y), _p(T))
+    return Y, T
+
+
+def fp8_linear(X: np.ndarray, W: np.ndarray, rows=None):
+    x8, sx = fp8_quantize(X)
+    w8, sw = fp8_quantize(W)
+    Y, T = fp8_gemm(x8, sx, w8, sw, rows)
+    return Y, T, (x8, sx), (w8, sw)
