@@ -1,0 +1,179 @@
+/*
+ * osc.h - C ABI of the B200 (sm_100a) OSC dual-path quantized linear layer.
+ *
+ * The calls follow the paper's statement of the problem:
+ *   offline  : suppression table + weight split            (Section 3.1; Section 3.3 "offline weight quantization")
+ *   online   : OSC-enhanced quantization                   (Algorithm 2)
+ *              dual-path GEMM  Y = (Q_X (x) Q_W).S + B.W_L (Eq. 5)
+ *   fallback : FP8 W8A8 linear for the down-projection     (Section 3.4)
+ *   grouped  : the same linears per MoE expert             (Section 4.1, Qwen3-30B-A3B: 128 experts, 8 active)
+ *
+ * Conventions
+ *   - Plain C, no exceptions cross the boundary.  Every call returns an osc_status
+ *     (0 = success, negative = error); osc_last_error() gives a thread-local detail string.
+ *   - "dev" pointers are device (HBM) addresses, "host" pointers are host addresses.
+ *     The caller owns every device buffer.  The library allocates no device memory and keeps
+ *     only small host handles (shapes, borrowed device pointers, TMA descriptors) created by
+ *     *_prepare_* and released by *_destroy.
+ *   - stream is a cudaStream_t passed as void*.  All work is enqueued on it; no call
+ *     synchronizes except osc_sync_check.  A failed validation launches nothing.
+ *   - Tensors: X bf16 [M, K] row-major (K contiguous, leading dimension ldx elements);
+ *     W bf16 [N, K] row-major (the nn.Linear layout, Y = X . W^T); Y bf16 [M, N] (ldy elements).
+ *   - Shape preconditions: K % 128 == 0, N % 64 == 0, M >= 0 (M == 0 is a successful no-op),
+ *     device pointers 16-byte aligned, leading dimensions multiples of 8 elements.
+ *   - Group size G = 32 (MXFP4).  The suppression table is lut[K/32][lut_c] int8 on the host:
+ *     local channel index 0..31 or -1 (no channel).  lut_c = 1 is the paper's one channel per
+ *     group; larger lut_c protects up to lut_c channels per group.
+ *
+ * Data layouts written by the library (and accepted back by osc_gemm_dual)
+ *   xq / wq  : packed E2M1 codes, [rows, K/2] bytes, element 2i in bits 3:0 and 2i+1 in bits 7:4.
+ *   sfa / sfw: E8M0 scale bytes, one per (row, 32-group), in 512-byte blocks of 128 rows x 4 groups:
+ *              offset(r, g) = ((r/128)*(K/128) + g/4)*512 + (r%32)*16 + ((r%128)/32)*4 + g%4.
+ *              Bytes of rows >= the row count are written as 0.
+ *   xo / wo  : the protected channels, bf16 [rows, K_o_pad], ascending channel order,
+ *              K_o_pad = roundup(K_o, 64), pad columns +0.
+ *   meta     : uint32 mask[K/32], int32 prefix[K/32], int32 idx_o[K_o] (device copy of the table).
+ *   x8 / w8  : E4M3 bytes [rows, K]; sx / sw: fp32 per-row scales (amax/448).
+ */
+#ifndef OSC_H_
+#define OSC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int osc_status;
+enum {
+    OSC_OK = 0,
+    OSC_ERR_INVALID_ARG = -1, /* null pointer, negative size, bad handle */
+    OSC_ERR_SHAPE = -2,       /* K % 128, N % 64, leading dimension too small */
+    OSC_ERR_LUT = -3,         /* table entry outside -1..31 or duplicated inside a group */
+    OSC_ERR_ALIGN = -4,       /* pointer not 16-byte aligned / leading dimension not a multiple of 8 */
+    OSC_ERR_WORKSPACE = -5,   /* workspace smaller than osc_*_act_sizes reports */
+    OSC_ERR_ARCH = -6,        /* current device is not compute capability 10.x */
+    OSC_ERR_CUDA = -7,        /* a CUDA runtime / driver call failed (detail in osc_last_error) */
+    OSC_ERR_TIMEOUT = -8      /* a device-side wait gave up (reported by osc_sync_check) */
+};
+
+const char* osc_status_string(osc_status s);
+const char* osc_last_error(void);
+
+/* Waits for `stream` and reports OSC_ERR_TIMEOUT if any kernel of this library gave up on a
+ * bounded device-side wait since the last check (the flag is cleared), OSC_ERR_CUDA if the
+ * stream is in error, else OSC_OK.  Test / debugging aid; never needed on the hot path. */
+osc_status osc_sync_check(void* stream);
+
+/* ------------------------------------------------------------------ OSC path */
+
+typedef struct osc_weights osc_weights; /* opaque host handle */
+
+typedef struct {
+    int32_t K_o;      /* protected channels listed in the table */
+    int32_t K_o_pad;  /* roundup(K_o, 64) */
+    size_t wq_bytes;  /* E * N * K/2 */
+    size_t sfw_bytes; /* E * ceil(N/128) * (K/128) * 512 */
+    size_t wo_bytes;  /* E * N * K_o_pad * 2 (0 when the table is empty) */
+    size_t meta_bytes;
+} osc_weight_sizes_t;
+
+typedef struct {
+    size_t xq_bytes;        /* M * K/2 */
+    size_t sfa_bytes;       /* 512-byte scale blocks: ceil(M/128) row blocks (grouped: M/128 + E) x K/128 */
+    size_t xo_bytes;        /* M * K_o_pad * 2 */
+    size_t sched_bytes;     /* grouped only: device-built tile schedule */
+    size_t xq_offset;       /* where osc_linear[_grouped] places each buffer inside its workspace */
+    size_t sfa_offset;
+    size_t xo_offset;
+    size_t sched_offset;
+    size_t workspace_bytes; /* total workspace osc_linear[_grouped] needs (each part 256-byte aligned) */
+} osc_act_sizes_t;
+
+/* Sizes of the buffers osc_prepare_weights[_grouped] fills (Section 3.3: FP4 weights plus
+ * the gathered high-precision rows).  E = number of experts (1 for a dense layer).
+ * lut: host [K/32][lut_c]. */
+osc_status osc_weight_sizes(int E, int N, int K, const int8_t* lut, int lut_c, osc_weight_sizes_t* out);
+
+/* Offline weight split (Section 3.3, first bullet; table semantics of Section 3.1):
+ * W_o = W[:, idx_o]; W_r = W with those columns zeroed; (wq, sfw) = MXFP4(W_r).
+ * W: dev bf16 [N, ldw].  wq/sfw/wo/meta: dev, caller-allocated with the sizes above; the
+ * handle borrows them and they must outlive it.  Work is enqueued on `stream`. */
+osc_status osc_prepare_weights(const void* W, int N, int K, int64_t ldw, const int8_t* lut, int lut_c,
+                               void* wq, void* sfw, void* wo, void* meta, void* stream, osc_weights** out);
+
+/* Same for E experts stacked as W[E][N][K] (dense, ldw = K); one table shared by all experts
+ * of the layer; wq/sfw/wo are stacked per expert in the same order. */
+osc_status osc_prepare_weights_grouped(const void* W, int E, int N, int K, const int8_t* lut, int lut_c,
+                                       void* wq, void* sfw, void* wo, void* meta, void* stream,
+                                       osc_weights** out);
+
+osc_status osc_weights_destroy(osc_weights* w);
+
+/* Buffer sizes for M activation rows (dense) or M_total rows in at most E expert segments (grouped). */
+osc_status osc_act_sizes(const osc_weights* w, int M, osc_act_sizes_t* out);
+
+/* Algorithm 2, fused: index lookup, back-up of the flagged channels into xo (the buffer B),
+ * zero-out, CalculateScale, Quantize.  X: dev bf16 [M, ldx]. */
+osc_status osc_quantize_extract(const osc_weights* w, const void* X, int M, int64_t ldx,
+                                void* xq, void* sfa, void* xo, void* stream);
+
+/* Eq. 5 on pre-quantized activations: block-scaled FP4 path and BF16 bypass path accumulate
+ * into one fp32 tile; Y = bf16(acc).  Y: dev bf16 [M, ldy]. */
+osc_status osc_gemm_dual(const osc_weights* w, const void* xq, const void* sfa, const void* xo, int M,
+                         void* Y, int64_t ldy, void* stream);
+
+/* osc_quantize_extract followed by osc_gemm_dual; workspace (dev) holds xq/sfa/xo. */
+osc_status osc_linear(const osc_weights* w, const void* X, int M, int64_t ldx, void* Y, int64_t ldy,
+                      void* workspace, size_t workspace_bytes, void* stream);
+
+/* Grouped (MoE) form: rows of X_perm are sorted by expert, expert e owns rows
+ * [off[e], off[e+1]); off: dev int32 [E+1], off[E] == M_total.  Expert e's scale rows start
+ * at scale row sum_{e'<e} roundup(m_e', 128).  The tile schedule is built on the device. */
+osc_status osc_linear_grouped(const osc_weights* w, const void* X_perm, const int32_t* off, int M_total,
+                              int64_t ldx, void* Y, int64_t ldy, void* workspace, size_t workspace_bytes,
+                              void* stream);
+
+/* ------------------------------------------------------------- FP8 fallback */
+
+typedef struct osc_fp8_weights osc_fp8_weights;
+
+typedef struct {
+    size_t x8_bytes;        /* M * K */
+    size_t sx_bytes;        /* M * 4 */
+    size_t sched_bytes;     /* grouped only */
+    size_t x8_offset;       /* placement inside the workspace of osc_fp8_linear[_grouped] */
+    size_t sx_offset;
+    size_t sched_offset;
+    size_t workspace_bytes;
+} osc_fp8_act_sizes_t;
+
+/* Section 3.4: the W2 / down-projection runs in FP8.  Offline: per output row n,
+ * sw[n] = max(amax_n, 2^-40)/448 and w8 = E4M3(W * 448/max(amax_n, 2^-40)) (nearest-even, saturating).
+ * w8: dev [E*N*K] bytes, sw: dev fp32 [E*N]. */
+osc_status osc_fp8_prepare_weights(const void* W, int N, int K, int64_t ldw, void* w8, void* sw,
+                                   void* stream, osc_fp8_weights** out);
+osc_status osc_fp8_prepare_weights_grouped(const void* W, int E, int N, int K, void* w8, void* sw,
+                                           void* stream, osc_fp8_weights** out);
+osc_status osc_fp8_weights_destroy(osc_fp8_weights* w);
+osc_status osc_fp8_act_sizes(const osc_fp8_weights* w, int M, osc_fp8_act_sizes_t* out);
+
+/* Per-token dynamic E4M3 quantization: sx[m] and x8[m,:] as above, per activation row. */
+osc_status osc_fp8_quantize(const void* X, int M, int K, int64_t ldx, void* x8, void* sx, void* stream);
+
+/* Y[m,n] = bf16(sx[m] * sw[n] * sum_k x8[m,k] * w8[n,k]), fp32 accumulation. */
+osc_status osc_fp8_gemm(const osc_fp8_weights* w, const void* x8, const void* sx, int M, void* Y,
+                        int64_t ldy, void* stream);
+
+osc_status osc_fp8_linear(const osc_fp8_weights* w, const void* X, int M, int64_t ldx, void* Y, int64_t ldy,
+                          void* workspace, size_t workspace_bytes, void* stream);
+
+osc_status osc_fp8_linear_grouped(const osc_fp8_weights* w, const void* X_perm, const int32_t* off,
+                                  int M_total, int64_t ldx, void* Y, int64_t ldy, void* workspace,
+                                  size_t workspace_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* OSC_H_ */

@@ -1,0 +1,279 @@
+"""Thin ctypes binding of the C ABI in include/osc.h (argument marshalling only).
+
+Every function here has the name of the C entry point it calls.  torch is used
+for device memory and streams; all arithmetic happens in the CUDA library.
+Importing this module loads `libosc_b200.so` from the package directory and
+raises if it is missing: there is no CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libosc_b200.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(f"{LIB_PATH} not found: build it with `python -c 'import __graft_entry__ as g; g.build()'` "
+                      "(nvcc, sm_100a). The OSC path has no CPU fallback.")
+_lib = C.CDLL(LIB_PATH)
+
+OSC_OK = 0
+STATUS = {0: "OSC_OK", -1: "OSC_ERR_INVALID_ARG", -2: "OSC_ERR_SHAPE", -3: "OSC_ERR_LUT", -4: "OSC_ERR_ALIGN",
+          -5: "OSC_ERR_WORKSPACE", -6: "OSC_ERR_ARCH", -7: "OSC_ERR_CUDA", -8: "OSC_ERR_TIMEOUT"}
+
+
+class OscError(RuntimeError):
+    def __init__(self, status: int, detail: str):
+        super().__init__(f"{STATUS.get(status, status)}: {detail}")
+        self.status = status
+
+
+class WeightSizes(C.Structure):
+    _fields_ = [("K_o", C.c_int32), ("K_o_pad", C.c_int32), ("wq_bytes", C.c_size_t), ("sfw_bytes", C.c_size_t),
+                ("wo_bytes", C.c_size_t), ("meta_bytes", C.c_size_t)]
+
+
+class ActSizes(C.Structure):
+    _fields_ = [(n, C.c_size_t) for n in ("xq_bytes", "sfa_bytes", "xo_bytes", "sched_bytes", "xq_offset",
+                                          "sfa_offset", "xo_offset", "sched_offset", "workspace_bytes")]
+
+
+class Fp8ActSizes(C.Structure):
+    _fields_ = [(n, C.c_size_t) for n in ("x8_bytes", "sx_bytes", "sched_bytes", "x8_offset", "sx_offset",
+                                          "sched_offset", "workspace_bytes")]
+
+
+_vp, _i, _i64, _sz = C.c_void_p, C.c_int, C.c_int64, C.c_size_t
+_SIGS = {
+    "osc_status_string": (C.c_char_p, [_i]),
+    "osc_last_error": (C.c_char_p, []),
+    "osc_sync_check": (_i, [_vp]),
+    "osc_weight_sizes": (_i, [_i, _i, _i, _vp, _i, C.POINTER(WeightSizes)]),
+    "osc_prepare_weights": (_i, [_vp, _i, _i, _i64, _vp, _i, _vp, _vp, _vp, _vp, _vp, C.POINTER(_vp)]),
+    "osc_prepare_weights_grouped": (_i, [_vp, _i, _i, _i, _vp, _i, _vp, _vp, _vp, _vp, _vp, C.POINTER(_vp)]),
+    "osc_weights_destroy": (_i, [_vp]),
+    "osc_act_sizes": (_i, [_vp, _i, C.POINTER(ActSizes)]),
+    "osc_quantize_extract": (_i, [_vp, _vp, _i, _i64, _vp, _vp, _vp, _vp]),
+    "osc_gemm_dual": (_i, [_vp, _vp, _vp, _vp, _i, _vp, _i64, _vp]),
+    "osc_linear": (_i, [_vp, _vp, _i, _i64, _vp, _i64, _vp, _sz, _vp]),
+    "osc_linear_grouped": (_i, [_vp, _vp, _vp, _i, _i64, _vp, _i64, _vp, _sz, _vp]),
+    "osc_fp8_prepare_weights": (_i, [_vp, _i, _i, _i64, _vp, _vp, _vp, C.POINTER(_vp)]),
+    "osc_fp8_prepare_weights_grouped": (_i, [_vp, _i, _i, _i, _vp, _vp, _vp, C.POINTER(_vp)]),
+    "osc_fp8_weights_destroy": (_i, [_vp]),
+    "osc_fp8_act_sizes": (_i, [_vp, _i, C.POINTER(Fp8ActSizes)]),
+    "osc_fp8_quantize": (_i, [_vp, _i, _i, _i64, _vp, _vp, _vp]),
+    "osc_fp8_gemm": (_i, [_vp, _vp, _vp, _i, _vp, _i64, _vp]),
+    "osc_fp8_linear": (_i, [_vp, _vp, _i, _i64, _vp, _i64, _vp, _sz, _vp]),
+    "osc_fp8_linear_grouped": (_i, [_vp, _vp, _vp, _i, _i64, _vp, _i64, _vp, _sz, _vp]),
+}
+for _name, (_res, _args) in _SIGS.items():
+    _f = getattr(_lib, _name)
+    _f.restype = _res
+    _f.argtypes = _args
+
+EXPORTS = tuple(_SIGS)
+
+
+def osc_last_error() -> str:
+    return _lib.osc_last_error().decode()
+
+
+def osc_status_string(s: int) -> str:
+    return _lib.osc_status_string(s).decode()
+
+
+def _check(status: int):
+    if status != OSC_OK:
+        raise OscError(status, osc_last_error())
+
+
+def _ptr(t):
+    if t is None:
+        return None
+    if isinstance(t, torch.Tensor):
+        return t.data_ptr() if t.numel() > 0 else None
+    return int(t)
+
+
+def _stream(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return s.cuda_stream
+
+
+def _lut(lut):
+    lut = np.ascontiguousarray(lut, dtype=np.int8)
+    if lut.ndim == 1:
+        lut = lut.reshape(-1, 1)
+    return lut
+
+
+def osc_sync_check(stream=None):
+    _check(_lib.osc_sync_check(_stream(stream)))
+
+
+def osc_weight_sizes(E: int, N: int, K: int, lut) -> WeightSizes:
+    lut = _lut(lut)
+    out = WeightSizes()
+    _check(_lib.osc_weight_sizes(E, N, K, lut.ctypes.data, lut.shape[1], C.byref(out)))
+    return out
+
+
+class _Handle:
+    _destroy = None
+
+    def __init__(self, ptr, keep):
+        self.ptr = ptr
+        self.keep = keep  # device buffers the handle borrows
+
+    def close(self):
+        if self.ptr:
+            self._destroy(self.ptr)
+            self.ptr = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+class OscWeights(_Handle):
+    _destroy = staticmethod(_lib.osc_weights_destroy)
+
+
+class Fp8Weights(_Handle):
+    _destroy = staticmethod(_lib.osc_fp8_weights_destroy)
+
+
+def _alloc(nbytes, dev):
+    return torch.empty(max(int(nbytes), 16), dtype=torch.uint8, device=dev)
+
+
+def osc_prepare_weights(W: torch.Tensor, lut, stream=None) -> OscWeights:
+    """W: cuda bf16 [N, K] (row stride = ldw). Returns a handle owning wq/sfw/wo/meta."""
+    N, K = W.shape
+    lut = _lut(lut)
+    sz = osc_weight_sizes(1, N, K, lut)
+    dev = W.device
+    bufs = {k: _alloc(getattr(sz, k + "_bytes"), dev) for k in ("wq", "sfw", "wo", "meta")}
+    h = _vp()
+    _check(_lib.osc_prepare_weights(_ptr(W), N, K, W.stride(0), lut.ctypes.data, lut.shape[1], _ptr(bufs["wq"]),
+                                    _ptr(bufs["sfw"]), _ptr(bufs["wo"]) if sz.wo_bytes else None, _ptr(bufs["meta"]),
+                                    _stream(stream), C.byref(h)))
+    w = OscWeights(h.value, bufs)
+    w.E, w.N, w.K, w.K_o, w.K_o_pad, w.sizes = 1, N, K, sz.K_o, sz.K_o_pad, sz
+    return w
+
+
+def osc_prepare_weights_grouped(W: torch.Tensor, lut, stream=None) -> OscWeights:
+    """W: cuda bf16 [E, N, K] contiguous."""
+    E, N, K = W.shape
+    assert W.is_contiguous()
+    lut = _lut(lut)
+    sz = osc_weight_sizes(E, N, K, lut)
+    dev = W.device
+    bufs = {k: _alloc(getattr(sz, k + "_bytes"), dev) for k in ("wq", "sfw", "wo", "meta")}
+    h = _vp()
+    _check(_lib.osc_prepare_weights_grouped(_ptr(W), E, N, K, lut.ctypes.data, lut.shape[1], _ptr(bufs["wq"]),
+                                            _ptr(bufs["sfw"]), _ptr(bufs["wo"]) if sz.wo_bytes else None,
+                                            _ptr(bufs["meta"]), _stream(stream), C.byref(h)))
+    w = OscWeights(h.value, bufs)
+    w.E, w.N, w.K, w.K_o, w.K_o_pad, w.sizes = E, N, K, sz.K_o, sz.K_o_pad, sz
+    return w
+
+
+def osc_weights_destroy(w: OscWeights):
+    w.close()
+
+
+def osc_act_sizes(w: OscWeights, M: int) -> ActSizes:
+    out = ActSizes()
+    _check(_lib.osc_act_sizes(w.ptr, M, C.byref(out)))
+    return out
+
+
+def osc_quantize_extract(w: OscWeights, X: torch.Tensor, xq, sfa, xo, stream=None):
+    M = X.shape[0]
+    _check(_lib.osc_quantize_extract(w.ptr, _ptr(X), M, X.stride(0) if M else w.K, _ptr(xq), _ptr(sfa),
+                                     _ptr(xo) if w.K_o_pad else None, _stream(stream)))
+
+
+def osc_gemm_dual(w: OscWeights, xq, sfa, xo, M: int, Y: torch.Tensor, stream=None):
+    _check(_lib.osc_gemm_dual(w.ptr, _ptr(xq), _ptr(sfa), _ptr(xo) if w.K_o_pad else None, M, _ptr(Y),
+                              Y.stride(0) if M else w.N, _stream(stream)))
+
+
+def osc_linear(w: OscWeights, X: torch.Tensor, Y: torch.Tensor, workspace: torch.Tensor, stream=None):
+    M = X.shape[0]
+    _check(_lib.osc_linear(w.ptr, _ptr(X), M, X.stride(0) if M else w.K, _ptr(Y), Y.stride(0) if M else w.N,
+                           _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)))
+
+
+def osc_linear_grouped(w: OscWeights, X: torch.Tensor, off: torch.Tensor, Y: torch.Tensor, workspace: torch.Tensor,
+                       stream=None):
+    M = X.shape[0]
+    _check(_lib.osc_linear_grouped(w.ptr, _ptr(X), _ptr(off), M, X.stride(0) if M else w.K, _ptr(Y),
+                                   Y.stride(0) if M else w.N, _ptr(workspace),
+                                   workspace.numel() * workspace.element_size(), _stream(stream)))
+
+
+def osc_fp8_prepare_weights(W: torch.Tensor, stream=None) -> Fp8Weights:
+    N, K = W.shape
+    dev = W.device
+    bufs = {"w8": _alloc(N * K, dev), "sw": torch.empty(N, dtype=torch.float32, device=dev)}
+    h = _vp()
+    _check(_lib.osc_fp8_prepare_weights(_ptr(W), N, K, W.stride(0), _ptr(bufs["w8"]), _ptr(bufs["sw"]),
+                                        _stream(stream), C.byref(h)))
+    w = Fp8Weights(h.value, bufs)
+    w.E, w.N, w.K = 1, N, K
+    return w
+
+
+def osc_fp8_prepare_weights_grouped(W: torch.Tensor, stream=None) -> Fp8Weights:
+    E, N, K = W.shape
+    assert W.is_contiguous()
+    dev = W.device
+    bufs = {"w8": _alloc(E * N * K, dev), "sw": torch.empty(E * N, dtype=torch.float32, device=dev)}
+    h = _vp()
+    _check(_lib.osc_fp8_prepare_weights_grouped(_ptr(W), E, N, K, _ptr(bufs["w8"]), _ptr(bufs["sw"]),
+                                                _stream(stream), C.byref(h)))
+    w = Fp8Weights(h.value, bufs)
+    w.E, w.N, w.K = E, N, K
+    return w
+
+
+def osc_fp8_weights_destroy(w: Fp8Weights):
+    w.close()
+
+
+def osc_fp8_act_sizes(w: Fp8Weights, M: int) -> Fp8ActSizes:
+    out = Fp8ActSizes()
+    _check(_lib.osc_fp8_act_sizes(w.ptr, M, C.byref(out)))
+    return out
+
+
+def osc_fp8_quantize(X: torch.Tensor, x8, sx, stream=None):
+    M, K = X.shape
+    _check(_lib.osc_fp8_quantize(_ptr(X), M, K, X.stride(0) if M else K, _ptr(x8), _ptr(sx), _stream(stream)))
+
+
+def osc_fp8_gemm(w: Fp8Weights, x8, sx, M: int, Y: torch.Tensor, stream=None):
+    _check(_lib.osc_fp8_gemm(w.ptr, _ptr(x8), _ptr(sx), M, _ptr(Y), Y.stride(0) if M else w.N, _stream(stream)))
+
+
+def osc_fp8_linear(w: Fp8Weights, X: torch.Tensor, Y: torch.Tensor, workspace: torch.Tensor, stream=None):
+    M = X.shape[0]
+    _check(_lib.osc_fp8_linear(w.ptr, _ptr(X), M, X.stride(0) if M else w.K, _ptr(Y), Y.stride(0) if M else w.N,
+                               _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)))
+
+
+def osc_fp8_linear_grouped(w: Fp8Weights, X: torch.Tensor, off: torch.Tensor, Y: torch.Tensor,
+                           workspace: torch.Tensor, stream=None):
+    M = X.shape[0]
+    _check(_lib.osc_fp8_linear_grouped(w.ptr, _ptr(X), _ptr(off), M, X.stride(0) if M else w.K, _ptr(Y),
+                                       Y.stride(0) if M else w.N, _ptr(workspace),
+                                       workspace.numel() * workspace.element_size(), _stream(stream)))

@@ -1,0 +1,520 @@
+// Host side of the C ABI declared in include/osc.h: validation, handles, TMA descriptors, launches.
+#include <stdarg.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "../../include/osc.h"
+#include "common.cuh"
+
+namespace osc {
+
+static thread_local char t_err[512] = "";
+
+static osc_status fail(osc_status s, const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(t_err, sizeof t_err, fmt, ap);
+    va_end(ap);
+    if (getenv("OSC_LOG")) fprintf(stderr, "[osc] %s: %s\n", osc_status_string(s), t_err);
+    return s;
+}
+static osc_status cuda_fail(cudaError_t e, const char* what) {
+    return fail(OSC_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+static size_t align256(size_t x) { return (x + 255u) & ~size_t(255); }
+
+// -------------------------------------------------------------- device facts
+struct DeviceInfo {
+    bool ok = false;
+    int num_sms = 0;
+};
+static osc_status device_info(DeviceInfo* out) {
+    int dev = 0, major = 0, sms = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+    e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceGetAttribute");
+    if (major != 10) return fail(OSC_ERR_ARCH, "device %d has compute capability %d.x; this library needs 10.x", dev, major);
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaDeviceGetAttribute");
+    out->ok = true;
+    out->num_sms = sms;
+    return OSC_OK;
+}
+
+// ------------------------------------------------------------ TMA descriptors
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// Row-major [rows, row_bytes] operand, tiles of box_rows x 128 bytes, 128-byte swizzle, zero fill.
+static osc_status make_tmap(CUtensorMap* tm, const void* base, bool bf16, uint64_t rows, uint64_t row_bytes,
+                            uint64_t pitch_bytes, uint32_t box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return fail(OSC_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+    if (rows == 0) rows = 1;  // never dereferenced: no tile is scheduled for an empty operand
+    const uint64_t esz = bf16 ? 2 : 1;
+    cuuint64_t gdim[2] = {row_bytes / esz, rows};
+    cuuint64_t gstr[1] = {pitch_bytes};
+    cuuint32_t box[2] = {static_cast<cuuint32_t>(128 / esz), box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(tm, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 2,
+                    const_cast<void*>(base), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(OSC_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
+    return OSC_OK;
+}
+
+// ----------------------------------------------------------------- the table
+struct Table {
+    int Ko = 0, Kop = 0;
+    std::vector<uint32_t> mask;
+    std::vector<int32_t> prefix, idx;
+};
+static osc_status parse_lut(const int8_t* lut, int K, int C, Table* t) {
+    if (K <= 0 || K % 128) return fail(OSC_ERR_SHAPE, "K = %d must be a positive multiple of 128", K);
+    if (C < 0 || C > 32) return fail(OSC_ERR_INVALID_ARG, "lut_c = %d outside 0..32", C);
+    if (C > 0 && !lut) return fail(OSC_ERR_INVALID_ARG, "lut is null");
+    const int Kg = K / 32;
+    t->mask.assign(Kg, 0);
+    t->prefix.assign(Kg, 0);
+    t->idx.clear();
+    for (int k = 0; k < Kg; ++k) {
+        uint32_t m = 0;
+        for (int c = 0; c < C; ++c) {
+            const int j = lut[(size_t)k * C + c];
+            if (j < -1 || j > 31) return fail(OSC_ERR_LUT, "table entry %d of group %d outside -1..31", j, k);
+            if (j < 0) continue;
+            if (m >> j & 1u) return fail(OSC_ERR_LUT, "channel %d listed twice in group %d", j, k);
+            m |= 1u << j;
+        }
+        t->mask[k] = m;
+        t->prefix[k] = (int32_t)t->idx.size();
+        for (int j = 0; j < 32; ++j)
+            if (m >> j & 1u) t->idx.push_back(k * 32 + j);
+    }
+    t->Ko = (int)t->idx.size();
+    t->Kop = (t->Ko + 63) / 64 * 64;
+    return OSC_OK;
+}
+
+static osc_status check_nk(int E, int N, int K) {
+    if (E < 1 || E > 1024) return fail(OSC_ERR_INVALID_ARG, "E = %d outside 1..1024", E);
+    if (N <= 0 || N % 64) return fail(OSC_ERR_SHAPE, "N = %d must be a positive multiple of 64", N);
+    if (K <= 0 || K % 128) return fail(OSC_ERR_SHAPE, "K = %d must be a positive multiple of 128", K);
+    if ((int64_t)E * N > 0x7FFFFFFF) return fail(OSC_ERR_SHAPE, "E*N too large");
+    return OSC_OK;
+}
+static size_t sf_bytes(int64_t rows, int K) { return (size_t)((rows + 127) / 128) * (K / 128) * 512; }
+
+}  // namespace osc
+
+using namespace osc;
+
+struct osc_weights {
+    int E, N, K, Ko, Kop;
+    bool grouped;
+    const uint8_t *wq, *sfw;
+    const uint16_t* wo;
+    const uint32_t* mask;
+    const int32_t* prefix;
+    int num_sms, block_n;
+    CUtensorMap tm_b, tm_bo;
+};
+struct osc_fp8_weights {
+    int E, N, K;
+    bool grouped;
+    const uint8_t* w8;
+    const float* sw;
+    int num_sms, block_n;
+    CUtensorMap tm_b;
+};
+
+extern "C" {
+
+const char* osc_status_string(osc_status s) {
+    switch (s) {
+        case OSC_OK: return "OSC_OK";
+        case OSC_ERR_INVALID_ARG: return "OSC_ERR_INVALID_ARG";
+        case OSC_ERR_SHAPE: return "OSC_ERR_SHAPE";
+        case OSC_ERR_LUT: return "OSC_ERR_LUT";
+        case OSC_ERR_ALIGN: return "OSC_ERR_ALIGN";
+        case OSC_ERR_WORKSPACE: return "OSC_ERR_WORKSPACE";
+        case OSC_ERR_ARCH: return "OSC_ERR_ARCH";
+        case OSC_ERR_CUDA: return "OSC_ERR_CUDA";
+        case OSC_ERR_TIMEOUT: return "OSC_ERR_TIMEOUT";
+        default: return "OSC_ERR_UNKNOWN";
+    }
+}
+const char* osc_last_error(void) { return t_err; }
+
+osc_status osc_sync_check(void* stream) {
+    cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
+    int st = 0;
+    e = cudaMemcpyFromSymbol(&st, g_dev_status, sizeof st);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpyFromSymbol");
+    if (st != 0) {
+        const int zero = 0;
+        cudaMemcpyToSymbol(g_dev_status, &zero, sizeof zero);
+        return fail(OSC_ERR_TIMEOUT, "a device-side wait gave up (site %d)", st >> 8);
+    }
+    return OSC_OK;
+}
+
+// ------------------------------------------------------------------ OSC path
+
+osc_status osc_weight_sizes(int E, int N, int K, const int8_t* lut, int lut_c, osc_weight_sizes_t* out) {
+    if (!out) return fail(OSC_ERR_INVALID_ARG, "out is null");
+    if (osc_status s = check_nk(E, N, K)) return s;
+    Table t;
+    if (osc_status s = parse_lut(lut, K, lut_c, &t)) return s;
+    out->K_o = t.Ko;
+    out->K_o_pad = t.Kop;
+    out->wq_bytes = (size_t)E * N * (K / 2);
+    out->sfw_bytes = (size_t)E * sf_bytes(N, K);
+    out->wo_bytes = (size_t)E * N * t.Kop * 2;
+    out->meta_bytes = align256((size_t)(K / 32) * 8 + (size_t)t.Ko * 4 + 16);
+    return OSC_OK;
+}
+
+static osc_status prepare_impl(const void* W, int E, int N, int K, int64_t ldw, const int8_t* lut, int lut_c,
+                               void* wq, void* sfw, void* wo, void* meta, void* stream, bool grouped,
+                               osc_weights** out) {
+    if (!out) return fail(OSC_ERR_INVALID_ARG, "out is null");
+    *out = nullptr;
+    if (osc_status s = check_nk(E, N, K)) return s;
+    Table t;
+    if (osc_status s = parse_lut(lut, K, lut_c, &t)) return s;
+    if (!W || !wq || !sfw || !meta || (t.Kop > 0 && !wo)) return fail(OSC_ERR_INVALID_ARG, "null device pointer");
+    if (ldw < K) return fail(OSC_ERR_SHAPE, "ldw = %lld < K", (long long)ldw);
+    if (ldw % 8 || !aligned16(W) || !aligned16(wq) || !aligned16(sfw) || !aligned16(meta) || !aligned16(wo))
+        return fail(OSC_ERR_ALIGN, "pointers must be 16-byte aligned and ldw a multiple of 8");
+    DeviceInfo di;
+    if (osc_status s = device_info(&di)) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+    const int Kg = K / 32;
+    uint8_t* m8 = static_cast<uint8_t*>(meta);
+    cudaError_t e = cudaMemcpyAsync(m8, t.mask.data(), (size_t)Kg * 4, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(m8 + (size_t)Kg * 4, t.prefix.data(), (size_t)Kg * 4, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess && t.Ko > 0)
+        e = cudaMemcpyAsync(m8 + (size_t)Kg * 8, t.idx.data(), (size_t)t.Ko * 4, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpyAsync(meta)");
+    const uint32_t* d_mask = reinterpret_cast<const uint32_t*>(m8);
+    const int32_t* d_prefix = reinterpret_cast<const int32_t*>(m8 + (size_t)Kg * 4);
+
+    const size_t sfw_e = sf_bytes(N, K);
+    for (int ex = 0; ex < E; ++ex) {
+        e = launch_quant_extract(static_cast<const uint16_t*>(W) + (size_t)ex * N * ldw, ldw, N, K, d_mask, d_prefix,
+                                 static_cast<uint8_t*>(wq) + (size_t)ex * N * (K / 2),
+                                 static_cast<uint8_t*>(sfw) + (size_t)ex * sfw_e,
+                                 t.Kop ? static_cast<uint16_t*>(wo) + (size_t)ex * N * t.Kop : nullptr, t.Ko, t.Kop,
+                                 nullptr, 0, st);
+        if (e != cudaSuccess) return cuda_fail(e, "quant_extract_kernel(weights)");
+    }
+
+    osc_weights* w = new (std::nothrow) osc_weights();
+    if (!w) return fail(OSC_ERR_INVALID_ARG, "out of host memory");
+    w->E = E; w->N = N; w->K = K; w->Ko = t.Ko; w->Kop = t.Kop; w->grouped = grouped;
+    w->wq = static_cast<const uint8_t*>(wq);
+    w->sfw = static_cast<const uint8_t*>(sfw);
+    w->wo = static_cast<const uint16_t*>(wo);
+    w->mask = d_mask; w->prefix = d_prefix;
+    w->num_sms = di.num_sms;
+    w->block_n = gemm_block_n();
+    osc_status s = make_tmap(&w->tm_b, wq, false, (uint64_t)E * N, K / 2, K / 2, w->block_n);
+    if (s == OSC_OK && t.Kop > 0)
+        s = make_tmap(&w->tm_bo, wo, true, (uint64_t)E * N, (uint64_t)t.Kop * 2, (uint64_t)t.Kop * 2, w->block_n);
+    if (s != OSC_OK) { delete w; return s; }
+    *out = w;
+    return OSC_OK;
+}
+
+osc_status osc_prepare_weights(const void* W, int N, int K, int64_t ldw, const int8_t* lut, int lut_c, void* wq,
+                               void* sfw, void* wo, void* meta, void* stream, osc_weights** out) {
+    return prepare_impl(W, 1, N, K, ldw, lut, lut_c, wq, sfw, wo, meta, stream, false, out);
+}
+osc_status osc_prepare_weights_grouped(const void* W, int E, int N, int K, const int8_t* lut, int lut_c, void* wq,
+                                       void* sfw, void* wo, void* meta, void* stream, osc_weights** out) {
+    return prepare_impl(W, E, N, K, K, lut, lut_c, wq, sfw, wo, meta, stream, true, out);
+}
+osc_status osc_weights_destroy(osc_weights* w) {
+    delete w;
+    return OSC_OK;
+}
+
+osc_status osc_act_sizes(const osc_weights* w, int M, osc_act_sizes_t* out) {
+    if (!w || !out) return fail(OSC_ERR_INVALID_ARG, "null argument");
+    if (M < 0) return fail(OSC_ERR_INVALID_ARG, "M = %d is negative", M);
+    const int64_t max_tiles = w->grouped ? (int64_t)M / 128 + w->E : ((int64_t)M + 127) / 128;
+    out->xq_bytes = (size_t)M * (w->K / 2);
+    out->sfa_bytes = (size_t)max_tiles * (w->K / 128) * 512;
+    out->xo_bytes = (size_t)M * w->Kop * 2;
+    out->sched_bytes = w->grouped ? (size_t)(1 + 4 * max_tiles) * 4 : 0;
+    out->xq_offset = 0;
+    out->sfa_offset = out->xq_offset + align256(out->xq_bytes);
+    out->xo_offset = out->sfa_offset + align256(out->sfa_bytes);
+    out->sched_offset = out->xo_offset + align256(out->xo_bytes);
+    out->workspace_bytes = out->sched_offset + align256(out->sched_bytes);
+    return OSC_OK;
+}
+
+static osc_status check_act(const osc_weights* w, const void* X, int M, int64_t ldx) {
+    if (!w) return fail(OSC_ERR_INVALID_ARG, "weights handle is null");
+    if (M < 0) return fail(OSC_ERR_INVALID_ARG, "M = %d is negative", M);
+    if (M > 0 && !X) return fail(OSC_ERR_INVALID_ARG, "X is null");
+    if (ldx < w->K) return fail(OSC_ERR_SHAPE, "ldx = %lld < K = %d", (long long)ldx, w->K);
+    if (ldx % 8 || !aligned16(X)) return fail(OSC_ERR_ALIGN, "X must be 16-byte aligned and ldx a multiple of 8");
+    return OSC_OK;
+}
+
+static osc_status quantize_impl(const osc_weights* w, const void* X, int M, int64_t ldx, void* xq, void* sfa,
+                                void* xo, const int32_t* sched, int max_tiles, cudaStream_t st) {
+    if (M == 0) return OSC_OK;
+    if (!xq || !sfa || (w->Kop > 0 && !xo)) return fail(OSC_ERR_INVALID_ARG, "null output pointer");
+    if (!aligned16(xq) || !aligned16(sfa) || !aligned16(xo)) return fail(OSC_ERR_ALIGN, "outputs must be 16-byte aligned");
+    cudaError_t e = launch_quant_extract(X, ldx, M, w->K, w->mask, w->prefix, xq, sfa, w->Kop ? xo : nullptr, w->Ko,
+                                         w->Kop, sched, max_tiles, st);
+    if (e != cudaSuccess) return cuda_fail(e, "quant_extract_kernel");
+    return OSC_OK;
+}
+
+osc_status osc_quantize_extract(const osc_weights* w, const void* X, int M, int64_t ldx, void* xq, void* sfa,
+                                void* xo, void* stream) {
+    if (osc_status s = check_act(w, X, M, ldx)) return s;
+    if (w->grouped) return fail(OSC_ERR_INVALID_ARG, "grouped weights: use osc_linear_grouped");
+    return quantize_impl(w, X, M, ldx, xq, sfa, xo, nullptr, 0, static_cast<cudaStream_t>(stream));
+}
+
+static osc_status gemm_impl(const osc_weights* w, const void* xq, const void* sfa, const void* xo, int M, void* Y,
+                            int64_t ldy, const int32_t* sched, int max_tiles, cudaStream_t st) {
+    if (M == 0) return OSC_OK;
+    if (!xq || !sfa || !Y || (w->Kop > 0 && !xo)) return fail(OSC_ERR_INVALID_ARG, "null device pointer");
+    if (ldy < w->N) return fail(OSC_ERR_SHAPE, "ldy = %lld < N = %d", (long long)ldy, w->N);
+    if (ldy % 8 || !aligned16(Y) || !aligned16(xq) || !aligned16(sfa) || !aligned16(xo))
+        return fail(OSC_ERR_ALIGN, "pointers must be 16-byte aligned and ldy a multiple of 8");
+    GemmArgs a;
+    memset(&a, 0, sizeof a);
+    if (osc_status s = make_tmap(&a.tm_a, xq, false, M, w->K / 2, w->K / 2, 128)) return s;
+    a.tm_b = w->tm_b;
+    if (w->Kop > 0) {
+        if (osc_status s = make_tmap(&a.tm_ao, xo, true, M, (uint64_t)w->Kop * 2, (uint64_t)w->Kop * 2, 128)) return s;
+        a.tm_bo = w->tm_bo;
+    }
+    a.sfa = static_cast<const uint8_t*>(sfa);
+    a.sfw = w->sfw;
+    a.Y = static_cast<uint16_t*>(Y);
+    a.ldy = ldy;
+    a.M = M; a.N = w->N; a.K = w->K; a.Kop = w->Kop;
+    a.sched = sched; a.max_tiles = max_tiles; a.num_sms = w->num_sms;
+    cudaError_t e = launch_gemm_dual(a, st);
+    if (e != cudaSuccess) return cuda_fail(e, "gemm_kernel(dual)");
+    return OSC_OK;
+}
+
+osc_status osc_gemm_dual(const osc_weights* w, const void* xq, const void* sfa, const void* xo, int M, void* Y,
+                         int64_t ldy, void* stream) {
+    if (!w) return fail(OSC_ERR_INVALID_ARG, "weights handle is null");
+    if (M < 0) return fail(OSC_ERR_INVALID_ARG, "M = %d is negative", M);
+    if (w->grouped) return fail(OSC_ERR_INVALID_ARG, "grouped weights: use osc_linear_grouped");
+    return gemm_impl(w, xq, sfa, xo, M, Y, ldy, nullptr, 0, static_cast<cudaStream_t>(stream));
+}
+
+osc_status osc_linear(const osc_weights* w, const void* X, int M, int64_t ldx, void* Y, int64_t ldy,
+                      void* workspace, size_t workspace_bytes, void* stream) {
+    if (osc_status s = check_act(w, X, M, ldx)) return s;
+    if (w->grouped) return fail(OSC_ERR_INVALID_ARG, "grouped weights: use osc_linear_grouped");
+    if (M == 0) return OSC_OK;
+    osc_act_sizes_t sz;
+    osc_act_sizes(w, M, &sz);
+    if (!workspace || !aligned16(workspace)) return fail(OSC_ERR_ALIGN, "workspace must be non-null and 16-byte aligned");
+    if (workspace_bytes < sz.workspace_bytes)
+        return fail(OSC_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", workspace_bytes, sz.workspace_bytes);
+    if (!Y) return fail(OSC_ERR_INVALID_ARG, "Y is null");
+    if (ldy < w->N) return fail(OSC_ERR_SHAPE, "ldy = %lld < N = %d", (long long)ldy, w->N);
+    if (ldy % 8 || !aligned16(Y)) return fail(OSC_ERR_ALIGN, "Y must be 16-byte aligned and ldy a multiple of 8");
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (osc_status s = quantize_impl(w, X, M, ldx, ws + sz.xq_offset, ws + sz.sfa_offset, ws + sz.xo_offset, nullptr, 0, st)) return s;
+    return gemm_impl(w, ws + sz.xq_offset, ws + sz.sfa_offset, ws + sz.xo_offset, M, Y, ldy, nullptr, 0, st);
+}
+
+osc_status osc_linear_grouped(const osc_weights* w, const void* X_perm, const int32_t* off, int M_total, int64_t ldx,
+                              void* Y, int64_t ldy, void* workspace, size_t workspace_bytes, void* stream) {
+    if (osc_status s = check_act(w, X_perm, M_total, ldx)) return s;
+    if (!w->grouped) return fail(OSC_ERR_INVALID_ARG, "dense weights: use osc_linear");
+    if (M_total == 0) return OSC_OK;
+    if (!off) return fail(OSC_ERR_INVALID_ARG, "off is null");
+    osc_act_sizes_t sz;
+    osc_act_sizes(w, M_total, &sz);
+    if (!workspace || !aligned16(workspace)) return fail(OSC_ERR_ALIGN, "workspace must be non-null and 16-byte aligned");
+    if (workspace_bytes < sz.workspace_bytes)
+        return fail(OSC_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", workspace_bytes, sz.workspace_bytes);
+    if (!Y) return fail(OSC_ERR_INVALID_ARG, "Y is null");
+    if (ldy < w->N) return fail(OSC_ERR_SHAPE, "ldy = %lld < N = %d", (long long)ldy, w->N);
+    if (ldy % 8 || !aligned16(Y)) return fail(OSC_ERR_ALIGN, "Y must be 16-byte aligned and ldy a multiple of 8");
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int max_tiles = M_total / 128 + w->E;
+    int32_t* sched = reinterpret_cast<int32_t*>(ws + sz.sched_offset);
+    cudaError_t e = launch_build_sched(off, w->E, sched, max_tiles, st);
+    if (e != cudaSuccess) return cuda_fail(e, "build_sched_kernel");
+    if (osc_status s = quantize_impl(w, X_perm, M_total, ldx, ws + sz.xq_offset, ws + sz.sfa_offset, ws + sz.xo_offset,
+                                     sched, max_tiles, st)) return s;
+    return gemm_impl(w, ws + sz.xq_offset, ws + sz.sfa_offset, ws + sz.xo_offset, M_total, Y, ldy, sched, max_tiles, st);
+}
+
+// -------------------------------------------------------------- FP8 fallback
+
+static osc_status fp8_prepare_impl(const void* W, int E, int N, int K, int64_t ldw, void* w8, void* sw, void* stream,
+                                   bool grouped, osc_fp8_weights** out) {
+    if (!out) return fail(OSC_ERR_INVALID_ARG, "out is null");
+    *out = nullptr;
+    if (osc_status s = check_nk(E, N, K)) return s;
+    if (!W || !w8 || !sw) return fail(OSC_ERR_INVALID_ARG, "null device pointer");
+    if (ldw < K) return fail(OSC_ERR_SHAPE, "ldw = %lld < K", (long long)ldw);
+    if (ldw % 8 || !aligned16(W) || !aligned16(w8) || !aligned16(sw))
+        return fail(OSC_ERR_ALIGN, "pointers must be 16-byte aligned and ldw a multiple of 8");
+    DeviceInfo di;
+    if (osc_status s = device_info(&di)) return s;
+    cudaError_t e = launch_fp8_quant(W, ldw, E * N, K, w8, sw, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(e, "fp8_quant_kernel(weights)");
+    osc_fp8_weights* w = new (std::nothrow) osc_fp8_weights();
+    if (!w) return fail(OSC_ERR_INVALID_ARG, "out of host memory");
+    w->E = E; w->N = N; w->K = K; w->grouped = grouped;
+    w->w8 = static_cast<const uint8_t*>(w8);
+    w->sw = static_cast<const float*>(sw);
+    w->num_sms = di.num_sms;
+    w->block_n = gemm_block_n();
+    if (osc_status s = make_tmap(&w->tm_b, w8, false, (uint64_t)E * N, K, K, w->block_n)) { delete w; return s; }
+    *out = w;
+    return OSC_OK;
+}
+
+osc_status osc_fp8_prepare_weights(const void* W, int N, int K, int64_t ldw, void* w8, void* sw, void* stream,
+                                   osc_fp8_weights** out) {
+    return fp8_prepare_impl(W, 1, N, K, ldw, w8, sw, stream, false, out);
+}
+osc_status osc_fp8_prepare_weights_grouped(const void* W, int E, int N, int K, void* w8, void* sw, void* stream,
+                                           osc_fp8_weights** out) {
+    return fp8_prepare_impl(W, E, N, K, K, w8, sw, stream, true, out);
+}
+osc_status osc_fp8_weights_destroy(osc_fp8_weights* w) {
+    delete w;
+    return OSC_OK;
+}
+
+osc_status osc_fp8_act_sizes(const osc_fp8_weights* w, int M, osc_fp8_act_sizes_t* out) {
+    if (!w || !out) return fail(OSC_ERR_INVALID_ARG, "null argument");
+    if (M < 0) return fail(OSC_ERR_INVALID_ARG, "M = %d is negative", M);
+    const int64_t max_tiles = w->grouped ? (int64_t)M / 128 + w->E : 0;
+    out->x8_bytes = (size_t)M * w->K;
+    out->sx_bytes = (size_t)M * 4;
+    out->sched_bytes = w->grouped ? (size_t)(1 + 4 * max_tiles) * 4 : 0;
+    out->x8_offset = 0;
+    out->sx_offset = align256(out->x8_bytes);
+    out->sched_offset = out->sx_offset + align256(out->sx_bytes);
+    out->workspace_bytes = out->sched_offset + align256(out->sched_bytes);
+    return OSC_OK;
+}
+
+osc_status osc_fp8_quantize(const void* X, int M, int K, int64_t ldx, void* x8, void* sx, void* stream) {
+    if (M < 0) return fail(OSC_ERR_INVALID_ARG, "M = %d is negative", M);
+    if (K <= 0 || K % 128) return fail(OSC_ERR_SHAPE, "K = %d must be a positive multiple of 128", K);
+    if (M == 0) return OSC_OK;
+    if (!X || !x8 || !sx) return fail(OSC_ERR_INVALID_ARG, "null device pointer");
+    if (ldx < K) return fail(OSC_ERR_SHAPE, "ldx = %lld < K", (long long)ldx);
+    if (ldx % 8 || !aligned16(X) || !aligned16(x8) || !aligned16(sx))
+        return fail(OSC_ERR_ALIGN, "pointers must be 16-byte aligned and ldx a multiple of 8");
+    cudaError_t e = launch_fp8_quant(X, ldx, M, K, x8, sx, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(e, "fp8_quant_kernel");
+    return OSC_OK;
+}
+
+static osc_status fp8_gemm_impl(const osc_fp8_weights* w, const void* x8, const void* sx, int M, void* Y, int64_t ldy,
+                                const int32_t* sched, int max_tiles, cudaStream_t st) {
+    if (M == 0) return OSC_OK;
+    if (!x8 || !sx || !Y) return fail(OSC_ERR_INVALID_ARG, "null device pointer");
+    if (ldy < w->N) return fail(OSC_ERR_SHAPE, "ldy = %lld < N = %d", (long long)ldy, w->N);
+    if (ldy % 8 || !aligned16(Y) || !aligned16(x8) || !aligned16(sx))
+        return fail(OSC_ERR_ALIGN, "pointers must be 16-byte aligned and ldy a multiple of 8");
+    GemmArgs a;
+    memset(&a, 0, sizeof a);
+    if (osc_status s = make_tmap(&a.tm_a, x8, false, M, w->K, w->K, 128)) return s;
+    a.tm_b = w->tm_b;
+    a.sx = static_cast<const float*>(sx);
+    a.sw = w->sw;
+    a.Y = static_cast<uint16_t*>(Y);
+    a.ldy = ldy;
+    a.M = M; a.N = w->N; a.K = w->K; a.Kop = 0;
+    a.sched = sched; a.max_tiles = max_tiles; a.num_sms = w->num_sms;
+    cudaError_t e = launch_gemm_fp8(a, st);
+    if (e != cudaSuccess) return cuda_fail(e, "gemm_kernel(fp8)");
+    return OSC_OK;
+}
+
+osc_status osc_fp8_gemm(const osc_fp8_weights* w, const void* x8, const void* sx, int M, void* Y, int64_t ldy,
+                        void* stream) {
+    if (!w) return fail(OSC_ERR_INVALID_ARG, "weights handle is null");
+    if (M < 0) return fail(OSC_ERR_INVALID_ARG, "M = %d is negative", M);
+    if (w->grouped) return fail(OSC_ERR_INVALID_ARG, "grouped weights: use osc_fp8_linear_grouped");
+    return fp8_gemm_impl(w, x8, sx, M, Y, ldy, nullptr, 0, static_cast<cudaStream_t>(stream));
+}
+
+static osc_status fp8_linear_impl(const osc_fp8_weights* w, const void* X, const int32_t* off, int M, int64_t ldx,
+                                  void* Y, int64_t ldy, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!w) return fail(OSC_ERR_INVALID_ARG, "weights handle is null");
+    if (M < 0) return fail(OSC_ERR_INVALID_ARG, "M = %d is negative", M);
+    if (M == 0) return OSC_OK;
+    if (w->grouped && !off) return fail(OSC_ERR_INVALID_ARG, "off is null");
+    osc_fp8_act_sizes_t sz;
+    osc_fp8_act_sizes(w, M, &sz);
+    if (!workspace || !aligned16(workspace)) return fail(OSC_ERR_ALIGN, "workspace must be non-null and 16-byte aligned");
+    if (workspace_bytes < sz.workspace_bytes)
+        return fail(OSC_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", workspace_bytes, sz.workspace_bytes);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int32_t* sched = nullptr;
+    int max_tiles = 0;
+    if (w->grouped) {
+        max_tiles = M / 128 + w->E;
+        int32_t* s = reinterpret_cast<int32_t*>(ws + sz.sched_offset);
+        cudaError_t e = launch_build_sched(off, w->E, s, max_tiles, st);
+        if (e != cudaSuccess) return cuda_fail(e, "build_sched_kernel");
+        sched = s;
+    }
+    if (osc_status s = osc_fp8_quantize(X, M, w->K, ldx, ws + sz.x8_offset, ws + sz.sx_offset, stream)) return s;
+    return fp8_gemm_impl(w, ws + sz.x8_offset, ws + sz.sx_offset, M, Y, ldy, sched, max_tiles, st);
+}
+
+osc_status osc_fp8_linear(const osc_fp8_weights* w, const void* X, int M, int64_t ldx, void* Y, int64_t ldy,
+                          void* workspace, size_t workspace_bytes, void* stream) {
+    if (w && w->grouped) return fail(OSC_ERR_INVALID_ARG, "grouped weights: use osc_fp8_linear_grouped");
+    return fp8_linear_impl(w, X, nullptr, M, ldx, Y, ldy, workspace, workspace_bytes, stream);
+}
+osc_status osc_fp8_linear_grouped(const osc_fp8_weights* w, const void* X_perm, const int32_t* off, int M_total,
+                                  int64_t ldx, void* Y, int64_t ldy, void* workspace, size_t workspace_bytes,
+                                  void* stream) {
+    if (w && !w->grouped) return fail(OSC_ERR_INVALID_ARG, "dense weights: use osc_fp8_linear");
+    return fp8_linear_impl(w, X_perm, off, M_total, ldx, Y, ldy, workspace, workspace_bytes, stream);
+}
+
+}  // extern "C"

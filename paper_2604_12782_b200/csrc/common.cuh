@@ -1,0 +1,40 @@
+// Declarations shared by the translation units of the library (host side + kernel launchers).
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "ptx.cuh"
+
+namespace osc {
+
+// quant_kernels.cu
+cudaError_t launch_quant_extract(const void* X, int64_t ldx, int M, int K, const uint32_t* mask,
+                                 const int32_t* prefix, void* xq, void* sf, void* xo, int Ko, int Kop,
+                                 const int32_t* sched, int max_tiles, cudaStream_t st);
+cudaError_t launch_fp8_quant(const void* X, int64_t ldx, int M, int K, void* x8, void* sx, cudaStream_t st);
+cudaError_t launch_build_sched(const int32_t* off, int E, int32_t* sched, int max_tiles, cudaStream_t st);
+
+// gemm_kernels.cu
+struct GemmArgs {
+    CUtensorMap tm_a;    // Path A activations: packed FP4 bytes [rows, K/2]  (FP8 mode: [rows, K])
+    CUtensorMap tm_b;    // Path A weights    : [E*N, K/2]                    (FP8 mode: [E*N, K])
+    CUtensorMap tm_ao;   // Path B activations: bf16 [rows, K_o_pad]
+    CUtensorMap tm_bo;   // Path B weights    : bf16 [E*N, K_o_pad]
+    const uint8_t* sfa;  // activation scales, block layout
+    const uint8_t* sfw;  // weight scales, block layout, per expert
+    const float* sx;     // FP8 mode: per-row activation scale
+    const float* sw;     // FP8 mode: per-output-row weight scale [E*N]
+    uint16_t* Y;         // bf16 [rows, ldy]
+    int64_t ldy;
+    int M;               // rows (dense) / total rows (grouped)
+    int N, K, Kop;
+    const int32_t* sched;  // grouped tile schedule or nullptr
+    int max_tiles;
+    int num_sms;
+};
+cudaError_t launch_gemm_dual(const GemmArgs& a, cudaStream_t st);
+cudaError_t launch_gemm_fp8(const GemmArgs& a, cudaStream_t st);
+int gemm_block_n();
+
+}  // namespace osc

@@ -1,0 +1,352 @@
+// Tensor-core kernels (tcgen05 + TMEM + TMA), one persistent CTA per SM, warp-specialised:
+//   warp 0    : TMA producer (operand tiles + scale-factor blocks into a shared-memory ring)
+//   warp 1    : MMA issuer (one thread) and TMEM owner
+//   warps 2-5 : epilogue (TMEM -> registers -> bf16 -> global)
+//
+// MODE_OSC : Eq. 5.  For every 128 x BN output tile the K loop first runs the block-scaled FP4
+//            blocks of Path A (256 channels = 128 bytes per row and stage, four K=64 MMAs with
+//            E8M0 scale vectors copied into TMEM), then the BF16 blocks of Path B over the
+//            gathered channels (64 channels = 128 bytes per row and stage, four K=16 MMAs) into the
+//            same fp32 accumulator.  Every stage carries 128 bytes per operand row, whatever the
+//            operand type, so one ring serves both paths.
+// MODE_FP8 : Section 3.4 fallback.  E4M3 x E4M3 (128 channels per stage, four K=32 MMAs); the
+//            per-row activation scale and per-output-row weight scale are applied in the epilogue.
+//
+// Dense and grouped (MoE) problems share the kernel: a tile's first row, last valid row, first
+// scale row and expert come either from arithmetic (dense) or from the device-built schedule.
+#include <cuda_bf16.h>
+
+#include "common.cuh"
+
+namespace osc {
+
+constexpr int MODE_OSC = 0;
+constexpr int MODE_FP8 = 1;
+
+constexpr int BM = 128;            // rows per tile = TMEM lanes
+constexpr int ROW_BYTES = 128;     // bytes per operand row and stage (one 128-byte swizzle row)
+constexpr int A_BYTES = BM * ROW_BYTES;
+constexpr int GEMM_THREADS = 192;
+constexpr int TMEM_COLS = 512;
+constexpr int BAND = 8;            // row tiles per scheduling band (L2 reuse of the weight tiles)
+
+template <int MODE, int BN>
+struct Cfg {
+    static constexpr int ACC_STAGES = (BN <= 192) ? 2 : 1;
+    static constexpr int SFB_ATOMS = (BN > 128) ? 2 : 1;  // 128-row scale blocks a tile can touch
+    static constexpr int B_BYTES = BN * ROW_BYTES;
+    static constexpr int SFA_BYTES = (MODE == MODE_OSC) ? 1024 : 0;
+    static constexpr int SFB_BYTES = (MODE == MODE_OSC) ? SFB_ATOMS * 1024 : 0;
+    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + SFA_BYTES + SFB_BYTES;  // multiple of 1024
+    static constexpr int STAGES = (200 * 1024) / STAGE_BYTES;
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+    static constexpr int TM_SFA = ACC_STAGES * BN;  // TMEM column of the activation scales (8 columns)
+    static constexpr int TM_SFB = TM_SFA + 8;       // weight scales: 2 K-blocks x SFB_ATOMS x 4 columns
+    static_assert(STAGE_BYTES % 1024 == 0, "stage must keep 1024-byte alignment");
+    static_assert(TM_SFB + 2 * SFB_ATOMS * 4 <= TMEM_COLS, "TMEM budget");
+};
+
+struct TileInfo {
+    int row0, row_end, sf_row0, expert, n0;
+};
+
+__device__ __forceinline__ int num_row_tiles(const GemmArgs& a) {
+    return a.sched ? a.sched[0] : (a.M + BM - 1) / BM;
+}
+
+template <int BN>
+__device__ __forceinline__ TileInfo tile_info(const GemmArgs& a, int t, int num_m, int num_n) {
+    const int per_band = BAND * num_n;
+    const int band = t / per_band;
+    const int rem = t - band * per_band;
+    const int m0 = band * BAND;
+    const int h = min(BAND, num_m - m0);
+    const int m = m0 + rem % h;
+    const int n = rem / h;
+    TileInfo ti;
+    ti.n0 = n * BN;
+    if (a.sched) {
+        ti.row0 = a.sched[1 + m];
+        ti.row_end = a.sched[1 + a.max_tiles + m];
+        ti.sf_row0 = a.sched[1 + 2 * a.max_tiles + m];
+        ti.expert = a.sched[1 + 3 * a.max_tiles + m];
+    } else {
+        ti.row0 = m * BM;
+        ti.row_end = a.M;
+        ti.sf_row0 = ti.row0;
+        ti.expert = 0;
+    }
+    return ti;
+}
+
+template <int MODE, int BN>
+__global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_constant__ GemmArgs args) {
+    using C = Cfg<MODE, BN>;
+    constexpr int STAGES = C::STAGES;
+    constexpr int ACC = C::ACC_STAGES;
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * C::STAGE_BYTES);
+    uint64_t* full_bar = bars;
+    uint64_t* empty_bar = bars + STAGES;
+    uint64_t* tfull_bar = bars + 2 * STAGES;
+    uint64_t* tempty_bar = bars + 2 * STAGES + ACC;
+    uint64_t* drain_bar = bars + 2 * STAGES + 2 * ACC;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 2 * ACC + 1);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < STAGES; ++i) {
+            mbar_init(&full_bar[i], 1);
+            mbar_init(&empty_bar[i], 1);
+        }
+        for (int i = 0; i < ACC; ++i) {
+            mbar_init(&tfull_bar[i], 1);
+            mbar_init(&tempty_bar[i], 4);
+        }
+        mbar_init(drain_bar, 1);
+        *abort_flag = 0;
+        fence_barrier_init();
+        prefetch_tmap(&args.tm_a);
+        prefetch_tmap(&args.tm_b);
+        if (MODE == MODE_OSC && args.Kop > 0) {
+            prefetch_tmap(&args.tm_ao);
+            prefetch_tmap(&args.tm_bo);
+        }
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int N = args.N, K = args.K;
+    const int num_m = num_row_tiles(args);
+    const int num_n = (N + BN - 1) / BN;
+    const int total = num_m * num_n;
+    // K blocks: Path A / FP8 first, then Path B
+    const int elems_per_kb = (MODE == MODE_OSC) ? 256 : 128;
+    const int nkb_a = (K + elems_per_kb - 1) / elems_per_kb;
+    const int nkb_b = (MODE == MODE_OSC) ? args.Kop / 64 : 0;
+    const int nkb = nkb_a + nkb_b;
+    const int katoms_total = K / 128;   // 128-channel scale blocks along K
+    const int natoms = (N + 127) / 128;  // 128-row scale blocks of one expert's weights
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            int s = 0;
+            uint32_t ph = 0;
+            for (int t = blockIdx.x; t < total; t += gridDim.x) {
+                const TileInfo ti = tile_info<BN>(args, t, num_m, num_n);
+                const int brow = ti.expert * N + ti.n0;
+                for (int kb = 0; kb < nkb; ++kb) {
+                    if (!wait_bounded(&empty_bar[s], ph ^ 1u, abort_flag, 1)) goto done;
+                    uint8_t* st = smem + s * C::STAGE_BYTES;
+                    if (kb < nkb_a) {
+                        if (MODE == MODE_OSC) {
+                            const int ka = min(2, katoms_total - 2 * kb);  // 128-channel scale blocks in this stage
+                            const uint32_t sfb = (uint32_t)ka * 512u;
+                            mbar_arrive_expect_tx(&full_bar[s], A_BYTES + C::B_BYTES + sfb * (1 + C::SFB_ATOMS));
+                            tma_load_2d(st, &args.tm_a, &full_bar[s], kb * ROW_BYTES, ti.row0);
+                            tma_load_2d(st + A_BYTES, &args.tm_b, &full_bar[s], kb * ROW_BYTES, brow);
+                            const uint8_t* sa = args.sfa + ((int64_t)(ti.sf_row0 / 128) * katoms_total + 2 * kb) * 512;
+                            bulk_load(st + A_BYTES + C::B_BYTES, sa, sfb, &full_bar[s]);
+#pragma unroll
+                            for (int j = 0; j < C::SFB_ATOMS; ++j) {
+                                const int atom = min(ti.n0 / 128 + j, natoms - 1);
+                                const uint8_t* sw = args.sfw +
+                                    (((int64_t)ti.expert * natoms + atom) * katoms_total + 2 * kb) * 512;
+                                bulk_load(st + A_BYTES + C::B_BYTES + C::SFA_BYTES + j * 1024, sw, sfb, &full_bar[s]);
+                            }
+                        } else {
+                            mbar_arrive_expect_tx(&full_bar[s], A_BYTES + C::B_BYTES);
+                            tma_load_2d(st, &args.tm_a, &full_bar[s], kb * ROW_BYTES, ti.row0);
+                            tma_load_2d(st + A_BYTES, &args.tm_b, &full_bar[s], kb * ROW_BYTES, brow);
+                        }
+                    } else {
+                        const int kk = kb - nkb_a;
+                        mbar_arrive_expect_tx(&full_bar[s], A_BYTES + C::B_BYTES);
+                        tma_load_2d(st, &args.tm_ao, &full_bar[s], kk * 64, ti.row0);
+                        tma_load_2d(st + A_BYTES, &args.tm_bo, &full_bar[s], kk * 64, brow);
+                    }
+                    if (++s == STAGES) { s = 0; ph ^= 1u; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // -------------------------------------------------------------- MMA issuer
+        if (lane == 0) {
+            int s = 0;
+            uint32_t ph = 0;
+            int acc = 0;
+            uint32_t acc_ph = 0;
+            constexpr uint32_t IDESC_A = (MODE == MODE_OSC) ? idesc_mxf4(BM, BN) : idesc_e4m3(BM, BN);
+            constexpr uint32_t IDESC_B = idesc_bf16(BM, BN);
+            for (int t = blockIdx.x; t < total; t += gridDim.x) {
+                const TileInfo ti = tile_info<BN>(args, t, num_m, num_n);
+                if (!wait_bounded(&tempty_bar[acc], acc_ph ^ 1u, abort_flag, 2)) goto done;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+                const uint32_t sfb_col_off = (uint32_t)((ti.n0 % 128) / 32);
+                for (int kb = 0; kb < nkb; ++kb) {
+                    if (!wait_bounded(&full_bar[s], ph, abort_flag, 3)) goto done;
+                    tc_fence_after();
+                    const uint32_t sbase = smem_u32(smem + s * C::STAGE_BYTES);
+                    const uint64_t adesc = smem_desc_sw128(sbase);
+                    const uint64_t bdesc = smem_desc_sw128(sbase + A_BYTES);
+                    if (MODE == MODE_OSC && kb < nkb_a) {
+                        const int ka = min(2, katoms_total - 2 * kb);
+                        const uint32_t sfa_s = sbase + A_BYTES + C::B_BYTES;
+                        const uint32_t sfb_s = sfa_s + C::SFA_BYTES;
+                        for (int a = 0; a < ka; ++a) {
+                            tc_copy_sf(tmem_base + C::TM_SFA + a * 4, smem_desc_sf(sfa_s + a * 512));
+#pragma unroll
+                            for (int j = 0; j < C::SFB_ATOMS; ++j)
+                                tc_copy_sf(tmem_base + C::TM_SFB + a * (C::SFB_ATOMS * 4) + j * 4,
+                                           smem_desc_sf(sfb_s + j * 1024 + a * 512));
+                        }
+                        for (int k = 0; k < 2 * ka; ++k) {
+                            const uint32_t sfid = (uint32_t)(k & 1) * 2u;  // byte pair inside the 4-byte scale column
+                            mma_mxf4(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC_A | idesc_sf_ids(sfid, sfid),
+                                     tmem_base + C::TM_SFA + (k >> 1) * 4,
+                                     tmem_base + C::TM_SFB + (k >> 1) * (C::SFB_ATOMS * 4) + sfb_col_off,
+                                     (kb | k) ? 1u : 0u);
+                        }
+                    } else if (MODE == MODE_OSC) {
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)
+                            mma_f16(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC_B, 1u);
+                    } else {
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)
+                            mma_f8(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC_A, (kb | k) ? 1u : 0u);
+                    }
+                    tc_commit(&empty_bar[s]);
+                    if (++s == STAGES) { s = 0; ph ^= 1u; }
+                }
+                tc_commit(&tfull_bar[acc]);
+                if (++acc == ACC) { acc = 0; acc_ph ^= 1u; }
+            }
+        }
+    } else {
+        // ---------------------------------------------------------------- epilogue
+        const int q = warp & 3;  // TMEM lane quarter this warp may read
+        int acc = 0;
+        uint32_t acc_ph = 0;
+        for (int t = blockIdx.x; t < total; t += gridDim.x) {
+            const TileInfo ti = tile_info<BN>(args, t, num_m, num_n);
+            if (!wait_bounded(&tfull_bar[acc], acc_ph, abort_flag, 4)) goto done;
+            tc_fence_after();
+            const int row = ti.row0 + q * 32 + lane;
+            const bool row_ok = row < ti.row_end;
+            float sxr = 1.0f;
+            if (MODE == MODE_FP8 && row_ok) sxr = args.sx[row];
+            uint16_t* yrow = args.Y + (int64_t)row * args.ldy;
+            const float* swp = (MODE == MODE_FP8) ? args.sw + (int64_t)ti.expert * N : nullptr;
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                uint32_t r[32];
+                tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + c * 32), r);
+                tmem_ld_wait();
+                const int col = ti.n0 + c * 32;
+                if (row_ok && col < N) {
+                    uint32_t o[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        float lo = __uint_as_float(r[2 * i]), hi = __uint_as_float(r[2 * i + 1]);
+                        if (MODE == MODE_FP8) {
+                            const float2 w2 = *reinterpret_cast<const float2*>(swp + col + 2 * i);
+                            lo = lo * (sxr * w2.x);
+                            hi = hi * (sxr * w2.y);
+                        }
+                        const __nv_bfloat162 b = __floats2bfloat162_rn(lo, hi);
+                        o[i] = *reinterpret_cast<const uint32_t*>(&b);
+                    }
+                    uint4* dst = reinterpret_cast<uint4*>(yrow + col);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) dst[i] = make_uint4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&tempty_bar[acc]);
+            if (++acc == ACC) { acc = 0; acc_ph ^= 1u; }
+        }
+    }
+
+done:
+    __syncwarp();
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        if (*abort_flag && lane == 0) {
+            // gave up somewhere: let outstanding tensor-core work retire before TMEM goes away
+            tc_commit(drain_bar);
+            int dummy = 0;
+            volatile int* never = &dummy;
+            wait_bounded(drain_bar, 0, never, 5);
+        }
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+// ---------------------------------------------------------------- launchers
+static int g_block_n = 0;
+
+int gemm_block_n() {
+    if (g_block_n == 0) {
+        g_block_n = 256;
+        if (const char* e = getenv("OSC_BLOCK_N")) {
+            const int v = atoi(e);
+            if (v == 128 || v == 192 || v == 256) g_block_n = v;
+        }
+    }
+    return g_block_n;
+}
+
+template <int MODE, int BN>
+static cudaError_t launch_cfg(const GemmArgs& a, cudaStream_t st) {
+    using C = Cfg<MODE, BN>;
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(gemm_kernel<MODE, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             C::SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    int grid = a.num_sms;
+    if (!a.sched) {
+        const int total = ((a.M + BM - 1) / BM) * ((a.N + BN - 1) / BN);
+        if (total <= 0) return cudaSuccess;
+        if (total < grid) grid = total;
+    }
+    gemm_kernel<MODE, BN><<<grid, GEMM_THREADS, C::SMEM_BYTES, st>>>(a);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_gemm_dual(const GemmArgs& a, cudaStream_t st) {
+    switch (gemm_block_n()) {
+        case 128: return launch_cfg<MODE_OSC, 128>(a, st);
+        case 192: return launch_cfg<MODE_OSC, 192>(a, st);
+        default: return launch_cfg<MODE_OSC, 256>(a, st);
+    }
+}
+cudaError_t launch_gemm_fp8(const GemmArgs& a, cudaStream_t st) {
+    switch (gemm_block_n()) {
+        case 128: return launch_cfg<MODE_FP8, 128>(a, st);
+        case 192: return launch_cfg<MODE_FP8, 192>(a, st);
+        default: return launch_cfg<MODE_FP8, 256>(a, st);
+    }
+}
+
+}  // namespace osc

@@ -1,0 +1,5 @@
+// Single translation unit of the library: the kernels share one device-side status word, so they
+// are compiled together (no relocatable device code needed).
+#include "quant_kernels.cu"
+#include "gemm_kernels.cu"
+#include "api.cu"

@@ -1,0 +1,266 @@
+// Memory-bound kernels of the OSC path:
+//   quant_extract_kernel : Algorithm 2 fused - table lookup, back-up of the flagged channels into
+//                          the dense buffer B (xo), zero-out, CalculateScale (E8M0), Quantize (E2M1),
+//                          scales written straight into the 128x4 block layout the tensor core reads.
+//   fp8_quant_kernel     : Section 3.4 fallback - per-row dynamic E4M3 with an fp32 scale.
+//   build_sched_kernel   : grouped (MoE) tile schedule from the expert offsets.
+// All three are used for activations (online) and for weights (offline preparation).
+#include "common.cuh"
+
+namespace osc {
+
+// ---------------------------------------------------------------- conversions
+__device__ __forceinline__ uint32_t e2m1x2(float lo, float hi) {
+    uint16_t r;
+    asm("{ .reg .b8 t;\n\t"
+        "cvt.rn.satfinite.e2m1x2.f32 t, %1, %2;\n\t"
+        "mov.b16 %0, {t, 0}; }"
+        : "=h"(r)
+        : "f"(hi), "f"(lo));
+    return r;
+}
+__device__ __forceinline__ uint32_t e4m3x2(float lo, float hi) {
+    uint16_t r;
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+// ------------------------------------------------------- Algorithm 2, fused
+// CTA tile: 128 rows x 128 channels (4 groups).  256 threads; thread t owns 8 consecutive
+// channels (t % 16) of row (t / 16) + 16 * pass.  Four neighbouring threads share a group.
+constexpr int QE_ROWS = 128;
+constexpr int QE_COLS = 128;
+constexpr int QE_THREADS = 256;
+constexpr int QE_PASSES = QE_ROWS / (QE_THREADS / 16);  // 8
+
+__global__ void __launch_bounds__(QE_THREADS)
+quant_extract_kernel(const uint16_t* __restrict__ X, int64_t ldx, int M, int K,
+                     const uint32_t* __restrict__ mask, const int32_t* __restrict__ prefix,
+                     uint8_t* __restrict__ xq, uint8_t* __restrict__ sf, uint16_t* __restrict__ xo,
+                     int Ko, int Kop, const int32_t* __restrict__ sched, int max_tiles) {
+    __shared__ __align__(16) uint8_t s_sf[512];
+
+    const int cb = blockIdx.x;  // 128-channel block
+    const int tile = blockIdx.y;
+    int row0, row_end, sf_row0;
+    if (sched != nullptr) {
+        if (tile >= sched[0]) return;
+        row0 = sched[1 + tile];
+        row_end = sched[1 + max_tiles + tile];
+        sf_row0 = sched[1 + 2 * max_tiles + tile];
+    } else {
+        row0 = tile * QE_ROWS;
+        row_end = M;
+        sf_row0 = row0;
+    }
+
+    const int tid = threadIdx.x;
+    const int cchunk = tid & 15;  // 8-channel chunk inside the 128-channel block
+    const int gi = cchunk >> 2;   // group inside the block
+    const int sub = cchunk & 3;   // which quarter of the group
+    const int rsub = tid >> 4;    // 0..15
+    const int g = cb * 4 + gi;
+
+    const uint32_t gmask = mask[g];
+    const uint32_t my8 = (gmask >> (sub * 8)) & 0xFFu;
+    const int my_pre = prefix[g] + __popc(gmask & ((1u << (sub * 8)) - 1u));
+
+    uint4 v[QE_PASSES];
+#pragma unroll
+    for (int p = 0; p < QE_PASSES; ++p) {
+        const int r = row0 + rsub + 16 * p;
+        if (r < row_end) {
+            v[p] = *reinterpret_cast<const uint4*>(X + (int64_t)r * ldx + cb * QE_COLS + cchunk * 8);
+        } else {
+            v[p] = make_uint4(0u, 0u, 0u, 0u);
+        }
+    }
+
+#pragma unroll
+    for (int p = 0; p < QE_PASSES; ++p) {
+        const int rl = rsub + 16 * p;  // row inside the tile
+        const int r = row0 + rl;
+        uint32_t w[4] = {v[p].x, v[p].y, v[p].z, v[p].w};
+        // back up + zero the flagged channels (rare: at most a few bits set)
+        if (my8 != 0u) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                if ((my8 >> j) & 1u) {
+                    const uint32_t word = w[j >> 1];
+                    const uint16_t bits = (j & 1) ? (uint16_t)(word >> 16) : (uint16_t)(word & 0xFFFFu);
+                    if (r < row_end) xo[(int64_t)r * Kop + my_pre + __popc(my8 & ((1u << j) - 1u))] = bits;
+                    w[j >> 1] = (j & 1) ? (word & 0x0000FFFFu) : (word & 0xFFFF0000u);
+                }
+            }
+        }
+        // amax over my 8 channels on the bf16 magnitude bits (monotone in the value)
+        uint32_t am = 0;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            am = max(am, w[i] & 0x7FFFu);
+            am = max(am, (w[i] >> 16) & 0x7FFFu);
+        }
+        am = max(am, __shfl_xor_sync(0xFFFFFFFFu, am, 1));
+        am = max(am, __shfl_xor_sync(0xFFFFFFFFu, am, 2));
+        // CalculateScale: E8M0 code = biased exponent of amax - 2, floored at 0 (2^(floor(log2 amax) - 2))
+        const int ex = (int)(am >> 7);
+        int code = max(ex - 2, 0);
+        if (ex == 255) code = 255;
+        // Quantize: x * 2^(127 - code) is exact in fp32, then hardware E2M1 rounding (nearest-even, saturating)
+        const float inv = __uint_as_float((uint32_t)(254 - min(code, 253)) << 23);
+        uint32_t packed = 0;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float lo = __uint_as_float(w[i] << 16) * inv;
+            const float hi = __uint_as_float(w[i] & 0xFFFF0000u) * inv;
+            packed |= (e2m1x2(lo, hi) & 0xFFu) << (8 * i);
+        }
+        if (r < row_end) {
+            *reinterpret_cast<uint32_t*>(xq + (int64_t)r * (K / 2) + cb * (QE_COLS / 2) + cchunk * 4) = packed;
+        }
+        if (sub == 0) s_sf[(rl & 31) * 16 + (rl >> 5) * 4 + gi] = (uint8_t)code;
+    }
+
+    // zero the pad columns of xo once per row tile
+    if (cb == 0 && Kop > Ko) {
+        const int npad = Kop - Ko;
+        for (int i = tid; i < QE_ROWS * npad; i += QE_THREADS) {
+            const int r = row0 + i / npad;
+            if (r < row_end) xo[(int64_t)r * Kop + Ko + i % npad] = 0;
+        }
+    }
+
+    __syncthreads();
+    if (tid < 32) {
+        const int64_t blk = (int64_t)(sf_row0 / 128) * (K / 128) + cb;
+        *reinterpret_cast<uint4*>(sf + blk * 512 + tid * 16) = *reinterpret_cast<const uint4*>(s_sf + tid * 16);
+    }
+}
+
+// ------------------------------------------------------ per-row dynamic E4M3
+// One CTA per row.  The row is kept in registers between the amax pass and the encode pass
+// when it fits (K <= 256 threads x 8 chunks x 8 elements = 16384), else re-read.
+constexpr int F8_THREADS = 256;
+constexpr int F8_MAXCH = 8;
+
+__global__ void __launch_bounds__(F8_THREADS)
+fp8_quant_kernel(const uint16_t* __restrict__ X, int64_t ldx, int M, int K, uint8_t* __restrict__ x8,
+                 float* __restrict__ sx) {
+    __shared__ float s_red[F8_THREADS / 32];
+    const int r = blockIdx.x;
+    const uint16_t* xrow = X + (int64_t)r * ldx;
+    const int nch = K / 8;  // 16-byte chunks in the row
+    const int tid = threadIdx.x;
+
+    uint4 v[F8_MAXCH];
+    uint32_t am = 0;
+#pragma unroll
+    for (int i = 0; i < F8_MAXCH; ++i) {
+        const int c = tid + i * F8_THREADS;
+        if (c < nch) {
+            v[i] = *reinterpret_cast<const uint4*>(xrow + c * 8);
+            am = max(am, max(max(v[i].x & 0x7FFFu, (v[i].x >> 16) & 0x7FFFu), max(v[i].y & 0x7FFFu, (v[i].y >> 16) & 0x7FFFu)));
+            am = max(am, max(max(v[i].z & 0x7FFFu, (v[i].z >> 16) & 0x7FFFu), max(v[i].w & 0x7FFFu, (v[i].w >> 16) & 0x7FFFu)));
+        }
+    }
+    for (int c = tid + F8_MAXCH * F8_THREADS; c < nch; c += F8_THREADS) {
+        const uint4 u = *reinterpret_cast<const uint4*>(xrow + c * 8);
+        am = max(am, max(max(u.x & 0x7FFFu, (u.x >> 16) & 0x7FFFu), max(u.y & 0x7FFFu, (u.y >> 16) & 0x7FFFu)));
+        am = max(am, max(max(u.z & 0x7FFFu, (u.z >> 16) & 0x7FFFu), max(u.w & 0x7FFFu, (u.w >> 16) & 0x7FFFu)));
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) am = max(am, __shfl_xor_sync(0xFFFFFFFFu, am, o));
+    if ((tid & 31) == 0) s_red[tid >> 5] = __uint_as_float(am << 16);
+    __syncthreads();
+    float amax = s_red[0];
+#pragma unroll
+    for (int i = 1; i < F8_THREADS / 32; ++i) amax = fmaxf(amax, s_red[i]);
+
+    // amax' = max(amax, 2^-40); sx = amax'/448; inv = 448/amax' (IEEE fp32 divisions)
+    const float amaxp = fmaxf(amax, __uint_as_float((uint32_t)(127 - 40) << 23));
+    const float scale = __fdiv_rn(amaxp, 448.0f);
+    const float inv = __fdiv_rn(448.0f, amaxp);
+    if (tid == 0) sx[r] = scale;
+
+    auto encode8 = [&](const uint4& u) -> uint2 {
+        const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+        uint32_t h[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float lo = __fmul_rn(__uint_as_float(w[i] << 16), inv);
+            const float hi = __fmul_rn(__uint_as_float(w[i] & 0xFFFF0000u), inv);
+            h[i] = e4m3x2(lo, hi) & 0xFFFFu;
+        }
+        return make_uint2(h[0] | (h[1] << 16), h[2] | (h[3] << 16));
+    };
+    uint8_t* orow = x8 + (int64_t)r * K;
+#pragma unroll
+    for (int i = 0; i < F8_MAXCH; ++i) {
+        const int c = tid + i * F8_THREADS;
+        if (c < nch) *reinterpret_cast<uint2*>(orow + c * 8) = encode8(v[i]);
+    }
+    for (int c = tid + F8_MAXCH * F8_THREADS; c < nch; c += F8_THREADS) {
+        const uint4 u = *reinterpret_cast<const uint4*>(xrow + c * 8);
+        *reinterpret_cast<uint2*>(orow + c * 8) = encode8(u);
+    }
+}
+
+// ------------------------------------------------------------ grouped schedule
+// sched[0] = number of 128-row tiles; then four arrays of max_tiles entries:
+// first row, end row (exclusive, the expert's end), first scale row, expert.
+__global__ void build_sched_kernel(const int32_t* __restrict__ off, int E, int32_t* __restrict__ sched,
+                                   int max_tiles) {
+    __shared__ int s_tiles[1024];
+    const int tid = threadIdx.x;
+    // serial prefix by one thread: E is small (hundreds) and this runs once per call
+    if (tid == 0) {
+        int acc = 0;
+        for (int e = 0; e < E; ++e) {
+            s_tiles[e] = acc;
+            acc += (off[e + 1] - off[e] + 127) / 128;
+        }
+        sched[0] = acc < max_tiles ? acc : max_tiles;
+    }
+    __syncthreads();
+    for (int e = tid; e < E; e += blockDim.x) {
+        const int m = off[e + 1] - off[e];
+        const int nt = (m + 127) / 128;
+        const int t0 = s_tiles[e];
+        for (int i = 0; i < nt; ++i) {
+            const int t = t0 + i;
+            if (t < max_tiles) {
+                sched[1 + t] = off[e] + i * 128;
+                sched[1 + max_tiles + t] = off[e + 1];
+                sched[1 + 2 * max_tiles + t] = t * 128;
+                sched[1 + 3 * max_tiles + t] = e;
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------ launchers
+cudaError_t launch_quant_extract(const void* X, int64_t ldx, int M, int K, const uint32_t* mask,
+                                 const int32_t* prefix, void* xq, void* sf, void* xo, int Ko, int Kop,
+                                 const int32_t* sched, int max_tiles, cudaStream_t st) {
+    const int tiles = sched ? max_tiles : (M + QE_ROWS - 1) / QE_ROWS;
+    if (tiles <= 0) return cudaSuccess;
+    dim3 grid(K / QE_COLS, tiles);
+    quant_extract_kernel<<<grid, QE_THREADS, 0, st>>>(static_cast<const uint16_t*>(X), ldx, M, K, mask, prefix,
+                                                      static_cast<uint8_t*>(xq), static_cast<uint8_t*>(sf),
+                                                      static_cast<uint16_t*>(xo), Ko, Kop, sched, max_tiles);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_fp8_quant(const void* X, int64_t ldx, int M, int K, void* x8, void* sx, cudaStream_t st) {
+    if (M <= 0) return cudaSuccess;
+    fp8_quant_kernel<<<M, F8_THREADS, 0, st>>>(static_cast<const uint16_t*>(X), ldx, M, K,
+                                               static_cast<uint8_t*>(x8), static_cast<float*>(sx));
+    return cudaGetLastError();
+}
+
+cudaError_t launch_build_sched(const int32_t* off, int E, int32_t* sched, int max_tiles, cudaStream_t st) {
+    build_sched_kernel<<<1, 256, 0, st>>>(off, E, sched, max_tiles);
+    return cudaGetLastError();
+}
+
+}  // namespace osc

@@ -1,0 +1,82 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports every symbol the
+header declares, and rejects bad arguments before touching the device."""
+import ctypes as C
+import os
+import re
+
+import numpy as np
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def B():
+    import __graft_entry__ as g
+    g.build()
+    from paper_2604_12782_b200 import binding
+    return binding
+
+
+def test_library_exports_every_declared_symbol(B):
+    with open(os.path.join(ROOT, "include", "osc.h")) as f:
+        text = f.read()
+    declared = set(re.findall(r"\b(osc_[a-z0-9_]+)\s*\(", text))
+    assert len(declared) >= 20
+    lib = C.CDLL(B.LIB_PATH)
+    for name in declared:
+        assert hasattr(lib, name), name
+    assert declared == set(B.EXPORTS), declared ^ set(B.EXPORTS)
+
+
+def test_status_strings(B):
+    assert B.osc_status_string(0) == "OSC_OK"
+    assert B.osc_status_string(-3) == "OSC_ERR_LUT"
+    assert B.osc_status_string(-8) == "OSC_ERR_TIMEOUT"
+
+
+def test_weight_sizes_and_table_validation(B):
+    lut = np.full((4096 // 32, 2), -1, np.int8)
+    lut[:, 0] = 3
+    lut[:, 1] = 17
+    sz = B.osc_weight_sizes(1, 6144, 4096, lut)
+    assert (sz.K_o, sz.K_o_pad) == (256, 256)
+    assert sz.wq_bytes == 6144 * 2048 and sz.sfw_bytes == 48 * 32 * 512 and sz.wo_bytes == 6144 * 256 * 2
+    lut1 = np.full((16, 1), -1, np.int8)
+    lut1[3] = 9
+    sz = B.osc_weight_sizes(2, 64, 512, lut1)
+    assert (sz.K_o, sz.K_o_pad) == (1, 64) and sz.sfw_bytes == 2 * 1 * 4 * 512
+    assert B.osc_weight_sizes(1, 64, 512, np.full((16, 1), -1, np.int8)).wo_bytes == 0
+
+    for bad, status in [((1, 64, 500), -2), ((1, 60, 512), -2), ((0, 64, 512), -1)]:
+        with pytest.raises(B.OscError) as e:
+            B.osc_weight_sizes(*bad, np.full((16, 1), -1, np.int8))
+        assert e.value.status == status
+    dup = np.full((16, 2), 5, np.int8)
+    with pytest.raises(B.OscError) as e:
+        B.osc_weight_sizes(1, 64, 512, dup)
+    assert e.value.status == -3 and "twice" in str(e.value)
+    oob = np.full((16, 1), 32, np.int8)
+    with pytest.raises(B.OscError) as e:
+        B.osc_weight_sizes(1, 64, 512, oob)
+    assert e.value.status == -3
+
+
+def test_null_and_misaligned_arguments_launch_nothing(B):
+    lib = C.CDLL(B.LIB_PATH)
+    lut = np.full((4, 1), -1, np.int8)
+    h = C.c_void_p()
+    f = lib.osc_prepare_weights
+    f.argtypes = B._SIGS["osc_prepare_weights"][1]
+    assert f(None, 64, 128, 128, lut.ctypes.data, 1, None, None, None, None, None, C.byref(h)) == -1
+    assert h.value is None
+    # misaligned device pointer (never dereferenced: validation comes first)
+    assert f(0x1008, 64, 128, 128, lut.ctypes.data, 1, 0x2000, 0x3000, None, 0x4000, None, C.byref(h)) == -4
+    assert f(0x1000, 64, 128, 100, lut.ctypes.data, 1, 0x2000, 0x3000, None, 0x4000, None, C.byref(h)) == -2
+    q = lib.osc_fp8_quantize
+    q.argtypes = B._SIGS["osc_fp8_quantize"][1]
+    assert q(0x1000, -1, 128, 128, 0x2000, 0x3000, None) == -1
+    assert q(0x1000, 4, 100, 128, 0x2000, 0x3000, None) == -2
+    assert q(0x1000, 0, 128, 128, None, None, None) == 0          # M == 0 is a no-op
+    assert q(0x1000, 4, 128, 132, 0x2000, 0x3000, None) == -4     # ldx not a multiple of 8
+    assert lib.osc_linear(None, None, 0, 0, None, 0, None, 0, None) == -1
