@@ -1,0 +1,501 @@
+#!/usr/bin/env python
+"""Benchmark of the OSC dual-path linear on B200 (one JSON line on stdout).
+
+A step is one pass of the online hot path over one batch: `osc_linear` (fused
+extract + MXFP4 quantize kernel, then the dual-path tcgen05 GEMM) on the
+Qwen3-8B QKV projection, M=8192 tokens, K=4096, N=6144, two protected channels
+per 32-group (K_o=256).  Inputs are seeded and synthetic (outlier-planted
+activations, N(0,0.02) weights); the offline weight split is done once before
+timing, as in the paper.
+
+  value       TFLOP/s of useful work, 2*M*N*(K+K_o) / step time, inputs resident in HBM
+  e2e         the same with X in pinned host memory and Y copied back, copies inside the timed region
+  roofline    the dual-path GEMM kernel against the tensor peak of its own FLOP mix
+              (FP4 peak = 4 x, measured BF16 peak from MEASURED_PEAKS.json)
+  cpu_baseline the CPU oracle timed on a bounded sample of the same workload (rank 0, N=1 only)
+  extra       the step against the dual-path roofline of the whole linear, the quantizer's
+              HBM fraction, and the same build's FP8 W8A8 linear on the same shape
+
+Between timed steps the buffers rotate over 4 independent sets (inputs, workspace,
+outputs and prepared weights: ~0.9 GB, 7x the L2), so no step finds its data in L2.
+
+`--impl reference` times the CPU oracle instead (host cores, bounded sample per step).
+`--sweep` prints a table over all benchmark shapes to stderr and gpurun_out/ (not a bench line).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2604_12782_b200 import roofline, synth  # noqa: E402
+
+WORKLOAD = {"name": "qwen3-8b-qkv", "M": 8192, "K": 4096, "N": 6144, "ch_per_group": 2}
+NSETS = 4
+METRIC = "OSC linear TFLOP/s"
+
+# DRAM traffic of one dual-path GEMM launch on the bench workload (dram__bytes_read.sum +
+# dram__bytes_write.sum from an ncu capture; see profiles/).  None until a capture exists.
+GEMM_TRAFFIC_BYTES = None
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"bf16_tflops": p["bf16_tflops"], "bf16_tflops_sustained": p.get("bf16_tflops_sustained"),
+                "hbm_gbs": p["hbm_gbs"], "source": "measured"}
+    return {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0, "source": "fallback"}
+
+
+# ----------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the GPU is busy."""
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        names = {"hw_slowdown": nv.nvmlClocksEventReasonHwSlowdown if hasattr(nv, "nvmlClocksEventReasonHwSlowdown") else 0x8,
+                 "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20, "sw_power_cap": 0x4,
+                 "hw_power_brake": 0x80}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for k, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(0.002)
+
+    def start(self):
+        if self.nv:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread:
+            self._thread.join()
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+# ---------------------------------------------------------------------- reference arm
+def oracle_sample_step(oracle, case, wts, rows):
+    """One bounded step of the CPU oracle: Algorithm 2 on `rows` activation rows, then Eq. 5."""
+    act = oracle.quantize_extract(case["X"][:rows], case["lut"])
+    oracle.gemm_dual(act, wts)
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    rows = args.ref_rows
+    case = synth.osc_linear_case(0, rows, WORKLOAD["K"], WORKLOAD["N"], WORKLOAD["ch_per_group"])
+    wts = oracle.prepare_weights(case["W"], case["lut"])
+    ko = wts["K_o"]
+    for _ in range(args.warmup):
+        oracle_sample_step(oracle, case, wts, min(rows, 8))
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_sample_step(oracle, case, wts, rows)
+    dt = (time.perf_counter() - t0) / max(args.steps, 1)
+    flops = 2.0 * rows * WORKLOAD["N"] * (WORKLOAD["K"] + ko)
+    val = flops / dt / 1e12
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": "TFLOP/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD["name"], **{k: WORKLOAD[k] for k in ("M", "K", "N")}, "K_o": ko},
+            "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": oracle.num_threads(), "kind": "oracle",
+                             "sample": f"{rows} of {WORKLOAD['M']} activation rows x all N per step "
+                                       "(weights prepared once, as on the GPU)"},
+            "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------ GPU arm
+def dev_bf16(torch, bits):
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).view(torch.bfloat16).cuda()
+
+
+class OscProblem:
+    """NSETS rotating buffer sets of one OSC linear."""
+
+    def __init__(self, torch, B, case, nsets):
+        self.B, self.M, self.K, self.N = B, case["M"], case["K"], case["N"]
+        X0, W0 = dev_bf16(torch, case["X"]), dev_bf16(torch, case["W"])
+        self.X = [X0 if i == 0 else torch.roll(X0, 97 * i, 0).contiguous() for i in range(nsets)]
+        self.w = []
+        for i in range(nsets):
+            Wi = W0 if i == 0 else torch.roll(W0, 61 * i, 0).contiguous()
+            self.w.append(B.osc_prepare_weights(Wi, case["lut"]))
+        self.sz = B.osc_act_sizes(self.w[0], self.M)
+        self.ws = [torch.empty(self.sz.workspace_bytes, dtype=torch.uint8, device="cuda") for _ in range(nsets)]
+        self.Y = [torch.empty(self.M, self.N, dtype=torch.bfloat16, device="cuda") for _ in range(nsets)]
+        self.K_o, self.K_o_pad = self.w[0].K_o, self.w[0].K_o_pad
+        self.n = nsets
+
+    def step(self, i):
+        j = i % self.n
+        self.B.osc_linear(self.w[j], self.X[j], self.Y[j], self.ws[j])
+
+    def views(self, j):
+        sz, ws = self.sz, self.ws[j]
+        return ws[sz.xq_offset:], ws[sz.sfa_offset:], ws[sz.xo_offset:]
+
+    def quant(self, i):
+        j = i % self.n
+        xq, sfa, xo = self.views(j)
+        self.B.osc_quantize_extract(self.w[j], self.X[j], xq, sfa, xo)
+
+    def gemm(self, i):
+        j = i % self.n
+        xq, sfa, xo = self.views(j)
+        self.B.osc_gemm_dual(self.w[j], xq, sfa, xo, self.M, self.Y[j])
+
+
+class Fp8Problem:
+    def __init__(self, torch, B, case, nsets):
+        self.B, self.M, self.K, self.N = B, case["M"], case["K"], case["N"]
+        X0, W0 = dev_bf16(torch, case["X"]), dev_bf16(torch, case["W"])
+        self.X = [X0 if i == 0 else torch.roll(X0, 97 * i, 0).contiguous() for i in range(nsets)]
+        self.w = [B.osc_fp8_prepare_weights(W0 if i == 0 else torch.roll(W0, 61 * i, 0).contiguous())
+                  for i in range(nsets)]
+        self.sz = B.osc_fp8_act_sizes(self.w[0], self.M)
+        self.ws = [torch.empty(self.sz.workspace_bytes, dtype=torch.uint8, device="cuda") for _ in range(nsets)]
+        self.Y = [torch.empty(self.M, self.N, dtype=torch.bfloat16, device="cuda") for _ in range(nsets)]
+        self.n = nsets
+
+    def step(self, i):
+        j = i % self.n
+        self.B.osc_fp8_linear(self.w[j], self.X[j], self.Y[j], self.ws[j])
+
+    def quant(self, i):
+        j = i % self.n
+        self.B.osc_fp8_quantize(self.X[j], self.ws[j][self.sz.x8_offset:], self.ws[j][self.sz.sx_offset:])
+
+    def gemm(self, i):
+        j = i % self.n
+        self.B.osc_fp8_gemm(self.w[j], self.ws[j][self.sz.x8_offset:], self.ws[j][self.sz.sx_offset:], self.M,
+                            self.Y[j])
+
+
+def time_loop(torch, fn, steps, warmup):
+    """Average milliseconds per call of fn(i) over `steps` calls, CUDA events on the current stream."""
+    for i in range(warmup):
+        fn(i)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(steps):
+        fn(i)
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / max(steps, 1)
+
+
+def time_split(torch, prob, steps):
+    """Per-kernel averages (ms): events between the quantizer and the GEMM of every step."""
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(steps)]
+    torch.cuda.synchronize()
+    for i in range(steps):
+        ev[i][0].record()
+        prob.quant(i)
+        ev[i][1].record()
+        prob.gemm(i)
+        ev[i][2].record()
+    torch.cuda.synchronize()
+    tq = sum(e[0].elapsed_time(e[1]) for e in ev) / steps
+    tg = sum(e[1].elapsed_time(e[2]) for e in ev) / steps
+    return tq, tg
+
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    from paper_2604_12782_b200 import binding as B   # raises if the CUDA library is missing
+
+    pk = load_peaks()
+    peaks = roofline.peaks(pk["bf16_tflops"], pk["hbm_gbs"])
+    M, K, N = WORKLOAD["M"], WORKLOAD["K"], WORKLOAD["N"]
+    case = synth.osc_linear_case(rank, M, K, N, WORKLOAD["ch_per_group"])   # replicas: one seed per rank
+    prob = OscProblem(torch, B, case, NSETS)
+    Ko, Kop = prob.K_o, prob.K_o_pad
+    torch.cuda.synchronize()
+    B.osc_sync_check()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(local)
+    # ---- timed region: K steps of osc_linear, inputs resident in HBM
+    for i in range(args.warmup):
+        prob.step(i)
+    barrier()
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(args.steps):
+        prob.step(i)
+    e1.record()
+    barrier()
+    ms = e0.elapsed_time(e1) / args.steps
+    # ---- same steps again with events between the two kernels (roofline of each kernel)
+    tq, tg = time_split(torch, prob, args.steps)
+    clocks = sampler.stop()
+    B.osc_sync_check()
+
+    if world > 1:
+        t = torch.tensor([ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    if args.only_osc:
+        print(f"osc_linear {ms:.4f} ms/step (quantizer {tq:.4f}, gemm {tg:.4f})", file=sys.stderr)
+        return
+
+    flops4, flops16 = roofline.osc_flops(M, N, K, Ko)
+    flops = flops4 + flops16
+    value = world * flops / (ms * 1e-3) / 1e12
+
+    # ---- end to end through the C ABI with host buffers (copies inside the timed region)
+    Xh = torch.from_numpy(case["X"].view(np.int16)).view(torch.bfloat16).pin_memory()
+    Yh = torch.empty(M, N, dtype=torch.bfloat16).pin_memory()
+    Xd, Yd = prob.X[0], prob.Y[0]
+
+    def e2e_step(i):
+        Xd.copy_(Xh, non_blocking=True)
+        B.osc_linear(prob.w[0], Xd, Yd, prob.ws[0])
+        Yh.copy_(Yd, non_blocking=True)
+
+    e2e_steps = max(3, min(args.steps, 20))
+    ms_e2e = time_loop(torch, e2e_step, e2e_steps, 3)
+    if world > 1:
+        t = torch.tensor([ms_e2e], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_e2e = float(t.item())
+    e2e_value = world * flops / (ms_e2e * 1e-3) / 1e12
+
+    # ---- the same build's FP8 W8A8 linear on the same shape (the paper's comparison point)
+    f8case = {"X": case["X"], "W": case["W"], "M": M, "K": K, "N": N}
+    f8 = Fp8Problem(torch, B, f8case, NSETS)
+    ms_f8 = time_loop(torch, f8.step, args.steps, args.warmup)
+    f8q, f8g = time_split(torch, f8, args.steps)
+    B.osc_sync_check()
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # roofline of the dominant kernel (dual-path GEMM): tensor peak of its own FLOP mix
+    p_mix = flops / (flops4 / peaks["fp4"] + flops16 / peaks["bf16"]) / 1e12
+    gemm_tflops = flops / (tg * 1e-3) / 1e12
+    roof = {"bound": "tensor", "kernel": "gemm_kernel<MODE_OSC>", "achieved": gemm_tflops, "peak": p_mix,
+            "unit": "TFLOP/s", "frac": gemm_tflops / p_mix, "traffic": GEMM_TRAFFIC_BYTES,
+            "peak_basis": f"{pk['source']} bf16 {pk['bf16_tflops']} TFLOP/s x4 for FP4 (burst), FLOP-mix weighted",
+            "ms": tg}
+    qbytes = roofline.quantize_extract_bytes(M, K, Kop)
+    t_roof = roofline.osc_roofline_seconds(M, N, K, Ko, peaks)
+    extra = {
+        "pct_dual_path_roofline": 100.0 * t_roof / (ms * 1e-3),
+        "roofline_us": t_roof * 1e6,
+        "quant_extract": {"ms": tq, "bytes": qbytes, "gbs": qbytes / (tq * 1e-3) / 1e9,
+                          "frac_hbm": qbytes / (tq * 1e-3) / peaks["hbm"]},
+        "fp8_linear": {"ms": ms_f8, "quant_ms": f8q, "gemm_ms": f8g,
+                       "tflops": roofline.fp8_flops(M, N, K) / (ms_f8 * 1e-3) / 1e12,
+                       "gemm_frac_fp8_peak": roofline.fp8_flops(M, N, K) / (f8g * 1e-3) / peaks["fp8"]},
+        "speedup_vs_own_fp8_linear": ms_f8 / ms,
+        "speedup_vs_own_fp8_gemm_only": f8g / tg,
+        "paper_analytic_speedup_vs_w8a8": roofline.analytic_speedup_vs_w8a8(32, WORKLOAD["ch_per_group"]),
+        "block_n": int(os.environ.get("OSC_BLOCK_N", "256")),
+    }
+
+    cpu = None
+    if world == 1 and not args.no_cpu:
+        import oracle
+        oracle.build()
+        rows = args.cpu_rows
+        wts = oracle.prepare_weights(case["W"], case["lut"])
+        t0 = time.perf_counter()
+        oracle_sample_step(oracle, case, wts, rows)
+        dt = time.perf_counter() - t0
+        cpu = {"value": 2.0 * rows * N * (K + Ko) / dt / 1e12, "unit": "TFLOP/s", "cores": oracle.num_threads(),
+               "kind": "oracle", "seconds": dt,
+               "sample": f"first {rows} of {M} activation rows x all N={N} (Algorithm 2 + Eq. 5; weights prepared once)"}
+
+    line = {"metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "fp4(e2m1)+e8m0 x bf16 branch, fp32 accumulate", "data": "synthetic",
+            "config": {"workload": WORKLOAD["name"], "M": M, "K": K, "N": N, "K_o": Ko,
+                       "l2": f"rotating {NSETS} buffer sets (inputs, weights, workspace, outputs)",
+                       "parallelism": "replicas only" if world > 1 else "1 gpu"},
+            "roofline": roof, "cpu_baseline": cpu,
+            "e2e": {"value": e2e_value, "unit": "TFLOP/s", "ms_per_step": ms_e2e,
+                    "h2d_bytes_per_step": int(Xh.numel() * 2), "d2h_bytes_per_step": int(Yh.numel() * 2)},
+            "gpu_launches": 2 * args.steps, "clocks": clocks, "extra": extra}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# -------------------------------------------------------------------------------- sweep
+def run_sweep(args):
+    """All benchmark shapes: OSC linears vs own FP8 on the same shape, FP8 down projection, MoE."""
+    import torch
+    from paper_2604_12782_b200 import binding as B
+    torch.cuda.set_device(0)
+    pk = load_peaks()
+    peaks = roofline.peaks(pk["bf16_tflops"], pk["hbm_gbs"])
+    rows = []
+    steps, warm = args.steps, args.warmup
+
+    def osc_row(name, M, K, N, cpg, seed=0):
+        case = synth.osc_linear_case(seed, M, K, N, cpg)
+        nsets = NSETS if M >= 1024 else 8
+        p = OscProblem(torch, B, case, nsets)
+        ms = time_loop(torch, p.step, steps, warm)
+        tq, tg = time_split(torch, p, steps)
+        f8 = Fp8Problem(torch, B, case, nsets)
+        ms8 = time_loop(torch, f8.step, steps, warm)
+        q8, g8 = time_split(torch, f8, steps)
+        B.osc_sync_check()
+        f4, f16 = roofline.osc_flops(M, N, K, p.K_o)
+        troof = roofline.osc_roofline_seconds(M, N, K, p.K_o, peaks)
+        rows.append({"name": name, "M": M, "K": K, "N": N, "K_o": p.K_o, "ms": ms, "quant_ms": tq, "gemm_ms": tg,
+                     "tflops": (f4 + f16) / ms / 1e9, "pct_roofline": 100 * troof / (ms * 1e-3),
+                     "roof_us": troof * 1e6, "fp8_ms": ms8, "fp8_quant_ms": q8, "fp8_gemm_ms": g8,
+                     "speedup_vs_fp8": ms8 / ms, "speedup_gemm_only": g8 / tg,
+                     "quant_gbs": roofline.quantize_extract_bytes(M, K, p.K_o_pad) / tq / 1e6})
+        del p, f8
+        torch.cuda.empty_cache()
+
+    def fp8_row(name, M, K, N, seed=0):
+        case = synth.fp8_linear_case(seed, M, K, N)
+        nsets = NSETS if M >= 1024 else 8
+        f8 = Fp8Problem(torch, B, case, nsets)
+        ms8 = time_loop(torch, f8.step, steps, warm)
+        q8, g8 = time_split(torch, f8, steps)
+        B.osc_sync_check()
+        troof = roofline.fp8_roofline_seconds(M, N, K, peaks)
+        rows.append({"name": name, "M": M, "K": K, "N": N, "ms": ms8, "quant_ms": q8, "gemm_ms": g8,
+                     "tflops": roofline.fp8_flops(M, N, K) / ms8 / 1e9, "pct_roofline": 100 * troof / (ms8 * 1e-3),
+                     "roof_us": troof * 1e6, "quant_gbs": roofline.fp8_quantize_bytes(M, K) / q8 / 1e6})
+        del f8
+        torch.cuda.empty_cache()
+
+    for M in (16, 128, 2048, 8192):
+        osc_row("qkv", M, 4096, 6144, 2)
+    for M in (128, 2048, 8192):
+        osc_row("gate_up", M, 4096, 24576, 1)
+        fp8_row("down_fp8", M, 12288, 4096)
+    osc_row("layer.qkv", 4096, 4096, 6144, 2)
+    osc_row("layer.o_proj", 4096, 4096, 4096, 1)
+    osc_row("layer.gate_up", 4096, 4096, 24576, 1)
+    fp8_row("layer.down_fp8", 4096, 12288, 4096)
+
+    # MoE: 128 experts, top-8 of 8192 tokens, Zipf(1.1) load
+    counts = synth.zipf_expert_rows()
+    E = counts.size
+    off = torch.from_numpy(synth.offsets_from_counts(counts)).cuda()
+    c = synth.moe_gate_up_case(E, counts, weight_pool=8)
+    Xd = dev_bf16(torch, c["X"])
+    Wd = dev_bf16(torch, c["W"].reshape(E * c["N"], c["K"])).view(E, c["N"], c["K"])
+    w = B.osc_prepare_weights_grouped(Wd, c["lut"])
+    sz = B.osc_act_sizes(w, c["M"])
+    ws = torch.empty(sz.workspace_bytes, dtype=torch.uint8, device="cuda")
+    Y = torch.empty(c["M"], c["N"], dtype=torch.bfloat16, device="cuda")
+    ms = time_loop(torch, lambda i: B.osc_linear_grouped(w, Xd, off, Y, ws), steps, warm)
+    B.osc_sync_check()
+    Mt, K, N = c["M"], c["K"], c["N"]
+    f4, f16 = roofline.osc_flops(Mt, N, K, w.K_o)
+    byts = 2.0 * Mt * K + E * (N * K / 2 + N * K / 32 + 2.0 * N * w.K_o) + 2.0 * Mt * N
+    troof = max(f4 / peaks["fp4"] + f16 / peaks["bf16"], byts / peaks["hbm"])
+    rows.append({"name": "moe.gate_up(grouped)", "M": Mt, "K": K, "N": N, "K_o": w.K_o, "ms": ms,
+                 "tflops": (f4 + f16) / ms / 1e9, "pct_roofline": 100 * troof / (ms * 1e-3), "roof_us": troof * 1e6})
+    del Xd, Wd, w, ws, Y
+    c = synth.moe_down_case(E, counts, weight_pool=8)
+    Xd = dev_bf16(torch, c["X"])
+    Wd = dev_bf16(torch, c["W"].reshape(E * c["N"], c["K"])).view(E, c["N"], c["K"])
+    w = B.osc_fp8_prepare_weights_grouped(Wd)
+    sz = B.osc_fp8_act_sizes(w, c["M"])
+    ws = torch.empty(sz.workspace_bytes, dtype=torch.uint8, device="cuda")
+    Y = torch.empty(c["M"], c["N"], dtype=torch.bfloat16, device="cuda")
+    ms = time_loop(torch, lambda i: B.osc_fp8_linear_grouped(w, Xd, off, Y, ws), steps, warm)
+    B.osc_sync_check()
+    Mt, K, N = c["M"], c["K"], c["N"]
+    byts = 2.0 * Mt * K + E * (N * K + 4.0 * N) + 2.0 * Mt * N
+    troof = max(roofline.fp8_flops(Mt, N, K) / peaks["fp8"], byts / peaks["hbm"])
+    rows.append({"name": "moe.down_fp8(grouped)", "M": Mt, "K": K, "N": N, "ms": ms,
+                 "tflops": roofline.fp8_flops(Mt, N, K) / ms / 1e9, "pct_roofline": 100 * troof / (ms * 1e-3),
+                 "roof_us": troof * 1e6})
+
+    os.makedirs(os.path.join(ROOT, "gpurun_out"), exist_ok=True)
+    with open(os.path.join(ROOT, "gpurun_out", "sweep.json"), "w") as f:
+        json.dump({"peaks": pk, "block_n": os.environ.get("OSC_BLOCK_N", "256"), "rows": rows}, f, indent=1)
+    for r in rows:
+        print(json.dumps(r), file=sys.stderr)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="osc", choices=["osc", "reference"])
+    ap.add_argument("--no-cpu", action="store_true", help="skip the cpu_baseline leg")
+    ap.add_argument("--cpu-rows", type=int, default=1024, help="activation rows of the cpu_baseline sample")
+    ap.add_argument("--ref-rows", type=int, default=128, help="activation rows per step of --impl reference")
+    ap.add_argument("--sweep", action="store_true")
+    ap.add_argument("--only-osc", action="store_true",
+                    help="skip the e2e, FP8 and cpu legs (short runs under a profiler; prints no bench line)")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "osc" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    elif args.sweep:
+        run_sweep(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

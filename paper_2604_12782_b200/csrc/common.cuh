@@ -32,6 +32,7 @@ struct GemmArgs {
     const int32_t* sched;  // grouped tile schedule or nullptr
     int max_tiles;
     int num_sms;
+    int dbg;             // timing experiments only (0 in normal use)
 };
 cudaError_t launch_gemm_dual(const GemmArgs& a, cudaStream_t st);
 cudaError_t launch_gemm_fp8(const GemmArgs& a, cudaStream_t st);
