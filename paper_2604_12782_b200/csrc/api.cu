@@ -82,6 +82,47 @@ static osc_status make_tmap(CUtensorMap* tm, const void* base, bool bf16, uint64
     return OSC_OK;
 }
 
+// bf16 [rows, cols] input of the quantizer: 128 x 128 tiles, no swizzle, zero fill.
+static osc_status make_tmap_x(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint64_t ld) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return fail(OSC_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+    if (rows == 0) rows = 1;
+    cuuint64_t gdim[2] = {cols, rows};
+    cuuint64_t gstr[1] = {ld * 2};
+    cuuint32_t box[2] = {128, 128};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstr, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(OSC_ERR_CUDA, "cuTensorMapEncodeTiled(X) failed with code %d", (int)r);
+    return OSC_OK;
+}
+
+// Scale-factor buffer as [blocks, 128] uint32 (512-byte blocks), tiles of 2 consecutive blocks.
+static osc_status make_tmap_sf(CUtensorMap* tm, const void* base, uint64_t blocks) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return fail(OSC_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+    if (blocks == 0) blocks = 1;
+    cuuint64_t gdim[2] = {128, blocks};
+    cuuint64_t gstr[1] = {512};
+    cuuint32_t box[2] = {128, 2};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void*>(base), gdim, gstr, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(OSC_ERR_CUDA, "cuTensorMapEncodeTiled(scales) failed with code %d", (int)r);
+    return OSC_OK;
+}
+
+static bool use_pair_kernel(bool grouped, int M) {
+    static int enabled = -1;
+    if (enabled < 0) {
+        const char* e = getenv("OSC_PAIR");
+        enabled = (e && atoi(e) == 0) ? 0 : 1;
+    }
+    return enabled && !grouped && M > 128;
+}
+
 // ----------------------------------------------------------------- the table
 struct Table {
     int Ko = 0, Kop = 0;
@@ -135,8 +176,10 @@ struct osc_weights {
     const uint16_t* wo;
     const uint32_t* mask;
     const int32_t* prefix;
+    const int32_t* idx_o;
     int num_sms, block_n;
-    CUtensorMap tm_b, tm_bo;
+    CUtensorMap tm_b, tm_bo;          // single-CTA kernel: weight tiles of block_n rows
+    CUtensorMap tm_b2, tm_bo2, tm_sfw;  // CTA-pair kernel: half tiles, scale blocks
 };
 struct osc_fp8_weights {
     int E, N, K;
@@ -144,7 +187,7 @@ struct osc_fp8_weights {
     const uint8_t* w8;
     const float* sw;
     int num_sms, block_n;
-    CUtensorMap tm_b;
+    CUtensorMap tm_b, tm_b2;
 };
 
 extern "C" {
@@ -223,11 +266,13 @@ static osc_status prepare_impl(const void* W, int E, int N, int K, int64_t ldw, 
 
     const size_t sfw_e = sf_bytes(N, K);
     for (int ex = 0; ex < E; ++ex) {
-        e = launch_quant_extract(static_cast<const uint16_t*>(W) + (size_t)ex * N * ldw, ldw, N, K, d_mask, d_prefix,
+        CUtensorMap tm_w;
+        if (osc_status s = make_tmap_x(&tm_w, static_cast<const uint16_t*>(W) + (size_t)ex * N * ldw, N, K, ldw)) return s;
+        e = launch_quant_extract(tm_w, N, K, d_mask, d_prefix, reinterpret_cast<const int32_t*>(m8 + (size_t)Kg * 8),
                                  static_cast<uint8_t*>(wq) + (size_t)ex * N * (K / 2),
                                  static_cast<uint8_t*>(sfw) + (size_t)ex * sfw_e,
                                  t.Kop ? static_cast<uint16_t*>(wo) + (size_t)ex * N * t.Kop : nullptr, t.Ko, t.Kop,
-                                 nullptr, 0, st);
+                                 nullptr, 0, di.num_sms, st);
         if (e != cudaSuccess) return cuda_fail(e, "quant_extract_kernel(weights)");
     }
 
@@ -238,11 +283,19 @@ static osc_status prepare_impl(const void* W, int E, int N, int K, int64_t ldw, 
     w->sfw = static_cast<const uint8_t*>(sfw);
     w->wo = static_cast<const uint16_t*>(wo);
     w->mask = d_mask; w->prefix = d_prefix;
+    w->idx_o = reinterpret_cast<const int32_t*>(m8 + (size_t)Kg * 8);
     w->num_sms = di.num_sms;
     w->block_n = gemm_block_n();
     osc_status s = make_tmap(&w->tm_b, wq, false, (uint64_t)E * N, K / 2, K / 2, w->block_n);
     if (s == OSC_OK && t.Kop > 0)
         s = make_tmap(&w->tm_bo, wo, true, (uint64_t)E * N, (uint64_t)t.Kop * 2, (uint64_t)t.Kop * 2, w->block_n);
+    if (s == OSC_OK && !grouped) {
+        const int half = gemm_pair_block_n() / 2;
+        s = make_tmap(&w->tm_b2, wq, false, (uint64_t)N, K / 2, K / 2, half);
+        if (s == OSC_OK && t.Kop > 0)
+            s = make_tmap(&w->tm_bo2, wo, true, (uint64_t)N, (uint64_t)t.Kop * 2, (uint64_t)t.Kop * 2, half);
+        if (s == OSC_OK) s = make_tmap_sf(&w->tm_sfw, sfw, (uint64_t)sfw_e / 512);
+    }
     if (s != OSC_OK) { delete w; return s; }
     *out = w;
     return OSC_OK;
@@ -291,8 +344,10 @@ static osc_status quantize_impl(const osc_weights* w, const void* X, int M, int6
     if (M == 0) return OSC_OK;
     if (!xq || !sfa || (w->Kop > 0 && !xo)) return fail(OSC_ERR_INVALID_ARG, "null output pointer");
     if (!aligned16(xq) || !aligned16(sfa) || !aligned16(xo)) return fail(OSC_ERR_ALIGN, "outputs must be 16-byte aligned");
-    cudaError_t e = launch_quant_extract(X, ldx, M, w->K, w->mask, w->prefix, xq, sfa, w->Kop ? xo : nullptr, w->Ko,
-                                         w->Kop, sched, max_tiles, st);
+    CUtensorMap tm_x;
+    if (osc_status s = make_tmap_x(&tm_x, X, M, w->K, ldx)) return s;
+    cudaError_t e = launch_quant_extract(tm_x, M, w->K, w->mask, w->prefix, w->idx_o, xq, sfa, w->Kop ? xo : nullptr, w->Ko,
+                                         w->Kop, sched, max_tiles, w->num_sms, st);
     if (e != cudaSuccess) return cuda_fail(e, "quant_extract_kernel");
     return OSC_OK;
 }
@@ -325,7 +380,17 @@ static osc_status gemm_impl(const osc_weights* w, const void* xq, const void* sf
     a.ldy = ldy;
     a.M = M; a.N = w->N; a.K = w->K; a.Kop = w->Kop;
     a.sched = sched; a.max_tiles = max_tiles; a.num_sms = w->num_sms;
-    cudaError_t e = launch_gemm_dual(a, st);
+    cudaError_t e;
+    if (use_pair_kernel(w->grouped, M)) {
+        a.tm_b = w->tm_b2;
+        a.tm_bo = w->tm_bo2;
+        a.tm_sfw = w->tm_sfw;
+        if (osc_status s = make_tmap_sf(&a.tm_sfa, sfa, (uint64_t)((M + 127) / 128) * (w->K / 128))) return s;
+        if (osc_status s = make_tmap(&a.tm_y, Y, true, M, (uint64_t)w->N * 2, (uint64_t)ldy * 2, 32)) return s;
+        e = launch_gemm_dual_pair(a, st);
+    } else {
+        e = launch_gemm_dual(a, st);
+    }
     if (e != cudaSuccess) return cuda_fail(e, "gemm_kernel(dual)");
     return OSC_OK;
 }
@@ -405,6 +470,9 @@ static osc_status fp8_prepare_impl(const void* W, int E, int N, int K, int64_t l
     w->num_sms = di.num_sms;
     w->block_n = gemm_block_n();
     if (osc_status s = make_tmap(&w->tm_b, w8, false, (uint64_t)E * N, K, K, w->block_n)) { delete w; return s; }
+    if (!grouped) {
+        if (osc_status s = make_tmap(&w->tm_b2, w8, false, (uint64_t)N, K, K, gemm_pair_block_n() / 2)) { delete w; return s; }
+    }
     *out = w;
     return OSC_OK;
 }
@@ -466,7 +534,14 @@ static osc_status fp8_gemm_impl(const osc_fp8_weights* w, const void* x8, const 
     a.ldy = ldy;
     a.M = M; a.N = w->N; a.K = w->K; a.Kop = 0;
     a.sched = sched; a.max_tiles = max_tiles; a.num_sms = w->num_sms;
-    cudaError_t e = launch_gemm_fp8(a, st);
+    cudaError_t e;
+    if (use_pair_kernel(w->grouped, M)) {
+        a.tm_b = w->tm_b2;
+        if (osc_status s = make_tmap(&a.tm_y, Y, true, M, (uint64_t)w->N * 2, (uint64_t)ldy * 2, 32)) return s;
+        e = launch_gemm_fp8_pair(a, st);
+    } else {
+        e = launch_gemm_fp8(a, st);
+    }
     if (e != cudaSuccess) return cuda_fail(e, "gemm_kernel(fp8)");
     return OSC_OK;
 }

@@ -9,9 +9,9 @@
 namespace osc {
 
 // quant_kernels.cu
-cudaError_t launch_quant_extract(const void* X, int64_t ldx, int M, int K, const uint32_t* mask,
-                                 const int32_t* prefix, void* xq, void* sf, void* xo, int Ko, int Kop,
-                                 const int32_t* sched, int max_tiles, cudaStream_t st);
+cudaError_t launch_quant_extract(const CUtensorMap& tm_x, int M, int K, const uint32_t* mask,
+                                 const int32_t* prefix, const int32_t* idx_o, void* xq, void* sf, void* xo, int Ko, int Kop,
+                                 const int32_t* sched, int max_tiles, int num_sms, cudaStream_t st);
 cudaError_t launch_fp8_quant(const void* X, int64_t ldx, int M, int K, void* x8, void* sx, cudaStream_t st);
 cudaError_t launch_build_sched(const int32_t* off, int E, int32_t* sched, int max_tiles, cudaStream_t st);
 
@@ -21,6 +21,9 @@ struct GemmArgs {
     CUtensorMap tm_b;    // Path A weights    : [E*N, K/2]                    (FP8 mode: [E*N, K])
     CUtensorMap tm_ao;   // Path B activations: bf16 [rows, K_o_pad]
     CUtensorMap tm_bo;   // Path B weights    : bf16 [E*N, K_o_pad]
+    CUtensorMap tm_sfa;  // activation scale blocks as uint32 [blocks, 128] (CTA-pair kernel only)
+    CUtensorMap tm_sfw;  // weight scale blocks, same form
+    CUtensorMap tm_y;    // output bf16 [rows, ldy], 32 x 64 store tiles (CTA-pair kernel only)
     const uint8_t* sfa;  // activation scales, block layout
     const uint8_t* sfw;  // weight scales, block layout, per expert
     const float* sx;     // FP8 mode: per-row activation scale
@@ -33,9 +36,15 @@ struct GemmArgs {
     int max_tiles;
     int num_sms;
     int dbg;             // timing experiments only (0 in normal use)
+    long long* trace;    // timing experiments only (builds with OSC_TRACE)
 };
 cudaError_t launch_gemm_dual(const GemmArgs& a, cudaStream_t st);
 cudaError_t launch_gemm_fp8(const GemmArgs& a, cudaStream_t st);
 int gemm_block_n();
+
+// gemm2_kernels.cu (CTA pairs, dense problems)
+cudaError_t launch_gemm_dual_pair(const GemmArgs& a, cudaStream_t st);
+cudaError_t launch_gemm_fp8_pair(const GemmArgs& a, cudaStream_t st);
+int gemm_pair_block_n();
 
 }  // namespace osc

@@ -1,0 +1,440 @@
+// CTA-pair variant of the tensor-core kernels for dense (non-grouped) problems with many rows.
+//
+// Two CTAs of a cluster (two SMs) compute one 256 x BN output tile with `cta_group::2` MMAs:
+// each CTA holds 128 rows of the activation tile and its 128 x BN slice of the fp32 accumulator in
+// its own TMEM, and loads only HALF of the weight tile (BN/2 rows); the tensor cores of the pair
+// exchange the halves.  Per stage a CTA therefore pulls 16 KB + BN/2 x 128 B from L2 instead of
+// 16 KB + BN x 128 B, which is what bounds the single-CTA kernel (L2 -> shared-memory feed).
+// No cluster-multicast loads are used: every CTA fetches its own operands.
+//
+// Roles per CTA: warp 0 TMA producer, warp 1 MMA issuer (only in the leader CTA, rank 0) and
+// TMEM owner, warps 2-5 epilogue.  Barriers:
+//   full[s]   leader's only: one arrive.expect_tx by the leader's producer for the bytes of BOTH
+//             CTAs; the peer's loads credit the leader's barrier (cta_group::2 loads).
+//   empty[s]  one per CTA, released for both CTAs by one multicast tcgen05.commit of the leader.
+//   tfull[a]  one per CTA (multicast commit); tempty[a] leader's only, 8 arrivals (4 epilogue warps
+//             of each CTA, the peer's arrive through the cluster window).
+// Stage layout and K-loop order are those of the single-CTA kernel (Path A FP4 blocks, then Path B
+// BF16 blocks, 128 bytes per operand row and stage).
+#include <cuda_bf16.h>
+#include <stdio.h>
+
+#include "common.cuh"
+
+namespace osc {
+
+namespace pair {
+
+#ifdef OSC_TRACE
+constexpr int TRACE_CAP = 96;
+__device__ __forceinline__ long long gtime() { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
+#define TRACE(role, idx, slot) do { if (args.trace && blockIdx.x < 4 && (idx) < TRACE_CAP) args.trace[(((blockIdx.x * 4 + (role)) * TRACE_CAP + (idx)) * 2) + (slot)] = gtime(); } while (0)
+#else
+#define TRACE(role, idx, slot) do {} while (0)
+#endif
+
+constexpr int MODE_OSC = 0;
+constexpr int MODE_FP8 = 1;
+constexpr int BM = 128;        // rows per CTA; the pair covers 256
+constexpr int ROW_BYTES = 128;
+constexpr int A_BYTES = BM * ROW_BYTES;
+constexpr int THREADS = 192;
+constexpr int TMEM_COLS = 512;
+constexpr int BAND = 4;        // 256-row tiles per scheduling band
+constexpr int EPI_TILE_BYTES = 32 * 128;            // 32 rows x 64 bf16 columns
+constexpr int EPI_BYTES = 4 * 2 * EPI_TILE_BYTES;   // 4 epilogue warps x 2 staging tiles
+
+template <int MODE, int BN>
+struct Cfg {
+    static constexpr int ACC_STAGES = (2 * BN + 2 * (8 + 2 * 4 * ((BN % 128 == 0) ? BN / 128 : BN / 128 + 2 - (BN % 128 == 64 ? 1 : 0))) <= TMEM_COLS) ? 2 : 1;
+    // 128-row scale blocks a BN-wide tile can touch, given that tiles start at multiples of BN
+    static constexpr int SFB_ATOMS = (BN % 128 == 0) ? BN / 128 : BN / 128 + 2 - (BN % 128 == 64 ? 1 : 0);
+    static constexpr int B_BYTES = (BN / 2) * ROW_BYTES;
+    static constexpr int SFA_BYTES = (MODE == MODE_OSC) ? 1024 : 0;
+    static constexpr int SFB_BYTES = (MODE == MODE_OSC) ? SFB_ATOMS * 1024 : 0;
+    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + SFA_BYTES + SFB_BYTES;
+#ifdef OSC_FORCE_STAGES
+    static constexpr int STAGES = OSC_FORCE_STAGES;
+#else
+    static constexpr int STAGES = (224 * 1024 - EPI_BYTES) / STAGE_BYTES;
+#endif
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/ + EPI_BYTES;
+    static constexpr int TM_SFA = ACC_STAGES * BN;
+    static constexpr int TM_SFB = TM_SFA + 8;
+    static constexpr int TM_SF_STRIDE = 8 + 2 * SFB_ATOMS * 4;  // columns of one scale buffer; two buffers alternate
+    static constexpr uint32_t TX_A = 2u * (A_BYTES + B_BYTES + SFA_BYTES + SFB_BYTES);  // both CTAs, Path A
+    static constexpr uint32_t TX_B = 2u * (A_BYTES + B_BYTES);                          // both CTAs, Path B / FP8
+    static_assert(STAGE_BYTES % 1024 == 0, "stage must keep 1024-byte alignment");
+    static_assert(B_BYTES % 1024 == 0, "weight half-tile must keep 1024-byte alignment");
+    static_assert(TM_SFA + 2 * TM_SF_STRIDE <= TMEM_COLS, "TMEM budget");
+    static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
+    // Tiles must start on an even 32-row scale column: a 224-wide tile (odd column offsets into the
+    // weight-scale region of TMEM) raised "misaligned address" on the block-scaled MMA.
+    static_assert(BN % 64 == 0 && BN <= 256, "tile width");
+};
+
+template <int MODE, int BN>
+__global__ void __launch_bounds__(THREADS, 1) gemm_pair_kernel(const __grid_constant__ GemmArgs args) {
+    using C = Cfg<MODE, BN>;
+    constexpr int STAGES = C::STAGES;
+    constexpr int ACC = C::ACC_STAGES;
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    // [operand ring][epilogue staging tiles, 1024-byte aligned for the swizzle][barriers]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * C::STAGE_BYTES + EPI_BYTES);
+    uint64_t* full_bar = bars;
+    uint64_t* empty_bar = bars + STAGES;
+    uint64_t* tfull_bar = bars + 2 * STAGES;
+    uint64_t* tempty_bar = bars + 2 * STAGES + ACC;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 2 * ACC);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    // warp-uniform values are passed through a shuffle so that the compiler keeps them (and all
+    // address arithmetic derived from them) in uniform registers: the TMA / tcgen05 instructions
+    // below are issued by one elected lane of a converged warp, not from a divergent branch
+    const int warp = __shfl_sync(0xFFFFFFFFu, (int)(threadIdx.x >> 5), 0);
+    const int lane = threadIdx.x & 31;
+    const uint32_t rank = __shfl_sync(0xFFFFFFFFu, cluster_ctarank(), 0);  // 0 = leader
+    const int pair_id = blockIdx.x >> 1;
+    const int num_pairs = gridDim.x >> 1;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < STAGES; ++i) {
+            mbar_init(&full_bar[i], 1);
+            mbar_init(&empty_bar[i], 1);
+        }
+        for (int i = 0; i < ACC; ++i) {
+            mbar_init(&tfull_bar[i], 1);
+            mbar_init(&tempty_bar[i], 8);
+        }
+        *abort_flag = 0;
+        fence_barrier_init();
+        prefetch_tmap(&args.tm_a);
+        prefetch_tmap(&args.tm_b);
+        prefetch_tmap(&args.tm_y);
+        if (MODE == MODE_OSC) {
+            prefetch_tmap(&args.tm_sfa);
+            prefetch_tmap(&args.tm_sfw);
+            if (args.Kop > 0) {
+                prefetch_tmap(&args.tm_ao);
+                prefetch_tmap(&args.tm_bo);
+            }
+        }
+    }
+    if (warp == 1) {
+        tmem_alloc_pair(tmem_slot, TMEM_COLS);
+        tmem_relinquish_pair();
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();
+    tc_fence_after();
+    const uint32_t tmem_base = __shfl_sync(0xFFFFFFFFu, *tmem_slot, 0);
+
+    const int N = args.N, K = args.K;
+    const int num_m = (args.M + 2 * BM - 1) / (2 * BM);
+    const int num_n = (N + BN - 1) / BN;
+    const int total = num_m * num_n;
+    const int elems_per_kb = (MODE == MODE_OSC) ? 256 : 128;
+    const int nkb_a = (K + elems_per_kb - 1) / elems_per_kb;
+    const int nkb_b = (MODE == MODE_OSC) ? args.Kop / 64 : 0;
+    const int nkb = nkb_a + nkb_b;
+    const int katoms_total = K / 128;
+    const int natoms = (N + 127) / 128;
+
+    auto tile_rc = [&](int t, int& row0, int& n0) {
+        const int per_band = BAND * num_n;
+        const int band = t / per_band;
+        const int rem = t - band * per_band;
+        const int m0 = band * BAND;
+        const int h = min(BAND, num_m - m0);
+        row0 = (m0 + rem % h) * (2 * BM);
+        n0 = (rem / h) * BN;
+    };
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer (both CTAs)
+        {
+            int s = 0;
+            uint32_t ph = 0;
+            const uint32_t full0 = map_to_cta(smem_u32(&full_bar[0]), 0);  // the leader's full barriers
+            int ev = 0;
+            for (int t = pair_id; t < total; t += num_pairs) {
+                int row0, n0;
+                tile_rc(t, row0, n0);
+                const int arow = row0 + (int)rank * BM;            // my 128 activation rows
+                const int brow = n0 + (int)rank * (BN / 2);        // my half of the weight rows
+                for (int kb = 0; kb < nkb; ++kb) {
+                    if (!wait_bounded_cluster(&empty_bar[s], ph ^ 1u, abort_flag, 11)) goto done;
+                    if (lane == 0) TRACE(0, ev, 0);
+                    const uint32_t st = smem_u32(smem + s * C::STAGE_BYTES);
+                    const uint32_t fb = full0 + (uint32_t)s * 8u;
+                    if (elect_one()) {
+                    if (kb < nkb_a) {
+                        if (rank == 0) mbar_arrive_expect_tx(&full_bar[s], MODE == MODE_OSC ? C::TX_A : C::TX_B);
+                        tma_load_2d_pair(st, &args.tm_a, fb, kb * ROW_BYTES, arow);
+                        tma_load_2d_pair(st + A_BYTES, &args.tm_b, fb, kb * ROW_BYTES, brow);
+                        if (MODE == MODE_OSC) {
+                            // scale blocks: 2 consecutive 512-byte blocks (256 channels) per 128 rows
+                            tma_load_2d_pair(st + A_BYTES + C::B_BYTES, &args.tm_sfa, fb, 0,
+                                             (arow / 128) * katoms_total + 2 * kb);
+#pragma unroll
+                            for (int j = 0; j < C::SFB_ATOMS; ++j) {
+                                const int atom = min(n0 / 128 + j, natoms - 1);
+                                tma_load_2d_pair(st + A_BYTES + C::B_BYTES + C::SFA_BYTES + j * 1024, &args.tm_sfw, fb, 0,
+                                                 atom * katoms_total + 2 * kb);
+                            }
+                        }
+                    } else {
+                        const int kk = kb - nkb_a;
+                        if (rank == 0) mbar_arrive_expect_tx(&full_bar[s], C::TX_B);
+                        tma_load_2d_pair(st, &args.tm_ao, fb, kk * 64, arow);
+                        tma_load_2d_pair(st + A_BYTES, &args.tm_bo, fb, kk * 64, brow);
+                    }
+                    TRACE(0, ev, 1);
+                    }
+                    __syncwarp();
+                    ++ev;
+                    if (++s == STAGES) { s = 0; ph ^= 1u; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------ MMA issuer (leader CTA only, one thread)
+        if (rank == 0) {
+            int s = 0;
+            uint32_t ph = 0;
+            int acc = 0;
+            uint32_t acc_ph = 0;
+            constexpr uint32_t IDESC_A = (MODE == MODE_OSC) ? idesc_mxf4(2 * BM, BN) : idesc_e4m3(2 * BM, BN);
+            constexpr uint32_t IDESC_B = idesc_bf16(2 * BM, BN);
+            const uint64_t desc_hi = smem_desc_sw128(0);  // everything but the start address
+            const uint64_t sf_hi = smem_desc_sf(0);
+            const uint32_t smem0 = smem_u32(smem);
+            int ev = 0;
+            for (int t = pair_id; t < total; t += num_pairs) {
+                int row0, n0;
+                tile_rc(t, row0, n0);
+                if (!wait_bounded_cluster(&tempty_bar[acc], acc_ph ^ 1u, abort_flag, 12)) goto done;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+                const uint32_t sfb_tm = tmem_base + C::TM_SFB + (uint32_t)((n0 % 128) / 32);
+                for (int kb = 0; kb < nkb; ++kb) {
+                    if (!wait_bounded_cluster(&full_bar[s], ph, abort_flag, 13)) goto done;
+                    if (lane == 0) TRACE(1, ev, 0);
+                    tc_fence_after();
+                    const uint32_t sbase = smem0 + s * C::STAGE_BYTES;
+                    const uint64_t adesc = desc_hi | (uint64_t)(sbase >> 4);
+                    const uint64_t bdesc = desc_hi | (uint64_t)((sbase + A_BYTES) >> 4);
+                    if (elect_one()) {
+                    if (MODE == MODE_OSC && kb < nkb_a) {
+                        const int ka = min(2, katoms_total - 2 * kb);
+                        const uint64_t sfa_d = sf_hi | (uint64_t)((sbase + A_BYTES + C::B_BYTES) >> 4);
+                        const uint64_t sfb_d = sf_hi | (uint64_t)((sbase + A_BYTES + C::B_BYTES + C::SFA_BYTES) >> 4);
+                        // two scale buffers in TMEM alternate, so this stage's copies do not wait for the
+                        // previous stage's MMAs to finish reading theirs
+                        const uint32_t sfo = (uint32_t)(kb & 1) * C::TM_SF_STRIDE;
+#pragma unroll
+                        for (int a = 0; a < 2; ++a) {
+                            if (a < ka && !(args.dbg & 1)) {
+                                tc_copy_sf_pair(tmem_base + sfo + C::TM_SFA + a * 4, sfa_d + (uint64_t)(a * 32));
+#pragma unroll
+                                for (int j = 0; j < C::SFB_ATOMS; ++j)
+                                    tc_copy_sf_pair(tmem_base + sfo + C::TM_SFB + a * (C::SFB_ATOMS * 4) + j * 4,
+                                                    sfb_d + (uint64_t)(j * 64 + a * 32));
+                            }
+                        }
+                        TRACE(1, ev, 1);
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            if (k < 2 * ka && !(args.dbg & 16)) {
+                                constexpr uint32_t SFID[2] = {idesc_sf_ids(0, 0), idesc_sf_ids(2, 2)};
+                                mma_mxf4_pair(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC_A | SFID[k & 1],
+                                              tmem_base + sfo + C::TM_SFA + (k >> 1) * 4,
+                                              sfb_tm + sfo + (k >> 1) * (C::SFB_ATOMS * 4), (kb | k) ? 1u : 0u);
+                            }
+                        }
+                    } else if (MODE == MODE_OSC) {
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) mma_f16_pair(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC_B, 1u);
+                    } else {
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)
+                            mma_f8_pair(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC_A, (kb | k) ? 1u : 0u);
+                    }
+                    TRACE(2, ev, 0);
+                    tc_commit_pair(&empty_bar[s], 3);  // frees the stage in both CTAs
+                    TRACE(2, ev, 1);
+                    }
+                    __syncwarp();
+                    ++ev;
+                    if (++s == STAGES) { s = 0; ph ^= 1u; }
+                }
+                if (elect_one()) tc_commit_pair(&tfull_bar[acc], 3);    // accumulator ready in both CTAs
+                __syncwarp();
+                if (++acc == ACC) { acc = 0; acc_ph ^= 1u; }
+            }
+        }
+    } else {
+        // ---------------------------------------------------------------- epilogue (both CTAs)
+        // Each warp owns 32 accumulator rows.  Per 64-column slice: TMEM -> registers -> bf16 ->
+        // a swizzled 32 x 128-byte staging tile in shared memory -> one TMA store.  Two staging
+        // tiles per warp alternate, so packing the next slice overlaps the store of the last one.
+        // Plain per-thread stores (32 rows x 16 bytes per instruction) kept the memory pipe busy for
+        // the whole epilogue and stalled the MMA issue of the next tile.
+        const int q = warp & 3;
+        int acc = 0;
+        uint32_t acc_ph = 0;
+        const uint32_t tempty0 = map_to_cta(smem_u32(&tempty_bar[0]), 0);
+        uint8_t* stage_buf = smem + STAGES * C::STAGE_BYTES + q * (2 * EPI_TILE_BYTES);
+        int nstore = 0;
+        int ev = 0;
+        for (int t = pair_id; t < total; t += num_pairs) {
+            int row0, n0;
+            tile_rc(t, row0, n0);
+            if (!wait_bounded_cluster(&tfull_bar[acc], acc_ph, abort_flag, 14)) goto done;
+            if (warp == 2 && lane == 0) TRACE(3, ev, 0);
+            tc_fence_after();
+            const int wrow0 = row0 + (int)rank * BM + q * 32;  // first row of this warp
+            const int row = wrow0 + lane;
+            float sxr = 1.0f;
+            if (MODE == MODE_FP8 && row < args.M) sxr = args.sx[row];
+#pragma unroll 1
+            for (int c = 0; c < BN / 64; ++c) {
+                uint32_t r0[32], r1[32];
+                const uint32_t tcol = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + c * 64);
+                tmem_ld_32x32(tcol, r0);
+                tmem_ld_32x32(tcol + 32, r1);
+                tmem_ld_wait();
+                const int col = n0 + c * 64;
+                uint8_t* buf = stage_buf + (nstore & 1) * EPI_TILE_BYTES;
+                // the store that last read this staging tile (two stores ago) must be done reading
+                if (lane == 0) tma_store_wait_read<1>();
+                __syncwarp();
+                if (col < N && !(args.dbg & 8)) {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {  // 8 chunks of 16 bytes = 8 columns each
+                        uint32_t o[4];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const int cc = j * 8 + 2 * i;  // column inside the 64-column slice
+                            float lo = __uint_as_float(cc < 32 ? r0[cc] : r1[cc - 32]);
+                            float hi = __uint_as_float(cc < 32 ? r0[cc + 1] : r1[cc - 31]);
+                            if (MODE == MODE_FP8) {
+                                const float2 w2 = *reinterpret_cast<const float2*>(args.sw + col + cc);
+                                lo = lo * (sxr * w2.x);
+                                hi = hi * (sxr * w2.y);
+                            }
+                            const __nv_bfloat162 b2 = __floats2bfloat162_rn(lo, hi);
+                            o[i] = *reinterpret_cast<const uint32_t*>(&b2);
+                        }
+                        // 128-byte swizzle: 16-byte chunk j of row `lane` lives at chunk j ^ (lane % 8)
+                        *reinterpret_cast<uint4*>(buf + lane * 128 + ((j ^ (lane & 7)) << 4)) =
+                            make_uint4(o[0], o[1], o[2], o[3]);
+                    }
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        tma_store_2d(&args.tm_y, buf, col, wrow0);
+                        tma_store_commit();
+                    }
+                    ++nstore;
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(tempty0 + (uint32_t)acc * 8u);
+            if (warp == 2 && lane == 0) TRACE(3, ev, 1);
+            ++ev;
+            if (++acc == ACC) { acc = 0; acc_ph ^= 1u; }
+        }
+        if (lane == 0) tma_store_wait_all<0>();
+        __syncwarp();
+    }
+
+done:
+    __syncwarp();
+    tc_fence_before();
+    __syncthreads();
+    // neither CTA may leave (or free TMEM) while the other can still touch its shared memory or barriers
+    cluster_sync_all();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc_pair(tmem_base, TMEM_COLS);
+    }
+}
+
+template <int MODE, int BN>
+static cudaError_t launch_cfg(const GemmArgs& a, cudaStream_t st) {
+    using C = Cfg<MODE, BN>;
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(gemm_pair_kernel<MODE, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             C::SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    const int total = ((a.M + 2 * BM - 1) / (2 * BM)) * ((a.N + BN - 1) / BN);
+    if (total <= 0) return cudaSuccess;
+    cudaLaunchConfig_t cfg = {};
+    cfg.blockDim = dim3(THREADS);
+    cfg.dynamicSmemBytes = C::SMEM_BYTES;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    // The kernel is persistent with static striping of tiles over pairs, so every pair must be
+    // resident at once: ask how many 2-CTA clusters of this footprint the device can hold.
+    static int max_pairs = 0;
+    if (max_pairs == 0) {
+        cfg.gridDim = dim3(a.num_sms);
+        int n = 0;
+        cudaError_t e = cudaOccupancyMaxActiveClusters(&n, gemm_pair_kernel<MODE, BN>, &cfg);
+        if (e != cudaSuccess) return e;
+        max_pairs = n > 0 ? n : 1;
+        if (getenv("OSC_LOG")) fprintf(stderr, "[osc] pair kernel BN=%d: %d resident clusters of 2\n", BN, max_pairs);
+    }
+    int pairs = a.num_sms / 2;
+    if (max_pairs < pairs) pairs = max_pairs;
+    if (const char* e = getenv("OSC_PAIRS")) { const int v = atoi(e); if (v > 0 && v < pairs) pairs = v; }
+    if (total < pairs) pairs = total;
+    cfg.gridDim = dim3(2 * pairs);
+    GemmArgs b = a;
+    if (const char* e = getenv("OSC_DEBUG")) b.dbg = atoi(e);
+    if (const char* e = getenv("OSC_TRACE_PTR")) b.trace = reinterpret_cast<long long*>(strtoull(e, nullptr, 0));
+    return cudaLaunchKernelEx(&cfg, gemm_pair_kernel<MODE, BN>, b);
+}
+
+}  // namespace pair
+
+static int g_pair_bn = 0;
+int gemm_pair_block_n() {
+    if (g_pair_bn == 0) {
+        g_pair_bn = 256;
+        if (const char* e = getenv("OSC_PAIR_BLOCK_N")) {
+            const int v = atoi(e);
+            if (v == 192 || v == 256) g_pair_bn = v;
+        }
+    }
+    return g_pair_bn;
+}
+
+cudaError_t launch_gemm_dual_pair(const GemmArgs& a, cudaStream_t st) {
+    switch (gemm_pair_block_n()) {
+        case 192: return pair::launch_cfg<pair::MODE_OSC, 192>(a, st);
+        default: return pair::launch_cfg<pair::MODE_OSC, 256>(a, st);
+    }
+}
+cudaError_t launch_gemm_fp8_pair(const GemmArgs& a, cudaStream_t st) {
+    switch (gemm_pair_block_n()) {
+        case 192: return pair::launch_cfg<pair::MODE_FP8, 192>(a, st);
+        default: return pair::launch_cfg<pair::MODE_FP8, 256>(a, st);
+    }
+}
+
+}  // namespace osc

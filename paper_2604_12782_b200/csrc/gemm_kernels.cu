@@ -154,13 +154,6 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
                         if (MODE == MODE_OSC) {
                             const int ka = min(2, katoms_total - 2 * kb);  // 128-channel scale blocks in this stage
                             const uint32_t sfb = (uint32_t)ka * 512u;
-                            if (args.dbg & 2) {
-                                mbar_arrive_expect_tx(&full_bar[s], A_BYTES + C::B_BYTES);
-                                tma_load_2d(st, &args.tm_a, &full_bar[s], kb * ROW_BYTES, ti.row0);
-                                tma_load_2d(st + A_BYTES, &args.tm_b, &full_bar[s], kb * ROW_BYTES, brow);
-                                if (++s == STAGES) { s = 0; ph ^= 1u; }
-                                continue;
-                            }
                             mbar_arrive_expect_tx(&full_bar[s], A_BYTES + C::B_BYTES + sfb * (1 + C::SFB_ATOMS));
                             tma_load_2d(st, &args.tm_a, &full_bar[s], kb * ROW_BYTES, ti.row0);
                             tma_load_2d(st + A_BYTES, &args.tm_b, &full_bar[s], kb * ROW_BYTES, brow);
@@ -213,18 +206,14 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
                         const int ka = min(2, katoms_total - 2 * kb);
                         const uint32_t sfa_s = sbase + A_BYTES + C::B_BYTES;
                         const uint32_t sfb_s = sfa_s + C::SFA_BYTES;
-                        for (int a = 0; a < ka && !(args.dbg & 1); ++a) {
+                        for (int a = 0; a < ka; ++a) {
                             tc_copy_sf(tmem_base + C::TM_SFA + a * 4, smem_desc_sf(sfa_s + a * 512));
 #pragma unroll
                             for (int j = 0; j < C::SFB_ATOMS; ++j)
                                 tc_copy_sf(tmem_base + C::TM_SFB + a * (C::SFB_ATOMS * 4) + j * 4,
                                            smem_desc_sf(sfb_s + j * 1024 + a * 512));
                         }
-                        for (int k = 0; k < 2 * ka && !(args.dbg & 16); ++k) {
-                            if (args.dbg & 4) {
-                                mma_f8(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc_e4m3(BM, BN), (kb | k) ? 1u : 0u);
-                                continue;
-                            }
+                        for (int k = 0; k < 2 * ka; ++k) {
                             const uint32_t sfid = (uint32_t)(k & 1) * 2u;  // byte pair inside the 4-byte scale column
                             mma_mxf4(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC_A | idesc_sf_ids(sfid, sfid),
                                      tmem_base + C::TM_SFA + (k >> 1) * 4,
@@ -268,7 +257,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
                 tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + c * 32), r);
                 tmem_ld_wait();
                 const int col = ti.n0 + c * 32;
-                if (row_ok && col < N && !(args.dbg & 8)) {
+                if (row_ok && col < N) {
                     uint32_t o[16];
 #pragma unroll
                     for (int i = 0; i < 16; ++i) {
@@ -341,9 +330,7 @@ static cudaError_t launch_cfg(const GemmArgs& a, cudaStream_t st) {
         if (total <= 0) return cudaSuccess;
         if (total < grid) grid = total;
     }
-    GemmArgs b = a;
-    if (const char* e = getenv("OSC_DEBUG")) b.dbg = atoi(e);
-    gemm_kernel<MODE, BN><<<grid, GEMM_THREADS, C::SMEM_BYTES, st>>>(b);
+    gemm_kernel<MODE, BN><<<grid, GEMM_THREADS, C::SMEM_BYTES, st>>>(a);
     return cudaGetLastError();
 }
 

@@ -2,4 +2,5 @@
 // are compiled together (no relocatable device code needed).
 #include "quant_kernels.cu"
 #include "gemm_kernels.cu"
+#include "gemm2_kernels.cu"
 #include "api.cu"

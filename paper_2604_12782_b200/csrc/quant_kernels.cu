@@ -5,6 +5,8 @@
 //   fp8_quant_kernel     : Section 3.4 fallback - per-row dynamic E4M3 with an fp32 scale.
 //   build_sched_kernel   : grouped (MoE) tile schedule from the expert offsets.
 // All three are used for activations (online) and for weights (offline preparation).
+#include <cuda_bf16.h>
+
 #include "common.cuh"
 
 namespace osc {
@@ -19,6 +21,8 @@ __device__ __forceinline__ uint32_t e2m1x2(float lo, float hi) {
         : "f"(hi), "f"(lo));
     return r;
 }
+__device__ __forceinline__ __nv_bfloat162 as_bf162(uint32_t u) { return *reinterpret_cast<__nv_bfloat162*>(&u); }
+__device__ __forceinline__ uint32_t bf162_bits(__nv_bfloat162 h) { return *reinterpret_cast<uint32_t*>(&h); }
 __device__ __forceinline__ uint32_t e4m3x2(float lo, float hi) {
     uint16_t r;
     asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
@@ -26,114 +30,174 @@ __device__ __forceinline__ uint32_t e4m3x2(float lo, float hi) {
 }
 
 // ------------------------------------------------------- Algorithm 2, fused
-// CTA tile: 128 rows x 128 channels (4 groups).  256 threads; thread t owns 8 consecutive
-// channels (t % 16) of row (t / 16) + 16 * pass.  Four neighbouring threads share a group.
+// Persistent kernel, one CTA per SM.  A producer warp streams 128-row x 128-channel tiles of X
+// (32 KB) through a shared-memory ring with TMA; eight consumer warps take a tile out of the ring
+// into registers, release the slot at once, and do the lookup / back-up / zero-out / scale /
+// quantize work while the next tiles are already in flight.  Thread t of the consumers owns 8
+// consecutive channels (t % 16) of row (t / 16) + 16 * pass; four neighbouring threads share a group.
 constexpr int QE_ROWS = 128;
 constexpr int QE_COLS = 128;
-constexpr int QE_THREADS = 256;
-constexpr int QE_PASSES = QE_ROWS / (QE_THREADS / 16);  // 8
+constexpr int QE_CONSUMERS = 512;
+constexpr int QE_THREADS = QE_CONSUMERS + 32;
+constexpr int QE_PASSES = QE_ROWS / (QE_CONSUMERS / 16);  // 8
+constexpr int QE_TILE_BYTES = QE_ROWS * QE_COLS * 2;
+constexpr int QE_STAGES = 3;
+constexpr int QE_CTAS_PER_SM = 2;
+constexpr int QE_SMEM = QE_STAGES * QE_TILE_BYTES + 1024 + 2 * 512 + 256;
 
-__global__ void __launch_bounds__(QE_THREADS)
-quant_extract_kernel(const uint16_t* __restrict__ X, int64_t ldx, int M, int K,
+__global__ void __launch_bounds__(QE_THREADS, QE_CTAS_PER_SM)
+quant_extract_kernel(const __grid_constant__ CUtensorMap tm_x, int M, int K,
                      const uint32_t* __restrict__ mask, const int32_t* __restrict__ prefix,
+                     const int32_t* __restrict__ idx_o,
                      uint8_t* __restrict__ xq, uint8_t* __restrict__ sf, uint16_t* __restrict__ xo,
                      int Ko, int Kop, const int32_t* __restrict__ sched, int max_tiles) {
-    __shared__ __align__(16) uint8_t s_sf[512];
+    extern __shared__ uint8_t qe_smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(qe_smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* s_sf = smem + QE_STAGES * QE_TILE_BYTES;                       // 2 x 512 bytes, alternating
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(s_sf + 2 * 512);
+    uint64_t* empty_bar = full_bar + QE_STAGES;
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(empty_bar + QE_STAGES);
 
-    const int cb = blockIdx.x;  // 128-channel block
-    const int tile = blockIdx.y;
-    int row0, row_end, sf_row0;
-    if (sched != nullptr) {
-        if (tile >= sched[0]) return;
-        row0 = sched[1 + tile];
-        row_end = sched[1 + max_tiles + tile];
-        sf_row0 = sched[1 + 2 * max_tiles + tile];
-    } else {
-        row0 = tile * QE_ROWS;
-        row_end = M;
-        sf_row0 = row0;
-    }
-
-    const int tid = threadIdx.x;
-    const int cchunk = tid & 15;  // 8-channel chunk inside the 128-channel block
-    const int gi = cchunk >> 2;   // group inside the block
-    const int sub = cchunk & 3;   // which quarter of the group
-    const int rsub = tid >> 4;    // 0..15
-    const int g = cb * 4 + gi;
-
-    const uint32_t gmask = mask[g];
-    const uint32_t my8 = (gmask >> (sub * 8)) & 0xFFu;
-    const int my_pre = prefix[g] + __popc(gmask & ((1u << (sub * 8)) - 1u));
-
-    uint4 v[QE_PASSES];
-#pragma unroll
-    for (int p = 0; p < QE_PASSES; ++p) {
-        const int r = row0 + rsub + 16 * p;
-        if (r < row_end) {
-            v[p] = *reinterpret_cast<const uint4*>(X + (int64_t)r * ldx + cb * QE_COLS + cchunk * 8);
-        } else {
-            v[p] = make_uint4(0u, 0u, 0u, 0u);
+    const int warp = __shfl_sync(0xFFFFFFFFu, (int)(threadIdx.x >> 5), 0);
+    const int lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < QE_STAGES; ++i) {
+            mbar_init(&full_bar[i], 1);
+            mbar_init(&empty_bar[i], QE_CONSUMERS / 32);
         }
+        *abort_flag = 0;
+        fence_barrier_init();
+        prefetch_tmap(&tm_x);
     }
+    __syncthreads();
 
+    const int ncb = K / QE_COLS;  // 128-channel blocks per row
+    const int nrt = sched ? sched[0] : (M + QE_ROWS - 1) / QE_ROWS;
+    const int total = nrt * ncb;
+
+    if (warp == QE_CONSUMERS / 32) {
+        // ------------------------------------------------------------------ producer
+        int s = 0;
+        uint32_t ph = 0;
+        for (int t = blockIdx.x; t < total; t += gridDim.x) {
+            const int rt = t / ncb, cb = t - rt * ncb;
+            const int row0 = sched ? sched[1 + rt] : rt * QE_ROWS;
+            if (!wait_bounded(&empty_bar[s], ph ^ 1u, abort_flag, 21)) break;
+            if (elect_one()) {
+                mbar_arrive_expect_tx(&full_bar[s], QE_TILE_BYTES);
+                tma_load_2d(smem + s * QE_TILE_BYTES, &tm_x, &full_bar[s], cb * QE_COLS, row0);
+            }
+            __syncwarp();
+            if (++s == QE_STAGES) { s = 0; ph ^= 1u; }
+        }
+    } else {
+        // ----------------------------------------------------------------- consumers
+        const int tid = threadIdx.x;
+        const int cchunk = tid & 15;  // 8-channel chunk inside the 128-channel block
+        const int gi = cchunk >> 2;   // group inside the block
+        const int sub = cchunk & 3;   // which quarter of the group
+        const int rsub = tid >> 4;    // 0 .. QE_CONSUMERS/16 - 1
+        int s = 0;
+        uint32_t ph = 0;
+        int parity = 0;
+        for (int t = blockIdx.x; t < total; t += gridDim.x) {
+            const int rt = t / ncb, cb = t - rt * ncb;
+            int row0, row_end, sf_row0;
+            if (sched) {
+                row0 = sched[1 + rt];
+                row_end = sched[1 + max_tiles + rt];
+                sf_row0 = sched[1 + 2 * max_tiles + rt];
+            } else {
+                row0 = rt * QE_ROWS;
+                row_end = M;
+                sf_row0 = row0;
+            }
+            // Per tile and thread: AND-masks that zero my flagged channels (the table is static, so the
+            // zero-out costs one logic op per register and no branch).
+            const uint32_t gmask = mask[cb * 4 + gi];
+            const uint32_t my8 = (gmask >> (sub * 8)) & 0xFFu;
+            uint32_t keep[4];
 #pragma unroll
-    for (int p = 0; p < QE_PASSES; ++p) {
-        const int rl = rsub + 16 * p;  // row inside the tile
-        const int r = row0 + rl;
-        uint32_t w[4] = {v[p].x, v[p].y, v[p].z, v[p].w};
-        // back up + zero the flagged channels (rare: at most a few bits set)
-        if (my8 != 0u) {
+            for (int i = 0; i < 4; ++i)
+                keep[i] = (((my8 >> (2 * i)) & 1u) ? 0u : 0x0000FFFFu) | (((my8 >> (2 * i + 1)) & 1u) ? 0u : 0xFFFF0000u);
+
+            if (!wait_bounded(&full_bar[s], ph, abort_flag, 22)) break;
+            const uint8_t* st = smem + s * QE_TILE_BYTES;
+            uint4 v[QE_PASSES];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                if ((my8 >> j) & 1u) {
-                    const uint32_t word = w[j >> 1];
-                    const uint16_t bits = (j & 1) ? (uint16_t)(word >> 16) : (uint16_t)(word & 0xFFFFu);
-                    if (r < row_end) xo[(int64_t)r * Kop + my_pre + __popc(my8 & ((1u << j) - 1u))] = bits;
-                    w[j >> 1] = (j & 1) ? (word & 0x0000FFFFu) : (word & 0xFFFF0000u);
+            for (int p = 0; p < QE_PASSES; ++p)
+                v[p] = *reinterpret_cast<const uint4*>(st + (rsub + (QE_CONSUMERS / 16) * p) * (QE_COLS * 2) + cchunk * 16);
+
+            // Back-up of the flagged channels of this 128-channel block into xo (the buffer B):
+            // one (row, channel) copy per task straight from the shared-memory tile, consecutive
+            // threads writing consecutive elements of a row.
+            {
+                const int o0 = prefix[cb * 4];
+                const int o1 = (cb * 4 + 4 < K / 32) ? prefix[cb * 4 + 4] : Ko;
+                const int nout = o1 - o0;
+                const int rows_here = min(QE_ROWS, row_end - row0);
+                for (int task = tid; task < rows_here * nout; task += QE_CONSUMERS) {
+                    const int rl = task / nout, k = task - rl * nout;
+                    const int col = idx_o[o0 + k] - cb * QE_COLS;
+                    xo[(int64_t)(row0 + rl) * Kop + o0 + k] =
+                        *reinterpret_cast<const uint16_t*>(st + rl * (QE_COLS * 2) + col * 2);
                 }
             }
-        }
-        // amax over my 8 channels on the bf16 magnitude bits (monotone in the value)
-        uint32_t am = 0;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            am = max(am, w[i] & 0x7FFFu);
-            am = max(am, (w[i] >> 16) & 0x7FFFu);
-        }
-        am = max(am, __shfl_xor_sync(0xFFFFFFFFu, am, 1));
-        am = max(am, __shfl_xor_sync(0xFFFFFFFFu, am, 2));
-        // CalculateScale: E8M0 code = biased exponent of amax - 2, floored at 0 (2^(floor(log2 amax) - 2))
-        const int ex = (int)(am >> 7);
-        int code = max(ex - 2, 0);
-        if (ex == 255) code = 255;
-        // Quantize: x * 2^(127 - code) is exact in fp32, then hardware E2M1 rounding (nearest-even, saturating)
-        const float inv = __uint_as_float((uint32_t)(254 - min(code, 253)) << 23);
-        uint32_t packed = 0;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const float lo = __uint_as_float(w[i] << 16) * inv;
-            const float hi = __uint_as_float(w[i] & 0xFFFF0000u) * inv;
-            packed |= (e2m1x2(lo, hi) & 0xFFu) << (8 * i);
-        }
-        if (r < row_end) {
-            *reinterpret_cast<uint32_t*>(xq + (int64_t)r * (K / 2) + cb * (QE_COLS / 2) + cchunk * 4) = packed;
-        }
-        if (sub == 0) s_sf[(rl & 31) * 16 + (rl >> 5) * 4 + gi] = (uint8_t)code;
-    }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&empty_bar[s]);  // the slot can be refilled while we work
+            if (++s == QE_STAGES) { s = 0; ph ^= 1u; }
 
-    // zero the pad columns of xo once per row tile
-    if (cb == 0 && Kop > Ko) {
-        const int npad = Kop - Ko;
-        for (int i = tid; i < QE_ROWS * npad; i += QE_THREADS) {
-            const int r = row0 + i / npad;
-            if (r < row_end) xo[(int64_t)r * Kop + Ko + i % npad] = 0;
-        }
-    }
+            uint8_t* sfb = s_sf + parity * 512;
+#pragma unroll
+            for (int p = 0; p < QE_PASSES; ++p) {
+                const int rl = rsub + (QE_CONSUMERS / 16) * p;  // row inside the tile
+                const int r = row0 + rl;
+                const bool live = r < row_end;  // rows past the end (next expert / padding) count as zeros
+                const uint32_t lm = live ? 0xFFFFFFFFu : 0u;
+                const uint32_t w[4] = {v[p].x & keep[0] & lm, v[p].y & keep[1] & lm, v[p].z & keep[2] & lm,
+                                       v[p].w & keep[3] & lm};
+                // amax over my 8 channels on the bf16 magnitudes (sign bits cleared: all values >= 0)
+                const __nv_bfloat162 m01 = __hmax2(as_bf162(w[0] & 0x7FFF7FFFu), as_bf162(w[1] & 0x7FFF7FFFu));
+                const __nv_bfloat162 m23 = __hmax2(as_bf162(w[2] & 0x7FFF7FFFu), as_bf162(w[3] & 0x7FFF7FFFu));
+                const uint32_t am2 = bf162_bits(__hmax2(m01, m23));
+                uint32_t am = max(am2 & 0xFFFFu, am2 >> 16);
+                am = max(am, __shfl_xor_sync(0xFFFFFFFFu, am, 1));
+                am = max(am, __shfl_xor_sync(0xFFFFFFFFu, am, 2));
+                // CalculateScale: E8M0 code = biased exponent of amax - 2, floored at 0 (2^(floor(log2 amax) - 2))
+                const int ex = (int)(am >> 7);
+                int code = max(ex - 2, 0);
+                if (ex == 255) code = 255;
+                // Quantize: x * 2^(127 - code) is exact in fp32, then hardware E2M1 rounding (nearest-even, saturating)
+                const float inv = __uint_as_float((uint32_t)(254 - min(code, 253)) << 23);
+                uint32_t packed = 0;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const float lo = __uint_as_float(w[i] << 16) * inv;
+                    const float hi = __uint_as_float(w[i] & 0xFFFF0000u) * inv;
+                    packed |= (e2m1x2(lo, hi) & 0xFFu) << (8 * i);
+                }
+                if (live)
+                    *reinterpret_cast<uint32_t*>(xq + (int64_t)r * (K / 2) + cb * (QE_COLS / 2) + cchunk * 4) = packed;
+                if (sub == 0) sfb[(rl & 31) * 16 + (rl >> 5) * 4 + gi] = (uint8_t)code;
+            }
 
-    __syncthreads();
-    if (tid < 32) {
-        const int64_t blk = (int64_t)(sf_row0 / 128) * (K / 128) + cb;
-        *reinterpret_cast<uint4*>(sf + blk * 512 + tid * 16) = *reinterpret_cast<const uint4*>(s_sf + tid * 16);
+            // zero the pad columns of xo once per row tile
+            if (cb == 0 && Kop > Ko) {
+                const int npad = Kop - Ko;
+                for (int i = tid; i < QE_ROWS * npad; i += QE_CONSUMERS) {
+                    const int r = row0 + i / npad;
+                    if (r < row_end) xo[(int64_t)r * Kop + Ko + i % npad] = 0;
+                }
+            }
+
+            // all 256 consumers have written their scale bytes of this tile
+            asm volatile("bar.sync 1, %0;" ::"n"(QE_CONSUMERS) : "memory");
+            if (tid < 32) {
+                const int64_t blk = (int64_t)(sf_row0 / 128) * (K / 128) + cb;
+                *reinterpret_cast<uint4*>(sf + blk * 512 + tid * 16) = *reinterpret_cast<const uint4*>(sfb + tid * 16);
+            }
+            parity ^= 1;  // the other staging block is free: its readers passed the previous barrier
+        }
     }
 }
 
@@ -239,15 +303,21 @@ __global__ void build_sched_kernel(const int32_t* __restrict__ off, int E, int32
 }
 
 // ------------------------------------------------------------------ launchers
-cudaError_t launch_quant_extract(const void* X, int64_t ldx, int M, int K, const uint32_t* mask,
-                                 const int32_t* prefix, void* xq, void* sf, void* xo, int Ko, int Kop,
-                                 const int32_t* sched, int max_tiles, cudaStream_t st) {
-    const int tiles = sched ? max_tiles : (M + QE_ROWS - 1) / QE_ROWS;
+cudaError_t launch_quant_extract(const CUtensorMap& tm_x, int M, int K, const uint32_t* mask,
+                                 const int32_t* prefix, const int32_t* idx_o, void* xq, void* sf, void* xo, int Ko, int Kop,
+                                 const int32_t* sched, int max_tiles, int num_sms, cudaStream_t st) {
+    const int tiles = (sched ? max_tiles : (M + QE_ROWS - 1) / QE_ROWS) * (K / QE_COLS);
     if (tiles <= 0) return cudaSuccess;
-    dim3 grid(K / QE_COLS, tiles);
-    quant_extract_kernel<<<grid, QE_THREADS, 0, st>>>(static_cast<const uint16_t*>(X), ldx, M, K, mask, prefix,
-                                                      static_cast<uint8_t*>(xq), static_cast<uint8_t*>(sf),
-                                                      static_cast<uint16_t*>(xo), Ko, Kop, sched, max_tiles);
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(quant_extract_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, QE_SMEM);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    const int grid = tiles < QE_CTAS_PER_SM * num_sms ? tiles : QE_CTAS_PER_SM * num_sms;
+    quant_extract_kernel<<<grid, QE_THREADS, QE_SMEM, st>>>(tm_x, M, K, mask, prefix, idx_o, static_cast<uint8_t*>(xq),
+                                                            static_cast<uint8_t*>(sf), static_cast<uint16_t*>(xo),
+                                                            Ko, Kop, sched, max_tiles);
     return cudaGetLastError();
 }
 
