@@ -329,7 +329,7 @@ def run_gpu(args):
     # roofline of the dominant kernel (dual-path GEMM): tensor peak of its own FLOP mix
     p_mix = flops / (flops4 / peaks["fp4"] + flops16 / peaks["bf16"]) / 1e12
     gemm_tflops = flops / (tg * 1e-3) / 1e12
-    roof = {"bound": "tensor", "kernel": "gemm_kernel<MODE_OSC>", "achieved": gemm_tflops, "peak": p_mix,
+    roof = {"bound": "tensor", "kernel": "gemm_pair_kernel<MODE_OSC> (dual-path GEMM, Eq. 5)", "achieved": gemm_tflops, "peak": p_mix,
             "unit": "TFLOP/s", "frac": gemm_tflops / p_mix, "traffic": GEMM_TRAFFIC_BYTES,
             "peak_basis": f"{pk['source']} bf16 {pk['bf16_tflops']} TFLOP/s x4 for FP4 (burst), FLOP-mix weighted",
             "ms": tg}
@@ -346,7 +346,6 @@ def run_gpu(args):
         "speedup_vs_own_fp8_linear": ms_f8 / ms,
         "speedup_vs_own_fp8_gemm_only": f8g / tg,
         "paper_analytic_speedup_vs_w8a8": roofline.analytic_speedup_vs_w8a8(32, WORKLOAD["ch_per_group"]),
-        "block_n": int(os.environ.get("OSC_BLOCK_N", "256")),
     }
 
     cpu = None
@@ -470,7 +469,7 @@ def run_sweep(args):
 
     os.makedirs(os.path.join(ROOT, "gpurun_out"), exist_ok=True)
     with open(os.path.join(ROOT, "gpurun_out", "sweep.json"), "w") as f:
-        json.dump({"peaks": pk, "block_n": os.environ.get("OSC_BLOCK_N", "256"), "rows": rows}, f, indent=1)
+        json.dump({"peaks": pk, "rows": rows}, f, indent=1)
     for r in rows:
         print(json.dumps(r), file=sys.stderr)
 

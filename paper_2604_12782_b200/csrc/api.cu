@@ -179,7 +179,7 @@ struct osc_weights {
     const int32_t* idx_o;
     int num_sms, block_n;
     CUtensorMap tm_b, tm_bo;          // single-CTA kernel: weight tiles of block_n rows
-    CUtensorMap tm_b2, tm_bo2, tm_sfw;  // CTA-pair kernel: half tiles, scale blocks
+    CUtensorMap tm_b2[2], tm_bo2[2], tm_sfw;  // CTA-pair kernel: half tiles for 192- and 256-wide tiles, scale blocks
 };
 struct osc_fp8_weights {
     int E, N, K;
@@ -187,7 +187,7 @@ struct osc_fp8_weights {
     const uint8_t* w8;
     const float* sw;
     int num_sms, block_n;
-    CUtensorMap tm_b, tm_b2;
+    CUtensorMap tm_b, tm_b2[2];
 };
 
 extern "C" {
@@ -289,13 +289,13 @@ static osc_status prepare_impl(const void* W, int E, int N, int K, int64_t ldw, 
     osc_status s = make_tmap(&w->tm_b, wq, false, (uint64_t)E * N, K / 2, K / 2, w->block_n);
     if (s == OSC_OK && t.Kop > 0)
         s = make_tmap(&w->tm_bo, wo, true, (uint64_t)E * N, (uint64_t)t.Kop * 2, (uint64_t)t.Kop * 2, w->block_n);
-    if (s == OSC_OK && !grouped) {
-        const int half = gemm_pair_block_n() / 2;
-        s = make_tmap(&w->tm_b2, wq, false, (uint64_t)N, K / 2, K / 2, half);
+    for (int v = 0; v < 2 && s == OSC_OK && !grouped; ++v) {
+        const int half = (v == 0 ? 192 : 256) / 2;
+        s = make_tmap(&w->tm_b2[v], wq, false, (uint64_t)N, K / 2, K / 2, half);
         if (s == OSC_OK && t.Kop > 0)
-            s = make_tmap(&w->tm_bo2, wo, true, (uint64_t)N, (uint64_t)t.Kop * 2, (uint64_t)t.Kop * 2, half);
-        if (s == OSC_OK) s = make_tmap_sf(&w->tm_sfw, sfw, (uint64_t)sfw_e / 512);
+            s = make_tmap(&w->tm_bo2[v], wo, true, (uint64_t)N, (uint64_t)t.Kop * 2, (uint64_t)t.Kop * 2, half);
     }
+    if (s == OSC_OK && !grouped) s = make_tmap_sf(&w->tm_sfw, sfw, (uint64_t)sfw_e / 512);
     if (s != OSC_OK) { delete w; return s; }
     *out = w;
     return OSC_OK;
@@ -382,12 +382,13 @@ static osc_status gemm_impl(const osc_weights* w, const void* xq, const void* sf
     a.sched = sched; a.max_tiles = max_tiles; a.num_sms = w->num_sms;
     cudaError_t e;
     if (use_pair_kernel(w->grouped, M)) {
-        a.tm_b = w->tm_b2;
-        a.tm_bo = w->tm_bo2;
+        const int bn = gemm_pair_block_n(M, w->N, w->num_sms);
+        a.tm_b = w->tm_b2[bn == 256];
+        a.tm_bo = w->tm_bo2[bn == 256];
         a.tm_sfw = w->tm_sfw;
         if (osc_status s = make_tmap_sf(&a.tm_sfa, sfa, (uint64_t)((M + 127) / 128) * (w->K / 128))) return s;
         if (osc_status s = make_tmap(&a.tm_y, Y, true, M, (uint64_t)w->N * 2, (uint64_t)ldy * 2, 32)) return s;
-        e = launch_gemm_dual_pair(a, st);
+        e = launch_gemm_dual_pair(a, bn, st);
     } else {
         e = launch_gemm_dual(a, st);
     }
@@ -470,8 +471,8 @@ static osc_status fp8_prepare_impl(const void* W, int E, int N, int K, int64_t l
     w->num_sms = di.num_sms;
     w->block_n = gemm_block_n();
     if (osc_status s = make_tmap(&w->tm_b, w8, false, (uint64_t)E * N, K, K, w->block_n)) { delete w; return s; }
-    if (!grouped) {
-        if (osc_status s = make_tmap(&w->tm_b2, w8, false, (uint64_t)N, K, K, gemm_pair_block_n() / 2)) { delete w; return s; }
+    for (int v = 0; v < 2 && !grouped; ++v) {
+        if (osc_status s = make_tmap(&w->tm_b2[v], w8, false, (uint64_t)N, K, K, (v == 0 ? 192 : 256) / 2)) { delete w; return s; }
     }
     *out = w;
     return OSC_OK;
@@ -536,9 +537,10 @@ static osc_status fp8_gemm_impl(const osc_fp8_weights* w, const void* x8, const 
     a.sched = sched; a.max_tiles = max_tiles; a.num_sms = w->num_sms;
     cudaError_t e;
     if (use_pair_kernel(w->grouped, M)) {
-        a.tm_b = w->tm_b2;
+        const int bn = gemm_pair_block_n(M, w->N, w->num_sms);
+        a.tm_b = w->tm_b2[bn == 256];
         if (osc_status s = make_tmap(&a.tm_y, Y, true, M, (uint64_t)w->N * 2, (uint64_t)ldy * 2, 32)) return s;
-        e = launch_gemm_fp8_pair(a, st);
+        e = launch_gemm_fp8_pair(a, bn, st);
     } else {
         e = launch_gemm_fp8(a, st);
     }

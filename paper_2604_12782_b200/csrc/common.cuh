@@ -35,16 +35,14 @@ struct GemmArgs {
     const int32_t* sched;  // grouped tile schedule or nullptr
     int max_tiles;
     int num_sms;
-    int dbg;             // timing experiments only (0 in normal use)
-    long long* trace;    // timing experiments only (builds with OSC_TRACE)
 };
 cudaError_t launch_gemm_dual(const GemmArgs& a, cudaStream_t st);
 cudaError_t launch_gemm_fp8(const GemmArgs& a, cudaStream_t st);
 int gemm_block_n();
 
 // gemm2_kernels.cu (CTA pairs, dense problems)
-cudaError_t launch_gemm_dual_pair(const GemmArgs& a, cudaStream_t st);
-cudaError_t launch_gemm_fp8_pair(const GemmArgs& a, cudaStream_t st);
-int gemm_pair_block_n();
+cudaError_t launch_gemm_dual_pair(const GemmArgs& a, int bn, cudaStream_t st);
+cudaError_t launch_gemm_fp8_pair(const GemmArgs& a, int bn, cudaStream_t st);
+int gemm_pair_block_n(int M, int N, int num_sms);
 
 }  // namespace osc

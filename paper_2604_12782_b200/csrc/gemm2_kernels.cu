@@ -8,12 +8,12 @@
 // No cluster-multicast loads are used: every CTA fetches its own operands.
 //
 // Roles per CTA: warp 0 TMA producer, warp 1 MMA issuer (only in the leader CTA, rank 0) and
-// TMEM owner, warps 2-5 epilogue.  Barriers:
+// TMEM owner, warps 2-9 epilogue.  Barriers:
 //   full[s]   leader's only: one arrive.expect_tx by the leader's producer for the bytes of BOTH
 //             CTAs; the peer's loads credit the leader's barrier (cta_group::2 loads).
 //   empty[s]  one per CTA, released for both CTAs by one multicast tcgen05.commit of the leader.
-//   tfull[a]  one per CTA (multicast commit); tempty[a] leader's only, 8 arrivals (4 epilogue warps
-//             of each CTA, the peer's arrive through the cluster window).
+//   tfull[a]  one per CTA (multicast commit); tempty[a] leader's only, one arrival per epilogue warp
+//             of both CTAs (the peer's arrive through the cluster window).
 // Stage layout and K-loop order are those of the single-CTA kernel (Path A FP4 blocks, then Path B
 // BF16 blocks, 128 bytes per operand row and stage).
 #include <cuda_bf16.h>
@@ -25,24 +25,16 @@ namespace osc {
 
 namespace pair {
 
-#ifdef OSC_TRACE
-constexpr int TRACE_CAP = 96;
-__device__ __forceinline__ long long gtime() { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
-#define TRACE(role, idx, slot) do { if (args.trace && blockIdx.x < 4 && (idx) < TRACE_CAP) args.trace[(((blockIdx.x * 4 + (role)) * TRACE_CAP + (idx)) * 2) + (slot)] = gtime(); } while (0)
-#else
-#define TRACE(role, idx, slot) do {} while (0)
-#endif
-
 constexpr int MODE_OSC = 0;
 constexpr int MODE_FP8 = 1;
 constexpr int BM = 128;        // rows per CTA; the pair covers 256
 constexpr int ROW_BYTES = 128;
 constexpr int A_BYTES = BM * ROW_BYTES;
-constexpr int THREADS = 192;
+constexpr int EPI_WARPS = 8;     // two per TMEM lane quarter, each draining every other 64-column slice
+constexpr int THREADS = 64 + 32 * EPI_WARPS;
 constexpr int TMEM_COLS = 512;
 constexpr int BAND = 4;        // 256-row tiles per scheduling band
-constexpr int EPI_TILE_BYTES = 32 * 128;            // 32 rows x 64 bf16 columns
-constexpr int EPI_BYTES = 4 * 2 * EPI_TILE_BYTES;   // 4 epilogue warps x 2 staging tiles
+constexpr int EPI_TILE_BYTES = 32 * 128;            // staging tile: 32 rows x 64 bf16 columns
 
 template <int MODE, int BN>
 struct Cfg {
@@ -53,11 +45,9 @@ struct Cfg {
     static constexpr int SFA_BYTES = (MODE == MODE_OSC) ? 1024 : 0;
     static constexpr int SFB_BYTES = (MODE == MODE_OSC) ? SFB_ATOMS * 1024 : 0;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + SFA_BYTES + SFB_BYTES;
-#ifdef OSC_FORCE_STAGES
-    static constexpr int STAGES = OSC_FORCE_STAGES;
-#else
+    static constexpr int EPI_WARP_BYTES = (BN / 64) * EPI_TILE_BYTES;  // one warp's 32 x BN output rows
+    static constexpr int EPI_BYTES = 4 * EPI_WARP_BYTES;
     static constexpr int STAGES = (224 * 1024 - EPI_BYTES) / STAGE_BYTES;
-#endif
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/ + EPI_BYTES;
     static constexpr int TM_SFA = ACC_STAGES * BN;
     static constexpr int TM_SFB = TM_SFA + 8;
@@ -82,7 +72,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_pair_kernel(const __grid_cons
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     // [operand ring][epilogue staging tiles, 1024-byte aligned for the swizzle][barriers]
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * C::STAGE_BYTES + EPI_BYTES);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * C::STAGE_BYTES + C::EPI_BYTES);
     uint64_t* full_bar = bars;
     uint64_t* empty_bar = bars + STAGES;
     uint64_t* tfull_bar = bars + 2 * STAGES;
@@ -106,7 +96,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_pair_kernel(const __grid_cons
         }
         for (int i = 0; i < ACC; ++i) {
             mbar_init(&tfull_bar[i], 1);
-            mbar_init(&tempty_bar[i], 8);
+            mbar_init(&tempty_bar[i], 2 * EPI_WARPS);
         }
         *abort_flag = 0;
         fence_barrier_init();
@@ -159,15 +149,13 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_pair_kernel(const __grid_cons
             int s = 0;
             uint32_t ph = 0;
             const uint32_t full0 = map_to_cta(smem_u32(&full_bar[0]), 0);  // the leader's full barriers
-            int ev = 0;
             for (int t = pair_id; t < total; t += num_pairs) {
                 int row0, n0;
                 tile_rc(t, row0, n0);
                 const int arow = row0 + (int)rank * BM;            // my 128 activation rows
                 const int brow = n0 + (int)rank * (BN / 2);        // my half of the weight rows
                 for (int kb = 0; kb < nkb; ++kb) {
-                    if (!wait_bounded_cluster(&empty_bar[s], ph ^ 1u, abort_flag, 11)) goto done;
-                    if (lane == 0) TRACE(0, ev, 0);
+                    if (!wait_bounded(&empty_bar[s], ph ^ 1u, abort_flag, 11)) goto done;
                     const uint32_t st = smem_u32(smem + s * C::STAGE_BYTES);
                     const uint32_t fb = full0 + (uint32_t)s * 8u;
                     if (elect_one()) {
@@ -192,10 +180,8 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_pair_kernel(const __grid_cons
                         tma_load_2d_pair(st, &args.tm_ao, fb, kk * 64, arow);
                         tma_load_2d_pair(st + A_BYTES, &args.tm_bo, fb, kk * 64, brow);
                     }
-                    TRACE(0, ev, 1);
                     }
                     __syncwarp();
-                    ++ev;
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
             }
@@ -212,7 +198,6 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_pair_kernel(const __grid_cons
             const uint64_t desc_hi = smem_desc_sw128(0);  // everything but the start address
             const uint64_t sf_hi = smem_desc_sf(0);
             const uint32_t smem0 = smem_u32(smem);
-            int ev = 0;
             for (int t = pair_id; t < total; t += num_pairs) {
                 int row0, n0;
                 tile_rc(t, row0, n0);
@@ -221,9 +206,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_pair_kernel(const __grid_cons
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
                 const uint32_t sfb_tm = tmem_base + C::TM_SFB + (uint32_t)((n0 % 128) / 32);
                 for (int kb = 0; kb < nkb; ++kb) {
-                    if (!wait_bounded_cluster(&full_bar[s], ph, abort_flag, 13)) goto done;
-                    if (lane == 0) TRACE(1, ev, 0);
-                    tc_fence_after();
+                    if (!wait_bounded(&full_bar[s], ph, abort_flag, 13)) goto done;
                     const uint32_t sbase = smem0 + s * C::STAGE_BYTES;
                     const uint64_t adesc = desc_hi | (uint64_t)(sbase >> 4);
                     const uint64_t bdesc = desc_hi | (uint64_t)((sbase + A_BYTES) >> 4);
@@ -237,7 +220,7 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_pair_kernel(const __grid_cons
                         const uint32_t sfo = (uint32_t)(kb & 1) * C::TM_SF_STRIDE;
 #pragma unroll
                         for (int a = 0; a < 2; ++a) {
-                            if (a < ka && !(args.dbg & 1)) {
+                            if (a < ka) {
                                 tc_copy_sf_pair(tmem_base + sfo + C::TM_SFA + a * 4, sfa_d + (uint64_t)(a * 32));
 #pragma unroll
                                 for (int j = 0; j < C::SFB_ATOMS; ++j)
@@ -245,10 +228,9 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_pair_kernel(const __grid_cons
                                                     sfb_d + (uint64_t)(j * 64 + a * 32));
                             }
                         }
-                        TRACE(1, ev, 1);
 #pragma unroll
                         for (int k = 0; k < 4; ++k) {
-                            if (k < 2 * ka && !(args.dbg & 16)) {
+                            if (k < 2 * ka) {
                                 constexpr uint32_t SFID[2] = {idesc_sf_ids(0, 0), idesc_sf_ids(2, 2)};
                                 mma_mxf4_pair(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC_A | SFID[k & 1],
                                               tmem_base + sfo + C::TM_SFA + (k >> 1) * 4,
@@ -263,12 +245,9 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_pair_kernel(const __grid_cons
                         for (int k = 0; k < 4; ++k)
                             mma_f8_pair(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC_A, (kb | k) ? 1u : 0u);
                     }
-                    TRACE(2, ev, 0);
                     tc_commit_pair(&empty_bar[s], 3);  // frees the stage in both CTAs
-                    TRACE(2, ev, 1);
                     }
                     __syncwarp();
-                    ++ev;
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
                 if (elect_one()) tc_commit_pair(&tfull_bar[acc], 3);    // accumulator ready in both CTAs
@@ -278,41 +257,40 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_pair_kernel(const __grid_cons
         }
     } else {
         // ---------------------------------------------------------------- epilogue (both CTAs)
-        // Each warp owns 32 accumulator rows.  Per 64-column slice: TMEM -> registers -> bf16 ->
-        // a swizzled 32 x 128-byte staging tile in shared memory -> one TMA store.  Two staging
-        // tiles per warp alternate, so packing the next slice overlaps the store of the last one.
-        // Plain per-thread stores (32 rows x 16 bytes per instruction) kept the memory pipe busy for
-        // the whole epilogue and stalled the MMA issue of the next tile.
-        const int q = warp & 3;
+        // Each warp owns 32 accumulator rows.  Drain: per 64-column slice TMEM -> registers -> bf16
+        // -> a swizzled 32 x 128-byte staging tile in shared memory (one tile per slice, so nothing
+        // waits inside the drain).  As soon as the last slice has left TMEM the accumulator is handed
+        // back to the MMA warp; only then are the TMA stores of the staged tile issued, and they
+        // drain to global memory while the next tile's MMAs run.  (Per-thread global stores, 32 rows
+        // x 16 bytes per instruction, kept the memory pipe busy and stalled the next tile's MMA issue.)
+        const int q = warp & 3;             // TMEM lane quarter this warp may read
+        const int half = (warp - 2) >> 2;   // which of the two warps of that quarter: slices c = half, half + 2, ...
         int acc = 0;
         uint32_t acc_ph = 0;
         const uint32_t tempty0 = map_to_cta(smem_u32(&tempty_bar[0]), 0);
-        uint8_t* stage_buf = smem + STAGES * C::STAGE_BYTES + q * (2 * EPI_TILE_BYTES);
-        int nstore = 0;
-        int ev = 0;
+        uint8_t* stage_buf = smem + STAGES * C::STAGE_BYTES + q * C::EPI_WARP_BYTES;
         for (int t = pair_id; t < total; t += num_pairs) {
             int row0, n0;
             tile_rc(t, row0, n0);
             if (!wait_bounded_cluster(&tfull_bar[acc], acc_ph, abort_flag, 14)) goto done;
-            if (warp == 2 && lane == 0) TRACE(3, ev, 0);
             tc_fence_after();
             const int wrow0 = row0 + (int)rank * BM + q * 32;  // first row of this warp
             const int row = wrow0 + lane;
             float sxr = 1.0f;
             if (MODE == MODE_FP8 && row < args.M) sxr = args.sx[row];
+            // the stores of the previous tile must be done reading the staging tiles
+            if (lane == 0) tma_store_wait_read<0>();
+            __syncwarp();
 #pragma unroll 1
-            for (int c = 0; c < BN / 64; ++c) {
+            for (int c = half; c < BN / 64; c += EPI_WARPS / 4) {
                 uint32_t r0[32], r1[32];
                 const uint32_t tcol = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + c * 64);
                 tmem_ld_32x32(tcol, r0);
                 tmem_ld_32x32(tcol + 32, r1);
                 tmem_ld_wait();
                 const int col = n0 + c * 64;
-                uint8_t* buf = stage_buf + (nstore & 1) * EPI_TILE_BYTES;
-                // the store that last read this staging tile (two stores ago) must be done reading
-                if (lane == 0) tma_store_wait_read<1>();
-                __syncwarp();
-                if (col < N && !(args.dbg & 8)) {
+                uint8_t* buf = stage_buf + c * EPI_TILE_BYTES;
+                if (col < N) {
 #pragma unroll
                     for (int j = 0; j < 8; ++j) {  // 8 chunks of 16 bytes = 8 columns each
                         uint32_t o[4];
@@ -333,20 +311,19 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_pair_kernel(const __grid_cons
                         *reinterpret_cast<uint4*>(buf + lane * 128 + ((j ^ (lane & 7)) << 4)) =
                             make_uint4(o[0], o[1], o[2], o[3]);
                     }
-                    fence_proxy_async_smem();
-                    __syncwarp();
-                    if (lane == 0) {
-                        tma_store_2d(&args.tm_y, buf, col, wrow0);
-                        tma_store_commit();
-                    }
-                    ++nstore;
                 }
             }
+            // accumulator drained: hand it back before the stores
             tc_fence_before();
+            fence_proxy_async_smem();
             __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(tempty0 + (uint32_t)acc * 8u);
-            if (warp == 2 && lane == 0) TRACE(3, ev, 1);
-            ++ev;
+            if (lane == 0) {
+                mbar_arrive_cluster(tempty0 + (uint32_t)acc * 8u);
+                for (int c = half; c < BN / 64; c += EPI_WARPS / 4)
+                    if (n0 + c * 64 < N) tma_store_2d(&args.tm_y, stage_buf + c * EPI_TILE_BYTES, n0 + c * 64, wrow0);
+                tma_store_commit();
+            }
+            __syncwarp();
             if (++acc == ACC) { acc = 0; acc_ph ^= 1u; }
         }
         if (lane == 0) tma_store_wait_all<0>();
@@ -404,37 +381,39 @@ static cudaError_t launch_cfg(const GemmArgs& a, cudaStream_t st) {
     if (const char* e = getenv("OSC_PAIRS")) { const int v = atoi(e); if (v > 0 && v < pairs) pairs = v; }
     if (total < pairs) pairs = total;
     cfg.gridDim = dim3(2 * pairs);
-    GemmArgs b = a;
-    if (const char* e = getenv("OSC_DEBUG")) b.dbg = atoi(e);
-    if (const char* e = getenv("OSC_TRACE_PTR")) b.trace = reinterpret_cast<long long*>(strtoull(e, nullptr, 0));
-    return cudaLaunchKernelEx(&cfg, gemm_pair_kernel<MODE, BN>, b);
+    return cudaLaunchKernelEx(&cfg, gemm_pair_kernel<MODE, BN>, a);
 }
 
 }  // namespace pair
 
-static int g_pair_bn = 0;
-int gemm_pair_block_n() {
-    if (g_pair_bn == 0) {
-        g_pair_bn = 256;
+// Tile width of the pair kernel for a given problem: the pair tile is 256 x BN and the kernel is
+// persistent over num_sms/2 pairs, so the cost is (rounds of tiles) x (time per tile).  Measured on
+// B200 a 256-wide tile (single accumulator, epilogue drain exposed) takes ~1.38x the time of a
+// 192-wide one (two accumulators, epilogue hidden).  OSC_PAIR_BLOCK_N overrides.
+int gemm_pair_block_n(int M, int N, int num_sms) {
+    static int forced = -1;
+    if (forced < 0) {
+        forced = 0;
         if (const char* e = getenv("OSC_PAIR_BLOCK_N")) {
             const int v = atoi(e);
-            if (v == 192 || v == 256) g_pair_bn = v;
+            if (v == 192 || v == 256) forced = v;
         }
     }
-    return g_pair_bn;
+    if (forced) return forced;
+    const int pairs = num_sms / 2 > 0 ? num_sms / 2 : 1;
+    const long mt = (M + 255) / 256;
+    const long r192 = (mt * ((N + 191) / 192) + pairs - 1) / pairs;
+    const long r256 = (mt * ((N + 255) / 256) + pairs - 1) / pairs;
+    return (100 * r192 <= 138 * r256) ? 192 : 256;
 }
 
-cudaError_t launch_gemm_dual_pair(const GemmArgs& a, cudaStream_t st) {
-    switch (gemm_pair_block_n()) {
-        case 192: return pair::launch_cfg<pair::MODE_OSC, 192>(a, st);
-        default: return pair::launch_cfg<pair::MODE_OSC, 256>(a, st);
-    }
+cudaError_t launch_gemm_dual_pair(const GemmArgs& a, int bn, cudaStream_t st) {
+    if (bn == 192) return pair::launch_cfg<pair::MODE_OSC, 192>(a, st);
+    return pair::launch_cfg<pair::MODE_OSC, 256>(a, st);
 }
-cudaError_t launch_gemm_fp8_pair(const GemmArgs& a, cudaStream_t st) {
-    switch (gemm_pair_block_n()) {
-        case 192: return pair::launch_cfg<pair::MODE_FP8, 192>(a, st);
-        default: return pair::launch_cfg<pair::MODE_FP8, 256>(a, st);
-    }
+cudaError_t launch_gemm_fp8_pair(const GemmArgs& a, int bn, cudaStream_t st) {
+    if (bn == 192) return pair::launch_cfg<pair::MODE_FP8, 192>(a, st);
+    return pair::launch_cfg<pair::MODE_FP8, 256>(a, st);
 }
 
 }  // namespace osc
