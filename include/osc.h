@@ -128,6 +128,24 @@ osc_status osc_gemm_dual(const osc_weights* w, const void* xq, const void* sfa, 
 osc_status osc_linear(const osc_weights* w, const void* X, int M, int64_t ldx, void* Y, int64_t ldy,
                       void* workspace, size_t workspace_bytes, void* stream);
 
+/* osc_linear without a caller workspace.  (The paper has no counterpart: this is a deployment aid.)
+ * For callers that cannot supply scratch memory - e.g. a plug-in whose host hands it only the input and
+ * output pointers, or code that must not allocate because an allocation would synchronise the device.
+ * The scratch between the two kernels lives in a fixed array of OSC_STATIC_SCRATCH_BYTES inside the
+ * library (every GPU that loads the library holds it until the process exits).  The call allocates
+ * nothing.  Limits and rules:
+ *   - dense weights only; the workspace size osc_act_sizes reports for M must not exceed
+ *     OSC_STATIC_SCRATCH_BYTES (e.g. M <= 1024 at K = 4096, K_o_pad = 256), else OSC_ERR_WORKSPACE;
+ *   - the first call on each device looks the array's device address up (one runtime query, with
+ *     that device current); make that first call before any stream capture;
+ *   - all calls on a device share the one array: two calls that may overlap on the GPU (different
+ *     streams without an ordering between them) race on it.  Calls on one stream are safe, and no call
+ *     depends on what an earlier one left behind.
+ * Arguments, layouts, status codes and asynchrony are those of osc_linear. */
+#define OSC_STATIC_SCRATCH_BYTES (4 * 1024 * 1024)
+osc_status osc_linear_static(const osc_weights* w, const void* X, int M, int64_t ldx, void* Y, int64_t ldy,
+                             void* stream);
+
 /* Grouped (MoE) form: rows of X_perm are sorted by expert, expert e owns rows
  * [off[e], off[e+1]); off: dev int32 [E+1], off[E] == M_total.  Expert e's scale rows start
  * at scale row sum_{e'<e} roundup(m_e', 128).  The tile schedule is built on the device. */

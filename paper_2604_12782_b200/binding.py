@@ -60,6 +60,7 @@ _SIGS = {
     "osc_quantize_extract": (_i, [_vp, _vp, _i, _i64, _vp, _vp, _vp, _vp]),
     "osc_gemm_dual": (_i, [_vp, _vp, _vp, _vp, _i, _vp, _i64, _vp]),
     "osc_linear": (_i, [_vp, _vp, _i, _i64, _vp, _i64, _vp, _sz, _vp]),
+    "osc_linear_static": (_i, [_vp, _vp, _i, _i64, _vp, _i64, _vp]),
     "osc_linear_grouped": (_i, [_vp, _vp, _vp, _i, _i64, _vp, _i64, _vp, _sz, _vp]),
     "osc_fp8_prepare_weights": (_i, [_vp, _i, _i, _i64, _vp, _vp, _vp, C.POINTER(_vp)]),
     "osc_fp8_prepare_weights_grouped": (_i, [_vp, _i, _i, _i, _vp, _vp, _vp, C.POINTER(_vp)]),
@@ -211,6 +212,14 @@ def osc_linear(w: OscWeights, X: torch.Tensor, Y: torch.Tensor, workspace: torch
     M = X.shape[0]
     _check(_lib.osc_linear(w.ptr, _ptr(X), M, X.stride(0) if M else w.K, _ptr(Y), Y.stride(0) if M else w.N,
                            _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)))
+
+
+def osc_linear_static(w: OscWeights, X: torch.Tensor, Y: torch.Tensor, stream=None):
+    """osc_linear for callers that cannot provide a workspace: the scratch is a fixed array inside the
+    library (limited size, shared by all calls on a device); nothing is allocated here or in the library."""
+    M = X.shape[0]
+    _check(_lib.osc_linear_static(w.ptr, _ptr(X), M, X.stride(0) if M else w.K, _ptr(Y), Y.stride(0) if M else w.N,
+                                  _stream(stream)))
 
 
 def osc_linear_grouped(w: OscWeights, X: torch.Tensor, off: torch.Tensor, Y: torch.Tensor, workspace: torch.Tensor,

@@ -4,3 +4,4 @@
 #include "gemm_kernels.cu"
 #include "gemm2_kernels.cu"
 #include "api.cu"
+#include "static_scratch.cu"
