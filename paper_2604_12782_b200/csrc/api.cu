@@ -382,7 +382,7 @@ static osc_status gemm_impl(const osc_weights* w, const void* xq, const void* sf
     a.sched = sched; a.max_tiles = max_tiles; a.num_sms = w->num_sms;
     cudaError_t e;
     if (use_pair_kernel(w->grouped, M)) {
-        const int bn = gemm_pair_block_n(M, w->N, w->num_sms);
+        const int bn = gemm_pair_block_n(M, w->N, (w->K + 255) / 256 + w->Kop / 64, w->num_sms);
         a.tm_b = w->tm_b2[bn == 256];
         a.tm_bo = w->tm_bo2[bn == 256];
         a.tm_sfw = w->tm_sfw;
@@ -537,7 +537,7 @@ static osc_status fp8_gemm_impl(const osc_fp8_weights* w, const void* x8, const 
     a.sched = sched; a.max_tiles = max_tiles; a.num_sms = w->num_sms;
     cudaError_t e;
     if (use_pair_kernel(w->grouped, M)) {
-        const int bn = gemm_pair_block_n(M, w->N, w->num_sms);
+        const int bn = gemm_pair_block_n(M, w->N, w->K / 128, w->num_sms);
         a.tm_b = w->tm_b2[bn == 256];
         if (osc_status s = make_tmap(&a.tm_y, Y, true, M, (uint64_t)w->N * 2, (uint64_t)ldy * 2, 32)) return s;
         e = launch_gemm_fp8_pair(a, bn, st);

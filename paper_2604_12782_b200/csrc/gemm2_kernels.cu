@@ -386,11 +386,12 @@ static cudaError_t launch_cfg(const GemmArgs& a, cudaStream_t st) {
 
 }  // namespace pair
 
-// Tile width of the pair kernel for a given problem: the pair tile is 256 x BN and the kernel is
-// persistent over num_sms/2 pairs, so the cost is (rounds of tiles) x (time per tile).  Measured on
-// B200 a 256-wide tile (single accumulator, epilogue drain exposed) takes ~1.38x the time of a
-// 192-wide one (two accumulators, epilogue hidden).  OSC_PAIR_BLOCK_N overrides.
-int gemm_pair_block_n(int M, int N, int num_sms) {
+// Tile width of the pair kernel for a given problem.  The pair tile is 256 x BN and the kernel is
+// persistent over num_sms/2 pairs, so the cost is (rounds of tiles) x (time per tile).  Per tile:
+// a 192-wide tile has two accumulators (epilogue drain hidden behind the next tile's K loop unless the
+// K loop is shorter than the drain), a 256-wide tile has one (drain exposed).  Stage and drain times are
+// the measured ones on B200 (ns).  OSC_PAIR_BLOCK_N overrides.
+int gemm_pair_block_n(int M, int N, int stages, int num_sms) {
     static int forced = -1;
     if (forced < 0) {
         forced = 0;
@@ -404,7 +405,10 @@ int gemm_pair_block_n(int M, int N, int num_sms) {
     const long mt = (M + 255) / 256;
     const long r192 = (mt * ((N + 191) / 192) + pairs - 1) / pairs;
     const long r256 = (mt * ((N + 255) / 256) + pairs - 1) / pairs;
-    return (100 * r192 <= 138 * r256) ? 192 : 256;
+    const long loop192 = 370L * stages, loop256 = 450L * stages;
+    const long t192 = loop192 > 2000 ? loop192 : 2000;  // drain of 192 columns ~2.0 us, overlapped
+    const long t256 = loop256 + 2500;                   // drain of 256 columns ~2.5 us, exposed
+    return (r192 * t192 <= r256 * t256) ? 192 : 256;
 }
 
 cudaError_t launch_gemm_dual_pair(const GemmArgs& a, int bn, cudaStream_t st) {

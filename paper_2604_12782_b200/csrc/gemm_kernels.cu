@@ -1,7 +1,10 @@
-// Tensor-core kernels (tcgen05 + TMEM + TMA), one persistent CTA per SM, warp-specialised:
+// Single-CTA tensor-core kernels (tcgen05 + TMEM + TMA), one persistent CTA per SM, warp-specialised.
+// Used for grouped (MoE) problems and for dense problems with few rows; dense problems with many rows
+// go to the CTA-pair kernel.
 //   warp 0    : TMA producer (operand tiles + scale-factor blocks into a shared-memory ring)
-//   warp 1    : MMA issuer (one thread) and TMEM owner
-//   warps 2-5 : epilogue (TMEM -> registers -> bf16 -> global)
+//   warp 1    : MMA issuer (one elected lane of the converged warp) and TMEM owner
+//   warps 2-9 : epilogue (TMEM -> registers -> bf16 -> swizzled shared-memory tile -> row-masked,
+//               line-wide global stores)
 //
 // MODE_OSC : Eq. 5.  For every 128 x BN output tile the K loop first runs the block-scaled FP4
 //            blocks of Path A (256 channels = 128 bytes per row and stage, four K=64 MMAs with
@@ -12,8 +15,9 @@
 // MODE_FP8 : Section 3.4 fallback.  E4M3 x E4M3 (128 channels per stage, four K=32 MMAs); the
 //            per-row activation scale and per-output-row weight scale are applied in the epilogue.
 //
-// Dense and grouped (MoE) problems share the kernel: a tile's first row, last valid row, first
-// scale row and expert come either from arithmetic (dense) or from the device-built schedule.
+// A tile's first row, last valid row, first scale row and expert come either from arithmetic
+// (dense) or from the device-built schedule (grouped): rows past an expert's end are computed
+// (they read the next expert's rows or zero fill) but never stored.
 #include <cuda_bf16.h>
 
 #include "common.cuh"
@@ -26,24 +30,31 @@ constexpr int MODE_FP8 = 1;
 constexpr int BM = 128;            // rows per tile = TMEM lanes
 constexpr int ROW_BYTES = 128;     // bytes per operand row and stage (one 128-byte swizzle row)
 constexpr int A_BYTES = BM * ROW_BYTES;
-constexpr int GEMM_THREADS = 192;
+constexpr int G_EPI_WARPS = 8;     // two per TMEM lane quarter, each draining every other 64-column slice
+constexpr int GEMM_THREADS = 64 + 32 * G_EPI_WARPS;
 constexpr int TMEM_COLS = 512;
 constexpr int BAND = 8;            // row tiles per scheduling band (L2 reuse of the weight tiles)
+constexpr int G_EPI_TILE_BYTES = 32 * 128;  // staging tile: 32 rows x 64 bf16 columns
 
 template <int MODE, int BN>
 struct Cfg {
-    static constexpr int ACC_STAGES = (BN <= 192) ? 2 : 1;
     static constexpr int SFB_ATOMS = (BN > 128) ? 2 : 1;  // 128-row scale blocks a tile can touch
+    static constexpr int SF_COLS = 8 + 2 * SFB_ATOMS * 4;  // TMEM columns of one stage's scales (A: 8, B: 2 x atoms x 4)
+    static constexpr int ACC_STAGES = (2 * BN + SF_COLS <= TMEM_COLS) ? 2 : 1;
     static constexpr int B_BYTES = BN * ROW_BYTES;
     static constexpr int SFA_BYTES = (MODE == MODE_OSC) ? 1024 : 0;
     static constexpr int SFB_BYTES = (MODE == MODE_OSC) ? SFB_ATOMS * 1024 : 0;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + SFA_BYTES + SFB_BYTES;  // multiple of 1024
-    static constexpr int STAGES = (200 * 1024) / STAGE_BYTES;
-    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
-    static constexpr int TM_SFA = ACC_STAGES * BN;  // TMEM column of the activation scales (8 columns)
-    static constexpr int TM_SFB = TM_SFA + 8;       // weight scales: 2 K-blocks x SFB_ATOMS x 4 columns
+    static constexpr int EPI_WARP_BYTES = (BN / 64) * G_EPI_TILE_BYTES;            // one lane quarter's 32 x BN outputs
+    static constexpr int EPI_BYTES = 4 * EPI_WARP_BYTES;
+    static constexpr int STAGES = (224 * 1024 - EPI_BYTES) / STAGE_BYTES;
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+    static constexpr int TM_SFA = ACC_STAGES * BN;  // TMEM column of the activation scales
+    static constexpr int TM_SFB = TM_SFA + 8;       // weight scales
     static_assert(STAGE_BYTES % 1024 == 0, "stage must keep 1024-byte alignment");
-    static_assert(TM_SFB + 2 * SFB_ATOMS * 4 <= TMEM_COLS, "TMEM budget");
+    static_assert(TM_SFA + SF_COLS <= TMEM_COLS, "TMEM budget");
+    static_assert(STAGES >= 3, "ring too shallow");
+    static_assert(BN % 64 == 0, "tile width");
 };
 
 struct TileInfo {
@@ -87,7 +98,8 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * C::STAGE_BYTES);
+    // [operand ring][epilogue staging tiles, 1024-byte aligned for the swizzle][barriers]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * C::STAGE_BYTES + C::EPI_BYTES);
     uint64_t* full_bar = bars;
     uint64_t* empty_bar = bars + STAGES;
     uint64_t* tfull_bar = bars + 2 * STAGES;
@@ -96,7 +108,9 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 2 * ACC + 1);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
-    const int warp = threadIdx.x >> 5;
+    // warp-uniform values go through a shuffle so that the address arithmetic of the TMA / tcgen05
+    // instructions stays in uniform registers (they are issued by one elected lane of a converged warp)
+    const int warp = __shfl_sync(0xFFFFFFFFu, (int)(threadIdx.x >> 5), 0);
     const int lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
@@ -106,7 +120,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
         }
         for (int i = 0; i < ACC; ++i) {
             mbar_init(&tfull_bar[i], 1);
-            mbar_init(&tempty_bar[i], 4);
+            mbar_init(&tempty_bar[i], G_EPI_WARPS);
         }
         mbar_init(drain_bar, 1);
         *abort_flag = 0;
@@ -125,7 +139,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t tmem_base = __shfl_sync(0xFFFFFFFFu, *tmem_slot, 0);
 
     const int N = args.N, K = args.K;
     const int num_m = num_row_tiles(args);
@@ -141,15 +155,15 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
-        if (lane == 0) {
-            int s = 0;
-            uint32_t ph = 0;
-            for (int t = blockIdx.x; t < total; t += gridDim.x) {
-                const TileInfo ti = tile_info<BN>(args, t, num_m, num_n);
-                const int brow = ti.expert * N + ti.n0;
-                for (int kb = 0; kb < nkb; ++kb) {
-                    if (!wait_bounded(&empty_bar[s], ph ^ 1u, abort_flag, 1)) goto done;
-                    uint8_t* st = smem + s * C::STAGE_BYTES;
+        int s = 0;
+        uint32_t ph = 0;
+        for (int t = blockIdx.x; t < total; t += gridDim.x) {
+            const TileInfo ti = tile_info<BN>(args, t, num_m, num_n);
+            const int brow = ti.expert * N + ti.n0;
+            for (int kb = 0; kb < nkb; ++kb) {
+                if (!wait_bounded(&empty_bar[s], ph ^ 1u, abort_flag, 1)) goto done;
+                uint8_t* st = smem + s * C::STAGE_BYTES;
+                if (elect_one()) {
                     if (kb < nkb_a) {
                         if (MODE == MODE_OSC) {
                             const int ka = min(2, katoms_total - 2 * kb);  // 128-channel scale blocks in this stage
@@ -177,107 +191,145 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
                         tma_load_2d(st, &args.tm_ao, &full_bar[s], kk * 64, ti.row0);
                         tma_load_2d(st + A_BYTES, &args.tm_bo, &full_bar[s], kk * 64, brow);
                     }
-                    if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
+                __syncwarp();
+                if (++s == STAGES) { s = 0; ph ^= 1u; }
             }
         }
     } else if (warp == 1) {
         // -------------------------------------------------------------- MMA issuer
-        if (lane == 0) {
-            int s = 0;
-            uint32_t ph = 0;
-            int acc = 0;
-            uint32_t acc_ph = 0;
-            constexpr uint32_t IDESC_A = (MODE == MODE_OSC) ? idesc_mxf4(BM, BN) : idesc_e4m3(BM, BN);
-            constexpr uint32_t IDESC_B = idesc_bf16(BM, BN);
-            for (int t = blockIdx.x; t < total; t += gridDim.x) {
-                const TileInfo ti = tile_info<BN>(args, t, num_m, num_n);
-                if (!wait_bounded(&tempty_bar[acc], acc_ph ^ 1u, abort_flag, 2)) goto done;
-                tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
-                const uint32_t sfb_col_off = (uint32_t)((ti.n0 % 128) / 32);
-                for (int kb = 0; kb < nkb; ++kb) {
-                    if (!wait_bounded(&full_bar[s], ph, abort_flag, 3)) goto done;
-                    tc_fence_after();
-                    const uint32_t sbase = smem_u32(smem + s * C::STAGE_BYTES);
-                    const uint64_t adesc = smem_desc_sw128(sbase);
-                    const uint64_t bdesc = smem_desc_sw128(sbase + A_BYTES);
+        int s = 0;
+        uint32_t ph = 0;
+        int acc = 0;
+        uint32_t acc_ph = 0;
+        constexpr uint32_t IDESC_A = (MODE == MODE_OSC) ? idesc_mxf4(BM, BN) : idesc_e4m3(BM, BN);
+        constexpr uint32_t IDESC_B = idesc_bf16(BM, BN);
+        const uint64_t desc_hi = smem_desc_sw128(0);  // everything but the start address
+        const uint64_t sf_hi = smem_desc_sf(0);
+        const uint32_t smem0 = smem_u32(smem);
+        for (int t = blockIdx.x; t < total; t += gridDim.x) {
+            const TileInfo ti = tile_info<BN>(args, t, num_m, num_n);
+            if (!wait_bounded(&tempty_bar[acc], acc_ph ^ 1u, abort_flag, 2)) goto done;
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+            const uint32_t sfb_tm = tmem_base + C::TM_SFB + (uint32_t)((ti.n0 % 128) / 32);
+            for (int kb = 0; kb < nkb; ++kb) {
+                if (!wait_bounded(&full_bar[s], ph, abort_flag, 3)) goto done;
+                const uint32_t sbase = smem0 + s * C::STAGE_BYTES;
+                const uint64_t adesc = desc_hi | (uint64_t)(sbase >> 4);
+                const uint64_t bdesc = desc_hi | (uint64_t)((sbase + A_BYTES) >> 4);
+                if (elect_one()) {
                     if (MODE == MODE_OSC && kb < nkb_a) {
                         const int ka = min(2, katoms_total - 2 * kb);
-                        const uint32_t sfa_s = sbase + A_BYTES + C::B_BYTES;
-                        const uint32_t sfb_s = sfa_s + C::SFA_BYTES;
-                        for (int a = 0; a < ka; ++a) {
-                            tc_copy_sf(tmem_base + C::TM_SFA + a * 4, smem_desc_sf(sfa_s + a * 512));
+                        const uint64_t sfa_d = sf_hi | (uint64_t)((sbase + A_BYTES + C::B_BYTES) >> 4);
+                        const uint64_t sfb_d = sf_hi | (uint64_t)((sbase + A_BYTES + C::B_BYTES + C::SFA_BYTES) >> 4);
 #pragma unroll
-                            for (int j = 0; j < C::SFB_ATOMS; ++j)
-                                tc_copy_sf(tmem_base + C::TM_SFB + a * (C::SFB_ATOMS * 4) + j * 4,
-                                           smem_desc_sf(sfb_s + j * 1024 + a * 512));
+                        for (int a = 0; a < 2; ++a) {
+                            if (a < ka) {
+                                tc_copy_sf(tmem_base + C::TM_SFA + a * 4, sfa_d + (uint64_t)(a * 32));
+#pragma unroll
+                                for (int j = 0; j < C::SFB_ATOMS; ++j)
+                                    tc_copy_sf(tmem_base + C::TM_SFB + a * (C::SFB_ATOMS * 4) + j * 4,
+                                               sfb_d + (uint64_t)(j * 64 + a * 32));
+                            }
                         }
-                        for (int k = 0; k < 2 * ka; ++k) {
-                            const uint32_t sfid = (uint32_t)(k & 1) * 2u;  // byte pair inside the 4-byte scale column
-                            mma_mxf4(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC_A | idesc_sf_ids(sfid, sfid),
-                                     tmem_base + C::TM_SFA + (k >> 1) * 4,
-                                     tmem_base + C::TM_SFB + (k >> 1) * (C::SFB_ATOMS * 4) + sfb_col_off,
-                                     (kb | k) ? 1u : 0u);
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            if (k < 2 * ka) {
+                                // byte pair inside the 4-byte scale column: 0 for the first, 2 for the second K=64 half
+                                constexpr uint32_t SFID[2] = {idesc_sf_ids(0, 0), idesc_sf_ids(2, 2)};
+                                mma_mxf4(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC_A | SFID[k & 1],
+                                         tmem_base + C::TM_SFA + (k >> 1) * 4, sfb_tm + (k >> 1) * (C::SFB_ATOMS * 4),
+                                         (kb | k) ? 1u : 0u);
+                            }
                         }
                     } else if (MODE == MODE_OSC) {
 #pragma unroll
-                        for (int k = 0; k < 4; ++k)
-                            mma_f16(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC_B, 1u);
+                        for (int k = 0; k < 4; ++k) mma_f16(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC_B, 1u);
                     } else {
 #pragma unroll
                         for (int k = 0; k < 4; ++k)
                             mma_f8(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC_A, (kb | k) ? 1u : 0u);
                     }
                     tc_commit(&empty_bar[s]);
-                    if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
-                tc_commit(&tfull_bar[acc]);
-                if (++acc == ACC) { acc = 0; acc_ph ^= 1u; }
+                __syncwarp();
+                if (++s == STAGES) { s = 0; ph ^= 1u; }
             }
+            if (elect_one()) tc_commit(&tfull_bar[acc]);
+            __syncwarp();
+            if (++acc == ACC) { acc = 0; acc_ph ^= 1u; }
         }
     } else {
         // ---------------------------------------------------------------- epilogue
-        const int q = warp & 3;  // TMEM lane quarter this warp may read
+        // Two warps per TMEM lane quarter (32 rows); each drains every other 64-column slice into a
+        // swizzled staging tile, hands the accumulator back, then writes the tile out with stores that
+        // cover whole 128-byte lines (8 lanes per row, 4 rows per instruction), skipping rows past the
+        // tile's last valid row.
+        const int q = warp & 3;
+        const int half = (warp - 2) >> 2;
         int acc = 0;
         uint32_t acc_ph = 0;
+        uint8_t* stage_buf = smem + STAGES * C::STAGE_BYTES + q * C::EPI_WARP_BYTES;
         for (int t = blockIdx.x; t < total; t += gridDim.x) {
             const TileInfo ti = tile_info<BN>(args, t, num_m, num_n);
             if (!wait_bounded(&tfull_bar[acc], acc_ph, abort_flag, 4)) goto done;
             tc_fence_after();
-            const int row = ti.row0 + q * 32 + lane;
-            const bool row_ok = row < ti.row_end;
+            const int wrow0 = ti.row0 + q * 32;
             float sxr = 1.0f;
-            if (MODE == MODE_FP8 && row_ok) sxr = args.sx[row];
-            uint16_t* yrow = args.Y + (int64_t)row * args.ldy;
+            if (MODE == MODE_FP8 && wrow0 + lane < ti.row_end) sxr = args.sx[wrow0 + lane];
             const float* swp = (MODE == MODE_FP8) ? args.sw + (int64_t)ti.expert * N : nullptr;
 #pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c) {
-                uint32_t r[32];
-                tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + c * 32), r);
+            for (int c = half; c < BN / 64; c += G_EPI_WARPS / 4) {
+                uint32_t r0[32], r1[32];
+                const uint32_t tcol = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + c * 64);
+                tmem_ld_32x32(tcol, r0);
+                tmem_ld_32x32(tcol + 32, r1);
                 tmem_ld_wait();
-                const int col = ti.n0 + c * 32;
-                if (row_ok && col < N) {
-                    uint32_t o[16];
+                const int col = ti.n0 + c * 64;
+                uint8_t* buf = stage_buf + c * G_EPI_TILE_BYTES;
+                if (col < N) {
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        float lo = __uint_as_float(r[2 * i]), hi = __uint_as_float(r[2 * i + 1]);
-                        if (MODE == MODE_FP8) {
-                            const float2 w2 = *reinterpret_cast<const float2*>(swp + col + 2 * i);
-                            lo = lo * (sxr * w2.x);
-                            hi = hi * (sxr * w2.y);
+                    for (int j = 0; j < 8; ++j) {  // 8 chunks of 16 bytes = 8 columns each
+                        uint32_t o[4];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const int cc = j * 8 + 2 * i;  // column inside the 64-column slice
+                            float lo = __uint_as_float(cc < 32 ? r0[cc] : r1[cc - 32]);
+                            float hi = __uint_as_float(cc < 32 ? r0[cc + 1] : r1[cc - 31]);
+                            if (MODE == MODE_FP8) {
+                                const float2 w2 = *reinterpret_cast<const float2*>(swp + col + cc);
+                                lo = lo * (sxr * w2.x);
+                                hi = hi * (sxr * w2.y);
+                            }
+                            const __nv_bfloat162 b2 = __floats2bfloat162_rn(lo, hi);
+                            o[i] = *reinterpret_cast<const uint32_t*>(&b2);
                         }
-                        const __nv_bfloat162 b = __floats2bfloat162_rn(lo, hi);
-                        o[i] = *reinterpret_cast<const uint32_t*>(&b);
+                        // 16-byte chunk j of row `lane` lives at chunk j ^ (lane % 8): conflict-free both ways
+                        *reinterpret_cast<uint4*>(buf + lane * 128 + ((j ^ (lane & 7)) << 4)) =
+                            make_uint4(o[0], o[1], o[2], o[3]);
                     }
-                    uint4* dst = reinterpret_cast<uint4*>(yrow + col);
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) dst[i] = make_uint4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
                 }
             }
+            // accumulator drained: hand it back before the stores
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&tempty_bar[acc]);
+#pragma unroll 1
+            for (int c = half; c < BN / 64; c += G_EPI_WARPS / 4) {
+                const int col = ti.n0 + c * 64;
+                if (col >= N) break;
+                const uint8_t* buf = stage_buf + c * G_EPI_TILE_BYTES;
+                const int j = lane & 7;  // 16-byte chunk of the row
+#pragma unroll
+                for (int rr = 0; rr < 8; ++rr) {
+                    const int rl = rr * 4 + (lane >> 3);  // row inside the warp's 32
+                    const int row = wrow0 + rl;
+                    const uint4 v = *reinterpret_cast<const uint4*>(buf + rl * 128 + ((j ^ (rl & 7)) << 4));
+                    if (row < ti.row_end) *reinterpret_cast<uint4*>(args.Y + (int64_t)row * args.ldy + col + j * 8) = v;
+                }
+            }
+            __syncwarp();
             if (++acc == ACC) { acc = 0; acc_ph ^= 1u; }
         }
     }

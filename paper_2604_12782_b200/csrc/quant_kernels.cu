@@ -269,6 +269,53 @@ fp8_quant_kernel(const uint16_t* __restrict__ X, int64_t ldx, int M, int K, uint
     }
 }
 
+// Short rows (K <= 2048): one warp per row, eight rows per CTA, the row held in registers
+// (at most 8 chunks of 8 elements per lane).  A CTA per row would leave most threads idle.
+constexpr int F8W_MAXCH = 8;
+__global__ void __launch_bounds__(256)
+fp8_quant_rows_kernel(const uint16_t* __restrict__ X, int64_t ldx, int M, int K, uint8_t* __restrict__ x8,
+                      float* __restrict__ sx) {
+    const int lane = threadIdx.x & 31;
+    const int r = blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (r >= M) return;
+    const uint16_t* xrow = X + (int64_t)r * ldx;
+    const int nch = K / 8;
+    uint4 v[F8W_MAXCH];
+    uint32_t am = 0;
+#pragma unroll
+    for (int i = 0; i < F8W_MAXCH; ++i) {
+        const int c = lane + i * 32;
+        if (c < nch) {
+            v[i] = *reinterpret_cast<const uint4*>(xrow + c * 8);
+            am = max(am, max(max(v[i].x & 0x7FFFu, (v[i].x >> 16) & 0x7FFFu), max(v[i].y & 0x7FFFu, (v[i].y >> 16) & 0x7FFFu)));
+            am = max(am, max(max(v[i].z & 0x7FFFu, (v[i].z >> 16) & 0x7FFFu), max(v[i].w & 0x7FFFu, (v[i].w >> 16) & 0x7FFFu)));
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) am = max(am, __shfl_xor_sync(0xFFFFFFFFu, am, o));
+    const float amax = __uint_as_float(am << 16);
+    const float amaxp = fmaxf(amax, __uint_as_float((uint32_t)(127 - 40) << 23));
+    const float scale = __fdiv_rn(amaxp, 448.0f);
+    const float inv = __fdiv_rn(448.0f, amaxp);
+    if (lane == 0) sx[r] = scale;
+    uint8_t* orow = x8 + (int64_t)r * K;
+#pragma unroll
+    for (int i = 0; i < F8W_MAXCH; ++i) {
+        const int c = lane + i * 32;
+        if (c < nch) {
+            const uint32_t w[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
+            uint32_t h[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const float lo = __fmul_rn(__uint_as_float(w[k] << 16), inv);
+                const float hi = __fmul_rn(__uint_as_float(w[k] & 0xFFFF0000u), inv);
+                h[k] = e4m3x2(lo, hi) & 0xFFFFu;
+            }
+            *reinterpret_cast<uint2*>(orow + c * 8) = make_uint2(h[0] | (h[1] << 16), h[2] | (h[3] << 16));
+        }
+    }
+}
+
 // ------------------------------------------------------------ grouped schedule
 // sched[0] = number of 128-row tiles; then four arrays of max_tiles entries:
 // first row, end row (exclusive, the expert's end), first scale row, expert.
@@ -323,6 +370,11 @@ cudaError_t launch_quant_extract(const CUtensorMap& tm_x, int M, int K, const ui
 
 cudaError_t launch_fp8_quant(const void* X, int64_t ldx, int M, int K, void* x8, void* sx, cudaStream_t st) {
     if (M <= 0) return cudaSuccess;
+    if (K <= F8W_MAXCH * 32 * 8) {
+        fp8_quant_rows_kernel<<<(M + 7) / 8, 256, 0, st>>>(static_cast<const uint16_t*>(X), ldx, M, K,
+                                                           static_cast<uint8_t*>(x8), static_cast<float*>(sx));
+        return cudaGetLastError();
+    }
     fp8_quant_kernel<<<M, F8_THREADS, 0, st>>>(static_cast<const uint16_t*>(X), ldx, M, K,
                                                static_cast<uint8_t*>(x8), static_cast<float*>(sx));
     return cudaGetLastError();
