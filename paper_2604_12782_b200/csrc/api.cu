@@ -82,17 +82,17 @@ static osc_status make_tmap(CUtensorMap* tm, const void* base, bool bf16, uint64
     return OSC_OK;
 }
 
-// bf16 [rows, cols] input of the quantizer: 128 x 128 tiles, no swizzle, zero fill.
+// bf16 [rows, cols] input of the quantizer: tiles of 128 rows x 64 channels (128 bytes), 128-byte swizzle, zero fill.
 static osc_status make_tmap_x(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint64_t ld) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return fail(OSC_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
     if (rows == 0) rows = 1;
     cuuint64_t gdim[2] = {cols, rows};
     cuuint64_t gstr[1] = {ld * 2};
-    cuuint32_t box[2] = {128, 128};
+    cuuint32_t box[2] = {64, 128};
     cuuint32_t estr[2] = {1, 1};
     CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstr, box, estr,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return fail(OSC_ERR_CUDA, "cuTensorMapEncodeTiled(X) failed with code %d", (int)r);
     return OSC_OK;

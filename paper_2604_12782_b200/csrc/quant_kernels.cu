@@ -30,20 +30,46 @@ __device__ __forceinline__ uint32_t e4m3x2(float lo, float hi) {
 }
 
 // ------------------------------------------------------- Algorithm 2, fused
-// Persistent kernel, one CTA per SM.  A producer warp streams 128-row x 128-channel tiles of X
-// (32 KB) through a shared-memory ring with TMA; eight consumer warps take a tile out of the ring
-// into registers, release the slot at once, and do the lookup / back-up / zero-out / scale /
-// quantize work while the next tiles are already in flight.  Thread t of the consumers owns 8
-// consecutive channels (t % 16) of row (t / 16) + 16 * pass; four neighbouring threads share a group.
+// Persistent kernel, two CTAs per SM.  A producer warp streams 128-row x 128-channel tiles of X
+// (32 KB, as two 64-channel halves with the 128-byte swizzle) through a shared-memory ring with
+// TMA.  512 consumer threads work on a tile in two steps:
+//   1. back-up + zero-out: one (row, flagged channel) task per thread copies the element from the
+//      shared tile into xo (the buffer B; consecutive threads write consecutive elements of a row)
+//      and overwrites it with +0 in shared memory;
+//   2. after a barrier every thread owns one 32-channel group of one row (64 bytes): amax, E8M0 code,
+//      exact fp32 scaling, hardware E2M1 conversion, one 16-byte store of the packed codes, one
+//      scale byte into the 512-byte scale block of the tile (staged in shared memory, written whole).
+// The slot is released as soon as the groups are in registers, so the next tiles stream in meanwhile.
 constexpr int QE_ROWS = 128;
 constexpr int QE_COLS = 128;
-constexpr int QE_CONSUMERS = 512;
+constexpr int QE_CONSUMERS = 512;               // = groups per tile
 constexpr int QE_THREADS = QE_CONSUMERS + 32;
-constexpr int QE_PASSES = QE_ROWS / (QE_CONSUMERS / 16);  // 8
-constexpr int QE_TILE_BYTES = QE_ROWS * QE_COLS * 2;
+constexpr int QE_HALF_BYTES = QE_ROWS * 128;    // 64 channels x 128 rows
+constexpr int QE_TILE_BYTES = 2 * QE_HALF_BYTES;
 constexpr int QE_STAGES = 3;
 constexpr int QE_CTAS_PER_SM = 2;
 constexpr int QE_SMEM = QE_STAGES * QE_TILE_BYTES + 1024 + 2 * 512 + 256;
+
+// byte offset of channel `col` (0..127) of row `row` inside a swizzled tile
+__device__ __forceinline__ int qe_elem_offset(int row, int col) {
+    const int half = col >> 6, within = (col & 63) * 2;
+    return half * QE_HALF_BYTES + row * 128 + ((((within >> 4) ^ (row & 7))) << 4) + (within & 15);
+}
+
+// eight fp32 values -> eight E2M1 codes packed into 32 bits (element 0 in the low nibble)
+__device__ __forceinline__ uint32_t e2m1x8(float f0, float f1, float f2, float f3, float f4, float f5, float f6,
+                                           float f7) {
+    uint32_t r;
+    asm("{ .reg .b8 t0, t1, t2, t3;\n\t"
+        "cvt.rn.satfinite.e2m1x2.f32 t0, %2, %1;\n\t"
+        "cvt.rn.satfinite.e2m1x2.f32 t1, %4, %3;\n\t"
+        "cvt.rn.satfinite.e2m1x2.f32 t2, %6, %5;\n\t"
+        "cvt.rn.satfinite.e2m1x2.f32 t3, %8, %7;\n\t"
+        "mov.b32 %0, {t0, t1, t2, t3}; }"
+        : "=r"(r)
+        : "f"(f0), "f"(f1), "f"(f2), "f"(f3), "f"(f4), "f"(f5), "f"(f6), "f"(f7));
+    return r;
+}
 
 __global__ void __launch_bounds__(QE_THREADS, QE_CTAS_PER_SM)
 quant_extract_kernel(const __grid_constant__ CUtensorMap tm_x, int M, int K,
@@ -74,34 +100,40 @@ quant_extract_kernel(const __grid_constant__ CUtensorMap tm_x, int M, int K,
     const int ncb = K / QE_COLS;  // 128-channel blocks per row
     const int nrt = sched ? sched[0] : (M + QE_ROWS - 1) / QE_ROWS;
     const int total = nrt * ncb;
+    // each CTA takes a contiguous run of tiles (channel block fastest), so neighbours in time are
+    // neighbours in memory and the (row tile, channel block) pair advances without divisions
+    const int per_cta = (total + gridDim.x - 1) / gridDim.x;
+    const int t_begin = min(total, (int)blockIdx.x * per_cta);
+    const int t_end = min(total, t_begin + per_cta);
 
     if (warp == QE_CONSUMERS / 32) {
         // ------------------------------------------------------------------ producer
         int s = 0;
         uint32_t ph = 0;
-        for (int t = blockIdx.x; t < total; t += gridDim.x) {
-            const int rt = t / ncb, cb = t - rt * ncb;
+        int rt = t_begin / ncb, cb = t_begin - rt * ncb;
+        for (int t = t_begin; t < t_end; ++t) {
             const int row0 = sched ? sched[1 + rt] : rt * QE_ROWS;
             if (!wait_bounded(&empty_bar[s], ph ^ 1u, abort_flag, 21)) break;
             if (elect_one()) {
                 mbar_arrive_expect_tx(&full_bar[s], QE_TILE_BYTES);
                 tma_load_2d(smem + s * QE_TILE_BYTES, &tm_x, &full_bar[s], cb * QE_COLS, row0);
+                tma_load_2d(smem + s * QE_TILE_BYTES + QE_HALF_BYTES, &tm_x, &full_bar[s], cb * QE_COLS + 64, row0);
             }
             __syncwarp();
             if (++s == QE_STAGES) { s = 0; ph ^= 1u; }
+            if (++cb == ncb) { cb = 0; ++rt; }
         }
     } else {
         // ----------------------------------------------------------------- consumers
         const int tid = threadIdx.x;
-        const int cchunk = tid & 15;  // 8-channel chunk inside the 128-channel block
-        const int gi = cchunk >> 2;   // group inside the block
-        const int sub = cchunk & 3;   // which quarter of the group
-        const int rsub = tid >> 4;    // 0 .. QE_CONSUMERS/16 - 1
+        const int grow = tid >> 2;  // my row inside the tile
+        const int gi = tid & 3;     // my group inside the 128-channel block
         int s = 0;
         uint32_t ph = 0;
         int parity = 0;
-        for (int t = blockIdx.x; t < total; t += gridDim.x) {
-            const int rt = t / ncb, cb = t - rt * ncb;
+        int rt = t_begin / ncb, cb = t_begin - rt * ncb;
+        int64_t prev_sf_blk = -1;
+        for (int t = t_begin; t < t_end; ++t) {
             int row0, row_end, sf_row0;
             if (sched) {
                 row0 = sched[1 + rt];
@@ -112,92 +144,95 @@ quant_extract_kernel(const __grid_constant__ CUtensorMap tm_x, int M, int K,
                 row_end = M;
                 sf_row0 = row0;
             }
-            // Per tile and thread: AND-masks that zero my flagged channels (the table is static, so the
-            // zero-out costs one logic op per register and no branch).
-            const uint32_t gmask = mask[cb * 4 + gi];
-            const uint32_t my8 = (gmask >> (sub * 8)) & 0xFFu;
-            uint32_t keep[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-                keep[i] = (((my8 >> (2 * i)) & 1u) ? 0u : 0x0000FFFFu) | (((my8 >> (2 * i + 1)) & 1u) ? 0u : 0xFFFF0000u);
-
             if (!wait_bounded(&full_bar[s], ph, abort_flag, 22)) break;
-            const uint8_t* st = smem + s * QE_TILE_BYTES;
-            uint4 v[QE_PASSES];
-#pragma unroll
-            for (int p = 0; p < QE_PASSES; ++p)
-                v[p] = *reinterpret_cast<const uint4*>(st + (rsub + (QE_CONSUMERS / 16) * p) * (QE_COLS * 2) + cchunk * 16);
+            uint8_t* st = smem + s * QE_TILE_BYTES;
 
-            // Back-up of the flagged channels of this 128-channel block into xo (the buffer B):
-            // one (row, channel) copy per task straight from the shared-memory tile, consecutive
-            // threads writing consecutive elements of a row.
-            {
-                const int o0 = prefix[cb * 4];
-                const int o1 = (cb * 4 + 4 < K / 32) ? prefix[cb * 4 + 4] : Ko;
-                const int nout = o1 - o0;
-                const int rows_here = min(QE_ROWS, row_end - row0);
-                for (int task = tid; task < rows_here * nout; task += QE_CONSUMERS) {
-                    const int rl = task / nout, k = task - rl * nout;
+            // step 1: back-up of the flagged channels of this block into xo, then zero them in the tile
+            const int o0 = prefix[cb * 4];
+            const int o1 = (cb * 4 + 4 < K / 32) ? prefix[cb * 4 + 4] : Ko;
+            const int nout = o1 - o0;
+            if (nout > 0) {
+                int shift = 0;
+                while ((1 << shift) < nout) ++shift;           // tasks: (row, k) with k < 2^shift
+                const int k = tid & ((1 << shift) - 1);
+                if (k < nout) {
                     const int col = idx_o[o0 + k] - cb * QE_COLS;
-                    xo[(int64_t)(row0 + rl) * Kop + o0 + k] =
-                        *reinterpret_cast<const uint16_t*>(st + rl * (QE_COLS * 2) + col * 2);
+                    const int rows_here = min(QE_ROWS, row_end - row0);
+                    for (int rl = tid >> shift; rl < QE_ROWS; rl += QE_CONSUMERS >> shift) {
+                        uint16_t* e = reinterpret_cast<uint16_t*>(st + qe_elem_offset(rl, col));
+                        if (rl < rows_here) xo[(int64_t)(row0 + rl) * Kop + o0 + k] = *e;
+                        *e = 0;
+                    }
+                }
+            }
+            // all flagged channels zeroed; all scale bytes of the previous tile staged
+            asm volatile("bar.sync 1, %0;" ::"n"(QE_CONSUMERS) : "memory");
+            if (prev_sf_blk >= 0 && tid < 32)
+                *reinterpret_cast<uint4*>(sf + prev_sf_blk * 512 + tid * 16) =
+                    *reinterpret_cast<const uint4*>(s_sf + (parity ^ 1) * 512 + tid * 16);
+
+            // step 2: my group into registers, then release the slot
+            uint32_t w[16];
+            {
+                const uint8_t* rowp = st + (gi >> 1) * QE_HALF_BYTES + grow * 128;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const uint4 v = *reinterpret_cast<const uint4*>(rowp + (((((gi & 1) << 2) + i) ^ (grow & 7)) << 4));
+                    w[4 * i] = v.x; w[4 * i + 1] = v.y; w[4 * i + 2] = v.z; w[4 * i + 3] = v.w;
                 }
             }
             __syncwarp();
-            if (lane == 0) mbar_arrive(&empty_bar[s]);  // the slot can be refilled while we work
+            if (lane == 0) mbar_arrive(&empty_bar[s]);
             if (++s == QE_STAGES) { s = 0; ph ^= 1u; }
 
-            uint8_t* sfb = s_sf + parity * 512;
+            const int r = row0 + grow;
+            int code = 0;
+            if (r < row_end) {  // rows past the end (next expert / padding) count as zeros: code 0, nothing stored
+                // amax on the bf16 magnitudes, two at a time
+                __nv_bfloat162 m2 = as_bf162(w[0] & 0x7FFF7FFFu);
 #pragma unroll
-            for (int p = 0; p < QE_PASSES; ++p) {
-                const int rl = rsub + (QE_CONSUMERS / 16) * p;  // row inside the tile
-                const int r = row0 + rl;
-                const bool live = r < row_end;  // rows past the end (next expert / padding) count as zeros
-                const uint32_t lm = live ? 0xFFFFFFFFu : 0u;
-                const uint32_t w[4] = {v[p].x & keep[0] & lm, v[p].y & keep[1] & lm, v[p].z & keep[2] & lm,
-                                       v[p].w & keep[3] & lm};
-                // amax over my 8 channels on the bf16 magnitudes (sign bits cleared: all values >= 0)
-                const __nv_bfloat162 m01 = __hmax2(as_bf162(w[0] & 0x7FFF7FFFu), as_bf162(w[1] & 0x7FFF7FFFu));
-                const __nv_bfloat162 m23 = __hmax2(as_bf162(w[2] & 0x7FFF7FFFu), as_bf162(w[3] & 0x7FFF7FFFu));
-                const uint32_t am2 = bf162_bits(__hmax2(m01, m23));
-                uint32_t am = max(am2 & 0xFFFFu, am2 >> 16);
-                am = max(am, __shfl_xor_sync(0xFFFFFFFFu, am, 1));
-                am = max(am, __shfl_xor_sync(0xFFFFFFFFu, am, 2));
+                for (int i = 1; i < 16; ++i) m2 = __hmax2(m2, as_bf162(w[i] & 0x7FFF7FFFu));
+                const uint32_t am2 = bf162_bits(m2);
+                const uint32_t am = max(am2 & 0xFFFFu, am2 >> 16);
                 // CalculateScale: E8M0 code = biased exponent of amax - 2, floored at 0 (2^(floor(log2 amax) - 2))
                 const int ex = (int)(am >> 7);
-                int code = max(ex - 2, 0);
+                code = max(ex - 2, 0);
                 if (ex == 255) code = 255;
                 // Quantize: x * 2^(127 - code) is exact in fp32, then hardware E2M1 rounding (nearest-even, saturating)
                 const float inv = __uint_as_float((uint32_t)(254 - min(code, 253)) << 23);
-                uint32_t packed = 0;
+                uint32_t q[4];
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
-                    const float lo = __uint_as_float(w[i] << 16) * inv;
-                    const float hi = __uint_as_float(w[i] & 0xFFFF0000u) * inv;
-                    packed |= (e2m1x2(lo, hi) & 0xFFu) << (8 * i);
+                    float f[8];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        f[2 * j] = __uint_as_float(w[4 * i + j] << 16) * inv;
+                        f[2 * j + 1] = __uint_as_float(w[4 * i + j] & 0xFFFF0000u) * inv;
+                    }
+                    q[i] = e2m1x8(f[0], f[1], f[2], f[3], f[4], f[5], f[6], f[7]);
                 }
-                if (live)
-                    *reinterpret_cast<uint32_t*>(xq + (int64_t)r * (K / 2) + cb * (QE_COLS / 2) + cchunk * 4) = packed;
-                if (sub == 0) sfb[(rl & 31) * 16 + (rl >> 5) * 4 + gi] = (uint8_t)code;
+                *reinterpret_cast<uint4*>(xq + (int64_t)r * (K / 2) + cb * (QE_COLS / 2) + gi * 16) =
+                    make_uint4(q[0], q[1], q[2], q[3]);
             }
+            s_sf[parity * 512 + (grow & 31) * 16 + (grow >> 5) * 4 + gi] = (uint8_t)code;
 
             // zero the pad columns of xo once per row tile
             if (cb == 0 && Kop > Ko) {
                 const int npad = Kop - Ko;
                 for (int i = tid; i < QE_ROWS * npad; i += QE_CONSUMERS) {
-                    const int r = row0 + i / npad;
-                    if (r < row_end) xo[(int64_t)r * Kop + Ko + i % npad] = 0;
+                    const int rr = row0 + i / npad;
+                    if (rr < row_end) xo[(int64_t)rr * Kop + Ko + i % npad] = 0;
                 }
             }
-
-            // all 256 consumers have written their scale bytes of this tile
-            asm volatile("bar.sync 1, %0;" ::"n"(QE_CONSUMERS) : "memory");
-            if (tid < 32) {
-                const int64_t blk = (int64_t)(sf_row0 / 128) * (K / 128) + cb;
-                *reinterpret_cast<uint4*>(sf + blk * 512 + tid * 16) = *reinterpret_cast<const uint4*>(sfb + tid * 16);
-            }
-            parity ^= 1;  // the other staging block is free: its readers passed the previous barrier
+            prev_sf_blk = (int64_t)(sf_row0 / 128) * (K / 128) + cb;
+            parity ^= 1;
+            if (++cb == ncb) { cb = 0; ++rt; }
         }
+        // scale block of the last tile
+        asm volatile("bar.sync 1, %0;" ::"n"(QE_CONSUMERS) : "memory");
+        if (prev_sf_blk >= 0 && tid < 32)
+            *reinterpret_cast<uint4*>(sf + prev_sf_blk * 512 + tid * 16) =
+                *reinterpret_cast<const uint4*>(s_sf + (parity ^ 1) * 512 + tid * 16);
     }
 }
 
