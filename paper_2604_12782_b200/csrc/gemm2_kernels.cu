@@ -121,6 +121,8 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_pair_kernel(const __grid_cons
     cluster_sync_all();
     tc_fence_after();
     const uint32_t tmem_base = __shfl_sync(0xFFFFFFFFu, *tmem_slot, 0);
+    grid_launch_dependents();
+    grid_dependency_wait();   // operands come from the kernel before this one
 
     const int N = args.N, K = args.K;
     const int num_m = (args.M + 2 * BM - 1) / (2 * BM);
@@ -358,13 +360,15 @@ static cudaError_t launch_cfg(const GemmArgs& a, cudaStream_t st) {
     cfg.blockDim = dim3(THREADS);
     cfg.dynamicSmemBytes = C::SMEM_BYTES;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     // The kernel is persistent with static striping of tiles over pairs, so every pair must be
     // resident at once: ask how many 2-CTA clusters of this footprint the device can hold.
     static int max_pairs = 0;

@@ -140,6 +140,8 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = __shfl_sync(0xFFFFFFFFu, *tmem_slot, 0);
+    grid_launch_dependents();
+    grid_dependency_wait();   // operands (and the grouped schedule) come from the kernels before this one
 
     const int N = args.N, K = args.K;
     const int num_m = num_row_tiles(args);
@@ -382,8 +384,7 @@ static cudaError_t launch_cfg(const GemmArgs& a, cudaStream_t st) {
         if (total <= 0) return cudaSuccess;
         if (total < grid) grid = total;
     }
-    gemm_kernel<MODE, BN><<<grid, GEMM_THREADS, C::SMEM_BYTES, st>>>(a);
-    return cudaGetLastError();
+    return launch_pdl(gemm_kernel<MODE, BN>, dim3(grid), dim3(GEMM_THREADS), C::SMEM_BYTES, st, a);
 }
 
 cudaError_t launch_gemm_dual(const GemmArgs& a, cudaStream_t st) {

@@ -25,6 +25,14 @@ __device__ __forceinline__ bool elect_one() {
     return pred != 0;
 }
 
+// ------------------------------------------------- programmatic dependent launch
+// Kernels of this library are launched so that a kernel's prologue (barrier set-up, TMEM
+// allocation, descriptor prefetch) may overlap the tail of the kernel before it on the stream.
+// grid_dependency_wait() returns once every earlier kernel has completed and its writes are
+// visible; it is called before the first global read or write of data another kernel touches.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ------------------------------------------------------------------ mbarrier
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));

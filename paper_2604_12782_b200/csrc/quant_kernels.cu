@@ -96,6 +96,8 @@ quant_extract_kernel(const __grid_constant__ CUtensorMap tm_x, int M, int K,
         prefetch_tmap(&tm_x);
     }
     __syncthreads();
+    grid_launch_dependents();
+    grid_dependency_wait();   // X may come from, and the outputs may still be read by, earlier kernels
 
     const int ncb = K / QE_COLS;  // 128-channel blocks per row
     const int nrt = sched ? sched[0] : (M + QE_ROWS - 1) / QE_ROWS;
@@ -246,6 +248,8 @@ __global__ void __launch_bounds__(F8_THREADS)
 fp8_quant_kernel(const uint16_t* __restrict__ X, int64_t ldx, int M, int K, uint8_t* __restrict__ x8,
                  float* __restrict__ sx) {
     __shared__ float s_red[F8_THREADS / 32];
+    grid_launch_dependents();
+    grid_dependency_wait();
     const int r = blockIdx.x;
     const uint16_t* xrow = X + (int64_t)r * ldx;
     const int nch = K / 8;  // 16-byte chunks in the row
@@ -310,6 +314,8 @@ constexpr int F8W_MAXCH = 8;
 __global__ void __launch_bounds__(256)
 fp8_quant_rows_kernel(const uint16_t* __restrict__ X, int64_t ldx, int M, int K, uint8_t* __restrict__ x8,
                       float* __restrict__ sx) {
+    grid_launch_dependents();
+    grid_dependency_wait();
     const int lane = threadIdx.x & 31;
     const int r = blockIdx.x * 8 + (threadIdx.x >> 5);
     if (r >= M) return;
@@ -357,6 +363,8 @@ fp8_quant_rows_kernel(const uint16_t* __restrict__ X, int64_t ldx, int M, int K,
 __global__ void build_sched_kernel(const int32_t* __restrict__ off, int E, int32_t* __restrict__ sched,
                                    int max_tiles) {
     __shared__ int s_tiles[1024];
+    grid_launch_dependents();
+    grid_dependency_wait();
     const int tid = threadIdx.x;
     // serial prefix by one thread: E is small (hundreds) and this runs once per call
     if (tid == 0) {
@@ -397,27 +405,23 @@ cudaError_t launch_quant_extract(const CUtensorMap& tm_x, int M, int K, const ui
         configured = true;
     }
     const int grid = tiles < QE_CTAS_PER_SM * num_sms ? tiles : QE_CTAS_PER_SM * num_sms;
-    quant_extract_kernel<<<grid, QE_THREADS, QE_SMEM, st>>>(tm_x, M, K, mask, prefix, idx_o, static_cast<uint8_t*>(xq),
-                                                            static_cast<uint8_t*>(sf), static_cast<uint16_t*>(xo),
-                                                            Ko, Kop, sched, max_tiles);
-    return cudaGetLastError();
+    return launch_pdl(quant_extract_kernel, dim3(grid), dim3(QE_THREADS), QE_SMEM, st, tm_x, M, K, mask, prefix, idx_o,
+                      static_cast<uint8_t*>(xq), static_cast<uint8_t*>(sf), static_cast<uint16_t*>(xo), Ko, Kop, sched,
+                      max_tiles);
 }
 
 cudaError_t launch_fp8_quant(const void* X, int64_t ldx, int M, int K, void* x8, void* sx, cudaStream_t st) {
     if (M <= 0) return cudaSuccess;
     if (K <= F8W_MAXCH * 32 * 8) {
-        fp8_quant_rows_kernel<<<(M + 7) / 8, 256, 0, st>>>(static_cast<const uint16_t*>(X), ldx, M, K,
-                                                           static_cast<uint8_t*>(x8), static_cast<float*>(sx));
-        return cudaGetLastError();
+        return launch_pdl(fp8_quant_rows_kernel, dim3((M + 7) / 8), dim3(256), 0, st, static_cast<const uint16_t*>(X), ldx,
+                          M, K, static_cast<uint8_t*>(x8), static_cast<float*>(sx));
     }
-    fp8_quant_kernel<<<M, F8_THREADS, 0, st>>>(static_cast<const uint16_t*>(X), ldx, M, K,
-                                               static_cast<uint8_t*>(x8), static_cast<float*>(sx));
-    return cudaGetLastError();
+    return launch_pdl(fp8_quant_kernel, dim3(M), dim3(F8_THREADS), 0, st, static_cast<const uint16_t*>(X), ldx, M, K,
+                      static_cast<uint8_t*>(x8), static_cast<float*>(sx));
 }
 
 cudaError_t launch_build_sched(const int32_t* off, int E, int32_t* sched, int max_tiles, cudaStream_t st) {
-    build_sched_kernel<<<1, 256, 0, st>>>(off, E, sched, max_tiles);
-    return cudaGetLastError();
+    return launch_pdl(build_sched_kernel, dim3(1), dim3(256), 0, st, off, E, sched, max_tiles);
 }
 
 }  // namespace osc
