@@ -7,8 +7,12 @@
 // 16 KB + BN x 128 B, which is what bounds the single-CTA kernel (L2 -> shared-memory feed).
 // No cluster-multicast loads are used: every CTA fetches its own operands.
 //
-// Roles per CTA: warp 0 TMA producer, warp 1 MMA issuer (only in the leader CTA, rank 0) and
-// TMEM owner, warps 2-9 epilogue.  Barriers:
+// Roles per CTA: per issue lane one TMA producer warp and one MMA issuer warp (the latter active only
+// in the leader CTA, rank 0; warp 1 also owns TMEM), then eight epilogue warps.  With two accumulators
+// (BN = 192) there are TWO issue lanes: lane L owns half of the shared-memory ring, accumulator L and
+// scale buffer L, and works on every other tile of the pair.  One elected thread issues all tcgen05
+// instructions of a tile, and its per-stage bookkeeping (barrier wait, commit, loop) leaves the tensor
+// pipe idle ~60 ns per stage; with two lanes the other lane's MMAs fill those gaps.  Barriers:
 //   full[s]   leader's only: one arrive.expect_tx by the leader's producer for the bytes of BOTH
 //             CTAs; the peer's loads credit the leader's barrier (cta_group::2 loads).
 //   empty[s]  one per CTA, released for both CTAs by one multicast tcgen05.commit of the leader.
@@ -31,7 +35,6 @@ constexpr int BM = 128;        // rows per CTA; the pair covers 256
 constexpr int ROW_BYTES = 128;
 constexpr int A_BYTES = BM * ROW_BYTES;
 constexpr int EPI_WARPS = 8;     // two per TMEM lane quarter, each draining every other 64-column slice
-constexpr int THREADS = 64 + 32 * EPI_WARPS;
 constexpr int TMEM_COLS = 512;
 constexpr int BAND = 4;        // 256-row tiles per scheduling band
 constexpr int EPI_TILE_BYTES = 32 * 128;            // staging tile: 32 rows x 64 bf16 columns
@@ -45,9 +48,15 @@ struct Cfg {
     static constexpr int SFA_BYTES = (MODE == MODE_OSC) ? 1024 : 0;
     static constexpr int SFB_BYTES = (MODE == MODE_OSC) ? SFB_ATOMS * 1024 : 0;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + SFA_BYTES + SFB_BYTES;
-    static constexpr int EPI_WARP_BYTES = (BN / 64) * EPI_TILE_BYTES;  // one warp's 32 x BN output rows
-    static constexpr int EPI_BYTES = 4 * EPI_WARP_BYTES;
-    static constexpr int STAGES = (224 * 1024 - EPI_BYTES) / STAGE_BYTES;
+    static constexpr int LANES = ACC_STAGES;            // issue lanes = accumulators
+    static constexpr int THREADS = 32 * (2 * LANES + EPI_WARPS);
+    static constexpr int EPI_FIRST_WARP = 2 * LANES;
+    // staging tiles per epilogue warp: 2 = the warp's whole share of a tile (accumulator released before any
+    // store is issued); 1 = one slice at a time (smaller footprint, used when two rings share the memory)
+    static constexpr int EPI_TPW = (LANES == 2) ? 1 : 2;
+    static constexpr int EPI_BYTES = EPI_WARPS * EPI_TPW * EPI_TILE_BYTES;
+    static constexpr int STAGES = ((224 * 1024 - EPI_BYTES) / STAGE_BYTES) / LANES * LANES;
+    static constexpr int SPL = STAGES / LANES;          // ring stages per lane
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/ + EPI_BYTES;
     static constexpr int TM_SFA = ACC_STAGES * BN;
     static constexpr int TM_SFB = TM_SFA + 8;
@@ -58,13 +67,15 @@ struct Cfg {
     static_assert(B_BYTES % 1024 == 0, "weight half-tile must keep 1024-byte alignment");
     static_assert(TM_SFA + 2 * TM_SF_STRIDE <= TMEM_COLS, "TMEM budget");
     static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
+    static_assert(SPL >= 3, "ring too shallow");
+    static_assert((BN / 64 + 1) / 2 <= 2, "an epilogue warp drains at most two slices of a tile");
     // Tiles must start on an even 32-row scale column: a 224-wide tile (odd column offsets into the
     // weight-scale region of TMEM) raised "misaligned address" on the block-scaled MMA.
     static_assert(BN % 64 == 0 && BN <= 256, "tile width");
 };
 
 template <int MODE, int BN>
-__global__ void __launch_bounds__(THREADS, 1) gemm_pair_kernel(const __grid_constant__ GemmArgs args) {
+__global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(const __grid_constant__ GemmArgs args) {
     using C = Cfg<MODE, BN>;
     constexpr int STAGES = C::STAGES;
     constexpr int ACC = C::ACC_STAGES;
@@ -145,24 +156,29 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_pair_kernel(const __grid_cons
         n0 = (rem / h) * BN;
     };
 
-    if (warp == 0) {
-        // ------------------------------------------------------------ TMA producer (both CTAs)
-        {
-            int s = 0;
-            uint32_t ph = 0;
-            const uint32_t full0 = map_to_cta(smem_u32(&full_bar[0]), 0);  // the leader's full barriers
-            for (int t = pair_id; t < total; t += num_pairs) {
-                int row0, n0;
-                tile_rc(t, row0, n0);
-                const int arow = row0 + (int)rank * BM;            // my 128 activation rows
-                const int brow = n0 + (int)rank * (BN / 2);        // my half of the weight rows
-                for (int kb = 0; kb < nkb; ++kb) {
-                    if (!wait_bounded(&empty_bar[s], ph ^ 1u, abort_flag, 11)) goto done;
-                    const uint32_t st = smem_u32(smem + s * C::STAGE_BYTES);
-                    const uint32_t fb = full0 + (uint32_t)s * 8u;
-                    if (elect_one()) {
+    constexpr int LANES = C::LANES;
+    constexpr int SPL = C::SPL;
+    if (warp < 2 * LANES && (warp & 1) == 0) {
+        // ------------------------------------------- TMA producer of issue lane L (both CTAs)
+        const int L = warp >> 1;
+        int s = 0;
+        uint32_t ph = 0;
+        uint64_t* fullL = full_bar + L * SPL;
+        uint64_t* emptyL = empty_bar + L * SPL;
+        uint8_t* ring = smem + L * SPL * C::STAGE_BYTES;
+        const uint32_t full0 = map_to_cta(smem_u32(fullL), 0);  // the leader's full barriers of this lane
+        for (int t = pair_id + L * num_pairs; t < total; t += LANES * num_pairs) {
+            int row0, n0;
+            tile_rc(t, row0, n0);
+            const int arow = row0 + (int)rank * BM;            // my 128 activation rows
+            const int brow = n0 + (int)rank * (BN / 2);        // my half of the weight rows
+            for (int kb = 0; kb < nkb; ++kb) {
+                if (!wait_bounded(&emptyL[s], ph ^ 1u, abort_flag, 11)) goto done;
+                const uint32_t st = smem_u32(ring + s * C::STAGE_BYTES);
+                const uint32_t fb = full0 + (uint32_t)s * 8u;
+                if (elect_one()) {
                     if (kb < nkb_a) {
-                        if (rank == 0) mbar_arrive_expect_tx(&full_bar[s], MODE == MODE_OSC ? C::TX_A : C::TX_B);
+                        if (rank == 0) mbar_arrive_expect_tx(&fullL[s], MODE == MODE_OSC ? C::TX_A : C::TX_B);
                         tma_load_2d_pair(st, &args.tm_a, fb, kb * ROW_BYTES, arow);
                         tma_load_2d_pair(st + A_BYTES, &args.tm_b, fb, kb * ROW_BYTES, brow);
                         if (MODE == MODE_OSC) {
@@ -178,29 +194,31 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_pair_kernel(const __grid_cons
                         }
                     } else {
                         const int kk = kb - nkb_a;
-                        if (rank == 0) mbar_arrive_expect_tx(&full_bar[s], C::TX_B);
+                        if (rank == 0) mbar_arrive_expect_tx(&fullL[s], C::TX_B);
                         tma_load_2d_pair(st, &args.tm_ao, fb, kk * 64, arow);
                         tma_load_2d_pair(st + A_BYTES, &args.tm_bo, fb, kk * 64, brow);
                     }
-                    }
-                    __syncwarp();
-                    if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
+                __syncwarp();
+                if (++s == SPL) { s = 0; ph ^= 1u; }
             }
         }
-    } else if (warp == 1) {
-        // ------------------------------------------------ MMA issuer (leader CTA only, one thread)
+    } else if (warp < 2 * LANES) {
+        // ---------------------- MMA issuer of issue lane L (leader CTA only, one elected lane)
         if (rank == 0) {
+            const int L = warp >> 1;
             int s = 0;
             uint32_t ph = 0;
-            int acc = 0;
-            uint32_t acc_ph = 0;
+            uint32_t acc_ph = 0;   // parity of this lane's accumulator barrier (single lane: toggles per tile)
+            int acc = (LANES == 2) ? L : 0;
+            uint64_t* fullL = full_bar + L * SPL;
+            uint64_t* emptyL = empty_bar + L * SPL;
             constexpr uint32_t IDESC_A = (MODE == MODE_OSC) ? idesc_mxf4(2 * BM, BN) : idesc_e4m3(2 * BM, BN);
             constexpr uint32_t IDESC_B = idesc_bf16(2 * BM, BN);
             const uint64_t desc_hi = smem_desc_sw128(0);  // everything but the start address
             const uint64_t sf_hi = smem_desc_sf(0);
-            const uint32_t smem0 = smem_u32(smem);
-            for (int t = pair_id; t < total; t += num_pairs) {
+            const uint32_t ring0 = smem_u32(smem + L * SPL * C::STAGE_BYTES);
+            for (int t = pair_id + L * num_pairs; t < total; t += LANES * num_pairs) {
                 int row0, n0;
                 tile_rc(t, row0, n0);
                 if (!wait_bounded_cluster(&tempty_bar[acc], acc_ph ^ 1u, abort_flag, 12)) goto done;
@@ -208,69 +226,72 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_pair_kernel(const __grid_cons
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
                 const uint32_t sfb_tm = tmem_base + C::TM_SFB + (uint32_t)((n0 % 128) / 32);
                 for (int kb = 0; kb < nkb; ++kb) {
-                    if (!wait_bounded(&full_bar[s], ph, abort_flag, 13)) goto done;
-                    const uint32_t sbase = smem0 + s * C::STAGE_BYTES;
+                    if (!wait_bounded(&fullL[s], ph, abort_flag, 13)) goto done;
+                    const uint32_t sbase = ring0 + s * C::STAGE_BYTES;
                     const uint64_t adesc = desc_hi | (uint64_t)(sbase >> 4);
                     const uint64_t bdesc = desc_hi | (uint64_t)((sbase + A_BYTES) >> 4);
                     if (elect_one()) {
-                    if (MODE == MODE_OSC && kb < nkb_a) {
-                        const int ka = min(2, katoms_total - 2 * kb);
-                        const uint64_t sfa_d = sf_hi | (uint64_t)((sbase + A_BYTES + C::B_BYTES) >> 4);
-                        const uint64_t sfb_d = sf_hi | (uint64_t)((sbase + A_BYTES + C::B_BYTES + C::SFA_BYTES) >> 4);
-                        // two scale buffers in TMEM alternate, so this stage's copies do not wait for the
-                        // previous stage's MMAs to finish reading theirs
-                        const uint32_t sfo = (uint32_t)(kb & 1) * C::TM_SF_STRIDE;
+                        if (MODE == MODE_OSC && kb < nkb_a) {
+                            const int ka = min(2, katoms_total - 2 * kb);
+                            const uint64_t sfa_d = sf_hi | (uint64_t)((sbase + A_BYTES + C::B_BYTES) >> 4);
+                            const uint64_t sfb_d = sf_hi | (uint64_t)((sbase + A_BYTES + C::B_BYTES + C::SFA_BYTES) >> 4);
+                            // two scale buffers in TMEM: one per issue lane, or alternating by stage with a single
+                            // lane (so a stage's copies never wait for another stage's MMAs still reading theirs)
+                            const uint32_t sfo = (uint32_t)((LANES == 2) ? L : (kb & 1)) * C::TM_SF_STRIDE;
 #pragma unroll
-                        for (int a = 0; a < 2; ++a) {
-                            if (a < ka) {
-                                tc_copy_sf_pair(tmem_base + sfo + C::TM_SFA + a * 4, sfa_d + (uint64_t)(a * 32));
+                            for (int a = 0; a < 2; ++a) {
+                                if (a < ka) {
+                                    tc_copy_sf_pair(tmem_base + sfo + C::TM_SFA + a * 4, sfa_d + (uint64_t)(a * 32));
 #pragma unroll
-                                for (int j = 0; j < C::SFB_ATOMS; ++j)
-                                    tc_copy_sf_pair(tmem_base + sfo + C::TM_SFB + a * (C::SFB_ATOMS * 4) + j * 4,
-                                                    sfb_d + (uint64_t)(j * 64 + a * 32));
+                                    for (int j = 0; j < C::SFB_ATOMS; ++j)
+                                        tc_copy_sf_pair(tmem_base + sfo + C::TM_SFB + a * (C::SFB_ATOMS * 4) + j * 4,
+                                                        sfb_d + (uint64_t)(j * 64 + a * 32));
+                                }
                             }
-                        }
 #pragma unroll
-                        for (int k = 0; k < 4; ++k) {
-                            if (k < 2 * ka) {
-                                constexpr uint32_t SFID[2] = {idesc_sf_ids(0, 0), idesc_sf_ids(2, 2)};
-                                mma_mxf4_pair(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC_A | SFID[k & 1],
-                                              tmem_base + sfo + C::TM_SFA + (k >> 1) * 4,
-                                              sfb_tm + sfo + (k >> 1) * (C::SFB_ATOMS * 4), (kb | k) ? 1u : 0u);
+                            for (int k = 0; k < 4; ++k) {
+                                if (k < 2 * ka) {
+                                    constexpr uint32_t SFID[2] = {idesc_sf_ids(0, 0), idesc_sf_ids(2, 2)};
+                                    mma_mxf4_pair(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC_A | SFID[k & 1],
+                                                  tmem_base + sfo + C::TM_SFA + (k >> 1) * 4,
+                                                  sfb_tm + sfo + (k >> 1) * (C::SFB_ATOMS * 4), (kb | k) ? 1u : 0u);
+                                }
                             }
+                        } else if (MODE == MODE_OSC) {
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) mma_f16_pair(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC_B, 1u);
+                        } else {
+#pragma unroll
+                            for (int k = 0; k < 4; ++k)
+                                mma_f8_pair(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC_A, (kb | k) ? 1u : 0u);
                         }
-                    } else if (MODE == MODE_OSC) {
-#pragma unroll
-                        for (int k = 0; k < 4; ++k) mma_f16_pair(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC_B, 1u);
-                    } else {
-#pragma unroll
-                        for (int k = 0; k < 4; ++k)
-                            mma_f8_pair(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC_A, (kb | k) ? 1u : 0u);
-                    }
-                    tc_commit_pair(&empty_bar[s], 3);  // frees the stage in both CTAs
+                        tc_commit_pair(&emptyL[s], 3);  // frees the stage in both CTAs
                     }
                     __syncwarp();
-                    if (++s == STAGES) { s = 0; ph ^= 1u; }
+                    if (++s == SPL) { s = 0; ph ^= 1u; }
                 }
                 if (elect_one()) tc_commit_pair(&tfull_bar[acc], 3);    // accumulator ready in both CTAs
                 __syncwarp();
-                if (++acc == ACC) { acc = 0; acc_ph ^= 1u; }
+                acc_ph ^= 1u;  // one use of this accumulator barrier per tile of the lane (both layouts: with a
+                               // single lane and one accumulator, or two lanes with one accumulator each)
+                if (LANES == 1 && ACC == 2) { acc ^= 1; if (acc) acc_ph ^= 1u; }
             }
         }
     } else {
         // ---------------------------------------------------------------- epilogue (both CTAs)
-        // Each warp owns 32 accumulator rows.  Drain: per 64-column slice TMEM -> registers -> bf16
-        // -> a swizzled 32 x 128-byte staging tile in shared memory (one tile per slice, so nothing
-        // waits inside the drain).  As soon as the last slice has left TMEM the accumulator is handed
-        // back to the MMA warp; only then are the TMA stores of the staged tile issued, and they
-        // drain to global memory while the next tile's MMAs run.  (Per-thread global stores, 32 rows
-        // x 16 bytes per instruction, kept the memory pipe busy and stalled the next tile's MMA issue.)
-        const int q = warp & 3;             // TMEM lane quarter this warp may read
-        const int half = (warp - 2) >> 2;   // which of the two warps of that quarter: slices c = half, half + 2, ...
+        // Two warps per TMEM lane quarter (32 accumulator rows), each draining every other 64-column
+        // slice: TMEM -> registers -> bf16 -> a swizzled 32 x 128-byte staging tile -> one TMA store.
+        // With two staging tiles per warp the accumulator is handed back before any store is issued;
+        // with one, stores go out slice by slice.  Either way they drain to global memory while the
+        // next tile's MMAs run.  (Per-thread global stores, 32 rows x 16 bytes per instruction, kept
+        // the memory pipe busy and stalled the next tile's MMA issue.)
+        const int q = warp & 3;                          // TMEM lane quarter this warp may read
+        const int half = (warp - C::EPI_FIRST_WARP) >> 2;  // which of the two warps of that quarter
+        constexpr int TPW = C::EPI_TPW;
         int acc = 0;
         uint32_t acc_ph = 0;
         const uint32_t tempty0 = map_to_cta(smem_u32(&tempty_bar[0]), 0);
-        uint8_t* stage_buf = smem + STAGES * C::STAGE_BYTES + q * C::EPI_WARP_BYTES;
+        uint8_t* stage_buf = smem + STAGES * C::STAGE_BYTES + (half * 4 + q) * (TPW * EPI_TILE_BYTES);
         for (int t = pair_id; t < total; t += num_pairs) {
             int row0, n0;
             tile_rc(t, row0, n0);
@@ -280,18 +301,25 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_pair_kernel(const __grid_cons
             const int row = wrow0 + lane;
             float sxr = 1.0f;
             if (MODE == MODE_FP8 && row < args.M) sxr = args.sx[row];
-            // the stores of the previous tile must be done reading the staging tiles
-            if (lane == 0) tma_store_wait_read<0>();
-            __syncwarp();
+            if (TPW == 2) {
+                // the stores of the previous tile must be done reading the staging tiles
+                if (lane == 0) tma_store_wait_read<0>();
+                __syncwarp();
+            }
+            int ord = 0;
 #pragma unroll 1
-            for (int c = half; c < BN / 64; c += EPI_WARPS / 4) {
+            for (int c = half; c < BN / 64; c += EPI_WARPS / 4, ++ord) {
                 uint32_t r0[32], r1[32];
                 const uint32_t tcol = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + c * 64);
                 tmem_ld_32x32(tcol, r0);
                 tmem_ld_32x32(tcol + 32, r1);
                 tmem_ld_wait();
                 const int col = n0 + c * 64;
-                uint8_t* buf = stage_buf + c * EPI_TILE_BYTES;
+                uint8_t* buf = stage_buf + (TPW == 2 ? ord : 0) * EPI_TILE_BYTES;
+                if (TPW == 1) {
+                    if (lane == 0) tma_store_wait_read<0>();  // the one staging tile must be free again
+                    __syncwarp();
+                }
                 if (col < N) {
 #pragma unroll
                     for (int j = 0; j < 8; ++j) {  // 8 chunks of 16 bytes = 8 columns each
@@ -313,17 +341,28 @@ __global__ void __launch_bounds__(THREADS, 1) gemm_pair_kernel(const __grid_cons
                         *reinterpret_cast<uint4*>(buf + lane * 128 + ((j ^ (lane & 7)) << 4)) =
                             make_uint4(o[0], o[1], o[2], o[3]);
                     }
+                    if (TPW == 1) {
+                        fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0) {
+                            tma_store_2d(&args.tm_y, buf, col, wrow0);
+                            tma_store_commit();
+                        }
+                    }
                 }
             }
-            // accumulator drained: hand it back before the stores
+            // accumulator drained: hand it back (before the stores when the whole share is staged)
             tc_fence_before();
-            fence_proxy_async_smem();
+            if (TPW == 2) fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) {
                 mbar_arrive_cluster(tempty0 + (uint32_t)acc * 8u);
-                for (int c = half; c < BN / 64; c += EPI_WARPS / 4)
-                    if (n0 + c * 64 < N) tma_store_2d(&args.tm_y, stage_buf + c * EPI_TILE_BYTES, n0 + c * 64, wrow0);
-                tma_store_commit();
+                if (TPW == 2) {
+                    int o2 = 0;
+                    for (int c = half; c < BN / 64; c += EPI_WARPS / 4, ++o2)
+                        if (n0 + c * 64 < N) tma_store_2d(&args.tm_y, stage_buf + o2 * EPI_TILE_BYTES, n0 + c * 64, wrow0);
+                    tma_store_commit();
+                }
             }
             __syncwarp();
             if (++acc == ACC) { acc = 0; acc_ph ^= 1u; }
@@ -357,7 +396,7 @@ static cudaError_t launch_cfg(const GemmArgs& a, cudaStream_t st) {
     const int total = ((a.M + 2 * BM - 1) / (2 * BM)) * ((a.N + BN - 1) / BN);
     if (total <= 0) return cudaSuccess;
     cudaLaunchConfig_t cfg = {};
-    cfg.blockDim = dim3(THREADS);
+    cfg.blockDim = dim3(C::THREADS);
     cfg.dynamicSmemBytes = C::SMEM_BYTES;
     cfg.stream = st;
     cudaLaunchAttribute attr[2];
