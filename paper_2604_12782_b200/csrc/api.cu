@@ -164,6 +164,12 @@ static osc_status check_nk(int E, int N, int K) {
     return OSC_OK;
 }
 static size_t sf_bytes(int64_t rows, int K) { return (size_t)((rows + 127) / 128) * (K / 128) * 512; }
+// meta = [mask | prefix | idx_o, padded to 1 KB][per-tile copy of the weight scales for 240-row tiles (dense only)]
+constexpr int kTiledBN = 240;
+static size_t meta_table_bytes(int K, int Ko) { return ((size_t)(K / 32) * 8 + (size_t)Ko * 4 + 16 + 1023) & ~size_t(1023); }
+static size_t tiled_sf_bytes(int N, int K) {
+    return (size_t)((N + kTiledBN - 1) / kTiledBN) * ((kTiledBN + 127) / 128) * (K / 128) * 512;
+}
 
 }  // namespace osc
 
@@ -179,7 +185,8 @@ struct osc_weights {
     const int32_t* idx_o;
     int num_sms, block_n;
     CUtensorMap tm_b, tm_bo;          // single-CTA kernel: weight tiles of block_n rows
-    CUtensorMap tm_b2[2], tm_bo2[2], tm_sfw;  // CTA-pair kernel: half tiles for 192- and 256-wide tiles, scale blocks
+    CUtensorMap tm_b2[3], tm_bo2[3];  // CTA-pair kernel: half tiles for 192-, 256- and 240-wide tiles
+    CUtensorMap tm_sfw, tm_sfw_tiled;  // scale blocks: standard layout / per-tile copy for 240-wide tiles
 };
 struct osc_fp8_weights {
     int E, N, K;
@@ -234,7 +241,7 @@ osc_status osc_weight_sizes(int E, int N, int K, const int8_t* lut, int lut_c, o
     out->wq_bytes = (size_t)E * N * (K / 2);
     out->sfw_bytes = (size_t)E * sf_bytes(N, K);
     out->wo_bytes = (size_t)E * N * t.Kop * 2;
-    out->meta_bytes = align256((size_t)(K / 32) * 8 + (size_t)t.Ko * 4 + 16);
+    out->meta_bytes = meta_table_bytes(K, t.Ko) + (E == 1 ? tiled_sf_bytes(N, K) : 0);
     return OSC_OK;
 }
 
@@ -289,13 +296,19 @@ static osc_status prepare_impl(const void* W, int E, int N, int K, int64_t ldw, 
     osc_status s = make_tmap(&w->tm_b, wq, false, (uint64_t)E * N, K / 2, K / 2, w->block_n);
     if (s == OSC_OK && t.Kop > 0)
         s = make_tmap(&w->tm_bo, wo, true, (uint64_t)E * N, (uint64_t)t.Kop * 2, (uint64_t)t.Kop * 2, w->block_n);
-    for (int v = 0; v < 2 && s == OSC_OK && !grouped; ++v) {
-        const int half = (v == 0 ? 192 : 256) / 2;
+    for (int v = 0; v < 3 && s == OSC_OK && !grouped; ++v) {
+        const int half = (v == 0 ? 192 : v == 1 ? 256 : kTiledBN) / 2;
         s = make_tmap(&w->tm_b2[v], wq, false, (uint64_t)N, K / 2, K / 2, half);
         if (s == OSC_OK && t.Kop > 0)
             s = make_tmap(&w->tm_bo2[v], wo, true, (uint64_t)N, (uint64_t)t.Kop * 2, (uint64_t)t.Kop * 2, half);
     }
     if (s == OSC_OK && !grouped) s = make_tmap_sf(&w->tm_sfw, sfw, (uint64_t)sfw_e / 512);
+    if (s == OSC_OK && !grouped) {
+        uint8_t* tiled = m8 + meta_table_bytes(K, t.Ko);
+        e = launch_retile_sf(static_cast<const uint8_t*>(sfw), tiled, N, K, kTiledBN, st);
+        if (e != cudaSuccess) { delete w; return cuda_fail(e, "retile_sf_kernel"); }
+        s = make_tmap_sf(&w->tm_sfw_tiled, tiled, (uint64_t)tiled_sf_bytes(N, K) / 512);
+    }
     if (s != OSC_OK) { delete w; return s; }
     *out = w;
     return OSC_OK;
@@ -382,10 +395,11 @@ static osc_status gemm_impl(const osc_weights* w, const void* xq, const void* sf
     a.sched = sched; a.max_tiles = max_tiles; a.num_sms = w->num_sms;
     cudaError_t e;
     if (use_pair_kernel(w->grouped, M)) {
-        const int bn = gemm_pair_block_n(M, w->N, (w->K + 255) / 256 + w->Kop / 64, w->num_sms);
-        a.tm_b = w->tm_b2[bn == 256];
-        a.tm_bo = w->tm_bo2[bn == 256];
-        a.tm_sfw = w->tm_sfw;
+        const int bn = gemm_pair_block_n(false, M, w->N, (w->K + 255) / 256 + w->Kop / 64, w->num_sms);
+        const int v = bn == 192 ? 0 : bn == 256 ? 1 : 2;
+        a.tm_b = w->tm_b2[v];
+        a.tm_bo = w->tm_bo2[v];
+        a.tm_sfw = (bn == kTiledBN) ? w->tm_sfw_tiled : w->tm_sfw;
         if (osc_status s = make_tmap_sf(&a.tm_sfa, sfa, (uint64_t)((M + 127) / 128) * (w->K / 128))) return s;
         if (osc_status s = make_tmap(&a.tm_y, Y, true, M, (uint64_t)w->N * 2, (uint64_t)ldy * 2, 32)) return s;
         e = launch_gemm_dual_pair(a, bn, st);
@@ -537,7 +551,7 @@ static osc_status fp8_gemm_impl(const osc_fp8_weights* w, const void* x8, const 
     a.sched = sched; a.max_tiles = max_tiles; a.num_sms = w->num_sms;
     cudaError_t e;
     if (use_pair_kernel(w->grouped, M)) {
-        const int bn = gemm_pair_block_n(M, w->N, w->K / 128, w->num_sms);
+        const int bn = gemm_pair_block_n(true, M, w->N, w->K / 128, w->num_sms);
         a.tm_b = w->tm_b2[bn == 256];
         if (osc_status s = make_tmap(&a.tm_y, Y, true, M, (uint64_t)w->N * 2, (uint64_t)ldy * 2, 32)) return s;
         e = launch_gemm_fp8_pair(a, bn, st);

@@ -61,6 +61,7 @@ int gemm_block_n();
 // gemm2_kernels.cu (CTA pairs, dense problems)
 cudaError_t launch_gemm_dual_pair(const GemmArgs& a, int bn, cudaStream_t st);
 cudaError_t launch_gemm_fp8_pair(const GemmArgs& a, int bn, cudaStream_t st);
-int gemm_pair_block_n(int M, int N, int stages, int num_sms);
+int gemm_pair_block_n(bool fp8, int M, int N, int stages, int num_sms);
+cudaError_t launch_retile_sf(const uint8_t* src, uint8_t* dst, int N, int K, int bn, cudaStream_t st);
 
 }  // namespace osc

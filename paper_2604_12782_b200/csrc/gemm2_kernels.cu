@@ -41,37 +41,50 @@ constexpr int EPI_TILE_BYTES = 32 * 128;            // staging tile: 32 rows x 6
 
 template <int MODE, int BN>
 struct Cfg {
-    static constexpr int ACC_STAGES = (2 * BN + 2 * (8 + 2 * 4 * ((BN % 128 == 0) ? BN / 128 : BN / 128 + 2 - (BN % 128 == 64 ? 1 : 0))) <= TMEM_COLS) ? 2 : 1;
-    // 128-row scale blocks a BN-wide tile can touch, given that tiles start at multiples of BN
-    static constexpr int SFB_ATOMS = (BN % 128 == 0) ? BN / 128 : BN / 128 + 2 - (BN % 128 == 64 ? 1 : 0);
+    // Weight scales in TMEM: a tile whose first row is not a multiple of 64 would start at an odd or
+    // fractional 32-row scale column (an odd column offset raised "misaligned address" on the
+    // block-scaled MMA).  Such widths (240) read a per-tile copy of the weight scales, laid out at
+    // weight-preparation time so that every tile starts at column 0 of its own two 128-row blocks.
+    static constexpr bool TILED_SF = (BN % 64) != 0;
+    // 128-row scale blocks a BN-wide tile can touch
+    static constexpr int SFB_ATOMS = TILED_SF ? (BN + 127) / 128 : ((BN % 128 == 0) ? BN / 128 : BN / 128 + 1);
+    static constexpr int SF_COLS = (MODE == MODE_OSC) ? 8 + 2 * SFB_ATOMS * 4 : 0;  // TMEM columns of one stage's scales
+    static constexpr int ACC_STAGES = (2 * BN + SF_COLS <= TMEM_COLS) ? 2 : 1;
+    static constexpr int SF_BUFS = (ACC_STAGES * BN + 2 * SF_COLS <= TMEM_COLS) ? 2 : 1;
     static constexpr int B_BYTES = (BN / 2) * ROW_BYTES;
     static constexpr int SFA_BYTES = (MODE == MODE_OSC) ? 1024 : 0;
     static constexpr int SFB_BYTES = (MODE == MODE_OSC) ? SFB_ATOMS * 1024 : 0;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + SFA_BYTES + SFB_BYTES;
-    static constexpr int LANES = ACC_STAGES;            // issue lanes = accumulators
+    static constexpr int LANES = 1;                      // issue lanes (a second one brought nothing, see above)
     static constexpr int THREADS = 32 * (2 * LANES + EPI_WARPS);
     static constexpr int EPI_FIRST_WARP = 2 * LANES;
+    static constexpr int SLICES = (BN + 63) / 64;        // 64-column output slices of a tile
+    static constexpr int LAST_W = BN - 64 * (SLICES - 1);  // width of the last one (64 or 48)
     // staging tiles per epilogue warp: 2 = the warp's whole share of a tile (accumulator released before any
-    // store is issued); 1 = one slice at a time (smaller footprint, used when two rings share the memory)
-    static constexpr int EPI_TPW = (LANES == 2) ? 1 : 2;
+    // store is issued); 1 = one slice at a time
+    static constexpr int EPI_TPW = 2;
     static constexpr int EPI_BYTES = EPI_WARPS * EPI_TPW * EPI_TILE_BYTES;
     static constexpr int STAGES = ((224 * 1024 - EPI_BYTES) / STAGE_BYTES) / LANES * LANES;
     static constexpr int SPL = STAGES / LANES;          // ring stages per lane
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/ + EPI_BYTES;
-    static constexpr int TM_SFA = ACC_STAGES * BN;
-    static constexpr int TM_SFB = TM_SFA + 8;
-    static constexpr int TM_SF_STRIDE = 8 + 2 * SFB_ATOMS * 4;  // columns of one scale buffer; two buffers alternate
+    // TMEM columns.  Accumulators start at multiples of ACC_STRIDE; a 240-wide tile keeps its second
+    // accumulator at column 256 and tucks the scales into the gaps (activation scales at 240..247,
+    // weight scales at 496..511).
+    static constexpr int ACC_STRIDE = TILED_SF ? 256 : BN;
+    static constexpr int TM_SFA = TILED_SF ? BN : ACC_STAGES * BN;
+    static constexpr int TM_SFB = TILED_SF ? 256 + BN : TM_SFA + 8;
+    static constexpr int TM_SF_STRIDE = SF_COLS;         // columns of one scale buffer (when there are two)
     static constexpr uint32_t TX_A = 2u * (A_BYTES + B_BYTES + SFA_BYTES + SFB_BYTES);  // both CTAs, Path A
     static constexpr uint32_t TX_B = 2u * (A_BYTES + B_BYTES);                          // both CTAs, Path B / FP8
     static_assert(STAGE_BYTES % 1024 == 0, "stage must keep 1024-byte alignment");
     static_assert(B_BYTES % 1024 == 0, "weight half-tile must keep 1024-byte alignment");
-    static_assert(TM_SFA + 2 * TM_SF_STRIDE <= TMEM_COLS, "TMEM budget");
+    static_assert(TILED_SF ? (TM_SFA + 8 <= 256 && TM_SFB + 2 * SFB_ATOMS * 4 <= TMEM_COLS && SF_BUFS == 1)
+                           : (TM_SFA + SF_BUFS * SF_COLS <= TMEM_COLS), "TMEM budget");
     static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
     static_assert(SPL >= 3, "ring too shallow");
-    static_assert((BN / 64 + 1) / 2 <= 2, "an epilogue warp drains at most two slices of a tile");
-    // Tiles must start on an even 32-row scale column: a 224-wide tile (odd column offsets into the
-    // weight-scale region of TMEM) raised "misaligned address" on the block-scaled MMA.
-    static_assert(BN % 64 == 0 && BN <= 256, "tile width");
+    static_assert((SLICES + 1) / 2 <= 2, "an epilogue warp drains at most two slices of a tile");
+    static_assert(BN % 16 == 0 && BN <= 256 && (LAST_W == 64 || LAST_W == 48), "tile width");
+    static_assert(LAST_W == 64 || EPI_TPW == 2, "the narrow last slice is written from a staged tile");
 };
 
 template <int MODE, int BN>
@@ -187,7 +200,7 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
                                              (arow / 128) * katoms_total + 2 * kb);
 #pragma unroll
                             for (int j = 0; j < C::SFB_ATOMS; ++j) {
-                                const int atom = min(n0 / 128 + j, natoms - 1);
+                                const int atom = C::TILED_SF ? (n0 / BN) * C::SFB_ATOMS + j : min(n0 / 128 + j, natoms - 1);
                                 tma_load_2d_pair(st + A_BYTES + C::B_BYTES + C::SFA_BYTES + j * 1024, &args.tm_sfw, fb, 0,
                                                  atom * katoms_total + 2 * kb);
                             }
@@ -209,7 +222,7 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
             const int L = warp >> 1;
             int s = 0;
             uint32_t ph = 0;
-            uint32_t acc_ph = 0;   // parity of this lane's accumulator barrier (single lane: toggles per tile)
+            uint32_t acc_ph = 0;
             int acc = (LANES == 2) ? L : 0;
             uint64_t* fullL = full_bar + L * SPL;
             uint64_t* emptyL = empty_bar + L * SPL;
@@ -223,8 +236,8 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
                 tile_rc(t, row0, n0);
                 if (!wait_bounded_cluster(&tempty_bar[acc], acc_ph ^ 1u, abort_flag, 12)) goto done;
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
-                const uint32_t sfb_tm = tmem_base + C::TM_SFB + (uint32_t)((n0 % 128) / 32);
+                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * C::ACC_STRIDE);
+                const uint32_t sfb_tm = tmem_base + C::TM_SFB + (C::TILED_SF ? 0u : (uint32_t)((n0 % 128) / 32));
                 for (int kb = 0; kb < nkb; ++kb) {
                     if (!wait_bounded(&fullL[s], ph, abort_flag, 13)) goto done;
                     const uint32_t sbase = ring0 + s * C::STAGE_BYTES;
@@ -237,7 +250,7 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
                             const uint64_t sfb_d = sf_hi | (uint64_t)((sbase + A_BYTES + C::B_BYTES + C::SFA_BYTES) >> 4);
                             // two scale buffers in TMEM: one per issue lane, or alternating by stage with a single
                             // lane (so a stage's copies never wait for another stage's MMAs still reading theirs)
-                            const uint32_t sfo = (uint32_t)((LANES == 2) ? L : (kb & 1)) * C::TM_SF_STRIDE;
+                            const uint32_t sfo = (uint32_t)((LANES == 2) ? L : (C::SF_BUFS == 2 ? (kb & 1) : 0)) * C::TM_SF_STRIDE;
 #pragma unroll
                             for (int a = 0; a < 2; ++a) {
                                 if (a < ka) {
@@ -272,9 +285,12 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
                 }
                 if (elect_one()) tc_commit_pair(&tfull_bar[acc], 3);    // accumulator ready in both CTAs
                 __syncwarp();
-                acc_ph ^= 1u;  // one use of this accumulator barrier per tile of the lane (both layouts: with a
-                               // single lane and one accumulator, or two lanes with one accumulator each)
-                if (LANES == 1 && ACC == 2) { acc ^= 1; if (acc) acc_ph ^= 1u; }
+                if (LANES == 2) {
+                    acc_ph ^= 1u;                                  // the lane keeps its own accumulator
+                } else if (++acc == ACC) {
+                    acc = 0;
+                    acc_ph ^= 1u;
+                }
             }
         }
     } else {
@@ -308,11 +324,12 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
             }
             int ord = 0;
 #pragma unroll 1
-            for (int c = half; c < BN / 64; c += EPI_WARPS / 4, ++ord) {
+            for (int c = half; c < C::SLICES; c += EPI_WARPS / 4, ++ord) {
                 uint32_t r0[32], r1[32];
-                const uint32_t tcol = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + c * 64);
+                const uint32_t tcol = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * C::ACC_STRIDE + c * 64);
+                const bool narrow = (C::LAST_W != 64) && (c == C::SLICES - 1);  // last slice of a 240-wide tile: 48 columns
                 tmem_ld_32x32(tcol, r0);
-                tmem_ld_32x32(tcol + 32, r1);
+                if (narrow) tmem_ld_32x16(tcol + 32, r1); else tmem_ld_32x32(tcol + 32, r1);
                 tmem_ld_wait();
                 const int col = n0 + c * 64;
                 uint8_t* buf = stage_buf + (TPW == 2 ? ord : 0) * EPI_TILE_BYTES;
@@ -323,6 +340,7 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
                 if (col < N) {
 #pragma unroll
                     for (int j = 0; j < 8; ++j) {  // 8 chunks of 16 bytes = 8 columns each
+                        if (narrow && j >= C::LAST_W / 8) break;
                         uint32_t o[4];
 #pragma unroll
                         for (int i = 0; i < 4; ++i) {
@@ -359,12 +377,32 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
                 mbar_arrive_cluster(tempty0 + (uint32_t)acc * 8u);
                 if (TPW == 2) {
                     int o2 = 0;
-                    for (int c = half; c < BN / 64; c += EPI_WARPS / 4, ++o2)
-                        if (n0 + c * 64 < N) tma_store_2d(&args.tm_y, stage_buf + o2 * EPI_TILE_BYTES, n0 + c * 64, wrow0);
+                    for (int c = half; c < C::SLICES; c += EPI_WARPS / 4, ++o2)
+                        if (n0 + c * 64 < N && !(C::LAST_W != 64 && c == C::SLICES - 1))
+                            tma_store_2d(&args.tm_y, stage_buf + o2 * EPI_TILE_BYTES, n0 + c * 64, wrow0);
                     tma_store_commit();
                 }
             }
             __syncwarp();
+            if (C::LAST_W != 64 && TPW == 2) {
+                // the 48-column last slice of a 240-wide tile: row-wise 16-byte stores from the staging tile
+                // (8 lanes per row, 4 rows per instruction), clipped at M and N
+                const int c = C::SLICES - 1;
+                if ((c & 1) == half && n0 + c * 64 < N) {
+                    const uint8_t* buf = stage_buf + (c >> 1) * EPI_TILE_BYTES;
+                    const int j = lane & 7;
+#pragma unroll
+                    for (int rr = 0; rr < 8; ++rr) {
+                        const int rl = rr * 4 + (lane >> 3);
+                        const int orow = wrow0 + rl;
+                        const int ocol = n0 + c * 64 + j * 8;
+                        if (j < C::LAST_W / 8 && orow < args.M && ocol < N)
+                            *reinterpret_cast<uint4*>(args.Y + (int64_t)orow * args.ldy + ocol) =
+                                *reinterpret_cast<const uint4*>(buf + rl * 128 + ((j ^ (rl & 7)) << 4));
+                    }
+                }
+                __syncwarp();
+            }
             if (++acc == ACC) { acc = 0; acc_ph ^= 1u; }
         }
         if (lane == 0) tma_store_wait_all<0>();
@@ -430,32 +468,43 @@ static cudaError_t launch_cfg(const GemmArgs& a, cudaStream_t st) {
 }  // namespace pair
 
 // Tile width of the pair kernel for a given problem.  The pair tile is 256 x BN and the kernel is
-// persistent over num_sms/2 pairs, so the cost is (rounds of tiles) x (time per tile).  Per tile:
-// a 192-wide tile has two accumulators (epilogue drain hidden behind the next tile's K loop unless the
-// K loop is shorter than the drain), a 256-wide tile has one (drain exposed).  Stage and drain times are
-// the measured ones on B200 (ns).  OSC_PAIR_BLOCK_N overrides.
-int gemm_pair_block_n(int M, int N, int stages, int num_sms) {
+// persistent over num_sms/2 pairs, so the cost is (rounds of tiles) x (time per tile).  Measured on B200
+// a K stage costs the same ~370 ns for 192, 240 and 256 columns (the MMA runs at the 256-column rate
+// for all three), so wide tiles win; 240 is the widest that leaves room in TMEM for two accumulators
+// plus the scale columns (epilogue hidden behind the next tile's K loop unless that loop is shorter
+// than the ~2 us drain), 256 has one accumulator (drain and hand-over exposed, ~2.7 us per tile).
+// The FP8 mode needs no scale columns: 256 wide with two accumulators.  OSC_PAIR_BLOCK_N overrides.
+int gemm_pair_block_n(bool fp8, int M, int N, int stages, int num_sms) {
     static int forced = -1;
     if (forced < 0) {
         forced = 0;
         if (const char* e = getenv("OSC_PAIR_BLOCK_N")) {
             const int v = atoi(e);
-            if (v == 192 || v == 256) forced = v;
+            if (v == 192 || v == 240 || v == 256) forced = v;
         }
     }
-    if (forced) return forced;
+    if (forced && !(fp8 && forced == 240)) return forced;
     const int pairs = num_sms / 2 > 0 ? num_sms / 2 : 1;
     const long mt = (M + 255) / 256;
-    const long r192 = (mt * ((N + 191) / 192) + pairs - 1) / pairs;
-    const long r256 = (mt * ((N + 255) / 256) + pairs - 1) / pairs;
-    const long loop192 = 370L * stages, loop256 = 450L * stages;
-    const long t192 = loop192 > 2000 ? loop192 : 2000;  // drain of 192 columns ~2.0 us, overlapped
-    const long t256 = loop256 + 2500;                   // drain of 256 columns ~2.5 us, exposed
-    return (r192 * t192 <= r256 * t256) ? 192 : 256;
+    const long loop = 370L * stages;
+    const long hidden = loop > 2000 ? loop : 2000;
+    long best = -1;
+    int best_bn = 256;
+    const int cand[3] = {256, 240, 192};
+    for (int i = 0; i < 3; ++i) {
+        const int bn = cand[i];
+        if (fp8 && bn == 240) continue;
+        const long rounds = (mt * ((N + bn - 1) / bn) + pairs - 1) / pairs;
+        const bool two_acc = fp8 || bn != 256;
+        const long cost = rounds * (two_acc ? hidden : loop + 2700);
+        if (best < 0 || cost < best) { best = cost; best_bn = bn; }
+    }
+    return best_bn;
 }
 
 cudaError_t launch_gemm_dual_pair(const GemmArgs& a, int bn, cudaStream_t st) {
     if (bn == 192) return pair::launch_cfg<pair::MODE_OSC, 192>(a, st);
+    if (bn == 240) return pair::launch_cfg<pair::MODE_OSC, 240>(a, st);
     return pair::launch_cfg<pair::MODE_OSC, 256>(a, st);
 }
 cudaError_t launch_gemm_fp8_pair(const GemmArgs& a, int bn, cudaStream_t st) {

@@ -392,6 +392,39 @@ __global__ void build_sched_kernel(const int32_t* __restrict__ off, int E, int32
     }
 }
 
+// ----------------------------------------------- per-tile copy of weight scales
+// dst holds, for every bn-row tile of the weight matrix, ceil(bn/128) 128-row scale blocks per
+// 128-channel block in which the tile's first row is row 0 (rows past the tile or past N: code 0).
+// Block order: [tile][block of the tile][K block]; inside a block the usual 512-byte arrangement.
+__global__ void retile_sf_kernel(const uint8_t* __restrict__ src, uint8_t* __restrict__ dst, int N, int K, int bn) {
+    const int katoms = K / 128;
+    const int atoms_per_tile = (bn + 127) / 128;
+    const int ntiles = (N + bn - 1) / bn;
+    const int64_t total = (int64_t)ntiles * atoms_per_tile * katoms * 512;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int byte = (int)(i & 511);
+        const int64_t blk = i >> 9;
+        const int ka = (int)(blk % katoms);
+        const int at = (int)((blk / katoms) % atoms_per_tile);
+        const int tile = (int)(blk / ((int64_t)katoms * atoms_per_tile));
+        const int r32 = byte >> 4, q = (byte >> 2) & 3, g4 = byte & 3;
+        const int j = at * 128 + q * 32 + r32;  // row inside the tile
+        const int n = tile * bn + j;
+        uint8_t v = 0;
+        if (j < bn && n < N)
+            v = src[((int64_t)(n / 128) * katoms + ka) * 512 + (n % 32) * 16 + ((n % 128) / 32) * 4 + g4];
+        dst[i] = v;
+    }
+}
+
+cudaError_t launch_retile_sf(const uint8_t* src, uint8_t* dst, int N, int K, int bn, cudaStream_t st) {
+    const int64_t total = (int64_t)((N + bn - 1) / bn) * ((bn + 127) / 128) * (K / 128) * 512;
+    if (total <= 0) return cudaSuccess;
+    const int blocks = (int)((total + 255) / 256 < 2048 ? (total + 255) / 256 : 2048);
+    retile_sf_kernel<<<blocks, 256, 0, st>>>(src, dst, N, K, bn);
+    return cudaGetLastError();
+}
+
 // ------------------------------------------------------------------ launchers
 cudaError_t launch_quant_extract(const CUtensorMap& tm_x, int M, int K, const uint32_t* mask,
                                  const int32_t* prefix, const int32_t* idx_o, void* xq, void* sf, void* xo, int Ko, int Kop,
