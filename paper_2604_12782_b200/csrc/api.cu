@@ -183,8 +183,8 @@ struct osc_weights {
     const uint32_t* mask;
     const int32_t* prefix;
     const int32_t* idx_o;
-    int num_sms, block_n;
-    CUtensorMap tm_b, tm_bo;          // single-CTA kernel: weight tiles of block_n rows
+    int num_sms;
+    CUtensorMap tm_b[4], tm_bo[4];    // single-CTA kernel: weight tiles of 64 / 128 / 192 / 256 rows
     CUtensorMap tm_b2[3], tm_bo2[3];  // CTA-pair kernel: half tiles for 192-, 256- and 240-wide tiles
     CUtensorMap tm_sfw, tm_sfw_tiled;  // scale blocks: standard layout / per-tile copy for 240-wide tiles
 };
@@ -193,8 +193,8 @@ struct osc_fp8_weights {
     bool grouped;
     const uint8_t* w8;
     const float* sw;
-    int num_sms, block_n;
-    CUtensorMap tm_b, tm_b2[2];
+    int num_sms;
+    CUtensorMap tm_b[4], tm_b2[2];
 };
 
 extern "C" {
@@ -292,10 +292,12 @@ static osc_status prepare_impl(const void* W, int E, int N, int K, int64_t ldw, 
     w->mask = d_mask; w->prefix = d_prefix;
     w->idx_o = reinterpret_cast<const int32_t*>(m8 + (size_t)Kg * 8);
     w->num_sms = di.num_sms;
-    w->block_n = gemm_block_n();
-    osc_status s = make_tmap(&w->tm_b, wq, false, (uint64_t)E * N, K / 2, K / 2, w->block_n);
-    if (s == OSC_OK && t.Kop > 0)
-        s = make_tmap(&w->tm_bo, wo, true, (uint64_t)E * N, (uint64_t)t.Kop * 2, (uint64_t)t.Kop * 2, w->block_n);
+    osc_status s = OSC_OK;
+    for (int v = 0; v < 4 && s == OSC_OK; ++v) {
+        s = make_tmap(&w->tm_b[v], wq, false, (uint64_t)E * N, K / 2, K / 2, 64 * (v + 1));
+        if (s == OSC_OK && t.Kop > 0)
+            s = make_tmap(&w->tm_bo[v], wo, true, (uint64_t)E * N, (uint64_t)t.Kop * 2, (uint64_t)t.Kop * 2, 64 * (v + 1));
+    }
     for (int v = 0; v < 3 && s == OSC_OK && !grouped; ++v) {
         const int half = (v == 0 ? 192 : v == 1 ? 256 : kTiledBN) / 2;
         s = make_tmap(&w->tm_b2[v], wq, false, (uint64_t)N, K / 2, K / 2, half);
@@ -382,10 +384,11 @@ static osc_status gemm_impl(const osc_weights* w, const void* xq, const void* sf
     GemmArgs a;
     memset(&a, 0, sizeof a);
     if (osc_status s = make_tmap(&a.tm_a, xq, false, M, w->K / 2, w->K / 2, 128)) return s;
-    a.tm_b = w->tm_b;
+    const int bn1 = gemm_block_n(sched ? max_tiles : (M + 127) / 128, w->N, w->num_sms);
+    a.tm_b = w->tm_b[bn1 / 64 - 1];
     if (w->Kop > 0) {
         if (osc_status s = make_tmap(&a.tm_ao, xo, true, M, (uint64_t)w->Kop * 2, (uint64_t)w->Kop * 2, 128)) return s;
-        a.tm_bo = w->tm_bo;
+        a.tm_bo = w->tm_bo[bn1 / 64 - 1];
     }
     a.sfa = static_cast<const uint8_t*>(sfa);
     a.sfw = w->sfw;
@@ -404,7 +407,7 @@ static osc_status gemm_impl(const osc_weights* w, const void* xq, const void* sf
         if (osc_status s = make_tmap(&a.tm_y, Y, true, M, (uint64_t)w->N * 2, (uint64_t)ldy * 2, 32)) return s;
         e = launch_gemm_dual_pair(a, bn, st);
     } else {
-        e = launch_gemm_dual(a, st);
+        e = launch_gemm_dual(a, bn1, st);
     }
     if (e != cudaSuccess) return cuda_fail(e, "gemm_kernel(dual)");
     return OSC_OK;
@@ -483,8 +486,9 @@ static osc_status fp8_prepare_impl(const void* W, int E, int N, int K, int64_t l
     w->w8 = static_cast<const uint8_t*>(w8);
     w->sw = static_cast<const float*>(sw);
     w->num_sms = di.num_sms;
-    w->block_n = gemm_block_n();
-    if (osc_status s = make_tmap(&w->tm_b, w8, false, (uint64_t)E * N, K, K, w->block_n)) { delete w; return s; }
+    for (int v = 0; v < 4; ++v) {
+        if (osc_status s = make_tmap(&w->tm_b[v], w8, false, (uint64_t)E * N, K, K, 64 * (v + 1))) { delete w; return s; }
+    }
     for (int v = 0; v < 2 && !grouped; ++v) {
         if (osc_status s = make_tmap(&w->tm_b2[v], w8, false, (uint64_t)N, K, K, (v == 0 ? 192 : 256) / 2)) { delete w; return s; }
     }
@@ -542,7 +546,8 @@ static osc_status fp8_gemm_impl(const osc_fp8_weights* w, const void* x8, const 
     GemmArgs a;
     memset(&a, 0, sizeof a);
     if (osc_status s = make_tmap(&a.tm_a, x8, false, M, w->K, w->K, 128)) return s;
-    a.tm_b = w->tm_b;
+    const int bn1 = gemm_block_n(sched ? max_tiles : (M + 127) / 128, w->N, w->num_sms);
+    a.tm_b = w->tm_b[bn1 / 64 - 1];
     a.sx = static_cast<const float*>(sx);
     a.sw = w->sw;
     a.Y = static_cast<uint16_t*>(Y);
@@ -556,7 +561,7 @@ static osc_status fp8_gemm_impl(const osc_fp8_weights* w, const void* x8, const 
         if (osc_status s = make_tmap(&a.tm_y, Y, true, M, (uint64_t)w->N * 2, (uint64_t)ldy * 2, 32)) return s;
         e = launch_gemm_fp8_pair(a, bn, st);
     } else {
-        e = launch_gemm_fp8(a, st);
+        e = launch_gemm_fp8(a, bn1, st);
     }
     if (e != cudaSuccess) return cuda_fail(e, "gemm_kernel(fp8)");
     return OSC_OK;

@@ -54,9 +54,9 @@ struct GemmArgs {
     int max_tiles;
     int num_sms;
 };
-cudaError_t launch_gemm_dual(const GemmArgs& a, cudaStream_t st);
-cudaError_t launch_gemm_fp8(const GemmArgs& a, cudaStream_t st);
-int gemm_block_n();
+cudaError_t launch_gemm_dual(const GemmArgs& a, int bn, cudaStream_t st);
+cudaError_t launch_gemm_fp8(const GemmArgs& a, int bn, cudaStream_t st);
+int gemm_block_n(int row_tiles, int N, int num_sms);
 
 // gemm2_kernels.cu (CTA pairs, dense problems)
 cudaError_t launch_gemm_dual_pair(const GemmArgs& a, int bn, cudaStream_t st);

@@ -355,17 +355,23 @@ done:
 }
 
 // ---------------------------------------------------------------- launchers
-static int g_block_n = 0;
-
-int gemm_block_n() {
-    if (g_block_n == 0) {
-        g_block_n = 256;
+// Tile width of the single-CTA kernel.  Few-row problems are weight streaming: every SM should pull
+// its share of the weights, so the width shrinks until there are about as many tiles as SMs.
+// Grouped problems have plenty of row tiles and take the widest tile.  OSC_BLOCK_N overrides.
+int gemm_block_n(int row_tiles, int N, int num_sms) {
+    static int forced = -1;
+    if (forced < 0) {
+        forced = 0;
         if (const char* e = getenv("OSC_BLOCK_N")) {
             const int v = atoi(e);
-            if (v == 128 || v == 192 || v == 256) g_block_n = v;
+            if (v == 64 || v == 128 || v == 192 || v == 256) forced = v;
         }
     }
-    return g_block_n;
+    if (forced) return forced;
+    const int cand[4] = {256, 192, 128, 64};
+    for (int i = 0; i < 4; ++i)
+        if ((long)row_tiles * ((N + cand[i] - 1) / cand[i]) >= num_sms) return cand[i];
+    return 64;
 }
 
 template <int MODE, int BN>
@@ -387,15 +393,17 @@ static cudaError_t launch_cfg(const GemmArgs& a, cudaStream_t st) {
     return launch_pdl(gemm_kernel<MODE, BN>, dim3(grid), dim3(GEMM_THREADS), C::SMEM_BYTES, st, a);
 }
 
-cudaError_t launch_gemm_dual(const GemmArgs& a, cudaStream_t st) {
-    switch (gemm_block_n()) {
+cudaError_t launch_gemm_dual(const GemmArgs& a, int bn, cudaStream_t st) {
+    switch (bn) {
+        case 64: return launch_cfg<MODE_OSC, 64>(a, st);
         case 128: return launch_cfg<MODE_OSC, 128>(a, st);
         case 192: return launch_cfg<MODE_OSC, 192>(a, st);
         default: return launch_cfg<MODE_OSC, 256>(a, st);
     }
 }
-cudaError_t launch_gemm_fp8(const GemmArgs& a, cudaStream_t st) {
-    switch (gemm_block_n()) {
+cudaError_t launch_gemm_fp8(const GemmArgs& a, int bn, cudaStream_t st) {
+    switch (bn) {
+        case 64: return launch_cfg<MODE_FP8, 64>(a, st);
         case 128: return launch_cfg<MODE_FP8, 128>(a, st);
         case 192: return launch_cfg<MODE_FP8, 192>(a, st);
         default: return launch_cfg<MODE_FP8, 256>(a, st);

@@ -308,9 +308,10 @@ fp8_quant_kernel(const uint16_t* __restrict__ X, int64_t ldx, int M, int K, uint
     }
 }
 
-// Short rows (K <= 2048): one warp per row, eight rows per CTA, the row held in registers
-// (at most 8 chunks of 8 elements per lane).  A CTA per row would leave most threads idle.
-constexpr int F8W_MAXCH = 8;
+// Short rows (K <= 4096): one warp per row, eight rows per CTA, the row held in registers
+// (at most 8 or 16 chunks of 8 elements per lane).  A CTA per row leaves most threads idle or
+// spends its time in the block-wide reduction.
+template <int F8W_MAXCH>
 __global__ void __launch_bounds__(256)
 fp8_quant_rows_kernel(const uint16_t* __restrict__ X, int64_t ldx, int M, int K, uint8_t* __restrict__ x8,
                       float* __restrict__ sx) {
@@ -445,9 +446,12 @@ cudaError_t launch_quant_extract(const CUtensorMap& tm_x, int M, int K, const ui
 
 cudaError_t launch_fp8_quant(const void* X, int64_t ldx, int M, int K, void* x8, void* sx, cudaStream_t st) {
     if (M <= 0) return cudaSuccess;
-    if (K <= F8W_MAXCH * 32 * 8) {
-        return launch_pdl(fp8_quant_rows_kernel, dim3((M + 7) / 8), dim3(256), 0, st, static_cast<const uint16_t*>(X), ldx,
-                          M, K, static_cast<uint8_t*>(x8), static_cast<float*>(sx));
+    if (K <= 8 * 32 * 8)
+        return launch_pdl(fp8_quant_rows_kernel<8>, dim3((M + 7) / 8), dim3(256), 0, st, static_cast<const uint16_t*>(X),
+                          ldx, M, K, static_cast<uint8_t*>(x8), static_cast<float*>(sx));
+    if (K <= 16 * 32 * 8) {
+        return launch_pdl(fp8_quant_rows_kernel<16>, dim3((M + 7) / 8), dim3(256), 0, st, static_cast<const uint16_t*>(X),
+                          ldx, M, K, static_cast<uint8_t*>(x8), static_cast<float*>(sx));
     }
     return launch_pdl(fp8_quant_kernel, dim3(M), dim3(F8_THREADS), 0, st, static_cast<const uint16_t*>(X), ldx, M, K,
                       static_cast<uint8_t*>(x8), static_cast<float*>(sx));
