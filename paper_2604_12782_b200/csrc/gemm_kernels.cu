@@ -39,7 +39,8 @@ constexpr int G_EPI_TILE_BYTES = 32 * 128;  // staging tile: 32 rows x 64 bf16 c
 template <int MODE, int BN>
 struct Cfg {
     static constexpr int SFB_ATOMS = (BN > 128) ? 2 : 1;  // 128-row scale blocks a tile can touch
-    static constexpr int SF_COLS = 8 + 2 * SFB_ATOMS * 4;  // TMEM columns of one stage's scales (A: 8, B: 2 x atoms x 4)
+    // TMEM columns of one stage's scales (A: 8, B: 2 x atoms x 4); the FP8 mode keeps no scales in TMEM
+    static constexpr int SF_COLS = (MODE == MODE_OSC) ? 8 + 2 * SFB_ATOMS * 4 : 0;
     static constexpr int ACC_STAGES = (2 * BN + SF_COLS <= TMEM_COLS) ? 2 : 1;
     static constexpr int B_BYTES = BN * ROW_BYTES;
     static constexpr int SFA_BYTES = (MODE == MODE_OSC) ? 1024 : 0;
