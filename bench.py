@@ -108,6 +108,25 @@ class ClockSampler:
                 "samples": len(self.samples)}
 
 
+# ------------------------------------------------------------------- multi-process glue
+def max_over_ranks(ms: float, device=None) -> float:
+    """Slowest rank's time (the job's time): all-reduce MAX over the default process group, if there is one.
+    Works with the nccl backend (device = a cuda device) and with gloo (device None -> CPU tensor)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(ms)
+    t = torch.tensor([float(ms)], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(units_per_rank: float, world: int, ms: float) -> float:
+    """Replicas only: every rank processes `units_per_rank` (FLOPs) per step; the job's rate is the sum over
+    ranks divided by the slowest rank's time, in TFLOP/s."""
+    return world * units_per_rank / (ms * 1e-3) / 1e12
+
+
 # ---------------------------------------------------------------------- reference arm
 def oracle_sample_step(oracle, case, wts, rows):
     """One bounded step of the CPU oracle: Algorithm 2 on `rows` activation rows, then Eq. 5."""
@@ -285,17 +304,14 @@ def run_gpu(args):
     clocks = sampler.stop()
     B.osc_sync_check()
 
-    if world > 1:
-        t = torch.tensor([ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(ms, torch.device("cuda", local))
     if args.only_osc:
         print(f"osc_linear {ms:.4f} ms/step (quantizer {tq:.4f}, gemm {tg:.4f})", file=sys.stderr)
         return
 
     flops4, flops16 = roofline.osc_flops(M, N, K, Ko)
     flops = flops4 + flops16
-    value = world * flops / (ms * 1e-3) / 1e12
+    value = whole_job_value(flops, world, ms)
 
     # ---- end to end through the C ABI with host buffers (copies inside the timed region)
     Xh = torch.from_numpy(case["X"].view(np.int16)).view(torch.bfloat16).pin_memory()
@@ -309,11 +325,8 @@ def run_gpu(args):
 
     e2e_steps = max(3, min(args.steps, 20))
     ms_e2e = time_loop(torch, e2e_step, e2e_steps, 3)
-    if world > 1:
-        t = torch.tensor([ms_e2e], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_e2e = float(t.item())
-    e2e_value = world * flops / (ms_e2e * 1e-3) / 1e12
+    ms_e2e = max_over_ranks(ms_e2e, torch.device("cuda", local))
+    e2e_value = whole_job_value(flops, world, ms_e2e)
 
     # ---- the same build's FP8 W8A8 linear on the same shape (the paper's comparison point)
     f8case = {"X": case["X"], "W": case["W"], "M": M, "K": K, "N": N}

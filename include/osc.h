@@ -153,6 +153,25 @@ osc_status osc_linear_grouped(const osc_weights* w, const void* X_perm, const in
                               int64_t ldx, void* Y, int64_t ldy, void* workspace, size_t workspace_bytes,
                               void* stream);
 
+/* ---------------------------------------------------- offline profiling */
+
+/* Scratch bytes osc_profile_lut needs for a K-channel slice (an fp64 sum and 32 counters per group). */
+osc_status osc_profile_scratch_bytes(int K, size_t* bytes);
+
+/* Offline profiling of one (position, layer) slice of calibration activations (Section 2.1-2.2, Eq. 1-4, and
+ * Algorithm 1 for that slice).  X: dev bf16 [S, ldx], S tokens, K channels, groups of 32.
+ *   T_l = alpha * mean|X|                                    (Eq. 1; the paper uses alpha = 5)
+ *   per token and group the first channel with the largest magnitude (Eq. 2) votes if that magnitude
+ *   exceeds T_l (Eq. 3); per group lut[k] = the channel with most votes (smallest index among equals) or -1
+ *   if no token voted (Algorithm 1), n_total[k] = votes, n_hit[k] = votes of the winner (Eq. 4: the clustering
+ *   density is n_hit[k] / n_total[k]).
+ * Outputs (dev): lut int8 [K/32], n_hit int32 [K/32], n_total int32 [K/32], threshold_bits uint32 [1] = bit
+ * pattern of the largest bf16 magnitude <= T_l (for bf16 data |x| > T_l is exactly bits(|x|) > that pattern;
+ * T_l itself is formed in fp64).  scratch: dev, zeroed by the call.  The resulting lut (copied to the host) is
+ * what osc_prepare_weights takes with lut_c = 1. */
+osc_status osc_profile_lut(const void* X, int S, int K, int64_t ldx, float alpha, void* scratch, size_t scratch_bytes,
+                           void* lut, void* n_hit, void* n_total, void* threshold_bits, void* stream);
+
 /* ------------------------------------------------------------- FP8 fallback */
 
 typedef struct osc_fp8_weights osc_fp8_weights;

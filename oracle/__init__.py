@@ -9,6 +9,7 @@ Function-to-paper map (details in the C file):
   quantize_extract / prepare_weights  Algorithm 2 (+ Section 3.3 weight split)
   gemm_dual / linear                   Eq. 5
   fp8_quantize / fp8_gemm / fp8_linear Section 3.4 fallback
+  threshold / profile_indexing / clustering_density   Eq. 1-4, Algorithm 1 (offline profiling)
 """
 from __future__ import annotations
 
@@ -48,6 +49,10 @@ def lib():
         _lib.osc_ref_sf_bytes.restype = C.c_int64
         _lib.osc_ref_sf_bytes.argtypes = [C.c_int64, C.c_int64]
         _lib.osc_ref_sf_row_base.restype = C.c_int64
+        _lib.osc_ref_threshold.restype = C.c_double
+        _lib.osc_ref_threshold.argtypes = [C.c_void_p, C.c_int64, C.c_int, C.c_int, C.c_double]
+        _lib.osc_ref_threshold_bits.restype = C.c_uint32
+        _lib.osc_ref_threshold_bits.argtypes = [C.c_double]
     return _lib
 
 
@@ -203,3 +208,33 @@ def fp8_linear(X: np.ndarray, W: np.ndarray, rows=None):
     w8, sw = fp8_quantize(W)
     Y, T = fp8_gemm(x8, sx, w8, sw, rows)
     return Y, T, (x8, sx), (w8, sw)
+
+
+def threshold(X: np.ndarray, alpha: float = 5.0) -> float:
+    """Eq. 1: T_l = alpha * mean|X|."""
+    X = np.ascontiguousarray(X, dtype=np.uint16)
+    S, H = X.shape
+    return float(lib().osc_ref_threshold(_p(X), H, S, H, float(alpha)))
+
+
+def threshold_bits(T: float) -> int:
+    return int(lib().osc_ref_threshold_bits(float(T)))
+
+
+def profile_indexing(X: np.ndarray, T: float):
+    """Algorithm 1 for one (position, layer) -> (L int8 [K], n_hit i32 [K], n_total i32 [K])."""
+    X = np.ascontiguousarray(X, dtype=np.uint16)
+    S, H = X.shape
+    K = H // 32
+    L = np.zeros(K, np.int8)
+    nh = np.zeros(K, np.int32)
+    nt = np.zeros(K, np.int32)
+    rc = lib().osc_ref_profile_indexing(_p(X), C.c_int64(H), S, H, C.c_double(T), _p(L), _p(nh), _p(nt))
+    assert rc == 0
+    return L, nh, nt
+
+
+def clustering_density(n_hit: np.ndarray, n_total: np.ndarray):
+    """Eq. 4 and the block mean: C_k = n_hit/n_total (0 for groups without outlier tokens), mean over all K groups."""
+    c = np.where(n_total > 0, n_hit / np.maximum(n_total, 1), 0.0)
+    return c, float(c.mean())

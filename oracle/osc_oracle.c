@@ -376,6 +376,61 @@ int osc_ref_fp8_gemm_rows(const uint8_t* x8, const float* sx, const int32_t* row
     return 0;
 }
 
+/* ------------------------------------------- offline profiling (Section 2, Algorithm 1) */
+
+/* Eq. 1: layer-wise threshold T_l = alpha * mean |x| over the S x H calibration activations. */
+double osc_ref_threshold(const uint16_t* X, int64_t ldx, int S, int H, double alpha) {
+    double sum = 0.0;
+    for (int s = 0; s < S; ++s)
+        for (int j = 0; j < H; ++j) sum += fabs(bf16_value(X[(int64_t)s * ldx + j]));
+    return alpha * (sum / ((double)S * (double)H));
+}
+
+/* Largest bf16 magnitude (bit pattern, sign clear) whose value is <= T: for bf16 inputs |x| > T is the
+ * same as bits(|x|) > this pattern, which makes the outlier test an integer comparison. */
+uint32_t osc_ref_threshold_bits(double T) {
+    if (!(T > 0.0)) return 0;
+    float f = (float)T;
+    if ((double)f > T) f = nextafterf(f, 0.0f);
+    uint32_t u;
+    memcpy(&u, &f, 4);
+    return u >> 16;
+}
+
+/* Algorithm 1 for one (position, layer): for every group k and token s take j* = argmax_j |x_{s,kG+j}|
+ * (first maximum wins); if |x_{s,kG+j*}| > T_l the token joins S_k with index j*.  L[k] = the most
+ * frequent index in S_k (smallest index among equally frequent ones), -1 if S_k is empty.
+ * Also returns Eq. 3-4: n_total[k] = |S_k| and n_hit[k] = how many of them carry the dominant index,
+ * so that the clustering density is C_k = n_hit[k] / n_total[k]. */
+int osc_ref_profile_indexing(const uint16_t* X, int64_t ldx, int S, int H, double T, int8_t* L, int32_t* n_hit,
+                             int32_t* n_total) {
+    if (H % G) return -3;
+    const int K = H / G;
+    for (int k = 0; k < K; ++k) {
+        int count[G];
+        for (int j = 0; j < G; ++j) count[j] = 0;
+        for (int s = 0; s < S; ++s) {
+            const int offset = k * G;
+            int jstar = 0;
+            double best = -1.0;
+            for (int j = 0; j < G; ++j) {
+                const double a = fabs(bf16_value(X[(int64_t)s * ldx + offset + j]));
+                if (a > best) { best = a; jstar = j; }
+            }
+            if (best > T) count[jstar] += 1;
+        }
+        int total = 0, hit = 0, mode = -1;
+        for (int j = 0; j < G; ++j) {
+            total += count[j];
+            if (count[j] > hit) { hit = count[j]; mode = j; }
+        }
+        L[k] = (int8_t)(total > 0 ? mode : -1);
+        n_hit[k] = hit;
+        n_total[k] = total;
+    }
+    return 0;
+}
+
 int osc_ref_num_threads(void) {
     int n = 1;
 #ifdef _OPENMP

@@ -62,6 +62,8 @@ _SIGS = {
     "osc_linear": (_i, [_vp, _vp, _i, _i64, _vp, _i64, _vp, _sz, _vp]),
     "osc_linear_static": (_i, [_vp, _vp, _i, _i64, _vp, _i64, _vp]),
     "osc_linear_grouped": (_i, [_vp, _vp, _vp, _i, _i64, _vp, _i64, _vp, _sz, _vp]),
+    "osc_profile_scratch_bytes": (_i, [_i, C.POINTER(_sz)]),
+    "osc_profile_lut": (_i, [_vp, _i, _i, _i64, C.c_float, _vp, _sz, _vp, _vp, _vp, _vp, _vp]),
     "osc_fp8_prepare_weights": (_i, [_vp, _i, _i, _i64, _vp, _vp, _vp, C.POINTER(_vp)]),
     "osc_fp8_prepare_weights_grouped": (_i, [_vp, _i, _i, _i, _vp, _vp, _vp, C.POINTER(_vp)]),
     "osc_fp8_weights_destroy": (_i, [_vp]),
@@ -228,6 +230,20 @@ def osc_linear_grouped(w: OscWeights, X: torch.Tensor, off: torch.Tensor, Y: tor
     _check(_lib.osc_linear_grouped(w.ptr, _ptr(X), _ptr(off), M, X.stride(0) if M else w.K, _ptr(Y),
                                    Y.stride(0) if M else w.N, _ptr(workspace),
                                    workspace.numel() * workspace.element_size(), _stream(stream)))
+
+
+def osc_profile_scratch_bytes(K: int) -> int:
+    out = _sz()
+    _check(_lib.osc_profile_scratch_bytes(K, C.byref(out)))
+    return int(out.value)
+
+
+def osc_profile_lut(X: torch.Tensor, alpha: float, scratch, lut, n_hit, n_total, threshold_bits, stream=None):
+    """X: cuda bf16 [S, K]; outputs are cuda tensors (int8 [K/32], int32 [K/32] x2, int32/uint32 [1])."""
+    S, K = X.shape
+    _check(_lib.osc_profile_lut(_ptr(X), S, K, X.stride(0), float(alpha), _ptr(scratch),
+                                scratch.numel() * scratch.element_size(), _ptr(lut), _ptr(n_hit), _ptr(n_total),
+                                _ptr(threshold_bits), _stream(stream)))
 
 
 def osc_fp8_prepare_weights(W: torch.Tensor, stream=None) -> Fp8Weights:

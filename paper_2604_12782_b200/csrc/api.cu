@@ -465,6 +465,38 @@ osc_status osc_linear_grouped(const osc_weights* w, const void* X_perm, const in
     return gemm_impl(w, ws + sz.xq_offset, ws + sz.sfa_offset, ws + sz.xo_offset, M_total, Y, ldy, sched, max_tiles, st);
 }
 
+// ------------------------------------------------------- offline profiling
+
+osc_status osc_profile_scratch_bytes(int K, size_t* bytes) {
+    if (!bytes) return fail(OSC_ERR_INVALID_ARG, "bytes is null");
+    if (K <= 0 || K % 128) return fail(OSC_ERR_SHAPE, "K = %d must be a positive multiple of 128", K);
+    *bytes = 256 + (size_t)(K / 32) * 32 * sizeof(int32_t);
+    return OSC_OK;
+}
+
+osc_status osc_profile_lut(const void* X, int S, int K, int64_t ldx, float alpha, void* scratch, size_t scratch_bytes,
+                           void* lut, void* n_hit, void* n_total, void* threshold_bits, void* stream) {
+    if (S <= 0) return fail(OSC_ERR_INVALID_ARG, "S = %d must be positive", S);
+    size_t need = 0;
+    if (osc_status s = osc_profile_scratch_bytes(K, &need)) return s;
+    if (!X || !scratch || !lut || !n_hit || !n_total || !threshold_bits) return fail(OSC_ERR_INVALID_ARG, "null device pointer");
+    if (ldx < K) return fail(OSC_ERR_SHAPE, "ldx = %lld < K", (long long)ldx);
+    if (ldx % 8 || !aligned16(X) || !aligned16(scratch) || (reinterpret_cast<uintptr_t>(n_hit) & 3) ||
+        (reinterpret_cast<uintptr_t>(n_total) & 3) || (reinterpret_cast<uintptr_t>(threshold_bits) & 3))
+        return fail(OSC_ERR_ALIGN, "X and scratch must be 16-byte aligned, ldx a multiple of 8, counters 4-byte aligned");
+    if (scratch_bytes < need) return fail(OSC_ERR_WORKSPACE, "scratch has %zu bytes, %zu needed", scratch_bytes, need);
+    if (!(alpha > 0.0f)) return fail(OSC_ERR_INVALID_ARG, "alpha must be positive");
+    DeviceInfo di;
+    if (osc_status s = device_info(&di)) return s;
+    uint8_t* sc = static_cast<uint8_t*>(scratch);
+    cudaError_t e = launch_profile(X, ldx, S, K, (double)alpha, reinterpret_cast<double*>(sc),
+                                   reinterpret_cast<int32_t*>(sc + 256), static_cast<int8_t*>(lut),
+                                   static_cast<int32_t*>(n_hit), static_cast<int32_t*>(n_total),
+                                   static_cast<uint32_t*>(threshold_bits), di.num_sms, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(e, "profile kernels");
+    return OSC_OK;
+}
+
 // -------------------------------------------------------------- FP8 fallback
 
 static osc_status fp8_prepare_impl(const void* W, int E, int N, int K, int64_t ldw, void* w8, void* sw, void* stream,

@@ -33,6 +33,11 @@ cudaError_t launch_quant_extract(const CUtensorMap& tm_x, int M, int K, const ui
 cudaError_t launch_fp8_quant(const void* X, int64_t ldx, int M, int K, void* x8, void* sx, cudaStream_t st);
 cudaError_t launch_build_sched(const int32_t* off, int E, int32_t* sched, int max_tiles, cudaStream_t st);
 
+// profile_kernels.cu
+cudaError_t launch_profile(const void* X, int64_t ldx, int S, int K, double alpha, double* sum, int32_t* counts,
+                           int8_t* lut, int32_t* n_hit, int32_t* n_total, uint32_t* threshold_bits, int num_sms,
+                           cudaStream_t st);
+
 // gemm_kernels.cu
 struct GemmArgs {
     CUtensorMap tm_a;    // Path A activations: packed FP4 bytes [rows, K/2]  (FP8 mode: [rows, K])

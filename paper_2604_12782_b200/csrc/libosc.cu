@@ -3,5 +3,6 @@
 #include "quant_kernels.cu"
 #include "gemm_kernels.cu"
 #include "gemm2_kernels.cu"
+#include "profile_kernels.cu"
 #include "api.cu"
 #include "static_scratch.cu"
