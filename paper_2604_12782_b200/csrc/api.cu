@@ -114,13 +114,16 @@ static osc_status make_tmap_sf(CUtensorMap* tm, const void* base, uint64_t block
     return OSC_OK;
 }
 
-static bool use_pair_kernel(bool grouped, int M) {
+// Dense problems with more than 128 rows, and grouped problems whose experts average at least 96 rows, run
+// on the CTA-pair kernel (256-row tiles); the rest on the single-CTA kernel (128-row tiles).
+static bool use_pair_kernel(bool grouped, int M, int E) {
     static int enabled = -1;
     if (enabled < 0) {
         const char* e = getenv("OSC_PAIR");
         enabled = (e && atoi(e) == 0) ? 0 : 1;
     }
-    return enabled && !grouped && M > 128;
+    if (!enabled) return false;
+    return grouped ? (M / E >= 96) : (M > 128);
 }
 
 // ----------------------------------------------------------------- the table
@@ -298,13 +301,14 @@ static osc_status prepare_impl(const void* W, int E, int N, int K, int64_t ldw, 
         if (s == OSC_OK && t.Kop > 0)
             s = make_tmap(&w->tm_bo[v], wo, true, (uint64_t)E * N, (uint64_t)t.Kop * 2, (uint64_t)t.Kop * 2, 64 * (v + 1));
     }
-    for (int v = 0; v < 3 && s == OSC_OK && !grouped; ++v) {
+    for (int v = 0; v < 3 && s == OSC_OK; ++v) {
+        if (grouped && v == 2) break;  // the per-tile scale copy exists for dense weights only
         const int half = (v == 0 ? 192 : v == 1 ? 256 : kTiledBN) / 2;
-        s = make_tmap(&w->tm_b2[v], wq, false, (uint64_t)N, K / 2, K / 2, half);
+        s = make_tmap(&w->tm_b2[v], wq, false, (uint64_t)E * N, K / 2, K / 2, half);
         if (s == OSC_OK && t.Kop > 0)
-            s = make_tmap(&w->tm_bo2[v], wo, true, (uint64_t)N, (uint64_t)t.Kop * 2, (uint64_t)t.Kop * 2, half);
+            s = make_tmap(&w->tm_bo2[v], wo, true, (uint64_t)E * N, (uint64_t)t.Kop * 2, (uint64_t)t.Kop * 2, half);
     }
-    if (s == OSC_OK && !grouped) s = make_tmap_sf(&w->tm_sfw, sfw, (uint64_t)sfw_e / 512);
+    if (s == OSC_OK) s = make_tmap_sf(&w->tm_sfw, sfw, (uint64_t)E * sfw_e / 512);
     if (s == OSC_OK && !grouped) {
         uint8_t* tiled = m8 + meta_table_bytes(K, t.Ko);
         e = launch_retile_sf(static_cast<const uint8_t*>(sfw), tiled, N, K, kTiledBN, st);
@@ -329,6 +333,11 @@ osc_status osc_weights_destroy(osc_weights* w) {
     return OSC_OK;
 }
 
+// A grouped workspace holds two tile schedules, back to back: 128-row tiles (quantizer, single-CTA GEMM) and
+// 256-row tiles (CTA-pair GEMM).  Each is 1 + 4 * max_tiles int32, rounded up to 64.
+static size_t sched_ints(int64_t max_tiles) { return (size_t)((1 + 4 * max_tiles + 63) / 64 * 64); }
+static int max_tiles256(int M, int E) { return M / 256 + E; }
+
 osc_status osc_act_sizes(const osc_weights* w, int M, osc_act_sizes_t* out) {
     if (!w || !out) return fail(OSC_ERR_INVALID_ARG, "null argument");
     if (M < 0) return fail(OSC_ERR_INVALID_ARG, "M = %d is negative", M);
@@ -336,7 +345,7 @@ osc_status osc_act_sizes(const osc_weights* w, int M, osc_act_sizes_t* out) {
     out->xq_bytes = (size_t)M * (w->K / 2);
     out->sfa_bytes = (size_t)max_tiles * (w->K / 128) * 512;
     out->xo_bytes = (size_t)M * w->Kop * 2;
-    out->sched_bytes = w->grouped ? (size_t)(1 + 4 * max_tiles) * 4 : 0;
+    out->sched_bytes = w->grouped ? sched_ints(max_tiles) * 4 + sched_ints(max_tiles256(M, w->E)) * 4 : 0;
     out->xq_offset = 0;
     out->sfa_offset = out->xq_offset + align256(out->xq_bytes);
     out->xo_offset = out->sfa_offset + align256(out->sfa_bytes);
@@ -375,7 +384,8 @@ osc_status osc_quantize_extract(const osc_weights* w, const void* X, int M, int6
 }
 
 static osc_status gemm_impl(const osc_weights* w, const void* xq, const void* sfa, const void* xo, int M, void* Y,
-                            int64_t ldy, const int32_t* sched, int max_tiles, cudaStream_t st) {
+                            int64_t ldy, const int32_t* sched, int max_tiles, const int32_t* sched2, int max_tiles2,
+                            cudaStream_t st) {
     if (M == 0) return OSC_OK;
     if (!xq || !sfa || !Y || (w->Kop > 0 && !xo)) return fail(OSC_ERR_INVALID_ARG, "null device pointer");
     if (ldy < w->N) return fail(OSC_ERR_SHAPE, "ldy = %lld < N = %d", (long long)ldy, w->N);
@@ -396,14 +406,17 @@ static osc_status gemm_impl(const osc_weights* w, const void* xq, const void* sf
     a.ldy = ldy;
     a.M = M; a.N = w->N; a.K = w->K; a.Kop = w->Kop;
     a.sched = sched; a.max_tiles = max_tiles; a.num_sms = w->num_sms;
+    a.sched2 = sched2; a.max_tiles2 = max_tiles2;
     cudaError_t e;
-    if (use_pair_kernel(w->grouped, M)) {
-        const int bn = gemm_pair_block_n(false, M, w->N, (w->K + 255) / 256 + w->Kop / 64, w->num_sms);
+    if (use_pair_kernel(w->grouped, M, w->E)) {
+        const long row_tiles = w->grouped ? max_tiles2 - w->E / 2 : (M + 255) / 256;
+        const int bn = gemm_pair_block_n(false, !w->grouped, row_tiles, w->N, (w->K + 255) / 256 + w->Kop / 64, w->num_sms);
         const int v = bn == 192 ? 0 : bn == 256 ? 1 : 2;
         a.tm_b = w->tm_b2[v];
         a.tm_bo = w->tm_bo2[v];
         a.tm_sfw = (bn == kTiledBN) ? w->tm_sfw_tiled : w->tm_sfw;
-        if (osc_status s = make_tmap_sf(&a.tm_sfa, sfa, (uint64_t)((M + 127) / 128) * (w->K / 128))) return s;
+        const uint64_t sf_row_blocks = w->grouped ? (uint64_t)max_tiles : (uint64_t)((M + 127) / 128);
+        if (osc_status s = make_tmap_sf(&a.tm_sfa, sfa, sf_row_blocks * (w->K / 128))) return s;
         if (osc_status s = make_tmap(&a.tm_y, Y, true, M, (uint64_t)w->N * 2, (uint64_t)ldy * 2, 32)) return s;
         e = launch_gemm_dual_pair(a, bn, st);
     } else {
@@ -418,7 +431,7 @@ osc_status osc_gemm_dual(const osc_weights* w, const void* xq, const void* sfa, 
     if (!w) return fail(OSC_ERR_INVALID_ARG, "weights handle is null");
     if (M < 0) return fail(OSC_ERR_INVALID_ARG, "M = %d is negative", M);
     if (w->grouped) return fail(OSC_ERR_INVALID_ARG, "grouped weights: use osc_linear_grouped");
-    return gemm_impl(w, xq, sfa, xo, M, Y, ldy, nullptr, 0, static_cast<cudaStream_t>(stream));
+    return gemm_impl(w, xq, sfa, xo, M, Y, ldy, nullptr, 0, nullptr, 0, static_cast<cudaStream_t>(stream));
 }
 
 osc_status osc_linear(const osc_weights* w, const void* X, int M, int64_t ldx, void* Y, int64_t ldy,
@@ -437,7 +450,7 @@ osc_status osc_linear(const osc_weights* w, const void* X, int M, int64_t ldx, v
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (osc_status s = quantize_impl(w, X, M, ldx, ws + sz.xq_offset, ws + sz.sfa_offset, ws + sz.xo_offset, nullptr, 0, st)) return s;
-    return gemm_impl(w, ws + sz.xq_offset, ws + sz.sfa_offset, ws + sz.xo_offset, M, Y, ldy, nullptr, 0, st);
+    return gemm_impl(w, ws + sz.xq_offset, ws + sz.sfa_offset, ws + sz.xo_offset, M, Y, ldy, nullptr, 0, nullptr, 0, st);
 }
 
 osc_status osc_linear_grouped(const osc_weights* w, const void* X_perm, const int32_t* off, int M_total, int64_t ldx,
@@ -457,12 +470,15 @@ osc_status osc_linear_grouped(const osc_weights* w, const void* X_perm, const in
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int max_tiles = M_total / 128 + w->E;
+    const int max_tiles2 = max_tiles256(M_total, w->E);
     int32_t* sched = reinterpret_cast<int32_t*>(ws + sz.sched_offset);
-    cudaError_t e = launch_build_sched(off, w->E, sched, max_tiles, st);
+    int32_t* sched2 = use_pair_kernel(true, M_total, w->E) ? sched + sched_ints(max_tiles) : nullptr;
+    cudaError_t e = launch_build_sched(off, w->E, sched, max_tiles, sched2, max_tiles2, st);
     if (e != cudaSuccess) return cuda_fail(e, "build_sched_kernel");
     if (osc_status s = quantize_impl(w, X_perm, M_total, ldx, ws + sz.xq_offset, ws + sz.sfa_offset, ws + sz.xo_offset,
                                      sched, max_tiles, st)) return s;
-    return gemm_impl(w, ws + sz.xq_offset, ws + sz.sfa_offset, ws + sz.xo_offset, M_total, Y, ldy, sched, max_tiles, st);
+    return gemm_impl(w, ws + sz.xq_offset, ws + sz.sfa_offset, ws + sz.xo_offset, M_total, Y, ldy, sched, max_tiles,
+                     sched2, max_tiles2, st);
 }
 
 // ------------------------------------------------------- offline profiling
@@ -521,8 +537,8 @@ static osc_status fp8_prepare_impl(const void* W, int E, int N, int K, int64_t l
     for (int v = 0; v < 4; ++v) {
         if (osc_status s = make_tmap(&w->tm_b[v], w8, false, (uint64_t)E * N, K, K, 64 * (v + 1))) { delete w; return s; }
     }
-    for (int v = 0; v < 2 && !grouped; ++v) {
-        if (osc_status s = make_tmap(&w->tm_b2[v], w8, false, (uint64_t)N, K, K, (v == 0 ? 192 : 256) / 2)) { delete w; return s; }
+    for (int v = 0; v < 2; ++v) {
+        if (osc_status s = make_tmap(&w->tm_b2[v], w8, false, (uint64_t)E * N, K, K, (v == 0 ? 192 : 256) / 2)) { delete w; return s; }
     }
     *out = w;
     return OSC_OK;
@@ -547,7 +563,7 @@ osc_status osc_fp8_act_sizes(const osc_fp8_weights* w, int M, osc_fp8_act_sizes_
     const int64_t max_tiles = w->grouped ? (int64_t)M / 128 + w->E : 0;
     out->x8_bytes = (size_t)M * w->K;
     out->sx_bytes = (size_t)M * 4;
-    out->sched_bytes = w->grouped ? (size_t)(1 + 4 * max_tiles) * 4 : 0;
+    out->sched_bytes = w->grouped ? sched_ints(max_tiles) * 4 + sched_ints(max_tiles256(M, w->E)) * 4 : 0;
     out->x8_offset = 0;
     out->sx_offset = align256(out->x8_bytes);
     out->sched_offset = out->sx_offset + align256(out->sx_bytes);
@@ -569,7 +585,8 @@ osc_status osc_fp8_quantize(const void* X, int M, int K, int64_t ldx, void* x8, 
 }
 
 static osc_status fp8_gemm_impl(const osc_fp8_weights* w, const void* x8, const void* sx, int M, void* Y, int64_t ldy,
-                                const int32_t* sched, int max_tiles, cudaStream_t st) {
+                                const int32_t* sched, int max_tiles, const int32_t* sched2, int max_tiles2,
+                                cudaStream_t st) {
     if (M == 0) return OSC_OK;
     if (!x8 || !sx || !Y) return fail(OSC_ERR_INVALID_ARG, "null device pointer");
     if (ldy < w->N) return fail(OSC_ERR_SHAPE, "ldy = %lld < N = %d", (long long)ldy, w->N);
@@ -586,9 +603,11 @@ static osc_status fp8_gemm_impl(const osc_fp8_weights* w, const void* x8, const 
     a.ldy = ldy;
     a.M = M; a.N = w->N; a.K = w->K; a.Kop = 0;
     a.sched = sched; a.max_tiles = max_tiles; a.num_sms = w->num_sms;
+    a.sched2 = sched2; a.max_tiles2 = max_tiles2;
     cudaError_t e;
-    if (use_pair_kernel(w->grouped, M)) {
-        const int bn = gemm_pair_block_n(true, M, w->N, w->K / 128, w->num_sms);
+    if (use_pair_kernel(w->grouped, M, w->E)) {
+        const long row_tiles = w->grouped ? max_tiles2 - w->E / 2 : (M + 255) / 256;
+        const int bn = gemm_pair_block_n(true, false, row_tiles, w->N, w->K / 128, w->num_sms);
         a.tm_b = w->tm_b2[bn == 256];
         if (osc_status s = make_tmap(&a.tm_y, Y, true, M, (uint64_t)w->N * 2, (uint64_t)ldy * 2, 32)) return s;
         e = launch_gemm_fp8_pair(a, bn, st);
@@ -604,7 +623,7 @@ osc_status osc_fp8_gemm(const osc_fp8_weights* w, const void* x8, const void* sx
     if (!w) return fail(OSC_ERR_INVALID_ARG, "weights handle is null");
     if (M < 0) return fail(OSC_ERR_INVALID_ARG, "M = %d is negative", M);
     if (w->grouped) return fail(OSC_ERR_INVALID_ARG, "grouped weights: use osc_fp8_linear_grouped");
-    return fp8_gemm_impl(w, x8, sx, M, Y, ldy, nullptr, 0, static_cast<cudaStream_t>(stream));
+    return fp8_gemm_impl(w, x8, sx, M, Y, ldy, nullptr, 0, nullptr, 0, static_cast<cudaStream_t>(stream));
 }
 
 static osc_status fp8_linear_impl(const osc_fp8_weights* w, const void* X, const int32_t* off, int M, int64_t ldx,
@@ -620,17 +639,21 @@ static osc_status fp8_linear_impl(const osc_fp8_weights* w, const void* X, const
         return fail(OSC_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", workspace_bytes, sz.workspace_bytes);
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const int32_t* sched = nullptr;
-    int max_tiles = 0;
+    const int32_t *sched = nullptr, *sched2 = nullptr;
+    int max_tiles = 0, max_tiles2 = 0;
     if (w->grouped) {
+        // only the schedule of the GEMM kernel that will run (the FP8 quantizer needs none)
         max_tiles = M / 128 + w->E;
+        max_tiles2 = max_tiles256(M, w->E);
         int32_t* s = reinterpret_cast<int32_t*>(ws + sz.sched_offset);
-        cudaError_t e = launch_build_sched(off, w->E, s, max_tiles, st);
+        const bool pair = use_pair_kernel(true, M, w->E);
+        cudaError_t e = launch_build_sched(off, w->E, pair ? nullptr : s, max_tiles, pair ? s + sched_ints(max_tiles) : nullptr,
+                                           max_tiles2, st);
         if (e != cudaSuccess) return cuda_fail(e, "build_sched_kernel");
-        sched = s;
+        if (pair) sched2 = s + sched_ints(max_tiles); else sched = s;
     }
     if (osc_status s = osc_fp8_quantize(X, M, w->K, ldx, ws + sz.x8_offset, ws + sz.sx_offset, stream)) return s;
-    return fp8_gemm_impl(w, ws + sz.x8_offset, ws + sz.sx_offset, M, Y, ldy, sched, max_tiles, st);
+    return fp8_gemm_impl(w, ws + sz.x8_offset, ws + sz.sx_offset, M, Y, ldy, sched, max_tiles, sched2, max_tiles2, st);
 }
 
 osc_status osc_fp8_linear(const osc_fp8_weights* w, const void* X, int M, int64_t ldx, void* Y, int64_t ldy,

@@ -31,7 +31,8 @@ cudaError_t launch_quant_extract(const CUtensorMap& tm_x, int M, int K, const ui
                                  const int32_t* prefix, const int32_t* idx_o, void* xq, void* sf, void* xo, int Ko, int Kop,
                                  const int32_t* sched, int max_tiles, int num_sms, cudaStream_t st);
 cudaError_t launch_fp8_quant(const void* X, int64_t ldx, int M, int K, void* x8, void* sx, cudaStream_t st);
-cudaError_t launch_build_sched(const int32_t* off, int E, int32_t* sched, int max_tiles, cudaStream_t st);
+cudaError_t launch_build_sched(const int32_t* off, int E, int32_t* sched128, int max_tiles128, int32_t* sched256,
+                               int max_tiles256, cudaStream_t st);
 
 // profile_kernels.cu
 cudaError_t launch_profile(const void* X, int64_t ldx, int S, int K, double alpha, double* sum, int32_t* counts,
@@ -55,18 +56,20 @@ struct GemmArgs {
     int64_t ldy;
     int M;               // rows (dense) / total rows (grouped)
     int N, K, Kop;
-    const int32_t* sched;  // grouped tile schedule or nullptr
+    const int32_t* sched;  // grouped tile schedule (128-row tiles) or nullptr
     int max_tiles;
+    const int32_t* sched2; // grouped tile schedule of the CTA-pair kernel (256-row tiles) or nullptr
+    int max_tiles2;
     int num_sms;
 };
 cudaError_t launch_gemm_dual(const GemmArgs& a, int bn, cudaStream_t st);
 cudaError_t launch_gemm_fp8(const GemmArgs& a, int bn, cudaStream_t st);
 int gemm_block_n(int row_tiles, int N, int num_sms);
 
-// gemm2_kernels.cu (CTA pairs, dense problems)
+// gemm2_kernels.cu (CTA pairs: 256-row tiles, dense or grouped)
 cudaError_t launch_gemm_dual_pair(const GemmArgs& a, int bn, cudaStream_t st);
 cudaError_t launch_gemm_fp8_pair(const GemmArgs& a, int bn, cudaStream_t st);
-int gemm_pair_block_n(bool fp8, int M, int N, int stages, int num_sms);
+int gemm_pair_block_n(bool fp8, bool allow_240, long row_tiles, int N, int stages, int num_sms);
 cudaError_t launch_retile_sf(const uint8_t* src, uint8_t* dst, int N, int K, int bn, cudaStream_t st);
 
 }  // namespace osc

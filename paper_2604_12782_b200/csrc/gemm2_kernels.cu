@@ -1,4 +1,6 @@
-// CTA-pair variant of the tensor-core kernels for dense (non-grouped) problems with many rows.
+// CTA-pair variant of the tensor-core kernels for problems with many rows: dense, or grouped (MoE) with a
+// schedule of 256-row tiles that never cross an expert boundary (rows past the expert's end are computed
+// but not written).
 //
 // Two CTAs of a cluster (two SMs) compute one 256 x BN output tile with `cta_group::2` MMAs:
 // each CTA holds 128 rows of the activation tile and its 128 x BN slice of the fp32 accumulator in
@@ -149,7 +151,8 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
     grid_dependency_wait();   // operands come from the kernel before this one
 
     const int N = args.N, K = args.K;
-    const int num_m = (args.M + 2 * BM - 1) / (2 * BM);
+    const int32_t* __restrict__ sched = args.sched2;
+    const int num_m = sched ? sched[0] : (args.M + 2 * BM - 1) / (2 * BM);
     const int num_n = (N + BN - 1) / BN;
     const int total = num_m * num_n;
     const int elems_per_kb = (MODE == MODE_OSC) ? 256 : 128;
@@ -159,14 +162,29 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
     const int katoms_total = K / 128;
     const int natoms = (N + 127) / 128;
 
-    auto tile_rc = [&](int t, int& row0, int& n0) {
+    // tile t -> first row, column, and (grouped) last valid row, first scale row, expert
+    struct Tile { int row0, n0, row_end, sf_row0, expert; };
+    auto tile_of = [&](int t) {
         const int per_band = BAND * num_n;
         const int band = t / per_band;
         const int rem = t - band * per_band;
         const int m0 = band * BAND;
         const int h = min(BAND, num_m - m0);
-        row0 = (m0 + rem % h) * (2 * BM);
-        n0 = (rem / h) * BN;
+        const int m = m0 + rem % h;
+        Tile ti;
+        ti.n0 = (rem / h) * BN;
+        if (sched) {
+            ti.row0 = sched[1 + m];
+            ti.row_end = sched[1 + args.max_tiles2 + m];
+            ti.sf_row0 = sched[1 + 2 * args.max_tiles2 + m];
+            ti.expert = sched[1 + 3 * args.max_tiles2 + m];
+        } else {
+            ti.row0 = m * (2 * BM);
+            ti.row_end = args.M;
+            ti.sf_row0 = ti.row0;
+            ti.expert = 0;
+        }
+        return ti;
     };
 
     constexpr int LANES = C::LANES;
@@ -181,10 +199,11 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
         uint8_t* ring = smem + L * SPL * C::STAGE_BYTES;
         const uint32_t full0 = map_to_cta(smem_u32(fullL), 0);  // the leader's full barriers of this lane
         for (int t = pair_id + L * num_pairs; t < total; t += LANES * num_pairs) {
-            int row0, n0;
-            tile_rc(t, row0, n0);
-            const int arow = row0 + (int)rank * BM;            // my 128 activation rows
-            const int brow = n0 + (int)rank * (BN / 2);        // my half of the weight rows
+            const Tile ti = tile_of(t);
+            const int n0 = ti.n0;
+            const int arow = ti.row0 + (int)rank * BM;                        // my 128 activation rows
+            const int brow = ti.expert * N + n0 + (int)rank * (BN / 2);       // my half of the weight rows
+            const int sfa_blk = (ti.sf_row0 / 128 + (int)rank) * katoms_total;  // my 128-row scale blocks
             for (int kb = 0; kb < nkb; ++kb) {
                 if (!wait_bounded(&emptyL[s], ph ^ 1u, abort_flag, 11)) goto done;
                 const uint32_t st = smem_u32(ring + s * C::STAGE_BYTES);
@@ -196,11 +215,11 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
                         tma_load_2d_pair(st + A_BYTES, &args.tm_b, fb, kb * ROW_BYTES, brow);
                         if (MODE == MODE_OSC) {
                             // scale blocks: 2 consecutive 512-byte blocks (256 channels) per 128 rows
-                            tma_load_2d_pair(st + A_BYTES + C::B_BYTES, &args.tm_sfa, fb, 0,
-                                             (arow / 128) * katoms_total + 2 * kb);
+                            tma_load_2d_pair(st + A_BYTES + C::B_BYTES, &args.tm_sfa, fb, 0, sfa_blk + 2 * kb);
 #pragma unroll
                             for (int j = 0; j < C::SFB_ATOMS; ++j) {
-                                const int atom = C::TILED_SF ? (n0 / BN) * C::SFB_ATOMS + j : min(n0 / 128 + j, natoms - 1);
+                                const int atom = C::TILED_SF ? (n0 / BN) * C::SFB_ATOMS + j
+                                                             : ti.expert * natoms + min(n0 / 128 + j, natoms - 1);
                                 tma_load_2d_pair(st + A_BYTES + C::B_BYTES + C::SFA_BYTES + j * 1024, &args.tm_sfw, fb, 0,
                                                  atom * katoms_total + 2 * kb);
                             }
@@ -232,9 +251,8 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
             const uint64_t sf_hi = smem_desc_sf(0);
             const uint32_t ring0 = smem_u32(smem + L * SPL * C::STAGE_BYTES);
             for (int t = pair_id + L * num_pairs; t < total; t += LANES * num_pairs) {
-                int row0, n0;
-                tile_rc(t, row0, n0);
-                if (!wait_bounded_cluster(&tempty_bar[acc], acc_ph ^ 1u, abort_flag, 12)) goto done;
+                const int n0 = tile_of(t).n0;
+                if (!wait_bounded(&tempty_bar[acc], acc_ph ^ 1u, abort_flag, 12)) goto done;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * C::ACC_STRIDE);
                 const uint32_t sfb_tm = tmem_base + C::TM_SFB + (C::TILED_SF ? 0u : (uint32_t)((n0 % 128) / 32));
@@ -309,14 +327,30 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
         const uint32_t tempty0 = map_to_cta(smem_u32(&tempty_bar[0]), 0);
         uint8_t* stage_buf = smem + STAGES * C::STAGE_BYTES + (half * 4 + q) * (TPW * EPI_TILE_BYTES);
         for (int t = pair_id; t < total; t += num_pairs) {
-            int row0, n0;
-            tile_rc(t, row0, n0);
-            if (!wait_bounded_cluster(&tfull_bar[acc], acc_ph, abort_flag, 14)) goto done;
-            tc_fence_after();
-            const int wrow0 = row0 + (int)rank * BM + q * 32;  // first row of this warp
+            const Tile ti = tile_of(t);
+            const int n0 = ti.n0;
+            const int wrow0 = ti.row0 + (int)rank * BM + q * 32;  // first row of this warp
             const int row = wrow0 + lane;
+            // FP8 scales, fetched before the wait so that their latency hides behind the K loop: the row's
+            // activation scale, and per slice one coalesced load of the 64 weight scales (lane l holds
+            // columns 2l, 2l+1; the conversion loop below broadcasts them with shuffles)
             float sxr = 1.0f;
-            if (MODE == MODE_FP8 && row < args.M) sxr = args.sx[row];
+            float2 wsc[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+            if (MODE == MODE_FP8) {
+                if (row < ti.row_end) sxr = args.sx[row];
+                const float* swp = args.sw + (int64_t)ti.expert * N;
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    const int col = n0 + (half + u * (EPI_WARPS / 4)) * 64 + 2 * lane;
+                    if (half + u * (EPI_WARPS / 4) < C::SLICES && col + 1 < N)
+                        wsc[u] = *reinterpret_cast<const float2*>(swp + col);
+                }
+            }
+            if (!wait_bounded(&tfull_bar[acc], acc_ph, abort_flag, 14)) goto done;
+            tc_fence_after();
+            // grouped problems: rows past the expert's end belong to the next expert and must not be written,
+            // so a warp whose 32 rows straddle the end writes its staged tiles with row-masked stores
+            const bool clip = sched != nullptr && wrow0 + 32 > ti.row_end;
             if (TPW == 2) {
                 // the stores of the previous tile must be done reading the staging tiles
                 if (lane == 0) tma_store_wait_read<0>();
@@ -326,6 +360,7 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
 #pragma unroll 1
             for (int c = half; c < C::SLICES; c += EPI_WARPS / 4, ++ord) {
                 uint32_t r0[32], r1[32];
+                const float2 wv = ord == 0 ? wsc[0] : wsc[1];
                 const uint32_t tcol = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * C::ACC_STRIDE + c * 64);
                 const bool narrow = (C::LAST_W != 64) && (c == C::SLICES - 1);  // last slice of a 240-wide tile: 48 columns
                 tmem_ld_32x32(tcol, r0);
@@ -348,9 +383,10 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
                             float lo = __uint_as_float(cc < 32 ? r0[cc] : r1[cc - 32]);
                             float hi = __uint_as_float(cc < 32 ? r0[cc + 1] : r1[cc - 31]);
                             if (MODE == MODE_FP8) {
-                                const float2 w2 = *reinterpret_cast<const float2*>(args.sw + col + cc);
-                                lo = lo * (sxr * w2.x);
-                                hi = hi * (sxr * w2.y);
+                                const float wx = __shfl_sync(0xFFFFFFFFu, wv.x, j * 4 + i);
+                                const float wy = __shfl_sync(0xFFFFFFFFu, wv.y, j * 4 + i);
+                                lo = lo * (sxr * wx);
+                                hi = hi * (sxr * wy);
                             }
                             const __nv_bfloat162 b2 = __floats2bfloat162_rn(lo, hi);
                             o[i] = *reinterpret_cast<const uint32_t*>(&b2);
@@ -362,7 +398,7 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
                     if (TPW == 1) {
                         fence_proxy_async_smem();
                         __syncwarp();
-                        if (lane == 0) {
+                        if (lane == 0 && !clip) {
                             tma_store_2d(&args.tm_y, buf, col, wrow0);
                             tma_store_commit();
                         }
@@ -378,12 +414,28 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
                 if (TPW == 2) {
                     int o2 = 0;
                     for (int c = half; c < C::SLICES; c += EPI_WARPS / 4, ++o2)
-                        if (n0 + c * 64 < N && !(C::LAST_W != 64 && c == C::SLICES - 1))
+                        if (!clip && n0 + c * 64 < N && !(C::LAST_W != 64 && c == C::SLICES - 1))
                             tma_store_2d(&args.tm_y, stage_buf + o2 * EPI_TILE_BYTES, n0 + c * 64, wrow0);
                     tma_store_commit();
                 }
             }
             __syncwarp();
+            if (clip && TPW == 2) {
+                int o2 = 0;
+                for (int c = half; c < C::SLICES; c += EPI_WARPS / 4, ++o2) {
+                    if (n0 + c * 64 >= N || (C::LAST_W != 64 && c == C::SLICES - 1)) continue;
+                    const uint8_t* buf = stage_buf + o2 * EPI_TILE_BYTES;
+                    const int j = lane & 7;
+#pragma unroll
+                    for (int rr = 0; rr < 8; ++rr) {
+                        const int rl = rr * 4 + (lane >> 3);
+                        if (wrow0 + rl < ti.row_end)
+                            *reinterpret_cast<uint4*>(args.Y + (int64_t)(wrow0 + rl) * args.ldy + n0 + c * 64 + j * 8) =
+                                *reinterpret_cast<const uint4*>(buf + rl * 128 + ((j ^ (rl & 7)) << 4));
+                    }
+                }
+                __syncwarp();
+            }
             if (C::LAST_W != 64 && TPW == 2) {
                 // the 48-column last slice of a 240-wide tile: row-wise 16-byte stores from the staging tile
                 // (8 lanes per row, 4 rows per instruction), clipped at M and N
@@ -396,7 +448,7 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
                         const int rl = rr * 4 + (lane >> 3);
                         const int orow = wrow0 + rl;
                         const int ocol = n0 + c * 64 + j * 8;
-                        if (j < C::LAST_W / 8 && orow < args.M && ocol < N)
+                        if (j < C::LAST_W / 8 && orow < ti.row_end && ocol < N)
                             *reinterpret_cast<uint4*>(args.Y + (int64_t)orow * args.ldy + ocol) =
                                 *reinterpret_cast<const uint4*>(buf + rl * 128 + ((j ^ (rl & 7)) << 4));
                     }
@@ -431,7 +483,7 @@ static cudaError_t launch_cfg(const GemmArgs& a, cudaStream_t st) {
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    const int total = ((a.M + 2 * BM - 1) / (2 * BM)) * ((a.N + BN - 1) / BN);
+    const int total = a.sched2 ? a.num_sms : ((a.M + 2 * BM - 1) / (2 * BM)) * ((a.N + BN - 1) / BN);
     if (total <= 0) return cudaSuccess;
     cudaLaunchConfig_t cfg = {};
     cfg.blockDim = dim3(C::THREADS);
@@ -474,7 +526,7 @@ static cudaError_t launch_cfg(const GemmArgs& a, cudaStream_t st) {
 // plus the scale columns (epilogue hidden behind the next tile's K loop unless that loop is shorter
 // than the ~2 us drain), 256 has one accumulator (drain and hand-over exposed, ~2.7 us per tile).
 // The FP8 mode needs no scale columns: 256 wide with two accumulators.  OSC_PAIR_BLOCK_N overrides.
-int gemm_pair_block_n(bool fp8, int M, int N, int stages, int num_sms) {
+int gemm_pair_block_n(bool fp8, bool allow_240, long row_tiles, int N, int stages, int num_sms) {
     static int forced = -1;
     if (forced < 0) {
         forced = 0;
@@ -483,9 +535,9 @@ int gemm_pair_block_n(bool fp8, int M, int N, int stages, int num_sms) {
             if (v == 192 || v == 240 || v == 256) forced = v;
         }
     }
-    if (forced && !(fp8 && forced == 240)) return forced;
+    if (forced && !((fp8 || !allow_240) && forced == 240)) return forced;
     const int pairs = num_sms / 2 > 0 ? num_sms / 2 : 1;
-    const long mt = (M + 255) / 256;
+    const long mt = row_tiles;
     const long loop = 370L * stages;
     const long hidden = loop > 2000 ? loop : 2000;
     long best = -1;
@@ -493,7 +545,7 @@ int gemm_pair_block_n(bool fp8, int M, int N, int stages, int num_sms) {
     const int cand[3] = {256, 240, 192};
     for (int i = 0; i < 3; ++i) {
         const int bn = cand[i];
-        if (fp8 && bn == 240) continue;
+        if ((fp8 || !allow_240) && bn == 240) continue;
         const long rounds = (mt * ((N + bn - 1) / bn) + pairs - 1) / pairs;
         const bool two_acc = fp8 || bn != 256;
         const long cost = rounds * (two_acc ? hidden : loop + 2700);

@@ -276,14 +276,28 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
         uint8_t* stage_buf = smem + STAGES * C::STAGE_BYTES + q * C::EPI_WARP_BYTES;
         for (int t = blockIdx.x; t < total; t += gridDim.x) {
             const TileInfo ti = tile_info<BN>(args, t, num_m, num_n);
+            const int wrow0 = ti.row0 + q * 32;
+            // FP8 scales, fetched before the wait so that their latency hides behind the K loop: the row's
+            // activation scale, and per slice one coalesced load of the 64 weight scales (lane l holds
+            // columns 2l, 2l+1; the conversion loop below broadcasts them with shuffles)
+            float sxr = 1.0f;
+            float2 wsc[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+            if (MODE == MODE_FP8) {
+                if (wrow0 + lane < ti.row_end) sxr = args.sx[wrow0 + lane];
+                const float* swp = args.sw + (int64_t)ti.expert * N;
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    const int col = ti.n0 + (half + u * (G_EPI_WARPS / 4)) * 64 + 2 * lane;
+                    if (half + u * (G_EPI_WARPS / 4) < BN / 64 && col + 1 < N)
+                        wsc[u] = *reinterpret_cast<const float2*>(swp + col);
+                }
+            }
             if (!wait_bounded(&tfull_bar[acc], acc_ph, abort_flag, 4)) goto done;
             tc_fence_after();
-            const int wrow0 = ti.row0 + q * 32;
-            float sxr = 1.0f;
-            if (MODE == MODE_FP8 && wrow0 + lane < ti.row_end) sxr = args.sx[wrow0 + lane];
-            const float* swp = (MODE == MODE_FP8) ? args.sw + (int64_t)ti.expert * N : nullptr;
+            int ord = 0;
 #pragma unroll 1
-            for (int c = half; c < BN / 64; c += G_EPI_WARPS / 4) {
+            for (int c = half; c < BN / 64; c += G_EPI_WARPS / 4, ++ord) {
+                const float2 wv = ord == 0 ? wsc[0] : wsc[1];
                 uint32_t r0[32], r1[32];
                 const uint32_t tcol = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + c * 64);
                 tmem_ld_32x32(tcol, r0);
@@ -301,9 +315,10 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
                             float lo = __uint_as_float(cc < 32 ? r0[cc] : r1[cc - 32]);
                             float hi = __uint_as_float(cc < 32 ? r0[cc + 1] : r1[cc - 31]);
                             if (MODE == MODE_FP8) {
-                                const float2 w2 = *reinterpret_cast<const float2*>(swp + col + cc);
-                                lo = lo * (sxr * w2.x);
-                                hi = hi * (sxr * w2.y);
+                                const float wx = __shfl_sync(0xFFFFFFFFu, wv.x, j * 4 + i);
+                                const float wy = __shfl_sync(0xFFFFFFFFu, wv.y, j * 4 + i);
+                                lo = lo * (sxr * wx);
+                                hi = hi * (sxr * wy);
                             }
                             const __nv_bfloat162 b2 = __floats2bfloat162_rn(lo, hi);
                             o[i] = *reinterpret_cast<const uint32_t*>(&b2);

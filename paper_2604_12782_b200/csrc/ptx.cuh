@@ -250,36 +250,12 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
     return r;
 }
+// Arrive on a barrier that may live in the other CTA of the pair.  CTA-scope release on purpose: the
+// barriers of the pair kernel order only tensor-memory traffic (bracketed by tcgen05 fences, with the
+// loads already waited for), never ordinary memory written by one CTA and read by the other, and a
+// cluster-scope release cost ~1400 cycles per arrival on B200.
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ bool wait_bounded_cluster(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
-                                                     int site) {
-    if (mbar_try_wait_cluster(bar, parity)) return true;
-    const long long t0 = clock64();
-    int spins = 0;
-    while (true) {
-        if (mbar_try_wait_cluster(bar, parity)) return true;
-        if ((++spins & 63) == 0) {
-            if (*abort_flag) return false;
-            if (clock64() - t0 > kWaitLimitCycles) {
-                *abort_flag = 1;
-                atomicCAS(&g_dev_status, 0, (site << 8) | 1);
-                return false;
-            }
-        }
-    }
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 // Tiled load into this CTA's shared memory whose byte count is credited to a barrier that may
 // live in the other CTA of the pair (`bar_cluster_addr` is a cluster-window address).

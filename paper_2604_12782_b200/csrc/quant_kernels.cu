@@ -359,34 +359,45 @@ fp8_quant_rows_kernel(const uint16_t* __restrict__ X, int64_t ldx, int M, int K,
 }
 
 // ------------------------------------------------------------ grouped schedule
-// sched[0] = number of 128-row tiles; then four arrays of max_tiles entries:
-// first row, end row (exclusive, the expert's end), first scale row, expert.
-__global__ void build_sched_kernel(const int32_t* __restrict__ off, int E, int32_t* __restrict__ sched,
-                                   int max_tiles) {
+// sched[0] = number of row tiles (tile_rows = 128 or 256 rows each, never crossing an expert boundary);
+// then four arrays of max_tiles entries: first row, end row (exclusive, the expert's end), first scale
+// row (scale rows are padded to 128 per expert whatever the tile height), expert.
+// Block 0 builds the 128-row schedule (if sched is given), block 1 the 256-row one (if sched2 is given).
+__global__ void build_sched_kernel(const int32_t* __restrict__ off, int E, int32_t* __restrict__ sched128,
+                                   int max_tiles128, int32_t* __restrict__ sched256, int max_tiles256) {
     __shared__ int s_tiles[1024];
+    __shared__ int s_sfbase[1024];
     grid_launch_dependents();
     grid_dependency_wait();
     const int tid = threadIdx.x;
+    const bool tall = blockIdx.x == 1 || sched128 == nullptr;
+    int32_t* sched = tall ? sched256 : sched128;
+    const int max_tiles = tall ? max_tiles256 : max_tiles128;
+    const int tile_rows = tall ? 256 : 128;
+    if (sched == nullptr) return;
     // serial prefix by one thread: E is small (hundreds) and this runs once per call
     if (tid == 0) {
-        int acc = 0;
+        int acc = 0, sfacc = 0;
         for (int e = 0; e < E; ++e) {
             s_tiles[e] = acc;
-            acc += (off[e + 1] - off[e] + 127) / 128;
+            s_sfbase[e] = sfacc;
+            const int m = off[e + 1] - off[e];
+            acc += (m + tile_rows - 1) / tile_rows;
+            sfacc += (m + 127) / 128 * 128;
         }
         sched[0] = acc < max_tiles ? acc : max_tiles;
     }
     __syncthreads();
     for (int e = tid; e < E; e += blockDim.x) {
         const int m = off[e + 1] - off[e];
-        const int nt = (m + 127) / 128;
+        const int nt = (m + tile_rows - 1) / tile_rows;
         const int t0 = s_tiles[e];
         for (int i = 0; i < nt; ++i) {
             const int t = t0 + i;
             if (t < max_tiles) {
-                sched[1 + t] = off[e] + i * 128;
+                sched[1 + t] = off[e] + i * tile_rows;
                 sched[1 + max_tiles + t] = off[e + 1];
-                sched[1 + 2 * max_tiles + t] = t * 128;
+                sched[1 + 2 * max_tiles + t] = s_sfbase[e] + i * tile_rows;
                 sched[1 + 3 * max_tiles + t] = e;
             }
         }
@@ -457,8 +468,12 @@ cudaError_t launch_fp8_quant(const void* X, int64_t ldx, int M, int K, void* x8,
                       static_cast<uint8_t*>(x8), static_cast<float*>(sx));
 }
 
-cudaError_t launch_build_sched(const int32_t* off, int E, int32_t* sched, int max_tiles, cudaStream_t st) {
-    return launch_pdl(build_sched_kernel, dim3(1), dim3(256), 0, st, off, E, sched, max_tiles);
+cudaError_t launch_build_sched(const int32_t* off, int E, int32_t* sched128, int max_tiles128, int32_t* sched256,
+                               int max_tiles256, cudaStream_t st) {
+    const int blocks = (sched128 != nullptr) + (sched256 != nullptr);
+    if (blocks == 0) return cudaSuccess;
+    return launch_pdl(build_sched_kernel, dim3(blocks), dim3(256), 0, st, off, E, sched128, max_tiles128, sched256,
+                      max_tiles256);
 }
 
 }  // namespace osc

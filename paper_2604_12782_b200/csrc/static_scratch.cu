@@ -60,5 +60,5 @@ extern "C" osc_status osc_linear_static(const osc_weights* w, const void* X, int
     // (codes and gathered channels of all M rows, pad columns, whole scale blocks incl. rows past M).
     if (osc_status s = quantize_impl(w, X, M, ldx, ws + sz.xq_offset, ws + sz.sfa_offset, ws + sz.xo_offset, nullptr, 0, st))
         return s;
-    return gemm_impl(w, ws + sz.xq_offset, ws + sz.sfa_offset, ws + sz.xo_offset, M, Y, ldy, nullptr, 0, st);
+    return gemm_impl(w, ws + sz.xq_offset, ws + sz.sfa_offset, ws + sz.xo_offset, M, Y, ldy, nullptr, 0, nullptr, 0, st);
 }

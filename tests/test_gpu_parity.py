@@ -230,15 +230,20 @@ def test_fp8_linear_within_tolerance(B, oracle, M, N, K, seed):
 
 
 def grouped_counts(kind):
+    """"small" averages under 96 rows per expert (128-row tiles, single-CTA kernel); "mid" and "zipf" run on the
+    CTA-pair kernel with 256-row tiles: experts ending inside the first / second half of a tile, on a tile edge,
+    empty experts, one-row experts."""
     if kind == "small":
         return np.array([3, 0, 130, 1, 257, 128])
+    if kind == "mid":
+        return np.array([300, 0, 5, 256, 129, 511, 1, 385])
     return synth.zipf_expert_rows(E=16, T=512, top_k=4, seed=1)
 
 
-@pytest.mark.parametrize("kind", ["small", "zipf"])
+@pytest.mark.parametrize("kind", ["small", "mid", "zipf"])
 def test_grouped_osc_linear(B, oracle, kind):
     counts = grouped_counts(kind)
-    E, K, N = counts.size, 256, 192
+    E, K, N = counts.size, 256, (320 if kind == "mid" else 192)
     c = synth.moe_gate_up_case(E, counts, K=K, N=N, seed=3)
     M = c["M"]
     w = B.osc_prepare_weights_grouped(dev_bf16(c["W"].reshape(E * N, K)).view(E, N, K), c["lut"])
@@ -270,9 +275,10 @@ def test_grouped_osc_linear(B, oracle, kind):
         assert_within_tolerance(Yh[r0:r1], Yref, T, f"grouped expert {e}")
 
 
-def test_grouped_fp8_linear(B, oracle):
-    counts = grouped_counts("small")
-    E, K, N = counts.size, 384, 128
+@pytest.mark.parametrize("kind", ["small", "mid"])
+def test_grouped_fp8_linear(B, oracle, kind):
+    counts = grouped_counts(kind)
+    E, K, N = counts.size, 384, (320 if kind == "mid" else 128)
     c = synth.moe_down_case(E, counts, K=K, N=N, seed=4)
     M = c["M"]
     w = B.osc_fp8_prepare_weights_grouped(dev_bf16(c["W"].reshape(E * N, K)).view(E, N, K))
