@@ -8,7 +8,8 @@ host memory; bf16 tensors are uint16 bit patterns.
 Function-to-paper map (details in the C file):
   quantize_extract / prepare_weights  Algorithm 2 (+ Section 3.3 weight split)
   gemm_dual / linear                   Eq. 5
-  fp8_quantize / fp8_gemm / fp8_linear Section 3.4 fallback
+  fp8_quantize / fp8_gemm / fp8_linear Section 3.4 fallback (per-token E4M3)
+  mxfp8_quantize / mxfp8_gemm / mxfp8_linear   Section 3.4 fallback in its 8-bit micro-scaling form (MXFP8)
   threshold / profile_indexing / clustering_density   Eq. 1-4, Algorithm 1 (offline profiling)
 """
 from __future__ import annotations
@@ -49,6 +50,7 @@ def lib():
         _lib.osc_ref_sf_bytes.restype = C.c_int64
         _lib.osc_ref_sf_bytes.argtypes = [C.c_int64, C.c_int64]
         _lib.osc_ref_sf_row_base.restype = C.c_int64
+        _lib.osc_ref_e8m0_from_amax_emax.argtypes = [C.c_double, C.c_int]
         _lib.osc_ref_threshold.restype = C.c_double
         _lib.osc_ref_threshold.argtypes = [C.c_void_p, C.c_int64, C.c_int, C.c_int, C.c_double]
         _lib.osc_ref_threshold_bits.restype = C.c_uint32
@@ -208,6 +210,40 @@ def fp8_linear(X: np.ndarray, W: np.ndarray, rows=None):
     w8, sw = fp8_quantize(W)
     Y, T = fp8_gemm(x8, sx, w8, sw, rows)
     return Y, T, (x8, sx), (w8, sw)
+
+
+def e8m0_from_amax_emax(a: float, emax: int) -> int:
+    return int(lib().osc_ref_e8m0_from_amax_emax(float(a), int(emax)))
+
+
+def mxfp8_quantize(X: np.ndarray):
+    """MXFP8 (E4M3 elements, E8M0 scale per 32) of bf16 rows X [M,K] -> (x8 [M,K] u8, sf u8 in block layout)."""
+    X = np.ascontiguousarray(X, dtype=np.uint16)
+    M, K = X.shape
+    x8 = np.zeros((M, K), np.uint8)
+    sf = np.zeros(sf_bytes(M, K), np.uint8)
+    lib().osc_ref_mxfp8_quantize(_p(X), C.c_int64(K), M, K, _p(x8), _p(sf))
+    return x8, sf
+
+
+def mxfp8_gemm(x8, sfa, w8, sfw, rows=None):
+    M, K = x8.shape
+    N = w8.shape[0]
+    if rows is None:
+        rows = np.arange(M, dtype=np.int32)
+    rows = np.ascontiguousarray(rows, dtype=np.int32)
+    Y = np.zeros((rows.size, N), np.float64)
+    T = np.zeros((rows.size, N), np.float64)
+    lib().osc_ref_mxfp8_gemm_rows(_p(np.ascontiguousarray(x8)), _p(np.ascontiguousarray(sfa)), _p(rows), rows.size,
+                                  _p(np.ascontiguousarray(w8)), _p(np.ascontiguousarray(sfw)), N, K, _p(Y), _p(T))
+    return Y, T
+
+
+def mxfp8_linear(X: np.ndarray, W: np.ndarray, rows=None):
+    x8, sfa = mxfp8_quantize(X)
+    w8, sfw = mxfp8_quantize(W)
+    Y, T = mxfp8_gemm(x8, sfa, w8, sfw, rows)
+    return Y, T, (x8, sfa), (w8, sfw)
 
 
 def threshold(X: np.ndarray, alpha: float = 5.0) -> float:

@@ -27,7 +27,9 @@
  * Pins (tests/test_oracle_*.py): E2M1/E4M3 tables against an independent
  * library codec, closed-form scale codes, the worked 32-element vectors under
  * tests/golden/, empty-table and full-table reductions against a numpy double
- * GEMM, brute force on tiny shapes, restoration identity, error ordering.
+ * GEMM, brute force on tiny shapes, restoration identity, error ordering;
+ * the MXFP8 fallback against a numpy + library-codec restatement, its own worked
+ * group and a dense product of the dequantized operands.
  * Unpinned: nothing in this file (the paper's accuracy tables are out of scope).
  */
 #include <math.h>
@@ -373,6 +375,91 @@ int osc_ref_fp8_gemm_rows(const uint8_t* x8, const float* sx, const int32_t* row
         free(w);
     }
     free(a);
+    return 0;
+}
+
+/* ------------------------- MXFP8 fallback (Section 3.4; Section 4 "Implementation Details") */
+
+/* The 8-bit micro-scaling form of the W2 fallback: groups of 32 along K share an
+ * E8M0 scale 2^(floor(log2 amax) - emax) with emax(E4M3) = 8 (OCP MX v1.0, MXFP8
+ * E4M3), elements are E4M3 with round-to-nearest-even and saturation at 448.
+ * No channel is extracted: the fallback applies to inputs whose outliers are
+ * diffuse.  Scales go to the same 128 x 4 block layout as the MXFP4 scales. */
+int osc_ref_e8m0_from_amax_emax(double amax, int emax) {
+    if (isnan(amax) || isinf(amax)) return 0xFF;
+    if (amax == 0.0) return 0;
+    int ex;
+    (void)frexp(amax, &ex); /* floor(log2 amax) = ex - 1 */
+    int code = (ex - 1) - emax + 127;
+    if (code < 0) code = 0;
+    if (code > 254) code = 254;
+    return code;
+}
+
+int osc_ref_mxfp8_quantize(const uint16_t* X, int64_t ldx, int M, int K, uint8_t* x8, uint8_t* sf) {
+    int Kg = K / G;
+#pragma omp parallel for schedule(static)
+    for (int m = 0; m < M; ++m) {
+        const uint16_t* xrow = X + (int64_t)m * ldx;
+        for (int g = 0; g < Kg; ++g) {
+            double amax = 0.0;
+            for (int c = g * G; c < (g + 1) * G; ++c) {
+                double a = fabs(bf16_value(xrow[c]));
+                if (a > amax || isnan(a)) amax = a;
+            }
+            int code = osc_ref_e8m0_from_amax_emax(amax, 8);
+            sf[osc_ref_sf_index(m, g, K)] = (uint8_t)code;
+            for (int c = g * G; c < (g + 1) * G; ++c) {
+                double v = ldexp(bf16_value(xrow[c]), 127 - code); /* exact: power-of-two scaling */
+                x8[(int64_t)m * K + c] = (uint8_t)osc_ref_e4m3_encode(v);
+            }
+        }
+    }
+    return 0;
+}
+
+/* Y[i][n] = sum_g 2^(sa-127) 2^(sw-127) sum_{c in g} a[c] w[c] over E4M3 elements;
+ * T = the same with absolute values.  Products are exact in double. */
+int osc_ref_mxfp8_gemm_rows(const uint8_t* x8, const uint8_t* sfa, const int32_t* rows, int nrows,
+                            const uint8_t* w8, const uint8_t* sfw, int N, int K, double* Y, double* T) {
+    int Kg = K / G;
+    double* a = (double*)malloc(sizeof(double) * (size_t)nrows * (size_t)(K > 0 ? K : 1));
+    int* sa = (int*)malloc(sizeof(int) * (size_t)nrows * (size_t)(Kg > 0 ? Kg : 1));
+    for (int i = 0; i < nrows; ++i) {
+        int64_t r = rows[i];
+        for (int c = 0; c < K; ++c) a[(int64_t)i * K + c] = osc_ref_e4m3_decode(x8[r * K + c]);
+        for (int g = 0; g < Kg; ++g) sa[(int64_t)i * Kg + g] = sfa[osc_ref_sf_index(r, g, K)];
+    }
+#pragma omp parallel
+    {
+        double* w = (double*)malloc(sizeof(double) * (size_t)(K > 0 ? K : 1));
+        int* sw = (int*)malloc(sizeof(int) * (size_t)(Kg > 0 ? Kg : 1));
+#pragma omp for schedule(static)
+        for (int n = 0; n < N; ++n) {
+            for (int c = 0; c < K; ++c) w[c] = osc_ref_e4m3_decode(w8[(int64_t)n * K + c]);
+            for (int g = 0; g < Kg; ++g) sw[g] = sfw[osc_ref_sf_index(n, g, K)];
+            for (int i = 0; i < nrows; ++i) {
+                const double* ai = a + (int64_t)i * K;
+                const int* sai = sa + (int64_t)i * Kg;
+                double acc = 0.0, tot = 0.0;
+                for (int g = 0; g < Kg; ++g) {
+                    double p = 0.0, q = 0.0;
+                    for (int c = g * G; c < (g + 1) * G; ++c) {
+                        double pr = ai[c] * w[c];
+                        p += pr;
+                        q += fabs(pr);
+                    }
+                    int e = sai[g] + sw[g] - 254;
+                    acc += ldexp(p, e);
+                    tot += ldexp(q, e);
+                }
+                Y[(int64_t)i * N + n] = acc;
+                T[(int64_t)i * N + n] = tot;
+            }
+        }
+        free(w); free(sw);
+    }
+    free(a); free(sa);
     return 0;
 }
 
