@@ -230,6 +230,34 @@ class Fp8Problem:
                             self.Y[j])
 
 
+class Mxfp8Problem:
+    """The fallback in its 8-bit micro-scaling form (MXFP8): same interface as Fp8Problem."""
+
+    def __init__(self, torch, B, case, nsets):
+        self.B, self.M, self.K, self.N = B, case["M"], case["K"], case["N"]
+        X0, W0 = dev_bf16(torch, case["X"]), dev_bf16(torch, case["W"])
+        self.X = [X0 if i == 0 else torch.roll(X0, 97 * i, 0).contiguous() for i in range(nsets)]
+        self.w = [B.osc_mxfp8_prepare_weights(W0 if i == 0 else torch.roll(W0, 61 * i, 0).contiguous())
+                  for i in range(nsets)]
+        self.sz = B.osc_mxfp8_act_sizes(self.w[0], self.M)
+        self.ws = [torch.empty(self.sz.workspace_bytes, dtype=torch.uint8, device="cuda") for _ in range(nsets)]
+        self.Y = [torch.empty(self.M, self.N, dtype=torch.bfloat16, device="cuda") for _ in range(nsets)]
+        self.n = nsets
+
+    def step(self, i):
+        j = i % self.n
+        self.B.osc_mxfp8_linear(self.w[j], self.X[j], self.Y[j], self.ws[j])
+
+    def quant(self, i):
+        j = i % self.n
+        self.B.osc_mxfp8_quantize(self.X[j], self.ws[j][self.sz.x8_offset:], self.ws[j][self.sz.sfa_offset:])
+
+    def gemm(self, i):
+        j = i % self.n
+        self.B.osc_mxfp8_gemm(self.w[j], self.ws[j][self.sz.x8_offset:], self.ws[j][self.sz.sfa_offset:], self.M,
+                              self.Y[j])
+
+
 def time_loop(torch, fn, steps, warmup):
     """Average milliseconds per call of fn(i) over `steps` calls, CUDA events on the current stream."""
     for i in range(warmup):
@@ -401,7 +429,12 @@ def run_sweep(args):
     rows = []
     steps, warm = args.steps, args.warmup
 
+    def want(name):
+        return not args.sweep_only or args.sweep_only in name
+
     def osc_row(name, M, K, N, cpg, seed=0):
+        if not want(name):
+            return
         case = synth.osc_linear_case(seed, M, K, N, cpg)
         nsets = NSETS if M >= 1024 else 8
         p = OscProblem(torch, B, case, nsets)
@@ -422,6 +455,8 @@ def run_sweep(args):
         torch.cuda.empty_cache()
 
     def fp8_row(name, M, K, N, seed=0):
+        if not want(name):
+            return
         case = synth.fp8_linear_case(seed, M, K, N)
         nsets = NSETS if M >= 1024 else 8
         f8 = Fp8Problem(torch, B, case, nsets)
@@ -435,11 +470,31 @@ def run_sweep(args):
         del f8
         torch.cuda.empty_cache()
 
+    def mxfp8_row(name, M, K, N, seed=0):
+        if not want(name):
+            return
+        case = synth.fp8_linear_case(seed, M, K, N)
+        nsets = NSETS if M >= 1024 else 8
+        p8 = Mxfp8Problem(torch, B, case, nsets)
+        ms8 = time_loop(torch, p8.step, steps, warm)
+        q8, g8 = time_split(torch, p8, steps)
+        B.osc_sync_check()
+        # same FLOPs and FP8 peak as the per-token form; bytes: X, W8 + its scales, Y (+ the two-kernel intermediates
+        # are implementation traffic, not counted)
+        byts = 2.0 * M * K + N * K * (1 + 1 / 32) + 2.0 * M * N
+        troof = max(roofline.fp8_flops(M, N, K) / peaks["fp8"], byts / peaks["hbm"])
+        rows.append({"name": name, "M": M, "K": K, "N": N, "ms": ms8, "quant_ms": q8, "gemm_ms": g8,
+                     "tflops": roofline.fp8_flops(M, N, K) / ms8 / 1e9, "pct_roofline": 100 * troof / (ms8 * 1e-3),
+                     "roof_us": troof * 1e6, "quant_gbs": (2.0 * M * K + M * K * (1 + 1 / 32)) / q8 / 1e6})
+        del p8
+        torch.cuda.empty_cache()
+
     for M in (16, 128, 2048, 8192):
         osc_row("qkv", M, 4096, 6144, 2)
     for M in (128, 2048, 8192):
         osc_row("gate_up", M, 4096, 24576, 1)
         fp8_row("down_fp8", M, 12288, 4096)
+        mxfp8_row("down_mxfp8", M, 12288, 4096)
     osc_row("layer.qkv", 4096, 4096, 6144, 2)
     osc_row("layer.o_proj", 4096, 4096, 4096, 1)
     osc_row("layer.gate_up", 4096, 4096, 24576, 1)
@@ -498,6 +553,7 @@ def main():
     ap.add_argument("--cpu-rows", type=int, default=1024, help="activation rows of the cpu_baseline sample")
     ap.add_argument("--ref-rows", type=int, default=128, help="activation rows per step of --impl reference")
     ap.add_argument("--sweep", action="store_true")
+    ap.add_argument("--sweep-only", default="", help="with --sweep: only the rows whose name contains this text")
     ap.add_argument("--only-osc", action="store_true",
                     help="skip the e2e, FP8 and cpu legs (short runs under a profiler; prints no bench line)")
     args = ap.parse_args()

@@ -210,6 +210,54 @@ osc_status osc_fp8_linear_grouped(const osc_fp8_weights* w, const void* X_perm, 
                                   int M_total, int64_t ldx, void* Y, int64_t ldy, void* workspace,
                                   size_t workspace_bytes, void* stream);
 
+/* ------------------------------------- MXFP8 form of the fallback (Section 3.4) */
+
+/* Section 3.4 allows "FP8 (or equivalent 8-bit micro-scaling formats)" for the W2 inputs and Section 4
+ * ("Implementation Details") states that the experiments fall back to MXFP8.  This group of calls is that
+ * form: E4M3 elements with one E8M0 scale per 32 channels along K (OCP MX v1.0: scale =
+ * 2^(floor(log2 amax) - 8), i.e. code = max(biased exponent of amax - 8, 0); elements rounded to nearest
+ * even, saturating at 448), for activations (online) and weights (offline) alike, no channel extracted.
+ * Scales use the same 128 x 4 block layout as the MXFP4 scales (see osc_quantize_extract):
+ * ceil(rows/128) * (K/128) * 512 bytes; bytes of rows past the end are written as 0.
+ * Dense problems only (no grouped variant).  Same conventions as the other calls: device pointers,
+ * 16-byte alignment, leading dimensions in elements and multiples of 8, asynchronous on `stream`,
+ * no allocation, M == 0 is a successful no-op, K % 128 == 0, N % 64 == 0. */
+typedef struct osc_mxfp8_weights osc_mxfp8_weights;
+
+typedef struct {
+    size_t w8_bytes;        /* N * K */
+    size_t sfw_bytes;       /* ceil(N/128) * (K/128) * 512 */
+} osc_mxfp8_weight_sizes_t;
+
+typedef struct {
+    size_t x8_bytes;        /* M * K */
+    size_t sfa_bytes;       /* ceil(M/128) * (K/128) * 512 */
+    size_t x8_offset;       /* placement inside the workspace of osc_mxfp8_linear */
+    size_t sfa_offset;
+    size_t workspace_bytes;
+} osc_mxfp8_act_sizes_t;
+
+osc_status osc_mxfp8_weight_sizes(int N, int K, osc_mxfp8_weight_sizes_t* out);
+
+/* Offline: w8 [N,K] E4M3 bytes and sfw (block layout) from W (dev bf16 [N, ldw]).  The handle borrows
+ * w8 and sfw, which must outlive it; the caller owns every buffer. */
+osc_status osc_mxfp8_prepare_weights(const void* W, int N, int K, int64_t ldw, void* w8, void* sfw, void* stream,
+                                     osc_mxfp8_weights** out);
+osc_status osc_mxfp8_weights_destroy(osc_mxfp8_weights* w);
+osc_status osc_mxfp8_act_sizes(const osc_mxfp8_weights* w, int M, osc_mxfp8_act_sizes_t* out);
+
+/* Online: x8 [M,K] bytes and sfa (block layout) from X (dev bf16 [M, ldx]). */
+osc_status osc_mxfp8_quantize(const void* X, int M, int K, int64_t ldx, void* x8, void* sfa, void* stream);
+
+/* Y[m,n] = bf16(sum_g 2^(sfa[m,g]-127) 2^(sfw[n,g]-127) sum_{k in g} x8[m,k] w8[n,k]), fp32 accumulation
+ * on the block-scaled tensor-core path. */
+osc_status osc_mxfp8_gemm(const osc_mxfp8_weights* w, const void* x8, const void* sfa, int M, void* Y, int64_t ldy,
+                          void* stream);
+
+/* quantize + gemm through a caller-provided workspace of at least osc_mxfp8_act_sizes().workspace_bytes. */
+osc_status osc_mxfp8_linear(const osc_mxfp8_weights* w, const void* X, int M, int64_t ldx, void* Y, int64_t ldy,
+                            void* workspace, size_t workspace_bytes, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -47,6 +47,14 @@ class Fp8ActSizes(C.Structure):
                                           "sched_offset", "workspace_bytes")]
 
 
+class Mxfp8WeightSizes(C.Structure):
+    _fields_ = [("w8_bytes", C.c_size_t), ("sfw_bytes", C.c_size_t)]
+
+
+class Mxfp8ActSizes(C.Structure):
+    _fields_ = [(n, C.c_size_t) for n in ("x8_bytes", "sfa_bytes", "x8_offset", "sfa_offset", "workspace_bytes")]
+
+
 _vp, _i, _i64, _sz = C.c_void_p, C.c_int, C.c_int64, C.c_size_t
 _SIGS = {
     "osc_status_string": (C.c_char_p, [_i]),
@@ -72,6 +80,13 @@ _SIGS = {
     "osc_fp8_gemm": (_i, [_vp, _vp, _vp, _i, _vp, _i64, _vp]),
     "osc_fp8_linear": (_i, [_vp, _vp, _i, _i64, _vp, _i64, _vp, _sz, _vp]),
     "osc_fp8_linear_grouped": (_i, [_vp, _vp, _vp, _i, _i64, _vp, _i64, _vp, _sz, _vp]),
+    "osc_mxfp8_weight_sizes": (_i, [_i, _i, C.POINTER(Mxfp8WeightSizes)]),
+    "osc_mxfp8_prepare_weights": (_i, [_vp, _i, _i, _i64, _vp, _vp, _vp, C.POINTER(_vp)]),
+    "osc_mxfp8_weights_destroy": (_i, [_vp]),
+    "osc_mxfp8_act_sizes": (_i, [_vp, _i, C.POINTER(Mxfp8ActSizes)]),
+    "osc_mxfp8_quantize": (_i, [_vp, _i, _i, _i64, _vp, _vp, _vp]),
+    "osc_mxfp8_gemm": (_i, [_vp, _vp, _vp, _i, _vp, _i64, _vp]),
+    "osc_mxfp8_linear": (_i, [_vp, _vp, _i, _i64, _vp, _i64, _vp, _sz, _vp]),
 }
 for _name, (_res, _args) in _SIGS.items():
     _f = getattr(_lib, _name)
@@ -150,6 +165,10 @@ class OscWeights(_Handle):
 
 class Fp8Weights(_Handle):
     _destroy = staticmethod(_lib.osc_fp8_weights_destroy)
+
+
+class Mxfp8Weights(_Handle):
+    _destroy = staticmethod(_lib.osc_mxfp8_weights_destroy)
 
 
 def _alloc(nbytes, dev):
@@ -302,3 +321,48 @@ def osc_fp8_linear_grouped(w: Fp8Weights, X: torch.Tensor, off: torch.Tensor, Y:
     _check(_lib.osc_fp8_linear_grouped(w.ptr, _ptr(X), _ptr(off), M, X.stride(0) if M else w.K, _ptr(Y),
                                        Y.stride(0) if M else w.N, _ptr(workspace),
                                        workspace.numel() * workspace.element_size(), _stream(stream)))
+
+
+# ------------------------------------------------------------- MXFP8 form of the fallback
+
+def osc_mxfp8_weight_sizes(N: int, K: int) -> Mxfp8WeightSizes:
+    out = Mxfp8WeightSizes()
+    _check(_lib.osc_mxfp8_weight_sizes(N, K, C.byref(out)))
+    return out
+
+
+def osc_mxfp8_prepare_weights(W: torch.Tensor, stream=None) -> Mxfp8Weights:
+    N, K = W.shape
+    sz = osc_mxfp8_weight_sizes(N, K)
+    bufs = {"w8": _alloc(sz.w8_bytes, W.device), "sfw": _alloc(sz.sfw_bytes, W.device)}
+    h = _vp()
+    _check(_lib.osc_mxfp8_prepare_weights(_ptr(W), N, K, W.stride(0), _ptr(bufs["w8"]), _ptr(bufs["sfw"]),
+                                          _stream(stream), C.byref(h)))
+    w = Mxfp8Weights(h.value, bufs)
+    w.N, w.K, w.sizes = N, K, sz
+    return w
+
+
+def osc_mxfp8_weights_destroy(w: Mxfp8Weights):
+    w.close()
+
+
+def osc_mxfp8_act_sizes(w: Mxfp8Weights, M: int) -> Mxfp8ActSizes:
+    out = Mxfp8ActSizes()
+    _check(_lib.osc_mxfp8_act_sizes(w.ptr, M, C.byref(out)))
+    return out
+
+
+def osc_mxfp8_quantize(X: torch.Tensor, x8, sfa, stream=None):
+    M, K = X.shape
+    _check(_lib.osc_mxfp8_quantize(_ptr(X), M, K, X.stride(0) if M else K, _ptr(x8), _ptr(sfa), _stream(stream)))
+
+
+def osc_mxfp8_gemm(w: Mxfp8Weights, x8, sfa, M: int, Y: torch.Tensor, stream=None):
+    _check(_lib.osc_mxfp8_gemm(w.ptr, _ptr(x8), _ptr(sfa), M, _ptr(Y), Y.stride(0) if M else w.N, _stream(stream)))
+
+
+def osc_mxfp8_linear(w: Mxfp8Weights, X: torch.Tensor, Y: torch.Tensor, workspace: torch.Tensor, stream=None):
+    M = X.shape[0]
+    _check(_lib.osc_mxfp8_linear(w.ptr, _ptr(X), M, X.stride(0) if M else w.K, _ptr(Y), Y.stride(0) if M else w.N,
+                                 _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)))

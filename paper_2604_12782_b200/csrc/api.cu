@@ -98,14 +98,15 @@ static osc_status make_tmap_x(CUtensorMap* tm, const void* base, uint64_t rows, 
     return OSC_OK;
 }
 
-// Scale-factor buffer as [blocks, 128] uint32 (512-byte blocks), tiles of 2 consecutive blocks.
-static osc_status make_tmap_sf(CUtensorMap* tm, const void* base, uint64_t blocks) {
+// Scale-factor buffer as [blocks, 128] uint32 (512-byte blocks), tiles of `box_blocks` consecutive blocks
+// (2 = the 256 FP4 channels of a GEMM stage, 1 = the 128 FP8 channels).
+static osc_status make_tmap_sf(CUtensorMap* tm, const void* base, uint64_t blocks, uint32_t box_blocks = 2) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return fail(OSC_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
     if (blocks == 0) blocks = 1;
     cuuint64_t gdim[2] = {128, blocks};
     cuuint64_t gstr[1] = {512};
-    cuuint32_t box[2] = {128, 2};
+    cuuint32_t box[2] = {128, box_blocks};
     cuuint32_t estr[2] = {1, 1};
     CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void*>(base), gdim, gstr, box, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -198,6 +199,14 @@ struct osc_fp8_weights {
     const float* sw;
     int num_sms;
     CUtensorMap tm_b[4], tm_b2[2];
+};
+
+struct osc_mxfp8_weights {
+    int N, K;
+    const uint8_t *w8, *sfw;
+    int num_sms;
+    CUtensorMap tm_b2[2];  // half tiles for 192- and 256-wide tiles
+    CUtensorMap tm_sfw;
 };
 
 extern "C" {
@@ -666,6 +675,110 @@ osc_status osc_fp8_linear_grouped(const osc_fp8_weights* w, const void* X_perm, 
                                   void* stream) {
     if (w && !w->grouped) return fail(OSC_ERR_INVALID_ARG, "dense weights: use osc_fp8_linear");
     return fp8_linear_impl(w, X_perm, off, M_total, ldx, Y, ldy, workspace, workspace_bytes, stream);
+}
+
+// ------------------------------------------------- MXFP8 form of the fallback
+
+osc_status osc_mxfp8_weight_sizes(int N, int K, osc_mxfp8_weight_sizes_t* out) {
+    if (!out) return fail(OSC_ERR_INVALID_ARG, "out is null");
+    if (osc_status s = check_nk(1, N, K)) return s;
+    out->w8_bytes = (size_t)N * K;
+    out->sfw_bytes = sf_bytes(N, K);
+    return OSC_OK;
+}
+
+osc_status osc_mxfp8_quantize(const void* X, int M, int K, int64_t ldx, void* x8, void* sfa, void* stream) {
+    if (M < 0) return fail(OSC_ERR_INVALID_ARG, "M = %d is negative", M);
+    if (K <= 0 || K % 128) return fail(OSC_ERR_SHAPE, "K = %d must be a positive multiple of 128", K);
+    if (M == 0) return OSC_OK;
+    if (!X || !x8 || !sfa) return fail(OSC_ERR_INVALID_ARG, "null device pointer");
+    if (ldx < K) return fail(OSC_ERR_SHAPE, "ldx = %lld < K", (long long)ldx);
+    if (ldx % 8 || !aligned16(X) || !aligned16(x8) || !aligned16(sfa))
+        return fail(OSC_ERR_ALIGN, "pointers must be 16-byte aligned and ldx a multiple of 8");
+    cudaError_t e = launch_mxfp8_quant(X, ldx, M, K, x8, sfa, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(e, "mxfp8_quant_kernel");
+    return OSC_OK;
+}
+
+osc_status osc_mxfp8_prepare_weights(const void* W, int N, int K, int64_t ldw, void* w8, void* sfw, void* stream,
+                                     osc_mxfp8_weights** out) {
+    if (!out) return fail(OSC_ERR_INVALID_ARG, "out is null");
+    *out = nullptr;
+    if (osc_status s = check_nk(1, N, K)) return s;
+    DeviceInfo di;
+    if (osc_status s = device_info(&di)) return s;
+    if (osc_status s = osc_mxfp8_quantize(W, N, K, ldw, w8, sfw, stream)) return s;
+    osc_mxfp8_weights* w = new (std::nothrow) osc_mxfp8_weights();
+    if (!w) return fail(OSC_ERR_INVALID_ARG, "out of host memory");
+    w->N = N; w->K = K;
+    w->w8 = static_cast<const uint8_t*>(w8);
+    w->sfw = static_cast<const uint8_t*>(sfw);
+    w->num_sms = di.num_sms;
+    osc_status s = OSC_OK;
+    for (int v = 0; v < 2 && s == OSC_OK; ++v) s = make_tmap(&w->tm_b2[v], w8, false, (uint64_t)N, K, K, (v == 0 ? 192 : 256) / 2);
+    if (s == OSC_OK) s = make_tmap_sf(&w->tm_sfw, sfw, (uint64_t)sf_bytes(N, K) / 512, 1);
+    if (s != OSC_OK) { delete w; return s; }
+    *out = w;
+    return OSC_OK;
+}
+osc_status osc_mxfp8_weights_destroy(osc_mxfp8_weights* w) {
+    delete w;
+    return OSC_OK;
+}
+
+osc_status osc_mxfp8_act_sizes(const osc_mxfp8_weights* w, int M, osc_mxfp8_act_sizes_t* out) {
+    if (!w || !out) return fail(OSC_ERR_INVALID_ARG, "null argument");
+    if (M < 0) return fail(OSC_ERR_INVALID_ARG, "M = %d is negative", M);
+    out->x8_bytes = (size_t)M * w->K;
+    out->sfa_bytes = sf_bytes(M, w->K);
+    out->x8_offset = 0;
+    out->sfa_offset = align256(out->x8_bytes);
+    out->workspace_bytes = out->sfa_offset + align256(out->sfa_bytes);
+    return OSC_OK;
+}
+
+osc_status osc_mxfp8_gemm(const osc_mxfp8_weights* w, const void* x8, const void* sfa, int M, void* Y, int64_t ldy,
+                          void* stream) {
+    if (!w) return fail(OSC_ERR_INVALID_ARG, "weights handle is null");
+    if (M < 0) return fail(OSC_ERR_INVALID_ARG, "M = %d is negative", M);
+    if (M == 0) return OSC_OK;
+    if (!x8 || !sfa || !Y) return fail(OSC_ERR_INVALID_ARG, "null device pointer");
+    if (ldy < w->N) return fail(OSC_ERR_SHAPE, "ldy = %lld < N = %d", (long long)ldy, w->N);
+    if (ldy % 8 || !aligned16(Y) || !aligned16(x8) || !aligned16(sfa))
+        return fail(OSC_ERR_ALIGN, "pointers must be 16-byte aligned and ldy a multiple of 8");
+    GemmArgs a;
+    memset(&a, 0, sizeof a);
+    if (osc_status s = make_tmap(&a.tm_a, x8, false, M, w->K, w->K, 128)) return s;
+    // every M runs on the CTA-pair kernel (256-row tiles); rows past M are zero-filled by the loads and never stored
+    const int bn = gemm_pair_block_n(false, false, (M + 255) / 256, w->N, w->K / 128, w->num_sms);
+    a.tm_b = w->tm_b2[bn == 256];
+    a.tm_sfw = w->tm_sfw;
+    if (osc_status s = make_tmap_sf(&a.tm_sfa, sfa, (uint64_t)sf_bytes(M, w->K) / 512, 1)) return s;
+    if (osc_status s = make_tmap(&a.tm_y, Y, true, M, (uint64_t)w->N * 2, (uint64_t)ldy * 2, 32)) return s;
+    a.sfa = static_cast<const uint8_t*>(sfa);
+    a.sfw = w->sfw;
+    a.Y = static_cast<uint16_t*>(Y);
+    a.ldy = ldy;
+    a.M = M; a.N = w->N; a.K = w->K; a.Kop = 0;
+    a.num_sms = w->num_sms;
+    cudaError_t e = launch_gemm_mxf8_pair(a, bn, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(e, "gemm_pair_kernel(mxfp8)");
+    return OSC_OK;
+}
+
+osc_status osc_mxfp8_linear(const osc_mxfp8_weights* w, const void* X, int M, int64_t ldx, void* Y, int64_t ldy,
+                            void* workspace, size_t workspace_bytes, void* stream) {
+    if (!w) return fail(OSC_ERR_INVALID_ARG, "weights handle is null");
+    if (M < 0) return fail(OSC_ERR_INVALID_ARG, "M = %d is negative", M);
+    if (M == 0) return OSC_OK;
+    osc_mxfp8_act_sizes_t sz;
+    osc_mxfp8_act_sizes(w, M, &sz);
+    if (!workspace || !aligned16(workspace)) return fail(OSC_ERR_ALIGN, "workspace must be non-null and 16-byte aligned");
+    if (workspace_bytes < sz.workspace_bytes)
+        return fail(OSC_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", workspace_bytes, sz.workspace_bytes);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    if (osc_status s = osc_mxfp8_quantize(X, M, w->K, ldx, ws + sz.x8_offset, ws + sz.sfa_offset, stream)) return s;
+    return osc_mxfp8_gemm(w, ws + sz.x8_offset, ws + sz.sfa_offset, M, Y, ldy, stream);
 }
 
 }  // extern "C"

@@ -31,6 +31,7 @@ cudaError_t launch_quant_extract(const CUtensorMap& tm_x, int M, int K, const ui
                                  const int32_t* prefix, const int32_t* idx_o, void* xq, void* sf, void* xo, int Ko, int Kop,
                                  const int32_t* sched, int max_tiles, int num_sms, cudaStream_t st);
 cudaError_t launch_fp8_quant(const void* X, int64_t ldx, int M, int K, void* x8, void* sx, cudaStream_t st);
+cudaError_t launch_mxfp8_quant(const void* X, int64_t ldx, int M, int K, void* x8, void* sf, cudaStream_t st);
 cudaError_t launch_build_sched(const int32_t* off, int E, int32_t* sched128, int max_tiles128, int32_t* sched256,
                                int max_tiles256, cudaStream_t st);
 
@@ -69,6 +70,7 @@ int gemm_block_n(int row_tiles, int N, int num_sms);
 // gemm2_kernels.cu (CTA pairs: 256-row tiles, dense or grouped)
 cudaError_t launch_gemm_dual_pair(const GemmArgs& a, int bn, cudaStream_t st);
 cudaError_t launch_gemm_fp8_pair(const GemmArgs& a, int bn, cudaStream_t st);
+cudaError_t launch_gemm_mxf8_pair(const GemmArgs& a, int bn, cudaStream_t st);
 int gemm_pair_block_n(bool fp8, bool allow_240, long row_tiles, int N, int stages, int num_sms);
 cudaError_t launch_retile_sf(const uint8_t* src, uint8_t* dst, int N, int K, int bn, cudaStream_t st);
 

@@ -33,6 +33,7 @@ namespace pair {
 
 constexpr int MODE_OSC = 0;
 constexpr int MODE_FP8 = 1;
+constexpr int MODE_MXF8 = 2;   // block-scaled FP8 (MXFP8): scales as in MODE_OSC, no BF16 branch
 constexpr int BM = 128;        // rows per CTA; the pair covers 256
 constexpr int ROW_BYTES = 128;
 constexpr int A_BYTES = BM * ROW_BYTES;
@@ -50,13 +51,16 @@ struct Cfg {
     static constexpr bool TILED_SF = (BN % 64) != 0;
     // 128-row scale blocks a BN-wide tile can touch
     static constexpr int SFB_ATOMS = TILED_SF ? (BN + 127) / 128 : ((BN % 128 == 0) ? BN / 128 : BN / 128 + 1);
-    static constexpr int SF_COLS = (MODE == MODE_OSC) ? 8 + 2 * SFB_ATOMS * 4 : 0;  // TMEM columns of one stage's scales
+    static constexpr bool SCALED = MODE != MODE_FP8;
+    // 128-channel scale blocks per stage and operand row block: a stage is 128 bytes per row = 256 FP4 or 128 FP8 channels
+    static constexpr int KA = (MODE == MODE_OSC) ? 2 : 1;
+    static constexpr int SF_COLS = SCALED ? KA * (4 + SFB_ATOMS * 4) : 0;  // TMEM columns of one stage's scales
     static constexpr int ACC_STAGES = (2 * BN + SF_COLS <= TMEM_COLS) ? 2 : 1;
     static constexpr int SF_BUFS = (ACC_STAGES * BN + 2 * SF_COLS <= TMEM_COLS) ? 2 : 1;
     static constexpr int B_BYTES = (BN / 2) * ROW_BYTES;
-    static constexpr int SFA_BYTES = (MODE == MODE_OSC) ? 1024 : 0;
-    static constexpr int SFB_BYTES = (MODE == MODE_OSC) ? SFB_ATOMS * 1024 : 0;
-    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + SFA_BYTES + SFB_BYTES;
+    static constexpr int SFA_BYTES = SCALED ? KA * 512 : 0;
+    static constexpr int SFB_BYTES = SCALED ? SFB_ATOMS * KA * 512 : 0;
+    static constexpr int STAGE_BYTES = (A_BYTES + B_BYTES + SFA_BYTES + SFB_BYTES + 1023) / 1024 * 1024;
     static constexpr int LANES = 1;                      // issue lanes (a second one brought nothing, see above)
     static constexpr int THREADS = 32 * (2 * LANES + EPI_WARPS);
     static constexpr int EPI_FIRST_WARP = 2 * LANES;
@@ -74,13 +78,13 @@ struct Cfg {
     // weight scales at 496..511).
     static constexpr int ACC_STRIDE = TILED_SF ? 256 : BN;
     static constexpr int TM_SFA = TILED_SF ? BN : ACC_STAGES * BN;
-    static constexpr int TM_SFB = TILED_SF ? 256 + BN : TM_SFA + 8;
+    static constexpr int TM_SFB = TILED_SF ? 256 + BN : TM_SFA + 4 * KA;
     static constexpr int TM_SF_STRIDE = SF_COLS;         // columns of one scale buffer (when there are two)
     static constexpr uint32_t TX_A = 2u * (A_BYTES + B_BYTES + SFA_BYTES + SFB_BYTES);  // both CTAs, Path A
     static constexpr uint32_t TX_B = 2u * (A_BYTES + B_BYTES);                          // both CTAs, Path B / FP8
     static_assert(STAGE_BYTES % 1024 == 0, "stage must keep 1024-byte alignment");
     static_assert(B_BYTES % 1024 == 0, "weight half-tile must keep 1024-byte alignment");
-    static_assert(TILED_SF ? (TM_SFA + 8 <= 256 && TM_SFB + 2 * SFB_ATOMS * 4 <= TMEM_COLS && SF_BUFS == 1)
+    static_assert(TILED_SF ? (TM_SFA + 4 * KA <= 256 && TM_SFB + KA * SFB_ATOMS * 4 <= TMEM_COLS && SF_BUFS == 1)
                            : (TM_SFA + SF_BUFS * SF_COLS <= TMEM_COLS), "TMEM budget");
     static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
     static_assert(SPL >= 3, "ring too shallow");
@@ -129,10 +133,10 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
         prefetch_tmap(&args.tm_a);
         prefetch_tmap(&args.tm_b);
         prefetch_tmap(&args.tm_y);
-        if (MODE == MODE_OSC) {
+        if (C::SCALED) {
             prefetch_tmap(&args.tm_sfa);
             prefetch_tmap(&args.tm_sfw);
-            if (args.Kop > 0) {
+            if (MODE == MODE_OSC && args.Kop > 0) {
                 prefetch_tmap(&args.tm_ao);
                 prefetch_tmap(&args.tm_bo);
             }
@@ -155,7 +159,7 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
     const int num_m = sched ? sched[0] : (args.M + 2 * BM - 1) / (2 * BM);
     const int num_n = (N + BN - 1) / BN;
     const int total = num_m * num_n;
-    const int elems_per_kb = (MODE == MODE_OSC) ? 256 : 128;
+    const int elems_per_kb = (MODE == MODE_OSC) ? 256 : 128;  // channels in 128 bytes of an operand row
     const int nkb_a = (K + elems_per_kb - 1) / elems_per_kb;
     const int nkb_b = (MODE == MODE_OSC) ? args.Kop / 64 : 0;
     const int nkb = nkb_a + nkb_b;
@@ -210,18 +214,18 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
                 const uint32_t fb = full0 + (uint32_t)s * 8u;
                 if (elect_one()) {
                     if (kb < nkb_a) {
-                        if (rank == 0) mbar_arrive_expect_tx(&fullL[s], MODE == MODE_OSC ? C::TX_A : C::TX_B);
+                        if (rank == 0) mbar_arrive_expect_tx(&fullL[s], C::SCALED ? C::TX_A : C::TX_B);
                         tma_load_2d_pair(st, &args.tm_a, fb, kb * ROW_BYTES, arow);
                         tma_load_2d_pair(st + A_BYTES, &args.tm_b, fb, kb * ROW_BYTES, brow);
-                        if (MODE == MODE_OSC) {
-                            // scale blocks: 2 consecutive 512-byte blocks (256 channels) per 128 rows
-                            tma_load_2d_pair(st + A_BYTES + C::B_BYTES, &args.tm_sfa, fb, 0, sfa_blk + 2 * kb);
+                        if (C::SCALED) {
+                            // scale blocks: KA consecutive 512-byte blocks (128 channels each) per 128 rows
+                            tma_load_2d_pair(st + A_BYTES + C::B_BYTES, &args.tm_sfa, fb, 0, sfa_blk + C::KA * kb);
 #pragma unroll
                             for (int j = 0; j < C::SFB_ATOMS; ++j) {
                                 const int atom = C::TILED_SF ? (n0 / BN) * C::SFB_ATOMS + j
                                                              : ti.expert * natoms + min(n0 / 128 + j, natoms - 1);
-                                tma_load_2d_pair(st + A_BYTES + C::B_BYTES + C::SFA_BYTES + j * 1024, &args.tm_sfw, fb, 0,
-                                                 atom * katoms_total + 2 * kb);
+                                tma_load_2d_pair(st + A_BYTES + C::B_BYTES + C::SFA_BYTES + j * (C::KA * 512), &args.tm_sfw,
+                                                 fb, 0, atom * katoms_total + C::KA * kb);
                             }
                         }
                     } else {
@@ -245,7 +249,9 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
             int acc = (LANES == 2) ? L : 0;
             uint64_t* fullL = full_bar + L * SPL;
             uint64_t* emptyL = empty_bar + L * SPL;
-            constexpr uint32_t IDESC_A = (MODE == MODE_OSC) ? idesc_mxf4(2 * BM, BN) : idesc_e4m3(2 * BM, BN);
+            constexpr uint32_t IDESC_A = (MODE == MODE_OSC)    ? idesc_mxf4(2 * BM, BN)
+                                         : (MODE == MODE_MXF8) ? idesc_mxf8(2 * BM, BN)
+                                                               : idesc_e4m3(2 * BM, BN);
             constexpr uint32_t IDESC_B = idesc_bf16(2 * BM, BN);
             const uint64_t desc_hi = smem_desc_sw128(0);  // everything but the start address
             const uint64_t sf_hi = smem_desc_sf(0);
@@ -291,6 +297,19 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
                         } else if (MODE == MODE_OSC) {
 #pragma unroll
                             for (int k = 0; k < 4; ++k) mma_f16_pair(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC_B, 1u);
+                        } else if (MODE == MODE_MXF8) {
+                            // one 128-channel scale block per stage: four K = 32 instructions, scale byte k of the column
+                            const uint64_t sfa_d = sf_hi | (uint64_t)((sbase + A_BYTES + C::B_BYTES) >> 4);
+                            const uint64_t sfb_d = sf_hi | (uint64_t)((sbase + A_BYTES + C::B_BYTES + C::SFA_BYTES) >> 4);
+                            const uint32_t sfo = (uint32_t)(C::SF_BUFS == 2 ? (kb & 1) : 0) * C::TM_SF_STRIDE;
+                            tc_copy_sf_pair(tmem_base + sfo + C::TM_SFA, sfa_d);
+#pragma unroll
+                            for (int j = 0; j < C::SFB_ATOMS; ++j)
+                                tc_copy_sf_pair(tmem_base + sfo + C::TM_SFB + j * 4, sfb_d + (uint64_t)(j * 32));
+#pragma unroll
+                            for (int k = 0; k < 4; ++k)
+                                mma_mxf8_pair(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC_A | idesc_sf_ids(k, k),
+                                              tmem_base + sfo + C::TM_SFA, sfb_tm + sfo, (kb | k) ? 1u : 0u);
                         } else {
 #pragma unroll
                             for (int k = 0; k < 4; ++k)
@@ -558,6 +577,10 @@ cudaError_t launch_gemm_dual_pair(const GemmArgs& a, int bn, cudaStream_t st) {
     if (bn == 192) return pair::launch_cfg<pair::MODE_OSC, 192>(a, st);
     if (bn == 240) return pair::launch_cfg<pair::MODE_OSC, 240>(a, st);
     return pair::launch_cfg<pair::MODE_OSC, 256>(a, st);
+}
+cudaError_t launch_gemm_mxf8_pair(const GemmArgs& a, int bn, cudaStream_t st) {
+    if (bn == 192) return pair::launch_cfg<pair::MODE_MXF8, 192>(a, st);
+    return pair::launch_cfg<pair::MODE_MXF8, 256>(a, st);
 }
 cudaError_t launch_gemm_fp8_pair(const GemmArgs& a, int bn, cudaStream_t st) {
     if (bn == 192) return pair::launch_cfg<pair::MODE_FP8, 192>(a, st);

@@ -358,6 +358,77 @@ fp8_quant_rows_kernel(const uint16_t* __restrict__ X, int64_t ldx, int M, int K,
     }
 }
 
+// ------------------------------------------------ MXFP8 (E4M3 elements, E8M0 scale per 32)
+// The 8-bit micro-scaling form of the fallback (Section 3.4).  One warp per row; per step the warp
+// reads 512 contiguous bytes (256 channels, 16 bytes per lane), so four neighbouring lanes hold one
+// 32-channel group: amax by two shuffles, scale code = biased exponent of amax - 8 (floored at 0),
+// exact power-of-two scaling in fp32, hardware E4M3 rounding, 8 bytes stored per lane (256
+// contiguous bytes per warp).  The scale bytes of four consecutive groups are one 32-bit word of the
+// 128 x 4 block layout; lanes 0 and 16 gather and store them.  Rows between M and the next multiple
+// of 128 only get zero scale bytes, so that the GEMM never reads an uninitialised scale block.
+constexpr int MX8_ROWS_PER_CTA = 8;
+
+__global__ void __launch_bounds__(32 * MX8_ROWS_PER_CTA)
+mxfp8_quant_kernel(const uint16_t* __restrict__ X, int64_t ldx, int M, int M_pad, int K, uint8_t* __restrict__ x8,
+                   uint8_t* __restrict__ sf) {
+    grid_launch_dependents();
+    grid_dependency_wait();
+    const int lane = threadIdx.x & 31;
+    const int r = blockIdx.x * MX8_ROWS_PER_CTA + (threadIdx.x >> 5);
+    if (r >= M_pad) return;
+    const int katoms = K / 128;
+    // scale word of (row r, 128-channel block a): block (r/128)*katoms + a, word (r%32)*4 + (r%128)/32
+    uint32_t* sf_row = reinterpret_cast<uint32_t*>(sf + (size_t)(r / 128) * katoms * 512) + (r & 31) * 4 + ((r & 127) >> 5);
+    if (r >= M) {
+        for (int a = lane; a < katoms; a += 32) sf_row[(size_t)a * 128] = 0u;
+        return;
+    }
+    const uint4* xrow = reinterpret_cast<const uint4*>(X + (int64_t)r * ldx);
+    uint2* orow = reinterpret_cast<uint2*>(x8 + (int64_t)r * K);
+    const int nch = K / 8;  // 16-byte chunks in the row
+    constexpr int U = 4;    // independent loads in flight per lane
+    for (int c0 = 0; c0 < nch; c0 += 32 * U) {
+        uint4 v[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int c = c0 + u * 32 + lane;
+            v[u] = (c < nch) ? xrow[c] : make_uint4(0u, 0u, 0u, 0u);
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int c = c0 + u * 32 + lane;
+            if (c0 + u * 32 >= nch) break;  // warp-uniform
+            const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+            uint32_t am = 0;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) am = max(am, max(w[i] & 0x7FFFu, (w[i] >> 16) & 0x7FFFu));
+            am = max(am, __shfl_xor_sync(0xFFFFFFFFu, am, 1));
+            am = max(am, __shfl_xor_sync(0xFFFFFFFFu, am, 2));
+            const int ex = (int)(am >> 7);
+            int code = max(ex - 8, 0);
+            if (ex == 255) code = 255;
+            const float inv = __uint_as_float((uint32_t)(254 - min(code, 253)) << 23);
+            uint32_t h[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float lo = __uint_as_float(w[i] << 16) * inv;
+                const float hi = __uint_as_float(w[i] & 0xFFFF0000u) * inv;
+                h[i] = e4m3x2(lo, hi) & 0xFFFFu;
+            }
+            if (c < nch) orow[c] = make_uint2(h[0] | (h[1] << 16), h[2] | (h[3] << 16));
+            // groups 0-3 of this step live in lanes 0,4,8,12 and groups 4-7 in lanes 16,20,24,28
+            const int base = lane & 16;
+            const uint32_t b0 = __shfl_sync(0xFFFFFFFFu, (uint32_t)code, base);
+            const uint32_t b1 = __shfl_sync(0xFFFFFFFFu, (uint32_t)code, base + 4);
+            const uint32_t b2 = __shfl_sync(0xFFFFFFFFu, (uint32_t)code, base + 8);
+            const uint32_t b3 = __shfl_sync(0xFFFFFFFFu, (uint32_t)code, base + 12);
+            const int a = (c0 + u * 32) / 16 + (lane >> 4);  // 128-channel block of this half-warp
+            if ((lane & 15) == 0 && a < katoms) sf_row[(size_t)a * 128] = b0 | (b1 << 8) | (b2 << 16) | (b3 << 24);
+        }
+    }
+}
+
+
 // ------------------------------------------------------------ grouped schedule
 // sched[0] = number of row tiles (tile_rows = 128 or 256 rows each, never crossing an expert boundary);
 // then four arrays of max_tiles entries: first row, end row (exclusive, the expert's end), first scale
@@ -466,6 +537,14 @@ cudaError_t launch_fp8_quant(const void* X, int64_t ldx, int M, int K, void* x8,
     }
     return launch_pdl(fp8_quant_kernel, dim3(M), dim3(F8_THREADS), 0, st, static_cast<const uint16_t*>(X), ldx, M, K,
                       static_cast<uint8_t*>(x8), static_cast<float*>(sx));
+}
+
+cudaError_t launch_mxfp8_quant(const void* X, int64_t ldx, int M, int K, void* x8, void* sf, cudaStream_t st) {
+    if (M <= 0) return cudaSuccess;
+    const int M_pad = (M + 127) / 128 * 128;
+    return launch_pdl(mxfp8_quant_kernel, dim3((M_pad + MX8_ROWS_PER_CTA - 1) / MX8_ROWS_PER_CTA),
+                      dim3(32 * MX8_ROWS_PER_CTA), 0, st, static_cast<const uint16_t*>(X), ldx, M, M_pad, K,
+                      static_cast<uint8_t*>(x8), static_cast<uint8_t*>(sf));
 }
 
 cudaError_t launch_build_sched(const int32_t* off, int E, int32_t* sched128, int max_tiles128, int32_t* sched256,
