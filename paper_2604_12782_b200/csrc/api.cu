@@ -127,6 +127,16 @@ static bool use_pair_kernel(bool grouped, int M, int E) {
     return grouped ? (M / E >= 96) : (M > 128);
 }
 
+// Dense problems with few rows run on the few-row kernel (operands swapped, K split over a cluster): up to 32
+// rows always, up to 64 rows when there are more 128-feature tiles than SMs (measured on B200: with 48 tiles
+// and 64 rows the 128-row-tile kernel is still ahead).  OSC_DECODE=0 disables, OSC_DECODE=2 forces it up to 64 rows.
+static bool use_decode_kernel(bool grouped, int M, int N, int num_sms) {
+    const char* e = getenv("OSC_DECODE");   // read per call: tests switch it inside one process
+    const int mode = e ? atoi(e) : 1;
+    if (mode == 0 || grouped || M > 64) return false;
+    return mode == 2 || M <= 32 || (N + 127) / 128 >= num_sms;
+}
+
 // ----------------------------------------------------------------- the table
 struct Table {
     int Ko = 0, Kop = 0;
@@ -402,6 +412,24 @@ static osc_status gemm_impl(const osc_weights* w, const void* xq, const void* sf
         return fail(OSC_ERR_ALIGN, "pointers must be 16-byte aligned and ldy a multiple of 8");
     GemmArgs a;
     memset(&a, 0, sizeof a);
+    if (use_decode_kernel(w->grouped, M, w->N, w->num_sms)) {
+        if (osc_status s = make_tmap(&a.tm_a, xq, false, M, w->K / 2, w->K / 2, 64)) return s;
+        a.tm_b = w->tm_b[1];
+        if (w->Kop > 0) {
+            if (osc_status s = make_tmap(&a.tm_ao, xo, true, M, (uint64_t)w->Kop * 2, (uint64_t)w->Kop * 2, 64)) return s;
+            a.tm_bo = w->tm_bo[1];
+        }
+        a.sfa = static_cast<const uint8_t*>(sfa);
+        a.sfw = w->sfw;
+        a.Y = static_cast<uint16_t*>(Y);
+        a.ldy = ldy;
+        a.M = M; a.N = w->N; a.K = w->K; a.Kop = w->Kop;
+        a.num_sms = w->num_sms;
+        const int S = gemm_decode_split(w->N, (w->K + 255) / 256 + w->Kop / 64, w->num_sms);
+        cudaError_t e = launch_gemm_dual_decode(a, S, st);
+        if (e != cudaSuccess) return cuda_fail(e, "gemm_decode_kernel(dual)");
+        return OSC_OK;
+    }
     if (osc_status s = make_tmap(&a.tm_a, xq, false, M, w->K / 2, w->K / 2, 128)) return s;
     const int bn1 = gemm_block_n(sched ? max_tiles : (M + 127) / 128, w->N, w->num_sms);
     a.tm_b = w->tm_b[bn1 / 64 - 1];
@@ -603,6 +631,20 @@ static osc_status fp8_gemm_impl(const osc_fp8_weights* w, const void* x8, const 
         return fail(OSC_ERR_ALIGN, "pointers must be 16-byte aligned and ldy a multiple of 8");
     GemmArgs a;
     memset(&a, 0, sizeof a);
+    if (use_decode_kernel(w->grouped, M, w->N, w->num_sms)) {
+        if (osc_status s = make_tmap(&a.tm_a, x8, false, M, w->K, w->K, 64)) return s;
+        a.tm_b = w->tm_b[1];
+        a.sx = static_cast<const float*>(sx);
+        a.sw = w->sw;
+        a.Y = static_cast<uint16_t*>(Y);
+        a.ldy = ldy;
+        a.M = M; a.N = w->N; a.K = w->K; a.Kop = 0;
+        a.num_sms = w->num_sms;
+        const int S = gemm_decode_split(w->N, w->K / 128, w->num_sms);
+        cudaError_t e = launch_gemm_fp8_decode(a, S, st);
+        if (e != cudaSuccess) return cuda_fail(e, "gemm_decode_kernel(fp8)");
+        return OSC_OK;
+    }
     if (osc_status s = make_tmap(&a.tm_a, x8, false, M, w->K, w->K, 128)) return s;
     const int bn1 = gemm_block_n(sched ? max_tiles : (M + 127) / 128, w->N, w->num_sms);
     a.tm_b = w->tm_b[bn1 / 64 - 1];

@@ -1,0 +1,393 @@
+// Few-row ("decode") variant of the tensor-core kernels: M <= 64 activation rows, dense weights.
+//
+// With a handful of tokens the linear layer streams its weights once and is bound by HBM bandwidth and
+// by latency, not by the tensor cores (the memory-bound column of the paper's efficiency table,
+// M = 16-64).  The roles of the operands are swapped: a CTA owns 128 OUTPUT FEATURES (weight rows), which
+// become the 128 rows of the MMA, and the tokens become its N dimension (16..64), so no tensor-core row
+// is spent on padding and a stage moves 16 KB of weights for 2-8 KB of activations.  To put every SM on
+// the weight stream, the K loop of one 128-feature tile is split over the S CTAs of a thread-block
+// cluster; each CTA accumulates its K slice in its own TMEM, parks the fp32 partial tile in its shared
+// memory, and after a cluster barrier every CTA adds, in rank order, the partials of its share of the
+// tokens through distributed shared memory (deterministic, no global scratch, no atomics) and writes
+// those bf16 outputs.
+//
+// The weight tiles do not depend on the kernel that quantized the activations, so the producer issues
+// its first ring of weight loads BEFORE the programmatic-dependency wait: the weight stream overlaps the
+// activation quantizer.
+//
+//   warp 0    : TMA producer          warp 1 : MMA issuer, TMEM owner        warps 2-5 : epilogue
+// Modes and K-block order are those of the other GEMM kernels (Path A block-scaled FP4 blocks, then the
+// BF16 blocks of Path B; or E4M3 blocks with per-row scales applied in the epilogue).
+#include <cuda_bf16.h>
+
+#include "common.cuh"
+
+namespace osc {
+
+namespace decode {
+
+constexpr int MODE_OSC = 0;
+constexpr int MODE_FP8 = 1;
+constexpr int BF = 128;                 // output features per CTA = MMA rows = TMEM lanes
+constexpr int MAX_TOK = 64;             // activation rows per call
+constexpr int ROW_BYTES = 128;
+constexpr int W_BYTES = BF * ROW_BYTES;        // 16 KB of weights per stage
+constexpr int X_BYTES = MAX_TOK * ROW_BYTES;   // 8 KB of activations per stage
+constexpr int THREADS = 192;
+constexpr int TMEM_COLS = 128;          // accumulator (<= 64 columns) + scale columns
+constexpr int TM_SFW = 64;              // weight scales: 2 K blocks x 4 columns
+constexpr int TM_SFX = 72;              // activation scales
+constexpr int MAX_CLUSTER = 8;
+constexpr int PSTR = MAX_TOK + 4;       // row stride (floats) of a parked partial tile
+
+template <int MODE>
+struct Cfg {
+    static constexpr int SF_BYTES = (MODE == MODE_OSC) ? 1024 : 0;   // per operand and stage
+    static constexpr int STAGE_BYTES = W_BYTES + X_BYTES + 2 * SF_BYTES;
+    static constexpr int STAGES = 4;   // ~105 KB per CTA: the CTAs of two consecutive launches share an SM, so the
+                                       // next call's weight loads overlap this call's reduction and stores
+    static constexpr int PARTIAL_BYTES = BF * PSTR * 4;               // aliases the first stages once the MMAs are done
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+    static_assert(STAGE_BYTES % 1024 == 0, "stage must keep 1024-byte alignment");
+    static_assert(PARTIAL_BYTES <= STAGES * STAGE_BYTES, "partial tile must fit in the ring");
+    static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
+};
+
+__device__ __forceinline__ uint32_t cluster_size() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ float4 ld_cluster_f32x4(uint32_t cluster_addr) {
+    float4 v;
+    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+                 : "r"(cluster_addr)
+                 : "memory");
+    return v;
+}
+
+template <int MODE>
+__global__ void __launch_bounds__(THREADS, 2) gemm_decode_kernel(const __grid_constant__ GemmArgs args) {
+    using C = Cfg<MODE>;
+    constexpr int STAGES = C::STAGES;
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * C::STAGE_BYTES);
+    uint64_t* full_bar = bars;
+    uint64_t* empty_bar = bars + STAGES;
+    uint64_t* tfull_bar = bars + 2 * STAGES;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 1);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = __shfl_sync(0xFFFFFFFFu, (int)(threadIdx.x >> 5), 0);
+    const int lane = threadIdx.x & 31;
+    const int S = (int)cluster_size();
+    const int rank = __shfl_sync(0xFFFFFFFFu, (int)cluster_ctarank(), 0);
+    const int tile = blockIdx.x / S;
+    const int n0 = tile * BF;             // first output feature of this cluster
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < STAGES; ++i) {
+            mbar_init(&full_bar[i], 1);
+            mbar_init(&empty_bar[i], 1);
+        }
+        mbar_init(tfull_bar, 1);
+        *abort_flag = 0;
+        fence_barrier_init();
+        prefetch_tmap(&args.tm_a);
+        prefetch_tmap(&args.tm_b);
+        if (MODE == MODE_OSC && args.Kop > 0) {
+            prefetch_tmap(&args.tm_ao);
+            prefetch_tmap(&args.tm_bo);
+        }
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = __shfl_sync(0xFFFFFFFFu, *tmem_slot, 0);
+    grid_launch_dependents();
+
+    const int N = args.N, K = args.K, M = args.M;
+    const int ntok = (M + 15) / 16 * 16;                       // MMA N
+    const int elems_per_kb = (MODE == MODE_OSC) ? 256 : 128;
+    const int nkb_a = (K + elems_per_kb - 1) / elems_per_kb;
+    const int nkb_b = (MODE == MODE_OSC) ? args.Kop / 64 : 0;
+    const int nkb = nkb_a + nkb_b;
+    const int katoms_total = K / 128;
+    // my K slice: blocks [kb0, kb1) of the tile's K loop
+    const int per = (nkb + S - 1) / S;
+    const int kb0 = min(nkb, rank * per);
+    const int kb1 = min(nkb, kb0 + per);
+    float acc[MAX_TOK];
+    const int q = warp & 3;                 // TMEM lane quarter an epilogue warp may read
+    const int f = q * 32 + lane;            // my feature inside the tile
+    float* partial = reinterpret_cast<float*>(smem);
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        // weights (and their scales) of the first ring before the dependency wait, activations after it
+        auto expect = [&](int kb, int s) {
+            uint32_t bytes = W_BYTES + X_BYTES;
+            if (MODE == MODE_OSC && kb < nkb_a) bytes += 2u * 512u * (uint32_t)min(2, katoms_total - 2 * kb);
+            mbar_arrive_expect_tx(&full_bar[s], bytes);
+        };
+        auto load_w = [&](int kb, int s) {
+            uint8_t* st = smem + s * C::STAGE_BYTES;
+            if (kb < nkb_a) {
+                tma_load_2d(st, &args.tm_b, &full_bar[s], kb * ROW_BYTES, n0);
+                if (MODE == MODE_OSC) {
+                    const int ka = min(2, katoms_total - 2 * kb);
+                    const uint8_t* sw = args.sfw + ((int64_t)tile * katoms_total + 2 * kb) * 512;
+                    bulk_load(st + W_BYTES + X_BYTES, sw, (uint32_t)ka * 512u, &full_bar[s]);
+                }
+            } else {
+                tma_load_2d(st, &args.tm_bo, &full_bar[s], (kb - nkb_a) * 64, n0);
+            }
+        };
+        auto load_x = [&](int kb, int s) {
+            uint8_t* st = smem + s * C::STAGE_BYTES;
+            if (kb < nkb_a) {
+                tma_load_2d(st + W_BYTES, &args.tm_a, &full_bar[s], kb * ROW_BYTES, 0);
+                if (MODE == MODE_OSC) {
+                    const int ka = min(2, katoms_total - 2 * kb);
+                    bulk_load(st + W_BYTES + X_BYTES + C::SF_BYTES, args.sfa + (int64_t)(2 * kb) * 512, (uint32_t)ka * 512u,
+                              &full_bar[s]);
+                }
+            } else {
+                tma_load_2d(st + W_BYTES, &args.tm_ao, &full_bar[s], (kb - nkb_a) * 64, 0);
+            }
+        };
+        const int first = min(kb1 - kb0, STAGES);
+        if (elect_one()) {
+            for (int i = 0; i < first; ++i) {
+                expect(kb0 + i, i);
+                load_w(kb0 + i, i);
+            }
+        }
+        __syncwarp();
+        grid_dependency_wait();   // the quantized activations come from the kernel before this one
+        if (elect_one()) {
+            for (int i = 0; i < first; ++i) load_x(kb0 + i, i);
+        }
+        __syncwarp();
+        int s = 0;
+        uint32_t ph = 1;          // the ring has been filled once
+        for (int kb = kb0 + first; kb < kb1; ++kb) {
+            if (!wait_bounded(&empty_bar[s], ph ^ 1u, abort_flag, 31)) goto done;
+            if (elect_one()) {
+                expect(kb, s);
+                load_w(kb, s);
+                load_x(kb, s);
+            }
+            __syncwarp();
+            if (++s == STAGES) { s = 0; ph ^= 1u; }
+        }
+    } else if (warp == 1) {
+        // -------------------------------------------------------------- MMA issuer
+        int s = 0;
+        uint32_t ph = 0;
+        const uint32_t idesc_a = (MODE == MODE_OSC) ? idesc_mxf4(BF, ntok) : idesc_e4m3(BF, ntok);
+        const uint32_t idesc_b = idesc_bf16(BF, ntok);
+        const uint64_t desc_hi = smem_desc_sw128(0);
+        const uint64_t sf_hi = smem_desc_sf(0);
+        const uint32_t smem0 = smem_u32(smem);
+        for (int kb = kb0; kb < kb1; ++kb) {
+            if (!wait_bounded(&full_bar[s], ph, abort_flag, 32)) goto done;
+            tc_fence_after();
+            const uint32_t sbase = smem0 + s * C::STAGE_BYTES;
+            const uint64_t wdesc = desc_hi | (uint64_t)(sbase >> 4);               // MMA operand A: weights
+            const uint64_t xdesc = desc_hi | (uint64_t)((sbase + W_BYTES) >> 4);   // MMA operand B: activations
+            const uint32_t first = (kb == kb0) ? 0u : 1u;
+            if (elect_one()) {
+                if (MODE == MODE_OSC && kb < nkb_a) {
+                    const int ka = min(2, katoms_total - 2 * kb);
+                    const uint64_t sfw_d = sf_hi | (uint64_t)((sbase + W_BYTES + X_BYTES) >> 4);
+                    const uint64_t sfx_d = sf_hi | (uint64_t)((sbase + W_BYTES + X_BYTES + C::SF_BYTES) >> 4);
+#pragma unroll
+                    for (int a = 0; a < 2; ++a) {
+                        if (a < ka) {
+                            tc_copy_sf(tmem_base + TM_SFW + a * 4, sfw_d + (uint64_t)(a * 32));
+                            tc_copy_sf(tmem_base + TM_SFX + a * 4, sfx_d + (uint64_t)(a * 32));
+                        }
+                    }
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        if (k < 2 * ka) {
+                            constexpr uint32_t SFID[2] = {idesc_sf_ids(0, 0), idesc_sf_ids(2, 2)};
+                            mma_mxf4(tmem_base, wdesc + 2 * k, xdesc + 2 * k, idesc_a | SFID[k & 1],
+                                     tmem_base + TM_SFW + (k >> 1) * 4, tmem_base + TM_SFX + (k >> 1) * 4,
+                                     (first | (uint32_t)k) ? 1u : 0u);
+                        }
+                    }
+                } else if (MODE == MODE_OSC) {
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        mma_f16(tmem_base, wdesc + 2 * k, xdesc + 2 * k, idesc_b, (first | (uint32_t)k) ? 1u : 0u);
+                } else {
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        mma_f8(tmem_base, wdesc + 2 * k, xdesc + 2 * k, idesc_a, (first | (uint32_t)k) ? 1u : 0u);
+                }
+                tc_commit(&empty_bar[s]);
+            }
+            __syncwarp();
+            if (++s == STAGES) { s = 0; ph ^= 1u; }
+        }
+        if (elect_one()) tc_commit(tfull_bar);
+        __syncwarp();
+    }
+
+done:
+    // ------------------------------------------------------------------ reduction + epilogue
+    // Every CTA of the cluster parks its partial tile as fp32 [feature][token] (row stride PSTR floats,
+    // conflict-free for 16-byte accesses) in its own shared memory: the ring is free once the accumulator
+    // is complete.  After a cluster barrier CTA r sums, in rank order, the four-token chunks c = r, r+S, ...
+    // of all partials through distributed shared memory and stores those tokens' outputs.
+    if (warp >= 2) {
+        bool have = kb1 > kb0;
+        if (have && !wait_bounded(tfull_bar, 0, abort_flag, 33)) have = false;
+        tc_fence_after();
+        if (have) {
+#pragma unroll
+            for (int c = 0; c < MAX_TOK / 16; ++c) {
+                if (c * 16 < ntok) {
+                    uint32_t r[32];
+                    tmem_ld_32x16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * 16), r);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) acc[c * 16 + i] = __uint_as_float(r[i]);
+                }
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < MAX_TOK; ++i) acc[i] = 0.0f;
+        }
+        tc_fence_before();
+        if (S > 1) {
+#pragma unroll
+            for (int c = 0; c < MAX_TOK / 4; ++c)
+                if (c * 4 < ntok)
+                    *reinterpret_cast<float4*>(partial + f * PSTR + c * 4) =
+                        make_float4(acc[4 * c], acc[4 * c + 1], acc[4 * c + 2], acc[4 * c + 3]);
+        }
+    }
+    __syncwarp();
+    __syncthreads();
+    if (S > 1) cluster_sync_all();          // partial tiles visible to the whole cluster
+    if (warp >= 2) {
+        grid_dependency_wait();             // Y may still be read by an earlier kernel
+        const int n = n0 + f;
+        float swn = 1.0f;
+        if (MODE == MODE_FP8 && n < N) swn = args.sw[n];
+        if (S == 1) {
+            if (n < N) {
+#pragma unroll
+                for (int t = 0; t < MAX_TOK; ++t) {
+                    if (t < M) {
+                        float v = acc[t];
+                        if (MODE == MODE_FP8) v = v * (args.sx[t] * swn);
+                        args.Y[(int64_t)t * args.ldy + n] = __bfloat16_as_ushort(__float2bfloat16_rn(v));
+                    }
+                }
+            }
+        } else {
+            const uint32_t mine = smem_u32(partial + f * PSTR);
+            uint32_t peer[MAX_CLUSTER];
+#pragma unroll
+            for (int r = 0; r < MAX_CLUSTER; ++r) peer[r] = map_to_cta(mine, (uint32_t)min(r, S - 1));
+            for (int c = rank; c * 4 < ntok; c += S) {
+                float4 p[MAX_CLUSTER];
+#pragma unroll
+                for (int r = 0; r < MAX_CLUSTER; ++r)
+                    if (r < S) p[r] = ld_cluster_f32x4(peer[r] + (uint32_t)(c * 16));
+                float4 v = p[0];
+#pragma unroll
+                for (int r = 1; r < MAX_CLUSTER; ++r)
+                    if (r < S) { v.x += p[r].x; v.y += p[r].y; v.z += p[r].z; v.w += p[r].w; }
+                if (n < N) {
+                    const float o[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int t = 4 * c + i;
+                        if (t < M) {
+                            float y = o[i];
+                            if (MODE == MODE_FP8) y = y * (args.sx[t] * swn);
+                            args.Y[(int64_t)t * args.ldy + n] = __bfloat16_as_ushort(__float2bfloat16_rn(y));
+                        }
+                    }
+                }
+            }
+        }
+    }
+    __syncwarp();
+    if (S > 1) cluster_sync_all();          // nobody leaves while a peer may still read its shared memory
+    __syncthreads();
+    if (warp == 1) {
+        if (*abort_flag && lane == 0) atomicCAS(&g_dev_status, 0, (39 << 8) | 1);
+        tc_fence_after();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+template <int MODE>
+static cudaError_t launch_cfg(const GemmArgs& a, int S, cudaStream_t st) {
+    using C = Cfg<MODE>;
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(gemm_decode_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             C::SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    const int tiles = (a.N + BF - 1) / BF;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(tiles * S);
+    cfg.blockDim = dim3(THREADS);
+    cfg.dynamicSmemBytes = C::SMEM_BYTES;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = S;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    return cudaLaunchKernelEx(&cfg, gemm_decode_kernel<MODE>, a);
+}
+
+}  // namespace decode
+
+// Cluster size (K split) of the few-row kernel: about one CTA per SM (measured on B200: with 48 feature tiles
+// S = 2, 3 and 4 are within 10 % of each other and ~15 % faster than S = 1; with more tiles than SMs any split
+// only adds reduction work and a second wave), every rank with at least one K block.  OSC_DECODE_SPLIT overrides.
+int gemm_decode_split(int N, int nkb, int num_sms) {
+    static int forced = -1;
+    if (forced < 0) {
+        forced = 0;
+        if (const char* e = getenv("OSC_DECODE_SPLIT")) forced = atoi(e);
+    }
+    const int tiles = (N + decode::BF - 1) / decode::BF;
+    int S = forced > 0 ? forced : num_sms / tiles;
+    if (S > 4 && forced <= 0) S = 4;
+    if (S > decode::MAX_CLUSTER) S = decode::MAX_CLUSTER;
+    if (S < 1) S = 1;
+    while (S > 1 && (S - 1) * ((nkb + S - 1) / S) >= nkb) --S;   // no rank without a K block
+    return S;
+}
+
+cudaError_t launch_gemm_dual_decode(const GemmArgs& a, int S, cudaStream_t st) {
+    return decode::launch_cfg<decode::MODE_OSC>(a, S, st);
+}
+cudaError_t launch_gemm_fp8_decode(const GemmArgs& a, int S, cudaStream_t st) {
+    return decode::launch_cfg<decode::MODE_FP8>(a, S, st);
+}
+
+}  // namespace osc

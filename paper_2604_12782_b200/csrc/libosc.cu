@@ -3,6 +3,7 @@
 #include "quant_kernels.cu"
 #include "gemm_kernels.cu"
 #include "gemm2_kernels.cu"
+#include "gemm3_kernels.cu"
 #include "profile_kernels.cu"
 #include "api.cu"
 #include "static_scratch.cu"

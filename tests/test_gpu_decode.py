@@ -1,0 +1,122 @@
+"""Few-row kernel (M <= 64: operands swapped, K split over a thread-block cluster) against the oracle.
+
+The library routes to it by itself for few rows; here OSC_DECODE=2 forces it for every M <= 64 and
+OSC_DECODE_SPLIT forces cluster sizes (1 = no reduction, up to 8), so that every reduction path, ranks whose
+K slice holds only Path-B blocks, odd numbers of 128-channel scale blocks, feature tiles cut by N and token
+counts that are not multiples of 16 are all covered.  OSC_DECODE=0 keeps the 128-row-tile kernel covered
+for the same shapes."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2604_12782_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+from gpu_util import assert_within_tolerance, dev_bf16, host_f64, poison  # noqa: E402
+
+
+@pytest.fixture(scope="module")
+def B():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2604_12782_b200 import binding
+    return binding
+
+
+@pytest.fixture
+def env():
+    saved = {k: os.environ.get(k) for k in ("OSC_DECODE", "OSC_DECODE_SPLIT")}
+
+    def set_(decode, split=None):
+        os.environ["OSC_DECODE"] = str(decode)
+        if split is None:
+            os.environ.pop("OSC_DECODE_SPLIT", None)
+        else:
+            os.environ["OSC_DECODE_SPLIT"] = str(split)
+    yield set_
+    for k, v in saved.items():
+        if v is None:
+            os.environ.pop(k, None)
+        else:
+            os.environ[k] = v
+
+
+def lut_for(rng, K, kind):
+    Kg = K // 32
+    if kind == "empty":
+        return np.full((Kg, 1), -1, np.int8)
+    if kind == "full":
+        return np.tile(np.arange(32, dtype=np.int8), (Kg, 1))
+    c = {"one": 1, "two": 2}[kind]
+    return np.stack([rng.permutation(32)[:c] for _ in range(Kg)]).astype(np.int8)
+
+
+CASES = [  # M, K, N, table, split (None = the library's choice)
+    (1, 128, 64, "one", None), (16, 512, 512, "two", None), (17, 384, 320, "one", 2), (33, 640, 192, "two", 3),
+    (64, 1024, 448, "one", 4), (48, 2048, 256, "two", 8), (5, 256, 128, "empty", 1), (64, 128, 64, "full", 2),
+    (31, 1536, 1024, "one", 5), (64, 4096, 512, "two", None), (20, 4096, 384, "two", 3), (64, 3072, 256, "one", 5),
+    (32, 4096, 128, "two", 7),
+]
+
+
+@pytest.mark.parametrize("M,K,N,kind,split", CASES)
+def test_decode_kernel_osc(B, oracle, env, M, K, N, kind, split):
+    rng = np.random.default_rng(M * 7 + K + N)
+    c = synth.osc_linear_case(M + N, M, K, N, 1)
+    lut = lut_for(rng, K, kind)
+    Yref, T, act, _ = oracle.linear(c["X"], c["W"], lut)
+    w = B.osc_prepare_weights(dev_bf16(c["W"]), lut)
+    sz = B.osc_act_sizes(w, M)
+    outs = {}
+    for mode in (2, 0):
+        env(mode, split if mode else None)
+        ws = poison(sz.workspace_bytes)
+        Ybig = torch.full((M + 2, N + 64), 7.0, dtype=torch.bfloat16, device="cuda")
+        Y = Ybig[1:M + 1, :N]
+        B.osc_linear(w, dev_bf16(c["X"]), Y, ws)
+        B.osc_sync_check()
+        assert np.array_equal(ws[sz.xq_offset:sz.xq_offset + sz.xq_bytes].cpu().numpy().reshape(M, K // 2), act["xq"])
+        assert_within_tolerance(host_f64(Y), Yref, T, f"decode={mode} M={M} K={K} N={N} {kind} S={split}")
+        guard = Ybig.clone()
+        guard[1:M + 1, :N] = 7.0
+        assert (guard == 7.0).all(), "wrote outside Y"
+        outs[mode] = Y.clone()
+    # the two kernels add the same exact products in different orders: equal up to fp32 rounding of the sums
+    d = (outs[2].float() - outs[0].float()).abs().cpu().numpy().astype(np.float64)
+    assert (d <= 2.0 ** -7 * np.abs(Yref) + 1e-3 * T).all()
+
+
+@pytest.mark.parametrize("M,K,N,split", [(1, 128, 64, None), (16, 768, 320, 3), (40, 1536, 1024, 4), (64, 12288, 256, 8),
+                                         (64, 256, 192, 2), (9, 4096, 128, 1)])
+def test_decode_kernel_fp8(B, oracle, env, M, K, N, split):
+    c = synth.fp8_linear_case(M + K, M, K, N)
+    Yref, T, (x8, sx), _ = oracle.fp8_linear(c["X"], c["W"])
+    w = B.osc_fp8_prepare_weights(dev_bf16(c["W"]))
+    sz = B.osc_fp8_act_sizes(w, M)
+    for mode in (2, 0):
+        env(mode, split if mode else None)
+        ws = poison(sz.workspace_bytes)
+        Y = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+        B.osc_fp8_linear(w, dev_bf16(c["X"]), Y, ws)
+        B.osc_sync_check()
+        assert np.array_equal(ws[sz.x8_offset:sz.x8_offset + M * K].cpu().numpy().reshape(M, K), x8)
+        assert_within_tolerance(host_f64(Y), Yref, T, f"fp8 decode={mode} M={M} K={K} N={N} S={split}")
+
+
+def test_decode_kernel_is_deterministic(B, env):
+    env(2, 4)
+    c = synth.osc_linear_case(3, 24, 2048, 768, 2)
+    w = B.osc_prepare_weights(dev_bf16(c["W"]), c["lut"])
+    sz = B.osc_act_sizes(w, 24)
+    ws = poison(sz.workspace_bytes)
+    X = dev_bf16(c["X"])
+    Ys = []
+    for _ in range(3):
+        Y = torch.empty((24, 768), dtype=torch.bfloat16, device="cuda")
+        B.osc_linear(w, X, Y, ws)
+        Ys.append(Y)
+    B.osc_sync_check()
+    assert torch.equal(Ys[0], Ys[1]) and torch.equal(Ys[0], Ys[2])
