@@ -272,6 +272,28 @@ def time_loop(torch, fn, steps, warmup):
     return e0.elapsed_time(e1) / max(steps, 1)
 
 
+def time_graph(torch, fn, n):
+    """Milliseconds of GPU time per call when `n` calls are captured once in a CUDA graph and replayed: what a
+    few-row (decode) step costs when the host does not pace the launches."""
+    st = torch.cuda.Stream()
+    with torch.cuda.stream(st):
+        for i in range(3):
+            fn(i)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=st):
+            for i in range(n):
+                fn(i)
+        g.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(st)
+        g.replay()
+        e1.record(st)
+        torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / n
+
+
 def time_split(torch, prob, steps):
     """Per-kernel averages (ms): events between the quantizer and the GEMM of every step."""
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(steps)]
@@ -446,7 +468,12 @@ def run_sweep(args):
         B.osc_sync_check()
         f4, f16 = roofline.osc_flops(M, N, K, p.K_o)
         troof = roofline.osc_roofline_seconds(M, N, K, p.K_o, peaks)
-        rows.append({"name": name, "M": M, "K": K, "N": N, "K_o": p.K_o, "ms": ms, "quant_ms": tq, "gemm_ms": tg,
+        extra = {}
+        if M <= 128:   # few rows: the plain loop above is paced by the host; also replay from a CUDA graph
+            gms, gms8 = time_graph(torch, p.step, 48), time_graph(torch, f8.step, 48)
+            extra = {"graph_ms": gms, "fp8_graph_ms": gms8, "pct_roofline_graph": 100 * troof / (gms * 1e-3),
+                     "speedup_vs_fp8_graph": gms8 / gms}
+        rows.append({**extra, "name": name, "M": M, "K": K, "N": N, "K_o": p.K_o, "ms": ms, "quant_ms": tq, "gemm_ms": tg,
                      "tflops": (f4 + f16) / ms / 1e9, "pct_roofline": 100 * troof / (ms * 1e-3),
                      "roof_us": troof * 1e6, "fp8_ms": ms8, "fp8_quant_ms": q8, "fp8_gemm_ms": g8,
                      "speedup_vs_fp8": ms8 / ms, "speedup_gemm_only": g8 / tg,
@@ -464,7 +491,11 @@ def run_sweep(args):
         q8, g8 = time_split(torch, f8, steps)
         B.osc_sync_check()
         troof = roofline.fp8_roofline_seconds(M, N, K, peaks)
-        rows.append({"name": name, "M": M, "K": K, "N": N, "ms": ms8, "quant_ms": q8, "gemm_ms": g8,
+        extra = {}
+        if M <= 128:
+            gms8 = time_graph(torch, f8.step, 48)
+            extra = {"graph_ms": gms8, "pct_roofline_graph": 100 * troof / (gms8 * 1e-3)}
+        rows.append({**extra, "name": name, "M": M, "K": K, "N": N, "ms": ms8, "quant_ms": q8, "gemm_ms": g8,
                      "tflops": roofline.fp8_flops(M, N, K) / ms8 / 1e9, "pct_roofline": 100 * troof / (ms8 * 1e-3),
                      "roof_us": troof * 1e6, "quant_gbs": roofline.fp8_quantize_bytes(M, K) / q8 / 1e6})
         del f8
@@ -489,12 +520,13 @@ def run_sweep(args):
         del p8
         torch.cuda.empty_cache()
 
-    for M in (16, 128, 2048, 8192):
+    for M in (16, 64, 128, 2048, 8192):
         osc_row("qkv", M, 4096, 6144, 2)
-    for M in (128, 2048, 8192):
+    for M in (16, 64, 128, 2048, 8192):
         osc_row("gate_up", M, 4096, 24576, 1)
         fp8_row("down_fp8", M, 12288, 4096)
-        mxfp8_row("down_mxfp8", M, 12288, 4096)
+        if M >= 128:
+            mxfp8_row("down_mxfp8", M, 12288, 4096)
     osc_row("layer.qkv", 4096, 4096, 6144, 2)
     osc_row("layer.o_proj", 4096, 4096, 4096, 1)
     osc_row("layer.gate_up", 4096, 4096, 24576, 1)
