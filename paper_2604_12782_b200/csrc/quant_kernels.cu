@@ -32,14 +32,16 @@ __device__ __forceinline__ uint32_t e4m3x2(float lo, float hi) {
 // ------------------------------------------------------- Algorithm 2, fused
 // Persistent kernel, two CTAs per SM.  A producer warp streams 128-row x 128-channel tiles of X
 // (32 KB, as two 64-channel halves with the 128-byte swizzle) through a shared-memory ring with
-// TMA.  512 consumer threads work on a tile in two steps:
-//   1. back-up + zero-out: one (row, flagged channel) task per thread copies the element from the
-//      shared tile into xo (the buffer B; consecutive threads write consecutive elements of a row)
-//      and overwrites it with +0 in shared memory;
-//   2. after a barrier every thread owns one 32-channel group of one row (64 bytes): amax, E8M0 code,
-//      exact fp32 scaling, hardware E2M1 conversion, one 16-byte store of the packed codes, one
-//      scale byte into the 512-byte scale block of the tile (staged in shared memory, written whole).
-// The slot is released as soon as the groups are in registers, so the next tiles stream in meanwhile.
+// TMA.  Each of the 512 consumer threads owns one 32-channel group of one row of the tile, 64 bytes
+// of shared memory that no other thread touches:
+//   1. back-up + zero-out: for every flagged channel of its group (bit mask of the table) the thread
+//      copies the element from the shared tile into xo (the buffer B) and overwrites it with +0;
+//   2. it loads its 64 bytes, releases the slot, then amax, E8M0 code, exact fp32 scaling, hardware
+//      E2M1 conversion, one 16-byte store of the packed codes; the four scale bytes of a row are
+//      gathered by shuffles into one 32-bit word of the 128 x 4 scale block.
+// No block-wide barrier: a version that first ran step 1 as (row, channel) tasks over all threads
+// and staged the scale block in shared memory spent a large part of its time waiting at the barrier
+// between the steps.
 constexpr int QE_ROWS = 128;
 constexpr int QE_COLS = 128;
 constexpr int QE_CONSUMERS = 512;               // = groups per tile
@@ -48,7 +50,7 @@ constexpr int QE_HALF_BYTES = QE_ROWS * 128;    // 64 channels x 128 rows
 constexpr int QE_TILE_BYTES = 2 * QE_HALF_BYTES;
 constexpr int QE_STAGES = 3;
 constexpr int QE_CTAS_PER_SM = 2;
-constexpr int QE_SMEM = QE_STAGES * QE_TILE_BYTES + 1024 + 2 * 512 + 256;
+constexpr int QE_SMEM = QE_STAGES * QE_TILE_BYTES + 1024 + 256;
 
 // byte offset of channel `col` (0..127) of row `row` inside a swizzled tile
 __device__ __forceinline__ int qe_elem_offset(int row, int col) {
@@ -79,8 +81,7 @@ quant_extract_kernel(const __grid_constant__ CUtensorMap tm_x, int M, int K,
                      int Ko, int Kop, const int32_t* __restrict__ sched, int max_tiles) {
     extern __shared__ uint8_t qe_smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(qe_smem_raw) + 1023) & ~uintptr_t(1023));
-    uint8_t* s_sf = smem + QE_STAGES * QE_TILE_BYTES;                       // 2 x 512 bytes, alternating
-    uint64_t* full_bar = reinterpret_cast<uint64_t*>(s_sf + 2 * 512);
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + QE_STAGES * QE_TILE_BYTES);
     uint64_t* empty_bar = full_bar + QE_STAGES;
     volatile int* abort_flag = reinterpret_cast<volatile int*>(empty_bar + QE_STAGES);
 
@@ -127,14 +128,21 @@ quant_extract_kernel(const __grid_constant__ CUtensorMap tm_x, int M, int K,
         }
     } else {
         // ----------------------------------------------------------------- consumers
+        // Every thread owns one 32-channel group of one row of the tile (64 bytes of the shared tile that no
+        // other thread touches), so back-up, zero-out, scale and quantization need no block-wide barrier.
         const int tid = threadIdx.x;
         const int grow = tid >> 2;  // my row inside the tile
         const int gi = tid & 3;     // my group inside the 128-channel block
         int s = 0;
         uint32_t ph = 0;
-        int parity = 0;
         int rt = t_begin / ncb, cb = t_begin - rt * ncb;
-        int64_t prev_sf_blk = -1;
+        // the table entries of the next tile are fetched one tile ahead, so their latency is off the critical path
+        uint32_t flagged_next = 0;
+        int slot_next = 0;
+        if (t_begin < t_end) {
+            flagged_next = mask[cb * 4 + gi];
+            slot_next = prefix[cb * 4 + gi];
+        }
         for (int t = t_begin; t < t_end; ++t) {
             int row0, row_end, sf_row0;
             if (sched) {
@@ -146,77 +154,85 @@ quant_extract_kernel(const __grid_constant__ CUtensorMap tm_x, int M, int K,
                 row_end = M;
                 sf_row0 = row0;
             }
+            const int r = row0 + grow;
+            uint32_t flagged = flagged_next;
+            int slot = slot_next;
+            if (t + 1 < t_end) {
+                const int cbn = (cb + 1 == ncb) ? 0 : cb + 1;
+                flagged_next = mask[cbn * 4 + gi];
+                slot_next = prefix[cbn * 4 + gi];
+            }
             if (!wait_bounded(&full_bar[s], ph, abort_flag, 22)) break;
             uint8_t* st = smem + s * QE_TILE_BYTES;
+            const uint8_t* rowp = st + (gi >> 1) * QE_HALF_BYTES + grow * 128;
 
-            // step 1: back-up of the flagged channels of this block into xo, then zero them in the tile
-            const int o0 = prefix[cb * 4];
-            const int o1 = (cb * 4 + 4 < K / 32) ? prefix[cb * 4 + 4] : Ko;
-            const int nout = o1 - o0;
-            if (nout > 0) {
-                int shift = 0;
-                while ((1 << shift) < nout) ++shift;           // tasks: (row, k) with k < 2^shift
-                const int k = tid & ((1 << shift) - 1);
-                if (k < nout) {
-                    const int col = idx_o[o0 + k] - cb * QE_COLS;
-                    const int rows_here = min(QE_ROWS, row_end - row0);
-                    for (int rl = tid >> shift; rl < QE_ROWS; rl += QE_CONSUMERS >> shift) {
-                        uint16_t* e = reinterpret_cast<uint16_t*>(st + qe_elem_offset(rl, col));
-                        if (rl < rows_here) xo[(int64_t)(row0 + rl) * Kop + o0 + k] = *e;
-                        *e = 0;
-                    }
-                }
+            // step 1: back-up of my group's flagged channels into xo, zero-out in the shared tile
+            const bool had_flagged = flagged != 0;
+            while (flagged) {
+                const int j = __ffs(flagged) - 1;
+                flagged &= flagged - 1;
+                const int within = (((gi & 1) << 5) + j) * 2;   // byte inside the 128-byte half row
+                uint16_t* e = reinterpret_cast<uint16_t*>(const_cast<uint8_t*>(rowp) +
+                                                          ((((within >> 4) ^ (grow & 7))) << 4) + (within & 15));
+                if (r < row_end) xo[(int64_t)r * Kop + slot] = *e;
+                ++slot;
+                *e = 0;
             }
-            // all flagged channels zeroed; all scale bytes of the previous tile staged
-            asm volatile("bar.sync 1, %0;" ::"n"(QE_CONSUMERS) : "memory");
-            if (prev_sf_blk >= 0 && tid < 32)
-                *reinterpret_cast<uint4*>(sf + prev_sf_blk * 512 + tid * 16) =
-                    *reinterpret_cast<const uint4*>(s_sf + (parity ^ 1) * 512 + tid * 16);
 
             // step 2: my group into registers, then release the slot
             uint32_t w[16];
-            {
-                const uint8_t* rowp = st + (gi >> 1) * QE_HALF_BYTES + grow * 128;
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const uint4 v = *reinterpret_cast<const uint4*>(rowp + (((((gi & 1) << 2) + i) ^ (grow & 7)) << 4));
-                    w[4 * i] = v.x; w[4 * i + 1] = v.y; w[4 * i + 2] = v.z; w[4 * i + 3] = v.w;
-                }
+            for (int i = 0; i < 4; ++i) {
+                const uint4 v = *reinterpret_cast<const uint4*>(rowp + (((((gi & 1) << 2) + i) ^ (grow & 7)) << 4));
+                w[4 * i] = v.x; w[4 * i + 1] = v.y; w[4 * i + 2] = v.z; w[4 * i + 3] = v.w;
             }
+            // the zero-out above wrote the slot through the generic proxy; the next TMA load overwrites it through
+            // the async proxy, so the writes are fenced before the slot is handed back
+            if (had_flagged) fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) mbar_arrive(&empty_bar[s]);
             if (++s == QE_STAGES) { s = 0; ph ^= 1u; }
 
-            const int r = row0 + grow;
             int code = 0;
             if (r < row_end) {  // rows past the end (next expert / padding) count as zeros: code 0, nothing stored
                 // amax on the bf16 magnitudes, two at a time
-                __nv_bfloat162 m2 = as_bf162(w[0] & 0x7FFF7FFFu);
+                __nv_bfloat162 m2 = __habs2(as_bf162(w[0]));
 #pragma unroll
-                for (int i = 1; i < 16; ++i) m2 = __hmax2(m2, as_bf162(w[i] & 0x7FFF7FFFu));
+                for (int i = 1; i < 16; ++i) m2 = __hmax2(m2, __habs2(as_bf162(w[i])));
                 const uint32_t am2 = bf162_bits(m2);
                 const uint32_t am = max(am2 & 0xFFFFu, am2 >> 16);
                 // CalculateScale: E8M0 code = biased exponent of amax - 2, floored at 0 (2^(floor(log2 amax) - 2))
                 const int ex = (int)(am >> 7);
                 code = max(ex - 2, 0);
                 if (ex == 255) code = 255;
-                // Quantize: x * 2^(127 - code) is exact in fp32, then hardware E2M1 rounding (nearest-even, saturating)
-                const float inv = __uint_as_float((uint32_t)(254 - min(code, 253)) << 23);
+                // Quantize: x * 2^(127 - code) is exact (a power of two, two bf16 values per multiply; results below
+                // the bf16 normal range are far under the 0.25 tie point and keep their sign), then hardware E2M1
+                // rounding (nearest-even, saturating) of the fp32 extensions
+                const __nv_bfloat162 inv2 = as_bf162(((uint32_t)(254 - min(code, 253)) << 7) * 0x10001u);
                 uint32_t q[4];
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     float f[8];
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
-                        f[2 * j] = __uint_as_float(w[4 * i + j] << 16) * inv;
-                        f[2 * j + 1] = __uint_as_float(w[4 * i + j] & 0xFFFF0000u) * inv;
+                        const uint32_t p = bf162_bits(__hmul2(as_bf162(w[4 * i + j]), inv2));
+                        f[2 * j] = __uint_as_float(p << 16);
+                        f[2 * j + 1] = __uint_as_float(p & 0xFFFF0000u);
                     }
                     q[i] = e2m1x8(f[0], f[1], f[2], f[3], f[4], f[5], f[6], f[7]);
                 }
                 *reinterpret_cast<uint4*>(xq + (int64_t)r * (K / 2) + cb * (QE_COLS / 2) + gi * 16) =
                     make_uint4(q[0], q[1], q[2], q[3]);
             }
-            s_sf[parity * 512 + (grow & 31) * 16 + (grow >> 5) * 4 + gi] = (uint8_t)code;
+            // the four scale bytes of a row and 128-channel block are one 32-bit word of the block layout:
+            // gather them from the four lanes of the row, lane gi == 0 stores
+            uint32_t word = (uint32_t)code << (8 * gi);
+            word |= __shfl_xor_sync(0xFFFFFFFFu, word, 1);
+            word |= __shfl_xor_sync(0xFFFFFFFFu, word, 2);
+            if (gi == 0) {
+                const int64_t blk = (int64_t)(sf_row0 / 128) * (K / 128) + cb;
+                *reinterpret_cast<uint32_t*>(sf + blk * 512 + (grow & 31) * 16 + (grow >> 5) * 4) = word;
+            }
 
             // zero the pad columns of xo once per row tile
             if (cb == 0 && Kop > Ko) {
@@ -226,15 +242,8 @@ quant_extract_kernel(const __grid_constant__ CUtensorMap tm_x, int M, int K,
                     if (rr < row_end) xo[(int64_t)rr * Kop + Ko + i % npad] = 0;
                 }
             }
-            prev_sf_blk = (int64_t)(sf_row0 / 128) * (K / 128) + cb;
-            parity ^= 1;
             if (++cb == ncb) { cb = 0; ++rt; }
         }
-        // scale block of the last tile
-        asm volatile("bar.sync 1, %0;" ::"n"(QE_CONSUMERS) : "memory");
-        if (prev_sf_blk >= 0 && tid < 32)
-            *reinterpret_cast<uint4*>(sf + prev_sf_blk * 512 + tid * 16) =
-                *reinterpret_cast<const uint4*>(s_sf + (parity ^ 1) * 512 + tid * 16);
     }
 }
 
