@@ -10,6 +10,7 @@ Function-to-paper map (details in the C file):
   gemm_dual / linear                   Eq. 5
   fp8_quantize / fp8_gemm / fp8_linear Section 3.4 fallback (per-token E4M3)
   mxfp8_quantize / mxfp8_gemm / mxfp8_linear   Section 3.4 fallback in its 8-bit micro-scaling form (MXFP8)
+  dyn_quantize_extract / dyn_prepare_weights / dyn_linear   the dynamic-protection control group of Section 4.2
   threshold / profile_indexing / clustering_density   Eq. 1-4, Algorithm 1 (offline profiling)
 """
 from __future__ import annotations
@@ -244,6 +245,40 @@ def mxfp8_linear(X: np.ndarray, W: np.ndarray, rows=None):
     w8, sfw = mxfp8_quantize(W)
     Y, T = mxfp8_gemm(x8, sfa, w8, sfw, rows)
     return Y, T, (x8, sfa), (w8, sfw)
+
+
+def dyn_quantize_extract(X: np.ndarray):
+    """Dynamic protection: per token and 32-group the run-time largest element is extracted (Section 4.2 control
+    group).  -> dict(xq, sf, idx u8 [M,K/32], val u16 [M,K/32], xo u16 [M,K] = the extracted elements scattered
+    back to their channels, zero elsewhere)."""
+    X = np.ascontiguousarray(X, dtype=np.uint16)
+    M, K = X.shape
+    Kg = K // 32
+    xq = np.zeros((M, K // 2), np.uint8)
+    sf = np.zeros(sf_bytes(M, K), np.uint8)
+    idx = np.zeros((M, Kg), np.uint8)
+    val = np.zeros((M, Kg), np.uint16)
+    lib().osc_ref_dyn_quantize_extract(_p(X), C.c_int64(K), M, K, _p(xq), _p(sf), _p(idx), _p(val))
+    xo = np.zeros((M, K), np.uint16)
+    cols = (np.arange(Kg, dtype=np.int64) * 32)[None, :] + idx
+    np.put_along_axis(xo, cols, val, axis=1)
+    return {"xq": xq, "sf": sf, "idx": idx, "val": val, "xo": xo, "K_o": K, "K_o_pad": K}
+
+
+def dyn_prepare_weights(W: np.ndarray):
+    """Weights of the dynamic baseline: MXFP4 of the whole matrix (no column zeroed) + the bf16 matrix itself
+    as the high-precision operand (any column can be picked by some token)."""
+    W = np.ascontiguousarray(W, dtype=np.uint16)
+    K = W.shape[1]
+    q = quantize_extract(W, np.full((K // 32, 1), -1, np.int8))
+    return {"xq": q["xq"], "sf": q["sf"], "xo": W.copy()}
+
+
+def dyn_linear(X: np.ndarray, W: np.ndarray, rows=None):
+    act = dyn_quantize_extract(X)
+    wts = dyn_prepare_weights(W)
+    Y, T = gemm_dual(act, wts, rows)
+    return Y, T, act, wts
 
 
 def threshold(X: np.ndarray, alpha: float = 5.0) -> float:

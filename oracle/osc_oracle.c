@@ -378,6 +378,55 @@ int osc_ref_fp8_gemm_rows(const uint8_t* x8, const float* sx, const int32_t* row
     return 0;
 }
 
+/* ---------------- dynamic-protection baseline (Section 4.2, "OSC vs. Optimized Dynamic Protection") */
+
+/* The control group the paper compares against: per token and per 32-group the
+ * element of largest magnitude is found AT RUN TIME, kept in high precision and
+ * removed before the group is scaled and quantized (same CalculateScale /
+ * Quantize as Algorithm 2).  Ties take the lowest channel; an all-zero group
+ * "extracts" its first element (a zero).  Outputs per row m and group g:
+ * idx[m][g] = local channel 0..31, val[m][g] = the bf16 element (bit copy);
+ * xq / sf as in osc_ref_quantize_extract.  The weights of this baseline are
+ * quantized whole (no column is zeroed: any column can be picked by some token). */
+int osc_ref_dyn_quantize_extract(const uint16_t* X, int64_t ldx, int M, int K, uint8_t* xq, uint8_t* sf,
+                                 uint8_t* idx, uint16_t* val) {
+    int Kg = K / G;
+#pragma omp parallel for schedule(static)
+    for (int m = 0; m < M; ++m) {
+        const uint16_t* xrow = X + (int64_t)m * ldx;
+        for (int g = 0; g < Kg; ++g) {
+            int best = 0;
+            double bestv = -1.0;
+            for (int j = 0; j < G; ++j) {
+                double a = fabs(bf16_value(xrow[g * G + j]));
+                if (a > bestv) {
+                    bestv = a;
+                    best = j;
+                }
+            }
+            idx[(int64_t)m * Kg + g] = (uint8_t)best;
+            val[(int64_t)m * Kg + g] = xrow[g * G + best];
+            double amax = 0.0;
+            for (int j = 0; j < G; ++j) {
+                if (j == best) continue;
+                double a = fabs(bf16_value(xrow[g * G + j]));
+                if (a > amax) amax = a;
+            }
+            int code = osc_ref_e8m0_from_amax(amax);
+            sf[osc_ref_sf_index(m, g, K)] = (uint8_t)code;
+            for (int j = 0; j < G; j += 2) {
+                int nib[2];
+                for (int t = 0; t < 2; ++t) {
+                    uint16_t b = (j + t == best) ? (uint16_t)0 : xrow[g * G + j + t];
+                    nib[t] = osc_ref_e2m1_encode(ldexp(bf16_value(b), 127 - code));
+                }
+                xq[(int64_t)m * (K / 2) + (g * G + j) / 2] = (uint8_t)(nib[0] | (nib[1] << 4));
+            }
+        }
+    }
+    return 0;
+}
+
 /* ------------------------- MXFP8 fallback (Section 3.4; Section 4 "Implementation Details") */
 
 /* The 8-bit micro-scaling form of the W2 fallback: groups of 32 along K share an
