@@ -520,6 +520,28 @@ def run_sweep(args):
         del p8
         torch.cuda.empty_cache()
 
+    def dyn_row(name, M, K, N, cpg, seed=0):
+        """The dynamic-protection control group (run-time per-group maximum) on the shape of an OSC row."""
+        if not want(name):
+            return
+        case = synth.osc_linear_case(seed, M, K, N, cpg)
+        X0, W0 = dev_bf16(torch, case["X"]), dev_bf16(torch, case["W"])
+        n = NSETS
+        Xs = [X0 if i == 0 else torch.roll(X0, 97 * i, 0).contiguous() for i in range(n)]
+        ws_ = [B.osc_dyn_prepare_weights(W0 if i == 0 else torch.roll(W0, 61 * i, 0).contiguous()) for i in range(n)]
+        sz = B.osc_dyn_act_sizes(ws_[0], M)
+        wk = [torch.empty(sz.workspace_bytes, dtype=torch.uint8, device="cuda") for _ in range(n)]
+        Ys = [torch.empty(M, N, dtype=torch.bfloat16, device="cuda") for _ in range(n)]
+        ms = time_loop(torch, lambda i: B.osc_dyn_linear(ws_[i % n], Xs[i % n], Ys[i % n], wk[i % n]), steps, warm)
+        tq = time_loop(torch, lambda i: B.osc_dyn_quantize_extract(
+            ws_[i % n], Xs[i % n], wk[i % n][sz.xq_offset:], wk[i % n][sz.sfa_offset:], wk[i % n][sz.xo_offset:],
+            wk[i % n][sz.idx_offset:], wk[i % n][sz.val_offset:]), steps, warm)
+        B.osc_sync_check()
+        rows.append({"name": name, "M": M, "K": K, "N": N, "ms": ms, "quant_ms": tq,
+                     "note": "high-precision branch over all K channels (one non-zero per 32), weights unzeroed"})
+        del ws_, wk, Ys, Xs
+        torch.cuda.empty_cache()
+
     for M in (16, 64, 128, 2048, 8192):
         osc_row("qkv", M, 4096, 6144, 2)
     for M in (16, 64, 128, 2048, 8192):
@@ -527,6 +549,8 @@ def run_sweep(args):
         fp8_row("down_fp8", M, 12288, 4096)
         if M >= 128:
             mxfp8_row("down_mxfp8", M, 12288, 4096)
+    dyn_row("qkv.dynamic_protection", 8192, 4096, 6144, 2)
+    dyn_row("qkv.dynamic_protection", 2048, 4096, 6144, 2)
     osc_row("layer.qkv", 4096, 4096, 6144, 2)
     osc_row("layer.o_proj", 4096, 4096, 4096, 1)
     osc_row("layer.gate_up", 4096, 4096, 24576, 1)

@@ -258,6 +258,41 @@ osc_status osc_mxfp8_gemm(const osc_mxfp8_weights* w, const void* x8, const void
 osc_status osc_mxfp8_linear(const osc_mxfp8_weights* w, const void* X, int M, int64_t ldx, void* Y, int64_t ldy,
                             void* workspace, size_t workspace_bytes, void* stream);
 
+/* ------------------- dynamic-protection control group (Section 4.2), a baseline */
+
+/* The paper compares OSC with an "idealized Dynamic Protection baseline": per token and per 32-group the
+ * element of largest magnitude is detected at run time, kept in high precision and removed before the group
+ * is scaled and quantized.  These calls are that baseline, built so that its cost can be measured beside
+ * osc_linear on the same shapes (Section 4.2, "Hardware-Efficiency Trade-offs").  Because any channel can be
+ * picked by some token, the weights are MXFP4 of the WHOLE matrix (no column zeroed) plus the bf16 matrix
+ * itself as the high-precision operand; the extracted elements are handed to the tensor cores as a dense
+ * [M, K] bf16 matrix xo that is +0 except at the extracted positions (one non-zero per 32 channels), so the
+ * high-precision branch of Eq. 5 runs over all K channels instead of K_o.  The handle is an osc_weights with
+ * K_o = K_o_pad = K; it is accepted by osc_gemm_dual, osc_weights_destroy and the osc_dyn_* calls only.
+ * Dense problems only.  osc_dyn_weight_sizes fills the same struct as osc_weight_sizes (wo_bytes = N*K*2). */
+typedef struct {
+    size_t xq_bytes, sfa_bytes;     /* as osc_act_sizes */
+    size_t xo_bytes;                /* M * K * 2: the dense high-precision operand */
+    size_t idx_bytes;               /* M * K/32: local channel 0..31 of the extracted element, uint8 */
+    size_t val_bytes;               /* M * K/32 * 2: the extracted elements, bf16 bit copies */
+    size_t xq_offset, sfa_offset, xo_offset, idx_offset, val_offset;
+    size_t workspace_bytes;
+} osc_dyn_act_sizes_t;
+
+osc_status osc_dyn_weight_sizes(int N, int K, osc_weight_sizes_t* out);
+osc_status osc_dyn_prepare_weights(const void* W, int N, int K, int64_t ldw, void* wq, void* sfw, void* wo, void* meta,
+                                   void* stream, osc_weights** out);
+osc_status osc_dyn_act_sizes(const osc_weights* w, int M, osc_dyn_act_sizes_t* out);
+
+/* Run-time extraction + MXFP4 of the rest.  Ties between equal magnitudes take the lowest channel; an all-zero
+ * group extracts its first element.  xq, sfa as osc_quantize_extract; xo, idx, val as described above. */
+osc_status osc_dyn_quantize_extract(const osc_weights* w, const void* X, int M, int64_t ldx, void* xq, void* sfa,
+                                    void* xo, void* idx, void* val, void* stream);
+
+/* osc_dyn_quantize_extract + the dual-path GEMM with K_o = K. */
+osc_status osc_dyn_linear(const osc_weights* w, const void* X, int M, int64_t ldx, void* Y, int64_t ldy,
+                          void* workspace, size_t workspace_bytes, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

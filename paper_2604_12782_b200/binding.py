@@ -47,6 +47,11 @@ class Fp8ActSizes(C.Structure):
                                           "sched_offset", "workspace_bytes")]
 
 
+class DynActSizes(C.Structure):
+    _fields_ = [(n, C.c_size_t) for n in ("xq_bytes", "sfa_bytes", "xo_bytes", "idx_bytes", "val_bytes", "xq_offset",
+                                          "sfa_offset", "xo_offset", "idx_offset", "val_offset", "workspace_bytes")]
+
+
 class Mxfp8WeightSizes(C.Structure):
     _fields_ = [("w8_bytes", C.c_size_t), ("sfw_bytes", C.c_size_t)]
 
@@ -80,6 +85,11 @@ _SIGS = {
     "osc_fp8_gemm": (_i, [_vp, _vp, _vp, _i, _vp, _i64, _vp]),
     "osc_fp8_linear": (_i, [_vp, _vp, _i, _i64, _vp, _i64, _vp, _sz, _vp]),
     "osc_fp8_linear_grouped": (_i, [_vp, _vp, _vp, _i, _i64, _vp, _i64, _vp, _sz, _vp]),
+    "osc_dyn_weight_sizes": (_i, [_i, _i, C.POINTER(WeightSizes)]),
+    "osc_dyn_prepare_weights": (_i, [_vp, _i, _i, _i64, _vp, _vp, _vp, _vp, _vp, C.POINTER(_vp)]),
+    "osc_dyn_act_sizes": (_i, [_vp, _i, C.POINTER(DynActSizes)]),
+    "osc_dyn_quantize_extract": (_i, [_vp, _vp, _i, _i64, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "osc_dyn_linear": (_i, [_vp, _vp, _i, _i64, _vp, _i64, _vp, _sz, _vp]),
     "osc_mxfp8_weight_sizes": (_i, [_i, _i, C.POINTER(Mxfp8WeightSizes)]),
     "osc_mxfp8_prepare_weights": (_i, [_vp, _i, _i, _i64, _vp, _vp, _vp, C.POINTER(_vp)]),
     "osc_mxfp8_weights_destroy": (_i, [_vp]),
@@ -366,3 +376,41 @@ def osc_mxfp8_linear(w: Mxfp8Weights, X: torch.Tensor, Y: torch.Tensor, workspac
     M = X.shape[0]
     _check(_lib.osc_mxfp8_linear(w.ptr, _ptr(X), M, X.stride(0) if M else w.K, _ptr(Y), Y.stride(0) if M else w.N,
                                  _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)))
+
+
+# ------------------------------------------- dynamic-protection control group (a baseline)
+
+def osc_dyn_weight_sizes(N: int, K: int) -> WeightSizes:
+    out = WeightSizes()
+    _check(_lib.osc_dyn_weight_sizes(N, K, C.byref(out)))
+    return out
+
+
+def osc_dyn_prepare_weights(W: torch.Tensor, stream=None) -> OscWeights:
+    N, K = W.shape
+    sz = osc_dyn_weight_sizes(N, K)
+    bufs = {k: _alloc(getattr(sz, k + "_bytes"), W.device) for k in ("wq", "sfw", "wo", "meta")}
+    h = _vp()
+    _check(_lib.osc_dyn_prepare_weights(_ptr(W), N, K, W.stride(0), _ptr(bufs["wq"]), _ptr(bufs["sfw"]),
+                                        _ptr(bufs["wo"]), _ptr(bufs["meta"]), _stream(stream), C.byref(h)))
+    w = OscWeights(h.value, bufs)
+    w.E, w.N, w.K, w.K_o, w.K_o_pad, w.sizes = 1, N, K, K, K, sz
+    return w
+
+
+def osc_dyn_act_sizes(w: OscWeights, M: int) -> DynActSizes:
+    out = DynActSizes()
+    _check(_lib.osc_dyn_act_sizes(w.ptr, M, C.byref(out)))
+    return out
+
+
+def osc_dyn_quantize_extract(w: OscWeights, X: torch.Tensor, xq, sfa, xo, idx, val, stream=None):
+    M = X.shape[0]
+    _check(_lib.osc_dyn_quantize_extract(w.ptr, _ptr(X), M, X.stride(0) if M else w.K, _ptr(xq), _ptr(sfa), _ptr(xo),
+                                         _ptr(idx), _ptr(val), _stream(stream)))
+
+
+def osc_dyn_linear(w: OscWeights, X: torch.Tensor, Y: torch.Tensor, workspace: torch.Tensor, stream=None):
+    M = X.shape[0]
+    _check(_lib.osc_dyn_linear(w.ptr, _ptr(X), M, X.stride(0) if M else w.K, _ptr(Y), Y.stride(0) if M else w.N,
+                               _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)))

@@ -192,6 +192,7 @@ using namespace osc;
 struct osc_weights {
     int E, N, K, Ko, Kop;
     bool grouped;
+    bool dynamic;   // weights of the dynamic-protection control group: whole-matrix MXFP4 + the bf16 matrix (Kop = K)
     const uint8_t *wq, *sfw;
     const uint16_t* wo;
     const uint32_t* mask;
@@ -269,13 +270,13 @@ osc_status osc_weight_sizes(int E, int N, int K, const int8_t* lut, int lut_c, o
 
 static osc_status prepare_impl(const void* W, int E, int N, int K, int64_t ldw, const int8_t* lut, int lut_c,
                                void* wq, void* sfw, void* wo, void* meta, void* stream, bool grouped,
-                               osc_weights** out) {
+                               osc_weights** out, bool dynamic = false) {
     if (!out) return fail(OSC_ERR_INVALID_ARG, "out is null");
     *out = nullptr;
     if (osc_status s = check_nk(E, N, K)) return s;
     Table t;
     if (osc_status s = parse_lut(lut, K, lut_c, &t)) return s;
-    if (!W || !wq || !sfw || !meta || (t.Kop > 0 && !wo)) return fail(OSC_ERR_INVALID_ARG, "null device pointer");
+    if (!W || !wq || !sfw || !meta || ((t.Kop > 0 || dynamic) && !wo)) return fail(OSC_ERR_INVALID_ARG, "null device pointer");
     if (ldw < K) return fail(OSC_ERR_SHAPE, "ldw = %lld < K", (long long)ldw);
     if (ldw % 8 || !aligned16(W) || !aligned16(wq) || !aligned16(sfw) || !aligned16(meta) || !aligned16(wo))
         return fail(OSC_ERR_ALIGN, "pointers must be 16-byte aligned and ldw a multiple of 8");
@@ -305,9 +306,17 @@ static osc_status prepare_impl(const void* W, int E, int N, int K, int64_t ldw, 
         if (e != cudaSuccess) return cuda_fail(e, "quant_extract_kernel(weights)");
     }
 
+    const size_t tiled_off = meta_table_bytes(K, t.Ko);   // the per-tile scale copy follows the table
+    if (dynamic) {
+        // the high-precision operand is the bf16 matrix itself, compacted to [N, K]; from here on the handle
+        // looks like one whose table lists every channel, except that no column was zeroed before quantization
+        e = cudaMemcpy2DAsync(wo, (size_t)K * 2, W, (size_t)ldw * 2, (size_t)K * 2, (size_t)N, cudaMemcpyDeviceToDevice, st);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpy2DAsync(weights)");
+        t.Ko = t.Kop = K;
+    }
     osc_weights* w = new (std::nothrow) osc_weights();
     if (!w) return fail(OSC_ERR_INVALID_ARG, "out of host memory");
-    w->E = E; w->N = N; w->K = K; w->Ko = t.Ko; w->Kop = t.Kop; w->grouped = grouped;
+    w->E = E; w->N = N; w->K = K; w->Ko = t.Ko; w->Kop = t.Kop; w->grouped = grouped; w->dynamic = dynamic;
     w->wq = static_cast<const uint8_t*>(wq);
     w->sfw = static_cast<const uint8_t*>(sfw);
     w->wo = static_cast<const uint16_t*>(wo);
@@ -329,7 +338,7 @@ static osc_status prepare_impl(const void* W, int E, int N, int K, int64_t ldw, 
     }
     if (s == OSC_OK) s = make_tmap_sf(&w->tm_sfw, sfw, (uint64_t)E * sfw_e / 512);
     if (s == OSC_OK && !grouped) {
-        uint8_t* tiled = m8 + meta_table_bytes(K, t.Ko);
+        uint8_t* tiled = m8 + tiled_off;
         e = launch_retile_sf(static_cast<const uint8_t*>(sfw), tiled, N, K, kTiledBN, st);
         if (e != cudaSuccess) { delete w; return cuda_fail(e, "retile_sf_kernel"); }
         s = make_tmap_sf(&w->tm_sfw_tiled, tiled, (uint64_t)tiled_sf_bytes(N, K) / 512);
@@ -373,8 +382,10 @@ osc_status osc_act_sizes(const osc_weights* w, int M, osc_act_sizes_t* out) {
     return OSC_OK;
 }
 
-static osc_status check_act(const osc_weights* w, const void* X, int M, int64_t ldx) {
+static osc_status check_act(const osc_weights* w, const void* X, int M, int64_t ldx, bool dynamic = false) {
     if (!w) return fail(OSC_ERR_INVALID_ARG, "weights handle is null");
+    if (w->dynamic != dynamic)
+        return fail(OSC_ERR_INVALID_ARG, dynamic ? "static-table weights: use osc_linear" : "dynamic-protection weights: use osc_dyn_linear");
     if (M < 0) return fail(OSC_ERR_INVALID_ARG, "M = %d is negative", M);
     if (M > 0 && !X) return fail(OSC_ERR_INVALID_ARG, "X is null");
     if (ldx < w->K) return fail(OSC_ERR_SHAPE, "ldx = %lld < K = %d", (long long)ldx, w->K);
@@ -821,6 +832,72 @@ osc_status osc_mxfp8_linear(const osc_mxfp8_weights* w, const void* X, int M, in
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     if (osc_status s = osc_mxfp8_quantize(X, M, w->K, ldx, ws + sz.x8_offset, ws + sz.sfa_offset, stream)) return s;
     return osc_mxfp8_gemm(w, ws + sz.x8_offset, ws + sz.sfa_offset, M, Y, ldy, stream);
+}
+
+// ------------------------------- dynamic-protection control group (Section 4.2)
+
+osc_status osc_dyn_weight_sizes(int N, int K, osc_weight_sizes_t* out) {
+    if (!out) return fail(OSC_ERR_INVALID_ARG, "out is null");
+    if (osc_status s = check_nk(1, N, K)) return s;
+    out->K_o = K;
+    out->K_o_pad = K;
+    out->wq_bytes = (size_t)N * (K / 2);
+    out->sfw_bytes = sf_bytes(N, K);
+    out->wo_bytes = (size_t)N * K * 2;
+    out->meta_bytes = meta_table_bytes(K, 0) + tiled_sf_bytes(N, K);
+    return OSC_OK;
+}
+
+osc_status osc_dyn_prepare_weights(const void* W, int N, int K, int64_t ldw, void* wq, void* sfw, void* wo, void* meta,
+                                   void* stream, osc_weights** out) {
+    return prepare_impl(W, 1, N, K, ldw, nullptr, 0, wq, sfw, wo, meta, stream, false, out, true);
+}
+
+osc_status osc_dyn_act_sizes(const osc_weights* w, int M, osc_dyn_act_sizes_t* out) {
+    if (!w || !out) return fail(OSC_ERR_INVALID_ARG, "null argument");
+    if (!w->dynamic) return fail(OSC_ERR_INVALID_ARG, "static-table weights: use osc_act_sizes");
+    if (M < 0) return fail(OSC_ERR_INVALID_ARG, "M = %d is negative", M);
+    out->xq_bytes = (size_t)M * (w->K / 2);
+    out->sfa_bytes = sf_bytes(M, w->K);
+    out->xo_bytes = (size_t)M * w->K * 2;
+    out->idx_bytes = (size_t)M * (w->K / 32);
+    out->val_bytes = (size_t)M * (w->K / 32) * 2;
+    out->xq_offset = 0;
+    out->sfa_offset = out->xq_offset + align256(out->xq_bytes);
+    out->xo_offset = out->sfa_offset + align256(out->sfa_bytes);
+    out->idx_offset = out->xo_offset + align256(out->xo_bytes);
+    out->val_offset = out->idx_offset + align256(out->idx_bytes);
+    out->workspace_bytes = out->val_offset + align256(out->val_bytes);
+    return OSC_OK;
+}
+
+osc_status osc_dyn_quantize_extract(const osc_weights* w, const void* X, int M, int64_t ldx, void* xq, void* sfa,
+                                    void* xo, void* idx, void* val, void* stream) {
+    if (osc_status s = check_act(w, X, M, ldx, true)) return s;
+    if (M == 0) return OSC_OK;
+    if (!xq || !sfa || !xo || !idx || !val) return fail(OSC_ERR_INVALID_ARG, "null output pointer");
+    if (!aligned16(xq) || !aligned16(sfa) || !aligned16(xo) || !aligned16(idx) || !aligned16(val))
+        return fail(OSC_ERR_ALIGN, "outputs must be 16-byte aligned");
+    cudaError_t e = launch_dyn_quant_extract(X, ldx, M, w->K, xq, sfa, xo, idx, val, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(e, "dyn_quant_extract_kernel");
+    return OSC_OK;
+}
+
+osc_status osc_dyn_linear(const osc_weights* w, const void* X, int M, int64_t ldx, void* Y, int64_t ldy,
+                          void* workspace, size_t workspace_bytes, void* stream) {
+    if (osc_status s = check_act(w, X, M, ldx, true)) return s;
+    if (M == 0) return OSC_OK;
+    osc_dyn_act_sizes_t sz;
+    osc_dyn_act_sizes(w, M, &sz);
+    if (!workspace || !aligned16(workspace)) return fail(OSC_ERR_ALIGN, "workspace must be non-null and 16-byte aligned");
+    if (workspace_bytes < sz.workspace_bytes)
+        return fail(OSC_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", workspace_bytes, sz.workspace_bytes);
+    if (!Y) return fail(OSC_ERR_INVALID_ARG, "Y is null");
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    if (osc_status s = osc_dyn_quantize_extract(w, X, M, ldx, ws + sz.xq_offset, ws + sz.sfa_offset, ws + sz.xo_offset,
+                                                ws + sz.idx_offset, ws + sz.val_offset, stream)) return s;
+    return gemm_impl(w, ws + sz.xq_offset, ws + sz.sfa_offset, ws + sz.xo_offset, M, Y, ldy, nullptr, 0, nullptr, 0,
+                     static_cast<cudaStream_t>(stream));
 }
 
 }  // extern "C"

@@ -438,6 +438,100 @@ mxfp8_quant_kernel(const uint16_t* __restrict__ X, int64_t ldx, int M, int M_pad
 }
 
 
+// ------------------------------- dynamic-protection control group (Section 4.2): run-time extraction
+// Per token and 32-channel group the element of largest magnitude is found at run time (ties: lowest
+// channel), kept in bf16 and removed; the rest is MXFP4 as in Algorithm 2.  Same thread layout as the
+// MXFP8 quantizer: one warp per row, 16 bytes (8 channels) per lane and step, four lanes per group.
+// Outputs per step: 4 bytes of packed codes per lane, the dense high-precision operand xo (the
+// extracted element at its own channel, +0 elsewhere: 16 bytes per lane), and per group one scale
+// byte, one index byte and the bf16 value (gathered by shuffles, written by lanes 0 and 16).
+__global__ void __launch_bounds__(32 * MX8_ROWS_PER_CTA)
+dyn_quant_extract_kernel(const uint16_t* __restrict__ X, int64_t ldx, int M, int M_pad, int K, uint8_t* __restrict__ xq,
+                         uint8_t* __restrict__ sf, uint16_t* __restrict__ xo, uint8_t* __restrict__ idx,
+                         uint16_t* __restrict__ val) {
+    grid_launch_dependents();
+    grid_dependency_wait();
+    const int lane = threadIdx.x & 31;
+    const int r = blockIdx.x * MX8_ROWS_PER_CTA + (threadIdx.x >> 5);
+    if (r >= M_pad) return;
+    const int katoms = K / 128;
+    const int Kg = K / 32;
+    uint32_t* sf_row = reinterpret_cast<uint32_t*>(sf + (size_t)(r / 128) * katoms * 512) + (r & 31) * 4 + ((r & 127) >> 5);
+    if (r >= M) {
+        for (int a = lane; a < katoms; a += 32) sf_row[(size_t)a * 128] = 0u;
+        return;
+    }
+    const uint4* xrow = reinterpret_cast<const uint4*>(X + (int64_t)r * ldx);
+    uint32_t* qrow = reinterpret_cast<uint32_t*>(xq + (int64_t)r * (K / 2));
+    uint4* orow = reinterpret_cast<uint4*>(xo + (int64_t)r * K);
+    const int nch = K / 8;
+    const int sub = lane & 3;       // my quarter of the group
+    for (int c0 = 0; c0 < nch; c0 += 32) {
+        const int c = c0 + lane;
+        const bool live = c < nch;  // K is a multiple of 128, so a group is never split by the end of the row
+        const uint4 v = live ? xrow[c] : make_uint4(0u, 0u, 0u, 0u);
+        uint32_t w[4] = {v.x, v.y, v.z, v.w};
+        // key = |x| (15 bits) above (31 - local channel): the maximum picks the largest magnitude, then the lowest channel
+        uint32_t key = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const uint32_t a = (w[i >> 1] >> ((i & 1) * 16)) & 0x7FFFu;
+            key = max(key, (a << 5) | (uint32_t)(31 - (sub * 8 + i)));
+        }
+        key = max(key, __shfl_xor_sync(0xFFFFFFFFu, key, 1));
+        key = max(key, __shfl_xor_sync(0xFFFFFFFFu, key, 2));
+        const int jstar = 31 - (int)(key & 31u);
+        const bool mine = (jstar >> 3) == sub;
+        const int istar = jstar & 7;
+        // the extracted element: bit copy out of the owning lane, +0 in its place
+        uint32_t picked = 0;
+        uint32_t o[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            if (mine && (istar >> 1) == k) {
+                const uint32_t keep = (istar & 1) ? 0x0000FFFFu : 0xFFFF0000u;
+                picked = (istar & 1) ? (w[k] >> 16) : (w[k] & 0xFFFFu);
+                o[k] = w[k] & ~keep;
+                w[k] &= keep;
+            }
+        }
+        picked = __shfl_sync(0xFFFFFFFFu, picked, (lane & ~3) + (jstar >> 3));
+        if (live) orow[c] = make_uint4(o[0], o[1], o[2], o[3]);
+        // CalculateScale / Quantize of what is left (as in Algorithm 2)
+        uint32_t am = 0;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) am = max(am, max(w[i] & 0x7FFFu, (w[i] >> 16) & 0x7FFFu));
+        am = max(am, __shfl_xor_sync(0xFFFFFFFFu, am, 1));
+        am = max(am, __shfl_xor_sync(0xFFFFFFFFu, am, 2));
+        const int ex = (int)(am >> 7);
+        int code = max(ex - 2, 0);
+        if (ex == 255) code = 255;
+        const float inv = __uint_as_float((uint32_t)(254 - min(code, 253)) << 23);
+        const uint32_t q = e2m1x8(__uint_as_float(w[0] << 16) * inv, __uint_as_float(w[0] & 0xFFFF0000u) * inv,
+                                  __uint_as_float(w[1] << 16) * inv, __uint_as_float(w[1] & 0xFFFF0000u) * inv,
+                                  __uint_as_float(w[2] << 16) * inv, __uint_as_float(w[2] & 0xFFFF0000u) * inv,
+                                  __uint_as_float(w[3] << 16) * inv, __uint_as_float(w[3] & 0xFFFF0000u) * inv);
+        if (live) qrow[c] = q;
+        // per-group outputs: groups 0-3 of the step sit in lanes 0,4,8,12, groups 4-7 in lanes 16,20,24,28
+        const int base = lane & 16;
+        uint32_t sfw = 0, idw = 0, v01 = 0, v23 = 0;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            sfw |= __shfl_sync(0xFFFFFFFFu, (uint32_t)code, base + 4 * k) << (8 * k);
+            idw |= __shfl_sync(0xFFFFFFFFu, (uint32_t)jstar, base + 4 * k) << (8 * k);
+            const uint32_t pv = __shfl_sync(0xFFFFFFFFu, picked, base + 4 * k);
+            if (k < 2) v01 |= pv << (16 * k); else v23 |= pv << (16 * (k - 2));
+        }
+        const int g0 = c0 / 4 + (lane >> 4) * 4;   // first of my half-warp's four groups
+        if ((lane & 15) == 0 && g0 < Kg) {
+            sf_row[(size_t)(g0 / 4) * 128] = sfw;
+            *reinterpret_cast<uint32_t*>(idx + (int64_t)r * Kg + g0) = idw;
+            *reinterpret_cast<uint2*>(val + (int64_t)r * Kg + g0) = make_uint2(v01, v23);
+        }
+    }
+}
+
+
 // ------------------------------------------------------------ grouped schedule
 // sched[0] = number of row tiles (tile_rows = 128 or 256 rows each, never crossing an expert boundary);
 // then four arrays of max_tiles entries: first row, end row (exclusive, the expert's end), first scale
@@ -554,6 +648,16 @@ cudaError_t launch_mxfp8_quant(const void* X, int64_t ldx, int M, int K, void* x
     return launch_pdl(mxfp8_quant_kernel, dim3((M_pad + MX8_ROWS_PER_CTA - 1) / MX8_ROWS_PER_CTA),
                       dim3(32 * MX8_ROWS_PER_CTA), 0, st, static_cast<const uint16_t*>(X), ldx, M, M_pad, K,
                       static_cast<uint8_t*>(x8), static_cast<uint8_t*>(sf));
+}
+
+cudaError_t launch_dyn_quant_extract(const void* X, int64_t ldx, int M, int K, void* xq, void* sf, void* xo, void* idx,
+                                     void* val, cudaStream_t st) {
+    if (M <= 0) return cudaSuccess;
+    const int M_pad = (M + 127) / 128 * 128;
+    return launch_pdl(dyn_quant_extract_kernel, dim3((M_pad + MX8_ROWS_PER_CTA - 1) / MX8_ROWS_PER_CTA),
+                      dim3(32 * MX8_ROWS_PER_CTA), 0, st, static_cast<const uint16_t*>(X), ldx, M, M_pad, K,
+                      static_cast<uint8_t*>(xq), static_cast<uint8_t*>(sf), static_cast<uint16_t*>(xo),
+                      static_cast<uint8_t*>(idx), static_cast<uint16_t*>(val));
 }
 
 cudaError_t launch_build_sched(const int32_t* off, int E, int32_t* sched128, int max_tiles128, int32_t* sched256,
