@@ -11,6 +11,7 @@ Function-to-paper map (details in the C file):
   fp8_quantize / fp8_gemm / fp8_linear Section 3.4 fallback (per-token E4M3)
   mxfp8_quantize / mxfp8_gemm / mxfp8_linear   Section 3.4 fallback in its 8-bit micro-scaling form (MXFP8)
   dyn_quantize_extract / dyn_prepare_weights / dyn_linear   the dynamic-protection control group of Section 4.2
+  nvfp4_quantize_extract / nvfp4_gemm / nvfp4_linear         the NVFP4 / G = 16 variant (efficiency table, G = 16)
   threshold / profile_indexing / clustering_density   Eq. 1-4, Algorithm 1 (offline profiling)
 """
 from __future__ import annotations
@@ -52,6 +53,10 @@ def lib():
         _lib.osc_ref_sf_bytes.argtypes = [C.c_int64, C.c_int64]
         _lib.osc_ref_sf_row_base.restype = C.c_int64
         _lib.osc_ref_e8m0_from_amax_emax.argtypes = [C.c_double, C.c_int]
+        _lib.osc_ref_sf16_index.restype = C.c_int64
+        _lib.osc_ref_sf16_index.argtypes = [C.c_int64, C.c_int64, C.c_int64]
+        _lib.osc_ref_sf16_bytes.restype = C.c_int64
+        _lib.osc_ref_sf16_bytes.argtypes = [C.c_int64, C.c_int64]
         _lib.osc_ref_threshold.restype = C.c_double
         _lib.osc_ref_threshold.argtypes = [C.c_void_p, C.c_int64, C.c_int, C.c_int, C.c_double]
         _lib.osc_ref_threshold_bits.restype = C.c_uint32
@@ -278,6 +283,55 @@ def dyn_linear(X: np.ndarray, W: np.ndarray, rows=None):
     act = dyn_quantize_extract(X)
     wts = dyn_prepare_weights(W)
     Y, T = gemm_dual(act, wts, rows)
+    return Y, T, act, wts
+
+
+def sf16_index(r: int, b: int, K: int) -> int:
+    return int(lib().osc_ref_sf16_index(r, b, K))
+
+
+def nvfp4_quantize_extract(X: np.ndarray, lut16: np.ndarray, e: int):
+    """NVFP4 / G = 16 form of Algorithm 2 with tensor-level scale 2^e: X bf16 [M,K], lut16 [K/16, C] entries -1..15
+    -> dict(xq [M,K/2], sf (E4M3 block scales, 128 x 4 block layout per 64 channels), xo [M,K_o_pad] scaled by 2^-e)."""
+    X = np.ascontiguousarray(X, dtype=np.uint16)
+    M, K = X.shape
+    lut16 = np.ascontiguousarray(lut16, dtype=np.int8).reshape(K // 16, -1)
+    Kg = K // 16
+    mask = np.zeros(Kg, np.uint32)
+    prefix = np.zeros(Kg, np.int32)
+    idx = np.zeros(max(K, 1), np.int32)
+    ko = lib().osc_ref_lut16_normalize(_p(lut16), Kg, lut16.shape[1], _p(mask), _p(prefix), _p(idx))
+    if ko < 0:
+        raise ValueError({-1: "lookup-table entry outside -1..15", -2: "duplicate channel in a group"}[ko])
+    kop = int(lib().osc_ref_ko_pad(ko))
+    xq = np.zeros((M, K // 2), np.uint8)
+    sf = np.zeros(int(lib().osc_ref_sf16_bytes(M, K)), np.uint8)
+    xo = np.zeros((M, kop), np.uint16)
+    rc = lib().osc_ref_nvfp4_quantize_extract(_p(X), C.c_int64(K), M, K, _p(lut16), lut16.shape[1], int(e), _p(xq),
+                                              _p(sf), _p(xo))
+    assert rc == ko
+    return {"xq": xq, "sf": sf, "xo": xo, "K_o": ko, "K_o_pad": kop, "idx_o": idx[:ko].copy(), "e": int(e)}
+
+
+def nvfp4_gemm(act: dict, wts: dict, rows=None):
+    xq, sfa, xo = act["xq"], act["sf"], act["xo"]
+    wq, sfw, wo = wts["xq"], wts["sf"], wts["xo"]
+    M, K2 = xq.shape
+    N = wq.shape[0]
+    if rows is None:
+        rows = np.arange(M, dtype=np.int32)
+    rows = np.ascontiguousarray(rows, dtype=np.int32)
+    Y = np.zeros((rows.size, N), np.float64)
+    T = np.zeros((rows.size, N), np.float64)
+    lib().osc_ref_nvfp4_gemm_rows(_p(xq), _p(sfa), _p(xo), _p(rows), rows.size, _p(wq), _p(sfw), _p(wo), N, 2 * K2,
+                                  xo.shape[1], act["e"] + wts["e"], _p(Y), _p(T))
+    return Y, T
+
+
+def nvfp4_linear(X, W, lut16, ex: int, ew: int, rows=None):
+    act = nvfp4_quantize_extract(X, lut16, ex)
+    wts = nvfp4_quantize_extract(W, lut16, ew)
+    Y, T = nvfp4_gemm(act, wts, rows)
     return Y, T, act, wts
 
 

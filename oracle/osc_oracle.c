@@ -378,6 +378,146 @@ int osc_ref_fp8_gemm_rows(const uint8_t* x8, const float* sx, const int32_t* row
     return 0;
 }
 
+/* ----------------- NVFP4 / G = 16 variant (Section 3.3 efficiency table, G = 16 row; Section 5) */
+
+/* The paper reports OSC on NVFP4 as well (blocks of 16, Table "Hardware Efficiency" row G = 16) without
+ * giving the arithmetic; this is the reading used here.  NVFP4 = E2M1 elements in blocks of 16 along K, one
+ * unsigned E4M3 scale per block, one tensor-level scale.  The tensor-level scale is restricted to a power of
+ * two, 2^e, so that the high-precision branch can live in the same scaled domain exactly:
+ *   x' = x * 2^-e                       (exact)
+ *   per block b (after the flagged channels are backed up and zeroed, as in Algorithm 2 with G = 16):
+ *     t  = fl32(amax_b' * fl32(1/6))                     amax_b' = max |x'| over the block
+ *     sb = E4M3_rne_sat(t)                               stored scale byte (0x00..0x7E)
+ *     q  = E2M1_rne_sat(fl32(x' * fl32(1 / value(sb))))  if value(sb) > 0, else the sign-only zero code
+ *   backed-up channels: xo = bf16 bits of x' (exponent shifted by -e: exact while it stays normal)
+ * The scale arithmetic is fp32 because it decides integer codes.  Scale bytes use the 128 x 4 block layout
+ * with one 512-byte block per 128 rows x 64 channels (four 16-blocks):
+ *   byte(r, b) = ((r/128)*(K/64) + b/4)*512 + (r%32)*16 + ((r%128)/32)*4 + b%4,  b = block index along K. */
+#define G16 16
+
+int64_t osc_ref_sf16_index(int64_t r, int64_t b, int64_t K) {
+    return ((r / 128) * (K / 64) + b / 4) * 512 + (r % 32) * 16 + ((r % 128) / 32) * 4 + (b % 4);
+}
+int64_t osc_ref_sf16_bytes(int64_t rows, int64_t K) { return ((rows + 127) / 128) * (K / 64) * 512; }
+
+/* table for 16-groups: lut[K/16][C], entries -1..15.  Same outputs as osc_ref_lut_normalize with one 16-bit
+ * mask per 16-group. Returns K_o, -1 (range) or -2 (duplicate). */
+int osc_ref_lut16_normalize(const int8_t* lut, int Kg, int C, uint32_t* mask, int32_t* prefix, int32_t* idx_o) {
+    int Ko = 0;
+    for (int k = 0; k < Kg; ++k) {
+        uint32_t m = 0;
+        for (int c = 0; c < C; ++c) {
+            int j = lut[(int64_t)k * C + c];
+            if (j < -1 || j >= G16) return -1;
+            if (j < 0) continue;
+            if (m & (1u << j)) return -2;
+            m |= 1u << j;
+        }
+        mask[k] = m;
+        prefix[k] = Ko;
+        for (int j = 0; j < G16; ++j)
+            if (m & (1u << j)) idx_o[Ko++] = k * G16 + j;
+    }
+    return Ko;
+}
+
+/* bf16 bits of v * 2^-e for a bf16 value v (exact for normal results; flushes to signed zero below) */
+static uint16_t bf16_scale_pow2(uint16_t b, int e) {
+    int ex = (b >> 7) & 0xFF;
+    if (ex == 0 || ex == 255) return b;              /* zero / subnormal / non-finite: left alone */
+    int ne = ex - e;
+    if (ne <= 0) return (uint16_t)(b & 0x8000);      /* underflow: signed zero */
+    if (ne >= 255) ne = 254;
+    return (uint16_t)((b & 0x807F) | (ne << 7));
+}
+
+int osc_ref_nvfp4_quantize_extract(const uint16_t* X, int64_t ldx, int M, int K, const int8_t* lut, int C, int e,
+                                   uint8_t* xq, uint8_t* sf, uint16_t* xo) {
+    if (K % 64) return -3;
+    int Kg = K / G16;
+    uint32_t* mask = (uint32_t*)malloc(sizeof(uint32_t) * (size_t)Kg);
+    int32_t* prefix = (int32_t*)malloc(sizeof(int32_t) * (size_t)Kg);
+    int32_t* idx_o = (int32_t*)malloc(sizeof(int32_t) * (size_t)K);
+    int Ko = osc_ref_lut16_normalize(lut, Kg, C, mask, prefix, idx_o);
+    if (Ko < 0) { free(mask); free(prefix); free(idx_o); return Ko; }
+    int Kop = osc_ref_ko_pad(Ko);
+    volatile float sixth = 1.0f / 6.0f;
+
+#pragma omp parallel for schedule(static)
+    for (int s = 0; s < M; ++s) {
+        const uint16_t* xrow = X + (int64_t)s * ldx;
+        for (int t = 0; t < Kop; ++t) xo[(int64_t)s * Kop + t] = 0;
+        for (int k = 0; k < Kg; ++k) {
+            float xr[G16];
+            int nib[G16];
+            for (int j = 0; j < G16; ++j) xr[j] = (float)bf16_value(bf16_scale_pow2(xrow[k * G16 + j], e));
+            int t = prefix[k];
+            for (int j = 0; j < G16; ++j) {
+                if (mask[k] & (1u << j)) {
+                    xo[(int64_t)s * Kop + t] = bf16_scale_pow2(xrow[k * G16 + j], e);
+                    ++t;
+                    xr[j] = 0.0f;
+                }
+            }
+            float amax = 0.0f;
+            for (int j = 0; j < G16; ++j) {
+                float a = fabsf(xr[j]);
+                if (a > amax) amax = a;
+            }
+            volatile float tt = amax * sixth;
+            int sb = osc_ref_e4m3_encode((double)tt) & 0x7F;
+            sf[osc_ref_sf16_index(s, k, K)] = (uint8_t)sb;
+            float sbv = (float)osc_ref_e4m3_decode(sb);
+            volatile float inv = sbv > 0.0f ? 1.0f / sbv : 0.0f;
+            for (int j = 0; j < G16; ++j) {
+                volatile float v = xr[j] * inv;
+                nib[j] = osc_ref_e2m1_encode((double)v);
+            }
+            for (int i = 0; i < G16 / 2; ++i)
+                xq[(int64_t)s * (K / 2) + k * (G16 / 2) + i] = (uint8_t)(nib[2 * i] | (nib[2 * i + 1] << 4));
+        }
+    }
+    free(mask); free(prefix); free(idx_o);
+    return Ko;
+}
+
+/* Y[i][n] = 2^(ex+ew) * ( sum_b sa*sw * sum_{c in b} a[c] w[c]  +  sum_t xo[t] wo[t] ), T likewise with
+ * absolute values; sa, sw = the E4M3 block scales. */
+int osc_ref_nvfp4_gemm_rows(const uint8_t* xq, const uint8_t* sfa, const uint16_t* xo, const int32_t* rows, int nrows,
+                            const uint8_t* wq, const uint8_t* sfw, const uint16_t* wo, int N, int K, int Kop,
+                            int e_sum, double* Y, double* T) {
+    int Kb = K / G16;
+#pragma omp parallel for schedule(static)
+    for (int n = 0; n < N; ++n) {
+        for (int i = 0; i < nrows; ++i) {
+            int64_t r = rows[i];
+            double acc = 0.0, tot = 0.0;
+            for (int b = 0; b < Kb; ++b) {
+                double p = 0.0, q = 0.0;
+                for (int c = b * G16; c < (b + 1) * G16; ++c) {
+                    int xa = xq[r * (K / 2) + c / 2], wa = wq[(int64_t)n * (K / 2) + c / 2];
+                    double pr = osc_ref_e2m1_decode((c & 1) ? (xa >> 4) : (xa & 15)) *
+                                osc_ref_e2m1_decode((c & 1) ? (wa >> 4) : (wa & 15));
+                    p += pr;
+                    q += fabs(pr);
+                }
+                double sc = osc_ref_e4m3_decode(sfa[osc_ref_sf16_index(r, b, K)]) *
+                            osc_ref_e4m3_decode(sfw[osc_ref_sf16_index(n, b, K)]);
+                acc += sc * p;
+                tot += sc * q;
+            }
+            for (int t = 0; t < Kop; ++t) {
+                double pr = bf16_value(xo[r * Kop + t]) * bf16_value(wo[(int64_t)n * Kop + t]);
+                acc += pr;
+                tot += fabs(pr);
+            }
+            Y[(int64_t)i * N + n] = ldexp(acc, e_sum);
+            T[(int64_t)i * N + n] = ldexp(tot, e_sum);
+        }
+    }
+    return 0;
+}
+
 /* ---------------- dynamic-protection baseline (Section 4.2, "OSC vs. Optimized Dynamic Protection") */
 
 /* The control group the paper compares against: per token and per 32-group the

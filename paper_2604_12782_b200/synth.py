@@ -174,3 +174,29 @@ def moe_down_case(E: int, counts: np.ndarray, K: int = 768, N: int = 2048, seed:
     W = Wp[np.arange(E) % pool]
     return {"X": _bf16(X), "W": np.ascontiguousarray(W), "off": offsets_from_counts(counts),
             "E": E, "K": K, "N": N, "M": Mtot}
+
+
+def nvfp4_tensor_exponent(bits: np.ndarray) -> int:
+    """Power-of-two tensor-level scale for an NVFP4 tensor: the smallest e with amax * 2^-e <= 6 * 448, so that
+    every block scale amax_b * 2^-e / 6 fits the E4M3 range.  An input recipe (calibration), handed to the oracle
+    and to the library alike."""
+    a = float(np.abs(bf16_bits_to_f64(bits)).max())
+    if a == 0.0:
+        return 0
+    return int(np.ceil(np.log2(a / (6.0 * 448.0))))
+
+
+def osc16_linear_case(seed: int, M: int, K: int, N: int):
+    """OSC inputs for 16-channel groups: one planted channel per 16-group (same recipe as osc_linear_case)."""
+    rng = np.random.default_rng(seed)
+    X = rng.standard_normal((M, K)).astype(np.float32)
+    Kg = K // 16
+    ch = rng.integers(0, 16, size=Kg)
+    cols = np.arange(Kg) * 16 + ch
+    factor = rng.uniform(20.0, 100.0, size=Kg).astype(np.float32)
+    hit = rng.random((M, Kg)) < 0.9
+    X[:, cols] *= np.where(hit, factor[None, :], 1.0).astype(np.float32)
+    X *= np.where(rng.random((M, K)) < 0.001, 30.0, 1.0).astype(np.float32)
+    W = (0.02 * rng.standard_normal((N, K))).astype(np.float32)
+    return {"X": f32_to_bf16_bits(X), "W": f32_to_bf16_bits(W), "lut16": ch.astype(np.int8).reshape(-1, 1),
+            "M": M, "K": K, "N": N}
