@@ -542,6 +542,36 @@ def run_sweep(args):
         del ws_, wk, Ys, Xs
         torch.cuda.empty_cache()
 
+    def nvfp4_row(name, M, K, N, seed=0):
+        """OSC on NVFP4 (blocks of 16, one flagged channel per block: K_o = K/16, as large as two per 32)."""
+        if not want(name):
+            return
+        case = synth.osc16_linear_case(seed, M, K, N)
+        ex, ew = synth.nvfp4_tensor_exponent(case["X"]), synth.nvfp4_tensor_exponent(case["W"])
+        X0, W0 = dev_bf16(torch, case["X"]), dev_bf16(torch, case["W"])
+        n = NSETS
+        Xs = [X0 if i == 0 else torch.roll(X0, 97 * i, 0).contiguous() for i in range(n)]
+        ws_ = [B.osc_nvfp4_prepare_weights(W0 if i == 0 else torch.roll(W0, 61 * i, 0).contiguous(), case["lut16"], ew)
+               for i in range(n)]
+        sz = B.osc_nvfp4_act_sizes(ws_[0], M)
+        wk = [torch.empty(sz.workspace_bytes, dtype=torch.uint8, device="cuda") for _ in range(n)]
+        Ys = [torch.empty(M, N, dtype=torch.bfloat16, device="cuda") for _ in range(n)]
+        ms = time_loop(torch, lambda i: B.osc_nvfp4_linear(ws_[i % n], Xs[i % n], ex, Ys[i % n], wk[i % n]), steps, warm)
+        tq = time_loop(torch, lambda i: B.osc_nvfp4_quantize_extract(
+            ws_[i % n], Xs[i % n], ex, wk[i % n][sz.xq_offset:], wk[i % n][sz.sfa_offset:], wk[i % n][sz.xo_offset:]),
+            steps, warm)
+        tg = time_loop(torch, lambda i: B.osc_nvfp4_gemm(
+            ws_[i % n], wk[i % n][sz.xq_offset:], wk[i % n][sz.sfa_offset:], wk[i % n][sz.xo_offset:], M, ex, Ys[i % n]),
+            steps, warm)
+        B.osc_sync_check()
+        Ko = ws_[0].K_o
+        f4, f16 = roofline.osc_flops(M, N, K, Ko)
+        troof = roofline.osc_roofline_seconds(M, N, K, Ko, peaks)
+        rows.append({"name": name, "M": M, "K": K, "N": N, "K_o": Ko, "ms": ms, "quant_ms": tq, "gemm_ms": tg,
+                     "tflops": (f4 + f16) / ms / 1e9, "pct_roofline": 100 * troof / (ms * 1e-3), "roof_us": troof * 1e6})
+        del ws_, wk, Ys, Xs
+        torch.cuda.empty_cache()
+
     for M in (16, 64, 128, 2048, 8192):
         osc_row("qkv", M, 4096, 6144, 2)
     for M in (16, 64, 128, 2048, 8192):
@@ -549,6 +579,8 @@ def run_sweep(args):
         fp8_row("down_fp8", M, 12288, 4096)
         if M >= 128:
             mxfp8_row("down_mxfp8", M, 12288, 4096)
+    nvfp4_row("qkv.nvfp4_g16", 8192, 4096, 6144)
+    nvfp4_row("qkv.nvfp4_g16", 2048, 4096, 6144)
     dyn_row("qkv.dynamic_protection", 8192, 4096, 6144, 2)
     dyn_row("qkv.dynamic_protection", 2048, 4096, 6144, 2)
     osc_row("layer.qkv", 4096, 4096, 6144, 2)

@@ -293,6 +293,34 @@ osc_status osc_dyn_quantize_extract(const osc_weights* w, const void* X, int M, 
 osc_status osc_dyn_linear(const osc_weights* w, const void* X, int M, int64_t ldx, void* Y, int64_t ldy,
                           void* workspace, size_t workspace_bytes, void* stream);
 
+/* --------------------------------------------- NVFP4 / G = 16 variant of the OSC path */
+
+/* The paper reports OSC on NVFP4 too (efficiency table, row G = 16; Section 5) without stating the arithmetic.
+ * These calls are the reading taken here: E2M1 elements in blocks of 16 along K, one unsigned E4M3 scale per
+ * block, and a tensor-level scale restricted to a power of two (2^ex for the activations, 2^ew for the weights,
+ * chosen by the caller, e.g. the smallest e with amax * 2^-e <= 6 * 448), so that the high-precision branch
+ * lives in the same scaled domain exactly and both paths share one accumulator:
+ *   x' = x * 2^-e;  per block, after the flagged channels are backed up (as bf16(x')) and zeroed:
+ *   t = fl32(amax' * fl32(1/6)), scale byte = E4M3(t) (nearest even, saturating),
+ *   codes = E2M1(fl32(x' * fl32(1/scale))) (sign-only zeros when the scale is zero);
+ *   Y = bf16( 2^(ex+ew) * ( sum_b sa*sw * sum_{k in b} xq*wq  +  sum_t xo*wo ) ).
+ * The table lists local channels 0..15 per 16-channel group: lut16 is host int8 [K/16][lut_c], -1 = none.
+ * Scale bytes: 512-byte blocks of 128 rows x 64 channels,
+ *   byte(r, b) = ((r/128)*(K/64) + b/4)*512 + (r%32)*16 + ((r%128)/32)*4 + b%4   (b = block index along K),
+ * ceil(rows/128) * (K/64) * 512 bytes per tensor.  Dense problems only; same conventions as osc_linear.
+ * The handle is an osc_weights accepted only by the osc_nvfp4_* calls and osc_weights_destroy;
+ * osc_nvfp4_weight_sizes and osc_nvfp4_act_sizes fill the structs of their MXFP4 counterparts. */
+osc_status osc_nvfp4_weight_sizes(int N, int K, const int8_t* lut16, int lut_c, osc_weight_sizes_t* out);
+osc_status osc_nvfp4_prepare_weights(const void* W, int N, int K, int64_t ldw, const int8_t* lut16, int lut_c, int ew,
+                                     void* wq, void* sfw, void* wo, void* meta, void* stream, osc_weights** out);
+osc_status osc_nvfp4_act_sizes(const osc_weights* w, int M, osc_act_sizes_t* out);
+osc_status osc_nvfp4_quantize_extract(const osc_weights* w, const void* X, int M, int64_t ldx, int ex, void* xq,
+                                      void* sfa, void* xo, void* stream);
+osc_status osc_nvfp4_gemm(const osc_weights* w, const void* xq, const void* sfa, const void* xo, int M, int ex, void* Y,
+                          int64_t ldy, void* stream);
+osc_status osc_nvfp4_linear(const osc_weights* w, const void* X, int M, int64_t ldx, int ex, void* Y, int64_t ldy,
+                            void* workspace, size_t workspace_bytes, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -389,7 +389,7 @@ int osc_ref_fp8_gemm_rows(const uint8_t* x8, const float* sx, const int32_t* row
  *     t  = fl32(amax_b' * fl32(1/6))                     amax_b' = max |x'| over the block
  *     sb = E4M3_rne_sat(t)                               stored scale byte (0x00..0x7E)
  *     q  = E2M1_rne_sat(fl32(x' * fl32(1 / value(sb))))  if value(sb) > 0, else the sign-only zero code
- *   backed-up channels: xo = bf16 bits of x' (exponent shifted by -e: exact while it stays normal)
+ *   backed-up channels: xo = x' rounded to bf16 (exact while x' is a normal bf16 number)
  * The scale arithmetic is fp32 because it decides integer codes.  Scale bytes use the 128 x 4 block layout
  * with one 512-byte block per 128 rows x 64 channels (four 16-blocks):
  *   byte(r, b) = ((r/128)*(K/64) + b/4)*512 + (r%32)*16 + ((r%128)/32)*4 + b%4,  b = block index along K. */
@@ -421,14 +421,15 @@ int osc_ref_lut16_normalize(const int8_t* lut, int Kg, int C, uint32_t* mask, in
     return Ko;
 }
 
-/* bf16 bits of v * 2^-e for a bf16 value v (exact for normal results; flushes to signed zero below) */
+/* bf16 bits of the value v * 2^-e rounded to bf16 (nearest even): exact whenever the result is a normal
+ * bf16 number, i.e. always for the tensor scales a calibration would pick. */
 static uint16_t bf16_scale_pow2(uint16_t b, int e) {
-    int ex = (b >> 7) & 0xFF;
-    if (ex == 0 || ex == 255) return b;              /* zero / subnormal / non-finite: left alone */
-    int ne = ex - e;
-    if (ne <= 0) return (uint16_t)(b & 0x8000);      /* underflow: signed zero */
-    if (ne >= 255) ne = 254;
-    return (uint16_t)((b & 0x807F) | (ne << 7));
+    float f = (float)ldexp(bf16_value(b), -e); /* exact: 8 significant bits, fp32 exponent range */
+    uint32_t u;
+    memcpy(&u, &f, sizeof u);
+    if ((u & 0x7F800000u) == 0x7F800000u) return (uint16_t)(u >> 16); /* non-finite: truncated */
+    u += 0x7FFFu + ((u >> 16) & 1u);
+    return (uint16_t)(u >> 16);
 }
 
 int osc_ref_nvfp4_quantize_extract(const uint16_t* X, int64_t ldx, int M, int K, const int8_t* lut, int C, int e,
@@ -450,7 +451,7 @@ int osc_ref_nvfp4_quantize_extract(const uint16_t* X, int64_t ldx, int M, int K,
         for (int k = 0; k < Kg; ++k) {
             float xr[G16];
             int nib[G16];
-            for (int j = 0; j < G16; ++j) xr[j] = (float)bf16_value(bf16_scale_pow2(xrow[k * G16 + j], e));
+            for (int j = 0; j < G16; ++j) xr[j] = (float)ldexp(bf16_value(xrow[k * G16 + j]), -e); /* exact */
             int t = prefix[k];
             for (int j = 0; j < G16; ++j) {
                 if (mask[k] & (1u << j)) {

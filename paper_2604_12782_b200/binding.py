@@ -90,6 +90,12 @@ _SIGS = {
     "osc_dyn_act_sizes": (_i, [_vp, _i, C.POINTER(DynActSizes)]),
     "osc_dyn_quantize_extract": (_i, [_vp, _vp, _i, _i64, _vp, _vp, _vp, _vp, _vp, _vp]),
     "osc_dyn_linear": (_i, [_vp, _vp, _i, _i64, _vp, _i64, _vp, _sz, _vp]),
+    "osc_nvfp4_weight_sizes": (_i, [_i, _i, _vp, _i, C.POINTER(WeightSizes)]),
+    "osc_nvfp4_prepare_weights": (_i, [_vp, _i, _i, _i64, _vp, _i, _i, _vp, _vp, _vp, _vp, _vp, C.POINTER(_vp)]),
+    "osc_nvfp4_act_sizes": (_i, [_vp, _i, C.POINTER(ActSizes)]),
+    "osc_nvfp4_quantize_extract": (_i, [_vp, _vp, _i, _i64, _i, _vp, _vp, _vp, _vp]),
+    "osc_nvfp4_gemm": (_i, [_vp, _vp, _vp, _vp, _i, _i, _vp, _i64, _vp]),
+    "osc_nvfp4_linear": (_i, [_vp, _vp, _i, _i64, _i, _vp, _i64, _vp, _sz, _vp]),
     "osc_mxfp8_weight_sizes": (_i, [_i, _i, C.POINTER(Mxfp8WeightSizes)]),
     "osc_mxfp8_prepare_weights": (_i, [_vp, _i, _i, _i64, _vp, _vp, _vp, C.POINTER(_vp)]),
     "osc_mxfp8_weights_destroy": (_i, [_vp]),
@@ -414,3 +420,55 @@ def osc_dyn_linear(w: OscWeights, X: torch.Tensor, Y: torch.Tensor, workspace: t
     M = X.shape[0]
     _check(_lib.osc_dyn_linear(w.ptr, _ptr(X), M, X.stride(0) if M else w.K, _ptr(Y), Y.stride(0) if M else w.N,
                                _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)))
+
+
+# --------------------------------------------------------------- NVFP4 / G = 16 variant
+
+def _lut16(lut, K):
+    lut = np.ascontiguousarray(lut, dtype=np.int8)
+    return lut.reshape(K // 16, -1)
+
+
+def osc_nvfp4_weight_sizes(N: int, K: int, lut16) -> WeightSizes:
+    lut16 = _lut16(lut16, K)
+    out = WeightSizes()
+    _check(_lib.osc_nvfp4_weight_sizes(N, K, lut16.ctypes.data, lut16.shape[1], C.byref(out)))
+    return out
+
+
+def osc_nvfp4_prepare_weights(W: torch.Tensor, lut16, ew: int, stream=None) -> OscWeights:
+    N, K = W.shape
+    lut16 = _lut16(lut16, K)
+    sz = osc_nvfp4_weight_sizes(N, K, lut16)
+    bufs = {k: _alloc(getattr(sz, k + "_bytes"), W.device) for k in ("wq", "sfw", "wo", "meta")}
+    h = _vp()
+    _check(_lib.osc_nvfp4_prepare_weights(_ptr(W), N, K, W.stride(0), lut16.ctypes.data, lut16.shape[1], int(ew),
+                                          _ptr(bufs["wq"]), _ptr(bufs["sfw"]), _ptr(bufs["wo"]) if sz.wo_bytes else None,
+                                          _ptr(bufs["meta"]), _stream(stream), C.byref(h)))
+    w = OscWeights(h.value, bufs)
+    w.E, w.N, w.K, w.K_o, w.K_o_pad, w.sizes, w.ew = 1, N, K, sz.K_o, sz.K_o_pad, sz, int(ew)
+    return w
+
+
+def osc_nvfp4_act_sizes(w: OscWeights, M: int) -> ActSizes:
+    out = ActSizes()
+    _check(_lib.osc_nvfp4_act_sizes(w.ptr, M, C.byref(out)))
+    return out
+
+
+def osc_nvfp4_quantize_extract(w: OscWeights, X: torch.Tensor, ex: int, xq, sfa, xo, stream=None):
+    M = X.shape[0]
+    _check(_lib.osc_nvfp4_quantize_extract(w.ptr, _ptr(X), M, X.stride(0) if M else w.K, int(ex), _ptr(xq), _ptr(sfa),
+                                           _ptr(xo) if w.K_o_pad else None, _stream(stream)))
+
+
+def osc_nvfp4_gemm(w: OscWeights, xq, sfa, xo, M: int, ex: int, Y: torch.Tensor, stream=None):
+    _check(_lib.osc_nvfp4_gemm(w.ptr, _ptr(xq), _ptr(sfa), _ptr(xo) if w.K_o_pad else None, M, int(ex), _ptr(Y),
+                               Y.stride(0) if M else w.N, _stream(stream)))
+
+
+def osc_nvfp4_linear(w: OscWeights, X: torch.Tensor, ex: int, Y: torch.Tensor, workspace: torch.Tensor, stream=None):
+    M = X.shape[0]
+    _check(_lib.osc_nvfp4_linear(w.ptr, _ptr(X), M, X.stride(0) if M else w.K, int(ex), _ptr(Y),
+                                 Y.stride(0) if M else w.N, _ptr(workspace),
+                                 workspace.numel() * workspace.element_size(), _stream(stream)))

@@ -193,6 +193,8 @@ struct osc_weights {
     int E, N, K, Ko, Kop;
     bool grouped;
     bool dynamic;   // weights of the dynamic-protection control group: whole-matrix MXFP4 + the bf16 matrix (Kop = K)
+    bool nvfp4;     // NVFP4 / G = 16 variant: E4M3 block scales per 16 channels, tensor-level scale 2^ew
+    int ew;
     const uint8_t *wq, *sfw;
     const uint16_t* wo;
     const uint32_t* mask;
@@ -368,6 +370,7 @@ static int max_tiles256(int M, int E) { return M / 256 + E; }
 
 osc_status osc_act_sizes(const osc_weights* w, int M, osc_act_sizes_t* out) {
     if (!w || !out) return fail(OSC_ERR_INVALID_ARG, "null argument");
+    if (w->nvfp4) return fail(OSC_ERR_INVALID_ARG, "NVFP4 weights: use osc_nvfp4_act_sizes");
     if (M < 0) return fail(OSC_ERR_INVALID_ARG, "M = %d is negative", M);
     const int64_t max_tiles = w->grouped ? (int64_t)M / 128 + w->E : ((int64_t)M + 127) / 128;
     out->xq_bytes = (size_t)M * (w->K / 2);
@@ -382,8 +385,11 @@ osc_status osc_act_sizes(const osc_weights* w, int M, osc_act_sizes_t* out) {
     return OSC_OK;
 }
 
-static osc_status check_act(const osc_weights* w, const void* X, int M, int64_t ldx, bool dynamic = false) {
+static osc_status check_act(const osc_weights* w, const void* X, int M, int64_t ldx, bool dynamic = false,
+                            bool nvfp4 = false) {
     if (!w) return fail(OSC_ERR_INVALID_ARG, "weights handle is null");
+    if (w->nvfp4 != nvfp4)
+        return fail(OSC_ERR_INVALID_ARG, nvfp4 ? "MXFP4 weights: use osc_linear" : "NVFP4 weights: use osc_nvfp4_linear");
     if (w->dynamic != dynamic)
         return fail(OSC_ERR_INVALID_ARG, dynamic ? "static-table weights: use osc_linear" : "dynamic-protection weights: use osc_dyn_linear");
     if (M < 0) return fail(OSC_ERR_INVALID_ARG, "M = %d is negative", M);
@@ -479,6 +485,7 @@ osc_status osc_gemm_dual(const osc_weights* w, const void* xq, const void* sfa, 
     if (!w) return fail(OSC_ERR_INVALID_ARG, "weights handle is null");
     if (M < 0) return fail(OSC_ERR_INVALID_ARG, "M = %d is negative", M);
     if (w->grouped) return fail(OSC_ERR_INVALID_ARG, "grouped weights: use osc_linear_grouped");
+    if (w->nvfp4) return fail(OSC_ERR_INVALID_ARG, "NVFP4 weights: use osc_nvfp4_gemm");
     return gemm_impl(w, xq, sfa, xo, M, Y, ldy, nullptr, 0, nullptr, 0, static_cast<cudaStream_t>(stream));
 }
 
@@ -898,6 +905,177 @@ osc_status osc_dyn_linear(const osc_weights* w, const void* X, int M, int64_t ld
                                                 ws + sz.idx_offset, ws + sz.val_offset, stream)) return s;
     return gemm_impl(w, ws + sz.xq_offset, ws + sz.sfa_offset, ws + sz.xo_offset, M, Y, ldy, nullptr, 0, nullptr, 0,
                      static_cast<cudaStream_t>(stream));
+}
+
+// ------------------------------------------------ NVFP4 / G = 16 variant
+
+static size_t sf16_bytes(int64_t rows, int K) { return (size_t)((rows + 127) / 128) * (K / 64) * 512; }
+
+// table for 16-channel groups [K/16][C] (entries -1..15) -> the 32-group form the kernels use [K/32][2C]
+static osc_status widen_lut16(const int8_t* lut16, int K, int C, std::vector<int8_t>* out) {
+    if (K <= 0 || K % 128) return fail(OSC_ERR_SHAPE, "K = %d must be a positive multiple of 128", K);
+    if (C < 0 || C > 16) return fail(OSC_ERR_INVALID_ARG, "lut_c = %d outside 0..16", C);
+    if (C > 0 && !lut16) return fail(OSC_ERR_INVALID_ARG, "lut is null");
+    out->assign((size_t)(K / 32) * 2 * (C > 0 ? C : 1), -1);
+    for (int g = 0; g < K / 16; ++g)
+        for (int c = 0; c < C; ++c) {
+            const int j = lut16[(size_t)g * C + c];
+            if (j < -1 || j > 15) return fail(OSC_ERR_LUT, "table entry %d of group %d outside -1..15", j, g);
+            if (j >= 0) (*out)[(size_t)(g / 2) * 2 * C + (g & 1) * C + c] = (int8_t)(j + 16 * (g & 1));
+        }
+    return OSC_OK;
+}
+
+osc_status osc_nvfp4_weight_sizes(int N, int K, const int8_t* lut16, int lut_c, osc_weight_sizes_t* out) {
+    if (!out) return fail(OSC_ERR_INVALID_ARG, "out is null");
+    if (osc_status s = check_nk(1, N, K)) return s;
+    std::vector<int8_t> lut;
+    if (osc_status s = widen_lut16(lut16, K, lut_c, &lut)) return s;
+    Table t;
+    if (osc_status s = parse_lut(lut.data(), K, 2 * (lut_c > 0 ? lut_c : 1), &t)) return s;
+    out->K_o = t.Ko;
+    out->K_o_pad = t.Kop;
+    out->wq_bytes = (size_t)N * (K / 2);
+    out->sfw_bytes = sf16_bytes(N, K);
+    out->wo_bytes = (size_t)N * t.Kop * 2;
+    out->meta_bytes = meta_table_bytes(K, t.Ko);
+    return OSC_OK;
+}
+
+osc_status osc_nvfp4_prepare_weights(const void* W, int N, int K, int64_t ldw, const int8_t* lut16, int lut_c, int ew,
+                                     void* wq, void* sfw, void* wo, void* meta, void* stream, osc_weights** out) {
+    if (!out) return fail(OSC_ERR_INVALID_ARG, "out is null");
+    *out = nullptr;
+    if (osc_status s = check_nk(1, N, K)) return s;
+    if (ew < -100 || ew > 100) return fail(OSC_ERR_INVALID_ARG, "tensor exponent %d outside -100..100", ew);
+    std::vector<int8_t> lut;
+    if (osc_status s = widen_lut16(lut16, K, lut_c, &lut)) return s;
+    Table t;
+    if (osc_status s = parse_lut(lut.data(), K, 2 * (lut_c > 0 ? lut_c : 1), &t)) return s;
+    if (!W || !wq || !sfw || !meta || (t.Kop > 0 && !wo)) return fail(OSC_ERR_INVALID_ARG, "null device pointer");
+    if (ldw < K) return fail(OSC_ERR_SHAPE, "ldw = %lld < K", (long long)ldw);
+    if (ldw % 8 || !aligned16(W) || !aligned16(wq) || !aligned16(sfw) || !aligned16(meta) || !aligned16(wo))
+        return fail(OSC_ERR_ALIGN, "pointers must be 16-byte aligned and ldw a multiple of 8");
+    DeviceInfo di;
+    if (osc_status s = device_info(&di)) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int Kg = K / 32;
+    uint8_t* m8 = static_cast<uint8_t*>(meta);
+    cudaError_t e = cudaMemcpyAsync(m8, t.mask.data(), (size_t)Kg * 4, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(m8 + (size_t)Kg * 4, t.prefix.data(), (size_t)Kg * 4, cudaMemcpyHostToDevice, st);
+    if (e == cudaSuccess && t.Ko > 0)
+        e = cudaMemcpyAsync(m8 + (size_t)Kg * 8, t.idx.data(), (size_t)t.Ko * 4, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpyAsync(meta)");
+    osc_weights* w = new (std::nothrow) osc_weights();
+    if (!w) return fail(OSC_ERR_INVALID_ARG, "out of host memory");
+    w->E = 1; w->N = N; w->K = K; w->Ko = t.Ko; w->Kop = t.Kop; w->grouped = false; w->dynamic = false;
+    w->nvfp4 = true; w->ew = ew;
+    w->wq = static_cast<const uint8_t*>(wq);
+    w->sfw = static_cast<const uint8_t*>(sfw);
+    w->wo = static_cast<const uint16_t*>(wo);
+    w->mask = reinterpret_cast<const uint32_t*>(m8);
+    w->prefix = reinterpret_cast<const int32_t*>(m8 + (size_t)Kg * 4);
+    w->idx_o = reinterpret_cast<const int32_t*>(m8 + (size_t)Kg * 8);
+    w->num_sms = di.num_sms;
+    CUtensorMap tm_w;
+    osc_status s = make_tmap_x(&tm_w, W, N, K, ldw);
+    if (s == OSC_OK) {
+        e = launch_quant_extract_nvfp4(tm_w, N, K, w->mask, w->prefix, w->idx_o, wq, sfw, t.Kop ? wo : nullptr, t.Ko, t.Kop,
+                                       di.num_sms, ew, st);
+        if (e != cudaSuccess) s = cuda_fail(e, "quant_extract_kernel(nvfp4 weights)");
+    }
+    for (int v = 0; v < 2 && s == OSC_OK; ++v) {
+        const int half = (v == 0 ? 192 : 256) / 2;
+        s = make_tmap(&w->tm_b2[v], wq, false, (uint64_t)N, K / 2, K / 2, half);
+        if (s == OSC_OK && t.Kop > 0)
+            s = make_tmap(&w->tm_bo2[v], wo, true, (uint64_t)N, (uint64_t)t.Kop * 2, (uint64_t)t.Kop * 2, half);
+    }
+    if (s == OSC_OK) s = make_tmap_sf(&w->tm_sfw, sfw, (uint64_t)sf16_bytes(N, K) / 512, 4);
+    if (s != OSC_OK) { delete w; return s; }
+    *out = w;
+    return OSC_OK;
+}
+
+osc_status osc_nvfp4_act_sizes(const osc_weights* w, int M, osc_act_sizes_t* out) {
+    if (!w || !out) return fail(OSC_ERR_INVALID_ARG, "null argument");
+    if (!w->nvfp4) return fail(OSC_ERR_INVALID_ARG, "MXFP4 weights: use osc_act_sizes");
+    if (M < 0) return fail(OSC_ERR_INVALID_ARG, "M = %d is negative", M);
+    out->xq_bytes = (size_t)M * (w->K / 2);
+    out->sfa_bytes = sf16_bytes(M, w->K);
+    out->xo_bytes = (size_t)M * w->Kop * 2;
+    out->sched_bytes = 0;
+    out->xq_offset = 0;
+    out->sfa_offset = out->xq_offset + align256(out->xq_bytes);
+    out->xo_offset = out->sfa_offset + align256(out->sfa_bytes);
+    out->sched_offset = out->xo_offset + align256(out->xo_bytes);
+    out->workspace_bytes = out->sched_offset;
+    return OSC_OK;
+}
+
+osc_status osc_nvfp4_quantize_extract(const osc_weights* w, const void* X, int M, int64_t ldx, int ex, void* xq,
+                                      void* sfa, void* xo, void* stream) {
+    if (osc_status s = check_act(w, X, M, ldx, false, true)) return s;
+    if (ex < -100 || ex > 100) return fail(OSC_ERR_INVALID_ARG, "tensor exponent %d outside -100..100", ex);
+    if (M == 0) return OSC_OK;
+    if (!xq || !sfa || (w->Kop > 0 && !xo)) return fail(OSC_ERR_INVALID_ARG, "null output pointer");
+    if (!aligned16(xq) || !aligned16(sfa) || !aligned16(xo)) return fail(OSC_ERR_ALIGN, "outputs must be 16-byte aligned");
+    CUtensorMap tm_x;
+    if (osc_status s = make_tmap_x(&tm_x, X, M, w->K, ldx)) return s;
+    cudaError_t e = launch_quant_extract_nvfp4(tm_x, M, w->K, w->mask, w->prefix, w->idx_o, xq, sfa, w->Kop ? xo : nullptr,
+                                               w->Ko, w->Kop, w->num_sms, ex, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(e, "quant_extract_kernel(nvfp4)");
+    return OSC_OK;
+}
+
+osc_status osc_nvfp4_gemm(const osc_weights* w, const void* xq, const void* sfa, const void* xo, int M, int ex, void* Y,
+                          int64_t ldy, void* stream) {
+    if (!w) return fail(OSC_ERR_INVALID_ARG, "weights handle is null");
+    if (!w->nvfp4) return fail(OSC_ERR_INVALID_ARG, "MXFP4 weights: use osc_gemm_dual");
+    if (M < 0) return fail(OSC_ERR_INVALID_ARG, "M = %d is negative", M);
+    if (M == 0) return OSC_OK;
+    if (!xq || !sfa || !Y || (w->Kop > 0 && !xo)) return fail(OSC_ERR_INVALID_ARG, "null device pointer");
+    if (ldy < w->N) return fail(OSC_ERR_SHAPE, "ldy = %lld < N = %d", (long long)ldy, w->N);
+    if (ldy % 8 || !aligned16(Y) || !aligned16(xq) || !aligned16(sfa) || !aligned16(xo))
+        return fail(OSC_ERR_ALIGN, "pointers must be 16-byte aligned and ldy a multiple of 8");
+    const int es = ex + w->ew;
+    if (es < -120 || es > 120) return fail(OSC_ERR_INVALID_ARG, "sum of the tensor exponents %d outside -120..120", es);
+    GemmArgs a;
+    memset(&a, 0, sizeof a);
+    if (osc_status s = make_tmap(&a.tm_a, xq, false, M, w->K / 2, w->K / 2, 128)) return s;
+    const int bn = gemm_pair_block_n(false, false, (M + 255) / 256, w->N, (w->K + 255) / 256 + w->Kop / 64, w->num_sms);
+    a.tm_b = w->tm_b2[bn == 256];
+    if (w->Kop > 0) {
+        if (osc_status s = make_tmap(&a.tm_ao, xo, true, M, (uint64_t)w->Kop * 2, (uint64_t)w->Kop * 2, 128)) return s;
+        a.tm_bo = w->tm_bo2[bn == 256];
+    }
+    a.tm_sfw = w->tm_sfw;
+    if (osc_status s = make_tmap_sf(&a.tm_sfa, sfa, (uint64_t)sf16_bytes(M, w->K) / 512, 4)) return s;
+    if (osc_status s = make_tmap(&a.tm_y, Y, true, M, (uint64_t)w->N * 2, (uint64_t)ldy * 2, 32)) return s;
+    a.sfa = static_cast<const uint8_t*>(sfa);
+    a.sfw = w->sfw;
+    a.Y = static_cast<uint16_t*>(Y);
+    a.ldy = ldy;
+    a.M = M; a.N = w->N; a.K = w->K; a.Kop = w->Kop;
+    a.num_sms = w->num_sms;
+    a.out_scale = ldexpf(1.0f, es);
+    cudaError_t e = launch_gemm_nvf4_pair(a, bn, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(e, "gemm_pair_kernel(nvfp4)");
+    return OSC_OK;
+}
+
+osc_status osc_nvfp4_linear(const osc_weights* w, const void* X, int M, int64_t ldx, int ex, void* Y, int64_t ldy,
+                            void* workspace, size_t workspace_bytes, void* stream) {
+    if (osc_status s = check_act(w, X, M, ldx, false, true)) return s;
+    if (M == 0) return OSC_OK;
+    osc_act_sizes_t sz;
+    osc_nvfp4_act_sizes(w, M, &sz);
+    if (!workspace || !aligned16(workspace)) return fail(OSC_ERR_ALIGN, "workspace must be non-null and 16-byte aligned");
+    if (workspace_bytes < sz.workspace_bytes)
+        return fail(OSC_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", workspace_bytes, sz.workspace_bytes);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    if (osc_status s = osc_nvfp4_quantize_extract(w, X, M, ldx, ex, ws + sz.xq_offset, ws + sz.sfa_offset,
+                                                  ws + sz.xo_offset, stream)) return s;
+    return osc_nvfp4_gemm(w, ws + sz.xq_offset, ws + sz.sfa_offset, ws + sz.xo_offset, M, ex, Y, ldy, stream);
 }
 
 }  // extern "C"

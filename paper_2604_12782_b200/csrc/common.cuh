@@ -30,6 +30,9 @@ static cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
 cudaError_t launch_quant_extract(const CUtensorMap& tm_x, int M, int K, const uint32_t* mask,
                                  const int32_t* prefix, const int32_t* idx_o, void* xq, void* sf, void* xo, int Ko, int Kop,
                                  const int32_t* sched, int max_tiles, int num_sms, cudaStream_t st);
+cudaError_t launch_quant_extract_nvfp4(const CUtensorMap& tm_x, int M, int K, const uint32_t* mask,
+                                       const int32_t* prefix, const int32_t* idx_o, void* xq, void* sf, void* xo, int Ko,
+                                       int Kop, int num_sms, int tensor_e, cudaStream_t st);
 cudaError_t launch_fp8_quant(const void* X, int64_t ldx, int M, int K, void* x8, void* sx, cudaStream_t st);
 cudaError_t launch_mxfp8_quant(const void* X, int64_t ldx, int M, int K, void* x8, void* sf, cudaStream_t st);
 cudaError_t launch_dyn_quant_extract(const void* X, int64_t ldx, int M, int K, void* xq, void* sf, void* xo, void* idx,
@@ -55,6 +58,7 @@ struct GemmArgs {
     const uint8_t* sfw;  // weight scales, block layout, per expert
     const float* sx;     // FP8 mode: per-row activation scale
     const float* sw;     // FP8 mode: per-output-row weight scale [E*N]
+    float out_scale;     // NVFP4 mode: product of the two power-of-two tensor scales, applied before the bf16 rounding
     uint16_t* Y;         // bf16 [rows, ldy]
     int64_t ldy;
     int M;               // rows (dense) / total rows (grouped)
@@ -73,6 +77,7 @@ int gemm_block_n(int row_tiles, int N, int num_sms);
 cudaError_t launch_gemm_dual_pair(const GemmArgs& a, int bn, cudaStream_t st);
 cudaError_t launch_gemm_fp8_pair(const GemmArgs& a, int bn, cudaStream_t st);
 cudaError_t launch_gemm_mxf8_pair(const GemmArgs& a, int bn, cudaStream_t st);
+cudaError_t launch_gemm_nvf4_pair(const GemmArgs& a, int bn, cudaStream_t st);
 int gemm_pair_block_n(bool fp8, bool allow_240, long row_tiles, int N, int stages, int num_sms);
 
 // gemm3_kernels.cu (few rows: operands swapped, K split over a cluster)

@@ -34,6 +34,7 @@ namespace pair {
 constexpr int MODE_OSC = 0;
 constexpr int MODE_FP8 = 1;
 constexpr int MODE_MXF8 = 2;   // block-scaled FP8 (MXFP8): scales as in MODE_OSC, no BF16 branch
+constexpr int MODE_NVF4 = 3;   // Eq. 5 on NVFP4: E2M1 with an E4M3 scale per 16 channels, BF16 branch, output scale
 constexpr int BM = 128;        // rows per CTA; the pair covers 256
 constexpr int ROW_BYTES = 128;
 constexpr int A_BYTES = BM * ROW_BYTES;
@@ -53,7 +54,10 @@ struct Cfg {
     static constexpr int SFB_ATOMS = TILED_SF ? (BN + 127) / 128 : ((BN % 128 == 0) ? BN / 128 : BN / 128 + 1);
     static constexpr bool SCALED = MODE != MODE_FP8;
     // 128-channel scale blocks per stage and operand row block: a stage is 128 bytes per row = 256 FP4 or 128 FP8 channels
-    static constexpr int KA = (MODE == MODE_OSC) ? 2 : 1;
+    // (NVFP4 scale blocks cover 64 channels: four per stage)
+    static constexpr int KA = (MODE == MODE_OSC) ? 2 : (MODE == MODE_NVF4) ? 4 : 1;
+    static constexpr bool DUAL = MODE == MODE_OSC || MODE == MODE_NVF4;   // has the BF16 branch (Path B)
+    static constexpr int SF_K = (MODE == MODE_NVF4) ? 64 : 128;           // channels per scale block
     static constexpr int SF_COLS = SCALED ? KA * (4 + SFB_ATOMS * 4) : 0;  // TMEM columns of one stage's scales
     static constexpr int ACC_STAGES = (2 * BN + SF_COLS <= TMEM_COLS) ? 2 : 1;
     static constexpr int SF_BUFS = (ACC_STAGES * BN + 2 * SF_COLS <= TMEM_COLS) ? 2 : 1;
@@ -136,7 +140,7 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
         if (C::SCALED) {
             prefetch_tmap(&args.tm_sfa);
             prefetch_tmap(&args.tm_sfw);
-            if (MODE == MODE_OSC && args.Kop > 0) {
+            if (C::DUAL && args.Kop > 0) {
                 prefetch_tmap(&args.tm_ao);
                 prefetch_tmap(&args.tm_bo);
             }
@@ -159,11 +163,11 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
     const int num_m = sched ? sched[0] : (args.M + 2 * BM - 1) / (2 * BM);
     const int num_n = (N + BN - 1) / BN;
     const int total = num_m * num_n;
-    const int elems_per_kb = (MODE == MODE_OSC) ? 256 : 128;  // channels in 128 bytes of an operand row
+    const int elems_per_kb = C::DUAL ? 256 : 128;  // channels in 128 bytes of an operand row
     const int nkb_a = (K + elems_per_kb - 1) / elems_per_kb;
-    const int nkb_b = (MODE == MODE_OSC) ? args.Kop / 64 : 0;
+    const int nkb_b = C::DUAL ? args.Kop / 64 : 0;
     const int nkb = nkb_a + nkb_b;
-    const int katoms_total = K / 128;
+    const int katoms_total = K / C::SF_K;   // scale blocks along K
     const int natoms = (N + 127) / 128;
 
     // tile t -> first row, column, and (grouped) last valid row, first scale row, expert
@@ -250,6 +254,7 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
             uint64_t* fullL = full_bar + L * SPL;
             uint64_t* emptyL = empty_bar + L * SPL;
             constexpr uint32_t IDESC_A = (MODE == MODE_OSC)    ? idesc_mxf4(2 * BM, BN)
+                                         : (MODE == MODE_NVF4) ? idesc_nvf4(2 * BM, BN)
                                          : (MODE == MODE_MXF8) ? idesc_mxf8(2 * BM, BN)
                                                                : idesc_e4m3(2 * BM, BN);
             constexpr uint32_t IDESC_B = idesc_bf16(2 * BM, BN);
@@ -294,7 +299,30 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
                                                   sfb_tm + sfo + (k >> 1) * (C::SFB_ATOMS * 4), (kb | k) ? 1u : 0u);
                                 }
                             }
-                        } else if (MODE == MODE_OSC) {
+                        } else if (MODE == MODE_NVF4 && kb < nkb_a) {
+                            // four 64-channel scale blocks per stage, one per K = 64 instruction (a whole scale column)
+                            const int ka = min(4, katoms_total - 4 * kb);
+                            const uint64_t sfa_d = sf_hi | (uint64_t)((sbase + A_BYTES + C::B_BYTES) >> 4);
+                            const uint64_t sfb_d = sf_hi | (uint64_t)((sbase + A_BYTES + C::B_BYTES + C::SFA_BYTES) >> 4);
+                            const uint32_t sfo = (uint32_t)(C::SF_BUFS == 2 ? (kb & 1) : 0) * C::TM_SF_STRIDE;
+#pragma unroll
+                            for (int a = 0; a < 4; ++a) {
+                                if (a < ka) {
+                                    tc_copy_sf_pair(tmem_base + sfo + C::TM_SFA + a * 4, sfa_d + (uint64_t)(a * 32));
+#pragma unroll
+                                    for (int j = 0; j < C::SFB_ATOMS; ++j)
+                                        tc_copy_sf_pair(tmem_base + sfo + C::TM_SFB + a * (C::SFB_ATOMS * 4) + j * 4,
+                                                        sfb_d + (uint64_t)(j * (C::KA * 32) + a * 32));
+                                }
+                            }
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) {
+                                if (k < ka)
+                                    mma_nvf4_pair(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC_A,
+                                                  tmem_base + sfo + C::TM_SFA + k * 4,
+                                                  sfb_tm + sfo + k * (C::SFB_ATOMS * 4), (kb | k) ? 1u : 0u);
+                            }
+                        } else if (C::DUAL) {
 #pragma unroll
                             for (int k = 0; k < 4; ++k) mma_f16_pair(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC_B, 1u);
                         } else if (MODE == MODE_MXF8) {
@@ -401,6 +429,10 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
                             const int cc = j * 8 + 2 * i;  // column inside the 64-column slice
                             float lo = __uint_as_float(cc < 32 ? r0[cc] : r1[cc - 32]);
                             float hi = __uint_as_float(cc < 32 ? r0[cc + 1] : r1[cc - 31]);
+                            if (MODE == MODE_NVF4) {   // back out of the scaled domain: an exact power of two
+                                lo *= args.out_scale;
+                                hi *= args.out_scale;
+                            }
                             if (MODE == MODE_FP8) {
                                 const float wx = __shfl_sync(0xFFFFFFFFu, wv.x, j * 4 + i);
                                 const float wy = __shfl_sync(0xFFFFFFFFu, wv.y, j * 4 + i);
@@ -581,6 +613,10 @@ cudaError_t launch_gemm_dual_pair(const GemmArgs& a, int bn, cudaStream_t st) {
 cudaError_t launch_gemm_mxf8_pair(const GemmArgs& a, int bn, cudaStream_t st) {
     if (bn == 192) return pair::launch_cfg<pair::MODE_MXF8, 192>(a, st);
     return pair::launch_cfg<pair::MODE_MXF8, 256>(a, st);
+}
+cudaError_t launch_gemm_nvf4_pair(const GemmArgs& a, int bn, cudaStream_t st) {
+    if (bn == 192) return pair::launch_cfg<pair::MODE_NVF4, 192>(a, st);
+    return pair::launch_cfg<pair::MODE_NVF4, 256>(a, st);
 }
 cudaError_t launch_gemm_fp8_pair(const GemmArgs& a, int bn, cudaStream_t st) {
     if (bn == 192) return pair::launch_cfg<pair::MODE_FP8, 192>(a, st);

@@ -73,12 +73,20 @@ __device__ __forceinline__ uint32_t e2m1x8(float f0, float f1, float f2, float f
     return r;
 }
 
+// FMT_MXFP4: groups of 32, E8M0 scale (Algorithm 2 as the paper states it).  FMT_NVFP4: blocks of 16, unsigned
+// E4M3 block scale, tensor-level scale 2^tensor_e (the G = 16 variant): t = fl32(amax' * fl32(1/6)),
+// scale byte = E4M3(t), elements = E2M1(fl32(x' * fl32(1/scale))) with x' = x * 2^-tensor_e, backed-up
+// channels stored as bf16(x').
+constexpr int FMT_MXFP4 = 0;
+constexpr int FMT_NVFP4 = 1;
+
+template <int FMT>
 __global__ void __launch_bounds__(QE_THREADS, QE_CTAS_PER_SM)
 quant_extract_kernel(const __grid_constant__ CUtensorMap tm_x, int M, int K,
                      const uint32_t* __restrict__ mask, const int32_t* __restrict__ prefix,
                      const int32_t* __restrict__ idx_o,
                      uint8_t* __restrict__ xq, uint8_t* __restrict__ sf, uint16_t* __restrict__ xo,
-                     int Ko, int Kop, const int32_t* __restrict__ sched, int max_tiles) {
+                     int Ko, int Kop, const int32_t* __restrict__ sched, int max_tiles, int tensor_e) {
     extern __shared__ uint8_t qe_smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(qe_smem_raw) + 1023) & ~uintptr_t(1023));
     uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + QE_STAGES * QE_TILE_BYTES);
@@ -174,7 +182,13 @@ quant_extract_kernel(const __grid_constant__ CUtensorMap tm_x, int M, int K,
                 const int within = (((gi & 1) << 5) + j) * 2;   // byte inside the 128-byte half row
                 uint16_t* e = reinterpret_cast<uint16_t*>(const_cast<uint8_t*>(rowp) +
                                                           ((((within >> 4) ^ (grow & 7))) << 4) + (within & 15));
-                if (r < row_end) xo[(int64_t)r * Kop + slot] = *e;
+                if (r < row_end) {
+                    uint16_t b = *e;
+                    if (FMT == FMT_NVFP4)   // into the scaled domain of the block-scaled path (exact for normal results)
+                        b = __bfloat16_as_ushort(__float2bfloat16_rn(
+                            __uint_as_float((uint32_t)b << 16) * __uint_as_float((uint32_t)(127 - tensor_e) << 23)));
+                    xo[(int64_t)r * Kop + slot] = b;
+                }
                 ++slot;
                 *e = 0;
             }
@@ -193,6 +207,7 @@ quant_extract_kernel(const __grid_constant__ CUtensorMap tm_x, int M, int K,
             if (lane == 0) mbar_arrive(&empty_bar[s]);
             if (++s == QE_STAGES) { s = 0; ph ^= 1u; }
 
+            if (FMT == FMT_MXFP4) {
             int code = 0;
             if (r < row_end) {  // rows past the end (next expert / padding) count as zeros: code 0, nothing stored
                 // amax on the bf16 magnitudes, two at a time
@@ -232,6 +247,51 @@ quant_extract_kernel(const __grid_constant__ CUtensorMap tm_x, int M, int K,
             if (gi == 0) {
                 const int64_t blk = (int64_t)(sf_row0 / 128) * (K / 128) + cb;
                 *reinterpret_cast<uint32_t*>(sf + blk * 512 + (grow & 31) * 16 + (grow >> 5) * 4) = word;
+            }
+            } else {
+            // NVFP4: my 32 channels are two blocks of 16
+            uint32_t codes = 0;
+            if (r < row_end) {
+                const float p2 = __uint_as_float((uint32_t)(127 - tensor_e) << 23);   // 2^-tensor_e
+                uint32_t q[4];
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    __nv_bfloat162 m2 = __habs2(as_bf162(w[8 * h]));
+#pragma unroll
+                    for (int i = 1; i < 8; ++i) m2 = __hmax2(m2, __habs2(as_bf162(w[8 * h + i])));
+                    const uint32_t am2 = bf162_bits(m2);
+                    const float amax = __uint_as_float(max(am2 & 0xFFFFu, am2 >> 16) << 16) * p2;   // exact
+                    const float t = __fmul_rn(amax, __fdiv_rn(1.0f, 6.0f));
+                    const uint32_t sb = e4m3x2(t, 0.0f) & 0xFFu;          // nearest-even, saturating at 448
+                    codes |= sb << (8 * h);
+                    // value of the scale byte: exponent field e, mantissa m -> (8 + m) * 2^(e - 10), or m * 2^-9
+                    const int se = (int)(sb >> 3), sm = (int)(sb & 7u);
+                    const float sbv = se ? __uint_as_float((uint32_t)(se + 120) << 23) * (1.0f + 0.125f * (float)sm)
+                                         : 0.001953125f * (float)sm;
+                    // one factor per block: fl32(1/scale) times the (exact) power of two of the tensor scale
+                    const float fac = sbv > 0.0f ? __fdiv_rn(1.0f, sbv) * p2 : 0.0f;
+#pragma unroll
+                    for (int i = 0; i < 2; ++i) {
+                        float f[8];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const uint32_t u = w[8 * h + 4 * i + j];
+                            f[2 * j] = __fmul_rn(__uint_as_float(u << 16), fac);
+                            f[2 * j + 1] = __fmul_rn(__uint_as_float(u & 0xFFFF0000u), fac);
+                        }
+                        q[2 * h + i] = e2m1x8(f[0], f[1], f[2], f[3], f[4], f[5], f[6], f[7]);
+                    }
+                }
+                *reinterpret_cast<uint4*>(xq + (int64_t)r * (K / 2) + cb * (QE_COLS / 2) + gi * 16) =
+                    make_uint4(q[0], q[1], q[2], q[3]);
+            }
+            // scale blocks cover 64 channels: lanes gi = 0,1 hold the four bytes of one word, gi = 2,3 of the next
+            uint32_t word = codes << (16 * (gi & 1));
+            word |= __shfl_xor_sync(0xFFFFFFFFu, word, 1);
+            if ((gi & 1) == 0) {
+                const int64_t blk = (int64_t)(sf_row0 / 128) * (K / 64) + cb * 2 + (gi >> 1);
+                *reinterpret_cast<uint32_t*>(sf + blk * 512 + (grow & 31) * 16 + (grow >> 5) * 4) = word;
+            }
             }
 
             // zero the pad columns of xo once per row tile
@@ -612,21 +672,37 @@ cudaError_t launch_retile_sf(const uint8_t* src, uint8_t* dst, int N, int K, int
 }
 
 // ------------------------------------------------------------------ launchers
-cudaError_t launch_quant_extract(const CUtensorMap& tm_x, int M, int K, const uint32_t* mask,
-                                 const int32_t* prefix, const int32_t* idx_o, void* xq, void* sf, void* xo, int Ko, int Kop,
-                                 const int32_t* sched, int max_tiles, int num_sms, cudaStream_t st) {
+template <int FMT>
+static cudaError_t launch_quant_extract_fmt(const CUtensorMap& tm_x, int M, int K, const uint32_t* mask,
+                                            const int32_t* prefix, const int32_t* idx_o, void* xq, void* sf, void* xo,
+                                            int Ko, int Kop, const int32_t* sched, int max_tiles, int num_sms,
+                                            int tensor_e, cudaStream_t st) {
     const int tiles = (sched ? max_tiles : (M + QE_ROWS - 1) / QE_ROWS) * (K / QE_COLS);
     if (tiles <= 0) return cudaSuccess;
     static bool configured = false;
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(quant_extract_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, QE_SMEM);
+        cudaError_t e = cudaFuncSetAttribute(quant_extract_kernel<FMT>, cudaFuncAttributeMaxDynamicSharedMemorySize, QE_SMEM);
         if (e != cudaSuccess) return e;
         configured = true;
     }
     const int grid = tiles < QE_CTAS_PER_SM * num_sms ? tiles : QE_CTAS_PER_SM * num_sms;
-    return launch_pdl(quant_extract_kernel, dim3(grid), dim3(QE_THREADS), QE_SMEM, st, tm_x, M, K, mask, prefix, idx_o,
-                      static_cast<uint8_t*>(xq), static_cast<uint8_t*>(sf), static_cast<uint16_t*>(xo), Ko, Kop, sched,
-                      max_tiles);
+    return launch_pdl(quant_extract_kernel<FMT>, dim3(grid), dim3(QE_THREADS), QE_SMEM, st, tm_x, M, K, mask, prefix,
+                      idx_o, static_cast<uint8_t*>(xq), static_cast<uint8_t*>(sf), static_cast<uint16_t*>(xo), Ko, Kop,
+                      sched, max_tiles, tensor_e);
+}
+
+cudaError_t launch_quant_extract(const CUtensorMap& tm_x, int M, int K, const uint32_t* mask,
+                                 const int32_t* prefix, const int32_t* idx_o, void* xq, void* sf, void* xo, int Ko, int Kop,
+                                 const int32_t* sched, int max_tiles, int num_sms, cudaStream_t st) {
+    return launch_quant_extract_fmt<FMT_MXFP4>(tm_x, M, K, mask, prefix, idx_o, xq, sf, xo, Ko, Kop, sched, max_tiles,
+                                               num_sms, 0, st);
+}
+// NVFP4 / G = 16 form (dense only): tensor-level scale 2^tensor_e
+cudaError_t launch_quant_extract_nvfp4(const CUtensorMap& tm_x, int M, int K, const uint32_t* mask,
+                                       const int32_t* prefix, const int32_t* idx_o, void* xq, void* sf, void* xo, int Ko,
+                                       int Kop, int num_sms, int tensor_e, cudaStream_t st) {
+    return launch_quant_extract_fmt<FMT_NVFP4>(tm_x, M, K, mask, prefix, idx_o, xq, sf, xo, Ko, Kop, nullptr, 0, num_sms,
+                                               tensor_e, st);
 }
 
 cudaError_t launch_fp8_quant(const void* X, int64_t ldx, int M, int K, void* x8, void* sx, cudaStream_t st) {

@@ -1,0 +1,106 @@
+"""GPU parity of the NVFP4 / G = 16 variant against the oracle: packed codes, E4M3 scale bytes and backed-up
+channels bit for bit (activations and weights), outputs within the stated tolerance."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2604_12782_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+from gpu_util import assert_within_tolerance, dev_bf16, host_f64, host_u8, poison  # noqa: E402
+
+
+@pytest.fixture(scope="module")
+def B():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2604_12782_b200 import binding
+    return binding
+
+
+def sf16_valid(rows, K):
+    r = np.arange(rows)[:, None]
+    b = np.arange(K // 16)[None, :]
+    return (((r // 128) * (K // 64) + b // 4) * 512 + (r % 32) * 16 + ((r % 128) // 32) * 4 + (b % 4)).ravel()
+
+
+def check_quantized(q, xq, sf, xo, rows, K):
+    assert np.array_equal(xq.reshape(rows, K // 2), q["xq"])
+    v = sf16_valid(rows, K)
+    assert np.array_equal(sf[:q["sf"].size][v], q["sf"][v])
+    if q["K_o_pad"]:
+        assert np.array_equal(xo.view(np.uint16).reshape(rows, q["K_o_pad"]), q["xo"])
+
+
+def run_case(B, oracle, Xb, Wb, lut16, what):
+    M, K = Xb.shape
+    N = Wb.shape[0]
+    ex, ew = synth.nvfp4_tensor_exponent(Xb), synth.nvfp4_tensor_exponent(Wb)
+    w = B.osc_nvfp4_prepare_weights(dev_bf16(Wb), lut16, ew)
+    sz = B.osc_nvfp4_act_sizes(w, M)
+    ws = poison(sz.workspace_bytes)
+    Y = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+    B.osc_nvfp4_linear(w, dev_bf16(Xb), ex, Y, ws)
+    B.osc_sync_check()
+    Yref, T, act, wts = oracle.nvfp4_linear(Xb, Wb, lut16, ex, ew)
+    h = host_u8(ws)
+    check_quantized(act, h[sz.xq_offset:sz.xq_offset + sz.xq_bytes], h[sz.sfa_offset:sz.sfa_offset + sz.sfa_bytes],
+                    h[sz.xo_offset:sz.xo_offset + sz.xo_bytes], M, K)
+    check_quantized(wts, host_u8(w.keep["wq"])[:w.sizes.wq_bytes], host_u8(w.keep["sfw"])[:w.sizes.sfw_bytes],
+                    host_u8(w.keep["wo"])[:w.sizes.wo_bytes], N, K)
+    assert_within_tolerance(host_f64(Y), Yref, T, what)
+    return w, sz, ws, Y, ex
+
+
+@pytest.mark.parametrize("M,K,N,kind", [(1, 128, 64, "one"), (64, 512, 512, "one"), (127, 384, 192, "two"),
+                                        (129, 256, 320, "empty"), (300, 640, 448, "one"), (515, 128, 64, "two")])
+def test_nvfp4_linear_small(B, oracle, M, K, N, kind):
+    c = synth.osc16_linear_case(M + K, M, K, N)
+    rng = np.random.default_rng(N)
+    lut16 = {"one": c["lut16"], "empty": np.full((K // 16, 1), -1, np.int8),
+             "two": np.stack([rng.permutation(16)[:2] for _ in range(K // 16)]).astype(np.int8)}[kind]
+    w, sz, ws, Y, ex = run_case(B, oracle, c["X"], c["W"], lut16, f"nvfp4 {M}x{K}x{N} {kind}")
+    Y2 = torch.full((M, N + 8), float("nan"), dtype=torch.bfloat16, device="cuda")
+    B.osc_nvfp4_gemm(w, ws[sz.xq_offset:], ws[sz.sfa_offset:], ws[sz.xo_offset:], M, ex, Y2)
+    B.osc_sync_check()
+    assert torch.equal(Y2[:, :N], Y) and torch.isnan(Y2[:, N:].float()).all()
+    with pytest.raises(B.OscError):
+        B.osc_linear(w, dev_bf16(c["X"]), Y, ws)      # an NVFP4 handle is refused by the MXFP4 entry points
+
+
+def test_nvfp4_edge_values(B, oracle):
+    rng = np.random.default_rng(41)
+    M, K = 40, 256
+    X = rng.standard_t(3, size=(M, K)).astype(np.float32)
+    X[2, 16:32] = 0.0                      # all-zero block: scale byte 0, sign-only codes
+    X[3, ::3] *= -1.0
+    X[4] *= 0.001                          # tiny blocks: subnormal E4M3 scales
+    X[5, 0:16] = [6.0, -3.0, 1.25, 0.75, 0.25, -0.0, 2.5, 3.5, 5.0] + [0.5] * 7
+    Xb = synth.f32_to_bf16_bits(X)
+    W = synth.f32_to_bf16_bits((0.02 * rng.standard_normal((64, K))).astype(np.float32))
+    run_case(B, oracle, Xb, W, np.full((K // 16, 1), 3, np.int8), "nvfp4 edge")
+
+
+def test_nvfp4_qkv_shape(B, oracle):
+    M, K, N = 1024, 4096, 6144
+    c = synth.osc16_linear_case(0, M, K, N)
+    ex, ew = synth.nvfp4_tensor_exponent(c["X"]), synth.nvfp4_tensor_exponent(c["W"])
+    w = B.osc_nvfp4_prepare_weights(dev_bf16(c["W"]), c["lut16"], ew)
+    sz = B.osc_nvfp4_act_sizes(w, M)
+    ws = poison(sz.workspace_bytes)
+    Y = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+    B.osc_nvfp4_linear(w, dev_bf16(c["X"]), ex, Y, ws)
+    B.osc_sync_check()
+    act = oracle.nvfp4_quantize_extract(c["X"], c["lut16"], ex)
+    wts = oracle.nvfp4_quantize_extract(c["W"], c["lut16"], ew)
+    h = host_u8(ws)
+    check_quantized(act, h[sz.xq_offset:sz.xq_offset + sz.xq_bytes], h[sz.sfa_offset:sz.sfa_offset + sz.sfa_bytes],
+                    h[sz.xo_offset:sz.xo_offset + sz.xo_bytes], M, K)
+    check_quantized(wts, host_u8(w.keep["wq"])[:w.sizes.wq_bytes], host_u8(w.keep["sfw"])[:w.sizes.sfw_bytes],
+                    host_u8(w.keep["wo"])[:w.sizes.wo_bytes], N, K)
+    rows = np.array(sorted({0, 1, 127, 128, 255, 256, 257, M - 257, M - 1}
+                           | set(int(r) for r in np.random.default_rng(0).integers(0, M, size=12))), np.int32)
+    Yref, T = oracle.nvfp4_gemm(act, wts, rows)
+    assert_within_tolerance(host_f64(Y[torch.from_numpy(rows.astype(np.int64)).cuda()]), Yref, T, "nvfp4 qkv")
+    assert not torch.isnan(Y.float()).any()
