@@ -638,7 +638,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="osc", choices=["osc", "reference"])
     ap.add_argument("--no-cpu", action="store_true", help="skip the cpu_baseline leg")
-    ap.add_argument("--cpu-rows", type=int, default=1024, help="activation rows of the cpu_baseline sample")
+    ap.add_argument("--cpu-rows", type=int, default=8192, help="activation rows of the cpu_baseline sample")
     ap.add_argument("--ref-rows", type=int, default=128, help="activation rows per step of --impl reference")
     ap.add_argument("--sweep", action="store_true")
     ap.add_argument("--sweep-only", default="", help="with --sweep: only the rows whose name contains this text")
