@@ -312,3 +312,37 @@ def test_error_ordering_on_device(B, oracle):
         return np.linalg.norm(host_f64(Y) - exact) / np.linalg.norm(exact)
 
     assert run(c["lut"]) < 0.3 * run(np.full((16, 1), -1, np.int8))
+
+
+def test_calls_can_be_captured_in_a_cuda_graph(B, oracle):
+    """The calls allocate nothing and never synchronise, so a sequence of them can be captured once and replayed:
+    the replay must give the bytes of a plain launch, for the dual-path, the few-row and the FP8 paths."""
+    outs = {}
+    for M in (24, 300):
+        X_bits, W_bits, lut = make_case("rand1", M, 320, 512, 5)
+        w = B.osc_prepare_weights(dev_bf16(W_bits), lut)
+        w8 = B.osc_fp8_prepare_weights(dev_bf16(W_bits))
+        sz, sz8 = B.osc_act_sizes(w, M), B.osc_fp8_act_sizes(w8, M)
+        ws, ws8 = poison(sz.workspace_bytes), poison(sz8.workspace_bytes)
+        X = dev_bf16(X_bits)
+        Y = torch.zeros((M, 320), dtype=torch.bfloat16, device="cuda")
+        Y8 = torch.zeros((M, 320), dtype=torch.bfloat16, device="cuda")
+        B.osc_linear(w, X, Y, ws)
+        B.osc_fp8_linear(w8, X, Y8, ws8)
+        B.osc_sync_check()
+        want, want8 = Y.clone(), Y8.clone()
+        st = torch.cuda.Stream()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(st):
+            with torch.cuda.graph(g, stream=st):
+                B.osc_linear(w, X, Y, ws, stream=st)
+                B.osc_fp8_linear(w8, X, Y8, ws8, stream=st)
+        for _ in range(2):
+            Y.zero_()
+            Y8.zero_()
+            g.replay()
+            torch.cuda.synchronize()
+            assert torch.equal(Y, want) and torch.equal(Y8, want8)
+        B.osc_sync_check()
+        outs[M] = want
+    assert outs[24].shape[0] == 24
