@@ -646,6 +646,17 @@ def run_sweep(args):
     rows.append({"name": "moe.down_fp8(grouped)", "M": Mt, "K": K, "N": N, "ms": ms,
                  "tflops": roofline.fp8_flops(Mt, N, K) / ms / 1e9, "pct_roofline": 100 * troof / (ms * 1e-3),
                  "roof_us": troof * 1e6})
+    del w, ws
+    w = B.osc_mxfp8_prepare_weights_grouped(Wd)
+    sz = B.osc_mxfp8_act_sizes(w, c["M"])
+    ws = torch.empty(sz.workspace_bytes, dtype=torch.uint8, device="cuda")
+    ms = time_loop(torch, lambda i: B.osc_mxfp8_linear_grouped(w, Xd, off, Y, ws), steps, warm)
+    B.osc_sync_check()
+    byts = 2.0 * Mt * K + E * N * K * (1 + 1 / 32) + 2.0 * Mt * N
+    troof = max(roofline.fp8_flops(Mt, N, K) / peaks["fp8"], byts / peaks["hbm"])
+    rows.append({"name": "moe.down_mxfp8(grouped)", "M": Mt, "K": K, "N": N, "ms": ms,
+                 "tflops": roofline.fp8_flops(Mt, N, K) / ms / 1e9, "pct_roofline": 100 * troof / (ms * 1e-3),
+                 "roof_us": troof * 1e6})
 
     os.makedirs(os.path.join(ROOT, "gpurun_out"), exist_ok=True)
     with open(os.path.join(ROOT, "gpurun_out", "sweep.json"), "w") as f:

@@ -219,30 +219,36 @@ osc_status osc_fp8_linear_grouped(const osc_fp8_weights* w, const void* X_perm, 
  * even, saturating at 448), for activations (online) and weights (offline) alike, no channel extracted.
  * Scales use the same 128 x 4 block layout as the MXFP4 scales (see osc_quantize_extract):
  * ceil(rows/128) * (K/128) * 512 bytes; bytes of rows past the end are written as 0.
- * Dense problems only (no grouped variant).  Same conventions as the other calls: device pointers,
+ * Dense and grouped (MoE) problems; the grouped calls follow osc_fp8_linear_grouped (rows sorted by expert,
+ * device-resident offsets, every expert's activation scales starting on a 128-row scale block, weights stacked
+ * [E, N, K] with per-expert scale blocks).  Same conventions as the other calls: device pointers,
  * 16-byte alignment, leading dimensions in elements and multiples of 8, asynchronous on `stream`,
  * no allocation, M == 0 is a successful no-op, K % 128 == 0, N % 64 == 0. */
 typedef struct osc_mxfp8_weights osc_mxfp8_weights;
 
 typedef struct {
-    size_t w8_bytes;        /* N * K */
-    size_t sfw_bytes;       /* ceil(N/128) * (K/128) * 512 */
+    size_t w8_bytes;        /* E * N * K */
+    size_t sfw_bytes;       /* E * ceil(N/128) * (K/128) * 512 */
 } osc_mxfp8_weight_sizes_t;
 
 typedef struct {
     size_t x8_bytes;        /* M * K */
-    size_t sfa_bytes;       /* ceil(M/128) * (K/128) * 512 */
-    size_t x8_offset;       /* placement inside the workspace of osc_mxfp8_linear */
+    size_t sfa_bytes;       /* ceil(M/128) * (K/128) * 512; grouped: (M/128 + E) row blocks */
+    size_t sched_bytes;     /* grouped only */
+    size_t x8_offset;       /* placement inside the workspace of osc_mxfp8_linear[_grouped] */
     size_t sfa_offset;
+    size_t sched_offset;
     size_t workspace_bytes;
 } osc_mxfp8_act_sizes_t;
 
-osc_status osc_mxfp8_weight_sizes(int N, int K, osc_mxfp8_weight_sizes_t* out);
+osc_status osc_mxfp8_weight_sizes(int E, int N, int K, osc_mxfp8_weight_sizes_t* out);
 
 /* Offline: w8 [N,K] E4M3 bytes and sfw (block layout) from W (dev bf16 [N, ldw]).  The handle borrows
  * w8 and sfw, which must outlive it; the caller owns every buffer. */
 osc_status osc_mxfp8_prepare_weights(const void* W, int N, int K, int64_t ldw, void* w8, void* sfw, void* stream,
                                      osc_mxfp8_weights** out);
+osc_status osc_mxfp8_prepare_weights_grouped(const void* W, int E, int N, int K, void* w8, void* sfw, void* stream,
+                                             osc_mxfp8_weights** out);
 osc_status osc_mxfp8_weights_destroy(osc_mxfp8_weights* w);
 osc_status osc_mxfp8_act_sizes(const osc_mxfp8_weights* w, int M, osc_mxfp8_act_sizes_t* out);
 
@@ -257,6 +263,9 @@ osc_status osc_mxfp8_gemm(const osc_mxfp8_weights* w, const void* x8, const void
 /* quantize + gemm through a caller-provided workspace of at least osc_mxfp8_act_sizes().workspace_bytes. */
 osc_status osc_mxfp8_linear(const osc_mxfp8_weights* w, const void* X, int M, int64_t ldx, void* Y, int64_t ldy,
                             void* workspace, size_t workspace_bytes, void* stream);
+osc_status osc_mxfp8_linear_grouped(const osc_mxfp8_weights* w, const void* X_perm, const int32_t* off, int M_total,
+                                    int64_t ldx, void* Y, int64_t ldy, void* workspace, size_t workspace_bytes,
+                                    void* stream);
 
 /* ------------------- dynamic-protection control group (Section 4.2), a baseline */
 

@@ -245,6 +245,20 @@ def mxfp8_gemm(x8, sfa, w8, sfw, rows=None):
     return Y, T
 
 
+def mxfp8_quantize_grouped(X: np.ndarray, off: np.ndarray):
+    """Rows sorted by expert: every expert is quantized on its own and its scale blocks (whole 128-row blocks,
+    rows numbered from 0 inside the expert) are laid end to end, so expert e starts at scale row
+    sum_{e'<e} roundup(m_e', 128).  -> (x8 [M,K], sf, per-expert (x8, sf) list)."""
+    X = np.ascontiguousarray(X, dtype=np.uint16)
+    parts, sfs = [], []
+    for e in range(off.size - 1):
+        x8e, sfe = mxfp8_quantize(X[int(off[e]):int(off[e + 1])])
+        parts.append((x8e, sfe))
+        sfs.append(sfe)
+    x8 = np.concatenate([p[0] for p in parts], axis=0) if parts else np.zeros((0, X.shape[1]), np.uint8)
+    return x8, (np.concatenate(sfs) if sfs else np.zeros(0, np.uint8)), parts
+
+
 def mxfp8_linear(X: np.ndarray, W: np.ndarray, rows=None):
     x8, sfa = mxfp8_quantize(X)
     w8, sfw = mxfp8_quantize(W)

@@ -57,7 +57,8 @@ class Mxfp8WeightSizes(C.Structure):
 
 
 class Mxfp8ActSizes(C.Structure):
-    _fields_ = [(n, C.c_size_t) for n in ("x8_bytes", "sfa_bytes", "x8_offset", "sfa_offset", "workspace_bytes")]
+    _fields_ = [(n, C.c_size_t) for n in ("x8_bytes", "sfa_bytes", "sched_bytes", "x8_offset", "sfa_offset",
+                                          "sched_offset", "workspace_bytes")]
 
 
 _vp, _i, _i64, _sz = C.c_void_p, C.c_int, C.c_int64, C.c_size_t
@@ -96,7 +97,9 @@ _SIGS = {
     "osc_nvfp4_quantize_extract": (_i, [_vp, _vp, _i, _i64, _i, _vp, _vp, _vp, _vp]),
     "osc_nvfp4_gemm": (_i, [_vp, _vp, _vp, _vp, _i, _i, _vp, _i64, _vp]),
     "osc_nvfp4_linear": (_i, [_vp, _vp, _i, _i64, _i, _vp, _i64, _vp, _sz, _vp]),
-    "osc_mxfp8_weight_sizes": (_i, [_i, _i, C.POINTER(Mxfp8WeightSizes)]),
+    "osc_mxfp8_weight_sizes": (_i, [_i, _i, _i, C.POINTER(Mxfp8WeightSizes)]),
+    "osc_mxfp8_prepare_weights_grouped": (_i, [_vp, _i, _i, _i, _vp, _vp, _vp, C.POINTER(_vp)]),
+    "osc_mxfp8_linear_grouped": (_i, [_vp, _vp, _vp, _i, _i64, _vp, _i64, _vp, _sz, _vp]),
     "osc_mxfp8_prepare_weights": (_i, [_vp, _i, _i, _i64, _vp, _vp, _vp, C.POINTER(_vp)]),
     "osc_mxfp8_weights_destroy": (_i, [_vp]),
     "osc_mxfp8_act_sizes": (_i, [_vp, _i, C.POINTER(Mxfp8ActSizes)]),
@@ -341,22 +344,43 @@ def osc_fp8_linear_grouped(w: Fp8Weights, X: torch.Tensor, off: torch.Tensor, Y:
 
 # ------------------------------------------------------------- MXFP8 form of the fallback
 
-def osc_mxfp8_weight_sizes(N: int, K: int) -> Mxfp8WeightSizes:
+def osc_mxfp8_weight_sizes(E: int, N: int, K: int) -> Mxfp8WeightSizes:
     out = Mxfp8WeightSizes()
-    _check(_lib.osc_mxfp8_weight_sizes(N, K, C.byref(out)))
+    _check(_lib.osc_mxfp8_weight_sizes(E, N, K, C.byref(out)))
     return out
 
 
 def osc_mxfp8_prepare_weights(W: torch.Tensor, stream=None) -> Mxfp8Weights:
     N, K = W.shape
-    sz = osc_mxfp8_weight_sizes(N, K)
+    sz = osc_mxfp8_weight_sizes(1, N, K)
     bufs = {"w8": _alloc(sz.w8_bytes, W.device), "sfw": _alloc(sz.sfw_bytes, W.device)}
     h = _vp()
     _check(_lib.osc_mxfp8_prepare_weights(_ptr(W), N, K, W.stride(0), _ptr(bufs["w8"]), _ptr(bufs["sfw"]),
                                           _stream(stream), C.byref(h)))
     w = Mxfp8Weights(h.value, bufs)
-    w.N, w.K, w.sizes = N, K, sz
+    w.E, w.N, w.K, w.sizes = 1, N, K, sz
     return w
+
+
+def osc_mxfp8_prepare_weights_grouped(W: torch.Tensor, stream=None) -> Mxfp8Weights:
+    E, N, K = W.shape
+    assert W.is_contiguous()
+    sz = osc_mxfp8_weight_sizes(E, N, K)
+    bufs = {"w8": _alloc(sz.w8_bytes, W.device), "sfw": _alloc(sz.sfw_bytes, W.device)}
+    h = _vp()
+    _check(_lib.osc_mxfp8_prepare_weights_grouped(_ptr(W), E, N, K, _ptr(bufs["w8"]), _ptr(bufs["sfw"]),
+                                                  _stream(stream), C.byref(h)))
+    w = Mxfp8Weights(h.value, bufs)
+    w.E, w.N, w.K, w.sizes = E, N, K, sz
+    return w
+
+
+def osc_mxfp8_linear_grouped(w: Mxfp8Weights, X: torch.Tensor, off: torch.Tensor, Y: torch.Tensor,
+                             workspace: torch.Tensor, stream=None):
+    M = X.shape[0]
+    _check(_lib.osc_mxfp8_linear_grouped(w.ptr, _ptr(X), _ptr(off), M, X.stride(0) if M else w.K, _ptr(Y),
+                                         Y.stride(0) if M else w.N, _ptr(workspace),
+                                         workspace.numel() * workspace.element_size(), _stream(stream)))
 
 
 def osc_mxfp8_weights_destroy(w: Mxfp8Weights):

@@ -215,7 +215,8 @@ struct osc_fp8_weights {
 };
 
 struct osc_mxfp8_weights {
-    int N, K;
+    int E, N, K;
+    bool grouped;
     const uint8_t *w8, *sfw;
     int num_sms;
     CUtensorMap tm_b2[2];  // half tiles for 192- and 256-wide tiles
@@ -739,15 +740,16 @@ osc_status osc_fp8_linear_grouped(const osc_fp8_weights* w, const void* X_perm, 
 
 // ------------------------------------------------- MXFP8 form of the fallback
 
-osc_status osc_mxfp8_weight_sizes(int N, int K, osc_mxfp8_weight_sizes_t* out) {
+osc_status osc_mxfp8_weight_sizes(int E, int N, int K, osc_mxfp8_weight_sizes_t* out) {
     if (!out) return fail(OSC_ERR_INVALID_ARG, "out is null");
-    if (osc_status s = check_nk(1, N, K)) return s;
-    out->w8_bytes = (size_t)N * K;
-    out->sfw_bytes = sf_bytes(N, K);
+    if (osc_status s = check_nk(E, N, K)) return s;
+    out->w8_bytes = (size_t)E * N * K;
+    out->sfw_bytes = (size_t)E * sf_bytes(N, K);
     return OSC_OK;
 }
 
-osc_status osc_mxfp8_quantize(const void* X, int M, int K, int64_t ldx, void* x8, void* sfa, void* stream) {
+static osc_status mxfp8_quantize_impl(const void* X, int M, int K, int64_t ldx, void* x8, void* sfa,
+                                      const int32_t* sched, int max_tiles, void* stream) {
     if (M < 0) return fail(OSC_ERR_INVALID_ARG, "M = %d is negative", M);
     if (K <= 0 || K % 128) return fail(OSC_ERR_SHAPE, "K = %d must be a positive multiple of 128", K);
     if (M == 0) return OSC_OK;
@@ -755,31 +757,50 @@ osc_status osc_mxfp8_quantize(const void* X, int M, int K, int64_t ldx, void* x8
     if (ldx < K) return fail(OSC_ERR_SHAPE, "ldx = %lld < K", (long long)ldx);
     if (ldx % 8 || !aligned16(X) || !aligned16(x8) || !aligned16(sfa))
         return fail(OSC_ERR_ALIGN, "pointers must be 16-byte aligned and ldx a multiple of 8");
-    cudaError_t e = launch_mxfp8_quant(X, ldx, M, K, x8, sfa, static_cast<cudaStream_t>(stream));
+    cudaError_t e = launch_mxfp8_quant(X, ldx, M, K, x8, sfa, sched, max_tiles, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return cuda_fail(e, "mxfp8_quant_kernel");
     return OSC_OK;
 }
 
-osc_status osc_mxfp8_prepare_weights(const void* W, int N, int K, int64_t ldw, void* w8, void* sfw, void* stream,
-                                     osc_mxfp8_weights** out) {
+osc_status osc_mxfp8_quantize(const void* X, int M, int K, int64_t ldx, void* x8, void* sfa, void* stream) {
+    return mxfp8_quantize_impl(X, M, K, ldx, x8, sfa, nullptr, 0, stream);
+}
+
+static osc_status mxfp8_prepare_impl(const void* W, int E, int N, int K, int64_t ldw, void* w8, void* sfw, void* stream,
+                                     bool grouped, osc_mxfp8_weights** out) {
     if (!out) return fail(OSC_ERR_INVALID_ARG, "out is null");
     *out = nullptr;
-    if (osc_status s = check_nk(1, N, K)) return s;
+    if (osc_status s = check_nk(E, N, K)) return s;
     DeviceInfo di;
     if (osc_status s = device_info(&di)) return s;
-    if (osc_status s = osc_mxfp8_quantize(W, N, K, ldw, w8, sfw, stream)) return s;
+    // expert by expert: every expert's scales start on a 128-row block of their own
+    for (int ex = 0; ex < E; ++ex) {
+        if (osc_status s = mxfp8_quantize_impl(static_cast<const uint16_t*>(W) + (size_t)ex * N * ldw, N, K, ldw,
+                                               static_cast<uint8_t*>(w8) + (size_t)ex * N * K,
+                                               static_cast<uint8_t*>(sfw) + (size_t)ex * sf_bytes(N, K), nullptr, 0, stream))
+            return s;
+    }
     osc_mxfp8_weights* w = new (std::nothrow) osc_mxfp8_weights();
     if (!w) return fail(OSC_ERR_INVALID_ARG, "out of host memory");
-    w->N = N; w->K = K;
+    w->E = E; w->N = N; w->K = K; w->grouped = grouped;
     w->w8 = static_cast<const uint8_t*>(w8);
     w->sfw = static_cast<const uint8_t*>(sfw);
     w->num_sms = di.num_sms;
     osc_status s = OSC_OK;
-    for (int v = 0; v < 2 && s == OSC_OK; ++v) s = make_tmap(&w->tm_b2[v], w8, false, (uint64_t)N, K, K, (v == 0 ? 192 : 256) / 2);
-    if (s == OSC_OK) s = make_tmap_sf(&w->tm_sfw, sfw, (uint64_t)sf_bytes(N, K) / 512, 1);
+    for (int v = 0; v < 2 && s == OSC_OK; ++v)
+        s = make_tmap(&w->tm_b2[v], w8, false, (uint64_t)E * N, K, K, (v == 0 ? 192 : 256) / 2);
+    if (s == OSC_OK) s = make_tmap_sf(&w->tm_sfw, sfw, (uint64_t)E * sf_bytes(N, K) / 512, 1);
     if (s != OSC_OK) { delete w; return s; }
     *out = w;
     return OSC_OK;
+}
+osc_status osc_mxfp8_prepare_weights(const void* W, int N, int K, int64_t ldw, void* w8, void* sfw, void* stream,
+                                     osc_mxfp8_weights** out) {
+    return mxfp8_prepare_impl(W, 1, N, K, ldw, w8, sfw, stream, false, out);
+}
+osc_status osc_mxfp8_prepare_weights_grouped(const void* W, int E, int N, int K, void* w8, void* sfw, void* stream,
+                                             osc_mxfp8_weights** out) {
+    return mxfp8_prepare_impl(W, E, N, K, K, w8, sfw, stream, true, out);
 }
 osc_status osc_mxfp8_weights_destroy(osc_mxfp8_weights* w) {
     delete w;
@@ -789,18 +810,19 @@ osc_status osc_mxfp8_weights_destroy(osc_mxfp8_weights* w) {
 osc_status osc_mxfp8_act_sizes(const osc_mxfp8_weights* w, int M, osc_mxfp8_act_sizes_t* out) {
     if (!w || !out) return fail(OSC_ERR_INVALID_ARG, "null argument");
     if (M < 0) return fail(OSC_ERR_INVALID_ARG, "M = %d is negative", M);
+    const int64_t max_tiles = w->grouped ? (int64_t)M / 128 + w->E : ((int64_t)M + 127) / 128;
     out->x8_bytes = (size_t)M * w->K;
-    out->sfa_bytes = sf_bytes(M, w->K);
+    out->sfa_bytes = (size_t)max_tiles * (w->K / 128) * 512;
+    out->sched_bytes = w->grouped ? sched_ints(max_tiles) * 4 + sched_ints(max_tiles256(M, w->E)) * 4 : 0;
     out->x8_offset = 0;
     out->sfa_offset = align256(out->x8_bytes);
-    out->workspace_bytes = out->sfa_offset + align256(out->sfa_bytes);
+    out->sched_offset = out->sfa_offset + align256(out->sfa_bytes);
+    out->workspace_bytes = out->sched_offset + align256(out->sched_bytes);
     return OSC_OK;
 }
 
-osc_status osc_mxfp8_gemm(const osc_mxfp8_weights* w, const void* x8, const void* sfa, int M, void* Y, int64_t ldy,
-                          void* stream) {
-    if (!w) return fail(OSC_ERR_INVALID_ARG, "weights handle is null");
-    if (M < 0) return fail(OSC_ERR_INVALID_ARG, "M = %d is negative", M);
+static osc_status mxfp8_gemm_impl(const osc_mxfp8_weights* w, const void* x8, const void* sfa, int M, void* Y,
+                                  int64_t ldy, const int32_t* sched2, int max_tiles, int max_tiles2, void* stream) {
     if (M == 0) return OSC_OK;
     if (!x8 || !sfa || !Y) return fail(OSC_ERR_INVALID_ARG, "null device pointer");
     if (ldy < w->N) return fail(OSC_ERR_SHAPE, "ldy = %lld < N = %d", (long long)ldy, w->N);
@@ -809,11 +831,14 @@ osc_status osc_mxfp8_gemm(const osc_mxfp8_weights* w, const void* x8, const void
     GemmArgs a;
     memset(&a, 0, sizeof a);
     if (osc_status s = make_tmap(&a.tm_a, x8, false, M, w->K, w->K, 128)) return s;
-    // every M runs on the CTA-pair kernel (256-row tiles); rows past M are zero-filled by the loads and never stored
-    const int bn = gemm_pair_block_n(false, false, (M + 255) / 256, w->N, w->K / 128, w->num_sms);
+    // every problem runs on the CTA-pair kernel (256-row tiles); rows past the end are zero-filled by the loads or
+    // belong to the next expert, and are never stored
+    const long row_tiles = w->grouped ? max_tiles2 - w->E / 2 : (M + 255) / 256;
+    const int bn = gemm_pair_block_n(false, false, row_tiles, w->N, w->K / 128, w->num_sms);
     a.tm_b = w->tm_b2[bn == 256];
     a.tm_sfw = w->tm_sfw;
-    if (osc_status s = make_tmap_sf(&a.tm_sfa, sfa, (uint64_t)sf_bytes(M, w->K) / 512, 1)) return s;
+    const uint64_t sf_row_blocks = w->grouped ? (uint64_t)max_tiles : (uint64_t)((M + 127) / 128);
+    if (osc_status s = make_tmap_sf(&a.tm_sfa, sfa, sf_row_blocks * (w->K / 128), 1)) return s;
     if (osc_status s = make_tmap(&a.tm_y, Y, true, M, (uint64_t)w->N * 2, (uint64_t)ldy * 2, 32)) return s;
     a.sfa = static_cast<const uint8_t*>(sfa);
     a.sfw = w->sfw;
@@ -821,24 +846,59 @@ osc_status osc_mxfp8_gemm(const osc_mxfp8_weights* w, const void* x8, const void
     a.ldy = ldy;
     a.M = M; a.N = w->N; a.K = w->K; a.Kop = 0;
     a.num_sms = w->num_sms;
+    a.sched2 = sched2; a.max_tiles2 = max_tiles2;
     cudaError_t e = launch_gemm_mxf8_pair(a, bn, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return cuda_fail(e, "gemm_pair_kernel(mxfp8)");
     return OSC_OK;
 }
 
-osc_status osc_mxfp8_linear(const osc_mxfp8_weights* w, const void* X, int M, int64_t ldx, void* Y, int64_t ldy,
-                            void* workspace, size_t workspace_bytes, void* stream) {
+osc_status osc_mxfp8_gemm(const osc_mxfp8_weights* w, const void* x8, const void* sfa, int M, void* Y, int64_t ldy,
+                          void* stream) {
+    if (!w) return fail(OSC_ERR_INVALID_ARG, "weights handle is null");
+    if (M < 0) return fail(OSC_ERR_INVALID_ARG, "M = %d is negative", M);
+    if (w->grouped) return fail(OSC_ERR_INVALID_ARG, "grouped weights: use osc_mxfp8_linear_grouped");
+    return mxfp8_gemm_impl(w, x8, sfa, M, Y, ldy, nullptr, 0, 0, stream);
+}
+
+static osc_status mxfp8_linear_impl(const osc_mxfp8_weights* w, const void* X, const int32_t* off, int M, int64_t ldx,
+                                    void* Y, int64_t ldy, void* workspace, size_t workspace_bytes, void* stream) {
     if (!w) return fail(OSC_ERR_INVALID_ARG, "weights handle is null");
     if (M < 0) return fail(OSC_ERR_INVALID_ARG, "M = %d is negative", M);
     if (M == 0) return OSC_OK;
+    if (w->grouped && !off) return fail(OSC_ERR_INVALID_ARG, "off is null");
     osc_mxfp8_act_sizes_t sz;
     osc_mxfp8_act_sizes(w, M, &sz);
     if (!workspace || !aligned16(workspace)) return fail(OSC_ERR_ALIGN, "workspace must be non-null and 16-byte aligned");
     if (workspace_bytes < sz.workspace_bytes)
         return fail(OSC_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", workspace_bytes, sz.workspace_bytes);
     uint8_t* ws = static_cast<uint8_t*>(workspace);
-    if (osc_status s = osc_mxfp8_quantize(X, M, w->K, ldx, ws + sz.x8_offset, ws + sz.sfa_offset, stream)) return s;
-    return osc_mxfp8_gemm(w, ws + sz.x8_offset, ws + sz.sfa_offset, M, Y, ldy, stream);
+    const int32_t *sched = nullptr, *sched2 = nullptr;
+    int max_tiles = 0, max_tiles2 = 0;
+    if (w->grouped) {
+        max_tiles = M / 128 + w->E;
+        max_tiles2 = max_tiles256(M, w->E);
+        int32_t* s1 = reinterpret_cast<int32_t*>(ws + sz.sched_offset);
+        int32_t* s2 = s1 + sched_ints(max_tiles);
+        cudaError_t e = launch_build_sched(off, w->E, s1, max_tiles, s2, max_tiles2, static_cast<cudaStream_t>(stream));
+        if (e != cudaSuccess) return cuda_fail(e, "build_sched_kernel");
+        sched = s1;
+        sched2 = s2;
+    }
+    if (osc_status s = mxfp8_quantize_impl(X, M, w->K, ldx, ws + sz.x8_offset, ws + sz.sfa_offset, sched, max_tiles, stream))
+        return s;
+    return mxfp8_gemm_impl(w, ws + sz.x8_offset, ws + sz.sfa_offset, M, Y, ldy, sched2, max_tiles, max_tiles2, stream);
+}
+
+osc_status osc_mxfp8_linear(const osc_mxfp8_weights* w, const void* X, int M, int64_t ldx, void* Y, int64_t ldy,
+                            void* workspace, size_t workspace_bytes, void* stream) {
+    if (w && w->grouped) return fail(OSC_ERR_INVALID_ARG, "grouped weights: use osc_mxfp8_linear_grouped");
+    return mxfp8_linear_impl(w, X, nullptr, M, ldx, Y, ldy, workspace, workspace_bytes, stream);
+}
+osc_status osc_mxfp8_linear_grouped(const osc_mxfp8_weights* w, const void* X_perm, const int32_t* off, int M_total,
+                                    int64_t ldx, void* Y, int64_t ldy, void* workspace, size_t workspace_bytes,
+                                    void* stream) {
+    if (w && !w->grouped) return fail(OSC_ERR_INVALID_ARG, "dense weights: use osc_mxfp8_linear");
+    return mxfp8_linear_impl(w, X_perm, off, M_total, ldx, Y, ldy, workspace, workspace_bytes, stream);
 }
 
 // ------------------------------- dynamic-protection control group (Section 4.2)

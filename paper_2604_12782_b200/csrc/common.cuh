@@ -34,7 +34,8 @@ cudaError_t launch_quant_extract_nvfp4(const CUtensorMap& tm_x, int M, int K, co
                                        const int32_t* prefix, const int32_t* idx_o, void* xq, void* sf, void* xo, int Ko,
                                        int Kop, int num_sms, int tensor_e, cudaStream_t st);
 cudaError_t launch_fp8_quant(const void* X, int64_t ldx, int M, int K, void* x8, void* sx, cudaStream_t st);
-cudaError_t launch_mxfp8_quant(const void* X, int64_t ldx, int M, int K, void* x8, void* sf, cudaStream_t st);
+cudaError_t launch_mxfp8_quant(const void* X, int64_t ldx, int M, int K, void* x8, void* sf, const int32_t* sched,
+                               int max_tiles, cudaStream_t st);
 cudaError_t launch_dyn_quant_extract(const void* X, int64_t ldx, int M, int K, void* xq, void* sf, void* xo, void* idx,
                                      void* val, cudaStream_t st);
 cudaError_t launch_build_sched(const int32_t* off, int E, int32_t* sched128, int max_tiles128, int32_t* sched256,

@@ -439,16 +439,28 @@ constexpr int MX8_ROWS_PER_CTA = 8;
 
 __global__ void __launch_bounds__(32 * MX8_ROWS_PER_CTA)
 mxfp8_quant_kernel(const uint16_t* __restrict__ X, int64_t ldx, int M, int M_pad, int K, uint8_t* __restrict__ x8,
-                   uint8_t* __restrict__ sf) {
+                   uint8_t* __restrict__ sf, const int32_t* __restrict__ sched, int max_tiles) {
     grid_launch_dependents();
     grid_dependency_wait();
     const int lane = threadIdx.x & 31;
-    const int r = blockIdx.x * MX8_ROWS_PER_CTA + (threadIdx.x >> 5);
-    if (r >= M_pad) return;
+    // Dense: scale row = tensor row.  Grouped: the warp index runs over the scale rows of the 128-row tile schedule
+    // (every expert starts on a 128-row scale block); scale rows past an expert's end get zero bytes.
+    const int v = blockIdx.x * MX8_ROWS_PER_CTA + (threadIdx.x >> 5);
+    int r = v, sr = v;
+    bool valid = v < M;
+    if (sched) {
+        const int tile = v >> 7;
+        if (tile >= sched[0]) return;
+        r = sched[1 + tile] + (v & 127);
+        valid = r < sched[1 + max_tiles + tile];
+        sr = sched[1 + 2 * max_tiles + tile] + (v & 127);
+    } else if (v >= M_pad) {
+        return;
+    }
     const int katoms = K / 128;
-    // scale word of (row r, 128-channel block a): block (r/128)*katoms + a, word (r%32)*4 + (r%128)/32
-    uint32_t* sf_row = reinterpret_cast<uint32_t*>(sf + (size_t)(r / 128) * katoms * 512) + (r & 31) * 4 + ((r & 127) >> 5);
-    if (r >= M) {
+    // scale word of (scale row sr, 128-channel block a): block (sr/128)*katoms + a, word (sr%32)*4 + (sr%128)/32
+    uint32_t* sf_row = reinterpret_cast<uint32_t*>(sf + (size_t)(sr / 128) * katoms * 512) + (sr & 31) * 4 + ((sr & 127) >> 5);
+    if (!valid) {
         for (int a = lane; a < katoms; a += 32) sf_row[(size_t)a * 128] = 0u;
         return;
     }
@@ -718,12 +730,13 @@ cudaError_t launch_fp8_quant(const void* X, int64_t ldx, int M, int K, void* x8,
                       static_cast<uint8_t*>(x8), static_cast<float*>(sx));
 }
 
-cudaError_t launch_mxfp8_quant(const void* X, int64_t ldx, int M, int K, void* x8, void* sf, cudaStream_t st) {
+cudaError_t launch_mxfp8_quant(const void* X, int64_t ldx, int M, int K, void* x8, void* sf, const int32_t* sched,
+                               int max_tiles, cudaStream_t st) {
     if (M <= 0) return cudaSuccess;
-    const int M_pad = (M + 127) / 128 * 128;
+    const int M_pad = sched ? max_tiles * 128 : (M + 127) / 128 * 128;
     return launch_pdl(mxfp8_quant_kernel, dim3((M_pad + MX8_ROWS_PER_CTA - 1) / MX8_ROWS_PER_CTA),
                       dim3(32 * MX8_ROWS_PER_CTA), 0, st, static_cast<const uint16_t*>(X), ldx, M, M_pad, K,
-                      static_cast<uint8_t*>(x8), static_cast<uint8_t*>(sf));
+                      static_cast<uint8_t*>(x8), static_cast<uint8_t*>(sf), sched, max_tiles);
 }
 
 cudaError_t launch_dyn_quant_extract(const void* X, int64_t ldx, int M, int K, void* xq, void* sf, void* xo, void* idx,

@@ -112,3 +112,55 @@ def test_mxfp8_down_projection_full_size(B, oracle):
     Yref, T = oracle.mxfp8_gemm(x8, sfa, w8, sfw, rows)
     assert_within_tolerance(host_f64(Y[torch.from_numpy(rows.astype(np.int64)).cuda()]), Yref, T, "mxfp8 down")
     assert not torch.isnan(Y.float()).any()
+
+
+def _grouped_check(B, oracle, counts, K, N, seed, sample=None):
+    E = counts.size
+    c = synth.moe_down_case(E, counts, K=K, N=N, seed=seed, weight_pool=min(E, 4))
+    M = c["M"]
+    off_h = synth.offsets_from_counts(counts)
+    w = B.osc_mxfp8_prepare_weights_grouped(dev_bf16(c["W"].reshape(E * N, K)).view(E, N, K))
+    sz = B.osc_mxfp8_act_sizes(w, M)
+    ws = poison(sz.workspace_bytes)
+    Y = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+    B.osc_mxfp8_linear_grouped(w, dev_bf16(c["X"]), torch.from_numpy(off_h).cuda(), Y, ws)
+    B.osc_sync_check()
+    x8, sf, parts = oracle.mxfp8_quantize_grouped(c["X"], off_h)
+    h = host_u8(ws)
+    assert np.array_equal(h[sz.x8_offset:sz.x8_offset + M * K].reshape(M, K), x8)
+    # activation scales, expert by expert (valid rows; padding rows of a block must be zero)
+    base = 0
+    sf_h = h[sz.sfa_offset:sz.sfa_offset + sz.sfa_bytes]
+    for e in range(E):
+        m = int(counts[e])
+        nb = (m + 127) // 128 * (K // 128) * 512
+        if m:
+            check_scales(oracle, sf_h[base:base + nb], parts[e][1], m, K)
+        base += nb
+    Yh = host_f64(Y)
+    wq = {}
+    experts = range(E) if sample is None else sample
+    for e in experts:
+        r0, r1 = int(off_h[e]), int(off_h[e + 1])
+        if r1 == r0:
+            continue
+        key = e % min(E, 4)
+        if key not in wq:
+            wq[key] = oracle.mxfp8_quantize(c["W"][e])
+        rows = np.arange(r1 - r0, dtype=np.int32) if sample is None else \
+            np.unique(np.array([0, r1 - r0 - 1, min(127, r1 - r0 - 1), min(128, r1 - r0 - 1), (r1 - r0) // 2], np.int32))
+        Yref, T = oracle.mxfp8_gemm(parts[e][0], parts[e][1], wq[key][0], wq[key][1], rows)
+        assert_within_tolerance(Yh[r0 + rows], Yref, T, f"grouped mxfp8 expert {e}")
+    assert not torch.isnan(Y.float()).any()
+
+
+@pytest.mark.parametrize("counts", [np.array([3, 0, 130, 1, 257, 128]), np.array([300, 0, 5, 256, 129, 511, 1, 385])])
+def test_mxfp8_grouped_small(B, oracle, counts):
+    _grouped_check(B, oracle, counts, 384, 320, 7)
+
+
+def test_mxfp8_grouped_moe_down_full_size(B, oracle):
+    counts = synth.zipf_expert_rows()
+    E = counts.size
+    big = np.argsort(-counts)
+    _grouped_check(B, oracle, counts, 768, 2048, 0, sample=[int(big[0]), int(big[-1]), 0, E - 1, E // 2])
