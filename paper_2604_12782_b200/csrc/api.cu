@@ -220,6 +220,7 @@ struct osc_mxfp8_weights {
     const uint8_t *w8, *sfw;
     int num_sms;
     CUtensorMap tm_b2[2];  // half tiles for 192- and 256-wide tiles
+    CUtensorMap tm_b128;   // 128-row weight tiles of the few-row kernel
     CUtensorMap tm_sfw;
 };
 
@@ -789,6 +790,7 @@ static osc_status mxfp8_prepare_impl(const void* W, int E, int N, int K, int64_t
     osc_status s = OSC_OK;
     for (int v = 0; v < 2 && s == OSC_OK; ++v)
         s = make_tmap(&w->tm_b2[v], w8, false, (uint64_t)E * N, K, K, (v == 0 ? 192 : 256) / 2);
+    if (s == OSC_OK) s = make_tmap(&w->tm_b128, w8, false, (uint64_t)E * N, K, K, 128);
     if (s == OSC_OK) s = make_tmap_sf(&w->tm_sfw, sfw, (uint64_t)E * sf_bytes(N, K) / 512, 1);
     if (s != OSC_OK) { delete w; return s; }
     *out = w;
@@ -830,8 +832,22 @@ static osc_status mxfp8_gemm_impl(const osc_mxfp8_weights* w, const void* x8, co
         return fail(OSC_ERR_ALIGN, "pointers must be 16-byte aligned and ldy a multiple of 8");
     GemmArgs a;
     memset(&a, 0, sizeof a);
+    if (use_decode_kernel(w->grouped, M, w->N, w->num_sms)) {
+        if (osc_status s = make_tmap(&a.tm_a, x8, false, M, w->K, w->K, 64)) return s;
+        a.tm_b = w->tm_b128;
+        a.sfa = static_cast<const uint8_t*>(sfa);
+        a.sfw = w->sfw;
+        a.Y = static_cast<uint16_t*>(Y);
+        a.ldy = ldy;
+        a.M = M; a.N = w->N; a.K = w->K; a.Kop = 0;
+        a.num_sms = w->num_sms;
+        const int S = gemm_decode_split(w->N, w->K / 128, w->num_sms);
+        cudaError_t e = launch_gemm_mxf8_decode(a, S, static_cast<cudaStream_t>(stream));
+        if (e != cudaSuccess) return cuda_fail(e, "gemm_decode_kernel(mxfp8)");
+        return OSC_OK;
+    }
     if (osc_status s = make_tmap(&a.tm_a, x8, false, M, w->K, w->K, 128)) return s;
-    // every problem runs on the CTA-pair kernel (256-row tiles); rows past the end are zero-filled by the loads or
+    // every other problem runs on the CTA-pair kernel (256-row tiles); rows past the end are zero-filled by the loads or
     // belong to the next expert, and are never stored
     const long row_tiles = w->grouped ? max_tiles2 - w->E / 2 : (M + 255) / 256;
     const int bn = gemm_pair_block_n(false, false, row_tiles, w->N, w->K / 128, w->num_sms);

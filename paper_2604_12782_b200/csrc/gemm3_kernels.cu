@@ -28,6 +28,7 @@ namespace decode {
 
 constexpr int MODE_OSC = 0;
 constexpr int MODE_FP8 = 1;
+constexpr int MODE_MXF8 = 2;            // block-scaled FP8 (MXFP8): one 128-channel scale block per stage and operand
 constexpr int BF = 128;                 // output features per CTA = MMA rows = TMEM lanes
 constexpr int MAX_TOK = 64;             // activation rows per call
 constexpr int ROW_BYTES = 128;
@@ -42,7 +43,9 @@ constexpr int PSTR = MAX_TOK + 4;       // row stride (floats) of a parked parti
 
 template <int MODE>
 struct Cfg {
-    static constexpr int SF_BYTES = (MODE == MODE_OSC) ? 1024 : 0;   // per operand and stage
+    static constexpr bool SCALED = MODE != MODE_FP8;
+    static constexpr int KA = (MODE == MODE_OSC) ? 2 : 1;            // 128-channel scale blocks per stage
+    static constexpr int SF_BYTES = SCALED ? 1024 : 0;               // per operand and stage (MXFP8 uses half of it)
     static constexpr int STAGE_BYTES = W_BYTES + X_BYTES + 2 * SF_BYTES;
     static constexpr int STAGES = 4;   // ~105 KB per CTA: the CTAs of two consecutive launches share an SM, so the
                                        // next call's weight loads overlap this call's reduction and stores
@@ -134,16 +137,16 @@ __global__ void __launch_bounds__(THREADS, 2) gemm_decode_kernel(const __grid_co
         // weights (and their scales) of the first ring before the dependency wait, activations after it
         auto expect = [&](int kb, int s) {
             uint32_t bytes = W_BYTES + X_BYTES;
-            if (MODE == MODE_OSC && kb < nkb_a) bytes += 2u * 512u * (uint32_t)min(2, katoms_total - 2 * kb);
+            if (C::SCALED && kb < nkb_a) bytes += 2u * 512u * (uint32_t)min(C::KA, katoms_total - C::KA * kb);
             mbar_arrive_expect_tx(&full_bar[s], bytes);
         };
         auto load_w = [&](int kb, int s) {
             uint8_t* st = smem + s * C::STAGE_BYTES;
             if (kb < nkb_a) {
                 tma_load_2d(st, &args.tm_b, &full_bar[s], kb * ROW_BYTES, n0);
-                if (MODE == MODE_OSC) {
-                    const int ka = min(2, katoms_total - 2 * kb);
-                    const uint8_t* sw = args.sfw + ((int64_t)tile * katoms_total + 2 * kb) * 512;
+                if (C::SCALED) {
+                    const int ka = min(C::KA, katoms_total - C::KA * kb);
+                    const uint8_t* sw = args.sfw + ((int64_t)tile * katoms_total + C::KA * kb) * 512;
                     bulk_load(st + W_BYTES + X_BYTES, sw, (uint32_t)ka * 512u, &full_bar[s]);
                 }
             } else {
@@ -154,9 +157,9 @@ __global__ void __launch_bounds__(THREADS, 2) gemm_decode_kernel(const __grid_co
             uint8_t* st = smem + s * C::STAGE_BYTES;
             if (kb < nkb_a) {
                 tma_load_2d(st + W_BYTES, &args.tm_a, &full_bar[s], kb * ROW_BYTES, 0);
-                if (MODE == MODE_OSC) {
-                    const int ka = min(2, katoms_total - 2 * kb);
-                    bulk_load(st + W_BYTES + X_BYTES + C::SF_BYTES, args.sfa + (int64_t)(2 * kb) * 512, (uint32_t)ka * 512u,
+                if (C::SCALED) {
+                    const int ka = min(C::KA, katoms_total - C::KA * kb);
+                    bulk_load(st + W_BYTES + X_BYTES + C::SF_BYTES, args.sfa + (int64_t)(C::KA * kb) * 512, (uint32_t)ka * 512u,
                               &full_bar[s]);
                 }
             } else {
@@ -192,7 +195,9 @@ __global__ void __launch_bounds__(THREADS, 2) gemm_decode_kernel(const __grid_co
         // -------------------------------------------------------------- MMA issuer
         int s = 0;
         uint32_t ph = 0;
-        const uint32_t idesc_a = (MODE == MODE_OSC) ? idesc_mxf4(BF, ntok) : idesc_e4m3(BF, ntok);
+        const uint32_t idesc_a = (MODE == MODE_OSC)    ? idesc_mxf4(BF, ntok)
+                                 : (MODE == MODE_MXF8) ? idesc_mxf8(BF, ntok)
+                                                       : idesc_e4m3(BF, ntok);
         const uint32_t idesc_b = idesc_bf16(BF, ntok);
         const uint64_t desc_hi = smem_desc_sw128(0);
         const uint64_t sf_hi = smem_desc_sf(0);
@@ -225,6 +230,15 @@ __global__ void __launch_bounds__(THREADS, 2) gemm_decode_kernel(const __grid_co
                                      (first | (uint32_t)k) ? 1u : 0u);
                         }
                     }
+                } else if (MODE == MODE_MXF8) {
+                    const uint64_t sfw_d = sf_hi | (uint64_t)((sbase + W_BYTES + X_BYTES) >> 4);
+                    const uint64_t sfx_d = sf_hi | (uint64_t)((sbase + W_BYTES + X_BYTES + C::SF_BYTES) >> 4);
+                    tc_copy_sf(tmem_base + TM_SFW, sfw_d);
+                    tc_copy_sf(tmem_base + TM_SFX, sfx_d);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        mma_mxf8(tmem_base, wdesc + 2 * k, xdesc + 2 * k, idesc_a | idesc_sf_ids(k, k), tmem_base + TM_SFW,
+                                 tmem_base + TM_SFX, (first | (uint32_t)k) ? 1u : 0u);
                 } else if (MODE == MODE_OSC) {
 #pragma unroll
                     for (int k = 0; k < 4; ++k)
@@ -385,6 +399,9 @@ int gemm_decode_split(int N, int nkb, int num_sms) {
 
 cudaError_t launch_gemm_dual_decode(const GemmArgs& a, int S, cudaStream_t st) {
     return decode::launch_cfg<decode::MODE_OSC>(a, S, st);
+}
+cudaError_t launch_gemm_mxf8_decode(const GemmArgs& a, int S, cudaStream_t st) {
+    return decode::launch_cfg<decode::MODE_MXF8>(a, S, st);
 }
 cudaError_t launch_gemm_fp8_decode(const GemmArgs& a, int S, cudaStream_t st) {
     return decode::launch_cfg<decode::MODE_FP8>(a, S, st);

@@ -120,3 +120,20 @@ def test_decode_kernel_is_deterministic(B, env):
         Ys.append(Y)
     B.osc_sync_check()
     assert torch.equal(Ys[0], Ys[1]) and torch.equal(Ys[0], Ys[2])
+
+
+@pytest.mark.parametrize("M,K,N,split", [(1, 128, 64, None), (16, 768, 320, 3), (40, 1536, 1024, 4), (64, 12288, 256, 8),
+                                         (33, 384, 192, 2)])
+def test_decode_kernel_mxfp8(B, oracle, env, M, K, N, split):
+    c = synth.fp8_linear_case(M + K + 1, M, K, N)
+    Yref, T, (x8, sfa), _ = oracle.mxfp8_linear(c["X"], c["W"])
+    w = B.osc_mxfp8_prepare_weights(dev_bf16(c["W"]))
+    sz = B.osc_mxfp8_act_sizes(w, M)
+    for mode in (2, 0):
+        env(mode, split if mode else None)
+        ws = poison(sz.workspace_bytes)
+        Y = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+        B.osc_mxfp8_linear(w, dev_bf16(c["X"]), Y, ws)
+        B.osc_sync_check()
+        assert np.array_equal(ws[sz.x8_offset:sz.x8_offset + M * K].cpu().numpy().reshape(M, K), x8)
+        assert_within_tolerance(host_f64(Y), Yref, T, f"mxfp8 decode={mode} M={M} K={K} N={N} S={split}")
