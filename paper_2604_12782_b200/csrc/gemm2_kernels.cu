@@ -226,7 +226,7 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
                             tma_load_2d_pair(st + A_BYTES + C::B_BYTES, &args.tm_sfa, fb, 0, sfa_blk + C::KA * kb);
 #pragma unroll
                             for (int j = 0; j < C::SFB_ATOMS; ++j) {
-                                const int atom = C::TILED_SF ? (n0 / BN) * C::SFB_ATOMS + j
+                                const int atom = C::TILED_SF ? (ti.expert * num_n + n0 / BN) * C::SFB_ATOMS + j
                                                              : ti.expert * natoms + min(n0 / 128 + j, natoms - 1);
                                 tma_load_2d_pair(st + A_BYTES + C::B_BYTES + C::SFA_BYTES + j * (C::KA * 512), &args.tm_sfw,
                                                  fb, 0, atom * katoms_total + C::KA * kb);
@@ -480,7 +480,7 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
 #pragma unroll
                     for (int rr = 0; rr < 8; ++rr) {
                         const int rl = rr * 4 + (lane >> 3);
-                        if (wrow0 + rl < ti.row_end)
+                        if (wrow0 + rl < ti.row_end && n0 + c * 64 + j * 8 < N)
                             *reinterpret_cast<uint4*>(args.Y + (int64_t)(wrow0 + rl) * args.ldy + n0 + c * 64 + j * 8) =
                                 *reinterpret_cast<const uint4*>(buf + rl * 128 + ((j ^ (rl & 7)) << 4));
                     }
