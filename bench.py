@@ -45,7 +45,7 @@ METRIC = "OSC linear TFLOP/s"
 # DRAM traffic of one dual-path GEMM launch on the bench workload: dram__bytes_read.sum (38.9 MB) +
 # dram__bytes_write.sum (55.5 MB) from the ncu capture summarised in
 # profiles/gemm_pair_and_quant_extract_qkv_M8192.md (same workload, one launch).
-GEMM_TRAFFIC_BYTES = 94.4e6
+GEMM_TRAFFIC_BYTES = 98.0e6
 
 
 def load_peaks():
