@@ -42,8 +42,8 @@ WORKLOAD = {"name": "qwen3-8b-qkv", "M": 8192, "K": 4096, "N": 6144, "ch_per_gro
 NSETS = 4
 METRIC = "OSC linear TFLOP/s"
 
-# DRAM traffic of one dual-path GEMM launch on the bench workload: dram__bytes_read.sum (38.9 MB) +
-# dram__bytes_write.sum (55.5 MB) from the ncu capture summarised in
+# DRAM traffic of one dual-path GEMM launch on the bench workload: dram__bytes_read.sum (38.8 MB) +
+# dram__bytes_write.sum (59.2 MB) from the ncu capture summarised in
 # profiles/gemm_pair_and_quant_extract_qkv_M8192.md (same workload, one launch).
 GEMM_TRAFFIC_BYTES = 98.0e6
 
