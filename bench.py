@@ -20,7 +20,8 @@ Between timed steps the buffers rotate over 4 independent sets (inputs, workspac
 outputs and prepared weights: ~0.9 GB, 7x the L2), so no step finds its data in L2.
 
 `--impl reference` times the CPU oracle instead (host cores, bounded sample per step).
-`--sweep` prints a table over all benchmark shapes to stderr and gpurun_out/ (not a bench line).
+`--sweep` prints a table over all benchmark shapes to stderr and writes sweep.json into the output folder
+(OSC_BENCH_OUT, a scratch folder beside this file by default); it prints no bench line.
 """
 from __future__ import annotations
 
@@ -658,8 +659,9 @@ def run_sweep(args):
                  "tflops": roofline.fp8_flops(Mt, N, K) / ms / 1e9, "pct_roofline": 100 * troof / (ms * 1e-3),
                  "roof_us": troof * 1e6})
 
-    os.makedirs(os.path.join(ROOT, "gpurun_out"), exist_ok=True)
-    with open(os.path.join(ROOT, "gpurun_out", "sweep.json"), "w") as f:
+    out_dir = os.environ.get("OSC_BENCH_OUT", os.path.join(ROOT, "gpurun_out"))
+    os.makedirs(out_dir, exist_ok=True)
+    with open(os.path.join(out_dir, "sweep.json"), "w") as f:
         json.dump({"peaks": pk, "rows": rows}, f, indent=1)
     for r in rows:
         print(json.dumps(r), file=sys.stderr)
