@@ -128,13 +128,15 @@ static bool use_pair_kernel(bool grouped, int M, int E) {
 }
 
 // Dense problems with few rows run on the few-row kernel (operands swapped, K split over a cluster): up to 32
-// rows always, up to 64 rows when there are more 128-feature tiles than SMs (measured on B200: with 48 tiles
-// and 64 rows the 128-row-tile kernel is still ahead).  OSC_DECODE=0 disables, OSC_DECODE=2 forces it up to 64 rows.
-static bool use_decode_kernel(bool grouped, int M, int N, int num_sms) {
+// rows always; up to 64 rows when there are more 128-feature tiles than SMs or the K loop is long (64 stages or
+// more) - measured on B200: with 48 tiles, 20 stages and 64 rows the 128-row-tile kernel is still ahead (11.5 vs
+// 14.4 us), with 32 tiles and 96 stages it is behind (24.4 vs 21.9 us).  OSC_DECODE=0 disables, OSC_DECODE=2 forces
+// it up to 64 rows.
+static bool use_decode_kernel(bool grouped, int M, int N, int nkb, int num_sms) {
     const char* e = getenv("OSC_DECODE");   // read per call: tests switch it inside one process
     const int mode = e ? atoi(e) : 1;
     if (mode == 0 || grouped || M > 64) return false;
-    return mode == 2 || M <= 32 || (N + 127) / 128 >= num_sms;
+    return mode == 2 || M <= 32 || (N + 127) / 128 >= num_sms || nkb >= 64;
 }
 
 // ----------------------------------------------------------------- the table
@@ -431,7 +433,7 @@ static osc_status gemm_impl(const osc_weights* w, const void* xq, const void* sf
         return fail(OSC_ERR_ALIGN, "pointers must be 16-byte aligned and ldy a multiple of 8");
     GemmArgs a;
     memset(&a, 0, sizeof a);
-    if (use_decode_kernel(w->grouped, M, w->N, w->num_sms)) {
+    if (use_decode_kernel(w->grouped, M, w->N, (w->K + 255) / 256 + w->Kop / 64, w->num_sms)) {
         if (osc_status s = make_tmap(&a.tm_a, xq, false, M, w->K / 2, w->K / 2, 64)) return s;
         a.tm_b = w->tm_b[1];
         if (w->Kop > 0) {
@@ -651,7 +653,7 @@ static osc_status fp8_gemm_impl(const osc_fp8_weights* w, const void* x8, const 
         return fail(OSC_ERR_ALIGN, "pointers must be 16-byte aligned and ldy a multiple of 8");
     GemmArgs a;
     memset(&a, 0, sizeof a);
-    if (use_decode_kernel(w->grouped, M, w->N, w->num_sms)) {
+    if (use_decode_kernel(w->grouped, M, w->N, w->K / 128, w->num_sms)) {
         if (osc_status s = make_tmap(&a.tm_a, x8, false, M, w->K, w->K, 64)) return s;
         a.tm_b = w->tm_b[1];
         a.sx = static_cast<const float*>(sx);
@@ -832,7 +834,7 @@ static osc_status mxfp8_gemm_impl(const osc_mxfp8_weights* w, const void* x8, co
         return fail(OSC_ERR_ALIGN, "pointers must be 16-byte aligned and ldy a multiple of 8");
     GemmArgs a;
     memset(&a, 0, sizeof a);
-    if (use_decode_kernel(w->grouped, M, w->N, w->num_sms)) {
+    if (use_decode_kernel(w->grouped, M, w->N, w->K / 128, w->num_sms)) {
         if (osc_status s = make_tmap(&a.tm_a, x8, false, M, w->K, w->K, 64)) return s;
         a.tm_b = w->tm_b128;
         a.sfa = static_cast<const uint8_t*>(sfa);

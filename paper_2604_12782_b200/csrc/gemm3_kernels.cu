@@ -315,24 +315,34 @@ done:
             uint32_t peer[MAX_CLUSTER];
 #pragma unroll
             for (int r = 0; r < MAX_CLUSTER; ++r) peer[r] = map_to_cta(mine, (uint32_t)min(r, S - 1));
-            for (int c = rank; c * 4 < ntok; c += S) {
-                float4 p[MAX_CLUSTER];
+            // two chunks per pass: the distributed-shared-memory loads of both (2 S round trips' worth) are in flight together
+            for (int c0 = rank; c0 * 4 < ntok; c0 += 2 * S) {
+                float4 p[2][MAX_CLUSTER];
 #pragma unroll
-                for (int r = 0; r < MAX_CLUSTER; ++r)
-                    if (r < S) p[r] = ld_cluster_f32x4(peer[r] + (uint32_t)(c * 16));
-                float4 v = p[0];
+                for (int h = 0; h < 2; ++h) {
+                    const int c = c0 + h * S;
 #pragma unroll
-                for (int r = 1; r < MAX_CLUSTER; ++r)
-                    if (r < S) { v.x += p[r].x; v.y += p[r].y; v.z += p[r].z; v.w += p[r].w; }
-                if (n < N) {
-                    const float o[4] = {v.x, v.y, v.z, v.w};
+                    for (int r = 0; r < MAX_CLUSTER; ++r)
+                        if (r < S && c * 4 < ntok) p[h][r] = ld_cluster_f32x4(peer[r] + (uint32_t)(c * 16));
+                }
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const int t = 4 * c + i;
-                        if (t < M) {
-                            float y = o[i];
-                            if (MODE == MODE_FP8) y = y * (args.sx[t] * swn);
-                            args.Y[(int64_t)t * args.ldy + n] = __bfloat16_as_ushort(__float2bfloat16_rn(y));
+                for (int h = 0; h < 2; ++h) {
+                    const int c = c0 + h * S;
+                    if (c * 4 >= ntok) break;
+                    float4 v = p[h][0];
+#pragma unroll
+                    for (int r = 1; r < MAX_CLUSTER; ++r)
+                        if (r < S) { v.x += p[h][r].x; v.y += p[h][r].y; v.z += p[h][r].z; v.w += p[h][r].w; }
+                    if (n < N) {
+                        const float o[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const int t = 4 * c + i;
+                            if (t < M) {
+                                float y = o[i];
+                                if (MODE == MODE_FP8) y = y * (args.sx[t] * swn);
+                                args.Y[(int64_t)t * args.ldy + n] = __bfloat16_as_ushort(__float2bfloat16_rn(y));
+                            }
                         }
                     }
                 }
