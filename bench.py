@@ -612,6 +612,30 @@ def run_sweep(args):
     osc_row("layer.gate_up", 4096, 4096, 24576, 1)
     fp8_row("layer.down_fp8", 4096, 12288, 4096)
 
+    # the four linears of one Qwen3-8B layer at M = 4096 back to back on one stream (independent tensors per linear):
+    # what the programmatic dependent launches between consecutive kernels are worth
+    if want("layer.chain"):
+        M = 4096
+        qkv = OscProblem(torch, B, synth.osc_linear_case(0, M, 4096, 6144, 2), 2)
+        opj = OscProblem(torch, B, synth.osc_linear_case(1, M, 4096, 4096, 1), 2)
+        gup = OscProblem(torch, B, synth.osc_linear_case(2, M, 4096, 24576, 1), 2)
+        dwn = Fp8Problem(torch, B, synth.fp8_linear_case(3, M, 12288, 4096), 2)
+        parts = [qkv, opj, gup, dwn]
+        each = [time_loop(torch, p.step, steps, warm) for p in parts]
+
+        def chain(i):
+            for p in parts:
+                p.step(i)
+        ms = time_loop(torch, chain, steps, warm)
+        gms = time_graph(torch, chain, 8)
+        B.osc_sync_check()
+        troof = (roofline.osc_roofline_seconds(M, 6144, 4096, qkv.K_o, peaks) + roofline.osc_roofline_seconds(M, 4096, 4096, opj.K_o, peaks)
+                 + roofline.osc_roofline_seconds(M, 24576, 4096, gup.K_o, peaks) + roofline.fp8_roofline_seconds(M, 4096, 12288, peaks))
+        rows.append({"name": "layer.chain(qkv,o_proj,gate_up,down_fp8)", "M": M, "ms": ms, "graph_ms": gms,
+                     "sum_of_separate_ms": sum(each), "pct_roofline": 100 * troof / (ms * 1e-3), "roof_us": troof * 1e6})
+        del parts, qkv, opj, gup, dwn
+        torch.cuda.empty_cache()
+
     # MoE: 128 experts, top-8 of 8192 tokens, Zipf(1.1) load
     counts = synth.zipf_expert_rows()
     E = counts.size
