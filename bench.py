@@ -601,8 +601,7 @@ def run_sweep(args):
     for M in (16, 64, 128, 2048, 8192):
         osc_row("gate_up", M, 4096, 24576, 1)
         fp8_row("down_fp8", M, 12288, 4096)
-        if M >= 128:
-            mxfp8_row("down_mxfp8", M, 12288, 4096)
+        mxfp8_row("down_mxfp8", M, 12288, 4096)
     nvfp4_row("qkv.nvfp4_g16", 8192, 4096, 6144)
     nvfp4_row("qkv.nvfp4_g16", 2048, 4096, 6144)
     dyn_row("qkv.dynamic_protection", 8192, 4096, 6144, 2)

@@ -439,7 +439,7 @@ constexpr int MX8_ROWS_PER_CTA = 8;
 
 __global__ void __launch_bounds__(32 * MX8_ROWS_PER_CTA)
 mxfp8_quant_kernel(const uint16_t* __restrict__ X, int64_t ldx, int M, int M_pad, int K, uint8_t* __restrict__ x8,
-                   uint8_t* __restrict__ sf, const int32_t* __restrict__ sched, int max_tiles) {
+                   uint8_t* __restrict__ sf, const int32_t* __restrict__ sched, int max_tiles, int kspan) {
     grid_launch_dependents();
     grid_dependency_wait();
     const int lane = threadIdx.x & 31;
@@ -460,15 +460,17 @@ mxfp8_quant_kernel(const uint16_t* __restrict__ X, int64_t ldx, int M, int M_pad
     const int katoms = K / 128;
     // scale word of (scale row sr, 128-channel block a): block (sr/128)*katoms + a, word (sr%32)*4 + (sr%128)/32
     uint32_t* sf_row = reinterpret_cast<uint32_t*>(sf + (size_t)(sr / 128) * katoms * 512) + (sr & 31) * 4 + ((sr & 127) >> 5);
+    // blockIdx.y splits the row into spans of kspan channels (a multiple of 1024), so that few rows still fill the GPU
+    const int k_begin = blockIdx.y * kspan, k_end = min(K, k_begin + kspan);
     if (!valid) {
-        for (int a = lane; a < katoms; a += 32) sf_row[(size_t)a * 128] = 0u;
+        for (int a = k_begin / 128 + lane; a < k_end / 128; a += 32) sf_row[(size_t)a * 128] = 0u;
         return;
     }
     const uint4* xrow = reinterpret_cast<const uint4*>(X + (int64_t)r * ldx);
     uint2* orow = reinterpret_cast<uint2*>(x8 + (int64_t)r * K);
-    const int nch = K / 8;  // 16-byte chunks in the row
-    constexpr int U = 4;    // independent loads in flight per lane
-    for (int c0 = 0; c0 < nch; c0 += 32 * U) {
+    const int nch = k_end / 8;  // 16-byte chunks up to the end of my span
+    constexpr int U = 4;        // independent loads in flight per lane
+    for (int c0 = k_begin / 8; c0 < nch; c0 += 32 * U) {
         uint4 v[U];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
@@ -734,9 +736,12 @@ cudaError_t launch_mxfp8_quant(const void* X, int64_t ldx, int M, int K, void* x
                                int max_tiles, cudaStream_t st) {
     if (M <= 0) return cudaSuccess;
     const int M_pad = sched ? max_tiles * 128 : (M + 127) / 128 * 128;
-    return launch_pdl(mxfp8_quant_kernel, dim3((M_pad + MX8_ROWS_PER_CTA - 1) / MX8_ROWS_PER_CTA),
+    // one warp per (row, span of 1024 channels = one pass of the warp's loop): few rows still fill the GPU, and
+    // with many rows it costs nothing (measured the same as whole rows per warp at M = 8192)
+    const int kspan = 1024;
+    return launch_pdl(mxfp8_quant_kernel, dim3((M_pad + MX8_ROWS_PER_CTA - 1) / MX8_ROWS_PER_CTA, (K + kspan - 1) / kspan),
                       dim3(32 * MX8_ROWS_PER_CTA), 0, st, static_cast<const uint16_t*>(X), ldx, M, M_pad, K,
-                      static_cast<uint8_t*>(x8), static_cast<uint8_t*>(sf), sched, max_tiles);
+                      static_cast<uint8_t*>(x8), static_cast<uint8_t*>(sf), sched, max_tiles, kspan);
 }
 
 cudaError_t launch_dyn_quant_extract(const void* X, int64_t ldx, int M, int K, void* xq, void* sf, void* xo, void* idx,
