@@ -434,10 +434,11 @@ static osc_status gemm_impl(const osc_weights* w, const void* xq, const void* sf
     GemmArgs a;
     memset(&a, 0, sizeof a);
     if (use_decode_kernel(w->grouped, M, w->N, (w->K + 255) / 256 + w->Kop / 64, w->num_sms)) {
-        if (osc_status s = make_tmap(&a.tm_a, xq, false, M, w->K / 2, w->K / 2, 64)) return s;
+        const uint32_t tok_box = (uint32_t)((M + 15) / 16 * 16);   // activation rows per tile = the MMA's N
+        if (osc_status s = make_tmap(&a.tm_a, xq, false, M, w->K / 2, w->K / 2, tok_box)) return s;
         a.tm_b = w->tm_b[1];
         if (w->Kop > 0) {
-            if (osc_status s = make_tmap(&a.tm_ao, xo, true, M, (uint64_t)w->Kop * 2, (uint64_t)w->Kop * 2, 64)) return s;
+            if (osc_status s = make_tmap(&a.tm_ao, xo, true, M, (uint64_t)w->Kop * 2, (uint64_t)w->Kop * 2, tok_box)) return s;
             a.tm_bo = w->tm_bo[1];
         }
         a.sfa = static_cast<const uint8_t*>(sfa);
@@ -654,7 +655,7 @@ static osc_status fp8_gemm_impl(const osc_fp8_weights* w, const void* x8, const 
     GemmArgs a;
     memset(&a, 0, sizeof a);
     if (use_decode_kernel(w->grouped, M, w->N, w->K / 128, w->num_sms)) {
-        if (osc_status s = make_tmap(&a.tm_a, x8, false, M, w->K, w->K, 64)) return s;
+        if (osc_status s = make_tmap(&a.tm_a, x8, false, M, w->K, w->K, (uint32_t)((M + 15) / 16 * 16))) return s;
         a.tm_b = w->tm_b[1];
         a.sx = static_cast<const float*>(sx);
         a.sw = w->sw;
@@ -835,7 +836,7 @@ static osc_status mxfp8_gemm_impl(const osc_mxfp8_weights* w, const void* x8, co
     GemmArgs a;
     memset(&a, 0, sizeof a);
     if (use_decode_kernel(w->grouped, M, w->N, w->K / 128, w->num_sms)) {
-        if (osc_status s = make_tmap(&a.tm_a, x8, false, M, w->K, w->K, 64)) return s;
+        if (osc_status s = make_tmap(&a.tm_a, x8, false, M, w->K, w->K, (uint32_t)((M + 15) / 16 * 16))) return s;
         a.tm_b = w->tm_b128;
         a.sfa = static_cast<const uint8_t*>(sfa);
         a.sfw = w->sfw;

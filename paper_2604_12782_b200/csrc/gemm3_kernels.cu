@@ -136,7 +136,7 @@ __global__ void __launch_bounds__(THREADS, 2) gemm_decode_kernel(const __grid_co
         // ------------------------------------------------------------ TMA producer
         // weights (and their scales) of the first ring before the dependency wait, activations after it
         auto expect = [&](int kb, int s) {
-            uint32_t bytes = W_BYTES + X_BYTES;
+            uint32_t bytes = W_BYTES + (uint32_t)(ntok * ROW_BYTES);   // the activation tile holds ntok rows
             if (C::SCALED && kb < nkb_a) bytes += 2u * 512u * (uint32_t)min(C::KA, katoms_total - C::KA * kb);
             mbar_arrive_expect_tx(&full_bar[s], bytes);
         };
@@ -389,9 +389,13 @@ static cudaError_t launch_cfg(const GemmArgs& a, int S, cudaStream_t st) {
 
 }  // namespace decode
 
-// Cluster size (K split) of the few-row kernel: about one CTA per SM (measured on B200: with 48 feature tiles
-// S = 2, 3 and 4 are within 10 % of each other and ~15 % faster than S = 1; with more tiles than SMs any split
-// only adds reduction work and a second wave), every rank with at least one K block.  OSC_DECODE_SPLIT overrides.
+// Cluster size (K split) of the few-row kernel: 4, 2 or 1, the largest with at most ~1.3 CTAs per SM.
+// Measured on B200 (rows = 16, K = 4096): a CTA alone on its SM streams its weights at ~107 GB/s and two CTAs on
+// one SM share that rate, so filling every second slot of every SM buys nothing (96 feature tiles: 9.2 us unsplit,
+// 9.6 us split in 2, 14.4 us split in 3 or 4); with 48 tiles (the QKV projection) the whole linear takes 10.0 us
+// with S = 4, 10.1 with S = 3, 10.9 with S = 2 or 1; with more tiles than SMs a split only adds reduction work and
+// a second wave (192 tiles: 15.1 / 18.1 / 23.1 us for S = 1 / 2 / 3).  Every rank gets at least one K block.
+// OSC_DECODE_SPLIT overrides.
 int gemm_decode_split(int N, int nkb, int num_sms) {
     static int forced = -1;
     if (forced < 0) {
@@ -399,10 +403,11 @@ int gemm_decode_split(int N, int nkb, int num_sms) {
         if (const char* e = getenv("OSC_DECODE_SPLIT")) forced = atoi(e);
     }
     const int tiles = (N + decode::BF - 1) / decode::BF;
-    int S = forced > 0 ? forced : num_sms / tiles;
-    if (S > 4 && forced <= 0) S = 4;
+    int S = 1;
+    if (forced > 0) S = forced;
+    else if (40 * tiles <= 13 * num_sms) S = 4;
+    else if (20 * tiles <= 13 * num_sms) S = 2;
     if (S > decode::MAX_CLUSTER) S = decode::MAX_CLUSTER;
-    if (S < 1) S = 1;
     while (S > 1 && (S - 1) * ((nkb + S - 1) / S) >= nkb) --S;   // no rank without a K block
     return S;
 }
