@@ -13,6 +13,7 @@ Function-to-paper map (details in the C file):
   dyn_quantize_extract / dyn_prepare_weights / dyn_linear   the dynamic-protection control group of Section 4.2
   nvfp4_quantize_extract / nvfp4_gemm / nvfp4_linear         the NVFP4 / G = 16 variant (efficiency table, G = 16)
   threshold / profile_indexing / clustering_density   Eq. 1-4, Algorithm 1 (offline profiling)
+  rmsnorm (oracle/rmsnorm.py)          the normalization in front of Algorithm 2 when the two are fused (Section 3.3)
 """
 from __future__ import annotations
 
@@ -377,3 +378,6 @@ def clustering_density(n_hit: np.ndarray, n_total: np.ndarray):
     """Eq. 4 and the block mean: C_k = n_hit/n_total (0 for groups without outlier tokens), mean over all K groups."""
     c = np.where(n_total > 0, n_hit / np.maximum(n_total, 1), 0.0)
     return c, float(c.mean())
+
+
+from .rmsnorm import f64_to_bf16_bits, rmsnorm  # noqa: E402,F401

@@ -1,0 +1,55 @@
+"""CPU oracle of the RMSNorm that feeds the quantizer when the two are fused (the producer of the QKV and
+gate/up inputs of a decoder layer; Section 3.3 places Algorithm 2 directly behind the operator that
+produces the activations).
+
+TEST INFRASTRUCTURE ONLY, like everything in this package.
+
+Definition (the plain one, in double):
+
+    y[m, k] = bf16( (x[m, k] * r[m]) * gamma[k] ),   r[m] = 1 / sqrt( (1/K) sum_k x[m, k]^2 + eps )
+
+with x, gamma bf16 values, eps an fp32 value, every operation in IEEE double and ONE final rounding
+(nearest, ties to even) to bf16.  The fused path is this function followed by Algorithm 2 on its output.
+
+Pins (tests/test_oracle_rmsnorm.py): torch's float64 rms_norm as the library routine, closed forms
+(constant rows, one non-zero per row, eps = 0 rows of +-1), power-of-two scale invariance at eps = 0,
+hand-worked double -> bf16 roundings (ties, subnormals, overflow, signed zero).
+"""
+from __future__ import annotations
+
+import math
+
+import numpy as np
+
+
+def _bf16_bits_to_f64(b: np.ndarray) -> np.ndarray:
+    u = np.ascontiguousarray(b, dtype=np.uint16).astype(np.uint32) << np.uint32(16)
+    return u.view(np.float32).astype(np.float64)
+
+
+def f64_to_bf16_bits(y: np.ndarray) -> np.ndarray:
+    """Nearest bf16 (ties to even) of doubles, in one rounding: scale so that the bf16 quantum of each value
+    is 1, round to integer, scale back.  bf16 = 8 significant bits, exponents as fp32 (subnormal quantum
+    2^-133, overflow to infinity at 2^128 - 2^119 and above)."""
+    y = np.asarray(y, dtype=np.float64)
+    _, e = np.frexp(y)                         # |y| in [2^(e-1), 2^e)
+    q = np.maximum(e - 8, -133)                # exponent of the quantum
+    n = np.rint(np.ldexp(y, -q))               # exact scaling; rint rounds halves to even
+    v = np.ldexp(n, q)                         # a bf16 value (or 2^128 after rounding up)
+    with np.errstate(over="ignore"):
+        f = v.astype(np.float32)               # exact for every finite bf16 value; 2^128 -> inf
+    bits = (f.view(np.uint32) >> np.uint32(16)).astype(np.uint16)
+    nan = np.isnan(y)
+    if nan.any():
+        bits = np.where(nan, np.uint16(0x7FC0), bits)
+    return bits
+
+
+def rmsnorm(H: np.ndarray, gamma: np.ndarray, eps: float) -> np.ndarray:
+    """H [M, K] bf16 bits, gamma [K] bf16 bits, eps -> normalized rows as bf16 bits [M, K]."""
+    x = _bf16_bits_to_f64(H)
+    g = _bf16_bits_to_f64(gamma)
+    K = x.shape[1]
+    ms = np.array([math.fsum(row) for row in x * x]) / K      # squares are exact in double; fsum is the exact sum, rounded once
+    r = 1.0 / np.sqrt(ms + float(np.float32(eps)))
+    return f64_to_bf16_bits((x * r[:, None]) * g[None, :])
