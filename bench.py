@@ -505,6 +505,51 @@ def run_sweep(args):
         del p, f8
         torch.cuda.empty_cache()
 
+    def rms_row(name, M, K, N, cpg, seed=0):
+        """RMSNorm in front of the OSC linear: fused into the quantizer against the two-step path (own RMSNorm kernel
+        writing bf16, then the stand-alone quantizer); the residual stream stands in for X."""
+        if not want(name):
+            return
+        case = synth.osc_linear_case(seed, M, K, N, cpg)
+        p = OscProblem(torch, B, case, NSETS)
+        gam = dev_bf16(torch, synth.f32_to_bf16_bits(np.random.default_rng(seed).uniform(0.5, 1.5, K).astype(np.float32)))
+        Xn = [torch.empty(M, K, dtype=torch.bfloat16, device="cuda") for _ in range(p.n)]
+        eps = 1e-6
+
+        def fused_q(i):
+            j = i % p.n
+            B.osc_rmsnorm_quantize_extract(p.w[j], p.X[j], gam, eps, *p.views(j))
+
+        def norm_only(i):
+            j = i % p.n
+            B.osc_rmsnorm(p.X[j], gam, eps, Xn[j])
+
+        def two_step_q(i):
+            j = i % p.n
+            B.osc_rmsnorm(p.X[j], gam, eps, Xn[j])
+            B.osc_quantize_extract(p.w[j], Xn[j], *p.views(j))
+
+        def fused_lin(i):
+            j = i % p.n
+            B.osc_rmsnorm_linear(p.w[j], p.X[j], gam, eps, p.Y[j], p.ws[j])
+
+        def two_step_lin(i):
+            j = i % p.n
+            B.osc_rmsnorm(p.X[j], gam, eps, Xn[j])
+            B.osc_linear(p.w[j], Xn[j], p.Y[j], p.ws[j])
+
+        t = {k: time_loop(torch, f, steps, warm) for k, f in
+             (("fused_quant_ms", fused_q), ("norm_ms", norm_only), ("two_step_quant_ms", two_step_q),
+              ("fused_linear_ms", fused_lin), ("two_step_linear_ms", two_step_lin))}
+        B.osc_sync_check()
+        byts = roofline.quantize_extract_bytes(M, K, p.K_o_pad)   # one read of the rows + the quantizer's outputs
+        rows.append({"name": name, "M": M, "K": K, "N": N, "K_o": p.K_o, **t, "ms": t["fused_linear_ms"],
+                     "fused_quant_gbs": byts / t["fused_quant_ms"] / 1e6,
+                     "fused_quant_frac_hbm": byts / (t["fused_quant_ms"] * 1e-3) / peaks["hbm"],
+                     "speedup_linear": t["two_step_linear_ms"] / t["fused_linear_ms"]})
+        del p, Xn
+        torch.cuda.empty_cache()
+
     def fp8_row(name, M, K, N, seed=0):
         if not want(name):
             return
@@ -602,6 +647,8 @@ def run_sweep(args):
         osc_row("gate_up", M, 4096, 24576, 1)
         fp8_row("down_fp8", M, 12288, 4096)
         mxfp8_row("down_mxfp8", M, 12288, 4096)
+    rms_row("qkv.rmsnorm_fused", 8192, 4096, 6144, 2)
+    rms_row("qkv.rmsnorm_fused", 2048, 4096, 6144, 2)
     nvfp4_row("qkv.nvfp4_g16", 8192, 4096, 6144)
     nvfp4_row("qkv.nvfp4_g16", 2048, 4096, 6144)
     dyn_row("qkv.dynamic_protection", 8192, 4096, 6144, 2)

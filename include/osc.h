@@ -159,6 +159,28 @@ osc_status osc_linear(const osc_weights* w, const void* X, int M, int64_t ldx, v
 osc_status osc_linear_static(const osc_weights* w, const void* X, int M, int64_t ldx, void* Y, int64_t ldy,
                              void* stream);
 
+/* ---- RMSNorm fused in front of Algorithm 2 -----------------------------------------------------------
+ * Section 3.3 places the OSC quantizer directly behind the operator that produces the activations; for the
+ * QKV and gate/up projections of a decoder layer that operator is an RMSNorm.  These calls read the residual
+ * stream H once and never write the normalized tensor:
+ *
+ *   r_m = 1 / sqrt( (1/K) sum_k H[m,k]^2 + eps ),   X[m,k] = bf16( (H[m,k] * r_m) * gamma[k] )
+ *
+ * with the squares, the sum, the division, the square root and the two multiplications in IEEE double and one
+ * rounding (nearest, ties to even) to bf16; Algorithm 2 then runs on X as in osc_quantize_extract.
+ *   H      dev bf16 [M, ldh] (ldh >= K, multiple of 8, 16-byte aligned); gamma dev bf16 [K], 16-byte aligned.
+ *   K <= 8192 (a row is held in registers), else OSC_ERR_SHAPE.  Dense weights only.
+ * osc_rmsnorm writes X itself (dev bf16 [M, ldx]): the unfused reference point for tests and measurements.
+ * osc_rmsnorm_quantize_extract's outputs equal osc_quantize_extract's on osc_rmsnorm's X bit for bit.
+ * osc_rmsnorm_linear = osc_rmsnorm_quantize_extract + osc_gemm_dual through the workspace of osc_act_sizes.
+ * Asynchronous on `stream`; status codes as above. */
+osc_status osc_rmsnorm(const void* H, int M, int K, int64_t ldh, const void* gamma, float eps, void* X, int64_t ldx,
+                       void* stream);
+osc_status osc_rmsnorm_quantize_extract(const osc_weights* w, const void* H, int M, int64_t ldh, const void* gamma,
+                                        float eps, void* xq, void* sfa, void* xo, void* stream);
+osc_status osc_rmsnorm_linear(const osc_weights* w, const void* H, int M, int64_t ldh, const void* gamma, float eps,
+                              void* Y, int64_t ldy, void* workspace, size_t workspace_bytes, void* stream);
+
 /* Grouped (MoE) form: rows of X_perm are sorted by expert, expert e owns rows
  * [off[e], off[e+1]); off: dev int32 [E+1], off[E] == M_total.  Expert e's scale rows start
  * at scale row sum_{e'<e} roundup(m_e', 128).  The tile schedule is built on the device. */

@@ -4,16 +4,19 @@ produces the activations).
 
 TEST INFRASTRUCTURE ONLY, like everything in this package.
 
-Definition (the plain one, in double):
+Definition (the paper does not state the arithmetic of the producer; this is the usual one: statistics in
+high precision, the element-wise part in fp32, one final rounding to bf16):
 
-    y[m, k] = bf16( (x[m, k] * r[m]) * gamma[k] ),   r[m] = 1 / sqrt( (1/K) sum_k x[m, k]^2 + eps )
+    r[m]    = fl32( 1 / sqrt( (1/K) sum_k x[m, k]^2 + eps ) )        sum exact, the rest in IEEE double
+    y[m, k] = bf16( fl32( fl32( x[m, k] * r[m] ) * gamma[k] ) )       two fp32 multiplications, then nearest-even
 
-with x, gamma bf16 values, eps an fp32 value, every operation in IEEE double and ONE final rounding
-(nearest, ties to even) to bf16.  The fused path is this function followed by Algorithm 2 on its output.
+with x, gamma bf16 values and eps an fp32 value.  The fused path is this function followed by Algorithm 2
+on its output.
 
-Pins (tests/test_oracle_rmsnorm.py): torch's float64 rms_norm as the library routine, closed forms
-(constant rows, one non-zero per row, eps = 0 rows of +-1), power-of-two scale invariance at eps = 0,
-hand-worked double -> bf16 roundings (ties, subnormals, overflow, signed zero).
+Pins (tests/test_oracle_rmsnorm.py): torch's float64 rms_norm as the library routine (agreement to one bf16
+unit, equality almost everywhere), closed forms (constant rows, one non-zero per row, eps = 0 rows of +-1),
+power-of-two scale invariance at eps = 0, hand-worked double -> bf16 roundings (ties, subnormals, overflow,
+signed zero).
 """
 from __future__ import annotations
 
@@ -48,8 +51,11 @@ def f64_to_bf16_bits(y: np.ndarray) -> np.ndarray:
 def rmsnorm(H: np.ndarray, gamma: np.ndarray, eps: float) -> np.ndarray:
     """H [M, K] bf16 bits, gamma [K] bf16 bits, eps -> normalized rows as bf16 bits [M, K]."""
     x = _bf16_bits_to_f64(H)
-    g = _bf16_bits_to_f64(gamma)
+    g32 = _bf16_bits_to_f64(gamma).astype(np.float32)
     K = x.shape[1]
     ms = np.array([math.fsum(row) for row in x * x]) / K      # squares are exact in double; fsum is the exact sum, rounded once
-    r = 1.0 / np.sqrt(ms + float(np.float32(eps)))
-    return f64_to_bf16_bits((x * r[:, None]) * g[None, :])
+    with np.errstate(divide="ignore", over="ignore", invalid="ignore"):
+        r32 = (1.0 / np.sqrt(ms + float(np.float32(eps)))).astype(np.float32)
+        t = x.astype(np.float32) * r32[:, None]                # fp32 product, rounded to nearest
+        y = t * g32[None, :]                                   # second fp32 product
+    return f64_to_bf16_bits(y.astype(np.float64))              # exact widening, then the one rounding to bf16

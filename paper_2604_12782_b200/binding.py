@@ -76,6 +76,9 @@ _SIGS = {
     "osc_linear": (_i, [_vp, _vp, _i, _i64, _vp, _i64, _vp, _sz, _vp]),
     "osc_linear_static": (_i, [_vp, _vp, _i, _i64, _vp, _i64, _vp]),
     "osc_linear_grouped": (_i, [_vp, _vp, _vp, _i, _i64, _vp, _i64, _vp, _sz, _vp]),
+    "osc_rmsnorm": (_i, [_vp, _i, _i, _i64, _vp, C.c_float, _vp, _i64, _vp]),
+    "osc_rmsnorm_quantize_extract": (_i, [_vp, _vp, _i, _i64, _vp, C.c_float, _vp, _vp, _vp, _vp]),
+    "osc_rmsnorm_linear": (_i, [_vp, _vp, _i, _i64, _vp, C.c_float, _vp, _i64, _vp, _sz, _vp]),
     "osc_profile_scratch_bytes": (_i, [_i, C.POINTER(_sz)]),
     "osc_profile_lut": (_i, [_vp, _i, _i, _i64, C.c_float, _vp, _sz, _vp, _vp, _vp, _vp, _vp]),
     "osc_fp8_prepare_weights": (_i, [_vp, _i, _i, _i64, _vp, _vp, _vp, C.POINTER(_vp)]),
@@ -260,6 +263,28 @@ def osc_linear_static(w: OscWeights, X: torch.Tensor, Y: torch.Tensor, stream=No
     M = X.shape[0]
     _check(_lib.osc_linear_static(w.ptr, _ptr(X), M, X.stride(0) if M else w.K, _ptr(Y), Y.stride(0) if M else w.N,
                                   _stream(stream)))
+
+
+def osc_rmsnorm(H: torch.Tensor, gamma: torch.Tensor, eps: float, X: torch.Tensor, stream=None):
+    """X = bf16(RMSNorm(H) * gamma), double arithmetic with one rounding: the unfused reference point."""
+    M, K = H.shape
+    _check(_lib.osc_rmsnorm(_ptr(H), M, K, H.stride(0) if M else K, _ptr(gamma), float(eps), _ptr(X),
+                            X.stride(0) if M else K, _stream(stream)))
+
+
+def osc_rmsnorm_quantize_extract(w: OscWeights, H: torch.Tensor, gamma: torch.Tensor, eps: float, xq, sfa, xo, stream=None):
+    """RMSNorm fused in front of Algorithm 2: H is read once, the normalized tensor is never written."""
+    M = H.shape[0]
+    _check(_lib.osc_rmsnorm_quantize_extract(w.ptr, _ptr(H), M, H.stride(0) if M else w.K, _ptr(gamma), float(eps),
+                                             _ptr(xq), _ptr(sfa), _ptr(xo) if w.K_o_pad else None, _stream(stream)))
+
+
+def osc_rmsnorm_linear(w: OscWeights, H: torch.Tensor, gamma: torch.Tensor, eps: float, Y: torch.Tensor,
+                       workspace: torch.Tensor, stream=None):
+    M = H.shape[0]
+    _check(_lib.osc_rmsnorm_linear(w.ptr, _ptr(H), M, H.stride(0) if M else w.K, _ptr(gamma), float(eps), _ptr(Y),
+                                   Y.stride(0) if M else w.N, _ptr(workspace),
+                                   workspace.numel() * workspace.element_size(), _stream(stream)))
 
 
 def osc_linear_grouped(w: OscWeights, X: torch.Tensor, off: torch.Tensor, Y: torch.Tensor, workspace: torch.Tensor,

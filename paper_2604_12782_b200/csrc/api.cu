@@ -513,6 +513,63 @@ osc_status osc_linear(const osc_weights* w, const void* X, int M, int64_t ldx, v
     return gemm_impl(w, ws + sz.xq_offset, ws + sz.sfa_offset, ws + sz.xo_offset, M, Y, ldy, nullptr, 0, nullptr, 0, st);
 }
 
+// ---- RMSNorm fused in front of Algorithm 2
+osc_status osc_rmsnorm(const void* H, int M, int K, int64_t ldh, const void* gamma, float eps, void* X, int64_t ldx,
+                       void* stream) {
+    if (M < 0) return fail(OSC_ERR_INVALID_ARG, "M = %d is negative", M);
+    if (K <= 0 || K % 128) return fail(OSC_ERR_SHAPE, "K = %d must be a positive multiple of 128", K);
+    if (K > 8192) return fail(OSC_ERR_SHAPE, "K = %d: the fused RMSNorm holds a row in registers, K <= 8192", K);
+    if (M == 0) return OSC_OK;
+    if (!H || !gamma || !X) return fail(OSC_ERR_INVALID_ARG, "null device pointer");
+    if (ldh < K || ldx < K) return fail(OSC_ERR_SHAPE, "ldh = %lld, ldx = %lld < K = %d", (long long)ldh, (long long)ldx, K);
+    if (ldh % 8 || ldx % 8 || !aligned16(H) || !aligned16(X) || !aligned16(gamma))
+        return fail(OSC_ERR_ALIGN, "H, X and gamma must be 16-byte aligned, ldh and ldx multiples of 8");
+    cudaError_t e = launch_rmsnorm_quant(false, H, ldh, M, K, gamma, eps, X, ldx, nullptr, nullptr, nullptr, nullptr,
+                                         0, 0, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(e, "rmsnorm_quant_kernel(norm only)");
+    return OSC_OK;
+}
+
+static osc_status rmsnorm_quantize_impl(const osc_weights* w, const void* H, int M, int64_t ldh, const void* gamma,
+                                        float eps, void* xq, void* sfa, void* xo, cudaStream_t st) {
+    if (w->grouped) return fail(OSC_ERR_INVALID_ARG, "grouped weights are not supported by the fused RMSNorm");
+    if (w->K > 8192) return fail(OSC_ERR_SHAPE, "K = %d: the fused RMSNorm holds a row in registers, K <= 8192", w->K);
+    if (M == 0) return OSC_OK;
+    if (!gamma || !aligned16(gamma)) return fail(OSC_ERR_ALIGN, "gamma must be non-null and 16-byte aligned");
+    if (!xq || !sfa || (w->Kop > 0 && !xo)) return fail(OSC_ERR_INVALID_ARG, "null output pointer");
+    if (!aligned16(xq) || !aligned16(sfa) || !aligned16(xo)) return fail(OSC_ERR_ALIGN, "outputs must be 16-byte aligned");
+    cudaError_t e = launch_rmsnorm_quant(true, H, ldh, M, w->K, gamma, eps, nullptr, 0, w->idx_o, xq, sfa,
+                                         w->Kop ? xo : nullptr, w->Ko, w->Kop, st);
+    if (e != cudaSuccess) return cuda_fail(e, "rmsnorm_quant_kernel");
+    return OSC_OK;
+}
+
+osc_status osc_rmsnorm_quantize_extract(const osc_weights* w, const void* H, int M, int64_t ldh, const void* gamma,
+                                        float eps, void* xq, void* sfa, void* xo, void* stream) {
+    if (osc_status s = check_act(w, H, M, ldh)) return s;
+    return rmsnorm_quantize_impl(w, H, M, ldh, gamma, eps, xq, sfa, xo, static_cast<cudaStream_t>(stream));
+}
+
+osc_status osc_rmsnorm_linear(const osc_weights* w, const void* H, int M, int64_t ldh, const void* gamma, float eps,
+                              void* Y, int64_t ldy, void* workspace, size_t workspace_bytes, void* stream) {
+    if (osc_status s = check_act(w, H, M, ldh)) return s;
+    if (w->grouped) return fail(OSC_ERR_INVALID_ARG, "grouped weights are not supported by the fused RMSNorm");
+    if (M == 0) return OSC_OK;
+    osc_act_sizes_t sz;
+    osc_act_sizes(w, M, &sz);
+    if (!workspace || !aligned16(workspace)) return fail(OSC_ERR_ALIGN, "workspace must be non-null and 16-byte aligned");
+    if (workspace_bytes < sz.workspace_bytes)
+        return fail(OSC_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", workspace_bytes, sz.workspace_bytes);
+    if (!Y) return fail(OSC_ERR_INVALID_ARG, "Y is null");
+    if (ldy < w->N) return fail(OSC_ERR_SHAPE, "ldy = %lld < N = %d", (long long)ldy, w->N);
+    if (ldy % 8 || !aligned16(Y)) return fail(OSC_ERR_ALIGN, "Y must be 16-byte aligned and ldy a multiple of 8");
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (osc_status s = rmsnorm_quantize_impl(w, H, M, ldh, gamma, eps, ws + sz.xq_offset, ws + sz.sfa_offset, ws + sz.xo_offset, st))
+        return s;
+    return gemm_impl(w, ws + sz.xq_offset, ws + sz.sfa_offset, ws + sz.xo_offset, M, Y, ldy, nullptr, 0, nullptr, 0, st);
+}
+
 osc_status osc_linear_grouped(const osc_weights* w, const void* X_perm, const int32_t* off, int M_total, int64_t ldx,
                               void* Y, int64_t ldy, void* workspace, size_t workspace_bytes, void* stream) {
     if (osc_status s = check_act(w, X_perm, M_total, ldx)) return s;

@@ -41,6 +41,11 @@ cudaError_t launch_dyn_quant_extract(const void* X, int64_t ldx, int M, int K, v
 cudaError_t launch_build_sched(const int32_t* off, int E, int32_t* sched128, int max_tiles128, int32_t* sched256,
                                int max_tiles256, cudaStream_t st);
 
+// norm_kernels.cu
+cudaError_t launch_rmsnorm_quant(bool quant, const void* H, int64_t ldh, int M, int K, const void* gamma, float eps,
+                                 void* Xn, int64_t ldx, const int32_t* idx_o, void* xq, void* sf,
+                                 void* xo, int Ko, int Kop, cudaStream_t st);
+
 // profile_kernels.cu
 cudaError_t launch_profile(const void* X, int64_t ldx, int S, int K, double alpha, double* sum, int32_t* counts,
                            int8_t* lut, int32_t* n_hit, int32_t* n_total, uint32_t* threshold_bits, int num_sms,

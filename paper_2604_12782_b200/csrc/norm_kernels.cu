@@ -1,0 +1,196 @@
+// RMSNorm fused in front of Algorithm 2 (Section 3.3 puts the OSC quantizer directly behind the operator that
+// produces the activations; in a decoder layer that operator is the RMSNorm in front of the QKV and gate/up
+// projections).  One pass over the residual stream instead of three (norm read + norm write + quantizer read).
+//
+// Arithmetic (statistics in double, element-wise part in fp32, one rounding to bf16):
+//   r   = fl32( 1 / sqrt( (1/K) sum_k x_k^2 + eps ) )     squares and sum in double (squares of bf16 are exact)
+//   y_k = bf16( fl32( fl32(x_k * r) * gamma_k ) )
+// followed by Algorithm 2 on the bf16 row y exactly as quant_extract_kernel does it (back-up of the flagged
+// channels, zero-out, E8M0 scale per 32, E2M1 codes).  The sum is a fixed tree (two partial sums per lane,
+// butterfly over the warp), so results are deterministic; against the exactly rounded sum it is off by a few
+// units of the 53rd bit, which changes r only if 1/sqrt(..) lies within ~1e-16 of an fp32 rounding boundary.
+//
+// One warp per row (K <= 8192): lane 0 fetches the row into shared memory with one bulk copy (cp.async.bulk, its
+// own mbarrier per warp); the first pass sums the squares; the second normalizes the row in place (bf16); then the
+// flagged channels are copied out through the channel list (lane t takes list entry t: 64-byte coalesced stores
+// into xo) and zeroed in the shared row; last, every lane quantizes whole 32-channel groups as in
+// quant_extract_kernel (amax without shuffles, one 16-byte store of codes, the four scale bytes of a 128-channel
+// block gathered by two shuffles).  Handling the flagged channels in registers, lane by lane through the bit mask,
+// made the lanes of a warp diverge at nearly every word (22 of 32 threads active on average, twice the
+// instructions).  A first version did the element-wise part in double too, with the
+// bf16 <-> double conversions as integer operations: ~90 instructions per element, the unrolled row loop no
+// longer fit the instruction cache, 172 us for 8192 x 4096 (ALU pipe and instruction fetch, fp64 pipe at 3 %).
+// Holding the row in registers needs the row loop fully unrolled, which made the compiler hoist every load of the
+// second pass and spill.
+#include "common.cuh"
+
+namespace osc {
+
+constexpr int RN_WARPS = 8;
+
+template <bool QUANT>
+__global__ void __launch_bounds__(32 * RN_WARPS)
+rmsnorm_quant_kernel(const uint16_t* __restrict__ H, int64_t ldh, int M, int M_pad, int K,
+                     const uint16_t* __restrict__ gamma, float eps, uint16_t* __restrict__ Xn, int64_t ldx,
+                     const int32_t* __restrict__ idx_o, uint8_t* __restrict__ xq,
+                     uint8_t* __restrict__ sf, uint16_t* __restrict__ xo, int Ko, int Kop) {
+    extern __shared__ uint4 rn_rows[];   // [RN_WARPS][K / 8], then one mbarrier and one give-up flag per warp
+    grid_launch_dependents();
+    const int lane = threadIdx.x & 31;
+    const int r = blockIdx.x * RN_WARPS + (threadIdx.x >> 5);
+    if (r >= M_pad) return;
+    const int katoms = K / 128;
+    // scale word of (row r, 128-channel block a): block (r/128)*katoms + a, word (r%32)*4 + (r%128)/32
+    uint32_t* sf_row = QUANT ? reinterpret_cast<uint32_t*>(sf + (size_t)(r / 128) * katoms * 512) + (r & 31) * 4 + ((r & 127) >> 5)
+                             : nullptr;
+    if (r >= M) {   // rows that only pad the last 128-row scale block
+        grid_dependency_wait();
+        if (QUANT)
+            for (int a = lane; a < katoms; a += 32) sf_row[(size_t)a * 128] = 0u;
+        return;
+    }
+    const uint4* hrow = reinterpret_cast<const uint4*>(H + (int64_t)r * ldh);
+    const uint4* grow = reinterpret_cast<const uint4*>(gamma);
+    const int nch = K / 8;   // 16-byte chunks in the row
+
+    const int warp = threadIdx.x >> 5;
+    uint4* row = rn_rows + (size_t)warp * nch;
+    uint64_t* bar = reinterpret_cast<uint64_t*>(rn_rows + (size_t)RN_WARPS * nch) + warp;
+    volatile int* give_up = reinterpret_cast<volatile int*>(reinterpret_cast<uint64_t*>(rn_rows + (size_t)RN_WARPS * nch) + RN_WARPS) + warp;
+    if (lane == 0) {
+        *give_up = 0;
+        mbar_init(bar, 1);
+        fence_barrier_init();
+    }
+    __syncwarp();
+    grid_dependency_wait();   // H may come from, and the outputs may still be read by, earlier kernels
+    if (lane == 0) {
+        mbar_arrive_expect_tx(bar, (uint32_t)K * 2u);
+        bulk_load(row, hrow, (uint32_t)K * 2u, bar);
+    }
+    __syncwarp();
+    if (!wait_bounded(bar, 0u, give_up, 41)) return;
+
+    const int nsteps = (nch + 31) / 32;
+    double ss0 = 0.0, ss1 = 0.0;
+#pragma unroll 2
+    for (int i = 0; i < nsteps; ++i) {
+        const int c = i * 32 + lane;
+        const uint4 v = (c < nch) ? row[c] : make_uint4(0u, 0u, 0u, 0u);
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const double a = (double)__uint_as_float(w[j] << 16), b = (double)__uint_as_float(w[j] & 0xFFFF0000u);
+            ss0 = fma(a, a, ss0);
+            ss1 = fma(b, b, ss1);
+        }
+    }
+    double ss = ss0 + ss1;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xFFFFFFFFu, ss, o);
+    ss = __shfl_sync(0xFFFFFFFFu, ss, 0);   // every lane continues with the same bits
+    const float r32 = (float)(1.0 / sqrt(ss / (double)K + (double)eps));
+
+    // ---- second pass: normalize; QUANT: in place in shared memory, else straight to global memory
+#pragma unroll 2
+    for (int i = 0; i < nsteps; ++i) {
+        const int c = i * 32 + lane;
+        if (c >= nch) break;
+        const uint4 g4 = grow[c], v = row[c];
+        const uint32_t gw[4] = {g4.x, g4.y, g4.z, g4.w};
+        uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float lo = __fmul_rn(__fmul_rn(__uint_as_float(w[j] << 16), r32), __uint_as_float(gw[j] << 16));
+            const float hi = __fmul_rn(__fmul_rn(__uint_as_float(w[j] & 0xFFFF0000u), r32), __uint_as_float(gw[j] & 0xFFFF0000u));
+            w[j] = bf162_bits(__floats2bfloat162_rn(lo, hi));   // nearest even; lo in the low half
+        }
+        if (QUANT) row[c] = make_uint4(w[0], w[1], w[2], w[3]);
+        else *reinterpret_cast<uint4*>(Xn + (int64_t)r * ldx + c * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+    if (!QUANT) return;
+    __syncwarp();
+
+    // ---- Algorithm 2 on the normalized row.  Back-up and zero-out: entry t of the (ascending) channel list goes to
+    // column t of xo; pad columns +0
+    uint16_t* row16 = reinterpret_cast<uint16_t*>(row);
+    for (int t = lane; t < Kop; t += 32) {
+        uint16_t e = 0;
+        if (t < Ko) {
+            const int ch = idx_o[t];
+            e = row16[ch];
+            row16[ch] = 0;
+        }
+        xo[(int64_t)r * Kop + t] = e;
+    }
+    __syncwarp();
+
+    // every lane quantizes whole 32-channel groups
+    const int ngrp = K / 32;
+    for (int g0 = 0; g0 < ngrp; g0 += 32) {
+        const int g = g0 + lane;
+        const bool in = g < ngrp;   // ngrp is a multiple of 4, so the four lanes of a scale word are in or out together
+        uint32_t w[16];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const uint4 v = in ? row[4 * g + j] : make_uint4(0u, 0u, 0u, 0u);
+            w[4 * j] = v.x; w[4 * j + 1] = v.y; w[4 * j + 2] = v.z; w[4 * j + 3] = v.w;
+        }
+        __nv_bfloat162 m2 = __habs2(as_bf162(w[0]));
+#pragma unroll
+        for (int t = 1; t < 16; ++t) m2 = __hmax2(m2, __habs2(as_bf162(w[t])));
+        const uint32_t am2 = bf162_bits(m2);
+        const uint32_t am = max(am2 & 0xFFFFu, am2 >> 16);
+        // CalculateScale: E8M0 code = biased exponent of amax - 2, floored at 0; Quantize: exact power-of-two
+        // scaling, hardware E2M1 rounding (nearest even, saturating)
+        const int ex = (int)(am >> 7);
+        int code = max(ex - 2, 0);
+        if (ex == 255) code = 255;
+        const __nv_bfloat162 inv2 = as_bf162(((uint32_t)(254 - min(code, 253)) << 7) * 0x10001u);
+        uint32_t q[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            float f[8];
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                const uint32_t p = bf162_bits(__hmul2(as_bf162(w[4 * j + t]), inv2));
+                f[2 * t] = __uint_as_float(p << 16);
+                f[2 * t + 1] = __uint_as_float(p & 0xFFFF0000u);
+            }
+            q[j] = e2m1x8(f[0], f[1], f[2], f[3], f[4], f[5], f[6], f[7]);
+        }
+        if (in) *reinterpret_cast<uint4*>(xq + (int64_t)r * (K / 2) + g * 16) = make_uint4(q[0], q[1], q[2], q[3]);
+        // the four scale bytes of a 128-channel block are one 32-bit word: gather from the four lanes that hold them
+        uint32_t word = (uint32_t)code << (8 * (g & 3));
+        word |= __shfl_xor_sync(0xFFFFFFFFu, word, 1);
+        word |= __shfl_xor_sync(0xFFFFFFFFu, word, 2);
+        if ((g & 3) == 0 && in) sf_row[(size_t)(g >> 2) * 128] = word;
+    }
+}
+
+// QUANT: Xn unused.  !QUANT: the quantizer arguments unused.  K <= 8192.
+cudaError_t launch_rmsnorm_quant(bool quant, const void* H, int64_t ldh, int M, int K, const void* gamma, float eps,
+                                 void* Xn, int64_t ldx, const int32_t* idx_o, void* xq, void* sf,
+                                 void* xo, int Ko, int Kop, cudaStream_t st) {
+    if (M <= 0) return cudaSuccess;
+    const int M_pad = quant ? (M + 127) / 128 * 128 : M;
+    const dim3 grid((M_pad + RN_WARPS - 1) / RN_WARPS), block(32 * RN_WARPS);
+    const size_t smem = (size_t)RN_WARPS * K * 2 + RN_WARPS * 16;
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(rmsnorm_quant_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, RN_WARPS * 8192 * 2 + RN_WARPS * 16);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(rmsnorm_quant_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, RN_WARPS * 8192 * 2 + RN_WARPS * 16);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    if (quant)
+        return launch_pdl(rmsnorm_quant_kernel<true>, grid, block, smem, st, static_cast<const uint16_t*>(H), ldh, M, M_pad, K,
+                          static_cast<const uint16_t*>(gamma), eps, static_cast<uint16_t*>(Xn), ldx, idx_o,
+                          static_cast<uint8_t*>(xq), static_cast<uint8_t*>(sf), static_cast<uint16_t*>(xo), Ko, Kop);
+    return launch_pdl(rmsnorm_quant_kernel<false>, grid, block, smem, st, static_cast<const uint16_t*>(H), ldh, M, M_pad, K,
+                      static_cast<const uint16_t*>(gamma), eps, static_cast<uint16_t*>(Xn), ldx, idx_o,
+                      static_cast<uint8_t*>(xq), static_cast<uint8_t*>(sf), static_cast<uint16_t*>(xo), Ko, Kop);
+}
+
+}  // namespace osc

@@ -83,11 +83,13 @@ def test_against_torch_float64_rms_norm(oracle):
     x = torch.from_numpy(synth.bf16_bits_to_f64(Hb))
     g = torch.from_numpy(synth.bf16_bits_to_f64(gb))
     y = torch.nn.functional.rms_norm(x, (K,), weight=g, eps=float(np.float32(eps)))
-    # the library's double result and the oracle's may differ in the last double bits (order of operations);
-    # the bf16 roundings agree unless a value sits within that distance of a rounding boundary
+    # the library works in double throughout, the oracle rounds r and the two products to fp32: the bf16 results
+    # agree unless the double value sits within ~2^-23 (relative) of a bf16 rounding boundary, and then by one unit
     want = oracle.f64_to_bf16_bits(y.numpy())
     got = oracle.rmsnorm(Hb, gb, eps)
-    assert np.count_nonzero(got != want) == 0
+    diff = np.abs(got.astype(np.int32) - want.astype(np.int32))
+    assert diff.max() <= 1
+    assert np.count_nonzero(diff) <= 1e-3 * got.size
     # and the result has unit mean square before gamma, to bf16 accuracy
     z = synth.bf16_bits_to_f64(got) / synth.bf16_bits_to_f64(gb)[None, :]
     assert np.allclose((z * z).mean(axis=1), 1.0, atol=5e-3)
