@@ -26,7 +26,7 @@
 
 namespace osc {
 
-constexpr int RN_WARPS = 8;
+constexpr int RN_WARPS = 14;
 
 template <bool QUANT>
 __global__ void __launch_bounds__(32 * RN_WARPS)
