@@ -115,16 +115,26 @@ static osc_status make_tmap_sf(CUtensorMap* tm, const void* base, uint64_t block
     return OSC_OK;
 }
 
-// Dense problems with more than 128 rows, and grouped problems whose experts average at least 96 rows, run
-// on the CTA-pair kernel (256-row tiles); the rest on the single-CTA kernel (128-row tiles).
-static bool use_pair_kernel(bool grouped, int M, int E) {
-    static int enabled = -1;
-    if (enabled < 0) {
+// Grouped problems whose experts average at least 96 rows run on the CTA-pair kernel (256-row tiles), the rest on
+// the single-CTA kernel (128-row tiles).  Dense problems with more than 128 rows take whichever kernel its cost
+// model puts ahead (single_ns / pair_ns: estimated time of the whole K loop over all waves of tiles): the pair
+// kernel is more than twice as efficient per tile, but with few rows and a long K loop its tiles fill a fraction
+// of the machine - down projection 12288 -> 4096 with 256 rows: 16 pair tiles on 74 pairs, 38 us, against 128
+// single-CTA tiles of 128 x 64 in one wave, 27 us.  The single-CTA estimate only holds while all its tiles run in
+// one wave (with more, the SMs compete for the L2 feed and it is about half as fast as the pair kernel), so it is
+// only considered then.  OSC_PAIR=0: never, OSC_PAIR=2: always when eligible.
+static bool use_pair_kernel(bool grouped, int M, int E, long single_ns = 0, long pair_ns = 0, bool single_one_wave = false) {
+    static int mode = -1;
+    if (mode < 0) {
         const char* e = getenv("OSC_PAIR");
-        enabled = (e && atoi(e) == 0) ? 0 : 1;
+        mode = e ? atoi(e) : 1;
+        if (mode < 0 || mode > 2) mode = 1;
     }
-    if (!enabled) return false;
-    return grouped ? (M / E >= 96) : (M > 128);
+    if (mode == 0) return false;
+    if (grouped) return M / E >= 96;
+    if (M <= 128) return false;
+    if (mode == 2 || single_ns <= 0 || pair_ns <= 0) return true;
+    return !single_one_wave || pair_ns <= single_ns;
 }
 
 // Dense problems with few rows run on the few-row kernel (operands swapped, K split over a cluster): up to 32
@@ -453,7 +463,11 @@ static osc_status gemm_impl(const osc_weights* w, const void* xq, const void* sf
         return OSC_OK;
     }
     if (osc_status s = make_tmap(&a.tm_a, xq, false, M, w->K / 2, w->K / 2, 128)) return s;
-    const int bn1 = gemm_block_n(sched ? max_tiles : (M + 127) / 128, w->N, w->num_sms);
+    const int nkb = (w->K + 255) / 256 + w->Kop / 64;
+    long single_ns = 0, pair_ns = 0;
+    const int bn1 = gemm_block_n(sched ? max_tiles : (M + 127) / 128, w->N, w->num_sms, &single_ns);
+    const long row_tiles2 = w->grouped ? (max_tiles2 > w->E / 2 ? max_tiles2 - w->E / 2 : 1) : (M + 255) / 256;
+    const int bn2 = gemm_pair_block_n(false, !w->grouped, row_tiles2, w->N, nkb, w->num_sms, &pair_ns);
     a.tm_b = w->tm_b[bn1 / 64 - 1];
     if (w->Kop > 0) {
         if (osc_status s = make_tmap(&a.tm_ao, xo, true, M, (uint64_t)w->Kop * 2, (uint64_t)w->Kop * 2, 128)) return s;
@@ -467,9 +481,8 @@ static osc_status gemm_impl(const osc_weights* w, const void* xq, const void* sf
     a.sched = sched; a.max_tiles = max_tiles; a.num_sms = w->num_sms;
     a.sched2 = sched2; a.max_tiles2 = max_tiles2;
     cudaError_t e;
-    if (use_pair_kernel(w->grouped, M, w->E)) {
-        const long row_tiles = w->grouped ? max_tiles2 - w->E / 2 : (M + 255) / 256;
-        const int bn = gemm_pair_block_n(false, !w->grouped, row_tiles, w->N, (w->K + 255) / 256 + w->Kop / 64, w->num_sms);
+    if (use_pair_kernel(w->grouped, M, w->E, single_ns * nkb, pair_ns, single_ns <= 470)) {
+        const int bn = bn2;
         const int v = bn == 192 ? 0 : bn == 256 ? 1 : 2;
         a.tm_b = w->tm_b2[v];
         a.tm_bo = w->tm_bo2[v];
@@ -726,7 +739,10 @@ static osc_status fp8_gemm_impl(const osc_fp8_weights* w, const void* x8, const 
         return OSC_OK;
     }
     if (osc_status s = make_tmap(&a.tm_a, x8, false, M, w->K, w->K, 128)) return s;
-    const int bn1 = gemm_block_n(sched ? max_tiles : (M + 127) / 128, w->N, w->num_sms);
+    long single_ns = 0, pair_ns = 0;
+    const int bn1 = gemm_block_n(sched ? max_tiles : (M + 127) / 128, w->N, w->num_sms, &single_ns);
+    const long row_tiles2 = w->grouped ? (max_tiles2 > w->E / 2 ? max_tiles2 - w->E / 2 : 1) : (M + 255) / 256;
+    const int bn2 = gemm_pair_block_n(true, false, row_tiles2, w->N, w->K / 128, w->num_sms, &pair_ns);
     a.tm_b = w->tm_b[bn1 / 64 - 1];
     a.sx = static_cast<const float*>(sx);
     a.sw = w->sw;
@@ -736,9 +752,8 @@ static osc_status fp8_gemm_impl(const osc_fp8_weights* w, const void* x8, const 
     a.sched = sched; a.max_tiles = max_tiles; a.num_sms = w->num_sms;
     a.sched2 = sched2; a.max_tiles2 = max_tiles2;
     cudaError_t e;
-    if (use_pair_kernel(w->grouped, M, w->E)) {
-        const long row_tiles = w->grouped ? max_tiles2 - w->E / 2 : (M + 255) / 256;
-        const int bn = gemm_pair_block_n(true, false, row_tiles, w->N, w->K / 128, w->num_sms);
+    if (use_pair_kernel(w->grouped, M, w->E, single_ns * (w->K / 128), pair_ns, single_ns <= 470)) {
+        const int bn = bn2;
         a.tm_b = w->tm_b2[bn == 256];
         if (osc_status s = make_tmap(&a.tm_y, Y, true, M, (uint64_t)w->N * 2, (uint64_t)ldy * 2, 32)) return s;
         e = launch_gemm_fp8_pair(a, bn, st);

@@ -77,14 +77,14 @@ struct GemmArgs {
 };
 cudaError_t launch_gemm_dual(const GemmArgs& a, int bn, cudaStream_t st);
 cudaError_t launch_gemm_fp8(const GemmArgs& a, int bn, cudaStream_t st);
-int gemm_block_n(int row_tiles, int N, int num_sms);
+int gemm_block_n(int row_tiles, int N, int num_sms, long* cost_ns = nullptr);
 
 // gemm2_kernels.cu (CTA pairs: 256-row tiles, dense or grouped)
 cudaError_t launch_gemm_dual_pair(const GemmArgs& a, int bn, cudaStream_t st);
 cudaError_t launch_gemm_fp8_pair(const GemmArgs& a, int bn, cudaStream_t st);
 cudaError_t launch_gemm_mxf8_pair(const GemmArgs& a, int bn, cudaStream_t st);
 cudaError_t launch_gemm_nvf4_pair(const GemmArgs& a, int bn, cudaStream_t st);
-int gemm_pair_block_n(bool fp8, bool allow_240, long row_tiles, int N, int stages, int num_sms);
+int gemm_pair_block_n(bool fp8, bool allow_240, long row_tiles, int N, int stages, int num_sms, long* cost_ns = nullptr);
 
 // gemm3_kernels.cu (few rows: operands swapped, K split over a cluster)
 cudaError_t launch_gemm_dual_decode(const GemmArgs& a, int S, cudaStream_t st);

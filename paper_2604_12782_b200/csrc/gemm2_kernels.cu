@@ -577,7 +577,7 @@ static cudaError_t launch_cfg(const GemmArgs& a, cudaStream_t st) {
 // plus the scale columns (epilogue hidden behind the next tile's K loop unless that loop is shorter
 // than the ~2 us drain), 256 has one accumulator (drain and hand-over exposed, ~2.7 us per tile).
 // The FP8 mode needs no scale columns: 256 wide with two accumulators.  OSC_PAIR_BLOCK_N overrides.
-int gemm_pair_block_n(bool fp8, bool allow_240, long row_tiles, int N, int stages, int num_sms) {
+int gemm_pair_block_n(bool fp8, bool allow_240, long row_tiles, int N, int stages, int num_sms, long* cost_ns) {
     static int forced = -1;
     if (forced < 0) {
         forced = 0;
@@ -586,6 +586,7 @@ int gemm_pair_block_n(bool fp8, bool allow_240, long row_tiles, int N, int stage
             if (v == 192 || v == 240 || v == 256) forced = v;
         }
     }
+    if (cost_ns) *cost_ns = 0;   // a forced width is never weighed against the other kernel
     if (forced && !((fp8 || !allow_240) && forced == 240)) return forced;
     const int pairs = num_sms / 2 > 0 ? num_sms / 2 : 1;
     const long mt = row_tiles;
@@ -602,6 +603,7 @@ int gemm_pair_block_n(bool fp8, bool allow_240, long row_tiles, int N, int stage
         const long cost = rounds * (two_acc ? hidden : loop + 2700);
         if (best < 0 || cost < best) { best = cost; best_bn = bn; }
     }
+    if (cost_ns) *cost_ns = best;
     return best_bn;
 }
 

@@ -371,10 +371,12 @@ done:
 }
 
 // ---------------------------------------------------------------- launchers
-// Tile width of the single-CTA kernel.  Few-row problems are weight streaming: every SM should pull
-// its share of the weights, so the width shrinks until there are about as many tiles as SMs.
-// Grouped problems have plenty of row tiles and take the widest tile.  OSC_BLOCK_N overrides.
-int gemm_block_n(int row_tiles, int N, int num_sms) {
+// Tile width of the single-CTA kernel: the one with the smallest (waves of tiles) x (time per K stage).  A stage
+// is bound by the SM's ingest of its operands (16 KB of activations + BN x 128 bytes of weights at ~107 GB/s),
+// measured on B200 at 96 stages: ~230 ns for 64 columns, ~265 ns for 128, ~390 ns for 192; 256 extrapolated.  With many
+// tiles the widest wins (least time per column), with few a narrower one that still fits in one wave.
+// cost_ns (optional) receives the estimate for one K stage times the waves.  OSC_BLOCK_N overrides.
+int gemm_block_n(int row_tiles, int N, int num_sms, long* cost_ns) {
     static int forced = -1;
     if (forced < 0) {
         forced = 0;
@@ -383,11 +385,20 @@ int gemm_block_n(int row_tiles, int N, int num_sms) {
             if (v == 64 || v == 128 || v == 192 || v == 256) forced = v;
         }
     }
+    if (cost_ns) *cost_ns = 0;
     if (forced) return forced;
     const int cand[4] = {256, 192, 128, 64};
-    for (int i = 0; i < 4; ++i)
-        if ((long)row_tiles * ((N + cand[i] - 1) / cand[i]) >= num_sms) return cand[i];
-    return 64;
+    const long stage_ns[4] = {470, 390, 265, 230};
+    long best = -1;
+    int best_bn = 64;
+    for (int i = 0; i < 4; ++i) {
+        const long tiles = (long)row_tiles * ((N + cand[i] - 1) / cand[i]);
+        const long waves = (tiles + num_sms - 1) / num_sms;
+        const long cost = waves * stage_ns[i];
+        if (best < 0 || cost < best) { best = cost; best_bn = cand[i]; }
+    }
+    if (cost_ns) *cost_ns = best;
+    return best_bn;
 }
 
 template <int MODE, int BN>
