@@ -233,6 +233,7 @@ struct osc_mxfp8_weights {
     int num_sms;
     CUtensorMap tm_b2[2];  // half tiles for 192- and 256-wide tiles
     CUtensorMap tm_b128;   // 128-row weight tiles of the few-row kernel
+    CUtensorMap tm_b1[4];  // single-CTA kernel: 64-, 128-, 192- and 256-row weight tiles
     CUtensorMap tm_sfw;
 };
 
@@ -866,6 +867,7 @@ static osc_status mxfp8_prepare_impl(const void* W, int E, int N, int K, int64_t
     for (int v = 0; v < 2 && s == OSC_OK; ++v)
         s = make_tmap(&w->tm_b2[v], w8, false, (uint64_t)E * N, K, K, (v == 0 ? 192 : 256) / 2);
     if (s == OSC_OK) s = make_tmap(&w->tm_b128, w8, false, (uint64_t)E * N, K, K, 128);
+    for (int v = 0; v < 4 && s == OSC_OK; ++v) s = make_tmap(&w->tm_b1[v], w8, false, (uint64_t)E * N, K, K, 64 * (v + 1));
     if (s == OSC_OK) s = make_tmap_sf(&w->tm_sfw, sfw, (uint64_t)E * sf_bytes(N, K) / 512, 1);
     if (s != OSC_OK) { delete w; return s; }
     *out = w;
@@ -922,10 +924,24 @@ static osc_status mxfp8_gemm_impl(const osc_mxfp8_weights* w, const void* x8, co
         return OSC_OK;
     }
     if (osc_status s = make_tmap(&a.tm_a, x8, false, M, w->K, w->K, 128)) return s;
-    // every other problem runs on the CTA-pair kernel (256-row tiles); rows past the end are zero-filled by the loads or
-    // belong to the next expert, and are never stored
+    // grouped problems run on the CTA-pair kernel (256-row tiles; rows past the end are zero-filled by the loads or
+    // belong to the next expert, and are never stored); dense ones on whichever kernel its cost model puts ahead
     const long row_tiles = w->grouped ? max_tiles2 - w->E / 2 : (M + 255) / 256;
-    const int bn = gemm_pair_block_n(false, false, row_tiles, w->N, w->K / 128, w->num_sms);
+    long single_ns = 0, pair_ns = 0;
+    const int bn1 = gemm_block_n((M + 127) / 128, w->N, w->num_sms, &single_ns);
+    const int bn = gemm_pair_block_n(false, false, row_tiles, w->N, w->K / 128, w->num_sms, &pair_ns);
+    if (!w->grouped && !use_pair_kernel(false, M, 1, single_ns * (w->K / 128), pair_ns, single_ns <= 470)) {
+        a.tm_b = w->tm_b1[bn1 / 64 - 1];
+        a.sfa = static_cast<const uint8_t*>(sfa);
+        a.sfw = w->sfw;
+        a.Y = static_cast<uint16_t*>(Y);
+        a.ldy = ldy;
+        a.M = M; a.N = w->N; a.K = w->K; a.Kop = 0;
+        a.num_sms = w->num_sms;
+        cudaError_t e1 = launch_gemm_mxf8(a, bn1, static_cast<cudaStream_t>(stream));
+        if (e1 != cudaSuccess) return cuda_fail(e1, "gemm_kernel(mxfp8)");
+        return OSC_OK;
+    }
     a.tm_b = w->tm_b2[bn == 256];
     a.tm_sfw = w->tm_sfw;
     const uint64_t sf_row_blocks = w->grouped ? (uint64_t)max_tiles : (uint64_t)((M + 127) / 128);

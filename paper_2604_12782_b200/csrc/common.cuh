@@ -77,6 +77,7 @@ struct GemmArgs {
 };
 cudaError_t launch_gemm_dual(const GemmArgs& a, int bn, cudaStream_t st);
 cudaError_t launch_gemm_fp8(const GemmArgs& a, int bn, cudaStream_t st);
+cudaError_t launch_gemm_mxf8(const GemmArgs& a, int bn, cudaStream_t st);
 int gemm_block_n(int row_tiles, int N, int num_sms, long* cost_ns = nullptr);
 
 // gemm2_kernels.cu (CTA pairs: 256-row tiles, dense or grouped)

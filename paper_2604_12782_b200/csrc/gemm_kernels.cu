@@ -15,6 +15,10 @@
 // MODE_FP8 : Section 3.4 fallback.  E4M3 x E4M3 (128 channels per stage, four K=32 MMAs); the
 //            per-row activation scale and per-output-row weight scale are applied in the epilogue.
 //
+// MODE_MXF8: the same fallback in its 8-bit micro-scaling form: E4M3 elements with one E8M0 scale per 32
+//            (128 channels and one 128-channel scale block per operand row block and stage, four K=32
+//            block-scaled MMAs taking scale byte k of the TMEM column); nothing to apply in the epilogue.
+//
 // A tile's first row, last valid row, first scale row and expert come either from arithmetic
 // (dense) or from the device-built schedule (grouped): rows past an expert's end are computed
 // (they read the next expert's rows or zero fill) but never stored.
@@ -26,6 +30,7 @@ namespace osc {
 
 constexpr int MODE_OSC = 0;
 constexpr int MODE_FP8 = 1;
+constexpr int MODE_MXF8 = 2;
 
 constexpr int BM = 128;            // rows per tile = TMEM lanes
 constexpr int ROW_BYTES = 128;     // bytes per operand row and stage (one 128-byte swizzle row)
@@ -39,12 +44,15 @@ constexpr int G_EPI_TILE_BYTES = 32 * 128;  // staging tile: 32 rows x 64 bf16 c
 template <int MODE, int BN>
 struct Cfg {
     static constexpr int SFB_ATOMS = (BN > 128) ? 2 : 1;  // 128-row scale blocks a tile can touch
-    // TMEM columns of one stage's scales (A: 8, B: 2 x atoms x 4); the FP8 mode keeps no scales in TMEM
-    static constexpr int SF_COLS = (MODE == MODE_OSC) ? 8 + 2 * SFB_ATOMS * 4 : 0;
+    static constexpr bool SCALED = MODE != MODE_FP8;
+    static constexpr int KA = (MODE == MODE_OSC) ? 2 : 1;   // 128-channel scale blocks per stage
+    // TMEM columns of one stage's scales (A: 8, B: 2 x atoms x 4; MXFP8 uses half of them); the FP8 mode keeps
+    // no scales in TMEM
+    static constexpr int SF_COLS = SCALED ? 8 + 2 * SFB_ATOMS * 4 : 0;
     static constexpr int ACC_STAGES = (2 * BN + SF_COLS <= TMEM_COLS) ? 2 : 1;
     static constexpr int B_BYTES = BN * ROW_BYTES;
-    static constexpr int SFA_BYTES = (MODE == MODE_OSC) ? 1024 : 0;
-    static constexpr int SFB_BYTES = (MODE == MODE_OSC) ? SFB_ATOMS * 1024 : 0;
+    static constexpr int SFA_BYTES = SCALED ? 1024 : 0;              // room for two blocks (MXFP8 fills one)
+    static constexpr int SFB_BYTES = SCALED ? SFB_ATOMS * 1024 : 0;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + SFA_BYTES + SFB_BYTES;  // multiple of 1024
     static constexpr int EPI_WARP_BYTES = (BN / 64) * G_EPI_TILE_BYTES;            // one lane quarter's 32 x BN outputs
     static constexpr int EPI_BYTES = 4 * EPI_WARP_BYTES;
@@ -155,6 +163,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
     const int nkb = nkb_a + nkb_b;
     const int katoms_total = K / 128;   // 128-channel scale blocks along K
     const int natoms = (N + 127) / 128;  // 128-row scale blocks of one expert's weights
+    constexpr int KA = C::KA;
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
@@ -168,19 +177,19 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
                 uint8_t* st = smem + s * C::STAGE_BYTES;
                 if (elect_one()) {
                     if (kb < nkb_a) {
-                        if (MODE == MODE_OSC) {
-                            const int ka = min(2, katoms_total - 2 * kb);  // 128-channel scale blocks in this stage
+                        if (C::SCALED) {
+                            const int ka = min(KA, katoms_total - KA * kb);  // 128-channel scale blocks in this stage
                             const uint32_t sfb = (uint32_t)ka * 512u;
                             mbar_arrive_expect_tx(&full_bar[s], A_BYTES + C::B_BYTES + sfb * (1 + C::SFB_ATOMS));
                             tma_load_2d(st, &args.tm_a, &full_bar[s], kb * ROW_BYTES, ti.row0);
                             tma_load_2d(st + A_BYTES, &args.tm_b, &full_bar[s], kb * ROW_BYTES, brow);
-                            const uint8_t* sa = args.sfa + ((int64_t)(ti.sf_row0 / 128) * katoms_total + 2 * kb) * 512;
+                            const uint8_t* sa = args.sfa + ((int64_t)(ti.sf_row0 / 128) * katoms_total + KA * kb) * 512;
                             bulk_load(st + A_BYTES + C::B_BYTES, sa, sfb, &full_bar[s]);
 #pragma unroll
                             for (int j = 0; j < C::SFB_ATOMS; ++j) {
                                 const int atom = min(ti.n0 / 128 + j, natoms - 1);
                                 const uint8_t* sw = args.sfw +
-                                    (((int64_t)ti.expert * natoms + atom) * katoms_total + 2 * kb) * 512;
+                                    (((int64_t)ti.expert * natoms + atom) * katoms_total + KA * kb) * 512;
                                 bulk_load(st + A_BYTES + C::B_BYTES + C::SFA_BYTES + j * 1024, sw, sfb, &full_bar[s]);
                             }
                         } else {
@@ -205,7 +214,9 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
         uint32_t ph = 0;
         int acc = 0;
         uint32_t acc_ph = 0;
-        constexpr uint32_t IDESC_A = (MODE == MODE_OSC) ? idesc_mxf4(BM, BN) : idesc_e4m3(BM, BN);
+        constexpr uint32_t IDESC_A = (MODE == MODE_OSC)    ? idesc_mxf4(BM, BN)
+                                     : (MODE == MODE_MXF8) ? idesc_mxf8(BM, BN)
+                                                           : idesc_e4m3(BM, BN);
         constexpr uint32_t IDESC_B = idesc_bf16(BM, BN);
         const uint64_t desc_hi = smem_desc_sw128(0);  // everything but the start address
         const uint64_t sf_hi = smem_desc_sf(0);
@@ -249,6 +260,18 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
                     } else if (MODE == MODE_OSC) {
 #pragma unroll
                         for (int k = 0; k < 4; ++k) mma_f16(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC_B, 1u);
+                    } else if (MODE == MODE_MXF8) {
+                        // one 128-channel scale block per stage: four K = 32 instructions, scale byte k of the column
+                        const uint64_t sfa_d = sf_hi | (uint64_t)((sbase + A_BYTES + C::B_BYTES) >> 4);
+                        const uint64_t sfb_d = sf_hi | (uint64_t)((sbase + A_BYTES + C::B_BYTES + C::SFA_BYTES) >> 4);
+                        tc_copy_sf(tmem_base + C::TM_SFA, sfa_d);
+#pragma unroll
+                        for (int j = 0; j < C::SFB_ATOMS; ++j)
+                            tc_copy_sf(tmem_base + C::TM_SFB + j * 4, sfb_d + (uint64_t)(j * 64));
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)
+                            mma_mxf8(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC_A | idesc_sf_ids(k, k), tmem_base + C::TM_SFA,
+                                     sfb_tm, (kb | k) ? 1u : 0u);
                     } else {
 #pragma unroll
                         for (int k = 0; k < 4; ++k)
@@ -434,6 +457,14 @@ cudaError_t launch_gemm_fp8(const GemmArgs& a, int bn, cudaStream_t st) {
         case 128: return launch_cfg<MODE_FP8, 128>(a, st);
         case 192: return launch_cfg<MODE_FP8, 192>(a, st);
         default: return launch_cfg<MODE_FP8, 256>(a, st);
+    }
+}
+cudaError_t launch_gemm_mxf8(const GemmArgs& a, int bn, cudaStream_t st) {
+    switch (bn) {
+        case 64: return launch_cfg<MODE_MXF8, 64>(a, st);
+        case 128: return launch_cfg<MODE_MXF8, 128>(a, st);
+        case 192: return launch_cfg<MODE_MXF8, 192>(a, st);
+        default: return launch_cfg<MODE_MXF8, 256>(a, st);
     }
 }
 

@@ -52,6 +52,21 @@ def test_mxfp8_linear_small(B, oracle, M, K, N):
     assert torch.equal(Y2[:, :N], Y) and torch.isnan(Y2[:, N:].float()).all()
 
 
+@pytest.mark.parametrize("N", [64, 9600, 19200, 28672])
+def test_mxfp8_128_row_tiles_all_widths(B, oracle, N):
+    """Up to 128 rows the dense MXFP8 GEMM runs on the 128-row-tile kernel; with one row tile its cost model takes
+    64-, 128-, 192- and 256-column tiles for these four N (the narrowest width whose tiles still fit in one wave)."""
+    M, K = 100, 256
+    c = synth.fp8_linear_case(N, M, K, N)
+    w = B.osc_mxfp8_prepare_weights(dev_bf16(c["W"]))
+    ws = poison(B.osc_mxfp8_act_sizes(w, M).workspace_bytes)
+    Y = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+    B.osc_mxfp8_linear(w, dev_bf16(c["X"]), Y, ws)
+    B.osc_sync_check()
+    Yref, T, *_ = oracle.mxfp8_linear(c["X"], c["W"])
+    assert_within_tolerance(host_f64(Y), Yref, T, f"mxfp8 128-row tiles N={N}")
+
+
 def test_mxfp8_quantizer_edge_values(B, oracle):
     """Ties, saturation, signed zeros, subnormal results, tiny and huge groups, all-zero groups, strided input."""
     rng = np.random.default_rng(11)
