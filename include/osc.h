@@ -39,15 +39,15 @@
  * the NVFP4 / G = 16 form of the OSC path, the dynamic-protection control group of Section 4.2 (a measured
  * baseline), offline profiling (Algorithm 1), and osc_linear_static (a deployment aid).
  *
- * Kernel selection is internal and depends only on the shape: few rows (M <= 32, or <= 64 for layers with
- * more 128-feature tiles than SMs or a long K loop) run on a weight-streaming kernel with the operands swapped
+ * Kernel selection is internal and depends only on the shape: few rows (M <= 32; <= 64 for layers with
+ * more 128-feature tiles than SMs or a long K loop; <= 256 for long K loops with few tiles) run on a weight-streaming kernel with the operands swapped
  * and K split over a thread-block cluster; grouped problems with large experts and dense problems with many
  * tiles on 256-row CTA-pair tiles; the rest (up to 128 rows, small experts, and dense problems whose 128-row
  * tiles fit in one wave and beat the pair kernel's estimate) on 128-row tiles.  Results of different kernels for
  * the same inputs agree within
  * the accumulation-order rounding of fp32, not bit for bit; one kernel is deterministic run to run.
  * Environment variables for experiments (read by the library, not part of the contract): OSC_DECODE (0 = never,
- * 2 = always up to 64 rows), OSC_DECODE_SPLIT, OSC_PAIR (0 = 128-row tiles only, 2 = pair tiles whenever eligible), OSC_PAIR_BLOCK_N, OSC_BLOCK_N,
+ * 2 = always up to 256 rows), OSC_DECODE_SPLIT, OSC_PAIR (0 = 128-row tiles only, 2 = pair tiles whenever eligible), OSC_PAIR_BLOCK_N, OSC_BLOCK_N,
  * OSC_LOG.
  */
 #ifndef OSC_H_

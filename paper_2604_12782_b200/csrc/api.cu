@@ -140,13 +140,18 @@ static bool use_pair_kernel(bool grouped, int M, int E, long single_ns = 0, long
 // Dense problems with few rows run on the few-row kernel (operands swapped, K split over a cluster): up to 32
 // rows always; up to 64 rows when there are more 128-feature tiles than SMs or the K loop is long (64 stages or
 // more) - measured on B200: with 48 tiles, 20 stages and 64 rows the 128-row-tile kernel is still ahead (11.5 vs
-// 14.4 us), with 32 tiles and 96 stages it is behind (24.4 vs 21.9 us).  OSC_DECODE=0 disables, OSC_DECODE=2 forces
-// it up to 64 rows.
+// 14.4 us), with 32 tiles and 96 stages it is behind (24.4 vs 21.9 us); up to 256 rows (its 256-token form, one
+// CTA per SM) when the K loop is long and the tiles with their K split still fit the machine, where the tile
+// kernels leave most SMs idle.  OSC_DECODE=0 disables, OSC_DECODE=2 forces it up to 256 rows.
 static bool use_decode_kernel(bool grouped, int M, int N, int nkb, int num_sms) {
     const char* e = getenv("OSC_DECODE");   // read per call: tests switch it inside one process
     const int mode = e ? atoi(e) : 1;
-    if (mode == 0 || grouped || M > 64) return false;
-    return mode == 2 || M <= 32 || (N + 127) / 128 >= num_sms || nkb >= 64;
+    if (mode == 0 || grouped || M > 256) return false;
+    if (mode == 2) return true;
+    const int tiles = (N + 127) / 128;
+    if (M <= 32) return true;
+    if (M <= 64) return tiles >= num_sms || nkb >= 64;
+    return nkb >= 64 && 2 * tiles <= num_sms;
 }
 
 // ----------------------------------------------------------------- the table

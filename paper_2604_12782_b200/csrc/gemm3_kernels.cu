@@ -30,26 +30,29 @@ constexpr int MODE_OSC = 0;
 constexpr int MODE_FP8 = 1;
 constexpr int MODE_MXF8 = 2;            // block-scaled FP8 (MXFP8): one 128-channel scale block per stage and operand
 constexpr int BF = 128;                 // output features per CTA = MMA rows = TMEM lanes
-constexpr int MAX_TOK = 64;             // activation rows per call
 constexpr int ROW_BYTES = 128;
 constexpr int W_BYTES = BF * ROW_BYTES;        // 16 KB of weights per stage
-constexpr int X_BYTES = MAX_TOK * ROW_BYTES;   // 8 KB of activations per stage
 constexpr int THREADS = 192;
-constexpr int TMEM_COLS = 128;          // accumulator (<= 64 columns) + scale columns
-constexpr int TM_SFW = 64;              // weight scales: 2 K blocks x 4 columns
-constexpr int TM_SFX = 72;              // activation scales
 constexpr int MAX_CLUSTER = 8;
-constexpr int PSTR = MAX_TOK + 4;       // row stride (floats) of a parked partial tile
 
-template <int MODE>
+// TOK = most activation rows per call: 64 (two CTAs per SM) or 256 (one CTA per SM; for long K loops, where a
+// 128-row-tile kernel would leave most SMs without a tile)
+template <int MODE, int TOK>
 struct Cfg {
     static constexpr bool SCALED = MODE != MODE_FP8;
     static constexpr int KA = (MODE == MODE_OSC) ? 2 : 1;            // 128-channel scale blocks per stage
-    static constexpr int SF_BYTES = SCALED ? 1024 : 0;               // per operand and stage (MXFP8 uses half of it)
-    static constexpr int STAGE_BYTES = W_BYTES + X_BYTES + 2 * SF_BYTES;
-    static constexpr int STAGES = 4;   // ~105 KB per CTA: the CTAs of two consecutive launches share an SM, so the
-                                       // next call's weight loads overlap this call's reduction and stores
-    static constexpr int PARTIAL_BYTES = BF * PSTR * 4;               // aliases the first stages once the MMAs are done
+    static constexpr int XATOMS = (TOK > 128) ? 2 : 1;               // 128-row scale blocks of the activations
+    static constexpr int X_BYTES = TOK * ROW_BYTES;                  // activations per stage
+    static constexpr int SFW_BYTES = SCALED ? 1024 : 0;              // weight scales per stage (MXFP8 uses half of it)
+    static constexpr int SFX_BYTES = SCALED ? XATOMS * 1024 : 0;     // activation scales
+    static constexpr int STAGE_BYTES = W_BYTES + X_BYTES + SFW_BYTES + SFX_BYTES;
+    static constexpr int STAGES = 4;   // TOK = 64: ~105 KB per CTA, the CTAs of two consecutive launches share an SM,
+                                       // so the next call's weight loads overlap this call's reduction and stores
+    static constexpr int CTAS_PER_SM = (TOK <= 64) ? 2 : 1;
+    static constexpr int TM_SFW = TOK;            // TMEM: accumulator (TOK columns), weight scales (2 K blocks x 4
+    static constexpr int TM_SFX = TOK + 8;        // columns), activation scales (2 K blocks x XATOMS x 4 columns)
+    static constexpr int TMEM_COLS = (TOK <= 64) ? 128 : 512;
+    static constexpr int PARTIAL_BYTES = TOK * BF * 4;   // parked partial tile [token][feature], aliases the first stages
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
     static_assert(STAGE_BYTES % 1024 == 0, "stage must keep 1024-byte alignment");
     static_assert(PARTIAL_BYTES <= STAGES * STAGE_BYTES, "partial tile must fit in the ring");
@@ -70,10 +73,11 @@ __device__ __forceinline__ float4 ld_cluster_f32x4(uint32_t cluster_addr) {
     return v;
 }
 
-template <int MODE>
-__global__ void __launch_bounds__(THREADS, 2) gemm_decode_kernel(const __grid_constant__ GemmArgs args) {
-    using C = Cfg<MODE>;
+template <int MODE, int TOK>
+__global__ void __launch_bounds__(THREADS, Cfg<MODE, TOK>::CTAS_PER_SM) gemm_decode_kernel(const __grid_constant__ GemmArgs args) {
+    using C = Cfg<MODE, TOK>;
     constexpr int STAGES = C::STAGES;
+    constexpr int X_BYTES = C::X_BYTES, TM_SFW = C::TM_SFW, TM_SFX = C::TM_SFX, TMEM_COLS = C::TMEM_COLS;
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -118,6 +122,7 @@ __global__ void __launch_bounds__(THREADS, 2) gemm_decode_kernel(const __grid_co
 
     const int N = args.N, K = args.K, M = args.M;
     const int ntok = (M + 15) / 16 * 16;                       // MMA N
+    const int xatoms = (ntok + 127) / 128;                     // 128-row scale blocks the activations span
     const int elems_per_kb = (MODE == MODE_OSC) ? 256 : 128;
     const int nkb_a = (K + elems_per_kb - 1) / elems_per_kb;
     const int nkb_b = (MODE == MODE_OSC) ? args.Kop / 64 : 0;
@@ -127,7 +132,6 @@ __global__ void __launch_bounds__(THREADS, 2) gemm_decode_kernel(const __grid_co
     const int per = (nkb + S - 1) / S;
     const int kb0 = min(nkb, rank * per);
     const int kb1 = min(nkb, kb0 + per);
-    float acc[MAX_TOK];
     const int q = warp & 3;                 // TMEM lane quarter an epilogue warp may read
     const int f = q * 32 + lane;            // my feature inside the tile
     float* partial = reinterpret_cast<float*>(smem);
@@ -137,7 +141,7 @@ __global__ void __launch_bounds__(THREADS, 2) gemm_decode_kernel(const __grid_co
         // weights (and their scales) of the first ring before the dependency wait, activations after it
         auto expect = [&](int kb, int s) {
             uint32_t bytes = W_BYTES + (uint32_t)(ntok * ROW_BYTES);   // the activation tile holds ntok rows
-            if (C::SCALED && kb < nkb_a) bytes += 2u * 512u * (uint32_t)min(C::KA, katoms_total - C::KA * kb);
+            if (C::SCALED && kb < nkb_a) bytes += (uint32_t)(1 + xatoms) * 512u * (uint32_t)min(C::KA, katoms_total - C::KA * kb);
             mbar_arrive_expect_tx(&full_bar[s], bytes);
         };
         auto load_w = [&](int kb, int s) {
@@ -159,8 +163,9 @@ __global__ void __launch_bounds__(THREADS, 2) gemm_decode_kernel(const __grid_co
                 tma_load_2d(st + W_BYTES, &args.tm_a, &full_bar[s], kb * ROW_BYTES, 0);
                 if (C::SCALED) {
                     const int ka = min(C::KA, katoms_total - C::KA * kb);
-                    bulk_load(st + W_BYTES + X_BYTES + C::SF_BYTES, args.sfa + (int64_t)(C::KA * kb) * 512, (uint32_t)ka * 512u,
-                              &full_bar[s]);
+                    for (int j = 0; j < xatoms; ++j)   // 128-row scale blocks of the activations
+                        bulk_load(st + W_BYTES + X_BYTES + C::SFW_BYTES + j * 1024,
+                                  args.sfa + ((int64_t)j * katoms_total + C::KA * kb) * 512, (uint32_t)ka * 512u, &full_bar[s]);
                 }
             } else {
                 tma_load_2d(st + W_BYTES, &args.tm_ao, &full_bar[s], (kb - nkb_a) * 64, 0);
@@ -213,12 +218,15 @@ __global__ void __launch_bounds__(THREADS, 2) gemm_decode_kernel(const __grid_co
                 if (MODE == MODE_OSC && kb < nkb_a) {
                     const int ka = min(2, katoms_total - 2 * kb);
                     const uint64_t sfw_d = sf_hi | (uint64_t)((sbase + W_BYTES + X_BYTES) >> 4);
-                    const uint64_t sfx_d = sf_hi | (uint64_t)((sbase + W_BYTES + X_BYTES + C::SF_BYTES) >> 4);
+                    const uint64_t sfx_d = sf_hi | (uint64_t)((sbase + W_BYTES + X_BYTES + C::SFW_BYTES) >> 4);
 #pragma unroll
                     for (int a = 0; a < 2; ++a) {
                         if (a < ka) {
                             tc_copy_sf(tmem_base + TM_SFW + a * 4, sfw_d + (uint64_t)(a * 32));
-                            tc_copy_sf(tmem_base + TM_SFX + a * 4, sfx_d + (uint64_t)(a * 32));
+#pragma unroll
+                            for (int j = 0; j < C::XATOMS; ++j)
+                                if (j < xatoms)
+                                    tc_copy_sf(tmem_base + TM_SFX + a * (C::XATOMS * 4) + j * 4, sfx_d + (uint64_t)(j * 64 + a * 32));
                         }
                     }
 #pragma unroll
@@ -226,15 +234,17 @@ __global__ void __launch_bounds__(THREADS, 2) gemm_decode_kernel(const __grid_co
                         if (k < 2 * ka) {
                             constexpr uint32_t SFID[2] = {idesc_sf_ids(0, 0), idesc_sf_ids(2, 2)};
                             mma_mxf4(tmem_base, wdesc + 2 * k, xdesc + 2 * k, idesc_a | SFID[k & 1],
-                                     tmem_base + TM_SFW + (k >> 1) * 4, tmem_base + TM_SFX + (k >> 1) * 4,
+                                     tmem_base + TM_SFW + (k >> 1) * 4, tmem_base + TM_SFX + (k >> 1) * (C::XATOMS * 4),
                                      (first | (uint32_t)k) ? 1u : 0u);
                         }
                     }
                 } else if (MODE == MODE_MXF8) {
                     const uint64_t sfw_d = sf_hi | (uint64_t)((sbase + W_BYTES + X_BYTES) >> 4);
-                    const uint64_t sfx_d = sf_hi | (uint64_t)((sbase + W_BYTES + X_BYTES + C::SF_BYTES) >> 4);
+                    const uint64_t sfx_d = sf_hi | (uint64_t)((sbase + W_BYTES + X_BYTES + C::SFW_BYTES) >> 4);
                     tc_copy_sf(tmem_base + TM_SFW, sfw_d);
-                    tc_copy_sf(tmem_base + TM_SFX, sfx_d);
+#pragma unroll
+                    for (int j = 0; j < C::XATOMS; ++j)
+                        if (j < xatoms) tc_copy_sf(tmem_base + TM_SFX + j * 4, sfx_d + (uint64_t)(j * 64));
 #pragma unroll
                     for (int k = 0; k < 4; ++k)
                         mma_mxf8(tmem_base, wdesc + 2 * k, xdesc + 2 * k, idesc_a | idesc_sf_ids(k, k), tmem_base + TM_SFW,
@@ -259,92 +269,99 @@ __global__ void __launch_bounds__(THREADS, 2) gemm_decode_kernel(const __grid_co
 
 done:
     // ------------------------------------------------------------------ reduction + epilogue
-    // Every CTA of the cluster parks its partial tile as fp32 [feature][token] (row stride PSTR floats,
-    // conflict-free for 16-byte accesses) in its own shared memory: the ring is free once the accumulator
-    // is complete.  After a cluster barrier CTA r sums, in rank order, the four-token chunks c = r, r+S, ...
-    // of all partials through distributed shared memory and stores those tokens' outputs.
+    // Every CTA of the cluster parks its partial tile as fp32 [token][feature] in its own shared memory (the ring
+    // is free once the accumulator is complete).  After a cluster barrier CTA r sums, in rank order, the tokens
+    // r, r+S, ... of all partials through distributed shared memory - a warp reads one token's 128 features as
+    // one contiguous 512-byte row per peer - and stores four features per lane (8 bytes, 256 per warp and token).
+    // (With the tile parked as [feature][token] every lane of a remote load hit a different row: the reduction
+    // of a 256-token tile took ~15 us.)
     if (warp >= 2) {
         bool have = kb1 > kb0;
         if (have && !wait_bounded(tfull_bar, 0, abort_flag, 33)) have = false;
         tc_fence_after();
-        if (have) {
-#pragma unroll
-            for (int c = 0; c < MAX_TOK / 16; ++c) {
-                if (c * 16 < ntok) {
-                    uint32_t r[32];
-                    tmem_ld_32x16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * 16), r);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) acc[c * 16 + i] = __uint_as_float(r[i]);
-                }
-            }
-        } else {
-#pragma unroll
-            for (int i = 0; i < MAX_TOK; ++i) acc[i] = 0.0f;
-        }
-        tc_fence_before();
-        if (S > 1) {
-#pragma unroll
-            for (int c = 0; c < MAX_TOK / 4; ++c)
-                if (c * 4 < ntok)
-                    *reinterpret_cast<float4*>(partial + f * PSTR + c * 4) =
-                        make_float4(acc[4 * c], acc[4 * c + 1], acc[4 * c + 2], acc[4 * c + 3]);
-        }
-    }
-    __syncwarp();
-    __syncthreads();
-    if (S > 1) cluster_sync_all();          // partial tiles visible to the whole cluster
-    if (warp >= 2) {
         grid_dependency_wait();             // Y may still be read by an earlier kernel
         const int n = n0 + f;
         float swn = 1.0f;
         if (MODE == MODE_FP8 && n < N) swn = args.sw[n];
-        if (S == 1) {
-            if (n < N) {
+        // sixteen tokens at a time: TMEM -> registers -> the parked partial tile (S > 1) or straight to Y (S == 1)
+        for (int c = 0; c * 16 < ntok; ++c) {
+            uint32_t r[32];   // the load fills r[0..15]
+            if (have) {
+                tmem_ld_32x16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * 16), r);
+                tmem_ld_wait();
+            } else {
 #pragma unroll
-                for (int t = 0; t < MAX_TOK; ++t) {
+                for (int i = 0; i < 16; ++i) r[i] = 0u;
+            }
+            if (S > 1) {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) partial[(c * 16 + i) * BF + f] = __uint_as_float(r[i]);
+            } else if (n < N) {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    const int t = c * 16 + i;
                     if (t < M) {
-                        float v = acc[t];
+                        float v = __uint_as_float(r[i]);
                         if (MODE == MODE_FP8) v = v * (args.sx[t] * swn);
                         args.Y[(int64_t)t * args.ldy + n] = __bfloat16_as_ushort(__float2bfloat16_rn(v));
                     }
                 }
             }
-        } else {
-            const uint32_t mine = smem_u32(partial + f * PSTR);
-            uint32_t peer[MAX_CLUSTER];
+        }
+        tc_fence_before();
+    }
+    __syncwarp();
+    __syncthreads();
+    if (S > 1) cluster_sync_all();          // partial tiles visible to the whole cluster
+    if (warp >= 2 && S > 1) {
+        const int wq = warp - 2;
+        const int n4 = n0 + 4 * lane;           // my four features
+        float4 sw4 = make_float4(1.0f, 1.0f, 1.0f, 1.0f);
+        if (MODE == MODE_FP8 && n4 < N) sw4 = *reinterpret_cast<const float4*>(args.sw + n4);
+        const uint32_t mine = smem_u32(partial) + (uint32_t)(lane * 16);
+        uint32_t peer[MAX_CLUSTER];
 #pragma unroll
-            for (int r = 0; r < MAX_CLUSTER; ++r) peer[r] = map_to_cta(mine, (uint32_t)min(r, S - 1));
-            // two chunks per pass: the distributed-shared-memory loads of both (2 S round trips' worth) are in flight together
-            for (int c0 = rank; c0 * 4 < ntok; c0 += 2 * S) {
-                float4 p[2][MAX_CLUSTER];
+        for (int r = 0; r < MAX_CLUSTER; ++r) peer[r] = map_to_cta(mine, (uint32_t)min(r, S - 1));
+        // tokens rank, rank + S, ...; the four warps take them in turn, four tokens per pass and four peers at a
+        // time (in rank order), so that up to sixteen remote loads per lane are in flight together
+        for (int j = wq; rank + S * j < M; j += 16) {
+            float4 v[4];
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    const int c = c0 + h * S;
+            for (int r0 = 0; r0 < MAX_CLUSTER; r0 += 4) {
+                if (r0 < S) {
+                    float4 p[4][4];
 #pragma unroll
-                    for (int r = 0; r < MAX_CLUSTER; ++r)
-                        if (r < S && c * 4 < ntok) p[h][r] = ld_cluster_f32x4(peer[r] + (uint32_t)(c * 16));
-                }
+                    for (int h = 0; h < 4; ++h) {
+                        const int t = rank + S * (j + 4 * h);
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    const int c = c0 + h * S;
-                    if (c * 4 >= ntok) break;
-                    float4 v = p[h][0];
+                        for (int r = 0; r < 4; ++r)
+                            if (r0 + r < S && t < M) p[h][r] = ld_cluster_f32x4(peer[r0 + r] + (uint32_t)(t * (BF * 4)));
+                    }
 #pragma unroll
-                    for (int r = 1; r < MAX_CLUSTER; ++r)
-                        if (r < S) { v.x += p[h][r].x; v.y += p[h][r].y; v.z += p[h][r].z; v.w += p[h][r].w; }
-                    if (n < N) {
-                        const float o[4] = {v.x, v.y, v.z, v.w};
+                    for (int h = 0; h < 4; ++h) {
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const int t = 4 * c + i;
-                            if (t < M) {
-                                float y = o[i];
-                                if (MODE == MODE_FP8) y = y * (args.sx[t] * swn);
-                                args.Y[(int64_t)t * args.ldy + n] = __bfloat16_as_ushort(__float2bfloat16_rn(y));
+                        for (int r = 0; r < 4; ++r) {
+                            if (r0 + r < S) {
+                                if (r0 + r == 0) v[h] = p[h][r];
+                                else { v[h].x += p[h][r].x; v[h].y += p[h][r].y; v[h].z += p[h][r].z; v[h].w += p[h][r].w; }
                             }
                         }
                     }
+                }
+            }
+#pragma unroll
+            for (int h = 0; h < 4; ++h) {
+                const int t = rank + S * (j + 4 * h);
+                if (t >= M) break;
+                float4 o = v[h];
+                if (MODE == MODE_FP8) {
+                    const float sxt = args.sx[t];
+                    o.x *= sxt * sw4.x; o.y *= sxt * sw4.y; o.z *= sxt * sw4.z; o.w *= sxt * sw4.w;
+                }
+                if (n4 < N) {
+                    const __nv_bfloat162 lo = __floats2bfloat162_rn(o.x, o.y), hi = __floats2bfloat162_rn(o.z, o.w);
+                    *reinterpret_cast<uint2*>(args.Y + (int64_t)t * args.ldy + n4) =
+                        make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
                 }
             }
         }
@@ -359,12 +376,12 @@ done:
     }
 }
 
-template <int MODE>
+template <int MODE, int TOK>
 static cudaError_t launch_cfg(const GemmArgs& a, int S, cudaStream_t st) {
-    using C = Cfg<MODE>;
+    using C = Cfg<MODE, TOK>;
     static bool configured = false;
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_decode_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(gemm_decode_kernel<MODE, TOK>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              C::SMEM_BYTES);
         if (e != cudaSuccess) return e;
         configured = true;
@@ -384,7 +401,7 @@ static cudaError_t launch_cfg(const GemmArgs& a, int S, cudaStream_t st) {
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, gemm_decode_kernel<MODE>, a);
+    return cudaLaunchKernelEx(&cfg, gemm_decode_kernel<MODE, TOK>, a);
 }
 
 }  // namespace decode
@@ -413,13 +430,13 @@ int gemm_decode_split(int N, int nkb, int num_sms) {
 }
 
 cudaError_t launch_gemm_dual_decode(const GemmArgs& a, int S, cudaStream_t st) {
-    return decode::launch_cfg<decode::MODE_OSC>(a, S, st);
+    return a.M <= 64 ? decode::launch_cfg<decode::MODE_OSC, 64>(a, S, st) : decode::launch_cfg<decode::MODE_OSC, 256>(a, S, st);
 }
 cudaError_t launch_gemm_mxf8_decode(const GemmArgs& a, int S, cudaStream_t st) {
-    return decode::launch_cfg<decode::MODE_MXF8>(a, S, st);
+    return a.M <= 64 ? decode::launch_cfg<decode::MODE_MXF8, 64>(a, S, st) : decode::launch_cfg<decode::MODE_MXF8, 256>(a, S, st);
 }
 cudaError_t launch_gemm_fp8_decode(const GemmArgs& a, int S, cudaStream_t st) {
-    return decode::launch_cfg<decode::MODE_FP8>(a, S, st);
+    return a.M <= 64 ? decode::launch_cfg<decode::MODE_FP8, 64>(a, S, st) : decode::launch_cfg<decode::MODE_FP8, 256>(a, S, st);
 }
 
 }  // namespace osc

@@ -1,6 +1,7 @@
-"""Few-row kernel (M <= 64: operands swapped, K split over a thread-block cluster) against the oracle.
+"""Few-row kernel (operands swapped, K split over a thread-block cluster; a 64-row and a 256-row form) against
+the oracle.
 
-The library routes to it by itself for few rows; here OSC_DECODE=2 forces it for every M <= 64 and
+The library routes to it by itself for few rows; here OSC_DECODE=2 forces it for every M <= 256 and
 OSC_DECODE_SPLIT forces cluster sizes (1 = no reduction, up to 8), so that every reduction path, ranks whose
 K slice holds only Path-B blocks, odd numbers of 128-channel scale blocks, feature tiles cut by N and token
 counts that are not multiples of 16 are all covered.  OSC_DECODE=0 keeps the 128-row-tile kernel covered
@@ -59,6 +60,9 @@ CASES = [  # M, K, N, table, split (None = the library's choice)
     (64, 1024, 448, "one", 4), (48, 2048, 256, "two", 8), (5, 256, 128, "empty", 1), (64, 128, 64, "full", 2),
     (31, 1536, 1024, "one", 5), (64, 4096, 512, "two", None), (20, 4096, 384, "two", 3), (64, 3072, 256, "one", 5),
     (32, 4096, 128, "two", 7),
+    # the 256-row form: one and two 128-row scale blocks of activations, token counts off the multiples of 16
+    (65, 512, 192, "two", None), (128, 1024, 256, "one", 2), (129, 384, 320, "two", 3), (200, 2048, 128, "one", 4),
+    (256, 640, 448, "two", 1), (250, 4096, 64, "two", 8), (144, 256, 128, "empty", 2), (256, 128, 64, "full", 2),
 ]
 
 
@@ -90,7 +94,9 @@ def test_decode_kernel_osc(B, oracle, env, M, K, N, kind, split):
 
 
 @pytest.mark.parametrize("M,K,N,split", [(1, 128, 64, None), (16, 768, 320, 3), (40, 1536, 1024, 4), (64, 12288, 256, 8),
-                                         (64, 256, 192, 2), (9, 4096, 128, 1)])
+                                         (64, 256, 192, 2), (9, 4096, 128, 1),
+                                         (65, 768, 192, None), (128, 8192, 256, 4), (200, 1536, 320, 3), (256, 12288, 128, 8),
+                                         (255, 128, 64, 1)])
 def test_decode_kernel_fp8(B, oracle, env, M, K, N, split):
     c = synth.fp8_linear_case(M + K, M, K, N)
     Yref, T, (x8, sx), _ = oracle.fp8_linear(c["X"], c["W"])
@@ -123,7 +129,9 @@ def test_decode_kernel_is_deterministic(B, env):
 
 
 @pytest.mark.parametrize("M,K,N,split", [(1, 128, 64, None), (16, 768, 320, 3), (40, 1536, 1024, 4), (64, 12288, 256, 8),
-                                         (33, 384, 192, 2)])
+                                         (33, 384, 192, 2),
+                                         (65, 768, 192, None), (128, 8192, 256, 4), (129, 1536, 320, 3), (256, 12288, 128, 8),
+                                         (250, 128, 64, 1)])
 def test_decode_kernel_mxfp8(B, oracle, env, M, K, N, split):
     c = synth.fp8_linear_case(M + K + 1, M, K, N)
     Yref, T, (x8, sfa), _ = oracle.mxfp8_linear(c["X"], c["W"])
