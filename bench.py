@@ -372,7 +372,7 @@ def run_gpu(args):
     # Rows are independent, so the step is cut into row chunks and pipelined over three streams: upload of chunk
     # c+1, osc_linear on chunk c and download of chunk c-1 overlap (PCIe is full duplex; the link, not the GPU,
     # bounds this number).  Every chunk goes through the same public call with its own slice of the workspace.
-    CH = 4
+    CH = 8
     rows_c = (M + CH - 1) // CH
     s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
     sz_c = B.osc_act_sizes(prob.w[0], rows_c)
