@@ -550,6 +550,28 @@ def run_sweep(args):
         del p, Xn
         torch.cuda.empty_cache()
 
+    def profile_row(name, S, K, seed=0):
+        """Algorithm 1 (offline): threshold of Eq. 1 over the slice, per-token per-group vote, table and Eq. 2-4 counters.
+        Two passes over the activations (the threshold needs the whole slice first): 2 x 2 bytes per element."""
+        if not want(name):
+            return
+        Xb, _ = synth.osc_activations_only(seed, S, K, 1)
+        X0 = dev_bf16(torch, Xb)
+        n = NSETS
+        Xs = [X0 if i == 0 else torch.roll(X0, 97 * i, 0).contiguous() for i in range(n)]
+        scratch = torch.empty(B.osc_profile_scratch_bytes(K), dtype=torch.uint8, device="cuda")
+        lut = torch.empty(K // 32, dtype=torch.int8, device="cuda")
+        nh, nt = (torch.empty(K // 32, dtype=torch.int32, device="cuda") for _ in range(2))
+        tb = torch.empty(1, dtype=torch.int32, device="cuda")
+        ms = time_loop(torch, lambda i: B.osc_profile_lut(Xs[i % n], 5.0, scratch, lut, nh, nt, tb), steps, warm)
+        B.osc_sync_check()
+        byts = 2 * 2.0 * S * K
+        rows.append({"name": name, "M": S, "K": K, "ms": ms, "gbs": byts / ms / 1e6,
+                     "frac_hbm": byts / (ms * 1e-3) / peaks["hbm"], "roof_us": byts / peaks["hbm"] * 1e6,
+                     "pct_roofline": 100 * byts / peaks["hbm"] / (ms * 1e-3)})
+        del Xs
+        torch.cuda.empty_cache()
+
     def fp8_row(name, M, K, N, seed=0):
         if not want(name):
             return
@@ -649,6 +671,7 @@ def run_sweep(args):
         mxfp8_row("down_mxfp8", M, 12288, 4096)
     rms_row("qkv.rmsnorm_fused", 8192, 4096, 6144, 2)
     rms_row("qkv.rmsnorm_fused", 2048, 4096, 6144, 2)
+    profile_row("profile.algorithm1", 8192, 4096)
     nvfp4_row("qkv.nvfp4_g16", 8192, 4096, 6144)
     nvfp4_row("qkv.nvfp4_g16", 2048, 4096, 6144)
     dyn_row("qkv.dynamic_protection", 8192, 4096, 6144, 2)
