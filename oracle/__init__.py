@@ -14,6 +14,7 @@ Function-to-paper map (details in the C file):
   nvfp4_quantize_extract / nvfp4_gemm / nvfp4_linear         the NVFP4 / G = 16 variant (efficiency table, G = 16)
   threshold / profile_indexing / clustering_density   Eq. 1-4, Algorithm 1 (offline profiling)
   rmsnorm (oracle/rmsnorm.py)          the normalization in front of Algorithm 2 when the two are fused (Section 3.3)
+  swiglu / silu32 / exp32              the activation in front of the FP8 quantizer of the down projection (Sections 3.3, 3.4)
 """
 from __future__ import annotations
 
@@ -378,6 +379,29 @@ def clustering_density(n_hit: np.ndarray, n_total: np.ndarray):
     """Eq. 4 and the block mean: C_k = n_hit/n_total (0 for groups without outlier tokens), mean over all K groups."""
     c = np.where(n_total > 0, n_hit / np.maximum(n_total, 1), 0.0)
     return c, float(c.mean())
+
+
+def exp32(z: float) -> float:
+    """The fp32 exponential the SwiGLU definition uses (see the C file)."""
+    f = lib().osc_ref_exp32
+    f.restype, f.argtypes = C.c_float, [C.c_float]
+    return float(f(C.c_float(z)))
+
+
+def silu32(g: float) -> float:
+    f = lib().osc_ref_silu32
+    f.restype, f.argtypes = C.c_float, [C.c_float]
+    return float(f(C.c_float(g)))
+
+
+def swiglu(GU: np.ndarray, I: int) -> np.ndarray:
+    """GU [M, >= 2I] bf16 bits (gate columns [0, I), up columns [I, 2I)) -> h = bf16(silu32(gate) * up) [M, I]."""
+    GU = np.ascontiguousarray(GU, dtype=np.uint16)
+    M = GU.shape[0]
+    H = np.zeros((M, I), np.uint16)
+    rc = lib().osc_ref_swiglu(_p(GU), C.c_int64(GU.shape[1]), M, I, _p(H))
+    assert rc == 0
+    return H
 
 
 from .rmsnorm import f64_to_bf16_bits, rmsnorm  # noqa: E402,F401

@@ -655,6 +655,55 @@ int osc_ref_mxfp8_gemm_rows(const uint8_t* x8, const uint8_t* sfa, const int32_t
 
 /* ------------------------------------------- offline profiling (Section 2, Algorithm 1) */
 
+/* ---- SwiGLU in front of the per-token FP8 quantizer (the producer of the down projection's input; Section 3.3
+ * places the quantizer directly behind the operator that produces the activations, Section 3.4 makes that
+ * quantizer FP8 for this input).  The paper does not give the activation's arithmetic; it is fixed here in
+ * fp32, every step an IEEE operation, so that the FP8 codes that follow are decided on identical values:
+ *
+ *   exp32(z):  t = fl32(z * LOG2E);  t > 127.4 -> +inf;  t < -64 -> 0 (1 + e is then 1 anyway);
+ *              n = rint(t) (ties to even), f = t - n (exact), p = Horner with fused multiply-adds of the
+ *              degree-6 Taylor polynomial of 2^f on [-1/2, 1/2]; e = p * 2^n (exact scaling)
+ *   silu32(g) = fl32( g / fl32(1 + exp32(-g)) )
+ *   h = bf16( fl32( silu32(g) * u ) )        g = GU[m][i], u = GU[m][I + i]
+ */
+static const float OSC_EXP2_C[7] = {1.0f, 0.693147182f, 0.240226507f, 0.0555041087f, 0.00961812911f,
+                                    0.00133335581f, 0.000154035304f};
+float osc_ref_exp32(float z) {
+    volatile float t = z * 1.44269502f;
+    if (t != t) return t;
+    if (t > 127.4f) return INFINITY;
+    if (t < -64.0f) return 0.0f;
+    float n = rintf(t);
+    float f = t - n;
+    float p = OSC_EXP2_C[6];
+    for (int i = 5; i >= 0; --i) p = fmaf(p, f, OSC_EXP2_C[i]);
+    return ldexpf(p, (int)n);
+}
+float osc_ref_silu32(float g) {
+    volatile float d = 1.0f + osc_ref_exp32(-g);
+    volatile float s = g / d;
+    return s;
+}
+static uint16_t bf16_from_float_rne(float v) {
+    uint32_t u;
+    memcpy(&u, &v, 4);
+    if ((u & 0x7FFFFFFFu) > 0x7F800000u) return 0x7FFF; /* NaN */
+    return (uint16_t)((u + 0x7FFFu + ((u >> 16) & 1u)) >> 16);
+}
+int osc_ref_swiglu(const uint16_t* GU, int64_t ldg, int M, int I, uint16_t* H) {
+#pragma omp parallel for schedule(static)
+    for (int m = 0; m < M; ++m) {
+        const uint16_t* row = GU + (int64_t)m * ldg;
+        for (int i = 0; i < I; ++i) {
+            float g = (float)bf16_value(row[i]), u = (float)bf16_value(row[I + i]);
+            volatile float hv = osc_ref_silu32(g) * u;
+            H[(int64_t)m * I + i] = bf16_from_float_rne(hv);
+        }
+    }
+    return 0;
+}
+
+
 /* Eq. 1: layer-wise threshold T_l = alpha * mean |x| over the S x H calibration activations. */
 double osc_ref_threshold(const uint16_t* X, int64_t ldx, int S, int H, double alpha) {
     double sum = 0.0;
