@@ -572,6 +572,58 @@ def run_sweep(args):
         del Xs
         torch.cuda.empty_cache()
 
+    def swiglu_row(name, M, I, N, seed=0):
+        """SwiGLU in front of the FP8 down projection: fused into the per-token quantizer against the two-step path (own
+        SwiGLU kernel writing bf16, then the stand-alone FP8 quantizer)."""
+        if not want(name):
+            return
+        rng = np.random.default_rng(seed)
+        case = synth.fp8_linear_case(seed, 1, I, N)
+        n = NSETS
+        GU0 = dev_bf16(torch, synth.f32_to_bf16_bits(np.concatenate(
+            [rng.standard_normal((M, I), dtype=np.float32) * 3.0, rng.standard_normal((M, I), dtype=np.float32)], axis=1)))
+        GUs = [GU0 if i == 0 else torch.roll(GU0, 97 * i, 0).contiguous() for i in range(n)]
+        W0 = dev_bf16(torch, case["W"])
+        ws_ = [B.osc_fp8_prepare_weights(W0 if i == 0 else torch.roll(W0, 61 * i, 0).contiguous()) for i in range(n)]
+        sz = B.osc_fp8_act_sizes(ws_[0], M)
+        wk = [torch.empty(sz.workspace_bytes, dtype=torch.uint8, device="cuda") for _ in range(n)]
+        Hs = [torch.empty(M, I, dtype=torch.bfloat16, device="cuda") for _ in range(n)]
+        Ys = [torch.empty(M, N, dtype=torch.bfloat16, device="cuda") for _ in range(n)]
+
+        def fused_q(i):
+            j = i % n
+            B.osc_swiglu_fp8_quantize(GUs[j], I, wk[j][sz.x8_offset:], wk[j][sz.sx_offset:])
+
+        def act_only(i):
+            j = i % n
+            B.osc_swiglu(GUs[j], I, Hs[j])
+
+        def two_step_q(i):
+            j = i % n
+            B.osc_swiglu(GUs[j], I, Hs[j])
+            B.osc_fp8_quantize(Hs[j], wk[j][sz.x8_offset:], wk[j][sz.sx_offset:])
+
+        def fused_lin(i):
+            j = i % n
+            B.osc_swiglu_fp8_linear(ws_[j], GUs[j], Ys[j], wk[j])
+
+        def two_step_lin(i):
+            j = i % n
+            B.osc_swiglu(GUs[j], I, Hs[j])
+            B.osc_fp8_linear(ws_[j], Hs[j], Ys[j], wk[j])
+
+        t = {k: time_loop(torch, f, steps, warm) for k, f in
+             (("fused_quant_ms", fused_q), ("swiglu_ms", act_only), ("two_step_quant_ms", two_step_q),
+              ("fused_linear_ms", fused_lin), ("two_step_linear_ms", two_step_lin))}
+        B.osc_sync_check()
+        byts = 2.0 * M * 2 * I + 1.0 * M * I + 4.0 * M     # gate and up read once, codes and scales written
+        rows.append({"name": name, "M": M, "K": I, "N": N, **t, "ms": t["fused_linear_ms"],
+                     "fused_quant_gbs": byts / t["fused_quant_ms"] / 1e6,
+                     "fused_quant_frac_hbm": byts / (t["fused_quant_ms"] * 1e-3) / peaks["hbm"],
+                     "speedup_linear": t["two_step_linear_ms"] / t["fused_linear_ms"]})
+        del GUs, ws_, wk, Hs, Ys
+        torch.cuda.empty_cache()
+
     def fp8_row(name, M, K, N, seed=0):
         if not want(name):
             return
@@ -671,6 +723,8 @@ def run_sweep(args):
         mxfp8_row("down_mxfp8", M, 12288, 4096)
     rms_row("qkv.rmsnorm_fused", 8192, 4096, 6144, 2)
     rms_row("qkv.rmsnorm_fused", 2048, 4096, 6144, 2)
+    swiglu_row("down.swiglu_fused", 8192, 12288, 4096)
+    swiglu_row("down.swiglu_fused", 2048, 12288, 4096)
     profile_row("profile.algorithm1", 8192, 4096)
     nvfp4_row("qkv.nvfp4_g16", 8192, 4096, 6144)
     nvfp4_row("qkv.nvfp4_g16", 2048, 4096, 6144)

@@ -247,6 +247,26 @@ osc_status osc_fp8_linear_grouped(const osc_fp8_weights* w, const void* X_perm, 
                                   int M_total, int64_t ldx, void* Y, int64_t ldy, void* workspace,
                                   size_t workspace_bytes, void* stream);
 
+/* ---- SwiGLU fused in front of the per-token FP8 quantizer ---------------------------------------------
+ * The producer of the down projection's input (Section 3.3 places the quantizer behind the operator that
+ * produces the activations; Section 3.4 makes it FP8 for this input):
+ *
+ *   h[m,i] = bf16( silu(GU[m,i]) * GU[m,I+i] ),   silu(g) = g * (1 / (1 + exp32(-g)))
+ *
+ * in fp32, every step an IEEE operation (two multiplications and one reciprocal in silu): exp32(z) takes
+ * t = z * log2(e) clamped to [-64, 126], n = rint(t), f = t - n, the degree-5 Taylor polynomial of 2^f by fused
+ * multiply-adds, times 2^n.  The
+ * per-token quantizer then works on the bf16 row h as osc_fp8_quantize does.
+ *   GU  dev bf16 [M, ldg]: gate columns [0, I), up columns [I, 2I); ldg >= 2I, multiple of 8, 16-byte aligned.
+ *   I   multiple of 128, <= 16384 (a row of h is held in registers), else OSC_ERR_SHAPE.
+ * osc_swiglu writes h itself (dev bf16 [M, ldh]): the unfused reference point.  osc_swiglu_fp8_quantize's
+ * outputs equal osc_fp8_quantize's on osc_swiglu's h bit for bit.  osc_swiglu_fp8_linear (dense weights with
+ * K = I) = osc_swiglu_fp8_quantize + osc_fp8_gemm through the workspace of osc_fp8_act_sizes. */
+osc_status osc_swiglu(const void* GU, int M, int I, int64_t ldg, void* H, int64_t ldh, void* stream);
+osc_status osc_swiglu_fp8_quantize(const void* GU, int M, int I, int64_t ldg, void* x8, void* sx, void* stream);
+osc_status osc_swiglu_fp8_linear(const osc_fp8_weights* w, const void* GU, int M, int64_t ldg, void* Y, int64_t ldy,
+                                 void* workspace, size_t workspace_bytes, void* stream);
+
 /* ------------------------------------- MXFP8 form of the fallback (Section 3.4) */
 
 /* Section 3.4 allows "FP8 (or equivalent 8-bit micro-scaling formats)" for the W2 inputs and Section 4

@@ -660,28 +660,27 @@ int osc_ref_mxfp8_gemm_rows(const uint8_t* x8, const uint8_t* sfa, const int32_t
  * quantizer FP8 for this input).  The paper does not give the activation's arithmetic; it is fixed here in
  * fp32, every step an IEEE operation, so that the FP8 codes that follow are decided on identical values:
  *
- *   exp32(z):  t = fl32(z * LOG2E);  t > 127.4 -> +inf;  t < -64 -> 0 (1 + e is then 1 anyway);
+ *   exp32(z):  t = fl32(z * LOG2E) clamped to [-64, 126] (beyond, 1 + e is 1 or the quotient g / (1 + e) is
+ *              below 1e-35 in magnitude: nothing a bf16 product with u can show);
  *              n = rint(t) (ties to even), f = t - n (exact), p = Horner with fused multiply-adds of the
- *              degree-6 Taylor polynomial of 2^f on [-1/2, 1/2]; e = p * 2^n (exact scaling)
- *   silu32(g) = fl32( g / fl32(1 + exp32(-g)) )
+ *              degree-5 Taylor polynomial of 2^f on [-1/2, 1/2]; e = p * 2^n (exact scaling)
+ *   silu32(g) = fl32( g * fl32( 1 / fl32(1 + exp32(-g)) ) )
  *   h = bf16( fl32( silu32(g) * u ) )        g = GU[m][i], u = GU[m][I + i]
  */
-static const float OSC_EXP2_C[7] = {1.0f, 0.693147182f, 0.240226507f, 0.0555041087f, 0.00961812911f,
-                                    0.00133335581f, 0.000154035304f};
+static const float OSC_EXP2_C[6] = {1.0f, 0.693147182f, 0.240226507f, 0.0555041097f, 0.00961812865f, 0.00133335579f};
 float osc_ref_exp32(float z) {
     volatile float t = z * 1.44269502f;
-    if (t != t) return t;
-    if (t > 127.4f) return INFINITY;
-    if (t < -64.0f) return 0.0f;
+    t = fminf(fmaxf(t, -64.0f), 126.0f); /* a NaN argument ends at -64: the NaN reaches the result through g itself */
     float n = rintf(t);
     float f = t - n;
-    float p = OSC_EXP2_C[6];
-    for (int i = 5; i >= 0; --i) p = fmaf(p, f, OSC_EXP2_C[i]);
+    float p = OSC_EXP2_C[5];
+    for (int i = 4; i >= 0; --i) p = fmaf(p, f, OSC_EXP2_C[i]);
     return ldexpf(p, (int)n);
 }
 float osc_ref_silu32(float g) {
     volatile float d = 1.0f + osc_ref_exp32(-g);
-    volatile float s = g / d;
+    volatile float r = 1.0f / d;
+    volatile float s = g * r;
     return s;
 }
 static uint16_t bf16_from_float_rne(float v) {

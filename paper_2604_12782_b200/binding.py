@@ -77,6 +77,9 @@ _SIGS = {
     "osc_linear_static": (_i, [_vp, _vp, _i, _i64, _vp, _i64, _vp]),
     "osc_linear_grouped": (_i, [_vp, _vp, _vp, _i, _i64, _vp, _i64, _vp, _sz, _vp]),
     "osc_rmsnorm": (_i, [_vp, _i, _i, _i64, _vp, C.c_float, _vp, _i64, _vp]),
+    "osc_swiglu": (_i, [_vp, _i, _i, _i64, _vp, _i64, _vp]),
+    "osc_swiglu_fp8_quantize": (_i, [_vp, _i, _i, _i64, _vp, _vp, _vp]),
+    "osc_swiglu_fp8_linear": (_i, [_vp, _vp, _i, _i64, _vp, _i64, _vp, _sz, _vp]),
     "osc_rmsnorm_quantize_extract": (_i, [_vp, _vp, _i, _i64, _vp, C.c_float, _vp, _vp, _vp, _vp]),
     "osc_rmsnorm_linear": (_i, [_vp, _vp, _i, _i64, _vp, C.c_float, _vp, _i64, _vp, _sz, _vp]),
     "osc_profile_scratch_bytes": (_i, [_i, C.POINTER(_sz)]),
@@ -285,6 +288,25 @@ def osc_rmsnorm_linear(w: OscWeights, H: torch.Tensor, gamma: torch.Tensor, eps:
     _check(_lib.osc_rmsnorm_linear(w.ptr, _ptr(H), M, H.stride(0) if M else w.K, _ptr(gamma), float(eps), _ptr(Y),
                                    Y.stride(0) if M else w.N, _ptr(workspace),
                                    workspace.numel() * workspace.element_size(), _stream(stream)))
+
+
+def osc_swiglu(GU: torch.Tensor, I: int, H: torch.Tensor, stream=None):
+    """H = bf16(silu(GU[:, :I]) * GU[:, I:2I]) in the library's fixed fp32 arithmetic: the unfused reference point."""
+    M = GU.shape[0]
+    _check(_lib.osc_swiglu(_ptr(GU), M, I, GU.stride(0) if M else 2 * I, _ptr(H), H.stride(0) if M else I, _stream(stream)))
+
+
+def osc_swiglu_fp8_quantize(GU: torch.Tensor, I: int, x8, sx, stream=None):
+    """SwiGLU fused in front of the per-token FP8 quantizer: the activation h is never written."""
+    M = GU.shape[0]
+    _check(_lib.osc_swiglu_fp8_quantize(_ptr(GU), M, I, GU.stride(0) if M else 2 * I, _ptr(x8), _ptr(sx), _stream(stream)))
+
+
+def osc_swiglu_fp8_linear(w: "Fp8Weights", GU: torch.Tensor, Y: torch.Tensor, workspace: torch.Tensor, stream=None):
+    M = GU.shape[0]
+    _check(_lib.osc_swiglu_fp8_linear(w.ptr, _ptr(GU), M, GU.stride(0) if M else 2 * w.K, _ptr(Y),
+                                      Y.stride(0) if M else w.N, _ptr(workspace),
+                                      workspace.numel() * workspace.element_size(), _stream(stream)))
 
 
 def osc_linear_grouped(w: OscWeights, X: torch.Tensor, off: torch.Tensor, Y: torch.Tensor, workspace: torch.Tensor,

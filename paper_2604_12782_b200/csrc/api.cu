@@ -820,6 +820,55 @@ osc_status osc_fp8_linear_grouped(const osc_fp8_weights* w, const void* X_perm, 
     return fp8_linear_impl(w, X_perm, off, M_total, ldx, Y, ldy, workspace, workspace_bytes, stream);
 }
 
+// ---- SwiGLU fused in front of the per-token FP8 quantizer
+static osc_status check_swiglu(const void* GU, int M, int I, int64_t ldg) {
+    if (M < 0) return fail(OSC_ERR_INVALID_ARG, "M = %d is negative", M);
+    if (I <= 0 || I % 128) return fail(OSC_ERR_SHAPE, "I = %d must be a positive multiple of 128", I);
+    if (I > 16384) return fail(OSC_ERR_SHAPE, "I = %d: the fused SwiGLU holds a row in registers, I <= 16384", I);
+    if (M > 0 && !GU) return fail(OSC_ERR_INVALID_ARG, "GU is null");
+    if (ldg < 2 * (int64_t)I) return fail(OSC_ERR_SHAPE, "ldg = %lld < 2 I = %d", (long long)ldg, 2 * I);
+    if (ldg % 8 || !aligned16(GU)) return fail(OSC_ERR_ALIGN, "GU must be 16-byte aligned and ldg a multiple of 8");
+    return OSC_OK;
+}
+
+osc_status osc_swiglu(const void* GU, int M, int I, int64_t ldg, void* H, int64_t ldh, void* stream) {
+    if (osc_status s = check_swiglu(GU, M, I, ldg)) return s;
+    if (M == 0) return OSC_OK;
+    if (!H) return fail(OSC_ERR_INVALID_ARG, "H is null");
+    if (ldh < I) return fail(OSC_ERR_SHAPE, "ldh = %lld < I = %d", (long long)ldh, I);
+    if (ldh % 8 || !aligned16(H)) return fail(OSC_ERR_ALIGN, "H must be 16-byte aligned and ldh a multiple of 8");
+    cudaError_t e = launch_swiglu_fp8(false, GU, ldg, M, I, H, ldh, nullptr, nullptr, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(e, "swiglu_fp8_kernel(activation only)");
+    return OSC_OK;
+}
+
+osc_status osc_swiglu_fp8_quantize(const void* GU, int M, int I, int64_t ldg, void* x8, void* sx, void* stream) {
+    if (osc_status s = check_swiglu(GU, M, I, ldg)) return s;
+    if (M == 0) return OSC_OK;
+    if (!x8 || !sx) return fail(OSC_ERR_INVALID_ARG, "null output pointer");
+    if (!aligned16(x8) || !aligned16(sx)) return fail(OSC_ERR_ALIGN, "outputs must be 16-byte aligned");
+    cudaError_t e = launch_swiglu_fp8(true, GU, ldg, M, I, nullptr, 0, x8, sx, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(e, "swiglu_fp8_kernel");
+    return OSC_OK;
+}
+
+osc_status osc_swiglu_fp8_linear(const osc_fp8_weights* w, const void* GU, int M, int64_t ldg, void* Y, int64_t ldy,
+                                 void* workspace, size_t workspace_bytes, void* stream) {
+    if (!w) return fail(OSC_ERR_INVALID_ARG, "weights handle is null");
+    if (w->grouped) return fail(OSC_ERR_INVALID_ARG, "grouped weights are not supported by the fused SwiGLU");
+    if (osc_status s = check_swiglu(GU, M, w->K, ldg)) return s;
+    if (M == 0) return OSC_OK;
+    osc_fp8_act_sizes_t sz;
+    osc_fp8_act_sizes(w, M, &sz);
+    if (!workspace || !aligned16(workspace)) return fail(OSC_ERR_ALIGN, "workspace must be non-null and 16-byte aligned");
+    if (workspace_bytes < sz.workspace_bytes)
+        return fail(OSC_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", workspace_bytes, sz.workspace_bytes);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    if (osc_status s = osc_swiglu_fp8_quantize(GU, M, w->K, ldg, ws + sz.x8_offset, ws + sz.sx_offset, stream)) return s;
+    return fp8_gemm_impl(w, ws + sz.x8_offset, ws + sz.sx_offset, M, Y, ldy, nullptr, 0, nullptr, 0,
+                         static_cast<cudaStream_t>(stream));
+}
+
 // ------------------------------------------------- MXFP8 form of the fallback
 
 osc_status osc_mxfp8_weight_sizes(int E, int N, int K, osc_mxfp8_weight_sizes_t* out) {

@@ -46,6 +46,9 @@ cudaError_t launch_rmsnorm_quant(bool quant, const void* H, int64_t ldh, int M, 
                                  void* Xn, int64_t ldx, const int32_t* idx_o, void* xq, void* sf,
                                  void* xo, int Ko, int Kop, cudaStream_t st);
 
+cudaError_t launch_swiglu_fp8(bool quant, const void* GU, int64_t ldg, int M, int I, void* Hout, int64_t ldh, void* x8,
+                              void* sx, cudaStream_t st);
+
 // profile_kernels.cu
 cudaError_t launch_profile(const void* X, int64_t ldx, int S, int K, double alpha, double* sum, int32_t* counts,
                            int8_t* lut, int32_t* n_hit, int32_t* n_total, uint32_t* threshold_bits, int num_sms,

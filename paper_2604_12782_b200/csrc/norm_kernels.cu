@@ -1,3 +1,5 @@
+// Producers fused with the quantizer that follows them: RMSNorm + Algorithm 2 (below), SwiGLU + per-token FP8 (end of file).
+//
 // RMSNorm fused in front of Algorithm 2 (Section 3.3 puts the OSC quantizer directly behind the operator that
 // produces the activations; in a decoder layer that operator is the RMSNorm in front of the QKV and gate/up
 // projections).  One pass over the residual stream instead of three (norm read + norm write + quantizer read).
@@ -191,6 +193,121 @@ cudaError_t launch_rmsnorm_quant(bool quant, const void* H, int64_t ldh, int M, 
     return launch_pdl(rmsnorm_quant_kernel<false>, grid, block, smem, st, static_cast<const uint16_t*>(H), ldh, M, M_pad, K,
                       static_cast<const uint16_t*>(gamma), eps, static_cast<uint16_t*>(Xn), ldx, idx_o,
                       static_cast<uint8_t*>(xq), static_cast<uint8_t*>(sf), static_cast<uint16_t*>(xo), Ko, Kop);
+}
+
+// ------------------------------------------------------------------ SwiGLU + per-token FP8
+// The producer of the down projection's input fused with its quantizer (Section 3.3 puts the quantizer behind the
+// producing operator; Section 3.4 makes it FP8 for this input): h = bf16(silu(gate) * up) is never written, the row
+// goes from the gate/up projection's output straight to E4M3 codes and a per-row scale.  Arithmetic (fp32, every
+// step an IEEE operation, so the codes are decided on identical values on every implementation):
+//   exp32(z): t = z * log2(e) clamped to [-64, 126]; n = rint(t), f = t - n, p = degree-5 Taylor polynomial of 2^f
+//             by fused multiply-adds, e = p * 2^n
+//   silu(g) = g * (1 / (1 + exp32(-g)));  h = bf16(silu(g) * u)
+// then amax' = max(amax, 2^-40), scale = amax'/448, codes = E4M3(h * (448/amax')) as in fp8_quant_kernel.
+// One CTA per row, the bf16 row h held in registers between the amax pass and the encode pass (I <= 16384).
+// The kernel is bound by instruction issue (ncu: issue slots 76 % busy at 47 instructions per element in a first
+// version with three range checks, a full division and a degree-6 polynomial), which is why the arithmetic above
+// is as lean as a reproducible definition allows.
+__device__ __forceinline__ float exp32(float z) {
+    const float t = fminf(fmaxf(__fmul_rn(z, 1.44269502f), -64.0f), 126.0f);   // NaN -> -64 (g itself carries the NaN on)
+    // n = rint(t), nearest with ties to even: adding 1.5 * 2^23 rounds t to an integer in the last mantissa bits
+    // (|t| < 2^22), and the integer can be read off the bit pattern; two additions instead of two conversions,
+    // which run at a quarter of the rate
+    const float tn = __fadd_rn(t, 12582912.0f);
+    const float n = __fsub_rn(tn, 12582912.0f);
+    const int ni = __float_as_int(tn) - 0x4B400000;
+    const float f = __fsub_rn(t, n);
+    float p = 0.00133335579f;
+    p = __fmaf_rn(p, f, 0.00961812865f);
+    p = __fmaf_rn(p, f, 0.0555041097f);
+    p = __fmaf_rn(p, f, 0.240226507f);
+    p = __fmaf_rn(p, f, 0.693147182f);
+    p = __fmaf_rn(p, f, 1.0f);
+    return __fmul_rn(p, __int_as_float((ni + 127) << 23));   // exact: -64 <= n <= 126 and p < 1.5
+}
+__device__ __forceinline__ float swiglu32(float g, float u) {
+    const float d = __fadd_rn(1.0f, exp32(-g));
+    return __fmul_rn(__fmul_rn(g, __frcp_rn(d)), u);
+}
+
+constexpr int SG_THREADS = 256;
+constexpr int SG_MAXCH = 8;   // 16-byte chunks of h per thread: I <= 256 x 8 x 8
+
+template <bool QUANT>
+__global__ void __launch_bounds__(SG_THREADS)
+swiglu_fp8_kernel(const uint16_t* __restrict__ GU, int64_t ldg, int M, int I, uint16_t* __restrict__ Hout, int64_t ldh,
+                  uint8_t* __restrict__ x8, float* __restrict__ sx) {
+    __shared__ float s_red[SG_THREADS / 32];
+    grid_launch_dependents();
+    grid_dependency_wait();
+    const int r = blockIdx.x;
+    const int tid = threadIdx.x;
+    const uint4* grow = reinterpret_cast<const uint4*>(GU + (int64_t)r * ldg);
+    const uint4* urow = reinterpret_cast<const uint4*>(GU + (int64_t)r * ldg + I);
+    const int nch = I / 8;
+
+    uint4 h[SG_MAXCH];
+    __nv_bfloat162 am2 = as_bf162(0u);
+#pragma unroll
+    for (int i = 0; i < SG_MAXCH; ++i) {
+        const int c = tid + i * SG_THREADS;
+        h[i] = make_uint4(0u, 0u, 0u, 0u);
+        if (c < nch) {
+            const uint4 g4 = grow[c], u4 = urow[c];
+            const uint32_t gw[4] = {g4.x, g4.y, g4.z, g4.w}, uw[4] = {u4.x, u4.y, u4.z, u4.w};
+            uint32_t o[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const float lo = swiglu32(__uint_as_float(gw[j] << 16), __uint_as_float(uw[j] << 16));
+                const float hi = swiglu32(__uint_as_float(gw[j] & 0xFFFF0000u), __uint_as_float(uw[j] & 0xFFFF0000u));
+                o[j] = bf162_bits(__floats2bfloat162_rn(lo, hi));
+            }
+            h[i] = make_uint4(o[0], o[1], o[2], o[3]);
+            if (QUANT) {   // packed bf16 magnitudes, two at a time
+                const __nv_bfloat162 m2 = __hmax2(__hmax2(__habs2(as_bf162(o[0])), __habs2(as_bf162(o[1]))),
+                                                  __hmax2(__habs2(as_bf162(o[2])), __habs2(as_bf162(o[3]))));
+                am2 = __hmax2(am2, m2);
+            }
+            if (!QUANT) *reinterpret_cast<uint4*>(Hout + (int64_t)r * ldh + c * 8) = h[i];
+        }
+    }
+    if (!QUANT) return;
+    uint32_t am = max(bf162_bits(am2) & 0xFFFFu, bf162_bits(am2) >> 16);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) am = max(am, __shfl_xor_sync(0xFFFFFFFFu, am, o));
+    if ((tid & 31) == 0) s_red[tid >> 5] = __uint_as_float(am << 16);
+    __syncthreads();
+    float amax = s_red[0];
+#pragma unroll
+    for (int i = 1; i < SG_THREADS / 32; ++i) amax = fmaxf(amax, s_red[i]);
+    const float amaxp = fmaxf(amax, __uint_as_float((uint32_t)(127 - 40) << 23));
+    const float scale = __fdiv_rn(amaxp, 448.0f);
+    const float inv = __fdiv_rn(448.0f, amaxp);
+    if (tid == 0) sx[r] = scale;
+    uint8_t* orow = x8 + (int64_t)r * I;
+#pragma unroll
+    for (int i = 0; i < SG_MAXCH; ++i) {
+        const int c = tid + i * SG_THREADS;
+        if (c < nch) {
+            const uint32_t w[4] = {h[i].x, h[i].y, h[i].z, h[i].w};
+            uint32_t e[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                e[j] = e4m3x2(__fmul_rn(__uint_as_float(w[j] << 16), inv), __fmul_rn(__uint_as_float(w[j] & 0xFFFF0000u), inv)) & 0xFFFFu;
+            *reinterpret_cast<uint2*>(orow + c * 8) = make_uint2(e[0] | (e[1] << 16), e[2] | (e[3] << 16));
+        }
+    }
+}
+
+// quant: Hout unused; else x8 / sx unused.  I <= 16384, a multiple of 8.
+cudaError_t launch_swiglu_fp8(bool quant, const void* GU, int64_t ldg, int M, int I, void* Hout, int64_t ldh, void* x8,
+                              void* sx, cudaStream_t st) {
+    if (M <= 0) return cudaSuccess;
+    if (quant)
+        return launch_pdl(swiglu_fp8_kernel<true>, dim3(M), dim3(SG_THREADS), 0, st, static_cast<const uint16_t*>(GU), ldg, M, I,
+                          static_cast<uint16_t*>(Hout), ldh, static_cast<uint8_t*>(x8), static_cast<float*>(sx));
+    return launch_pdl(swiglu_fp8_kernel<false>, dim3(M), dim3(SG_THREADS), 0, st, static_cast<const uint16_t*>(GU), ldg, M, I,
+                      static_cast<uint16_t*>(Hout), ldh, static_cast<uint8_t*>(x8), static_cast<float*>(sx));
 }
 
 }  // namespace osc

@@ -18,23 +18,24 @@ def bits(a):
 
 def test_exp32_against_the_library_exponential(oracle):
     worst = 0.0
-    for z in np.linspace(-44.0, 88.0, 20001):
+    for z in np.linspace(-44.0, 87.0, 20001):   # t = z log2(e) inside the clamp [-64, 126]
         z = float(np.float32(z))
         worst = max(worst, abs(oracle.exp32(z) - math.exp(z)) / math.exp(z))
-    assert worst < 5e-6                      # the product z * log2(e) is rounded to fp32: ~2^-24 * |t| absolute in t
-    for z in np.linspace(-1.0, 1.0, 2001):   # small arguments: a few fp32 units (degree-6 truncation ~1.2e-7 + roundings)
+    assert worst < 8e-6                      # z * log2(e) rounded to fp32 (~2^-24 |t| absolute in t) + the degree-5 truncation (2.4e-6)
+    for z in np.linspace(-1.0, 1.0, 2001):   # small arguments: the truncation error of the polynomial dominates
         z = float(np.float32(z))
-        assert abs(oracle.exp32(z) - math.exp(z)) <= 4 * 2.0 ** -24 * math.exp(z)
+        assert abs(oracle.exp32(z) - math.exp(z)) <= 3.5e-6 * math.exp(z)
     assert oracle.exp32(0.0) == 1.0
     assert oracle.exp32(1.0) == float(np.float32(math.e)) or abs(oracle.exp32(1.0) - math.e) < 3e-7
-    assert oracle.exp32(89.0) == math.inf and oracle.exp32(-50.0) == 0.0
+    assert oracle.exp32(200.0) == oracle.exp32(126.0 / 1.4426950408889634 + 1.0)      # clamped at 2^126
+    assert 0.0 < oracle.exp32(-200.0) <= 2.0 ** -64 * 1.0001                            # and at 2^-64
 
 
 def test_silu32_special_values_and_identity(oracle):
     assert oracle.silu32(0.0) == 0.0
     for g in (45.0, 100.0, float(np.float32(3e30))):   # exp(-g) is dropped: silu(g) = g exactly
         assert oracle.silu32(g) == g
-    assert oracle.silu32(-100.0) == 0.0 and math.copysign(1.0, oracle.silu32(-100.0)) == -1.0
+    assert -2e-36 < oracle.silu32(-100.0) < 0.0          # -100 / (1 + 2^126): far below anything bf16 h can show
     for g in np.linspace(0.01, 30.0, 500):
         g = float(np.float32(g))
         assert abs(oracle.silu32(g) - g / (1.0 + math.exp(-g))) <= 6e-6 * g
