@@ -234,7 +234,7 @@ constexpr int SG_THREADS = 256;
 constexpr int SG_MAXCH = 8;   // 16-byte chunks of h per thread: I <= 256 x 8 x 8
 
 template <bool QUANT>
-__global__ void __launch_bounds__(SG_THREADS)
+__global__ void __launch_bounds__(SG_THREADS, 5)
 swiglu_fp8_kernel(const uint16_t* __restrict__ GU, int64_t ldg, int M, int I, uint16_t* __restrict__ Hout, int64_t ldh,
                   uint8_t* __restrict__ x8, float* __restrict__ sx) {
     __shared__ float s_red[SG_THREADS / 32];
