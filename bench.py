@@ -759,6 +759,42 @@ def run_sweep(args):
         del parts, qkv, opj, gup, dwn
         torch.cuda.empty_cache()
 
+    # the same layer with its producers: RMSNorm in front of QKV and gate/up, SwiGLU between gate/up and down (the down
+    # projection really consumes the gate/up output); fused into the quantizers against separate kernels
+    if want("layer.fused"):
+        M, eps = 4096, 1e-6
+        qkv = OscProblem(torch, B, synth.osc_linear_case(0, M, 4096, 6144, 2), 2)
+        opj = OscProblem(torch, B, synth.osc_linear_case(1, M, 4096, 4096, 1), 2)
+        gup = OscProblem(torch, B, synth.osc_linear_case(2, M, 4096, 24576, 1), 2)
+        dwn = Fp8Problem(torch, B, synth.fp8_linear_case(3, M, 12288, 4096), 2)
+        gam = dev_bf16(torch, synth.f32_to_bf16_bits(np.random.default_rng(0).uniform(0.5, 1.5, 4096).astype(np.float32)))
+        Xn = torch.empty(M, 4096, dtype=torch.bfloat16, device="cuda")
+        Hh = torch.empty(M, 12288, dtype=torch.bfloat16, device="cuda")
+
+        def fused(i):
+            j = i % 2
+            B.osc_rmsnorm_linear(qkv.w[j], qkv.X[j], gam, eps, qkv.Y[j], qkv.ws[j])
+            B.osc_linear(opj.w[j], opj.X[j], opj.Y[j], opj.ws[j])
+            B.osc_rmsnorm_linear(gup.w[j], gup.X[j], gam, eps, gup.Y[j], gup.ws[j])
+            B.osc_swiglu_fp8_linear(dwn.w[j], gup.Y[j], dwn.Y[j], dwn.ws[j])
+
+        def separate(i):
+            j = i % 2
+            B.osc_rmsnorm(qkv.X[j], gam, eps, Xn)
+            B.osc_linear(qkv.w[j], Xn, qkv.Y[j], qkv.ws[j])
+            B.osc_linear(opj.w[j], opj.X[j], opj.Y[j], opj.ws[j])
+            B.osc_rmsnorm(gup.X[j], gam, eps, Xn)
+            B.osc_linear(gup.w[j], Xn, gup.Y[j], gup.ws[j])
+            B.osc_swiglu(gup.Y[j], 12288, Hh)
+            B.osc_fp8_linear(dwn.w[j], Hh, dwn.Y[j], dwn.ws[j])
+
+        ms_f, ms_s = time_loop(torch, fused, steps, warm), time_loop(torch, separate, steps, warm)
+        B.osc_sync_check()
+        rows.append({"name": "layer.fused(rmsnorm+qkv,o_proj,rmsnorm+gate_up,swiglu+down_fp8)", "M": M, "ms": ms_f,
+                     "separate_kernels_ms": ms_s, "speedup": ms_s / ms_f})
+        del qkv, opj, gup, dwn, Xn, Hh
+        torch.cuda.empty_cache()
+
     # MoE: 128 experts, top-8 of 8192 tokens, Zipf(1.1) load
     counts = synth.zipf_expert_rows()
     E = counts.size
