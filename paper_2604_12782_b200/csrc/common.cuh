@@ -26,6 +26,28 @@ static cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
+// Function attributes (the shared-memory opt-in) and occupancy answers belong to a device, not to the process:
+// every kernel instantiation keeps one of these and sets itself up once on each device it is launched on.
+constexpr int kMaxDevicesPerProcess = 64;
+struct PerDevice {
+    bool done[kMaxDevicesPerProcess] = {};
+    int value[kMaxDevicesPerProcess] = {};
+};
+// index of the current device in a PerDevice, or -1 (no caching) if it cannot be had or is out of range
+static inline int per_device_slot() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevicesPerProcess) return -1;
+    return dev;
+}
+template <typename Kernel>
+static cudaError_t opt_in_shared_memory(PerDevice& pd, Kernel kernel, int bytes) {
+    const int slot = per_device_slot();
+    if (slot >= 0 && pd.done[slot]) return cudaSuccess;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess && slot >= 0) pd.done[slot] = true;
+    return e;
+}
+
 // quant_kernels.cu
 cudaError_t launch_quant_extract(const CUtensorMap& tm_x, int M, int K, const uint32_t* mask,
                                  const int32_t* prefix, const int32_t* idx_o, void* xq, void* sf, void* xo, int Ko, int Kop,

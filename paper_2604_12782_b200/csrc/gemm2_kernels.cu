@@ -527,13 +527,8 @@ done:
 template <int MODE, int BN>
 static cudaError_t launch_cfg(const GemmArgs& a, cudaStream_t st) {
     using C = Cfg<MODE, BN>;
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_pair_kernel<MODE, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             C::SMEM_BYTES);
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
+    static PerDevice configured, resident;
+    if (cudaError_t e = opt_in_shared_memory(configured, gemm_pair_kernel<MODE, BN>, C::SMEM_BYTES)) return e;
     const int total = a.sched2 ? a.num_sms : ((a.M + 2 * BM - 1) / (2 * BM)) * ((a.N + BN - 1) / BN);
     if (total <= 0) return cudaSuccess;
     cudaLaunchConfig_t cfg = {};
@@ -551,13 +546,15 @@ static cudaError_t launch_cfg(const GemmArgs& a, cudaStream_t st) {
     cfg.numAttrs = 2;
     // The kernel is persistent with static striping of tiles over pairs, so every pair must be
     // resident at once: ask how many 2-CTA clusters of this footprint the device can hold.
-    static int max_pairs = 0;
+    const int slot = per_device_slot();
+    int max_pairs = (slot >= 0 && resident.done[slot]) ? resident.value[slot] : 0;
     if (max_pairs == 0) {
         cfg.gridDim = dim3(a.num_sms);
         int n = 0;
         cudaError_t e = cudaOccupancyMaxActiveClusters(&n, gemm_pair_kernel<MODE, BN>, &cfg);
         if (e != cudaSuccess) return e;
         max_pairs = n > 0 ? n : 1;
+        if (slot >= 0) { resident.value[slot] = max_pairs; resident.done[slot] = true; }
         if (getenv("OSC_LOG")) fprintf(stderr, "[osc] pair kernel BN=%d: %d resident clusters of 2\n", BN, max_pairs);
     }
     int pairs = a.num_sms / 2;

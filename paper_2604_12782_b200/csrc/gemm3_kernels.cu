@@ -379,13 +379,8 @@ done:
 template <int MODE, int TOK>
 static cudaError_t launch_cfg(const GemmArgs& a, int S, cudaStream_t st) {
     using C = Cfg<MODE, TOK>;
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_decode_kernel<MODE, TOK>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             C::SMEM_BYTES);
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
+    static PerDevice configured;
+    if (cudaError_t e = opt_in_shared_memory(configured, gemm_decode_kernel<MODE, TOK>, C::SMEM_BYTES)) return e;
     const int tiles = (a.N + BF - 1) / BF;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(tiles * S);

@@ -427,13 +427,8 @@ int gemm_block_n(int row_tiles, int N, int num_sms, long* cost_ns) {
 template <int MODE, int BN>
 static cudaError_t launch_cfg(const GemmArgs& a, cudaStream_t st) {
     using C = Cfg<MODE, BN>;
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_kernel<MODE, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             C::SMEM_BYTES);
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
+    static PerDevice configured;
+    if (cudaError_t e = opt_in_shared_memory(configured, gemm_kernel<MODE, BN>, C::SMEM_BYTES)) return e;
     int grid = a.num_sms;
     if (!a.sched) {
         const int total = ((a.M + BM - 1) / BM) * ((a.N + BN - 1) / BN);

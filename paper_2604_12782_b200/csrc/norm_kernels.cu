@@ -178,14 +178,9 @@ cudaError_t launch_rmsnorm_quant(bool quant, const void* H, int64_t ldh, int M, 
     const int M_pad = quant ? (M + 127) / 128 * 128 : M;
     const dim3 grid((M_pad + RN_WARPS - 1) / RN_WARPS), block(32 * RN_WARPS);
     const size_t smem = (size_t)RN_WARPS * K * 2 + RN_WARPS * 16;
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(rmsnorm_quant_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, RN_WARPS * 8192 * 2 + RN_WARPS * 16);
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(rmsnorm_quant_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, RN_WARPS * 8192 * 2 + RN_WARPS * 16);
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
+    static PerDevice configured_q, configured_n;
+    if (cudaError_t e = opt_in_shared_memory(configured_q, rmsnorm_quant_kernel<true>, RN_WARPS * 8192 * 2 + RN_WARPS * 16)) return e;
+    if (cudaError_t e = opt_in_shared_memory(configured_n, rmsnorm_quant_kernel<false>, RN_WARPS * 8192 * 2 + RN_WARPS * 16)) return e;
     if (quant)
         return launch_pdl(rmsnorm_quant_kernel<true>, grid, block, smem, st, static_cast<const uint16_t*>(H), ldh, M, M_pad, K,
                           static_cast<const uint16_t*>(gamma), eps, static_cast<uint16_t*>(Xn), ldx, idx_o,

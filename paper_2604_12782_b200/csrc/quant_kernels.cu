@@ -693,12 +693,8 @@ static cudaError_t launch_quant_extract_fmt(const CUtensorMap& tm_x, int M, int 
                                             int tensor_e, cudaStream_t st) {
     const int tiles = (sched ? max_tiles : (M + QE_ROWS - 1) / QE_ROWS) * (K / QE_COLS);
     if (tiles <= 0) return cudaSuccess;
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(quant_extract_kernel<FMT>, cudaFuncAttributeMaxDynamicSharedMemorySize, QE_SMEM);
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
+    static PerDevice configured;
+    if (cudaError_t e = opt_in_shared_memory(configured, quant_extract_kernel<FMT>, QE_SMEM)) return e;
     const int grid = tiles < QE_CTAS_PER_SM * num_sms ? tiles : QE_CTAS_PER_SM * num_sms;
     return launch_pdl(quant_extract_kernel<FMT>, dim3(grid), dim3(QE_THREADS), QE_SMEM, st, tm_x, M, K, mask, prefix,
                       idx_o, static_cast<uint8_t*>(xq), static_cast<uint8_t*>(sf), static_cast<uint16_t*>(xo), Ko, Kop,
