@@ -955,7 +955,8 @@ osc_status osc_mxfp8_act_sizes(const osc_mxfp8_weights* w, int M, osc_mxfp8_act_
 }
 
 static osc_status mxfp8_gemm_impl(const osc_mxfp8_weights* w, const void* x8, const void* sfa, int M, void* Y,
-                                  int64_t ldy, const int32_t* sched2, int max_tiles, int max_tiles2, void* stream) {
+                                  int64_t ldy, const int32_t* sched, const int32_t* sched2, int max_tiles, int max_tiles2,
+                                  void* stream) {
     if (M == 0) return OSC_OK;
     if (!x8 || !sfa || !Y) return fail(OSC_ERR_INVALID_ARG, "null device pointer");
     if (ldy < w->N) return fail(OSC_ERR_SHAPE, "ldy = %lld < N = %d", (long long)ldy, w->N);
@@ -978,14 +979,16 @@ static osc_status mxfp8_gemm_impl(const osc_mxfp8_weights* w, const void* x8, co
         return OSC_OK;
     }
     if (osc_status s = make_tmap(&a.tm_a, x8, false, M, w->K, w->K, 128)) return s;
-    // grouped problems run on the CTA-pair kernel (256-row tiles; rows past the end are zero-filled by the loads or
-    // belong to the next expert, and are never stored); dense ones on whichever kernel its cost model puts ahead
-    const long row_tiles = w->grouped ? max_tiles2 - w->E / 2 : (M + 255) / 256;
+    // grouped problems with large experts run on the CTA-pair kernel (256-row tiles; rows past the end are zero-filled by
+    // the loads or belong to the next expert, and are never stored), those with small experts on 128-row tiles; dense
+    // ones on whichever kernel its cost model puts ahead
+    const long row_tiles = w->grouped ? (max_tiles2 > w->E / 2 ? max_tiles2 - w->E / 2 : 1) : (M + 255) / 256;
     long single_ns = 0, pair_ns = 0;
-    const int bn1 = gemm_block_n((M + 127) / 128, w->N, w->num_sms, &single_ns);
+    const int bn1 = gemm_block_n(w->grouped ? max_tiles : (M + 127) / 128, w->N, w->num_sms, &single_ns);
     const int bn = gemm_pair_block_n(false, false, row_tiles, w->N, w->K / 128, w->num_sms, &pair_ns);
-    if (!w->grouped && !use_pair_kernel(false, M, 1, single_ns * (w->K / 128), pair_ns, single_ns <= 470)) {
+    if (!use_pair_kernel(w->grouped, M, w->E, single_ns * (w->K / 128), pair_ns, single_ns <= 470)) {
         a.tm_b = w->tm_b1[bn1 / 64 - 1];
+        a.sched = sched; a.max_tiles = max_tiles;
         a.sfa = static_cast<const uint8_t*>(sfa);
         a.sfw = w->sfw;
         a.Y = static_cast<uint16_t*>(Y);
@@ -1018,7 +1021,7 @@ osc_status osc_mxfp8_gemm(const osc_mxfp8_weights* w, const void* x8, const void
     if (!w) return fail(OSC_ERR_INVALID_ARG, "weights handle is null");
     if (M < 0) return fail(OSC_ERR_INVALID_ARG, "M = %d is negative", M);
     if (w->grouped) return fail(OSC_ERR_INVALID_ARG, "grouped weights: use osc_mxfp8_linear_grouped");
-    return mxfp8_gemm_impl(w, x8, sfa, M, Y, ldy, nullptr, 0, 0, stream);
+    return mxfp8_gemm_impl(w, x8, sfa, M, Y, ldy, nullptr, nullptr, 0, 0, stream);
 }
 
 static osc_status mxfp8_linear_impl(const osc_mxfp8_weights* w, const void* X, const int32_t* off, int M, int64_t ldx,
@@ -1047,7 +1050,7 @@ static osc_status mxfp8_linear_impl(const osc_mxfp8_weights* w, const void* X, c
     }
     if (osc_status s = mxfp8_quantize_impl(X, M, w->K, ldx, ws + sz.x8_offset, ws + sz.sfa_offset, sched, max_tiles, stream))
         return s;
-    return mxfp8_gemm_impl(w, ws + sz.x8_offset, ws + sz.sfa_offset, M, Y, ldy, sched2, max_tiles, max_tiles2, stream);
+    return mxfp8_gemm_impl(w, ws + sz.x8_offset, ws + sz.sfa_offset, M, Y, ldy, sched, sched2, max_tiles, max_tiles2, stream);
 }
 
 osc_status osc_mxfp8_linear(const osc_mxfp8_weights* w, const void* X, int M, int64_t ldx, void* Y, int64_t ldy,

@@ -169,7 +169,9 @@ def _grouped_check(B, oracle, counts, K, N, seed, sample=None):
     assert not torch.isnan(Y.float()).any()
 
 
-@pytest.mark.parametrize("counts", [np.array([3, 0, 130, 1, 257, 128]), np.array([300, 0, 5, 256, 129, 511, 1, 385])])
+# experts averaging under 96 rows run on 128-row tiles, larger ones on 256-row pair tiles
+@pytest.mark.parametrize("counts", [np.array([3, 0, 130, 1, 257, 128]), np.array([300, 0, 5, 256, 129, 511, 1, 385]),
+                                    np.array([1, 64, 0, 0, 127, 5, 90, 33, 128, 2])])
 def test_mxfp8_grouped_small(B, oracle, counts):
     _grouped_check(B, oracle, counts, 384, 320, 7)
 
