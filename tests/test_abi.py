@@ -80,3 +80,32 @@ def test_null_and_misaligned_arguments_launch_nothing(B):
     assert q(0x1000, 0, 128, 128, None, None, None) == 0          # M == 0 is a no-op
     assert q(0x1000, 4, 128, 132, 0x2000, 0x3000, None) == -4     # ldx not a multiple of 8
     assert lib.osc_linear(None, None, 0, 0, None, 0, None, 0, None) == -1
+
+
+def test_producer_fusions_validate_before_launching(B):
+    """RMSNorm / SwiGLU entry points: shape, range, alignment and null checks come before any device work."""
+    lib = C.CDLL(B.LIB_PATH)
+    rn = lib.osc_rmsnorm
+    rn.argtypes = B._SIGS["osc_rmsnorm"][1]
+    assert rn(0x1000, 4, 100, 128, 0x2000, 1e-6, 0x3000, 128, None) == -2       # K not a multiple of 128
+    assert rn(0x1000, 4, 8320, 8320, 0x2000, 1e-6, 0x3000, 8320, None) == -2    # a row must fit on chip: K <= 8192
+    assert rn(0x1000, -1, 128, 128, 0x2000, 1e-6, 0x3000, 128, None) == -1
+    assert rn(0x1000, 0, 128, 128, None, 1e-6, None, 128, None) == 0            # M == 0 is a no-op
+    assert rn(0x1000, 4, 128, 128, None, 1e-6, 0x3000, 128, None) == -1         # gamma is null
+    assert rn(0x1000, 4, 128, 120, 0x2000, 1e-6, 0x3000, 128, None) == -2       # ldh < K
+    assert rn(0x1008, 4, 128, 128, 0x2000, 1e-6, 0x3000, 128, None) == -4
+    assert rn(0x1000, 4, 128, 132, 0x2000, 1e-6, 0x3000, 128, None) == -4       # ldh not a multiple of 8
+    sg = lib.osc_swiglu
+    sg.argtypes = B._SIGS["osc_swiglu"][1]
+    assert sg(0x1000, 4, 100, 256, 0x2000, 128, None) == -2                     # I not a multiple of 128
+    assert sg(0x1000, 4, 16512, 33024, 0x2000, 16512, None) == -2               # I <= 16384
+    assert sg(0x1000, 4, 128, 200, 0x2000, 128, None) == -2                     # ldg < 2 I
+    assert sg(0x1000, 4, 128, 256, None, 128, None) == -1
+    assert sg(0x1000, 4, 128, 256, 0x2008, 128, None) == -4
+    assert sg(0x1000, 0, 128, 256, None, 128, None) == 0
+    sq = lib.osc_swiglu_fp8_quantize
+    sq.argtypes = B._SIGS["osc_swiglu_fp8_quantize"][1]
+    assert sq(0x1000, 4, 128, 256, None, 0x3000, None) == -1
+    assert sq(0x1000, 4, 128, 256, 0x2004, 0x3000, None) == -4
+    assert lib.osc_rmsnorm_linear(None, None, 0, 0, None, C.c_float(0), None, 0, None, 0, None) == -1
+    assert lib.osc_swiglu_fp8_linear(None, None, 0, 0, None, 0, None, 0, None) == -1
