@@ -129,8 +129,8 @@ def test_fused_equals_two_step_path_byte_for_byte(B, M, K):
         assert torch.equal(u[:n], v[:n])
 
 
-def test_rmsnorm_linear_within_tolerance(B, oracle):
-    M, K, N = 200, 1024, 320
+@pytest.mark.parametrize("M,K,N", [(200, 1024, 320), (24, 4096, 256), (1500, 512, 768)])   # 128-row tiles, few-row kernel, pair tiles
+def test_rmsnorm_linear_within_tolerance(B, oracle, M, K, N):
     rng = np.random.default_rng(9)
     Hb, gb = residual_rows(rng, M, K), gamma_bits(rng, K)
     c = synth.osc_linear_case(3, M, K, N, 2)

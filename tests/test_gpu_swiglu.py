@@ -73,8 +73,8 @@ def test_fused_equals_two_step_path_byte_for_byte(B, M, I):
     assert torch.equal(a8[:M * I], b8[:M * I]) and torch.equal(asx.view(torch.int32), bsx.view(torch.int32))
 
 
-def test_swiglu_fp8_linear_within_tolerance(B, oracle):
-    M, I, N = 200, 1024, 320
+@pytest.mark.parametrize("M,I,N", [(200, 1024, 320), (16, 2048, 256), (1200, 512, 512)])   # 128-row tiles, few-row kernel, pair tiles
+def test_swiglu_fp8_linear_within_tolerance(B, oracle, M, I, N):
     rng = np.random.default_rng(9)
     GUb = gate_up(rng, M, I)
     W = synth.fp8_linear_case(3, 1, I, N)["W"]
