@@ -12,8 +12,8 @@
 // butterfly over the warp), so results are deterministic; against the exactly rounded sum it is off by a few
 // units of the 53rd bit, which changes r only if 1/sqrt(..) lies within ~1e-16 of an fp32 rounding boundary.
 //
-// One warp per row (K <= 8192): lane 0 fetches the row into shared memory with one bulk copy (cp.async.bulk, its
-// own mbarrier per warp); the first pass sums the squares; the second normalizes the row in place (bf16); then the
+// Two warps per row (K <= 8192; named barriers keep the pair in step): one lane fetches the row into shared memory
+// with one bulk copy (cp.async.bulk, one mbarrier per row); the first pass sums the squares; the second normalizes the row in place (bf16); then the
 // flagged channels are copied out through the channel list (lane t takes list entry t: 64-byte coalesced stores
 // into xo) and zeroed in the shared row; last, every lane quantizes whole 32-channel groups as in
 // quant_extract_kernel (amax without shuffles, one 16-byte store of codes, the four scale bytes of a 128-channel
@@ -28,19 +28,30 @@
 
 namespace osc {
 
-constexpr int RN_WARPS = 14;
+constexpr int RN_ROWS = 14;    // rows per CTA (28 rows in flight per SM: 8 KB of shared memory per row at K = 4096)
+constexpr int RN_WPR = 2;      // warps per row: twice the warps to hide latency with, for the same shared memory
+constexpr int RN_TEAM = 32 * RN_WPR;
+constexpr int RN_THREADS = RN_ROWS * RN_TEAM;
+
+// barrier of the two warps of a row (named barriers 1..RN_ROWS; 0 is the CTA's)
+__device__ __forceinline__ void team_sync(int slot) {
+    asm volatile("bar.sync %0, %1;" ::"r"(slot + 1), "r"(RN_TEAM) : "memory");
+}
 
 template <bool QUANT>
-__global__ void __launch_bounds__(32 * RN_WARPS)
+__global__ void __launch_bounds__(RN_THREADS)
 rmsnorm_quant_kernel(const uint16_t* __restrict__ H, int64_t ldh, int M, int M_pad, int K,
                      const uint16_t* __restrict__ gamma, float eps, uint16_t* __restrict__ Xn, int64_t ldx,
                      const int32_t* __restrict__ idx_o, uint8_t* __restrict__ xq,
                      uint8_t* __restrict__ sf, uint16_t* __restrict__ xo, int Ko, int Kop) {
-    extern __shared__ uint4 rn_rows[];   // [RN_WARPS][K / 8], then one mbarrier and one give-up flag per warp
+    // [RN_ROWS][K / 8] rows, then per row: one mbarrier, two partial sums (double), one give-up flag
+    extern __shared__ uint4 rn_rows[];
     grid_launch_dependents();
+    const int slot = threadIdx.x / RN_TEAM;          // my row inside the CTA
+    const int tl = threadIdx.x % RN_TEAM;            // my lane inside the row's team of two warps
     const int lane = threadIdx.x & 31;
-    const int r = blockIdx.x * RN_WARPS + (threadIdx.x >> 5);
-    if (r >= M_pad) return;
+    const int r = blockIdx.x * RN_ROWS + slot;
+    if (r >= M_pad) return;                          // both warps of a team take every exit together
     const int katoms = K / 128;
     // scale word of (row r, 128-channel block a): block (r/128)*katoms + a, word (r%32)*4 + (r%128)/32
     uint32_t* sf_row = QUANT ? reinterpret_cast<uint32_t*>(sf + (size_t)(r / 128) * katoms * 512) + (r & 31) * 4 + ((r & 127) >> 5)
@@ -48,55 +59,63 @@ rmsnorm_quant_kernel(const uint16_t* __restrict__ H, int64_t ldh, int M, int M_p
     if (r >= M) {   // rows that only pad the last 128-row scale block
         grid_dependency_wait();
         if (QUANT)
-            for (int a = lane; a < katoms; a += 32) sf_row[(size_t)a * 128] = 0u;
+            for (int a = tl; a < katoms; a += RN_TEAM) sf_row[(size_t)a * 128] = 0u;
         return;
     }
     const uint4* hrow = reinterpret_cast<const uint4*>(H + (int64_t)r * ldh);
     const uint4* grow = reinterpret_cast<const uint4*>(gamma);
     const int nch = K / 8;   // 16-byte chunks in the row
 
-    const int warp = threadIdx.x >> 5;
-    uint4* row = rn_rows + (size_t)warp * nch;
-    uint64_t* bar = reinterpret_cast<uint64_t*>(rn_rows + (size_t)RN_WARPS * nch) + warp;
-    volatile int* give_up = reinterpret_cast<volatile int*>(reinterpret_cast<uint64_t*>(rn_rows + (size_t)RN_WARPS * nch) + RN_WARPS) + warp;
-    if (lane == 0) {
+    uint4* row = rn_rows + (size_t)slot * nch;
+    uint8_t* tail = reinterpret_cast<uint8_t*>(rn_rows + (size_t)RN_ROWS * nch);
+    uint64_t* bar = reinterpret_cast<uint64_t*>(tail) + slot;
+    double* part = reinterpret_cast<double*>(tail + RN_ROWS * 8) + slot * RN_WPR;
+    volatile int* give_up = reinterpret_cast<volatile int*>(tail + RN_ROWS * 8 + RN_ROWS * RN_WPR * 8) + slot;
+    if (tl == 0) {
         *give_up = 0;
         mbar_init(bar, 1);
         fence_barrier_init();
     }
-    __syncwarp();
+    team_sync(slot);
     grid_dependency_wait();   // H may come from, and the outputs may still be read by, earlier kernels
-    if (lane == 0) {
+    if (tl == 0) {
         mbar_arrive_expect_tx(bar, (uint32_t)K * 2u);
         bulk_load(row, hrow, (uint32_t)K * 2u, bar);
     }
-    __syncwarp();
-    if (!wait_bounded(bar, 0u, give_up, 41)) return;
+    // a wait that gives up has recorded it in the device status word; the team carries on (with whatever the row
+    // buffer holds) so that its barriers below stay matched
+    wait_bounded(bar, 0u, give_up, 41);
 
-    const int nsteps = (nch + 31) / 32;
-    double ss0 = 0.0, ss1 = 0.0;
-#pragma unroll 2
+    // ---- first pass: sum of squares, each warp over every second step of chunks
+    const int nsteps = (nch + RN_TEAM - 1) / RN_TEAM;
+    double ss0 = 0.0, ss1 = 0.0, ss2 = 0.0, ss3 = 0.0;   // four chains: the fp64 pipe's latency is long
+#pragma unroll 4
     for (int i = 0; i < nsteps; ++i) {
-        const int c = i * 32 + lane;
+        const int c = i * RN_TEAM + tl;
         const uint4 v = (c < nch) ? row[c] : make_uint4(0u, 0u, 0u, 0u);
         const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const double a = (double)__uint_as_float(w[j] << 16), b = (double)__uint_as_float(w[j] & 0xFFFF0000u);
-            ss0 = fma(a, a, ss0);
-            ss1 = fma(b, b, ss1);
+        for (int j = 0; j < 4; j += 2) {
+            const double a0 = (double)__uint_as_float(w[j] << 16), b0 = (double)__uint_as_float(w[j] & 0xFFFF0000u);
+            const double a1 = (double)__uint_as_float(w[j + 1] << 16), b1 = (double)__uint_as_float(w[j + 1] & 0xFFFF0000u);
+            ss0 = fma(a0, a0, ss0);
+            ss1 = fma(b0, b0, ss1);
+            ss2 = fma(a1, a1, ss2);
+            ss3 = fma(b1, b1, ss3);
         }
     }
-    double ss = ss0 + ss1;
+    double ss = (ss0 + ss1) + (ss2 + ss3);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xFFFFFFFFu, ss, o);
-    ss = __shfl_sync(0xFFFFFFFFu, ss, 0);   // every lane continues with the same bits
+    if (lane == 0) part[tl >> 5] = ss;
+    team_sync(slot);
+    ss = part[0] + part[1];   // the same two values in the same order in every lane of the team
     const float r32 = (float)(1.0 / sqrt(ss / (double)K + (double)eps));
 
     // ---- second pass: normalize; QUANT: in place in shared memory, else straight to global memory
-#pragma unroll 2
+#pragma unroll 4
     for (int i = 0; i < nsteps; ++i) {
-        const int c = i * 32 + lane;
+        const int c = i * RN_TEAM + tl;
         if (c >= nch) break;
         const uint4 g4 = grow[c], v = row[c];
         const uint32_t gw[4] = {g4.x, g4.y, g4.z, g4.w};
@@ -111,12 +130,12 @@ rmsnorm_quant_kernel(const uint16_t* __restrict__ H, int64_t ldh, int M, int M_p
         else *reinterpret_cast<uint4*>(Xn + (int64_t)r * ldx + c * 8) = make_uint4(w[0], w[1], w[2], w[3]);
     }
     if (!QUANT) return;
-    __syncwarp();
+    team_sync(slot);
 
     // ---- Algorithm 2 on the normalized row.  Back-up and zero-out: entry t of the (ascending) channel list goes to
     // column t of xo; pad columns +0
     uint16_t* row16 = reinterpret_cast<uint16_t*>(row);
-    for (int t = lane; t < Kop; t += 32) {
+    for (int t = tl; t < Kop; t += RN_TEAM) {
         uint16_t e = 0;
         if (t < Ko) {
             const int ch = idx_o[t];
@@ -125,12 +144,12 @@ rmsnorm_quant_kernel(const uint16_t* __restrict__ H, int64_t ldh, int M, int M_p
         }
         xo[(int64_t)r * Kop + t] = e;
     }
-    __syncwarp();
+    team_sync(slot);
 
     // every lane quantizes whole 32-channel groups
     const int ngrp = K / 32;
-    for (int g0 = 0; g0 < ngrp; g0 += 32) {
-        const int g = g0 + lane;
+    for (int g0 = 0; g0 < ngrp; g0 += RN_TEAM) {
+        const int g = g0 + tl;
         const bool in = g < ngrp;   // ngrp is a multiple of 4, so the four lanes of a scale word are in or out together
         uint32_t w[16];
 #pragma unroll
@@ -176,11 +195,12 @@ cudaError_t launch_rmsnorm_quant(bool quant, const void* H, int64_t ldh, int M, 
                                  void* xo, int Ko, int Kop, cudaStream_t st) {
     if (M <= 0) return cudaSuccess;
     const int M_pad = quant ? (M + 127) / 128 * 128 : M;
-    const dim3 grid((M_pad + RN_WARPS - 1) / RN_WARPS), block(32 * RN_WARPS);
-    const size_t smem = (size_t)RN_WARPS * K * 2 + RN_WARPS * 16;
+    const dim3 grid((M_pad + RN_ROWS - 1) / RN_ROWS), block(RN_THREADS);
+    constexpr int kTail = RN_ROWS * (8 + RN_WPR * 8 + 4) + 8;   // mbarriers, partial sums, give-up flags
+    const size_t smem = (size_t)RN_ROWS * K * 2 + kTail;
     static PerDevice configured_q, configured_n;
-    if (cudaError_t e = opt_in_shared_memory(configured_q, rmsnorm_quant_kernel<true>, RN_WARPS * 8192 * 2 + RN_WARPS * 16)) return e;
-    if (cudaError_t e = opt_in_shared_memory(configured_n, rmsnorm_quant_kernel<false>, RN_WARPS * 8192 * 2 + RN_WARPS * 16)) return e;
+    if (cudaError_t e = opt_in_shared_memory(configured_q, rmsnorm_quant_kernel<true>, RN_ROWS * 8192 * 2 + kTail)) return e;
+    if (cudaError_t e = opt_in_shared_memory(configured_n, rmsnorm_quant_kernel<false>, RN_ROWS * 8192 * 2 + kTail)) return e;
     if (quant)
         return launch_pdl(rmsnorm_quant_kernel<true>, grid, block, smem, st, static_cast<const uint16_t*>(H), ldh, M, M_pad, K,
                           static_cast<const uint16_t*>(gamma), eps, static_cast<uint16_t*>(Xn), ldx, idx_o,
