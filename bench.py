@@ -814,7 +814,20 @@ def run_sweep(args):
     troof = max(f4 / peaks["fp4"] + f16 / peaks["bf16"], byts / peaks["hbm"])
     rows.append({"name": "moe.gate_up(grouped)", "M": Mt, "K": K, "N": N, "K_o": w.K_o, "ms": ms,
                  "tflops": (f4 + f16) / ms / 1e9, "pct_roofline": 100 * troof / (ms * 1e-3), "roof_us": troof * 1e6})
-    del Xd, Wd, w, ws, Y
+    # the same layer with the dispatch fused behind the quantizer: 8192 tokens quantized once, their quantized rows
+    # gathered to the 65536 (token, expert) rows; the caller never builds the permuted bf16 matrix
+    T_tok = Mt // 8
+    Xtok = Xd[:T_tok].contiguous()
+    row_token = torch.from_numpy(np.random.default_rng(0).integers(0, T_tok, size=Mt).astype(np.int32)).cuda()
+    wsg = torch.empty(B.osc_gather_workspace_bytes(w, T_tok, Mt), dtype=torch.uint8, device="cuda")
+    msg = time_loop(torch, lambda i: B.osc_linear_grouped_gather(w, Xtok, row_token, off, Y, wsg), steps, warm)
+    B.osc_sync_check()
+    bytsg = 2.0 * T_tok * K + E * (N * K / 2 + N * K / 32 + 2.0 * N * w.K_o) + 2.0 * Mt * N
+    troofg = max(f4 / peaks["fp4"] + f16 / peaks["bf16"], bytsg / peaks["hbm"])
+    rows.append({"name": "moe.gate_up(grouped, gathered from 8192 tokens)", "M": Mt, "K": K, "N": N, "K_o": w.K_o, "ms": msg,
+                 "tflops": (f4 + f16) / msg / 1e9, "pct_roofline": 100 * troofg / (msg * 1e-3), "roof_us": troofg * 1e6,
+                 "speedup_vs_permuted_input": ms / msg})
+    del Xd, Wd, w, ws, Y, wsg, Xtok
     c = synth.moe_down_case(E, counts, weight_pool=8)
     Xd = dev_bf16(torch, c["X"])
     Wd = dev_bf16(torch, c["W"].reshape(E * c["N"], c["K"])).view(E, c["N"], c["K"])

@@ -190,6 +190,18 @@ osc_status osc_linear_grouped(const osc_weights* w, const void* X_perm, const in
                               int64_t ldx, void* Y, int64_t ldy, void* workspace, size_t workspace_bytes,
                               void* stream);
 
+/* Grouped form with the dispatch fused behind the quantizer.  In a mixture-of-experts layer a token goes to several
+ * experts and Algorithm 2 does not depend on the expert (one table per layer): X holds the T tokens once
+ * (dev bf16 [T, ldx]), row_token (dev int32 [M_total]) names the source token of every permuted row, off as in
+ * osc_linear_grouped.  The tokens are quantized once and their packed codes, scale bytes and backed-up channels are
+ * copied to the rows their experts own; the result equals osc_linear_grouped on X_perm[r] = X[row_token[r]] bit for
+ * bit, without X_perm ever existing.  Indices outside [0, T) are clamped.  The workspace holds the grouped buffers
+ * of osc_act_sizes(w, M_total) followed by the T tokens' quantized form: ask osc_gather_workspace_bytes. */
+osc_status osc_gather_workspace_bytes(const osc_weights* w, int T, int M_total, size_t* bytes);
+osc_status osc_linear_grouped_gather(const osc_weights* w, const void* X, int T, int64_t ldx, const int32_t* row_token,
+                                     const int32_t* off, int M_total, void* Y, int64_t ldy, void* workspace,
+                                     size_t workspace_bytes, void* stream);
+
 /* ---------------------------------------------------- offline profiling */
 
 /* Scratch bytes osc_profile_lut needs for a K-channel slice (an fp64 sum and 32 counters per group). */

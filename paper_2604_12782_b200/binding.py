@@ -76,6 +76,8 @@ _SIGS = {
     "osc_linear": (_i, [_vp, _vp, _i, _i64, _vp, _i64, _vp, _sz, _vp]),
     "osc_linear_static": (_i, [_vp, _vp, _i, _i64, _vp, _i64, _vp]),
     "osc_linear_grouped": (_i, [_vp, _vp, _vp, _i, _i64, _vp, _i64, _vp, _sz, _vp]),
+    "osc_gather_workspace_bytes": (_i, [_vp, _i, _i, C.POINTER(_sz)]),
+    "osc_linear_grouped_gather": (_i, [_vp, _vp, _i, _i64, _vp, _vp, _i, _vp, _i64, _vp, _sz, _vp]),
     "osc_rmsnorm": (_i, [_vp, _i, _i, _i64, _vp, C.c_float, _vp, _i64, _vp]),
     "osc_swiglu": (_i, [_vp, _i, _i, _i64, _vp, _i64, _vp]),
     "osc_swiglu_fp8_quantize": (_i, [_vp, _i, _i, _i64, _vp, _vp, _vp]),
@@ -266,6 +268,21 @@ def osc_linear_static(w: OscWeights, X: torch.Tensor, Y: torch.Tensor, stream=No
     M = X.shape[0]
     _check(_lib.osc_linear_static(w.ptr, _ptr(X), M, X.stride(0) if M else w.K, _ptr(Y), Y.stride(0) if M else w.N,
                                   _stream(stream)))
+
+
+def osc_gather_workspace_bytes(w: OscWeights, T: int, M_total: int) -> int:
+    out = _sz()
+    _check(_lib.osc_gather_workspace_bytes(w.ptr, T, M_total, C.byref(out)))
+    return int(out.value)
+
+
+def osc_linear_grouped_gather(w: OscWeights, X: torch.Tensor, row_token: torch.Tensor, off: torch.Tensor, Y: torch.Tensor,
+                              workspace: torch.Tensor, stream=None):
+    """Grouped linear on X[row_token] without materialising it: tokens quantized once, quantized rows gathered."""
+    T, M = X.shape[0], row_token.shape[0]
+    _check(_lib.osc_linear_grouped_gather(w.ptr, _ptr(X), T, X.stride(0) if T else w.K, _ptr(row_token), _ptr(off), M,
+                                          _ptr(Y), Y.stride(0) if M else w.N, _ptr(workspace),
+                                          workspace.numel() * workspace.element_size(), _stream(stream)))
 
 
 def osc_rmsnorm(H: torch.Tensor, gamma: torch.Tensor, eps: float, X: torch.Tensor, stream=None):

@@ -617,6 +617,64 @@ osc_status osc_linear_grouped(const osc_weights* w, const void* X_perm, const in
                      sched2, max_tiles2, st);
 }
 
+// ---- grouped linear with the dispatch fused behind the quantizer: tokens quantized once, quantized rows gathered
+struct GatherLayout {
+    size_t xq_u, sf_u, xo_u, total;   // offsets of the unique tokens' buffers behind the grouped workspace, and the total
+};
+static GatherLayout gather_layout(const osc_weights* w, int T, const osc_act_sizes_t& sz) {
+    GatherLayout g;
+    g.xq_u = sz.workspace_bytes;
+    g.sf_u = g.xq_u + align256((size_t)T * (w->K / 2));
+    g.xo_u = g.sf_u + align256((size_t)((T + 127) / 128) * (w->K / 128) * 512);
+    g.total = g.xo_u + align256((size_t)T * w->Kop * 2);
+    return g;
+}
+
+osc_status osc_gather_workspace_bytes(const osc_weights* w, int T, int M_total, size_t* bytes) {
+    if (!w || !bytes) return fail(OSC_ERR_INVALID_ARG, "null argument");
+    if (!w->grouped) return fail(OSC_ERR_INVALID_ARG, "dense weights have no dispatch");
+    if (T < 0 || M_total < 0) return fail(OSC_ERR_INVALID_ARG, "negative size");
+    osc_act_sizes_t sz;
+    if (osc_status s = osc_act_sizes(w, M_total, &sz)) return s;
+    *bytes = gather_layout(w, T, sz).total;
+    return OSC_OK;
+}
+
+osc_status osc_linear_grouped_gather(const osc_weights* w, const void* X, int T, int64_t ldx, const int32_t* row_token,
+                                     const int32_t* off, int M_total, void* Y, int64_t ldy, void* workspace,
+                                     size_t workspace_bytes, void* stream) {
+    if (osc_status s = check_act(w, X, T, ldx)) return s;
+    if (!w->grouped) return fail(OSC_ERR_INVALID_ARG, "dense weights: use osc_linear");
+    if (M_total < 0) return fail(OSC_ERR_INVALID_ARG, "M_total = %d is negative", M_total);
+    if (M_total == 0) return OSC_OK;
+    if (T == 0) return fail(OSC_ERR_INVALID_ARG, "rows to dispatch but no tokens");
+    if (!off || !row_token) return fail(OSC_ERR_INVALID_ARG, "off / row_token is null");
+    osc_act_sizes_t sz;
+    osc_act_sizes(w, M_total, &sz);
+    const GatherLayout g = gather_layout(w, T, sz);
+    if (!workspace || !aligned16(workspace)) return fail(OSC_ERR_ALIGN, "workspace must be non-null and 16-byte aligned");
+    if (workspace_bytes < g.total)
+        return fail(OSC_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", workspace_bytes, g.total);
+    if (!Y) return fail(OSC_ERR_INVALID_ARG, "Y is null");
+    if (ldy < w->N) return fail(OSC_ERR_SHAPE, "ldy = %lld < N = %d", (long long)ldy, w->N);
+    if (ldy % 8 || !aligned16(Y)) return fail(OSC_ERR_ALIGN, "Y must be 16-byte aligned and ldy a multiple of 8");
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int max_tiles = M_total / 128 + w->E;
+    const int max_tiles2 = max_tiles256(M_total, w->E);
+    int32_t* sched = reinterpret_cast<int32_t*>(ws + sz.sched_offset);
+    int32_t* sched2 = use_pair_kernel(true, M_total, w->E) ? sched + sched_ints(max_tiles) : nullptr;
+    cudaError_t e = launch_build_sched(off, w->E, sched, max_tiles, sched2, max_tiles2, st);
+    if (e != cudaSuccess) return cuda_fail(e, "build_sched_kernel");
+    // Algorithm 2 once per token (it does not depend on the expert), as a dense problem of T rows
+    if (osc_status s = quantize_impl(w, X, T, ldx, ws + g.xq_u, ws + g.sf_u, ws + g.xo_u, nullptr, 0, st)) return s;
+    e = launch_gather_quantized(row_token, T, w->K, w->Kop, ws + g.xq_u, ws + g.sf_u, ws + g.xo_u, ws + sz.xq_offset,
+                                ws + sz.sfa_offset, ws + sz.xo_offset, sched, max_tiles, st);
+    if (e != cudaSuccess) return cuda_fail(e, "gather_quantized_kernel");
+    return gemm_impl(w, ws + sz.xq_offset, ws + sz.sfa_offset, ws + sz.xo_offset, M_total, Y, ldy, sched, max_tiles,
+                     sched2, max_tiles2, st);
+}
+
 // ------------------------------------------------------- offline profiling
 
 osc_status osc_profile_scratch_bytes(int K, size_t* bytes) {

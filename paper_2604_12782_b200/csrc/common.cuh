@@ -63,6 +63,10 @@ cudaError_t launch_dyn_quant_extract(const void* X, int64_t ldx, int M, int K, v
 cudaError_t launch_build_sched(const int32_t* off, int E, int32_t* sched128, int max_tiles128, int32_t* sched256,
                                int max_tiles256, cudaStream_t st);
 
+cudaError_t launch_gather_quantized(const int32_t* row_token, int T, int K, int Kop, const void* xq_u, const void* sf_u,
+                                    const void* xo_u, void* xq, void* sf, void* xo, const int32_t* sched, int max_tiles,
+                                    cudaStream_t st);
+
 // norm_kernels.cu
 cudaError_t launch_rmsnorm_quant(bool quant, const void* H, int64_t ldh, int M, int K, const void* gamma, float eps,
                                  void* Xn, int64_t ldx, const int32_t* idx_o, void* xq, void* sf,

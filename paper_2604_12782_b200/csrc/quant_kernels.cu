@@ -610,45 +610,69 @@ dyn_quant_extract_kernel(const uint16_t* __restrict__ X, int64_t ldx, int M, int
 // sched[0] = number of row tiles (tile_rows = 128 or 256 rows each, never crossing an expert boundary);
 // then four arrays of max_tiles entries: first row, end row (exclusive, the expert's end), first scale
 // row (scale rows are padded to 128 per expert whatever the tile height), expert.
-// Block 0 builds the 128-row schedule (if sched is given), block 1 the 256-row one (if sched2 is given).
-__global__ void build_sched_kernel(const int32_t* __restrict__ off, int E, int32_t* __restrict__ sched128,
-                                   int max_tiles128, int32_t* __restrict__ sched256, int max_tiles256) {
-    __shared__ int s_tiles[1024];
-    __shared__ int s_sfbase[1024];
+// Block 0 builds the 128-row schedule (if sched is given), block 1 the 256-row one (if sched2 is given).  Thread e scans
+// expert e's tile count and padded scale rows block-wide, then thread t writes tile t (binary search for its expert):
+// a version with a serial prefix by one thread and one thread per expert took ~14 us for 128 experts.
+constexpr int SCHED_THREADS = 1024;   // = the most experts a schedule can be built for
+
+__global__ void __launch_bounds__(SCHED_THREADS)
+build_sched_kernel(const int32_t* __restrict__ off, int E, int32_t* __restrict__ sched128, int max_tiles128,
+                   int32_t* __restrict__ sched256, int max_tiles256) {
+    __shared__ int s_tiles[SCHED_THREADS + 1];    // exclusive prefix of the experts' tile counts (+ the total)
+    __shared__ int s_sfbase[SCHED_THREADS];       // exclusive prefix of the experts' padded scale rows
+    __shared__ int s_wt[32], s_ws[32];
     grid_launch_dependents();
     grid_dependency_wait();
-    const int tid = threadIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const bool tall = blockIdx.x == 1 || sched128 == nullptr;
     int32_t* sched = tall ? sched256 : sched128;
     const int max_tiles = tall ? max_tiles256 : max_tiles128;
     const int tile_rows = tall ? 256 : 128;
     if (sched == nullptr) return;
-    // serial prefix by one thread: E is small (hundreds) and this runs once per call
-    if (tid == 0) {
-        int acc = 0, sfacc = 0;
-        for (int e = 0; e < E; ++e) {
-            s_tiles[e] = acc;
-            s_sfbase[e] = sfacc;
-            const int m = off[e + 1] - off[e];
-            acc += (m + tile_rows - 1) / tile_rows;
-            sfacc += (m + 127) / 128 * 128;
+    // thread e owns expert e: block-wide exclusive scan of (tiles, padded scale rows)
+    const int m = tid < E ? off[tid + 1] - off[tid] : 0;
+    const int nt = (m + tile_rows - 1) / tile_rows, ns = (m + 127) / 128 * 128;
+    int it = nt, is = ns;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int a = __shfl_up_sync(0xFFFFFFFFu, it, o), b = __shfl_up_sync(0xFFFFFFFFu, is, o);
+        if (lane >= o) { it += a; is += b; }
+    }
+    if (lane == 31) { s_wt[warp] = it; s_ws[warp] = is; }
+    __syncthreads();
+    if (warp == 0) {
+        int a = s_wt[lane], b = s_ws[lane];
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int x = __shfl_up_sync(0xFFFFFFFFu, a, o), y = __shfl_up_sync(0xFFFFFFFFu, b, o);
+            if (lane >= o) { a += x; b += y; }
         }
-        sched[0] = acc < max_tiles ? acc : max_tiles;
+        s_wt[lane] = a;
+        s_ws[lane] = b;
     }
     __syncthreads();
-    for (int e = tid; e < E; e += blockDim.x) {
-        const int m = off[e + 1] - off[e];
-        const int nt = (m + tile_rows - 1) / tile_rows;
-        const int t0 = s_tiles[e];
-        for (int i = 0; i < nt; ++i) {
-            const int t = t0 + i;
-            if (t < max_tiles) {
-                sched[1 + t] = off[e] + i * tile_rows;
-                sched[1 + max_tiles + t] = off[e + 1];
-                sched[1 + 2 * max_tiles + t] = s_sfbase[e] + i * tile_rows;
-                sched[1 + 3 * max_tiles + t] = e;
-            }
+    const int base_t = warp ? s_wt[warp - 1] : 0, base_s = warp ? s_ws[warp - 1] : 0;
+    s_tiles[tid] = base_t + it - nt;
+    s_sfbase[tid] = base_s + is - ns;
+    const int total = s_wt[31];
+    if (tid == 0) {
+        s_tiles[SCHED_THREADS] = total;
+        sched[0] = total < max_tiles ? total : max_tiles;
+    }
+    __syncthreads();
+    // thread t owns tile t: its expert is the last one whose first tile is <= t
+    for (int t = tid; t < total && t < max_tiles; t += SCHED_THREADS) {
+        int lo = 0, hi = E - 1;
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (s_tiles[mid] <= t) lo = mid; else hi = mid - 1;
         }
+        const int e = lo;   // (experts without rows share their first tile index with the next one; the last of them owns it)
+        const int i = t - s_tiles[e];
+        sched[1 + t] = off[e] + i * tile_rows;
+        sched[1 + max_tiles + t] = off[e + 1];
+        sched[1 + 2 * max_tiles + t] = s_sfbase[e] + i * tile_rows;
+        sched[1 + 3 * max_tiles + t] = e;
     }
 }
 
@@ -683,6 +707,88 @@ cudaError_t launch_retile_sf(const uint8_t* src, uint8_t* dst, int N, int K, int
     const int blocks = (int)((total + 255) / 256 < 2048 ? (total + 255) / 256 : 2048);
     retile_sf_kernel<<<blocks, 256, 0, st>>>(src, dst, N, K, bn);
     return cudaGetLastError();
+}
+
+// ------------------------------------------------- gather of quantized rows (MoE dispatch)
+// In a mixture-of-experts layer every token goes to several experts, and Algorithm 2 does not depend on the expert
+// (one table per layer): the tokens are quantized once, and this kernel copies each token's packed codes, scale bytes
+// and backed-up channels to the rows its experts own (row_token[r] = source token of permuted row r).  One block per
+// 128-row tile of the schedule, one warp per row at a time; scale bytes move as the 32-bit words of the 128 x 4 block
+// layout; the scale rows that only pad an expert's last block are written as zeros.
+__global__ void __launch_bounds__(256)
+gather_quantized_kernel(const int32_t* __restrict__ row_token, int T, int K, int Kop,
+                        const uint8_t* __restrict__ xq_u, const uint8_t* __restrict__ sf_u, const uint16_t* __restrict__ xo_u,
+                        uint8_t* __restrict__ xq, uint8_t* __restrict__ sf, uint16_t* __restrict__ xo,
+                        const int32_t* __restrict__ sched, int max_tiles) {
+    extern __shared__ uint32_t gq_sf[];   // the tile's scale block row: [K / 128][128] words, written out in one piece
+    grid_launch_dependents();
+    grid_dependency_wait();
+    const int tile = blockIdx.x;
+    if (tile >= sched[0]) return;
+    const int row0 = sched[1 + tile], row_end = sched[1 + max_tiles + tile], sf_row0 = sched[1 + 2 * max_tiles + tile];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int katoms = K / 128;
+    const int nq = K / 32;          // 16-byte chunks of a row of packed codes
+    const int no = Kop / 8;         // 16-byte chunks of a row of backed-up channels
+    const uint32_t* sfu32 = reinterpret_cast<const uint32_t*>(sf_u);
+    uint32_t* sf32 = reinterpret_cast<uint32_t*>(sf);
+    // the warp's sixteen rows (rr = warp, warp + 8, ...): lane i holds the token of row i; four rows per pass, all
+    // their loads issued before the first store
+    const int my_r = row0 + warp + 8 * (lane & 15);
+    const int my_t = (my_r < row_end) ? min(max(row_token[my_r], 0), T - 1) : -1;   // an index outside the token range
+                                                                                 // must not become an address
+    for (int i0 = 0; i0 < 16; i0 += 4) {
+        uint4 q[4][2], o4[4];
+        uint32_t sw[4];
+        int tk[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            tk[u] = __shfl_sync(0xFFFFFFFFu, my_t, i0 + u);
+            q[u][0] = q[u][1] = o4[u] = make_uint4(0u, 0u, 0u, 0u);
+            sw[u] = 0u;
+            if (tk[u] >= 0) {
+                const uint4* src_q = reinterpret_cast<const uint4*>(xq_u + (size_t)tk[u] * (K / 2));
+                if (lane < nq) q[u][0] = src_q[lane];
+                if (lane + 32 < nq) q[u][1] = src_q[lane + 32];
+                if (lane < no) o4[u] = reinterpret_cast<const uint4*>(xo_u + (size_t)tk[u] * Kop)[lane];
+                if (lane < katoms)
+                    sw[u] = sfu32[((size_t)(tk[u] >> 7) * katoms + lane) * 128 + (tk[u] & 31) * 4 + ((tk[u] & 127) >> 5)];
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int rr = warp + 8 * (i0 + u);
+            const int r = row0 + rr, sr = sf_row0 + rr;
+            // scale words: the row's own, or zeros for the rows that only pad the expert's last scale block; staged
+            // in shared memory (every tile starts a 128-row scale block, so rr is the row inside the block)
+            uint32_t* dst_sf = gq_sf + (rr & 31) * 4 + (rr >> 5);
+            if (lane < katoms) dst_sf[lane * 128] = sw[u];
+            for (int a = lane + 32; a < katoms; a += 32)
+                dst_sf[a * 128] = tk[u] >= 0 ? sfu32[((size_t)(tk[u] >> 7) * katoms + a) * 128 + (tk[u] & 31) * 4 + ((tk[u] & 127) >> 5)] : 0u;
+            (void)sr;
+            if (tk[u] < 0) continue;
+            uint4* dst_q = reinterpret_cast<uint4*>(xq + (size_t)r * (K / 2));
+            if (lane < nq) dst_q[lane] = q[u][0];
+            if (lane + 32 < nq) dst_q[lane + 32] = q[u][1];
+            for (int c = lane + 64; c < nq; c += 32)
+                dst_q[c] = reinterpret_cast<const uint4*>(xq_u + (size_t)tk[u] * (K / 2))[c];
+            uint4* dst_o = reinterpret_cast<uint4*>(xo + (size_t)r * Kop);
+            if (lane < no) dst_o[lane] = o4[u];
+            for (int c = lane + 32; c < no; c += 32) dst_o[c] = reinterpret_cast<const uint4*>(xo_u + (size_t)tk[u] * Kop)[c];
+        }
+    }
+    __syncthreads();
+    uint4* dst_blk = reinterpret_cast<uint4*>(sf32 + (size_t)(sf_row0 >> 7) * katoms * 128);
+    for (int i = threadIdx.x; i < katoms * 32; i += blockDim.x) dst_blk[i] = reinterpret_cast<const uint4*>(gq_sf)[i];
+}
+
+cudaError_t launch_gather_quantized(const int32_t* row_token, int T, int K, int Kop, const void* xq_u, const void* sf_u,
+                                    const void* xo_u, void* xq, void* sf, void* xo, const int32_t* sched, int max_tiles,
+                                    cudaStream_t st) {
+    if (max_tiles <= 0) return cudaSuccess;
+    return launch_pdl(gather_quantized_kernel, dim3(max_tiles), dim3(256), (size_t)(K / 128) * 512, st, row_token, T, K, Kop,
+                      static_cast<const uint8_t*>(xq_u), static_cast<const uint8_t*>(sf_u), static_cast<const uint16_t*>(xo_u),
+                      static_cast<uint8_t*>(xq), static_cast<uint8_t*>(sf), static_cast<uint16_t*>(xo), sched, max_tiles);
 }
 
 // ------------------------------------------------------------------ launchers
@@ -754,7 +860,7 @@ cudaError_t launch_build_sched(const int32_t* off, int E, int32_t* sched128, int
                                int max_tiles256, cudaStream_t st) {
     const int blocks = (sched128 != nullptr) + (sched256 != nullptr);
     if (blocks == 0) return cudaSuccess;
-    return launch_pdl(build_sched_kernel, dim3(blocks), dim3(256), 0, st, off, E, sched128, max_tiles128, sched256,
+    return launch_pdl(build_sched_kernel, dim3(blocks), dim3(SCHED_THREADS), 0, st, off, E, sched128, max_tiles128, sched256,
                       max_tiles256);
 }
 

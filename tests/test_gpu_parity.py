@@ -346,3 +346,50 @@ def test_calls_can_be_captured_in_a_cuda_graph(B, oracle):
         B.osc_sync_check()
         outs[M] = want
     assert outs[24].shape[0] == 24
+
+
+@pytest.mark.parametrize("kind", ["small", "mid"])
+def test_grouped_gather_equals_grouped_on_permuted_rows(B, oracle, kind):
+    """Dispatch fused behind the quantizer: tokens quantized once, quantized rows gathered per expert.  Must equal the
+    grouped linear on X[row_token] byte for byte (same kernels on identical operands), and the oracle within tolerance."""
+    counts = grouped_counts(kind)
+    E, K, N, T = counts.size, 384, (320 if kind == "mid" else 192), 200
+    c = synth.moe_gate_up_case(E, counts, K=K, N=N, seed=5)
+    M = c["M"]
+    rng = np.random.default_rng(11)
+    Xtok, _ = synth.osc_activations_only(9, T, K, 1)
+    row_token = rng.integers(0, T, size=M).astype(np.int32)
+    row_token[:3] = [0, T - 1, 0]                      # repeated and extreme tokens
+    Xperm = Xtok[row_token]
+    w = B.osc_prepare_weights_grouped(dev_bf16(c["W"].reshape(E * N, K)).view(E, N, K), c["lut"])
+    off = torch.from_numpy(c["off"]).cuda()
+    sz = B.osc_act_sizes(w, M)
+    ws_a = poison(sz.workspace_bytes)
+    Ya = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+    B.osc_linear_grouped(w, dev_bf16(Xperm), off, Ya, ws_a)
+    nbytes = B.osc_gather_workspace_bytes(w, T, M)
+    assert nbytes > sz.workspace_bytes
+    ws_b = poison(nbytes)
+    Yb = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+    B.osc_linear_grouped_gather(w, dev_bf16(Xtok), torch.from_numpy(row_token).cuda(), off, Yb, ws_b)
+    B.osc_sync_check()
+    assert torch.equal(Ya.view(torch.int16), Yb.view(torch.int16))
+    for o, n in ((sz.xq_offset, sz.xq_bytes), (sz.xo_offset, sz.xo_bytes)):
+        assert torch.equal(ws_a[o:o + n], ws_b[o:o + n])
+    # scale bytes: every block either side wrote (the blocks of the schedule's tiles) agrees; compare on the valid rows
+    gq = oracle.quantize_extract_grouped(Xperm, c["off"], c["lut"])
+    sfa, sfb = host_u8(ws_a)[sz.sfa_offset:], host_u8(ws_b)[sz.sfa_offset:]
+    for e in range(E):
+        if counts[e]:
+            v = valid_sf_bytes(oracle, int(counts[e]), K, int(gq["sf_row_base"][e]))
+            assert np.array_equal(sfa[v], sfb[v]) and np.array_equal(sfb[v], gq["sf"][v])
+    Yh = host_f64(Yb)
+    for e in range(E):
+        r0, r1 = int(c["off"][e]), int(c["off"][e + 1])
+        if r1 > r0:
+            Yref, Tb, *_ = oracle.linear(Xperm[r0:r1], c["W"][e], c["lut"])
+            assert_within_tolerance(Yh[r0:r1], Yref, Tb, f"gathered grouped expert {e}")
+    # too small a workspace is refused before any launch
+    with pytest.raises(B.OscError) as err:
+        B.osc_linear_grouped_gather(w, dev_bf16(Xtok), torch.from_numpy(row_token).cuda(), off, Yb, ws_b[:sz.workspace_bytes])
+    assert err.value.status == -5
