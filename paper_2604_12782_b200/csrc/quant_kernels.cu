@@ -715,7 +715,10 @@ cudaError_t launch_retile_sf(const uint8_t* src, uint8_t* dst, int N, int K, int
 // and backed-up channels to the rows its experts own (row_token[r] = source token of permuted row r).  One block per
 // 128-row tile of the schedule, one warp per row at a time; scale bytes move as the 32-bit words of the 128 x 4 block
 // layout; the scale rows that only pad an expert's last block are written as zeros.
-__global__ void __launch_bounds__(256)
+constexpr int GQ_WARPS = 16;              // warps per block; each takes 128 / GQ_WARPS rows of the tile
+constexpr int GQ_RPW = 128 / GQ_WARPS;
+
+__global__ void __launch_bounds__(32 * GQ_WARPS)
 gather_quantized_kernel(const int32_t* __restrict__ row_token, int T, int K, int Kop,
                         const uint8_t* __restrict__ xq_u, const uint8_t* __restrict__ sf_u, const uint16_t* __restrict__ xo_u,
                         uint8_t* __restrict__ xq, uint8_t* __restrict__ sf, uint16_t* __restrict__ xo,
@@ -732,12 +735,12 @@ gather_quantized_kernel(const int32_t* __restrict__ row_token, int T, int K, int
     const int no = Kop / 8;         // 16-byte chunks of a row of backed-up channels
     const uint32_t* sfu32 = reinterpret_cast<const uint32_t*>(sf_u);
     uint32_t* sf32 = reinterpret_cast<uint32_t*>(sf);
-    // the warp's sixteen rows (rr = warp, warp + 8, ...): lane i holds the token of row i; four rows per pass, all
+    // the warp's rows (rr = warp, warp + GQ_WARPS, ...): lane i holds the token of row i; four rows per pass, all
     // their loads issued before the first store
-    const int my_r = row0 + warp + 8 * (lane & 15);
+    const int my_r = row0 + warp + GQ_WARPS * (lane % GQ_RPW);
     const int my_t = (my_r < row_end) ? min(max(row_token[my_r], 0), T - 1) : -1;   // an index outside the token range
                                                                                  // must not become an address
-    for (int i0 = 0; i0 < 16; i0 += 4) {
+    for (int i0 = 0; i0 < GQ_RPW; i0 += 4) {
         uint4 q[4][2], o4[4];
         uint32_t sw[4];
         int tk[4];
@@ -757,7 +760,7 @@ gather_quantized_kernel(const int32_t* __restrict__ row_token, int T, int K, int
         }
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-            const int rr = warp + 8 * (i0 + u);
+            const int rr = warp + GQ_WARPS * (i0 + u);
             const int r = row0 + rr, sr = sf_row0 + rr;
             // scale words: the row's own, or zeros for the rows that only pad the expert's last scale block; staged
             // in shared memory (every tile starts a 128-row scale block, so rr is the row inside the block)
@@ -786,7 +789,7 @@ cudaError_t launch_gather_quantized(const int32_t* row_token, int T, int K, int 
                                     const void* xo_u, void* xq, void* sf, void* xo, const int32_t* sched, int max_tiles,
                                     cudaStream_t st) {
     if (max_tiles <= 0) return cudaSuccess;
-    return launch_pdl(gather_quantized_kernel, dim3(max_tiles), dim3(256), (size_t)(K / 128) * 512, st, row_token, T, K, Kop,
+    return launch_pdl(gather_quantized_kernel, dim3(max_tiles), dim3(32 * GQ_WARPS), (size_t)(K / 128) * 512, st, row_token, T, K, Kop,
                       static_cast<const uint8_t*>(xq_u), static_cast<const uint8_t*>(sf_u), static_cast<const uint16_t*>(xo_u),
                       static_cast<uint8_t*>(xq), static_cast<uint8_t*>(sf), static_cast<uint16_t*>(xo), sched, max_tiles);
 }
