@@ -72,7 +72,7 @@ struct Cfg {
     static constexpr int LAST_W = BN - 64 * (SLICES - 1);  // width of the last one (64 or 48)
     // staging tiles per epilogue warp: 2 = the warp's whole share of a tile (accumulator released before any
     // store is issued); 1 = one slice at a time
-    static constexpr int EPI_TPW = (LAST_W != 64) ? 2 : 1;
+    static constexpr int EPI_TPW = 1;
     static constexpr int EPI_BYTES = EPI_WARPS * EPI_TPW * EPI_TILE_BYTES;
     static constexpr int STAGES = ((224 * 1024 - EPI_BYTES) / STAGE_BYTES) / LANES * LANES;
     static constexpr int SPL = STAGES / LANES;          // ring stages per lane
@@ -94,7 +94,6 @@ struct Cfg {
     static_assert(SPL >= 3, "ring too shallow");
     static_assert((SLICES + 1) / 2 <= 2, "an epilogue warp drains at most two slices of a tile");
     static_assert(BN % 16 == 0 && BN <= 256 && (LAST_W == 64 || LAST_W == 48), "tile width");
-    static_assert(LAST_W == 64 || EPI_TPW == 2, "the narrow last slice is written from a staged tile");
 };
 
 template <int MODE, int BN>
@@ -449,18 +448,19 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
                     if (TPW == 1) {
                         fence_proxy_async_smem();
                         __syncwarp();
-                        if (!clip) {
+                        if (!clip && !narrow) {
                             if (lane == 0) {
                                 tma_store_2d(&args.tm_y, buf, col, wrow0);
                                 tma_store_commit();
                             }
                         } else {
-                            // rows past the expert's end must stay untouched: row-masked 16-byte stores from the staged tile
+                            // rows past the expert's end must stay untouched, and the 48-column last slice of a 240-wide
+                            // tile is no TMA box: row-masked 16-byte stores from the staged tile
                             const int j8 = lane & 7;
 #pragma unroll
                             for (int rr = 0; rr < 8; ++rr) {
                                 const int rl = rr * 4 + (lane >> 3);
-                                if (wrow0 + rl < ti.row_end && col + j8 * 8 < N)
+                                if (wrow0 + rl < ti.row_end && col + j8 * 8 < N && (!narrow || j8 < C::LAST_W / 8))
                                     *reinterpret_cast<uint4*>(args.Y + (int64_t)(wrow0 + rl) * args.ldy + col + j8 * 8) =
                                         *reinterpret_cast<const uint4*>(buf + rl * 128 + ((j8 ^ (rl & 7)) << 4));
                             }
