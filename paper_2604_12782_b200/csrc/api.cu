@@ -496,6 +496,7 @@ static osc_status gemm_impl(const osc_weights* w, const void* xq, const void* sf
         const uint64_t sf_row_blocks = w->grouped ? (uint64_t)max_tiles : (uint64_t)((M + 127) / 128);
         if (osc_status s = make_tmap_sf(&a.tm_sfa, sfa, sf_row_blocks * (w->K / 128))) return s;
         if (osc_status s = make_tmap(&a.tm_y, Y, true, M, (uint64_t)w->N * 2, (uint64_t)ldy * 2, 32)) return s;
+        if (osc_status s = make_tmap(&a.tm_y16, Y, true, M, (uint64_t)w->N * 2, (uint64_t)ldy * 2, 16)) return s;
         e = launch_gemm_dual_pair(a, bn, st);
     } else {
         e = launch_gemm_dual(a, bn1, st);
@@ -820,6 +821,7 @@ static osc_status fp8_gemm_impl(const osc_fp8_weights* w, const void* x8, const 
         const int bn = bn2;
         a.tm_b = w->tm_b2[bn == 256];
         if (osc_status s = make_tmap(&a.tm_y, Y, true, M, (uint64_t)w->N * 2, (uint64_t)ldy * 2, 32)) return s;
+        if (osc_status s = make_tmap(&a.tm_y16, Y, true, M, (uint64_t)w->N * 2, (uint64_t)ldy * 2, 16)) return s;
         e = launch_gemm_fp8_pair(a, bn, st);
     } else {
         e = launch_gemm_fp8(a, bn1, st);
@@ -1062,6 +1064,7 @@ static osc_status mxfp8_gemm_impl(const osc_mxfp8_weights* w, const void* x8, co
     const uint64_t sf_row_blocks = w->grouped ? (uint64_t)max_tiles : (uint64_t)((M + 127) / 128);
     if (osc_status s = make_tmap_sf(&a.tm_sfa, sfa, sf_row_blocks * (w->K / 128), 1)) return s;
     if (osc_status s = make_tmap(&a.tm_y, Y, true, M, (uint64_t)w->N * 2, (uint64_t)ldy * 2, 32)) return s;
+    if (osc_status s = make_tmap(&a.tm_y16, Y, true, M, (uint64_t)w->N * 2, (uint64_t)ldy * 2, 16)) return s;
     a.sfa = static_cast<const uint8_t*>(sfa);
     a.sfw = w->sfw;
     a.Y = static_cast<uint16_t*>(Y);
@@ -1333,6 +1336,7 @@ osc_status osc_nvfp4_gemm(const osc_weights* w, const void* xq, const void* sfa,
     a.tm_sfw = w->tm_sfw;
     if (osc_status s = make_tmap_sf(&a.tm_sfa, sfa, (uint64_t)sf16_bytes(M, w->K) / 512, 4)) return s;
     if (osc_status s = make_tmap(&a.tm_y, Y, true, M, (uint64_t)w->N * 2, (uint64_t)ldy * 2, 32)) return s;
+    if (osc_status s = make_tmap(&a.tm_y16, Y, true, M, (uint64_t)w->N * 2, (uint64_t)ldy * 2, 16)) return s;
     a.sfa = static_cast<const uint8_t*>(sfa);
     a.sfw = w->sfw;
     a.Y = static_cast<uint16_t*>(Y);

@@ -89,6 +89,7 @@ struct GemmArgs {
     CUtensorMap tm_sfa;  // activation scale blocks as uint32 [blocks, 128] (CTA-pair kernel only)
     CUtensorMap tm_sfw;  // weight scale blocks, same form
     CUtensorMap tm_y;    // output bf16 [rows, ldy], 32 x 64 store tiles (CTA-pair kernel only)
+    CUtensorMap tm_y16;  // the same with 16 x 64 store tiles (240-wide tiles of the CTA-pair kernel)
     const uint8_t* sfa;  // activation scales, block layout
     const uint8_t* sfw;  // weight scales, block layout, per expert
     const float* sx;     // FP8 mode: per-row activation scale

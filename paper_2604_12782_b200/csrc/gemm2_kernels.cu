@@ -73,8 +73,14 @@ struct Cfg {
     // staging tiles per epilogue warp: 2 = the warp's whole share of a tile (accumulator released before any
     // store is issued); 1 = one slice at a time
     static constexpr int EPI_TPW = 1;
-    static constexpr int EPI_BYTES = EPI_WARPS * EPI_TPW * EPI_TILE_BYTES;
-    static constexpr int STAGES = ((224 * 1024 - EPI_BYTES) / STAGE_BYTES) / LANES * LANES;
+    // The ring's depth decides how well the operand feed rides out latency (240-wide tiles: 4 / 5 / 6 stages =
+    // 112.6 / 109.5 / 106.6 us per QKV step), so the staging tiles give way to it: where staging 16 rows at a time
+    // (two stores per slice) instead of 32 buys another stage, it is done.
+    static constexpr int SMEM_BUDGET = 227 * 1024 - 1024 /*alignment slack*/ - 256 /*barriers*/;
+    static constexpr int EPI_FULL = EPI_WARPS * EPI_TPW * EPI_TILE_BYTES;
+    static constexpr int EPI_HALVES = ((SMEM_BUDGET - EPI_FULL / 2) / STAGE_BYTES > (SMEM_BUDGET - EPI_FULL) / STAGE_BYTES) ? 2 : 1;
+    static constexpr int EPI_BYTES = EPI_FULL / EPI_HALVES;
+    static constexpr int STAGES = ((SMEM_BUDGET - EPI_BYTES) / STAGE_BYTES) / LANES * LANES;
     static constexpr int SPL = STAGES / LANES;          // ring stages per lane
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/ + EPI_BYTES;
     // TMEM columns.  Accumulators start at multiples of ACC_STRIDE; a 240-wide tile keeps its second
@@ -371,7 +377,7 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
         int acc = 0;
         uint32_t acc_ph = 0;
         const uint32_t tempty0 = map_to_cta(smem_u32(&tempty_bar[0]), 0);
-        uint8_t* stage_buf = smem + STAGES * C::STAGE_BYTES + (half * 4 + q) * (TPW * EPI_TILE_BYTES);
+        uint8_t* stage_buf = smem + STAGES * C::STAGE_BYTES + (half * 4 + q) * (TPW * EPI_TILE_BYTES / C::EPI_HALVES);
         for (int t = pair_id; t < total; t += num_pairs) {
             const Tile ti = tile_of(t);
             const int n0 = ti.n0;
@@ -413,44 +419,52 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
                 if (narrow) tmem_ld_32x16(tcol + 32, r1); else tmem_ld_32x32(tcol + 32, r1);
                 tmem_ld_wait();
                 const int col = n0 + c * 64;
-                uint8_t* buf = stage_buf + (TPW == 2 ? ord : 0) * EPI_TILE_BYTES;
-                if (TPW == 1) {
-                    if (lane == 0) tma_store_wait_read<0>();  // the one staging tile must be free again
-                    __syncwarp();
-                }
+                uint8_t* buf = stage_buf;
                 if (col < N) {
+                    uint4 pk[8];   // the row's 64 outputs as bf16: 8 chunks of 16 bytes = 8 columns each
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) {  // 8 chunks of 16 bytes = 8 columns each
-                        if (narrow && j >= C::LAST_W / 8) break;
-                        uint32_t o[4];
+                    for (int j = 0; j < 8; ++j) {
+                        uint32_t o[4] = {0u, 0u, 0u, 0u};
+                        if (!(narrow && j >= C::LAST_W / 8)) {
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const int cc = j * 8 + 2 * i;  // column inside the 64-column slice
-                            float lo = __uint_as_float(cc < 32 ? r0[cc] : r1[cc - 32]);
-                            float hi = __uint_as_float(cc < 32 ? r0[cc + 1] : r1[cc - 31]);
-                            if (MODE == MODE_NVF4) {   // back out of the scaled domain: an exact power of two
-                                lo *= args.out_scale;
-                                hi *= args.out_scale;
+                            for (int i = 0; i < 4; ++i) {
+                                const int cc = j * 8 + 2 * i;  // column inside the 64-column slice
+                                float lo = __uint_as_float(cc < 32 ? r0[cc] : r1[cc - 32]);
+                                float hi = __uint_as_float(cc < 32 ? r0[cc + 1] : r1[cc - 31]);
+                                if (MODE == MODE_NVF4) {   // back out of the scaled domain: an exact power of two
+                                    lo *= args.out_scale;
+                                    hi *= args.out_scale;
+                                }
+                                if (MODE == MODE_FP8) {
+                                    const float wx = __shfl_sync(0xFFFFFFFFu, wv.x, j * 4 + i);
+                                    const float wy = __shfl_sync(0xFFFFFFFFu, wv.y, j * 4 + i);
+                                    lo = lo * (sxr * wx);
+                                    hi = hi * (sxr * wy);
+                                }
+                                const __nv_bfloat162 b2 = __floats2bfloat162_rn(lo, hi);
+                                o[i] = *reinterpret_cast<const uint32_t*>(&b2);
                             }
-                            if (MODE == MODE_FP8) {
-                                const float wx = __shfl_sync(0xFFFFFFFFu, wv.x, j * 4 + i);
-                                const float wy = __shfl_sync(0xFFFFFFFFu, wv.y, j * 4 + i);
-                                lo = lo * (sxr * wx);
-                                hi = hi * (sxr * wy);
-                            }
-                            const __nv_bfloat162 b2 = __floats2bfloat162_rn(lo, hi);
-                            o[i] = *reinterpret_cast<const uint32_t*>(&b2);
                         }
-                        // 128-byte swizzle: 16-byte chunk j of row `lane` lives at chunk j ^ (lane % 8)
-                        *reinterpret_cast<uint4*>(buf + lane * 128 + ((j ^ (lane & 7)) << 4)) =
-                            make_uint4(o[0], o[1], o[2], o[3]);
+                        pk[j] = make_uint4(o[0], o[1], o[2], o[3]);
                     }
-                    if (TPW == 1) {
+                    constexpr int HV = C::EPI_HALVES, RPH = 32 / HV;   // staging passes per slice, rows per pass
+#pragma unroll
+                    for (int hh = 0; hh < HV; ++hh) {
+                        if (lane == 0) tma_store_wait_read<0>();  // the one staging tile must be free again
+                        __syncwarp();
+                        if (HV == 1 || (lane / RPH) == hh) {
+                            const int rl = lane % RPH;
+                            // 128-byte swizzle: 16-byte chunk j of row rl lives at chunk j ^ (rl % 8)
+#pragma unroll
+                            for (int j = 0; j < 8; ++j)
+                                *reinterpret_cast<uint4*>(buf + rl * 128 + ((j ^ (rl & 7)) << 4)) = pk[j];
+                        }
                         fence_proxy_async_smem();
                         __syncwarp();
+                        const int prow0 = wrow0 + hh * RPH;   // first output row of this pass
                         if (!clip && !narrow) {
                             if (lane == 0) {
-                                tma_store_2d(&args.tm_y, buf, col, wrow0);
+                                tma_store_2d(HV == 1 ? &args.tm_y : &args.tm_y16, buf, col, prow0);
                                 tma_store_commit();
                             }
                         } else {
@@ -458,10 +472,10 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
                             // tile is no TMA box: row-masked 16-byte stores from the staged tile
                             const int j8 = lane & 7;
 #pragma unroll
-                            for (int rr = 0; rr < 8; ++rr) {
+                            for (int rr = 0; rr < RPH / 4; ++rr) {
                                 const int rl = rr * 4 + (lane >> 3);
-                                if (wrow0 + rl < ti.row_end && col + j8 * 8 < N && (!narrow || j8 < C::LAST_W / 8))
-                                    *reinterpret_cast<uint4*>(args.Y + (int64_t)(wrow0 + rl) * args.ldy + col + j8 * 8) =
+                                if (prow0 + rl < ti.row_end && col + j8 * 8 < N && (!narrow || j8 < C::LAST_W / 8))
+                                    *reinterpret_cast<uint4*>(args.Y + (int64_t)(prow0 + rl) * args.ldy + col + j8 * 8) =
                                         *reinterpret_cast<const uint4*>(buf + rl * 128 + ((j8 ^ (rl & 7)) << 4));
                             }
                             __syncwarp();
