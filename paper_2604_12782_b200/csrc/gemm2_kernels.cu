@@ -70,14 +70,11 @@ struct Cfg {
     static constexpr int EPI_FIRST_WARP = 2 * LANES;
     static constexpr int SLICES = (BN + 63) / 64;        // 64-column output slices of a tile
     static constexpr int LAST_W = BN - 64 * (SLICES - 1);  // width of the last one (64 or 48)
-    // staging tiles per epilogue warp: 2 = the warp's whole share of a tile (accumulator released before any
-    // store is issued); 1 = one slice at a time
-    static constexpr int EPI_TPW = 1;
     // The ring's depth decides how well the operand feed rides out latency (240-wide tiles: 4 / 5 / 6 stages =
     // 112.6 / 109.5 / 106.6 us per QKV step), so the staging tiles give way to it: where staging 16 rows at a time
     // (two stores per slice) instead of 32 buys another stage, it is done.
     static constexpr int SMEM_BUDGET = 227 * 1024 - 1024 /*alignment slack*/ - 256 /*barriers*/;
-    static constexpr int EPI_FULL = EPI_WARPS * EPI_TPW * EPI_TILE_BYTES;
+    static constexpr int EPI_FULL = EPI_WARPS * EPI_TILE_BYTES;   // one 32 x 64 staging tile per epilogue warp
     static constexpr int EPI_HALVES = ((SMEM_BUDGET - EPI_FULL / 2) / STAGE_BYTES > (SMEM_BUDGET - EPI_FULL) / STAGE_BYTES) ? 2 : 1;
     static constexpr int EPI_BYTES = EPI_FULL / EPI_HALVES;
     static constexpr int STAGES = ((SMEM_BUDGET - EPI_BYTES) / STAGE_BYTES) / LANES * LANES;
@@ -366,18 +363,16 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
     } else {
         // ---------------------------------------------------------------- epilogue (both CTAs)
         // Two warps per TMEM lane quarter (32 accumulator rows), each draining every other 64-column
-        // slice: TMEM -> registers -> bf16 -> a swizzled 32 x 128-byte staging tile -> one TMA store.
-        // With two staging tiles per warp the accumulator is handed back before any store is issued;
-        // with one, stores go out slice by slice.  Either way they drain to global memory while the
-        // next tile's MMAs run.  (Per-thread global stores, 32 rows x 16 bytes per instruction, kept
-        // the memory pipe busy and stalled the next tile's MMA issue.)
+        // slice: TMEM -> registers -> bf16 -> the warp's swizzled staging tile (32 or 16 rows x 128 bytes) ->
+        // TMA store, slice by slice; the stores drain to global memory while the next tile's MMAs run.
+        // (Per-thread global stores, 32 rows x 16 bytes per instruction, kept the memory pipe busy and
+        // stalled the next tile's MMA issue.)
         const int q = warp & 3;                          // TMEM lane quarter this warp may read
         const int half = (warp - C::EPI_FIRST_WARP) >> 2;  // which of the two warps of that quarter
-        constexpr int TPW = C::EPI_TPW;
         int acc = 0;
         uint32_t acc_ph = 0;
         const uint32_t tempty0 = map_to_cta(smem_u32(&tempty_bar[0]), 0);
-        uint8_t* stage_buf = smem + STAGES * C::STAGE_BYTES + (half * 4 + q) * (TPW * EPI_TILE_BYTES / C::EPI_HALVES);
+        uint8_t* stage_buf = smem + STAGES * C::STAGE_BYTES + (half * 4 + q) * (EPI_TILE_BYTES / C::EPI_HALVES);
         for (int t = pair_id; t < total; t += num_pairs) {
             const Tile ti = tile_of(t);
             const int n0 = ti.n0;
@@ -403,11 +398,6 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
             // grouped problems: rows past the expert's end belong to the next expert and must not be written,
             // so a warp whose 32 rows straddle the end writes its staged tiles with row-masked stores
             const bool clip = sched != nullptr && wrow0 + 32 > ti.row_end;
-            if (TPW == 2) {
-                // the stores of the previous tile must be done reading the staging tiles
-                if (lane == 0) tma_store_wait_read<0>();
-                __syncwarp();
-            }
             int ord = 0;
 #pragma unroll 1
             for (int c = half; c < C::SLICES; c += EPI_WARPS / 4, ++ord) {
@@ -483,56 +473,11 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
                     }
                 }
             }
-            // accumulator drained: hand it back (before the stores when the whole share is staged)
+            // accumulator drained: hand it back
             tc_fence_before();
-            if (TPW == 2) fence_proxy_async_smem();
             __syncwarp();
-            if (lane == 0) {
-                mbar_arrive_cluster(tempty0 + (uint32_t)acc * 8u);
-                if (TPW == 2) {
-                    int o2 = 0;
-                    for (int c = half; c < C::SLICES; c += EPI_WARPS / 4, ++o2)
-                        if (!clip && n0 + c * 64 < N && !(C::LAST_W != 64 && c == C::SLICES - 1))
-                            tma_store_2d(&args.tm_y, stage_buf + o2 * EPI_TILE_BYTES, n0 + c * 64, wrow0);
-                    tma_store_commit();
-                }
-            }
+            if (lane == 0) mbar_arrive_cluster(tempty0 + (uint32_t)acc * 8u);
             __syncwarp();
-            if (clip && TPW == 2) {
-                int o2 = 0;
-                for (int c = half; c < C::SLICES; c += EPI_WARPS / 4, ++o2) {
-                    if (n0 + c * 64 >= N || (C::LAST_W != 64 && c == C::SLICES - 1)) continue;
-                    const uint8_t* buf = stage_buf + o2 * EPI_TILE_BYTES;
-                    const int j = lane & 7;
-#pragma unroll
-                    for (int rr = 0; rr < 8; ++rr) {
-                        const int rl = rr * 4 + (lane >> 3);
-                        if (wrow0 + rl < ti.row_end && n0 + c * 64 + j * 8 < N)
-                            *reinterpret_cast<uint4*>(args.Y + (int64_t)(wrow0 + rl) * args.ldy + n0 + c * 64 + j * 8) =
-                                *reinterpret_cast<const uint4*>(buf + rl * 128 + ((j ^ (rl & 7)) << 4));
-                    }
-                }
-                __syncwarp();
-            }
-            if (C::LAST_W != 64 && TPW == 2) {
-                // the 48-column last slice of a 240-wide tile: row-wise 16-byte stores from the staging tile
-                // (8 lanes per row, 4 rows per instruction), clipped at M and N
-                const int c = C::SLICES - 1;
-                if ((c & 1) == half && n0 + c * 64 < N) {
-                    const uint8_t* buf = stage_buf + (c >> 1) * EPI_TILE_BYTES;
-                    const int j = lane & 7;
-#pragma unroll
-                    for (int rr = 0; rr < 8; ++rr) {
-                        const int rl = rr * 4 + (lane >> 3);
-                        const int orow = wrow0 + rl;
-                        const int ocol = n0 + c * 64 + j * 8;
-                        if (j < C::LAST_W / 8 && orow < ti.row_end && ocol < N)
-                            *reinterpret_cast<uint4*>(args.Y + (int64_t)orow * args.ldy + ocol) =
-                                *reinterpret_cast<const uint4*>(buf + rl * 128 + ((j ^ (rl & 7)) << 4));
-                    }
-                }
-                __syncwarp();
-            }
             if (++acc == ACC) { acc = 0; acc_ph ^= 1u; }
         }
         if (lane == 0) tma_store_wait_all<0>();
