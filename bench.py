@@ -44,9 +44,9 @@ NSETS = 4
 METRIC = "OSC linear TFLOP/s"
 
 # DRAM traffic of one dual-path GEMM launch on the bench workload: dram__bytes_read.sum (38.8 MB) +
-# dram__bytes_write.sum (59.2 MB) from the ncu capture summarised in
+# dram__bytes_write.sum (56.4 MB) from the ncu capture summarised in
 # profiles/gemm_pair_and_quant_extract_qkv_M8192.md (same workload, one launch).
-GEMM_TRAFFIC_BYTES = 98.0e6
+GEMM_TRAFFIC_BYTES = 95.2e6
 
 
 def load_peaks():
