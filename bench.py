@@ -424,6 +424,8 @@ def run_gpu(args):
             "unit": "TFLOP/s", "frac": gemm_tflops / p_mix, "traffic": GEMM_TRAFFIC_BYTES,
             "peak_basis": f"{pk['source']} bf16 {pk['bf16_tflops']} TFLOP/s x4 for FP4 (burst), FLOP-mix weighted",
             "ms": tg_loop, "timing": "average over back-to-back launches between two events, rotating buffer sets",
+            "frac_of_sustained_peak": (gemm_tflops / (p_mix * pk["bf16_tflops_sustained"] / pk["bf16_tflops"])
+                                       if pk.get("bf16_tflops_sustained") else None),
             "ms_between_events_inside_the_step": tg}
     qbytes = roofline.quantize_extract_bytes(M, K, Kop)
     t_roof = roofline.osc_roofline_seconds(M, N, K, Ko, peaks)
