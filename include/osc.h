@@ -35,20 +35,22 @@
  *   meta     : uint32 mask[K/32], int32 prefix[K/32], int32 idx_o[K_o] (device copy of the table).
  *   x8 / w8  : E4M3 bytes [rows, K]; sx / sw: fp32 per-row scales (amax/448).
  *
- * Variants beyond the paper's main path, each in its own section below: the MXFP8 form of the fallback,
- * the NVFP4 / G = 16 form of the OSC path, the dynamic-protection control group of Section 4.2 (a measured
- * baseline), offline profiling (Algorithm 1), and osc_linear_static (a deployment aid).
+ * Beyond the paper's main path, each in its own section below: the quantizers fused into their producers
+ * (RMSNorm + Algorithm 2, SwiGLU + per-token FP8), the grouped form with the MoE dispatch fused behind the
+ * quantizer, the MXFP8 form of the fallback, the NVFP4 / G = 16 form of the OSC path, the dynamic-protection
+ * control group of Section 4.2 (a measured baseline), offline profiling (Algorithm 1), and osc_linear_static
+ * (a deployment aid).
  *
- * Kernel selection is internal and depends only on the shape: few rows (M <= 32; <= 64 for layers with
- * more 128-feature tiles than SMs or a long K loop; <= 256 for long K loops with few tiles) run on a weight-streaming kernel with the operands swapped
- * and K split over a thread-block cluster; grouped problems with large experts and dense problems with many
- * tiles on 256-row CTA-pair tiles; the rest (up to 128 rows, small experts, and dense problems whose 128-row
- * tiles fit in one wave and beat the pair kernel's estimate) on 128-row tiles.  Results of different kernels for
- * the same inputs agree within
- * the accumulation-order rounding of fp32, not bit for bit; one kernel is deterministic run to run.
+ * Kernel selection is internal and depends only on the shape.  Few rows (M <= 32; <= 64 for layers with more
+ * 128-feature tiles than SMs or a long K loop; <= 256 for long K loops with few tiles) run on a
+ * weight-streaming kernel with the operands swapped and K split over a thread-block cluster; grouped problems
+ * with large experts and dense problems with many tiles on 256-row CTA-pair tiles; the rest (up to 128 rows,
+ * small experts, and dense problems whose 128-row tiles fit in one wave and beat the pair kernel's estimate) on
+ * 128-row tiles.  Results of different kernels for the same inputs agree within the accumulation-order rounding
+ * of fp32, not bit for bit; one kernel is deterministic run to run.
  * Environment variables for experiments (read by the library, not part of the contract): OSC_DECODE (0 = never,
- * 2 = always up to 256 rows), OSC_DECODE_SPLIT, OSC_PAIR (0 = 128-row tiles only, 2 = pair tiles whenever eligible), OSC_PAIR_BLOCK_N, OSC_BLOCK_N,
- * OSC_LOG.
+ * 2 = always up to 256 rows), OSC_DECODE_SPLIT, OSC_PAIR (0 = 128-row tiles only, 2 = pair tiles whenever
+ * eligible), OSC_PAIR_BLOCK_N, OSC_BLOCK_N, OSC_LOG.
  */
 #ifndef OSC_H_
 #define OSC_H_
