@@ -211,9 +211,11 @@ quant_extract_kernel(const __grid_constant__ CUtensorMap tm_x, int M, int K,
             int code = 0;
             if (r < row_end) {  // rows past the end (next expert / padding) count as zeros: code 0, nothing stored
                 // amax on the bf16 magnitudes, two at a time
-                __nv_bfloat162 m2 = __habs2(as_bf162(w[0]));
+                __nv_bfloat162 m8[8];   // a tree, not a chain of sixteen: the thread has little else to overlap it with
 #pragma unroll
-                for (int i = 1; i < 16; ++i) m2 = __hmax2(m2, __habs2(as_bf162(w[i])));
+                for (int i = 0; i < 8; ++i) m8[i] = __hmax2(__habs2(as_bf162(w[2 * i])), __habs2(as_bf162(w[2 * i + 1])));
+                const __nv_bfloat162 m2 = __hmax2(__hmax2(__hmax2(m8[0], m8[1]), __hmax2(m8[2], m8[3])),
+                                                  __hmax2(__hmax2(m8[4], m8[5]), __hmax2(m8[6], m8[7])));
                 const uint32_t am2 = bf162_bits(m2);
                 const uint32_t am = max(am2 & 0xFFFFu, am2 >> 16);
                 // CalculateScale: E8M0 code = biased exponent of amax - 2, floored at 0 (2^(floor(log2 amax) - 2))
