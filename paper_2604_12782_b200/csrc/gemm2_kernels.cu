@@ -368,6 +368,7 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
         // (Per-thread global stores, 32 rows x 16 bytes per instruction, kept the memory pipe busy and
         // stalled the next tile's MMA issue.)
         const int q = warp & 3;                          // TMEM lane quarter this warp may read
+        const uint64_t y_policy = l2_policy_evict_first();
         const int half = (warp - C::EPI_FIRST_WARP) >> 2;  // which of the two warps of that quarter
         int acc = 0;
         uint32_t acc_ph = 0;
@@ -454,7 +455,7 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
                         const int prow0 = wrow0 + hh * RPH;   // first output row of this pass
                         if (!clip && !narrow) {
                             if (lane == 0) {
-                                tma_store_2d(HV == 1 ? &args.tm_y : &args.tm_y16, buf, col, prow0);
+                                tma_store_2d_hint(HV == 1 ? &args.tm_y : &args.tm_y16, buf, col, prow0, y_policy);
                                 tma_store_commit();
                             }
                         } else {
