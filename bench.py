@@ -861,7 +861,7 @@ def run_sweep(args):
                  "tflops": roofline.fp8_flops(Mt, N, K) / ms / 1e9, "pct_roofline": 100 * troof / (ms * 1e-3),
                  "roof_us": troof * 1e6})
 
-    out_dir = os.environ.get("OSC_BENCH_OUT", os.path.join(ROOT, "gpurun_out"))
+    out_dir = os.environ.get("OSC_BENCH_OUT", os.path.join(ROOT, "bench_out"))
     os.makedirs(out_dir, exist_ok=True)
     with open(os.path.join(out_dir, "sweep.json"), "w") as f:
         json.dump({"peaks": pk, "rows": rows}, f, indent=1)
