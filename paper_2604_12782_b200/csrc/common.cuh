@@ -104,6 +104,7 @@ struct GemmArgs {
     const int32_t* sched2; // grouped tile schedule of the CTA-pair kernel (256-row tiles) or nullptr
     int max_tiles2;
     int num_sms;
+    int band;            // CTA-pair kernel: 256-row tiles per scheduling band (set by its launcher)
 };
 cudaError_t launch_gemm_dual(const GemmArgs& a, int bn, cudaStream_t st);
 cudaError_t launch_gemm_fp8(const GemmArgs& a, int bn, cudaStream_t st);
