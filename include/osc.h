@@ -168,12 +168,13 @@ osc_status osc_linear_static(const osc_weights* w, const void* X, int M, int64_t
  * QKV and gate/up projections of a decoder layer that operator is an RMSNorm.  These calls read the residual
  * stream H once and never write the normalized tensor:
  *
- *   r_m = 1 / sqrt( (1/K) sum_k H[m,k]^2 + eps ),   X[m,k] = bf16( (H[m,k] * r_m) * gamma[k] )
+ *   r_m = fl32( 1 / sqrt( (1/K) sum_k H[m,k]^2 + eps ) ),   X[m,k] = bf16( fl32( fl32( H[m,k] * r_m ) * gamma[k] ) )
  *
- * with the squares, the sum, the division, the square root and the two multiplications in IEEE double and one
- * rounding (nearest, ties to even) to bf16; Algorithm 2 then runs on X as in osc_quantize_extract.
+ * the statistic in IEEE double (squares exact, the sum accumulated in double, division and square root in
+ * double, then one rounding to fp32), the element-wise part as two fp32 multiplications and one rounding
+ * (nearest, ties to even) to bf16; Algorithm 2 then runs on X as in osc_quantize_extract.
  *   H      dev bf16 [M, ldh] (ldh >= K, multiple of 8, 16-byte aligned); gamma dev bf16 [K], 16-byte aligned.
- *   K <= 8192 (a row is held in registers), else OSC_ERR_SHAPE.  Dense weights only.
+ *   K <= 8192 (a row is staged in shared memory), else OSC_ERR_SHAPE.  Dense weights only.
  * osc_rmsnorm writes X itself (dev bf16 [M, ldx]): the unfused reference point for tests and measurements.
  * osc_rmsnorm_quantize_extract's outputs equal osc_quantize_extract's on osc_rmsnorm's X bit for bit.
  * osc_rmsnorm_linear = osc_rmsnorm_quantize_extract + osc_gemm_dual through the workspace of osc_act_sizes.

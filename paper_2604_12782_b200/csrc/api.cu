@@ -538,7 +538,7 @@ osc_status osc_rmsnorm(const void* H, int M, int K, int64_t ldh, const void* gam
                        void* stream) {
     if (M < 0) return fail(OSC_ERR_INVALID_ARG, "M = %d is negative", M);
     if (K <= 0 || K % 128) return fail(OSC_ERR_SHAPE, "K = %d must be a positive multiple of 128", K);
-    if (K > 8192) return fail(OSC_ERR_SHAPE, "K = %d: the fused RMSNorm holds a row in registers, K <= 8192", K);
+    if (K > 8192) return fail(OSC_ERR_SHAPE, "K = %d: the fused RMSNorm stages a row in shared memory, K <= 8192", K);
     if (M == 0) return OSC_OK;
     if (!H || !gamma || !X) return fail(OSC_ERR_INVALID_ARG, "null device pointer");
     if (ldh < K || ldx < K) return fail(OSC_ERR_SHAPE, "ldh = %lld, ldx = %lld < K = %d", (long long)ldh, (long long)ldx, K);
@@ -553,7 +553,7 @@ osc_status osc_rmsnorm(const void* H, int M, int K, int64_t ldh, const void* gam
 static osc_status rmsnorm_quantize_impl(const osc_weights* w, const void* H, int M, int64_t ldh, const void* gamma,
                                         float eps, void* xq, void* sfa, void* xo, cudaStream_t st) {
     if (w->grouped) return fail(OSC_ERR_INVALID_ARG, "grouped weights are not supported by the fused RMSNorm");
-    if (w->K > 8192) return fail(OSC_ERR_SHAPE, "K = %d: the fused RMSNorm holds a row in registers, K <= 8192", w->K);
+    if (w->K > 8192) return fail(OSC_ERR_SHAPE, "K = %d: the fused RMSNorm stages a row in shared memory, K <= 8192", w->K);
     if (M == 0) return OSC_OK;
     if (!gamma || !aligned16(gamma)) return fail(OSC_ERR_ALIGN, "gamma must be non-null and 16-byte aligned");
     if (!xq || !sfa || (w->Kop > 0 && !xo)) return fail(OSC_ERR_INVALID_ARG, "null output pointer");
