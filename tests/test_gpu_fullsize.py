@@ -150,3 +150,116 @@ def test_moe_grouped_full_size(B, oracle):
         Yref, T = oracle.fp8_gemm(x8, sx, q[key][0], q[key][1], np.array([r], np.int32))
         assert_within_tolerance(Y2h[i:i + 1], Yref, T, f"moe down row {r} expert {e}")
     assert not torch.isnan(Y2.float()).any()
+
+
+# ---- more than 2^31 elements in one activation matrix --------------------------------------------------------
+
+BIG_K = 4096
+BIG_M = (1 << 19) + 77            # M * K = 2^31 + 315392 elements; the FP8 code matrix alone exceeds 2^31 bytes
+BIG_BASE = 5000                   # distinct rows, repeated: 2^31 / K = 524288 is not a multiple of 5000, so a row
+                                  # offset that wrapped at 32 bits would land on a different base row
+
+
+def big_rows():
+    wrap = (1 << 31) // BIG_K
+    edge = [0, 127, 128, BIG_BASE - 1, BIG_BASE, wrap - 1, wrap, wrap + 1, BIG_M - 78, BIG_M - 77, BIG_M - 1]
+    rng = np.random.default_rng(7)
+    return np.array(sorted(set(edge) | set(int(r) for r in rng.integers(0, BIG_M, size=28))), np.int64)
+
+
+def sf_positions(rows, K):
+    r = np.asarray(rows)[:, None]
+    g = np.arange(K // 32)[None, :]
+    return ((r // 128) * (K // 128) + g // 4) * 512 + (r % 32) * 16 + ((r % 128) // 32) * 4 + (g % 4)
+
+
+def repeated_rows(base_bits):
+    Xb = dev_bf16(base_bits)
+    return Xb.repeat((BIG_M + BIG_BASE - 1) // BIG_BASE, 1)[:BIG_M]
+
+
+@pytest.mark.parametrize("which", ["osc", "fp8", "mxfp8"])
+def test_more_than_2_31_elements(B, oracle, which):
+    """Row offsets are 64-bit everywhere: sampled rows on both sides of the 2^31-element mark, and the ragged
+    last tile, match the oracle (quantizer outputs bit for bit, GEMM rows within the tolerance)."""
+    K, N, M = BIG_K, 128, BIG_M
+    rows = big_rows()
+    src = rows % BIG_BASE
+    rows_d = torch.from_numpy(rows).cuda()
+    local = np.arange(rows.size)
+    Y = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+    if which == "osc":
+        c = synth.osc_linear_case(3, BIG_BASE, K, N, 2)
+        X = repeated_rows(c["X"])
+        w = B.osc_prepare_weights(dev_bf16(c["W"]), c["lut"])
+        sz = B.osc_act_sizes(w, M)
+        ws = poison(sz.workspace_bytes)
+        B.osc_linear(w, X, Y, ws)
+        B.osc_sync_check()
+        act = oracle.quantize_extract(c["X"][src], c["lut"])
+        xq = ws[sz.xq_offset:sz.xq_offset + sz.xq_bytes].view(M, K // 2)[rows_d]
+        assert np.array_equal(host_u8(xq), act["xq"])
+        xo = ws[sz.xo_offset:sz.xo_offset + sz.xo_bytes].view(torch.int16).view(M, -1)[rows_d]
+        assert np.array_equal(host_u8(xo).view(np.uint16), act["xo"])
+        sf = ws[sz.sfa_offset:sz.sfa_offset + sz.sfa_bytes][torch.from_numpy(sf_positions(rows, K)).cuda()]
+        assert np.array_equal(host_u8(sf), act["sf"][sf_positions(local, K)])
+        Yref, T, *_ = oracle.linear(c["X"][src], c["W"], c["lut"])
+    elif which == "fp8":
+        c = synth.fp8_linear_case(3, BIG_BASE, K, N)
+        X = repeated_rows(c["X"])
+        w = B.osc_fp8_prepare_weights(dev_bf16(c["W"]))
+        sz = B.osc_fp8_act_sizes(w, M)
+        ws = poison(sz.workspace_bytes)
+        B.osc_fp8_linear(w, X, Y, ws)
+        B.osc_sync_check()
+        Yref, T, (x8, sx), _ = oracle.fp8_linear(c["X"][src], c["W"])
+        got8 = ws[sz.x8_offset:sz.x8_offset + M * K].view(M, K)[rows_d]
+        assert np.array_equal(host_u8(got8), x8)
+        gots = ws[sz.sx_offset:sz.sx_offset + 4 * M].view(torch.int32)[rows_d]
+        assert np.array_equal(host_u8(gots).view(np.uint32), sx.view(np.uint32))
+    else:
+        c = synth.fp8_linear_case(4, BIG_BASE, K, N)
+        X = repeated_rows(c["X"])
+        w = B.osc_mxfp8_prepare_weights(dev_bf16(c["W"]))
+        sz = B.osc_mxfp8_act_sizes(w, M)
+        ws = poison(sz.workspace_bytes)
+        B.osc_mxfp8_linear(w, X, Y, ws)
+        B.osc_sync_check()
+        Yref, T, (x8, sfa), _ = oracle.mxfp8_linear(c["X"][src], c["W"])
+        got8 = ws[sz.x8_offset:sz.x8_offset + M * K].view(M, K)[rows_d]
+        assert np.array_equal(host_u8(got8), x8)
+        sf = ws[sz.sfa_offset:sz.sfa_offset + sz.sfa_bytes][torch.from_numpy(sf_positions(rows, K)).cuda()]
+        assert np.array_equal(host_u8(sf), sfa[sf_positions(local, K)])
+    assert_within_tolerance(host_f64(Y[rows_d]), Yref, T, f"{which} M={M}")
+    assert not torch.isnan(Y.float()).any()
+
+
+@pytest.mark.parametrize("which", ["rmsnorm", "swiglu"])
+def test_more_than_2_31_elements_behind_a_producer(B, oracle, which):
+    """The same for the quantizers fused into their producers (the residual stream, the gate|up matrix)."""
+    M, N = BIG_M, 128
+    rows = big_rows()
+    src = rows % BIG_BASE
+    rows_d = torch.from_numpy(rows).cuda()
+    Y = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+    rng = np.random.default_rng(11)
+    if which == "rmsnorm":
+        K = BIG_K
+        c = synth.osc_linear_case(5, BIG_BASE, K, N, 2)
+        gb = synth.f32_to_bf16_bits(rng.uniform(0.5, 2.0, K).astype(np.float32))
+        w = B.osc_prepare_weights(dev_bf16(c["W"]), c["lut"])
+        ws = poison(B.osc_act_sizes(w, M).workspace_bytes)
+        B.osc_rmsnorm_linear(w, repeated_rows(c["X"]), dev_bf16(gb), 1e-6, Y, ws)
+        B.osc_sync_check()
+        Yref, T, *_ = oracle.linear(oracle.rmsnorm(c["X"][src], gb, 1e-6), c["W"], c["lut"])
+    else:
+        I = BIG_K // 2                                 # gate|up rows of 4096 columns
+        GUb = synth.f32_to_bf16_bits(rng.normal(0.0, 1.5, (BIG_BASE, 2 * I)).astype(np.float32))
+        W = synth.fp8_linear_case(3, 1, I, N)["W"]
+        w = B.osc_fp8_prepare_weights(dev_bf16(W))
+        ws = poison(B.osc_fp8_act_sizes(w, M).workspace_bytes)
+        B.osc_swiglu_fp8_linear(w, repeated_rows(GUb), Y, ws)
+        B.osc_sync_check()
+        Yref, T, *_ = oracle.fp8_linear(oracle.swiglu(GUb[src], I), W)
+    assert_within_tolerance(host_f64(Y[rows_d]), Yref, T, f"{which} M={M}")
+    assert not torch.isnan(Y.float()).any()
