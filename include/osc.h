@@ -17,6 +17,10 @@
  *     *_prepare_* and released by *_destroy.
  *   - stream is a cudaStream_t passed as void*.  All work is enqueued on it; no call
  *     synchronizes except osc_sync_check.  A failed validation launches nothing.
+ *   - Threads: calls on distinct handles (or on one handle with distinct activation buffers and workspaces)
+ *     may be made from several host threads at once; the library keeps no mutable state of its own beyond
+ *     once-only caches (driver entry point, per-device kernel attributes) that are safe to race on.  Two
+ *     calls that share a workspace must be ordered by the caller (one stream, or events).
  *   - Tensors: X bf16 [M, K] row-major (K contiguous, leading dimension ldx elements);
  *     W bf16 [N, K] row-major (the nn.Linear layout, Y = X . W^T); Y bf16 [M, N] (ldy elements).
  *   - Shape preconditions: K % 128 == 0, N % 64 == 0, M >= 0 (M == 0 is a successful no-op),

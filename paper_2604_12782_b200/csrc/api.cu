@@ -53,14 +53,14 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 static EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
+    static const EncodeTiledFn fn = [] {   // looked up once; initialisation of a local static is thread-safe
         void* p = nullptr;
         cudaDriverEntryPointQueryResult q;
         if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
             q == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(p);
-    }
+            return reinterpret_cast<EncodeTiledFn>(p);
+        return static_cast<EncodeTiledFn>(nullptr);
+    }();
     return fn;
 }
 
@@ -124,12 +124,11 @@ static osc_status make_tmap_sf(CUtensorMap* tm, const void* base, uint64_t block
 // one wave (with more, the SMs compete for the L2 feed and it is about half as fast as the pair kernel), so it is
 // only considered then.  OSC_PAIR=0: never, OSC_PAIR=2: always when eligible.
 static bool use_pair_kernel(bool grouped, int M, int E, long single_ns = 0, long pair_ns = 0, bool single_one_wave = false) {
-    static int mode = -1;
-    if (mode < 0) {
+    static const int mode = [] {
         const char* e = getenv("OSC_PAIR");
-        mode = e ? atoi(e) : 1;
-        if (mode < 0 || mode > 2) mode = 1;
-    }
+        const int v = e ? atoi(e) : 1;
+        return (v < 0 || v > 2) ? 1 : v;
+    }();
     if (mode == 0) return false;
     if (grouped) return M / E >= 96;
     if (M <= 128) return false;

@@ -4,6 +4,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "ptx.cuh"
 
 namespace osc {
@@ -29,9 +31,10 @@ static cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
 // Function attributes (the shared-memory opt-in) and occupancy answers belong to a device, not to the process:
 // every kernel instantiation keeps one of these and sets itself up once on each device it is launched on.
 constexpr int kMaxDevicesPerProcess = 64;
-struct PerDevice {
-    bool done[kMaxDevicesPerProcess] = {};
-    int value[kMaxDevicesPerProcess] = {};
+struct PerDevice {   // threads may race to fill a slot: both then store the same values, and a reader that sees
+                     // `done` also sees `value` (sequentially consistent atomics)
+    std::atomic<bool> done[kMaxDevicesPerProcess] = {};
+    std::atomic<int> value[kMaxDevicesPerProcess] = {};
 };
 // index of the current device in a PerDevice, or -1 (no caching) if it cannot be had or is out of range
 static inline int per_device_slot() {

@@ -536,7 +536,7 @@ static cudaError_t launch_cfg(const GemmArgs& a, cudaStream_t st) {
     // The kernel is persistent with static striping of tiles over pairs, so every pair must be
     // resident at once: ask how many 2-CTA clusters of this footprint the device can hold.
     const int slot = per_device_slot();
-    int max_pairs = (slot >= 0 && resident.done[slot]) ? resident.value[slot] : 0;
+    int max_pairs = (slot >= 0 && resident.done[slot]) ? resident.value[slot].load() : 0;
     if (max_pairs == 0) {
         cfg.gridDim = dim3(a.num_sms);
         int n = 0;
@@ -566,14 +566,11 @@ static cudaError_t launch_cfg(const GemmArgs& a, cudaStream_t st) {
 // than the ~2 us drain), 256 has one accumulator (drain and hand-over exposed, ~2.7 us per tile).
 // The FP8 mode needs no scale columns: 256 wide with two accumulators.  OSC_PAIR_BLOCK_N overrides.
 int gemm_pair_block_n(bool fp8, bool allow_240, long row_tiles, int N, int stages, int num_sms, long* cost_ns) {
-    static int forced = -1;
-    if (forced < 0) {
-        forced = 0;
-        if (const char* e = getenv("OSC_PAIR_BLOCK_N")) {
-            const int v = atoi(e);
-            if (v == 192 || v == 240 || v == 256) forced = v;
-        }
-    }
+    static const int forced = [] {
+        const char* e = getenv("OSC_PAIR_BLOCK_N");
+        const int v = e ? atoi(e) : 0;
+        return (v == 192 || v == 240 || v == 256) ? v : 0;
+    }();
     if (cost_ns) *cost_ns = 0;   // a forced width is never weighed against the other kernel
     if (forced && !((fp8 || !allow_240) && forced == 240)) return forced;
     const int pairs = num_sms / 2 > 0 ? num_sms / 2 : 1;

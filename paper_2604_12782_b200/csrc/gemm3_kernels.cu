@@ -409,11 +409,7 @@ static cudaError_t launch_cfg(const GemmArgs& a, int S, cudaStream_t st) {
 // a second wave (192 tiles: 15.1 / 18.1 / 23.1 us for S = 1 / 2 / 3).  Every rank gets at least one K block.
 // OSC_DECODE_SPLIT overrides.
 int gemm_decode_split(int N, int nkb, int num_sms) {
-    static int forced = -1;
-    if (forced < 0) {
-        forced = 0;
-        if (const char* e = getenv("OSC_DECODE_SPLIT")) forced = atoi(e);
-    }
+    static const int forced = [] { const char* e = getenv("OSC_DECODE_SPLIT"); return e ? atoi(e) : 0; }();
     const int tiles = (N + decode::BF - 1) / decode::BF;
     int S = 1;
     if (forced > 0) S = forced;

@@ -400,14 +400,11 @@ done:
 // tiles the widest wins (least time per column), with few a narrower one that still fits in one wave.
 // cost_ns (optional) receives the estimate for one K stage times the waves.  OSC_BLOCK_N overrides.
 int gemm_block_n(int row_tiles, int N, int num_sms, long* cost_ns) {
-    static int forced = -1;
-    if (forced < 0) {
-        forced = 0;
-        if (const char* e = getenv("OSC_BLOCK_N")) {
-            const int v = atoi(e);
-            if (v == 64 || v == 128 || v == 192 || v == 256) forced = v;
-        }
-    }
+    static const int forced = [] {
+        const char* e = getenv("OSC_BLOCK_N");
+        const int v = e ? atoi(e) : 0;
+        return (v == 64 || v == 128 || v == 192 || v == 256) ? v : 0;
+    }();
     if (cost_ns) *cost_ns = 0;
     if (forced) return forced;
     const int cand[4] = {256, 192, 128, 64};
