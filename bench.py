@@ -833,7 +833,8 @@ def run_sweep(args):
     rows.append({"name": "moe.gate_up(grouped, gathered from 8192 tokens)", "M": Mt, "K": K, "N": N, "K_o": w.K_o, "ms": msg,
                  "tflops": (f4 + f16) / msg / 1e9, "pct_roofline": 100 * troofg / (msg * 1e-3), "roof_us": troofg * 1e6,
                  "speedup_vs_permuted_input": ms / msg})
-    del Xd, Wd, w, ws, Y, wsg, Xtok
+    wg, Yg = w, Y
+    del Xd, Wd, ws
     c = synth.moe_down_case(E, counts, weight_pool=8)
     Xd = dev_bf16(torch, c["X"])
     Wd = dev_bf16(torch, c["W"].reshape(E * c["N"], c["K"])).view(E, c["N"], c["K"])
@@ -849,7 +850,27 @@ def run_sweep(args):
     rows.append({"name": "moe.down_fp8(grouped)", "M": Mt, "K": K, "N": N, "ms": ms,
                  "tflops": roofline.fp8_flops(Mt, N, K) / ms / 1e9, "pct_roofline": 100 * troof / (ms * 1e-3),
                  "roof_us": troof * 1e6})
-    del w, ws
+    # the expert layer with its producers: RMSNorm of the 8192 tokens fused into the quantizer in front of the gather,
+    # SwiGLU of the experts' gate|up rows fused into the FP8 quantizer in front of the down projection (I = 768)
+    gamma = torch.ones(wg.K, dtype=torch.bfloat16, device="cuda")
+    Xn = torch.empty_like(Xtok)
+    Hh = torch.empty(Mt, K, dtype=torch.bfloat16, device="cuda")
+
+    def moe_fused(i):
+        B.osc_rmsnorm_linear_grouped_gather(wg, Xtok, gamma, 1e-6, row_token, off, Yg, wsg)
+        B.osc_swiglu_fp8_linear_grouped(w, Yg, off, Y, ws)
+
+    def moe_separate(i):
+        B.osc_rmsnorm(Xtok, gamma, 1e-6, Xn)
+        B.osc_linear_grouped_gather(wg, Xn, row_token, off, Yg, wsg)
+        B.osc_swiglu(Yg, K, Hh)
+        B.osc_fp8_linear_grouped(w, Hh, off, Y, ws)
+
+    ms_f, ms_s = time_loop(torch, moe_fused, steps, warm), time_loop(torch, moe_separate, steps, warm)
+    B.osc_sync_check()
+    rows.append({"name": "moe.layer.fused(rmsnorm+gather+gate_up, swiglu+down_fp8)", "M": Mt, "ms": ms_f,
+                 "separate_kernels_ms": ms_s, "speedup": ms_s / ms_f})
+    del w, ws, wg, Yg, wsg, Xtok, Xn, Hh
     w = B.osc_mxfp8_prepare_weights_grouped(Wd)
     sz = B.osc_mxfp8_act_sizes(w, c["M"])
     ws = torch.empty(sz.workspace_bytes, dtype=torch.uint8, device="cuda")

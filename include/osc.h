@@ -211,6 +211,13 @@ osc_status osc_linear_grouped_gather(const osc_weights* w, const void* X, int T,
                                      const int32_t* off, int M_total, void* Y, int64_t ldy, void* workspace,
                                      size_t workspace_bytes, void* stream);
 
+/* The same behind an RMSNorm (the router's tokens come straight from the residual stream H, dev bf16 [T, ldh]):
+ * osc_rmsnorm_quantize_extract's kernel on the T tokens, then the gather.  Equals osc_linear_grouped_gather on
+ * osc_rmsnorm's output bit for bit; K <= 8192; workspace as above. */
+osc_status osc_rmsnorm_linear_grouped_gather(const osc_weights* w, const void* H, int T, int64_t ldh, const void* gamma,
+                                             float eps, const int32_t* row_token, const int32_t* off, int M_total, void* Y,
+                                             int64_t ldy, void* workspace, size_t workspace_bytes, void* stream);
+
 /* ---------------------------------------------------- offline profiling */
 
 /* Scratch bytes osc_profile_lut needs for a K-channel slice (an fp64 sum and 32 counters per group). */
@@ -287,6 +294,12 @@ osc_status osc_swiglu(const void* GU, int M, int I, int64_t ldg, void* H, int64_
 osc_status osc_swiglu_fp8_quantize(const void* GU, int M, int I, int64_t ldg, void* x8, void* sx, void* stream);
 osc_status osc_swiglu_fp8_linear(const osc_fp8_weights* w, const void* GU, int M, int64_t ldg, void* Y, int64_t ldy,
                                  void* workspace, size_t workspace_bytes, void* stream);
+/* Grouped (MoE) form: rows of GU_perm (dev bf16 [M_total, ldg], the experts' gate|up outputs) sorted by expert as in
+ * osc_fp8_linear_grouped; the per-token quantizer does not depend on the expert, so this is
+ * osc_swiglu_fp8_quantize on all rows + the grouped FP8 GEMM.  Workspace: osc_fp8_act_sizes(w, M_total). */
+osc_status osc_swiglu_fp8_linear_grouped(const osc_fp8_weights* w, const void* GU_perm, const int32_t* off, int M_total,
+                                         int64_t ldg, void* Y, int64_t ldy, void* workspace, size_t workspace_bytes,
+                                         void* stream);
 
 /* ------------------------------------- MXFP8 form of the fallback (Section 3.4) */
 

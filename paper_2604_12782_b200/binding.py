@@ -78,6 +78,8 @@ _SIGS = {
     "osc_linear_grouped": (_i, [_vp, _vp, _vp, _i, _i64, _vp, _i64, _vp, _sz, _vp]),
     "osc_gather_workspace_bytes": (_i, [_vp, _i, _i, C.POINTER(_sz)]),
     "osc_linear_grouped_gather": (_i, [_vp, _vp, _i, _i64, _vp, _vp, _i, _vp, _i64, _vp, _sz, _vp]),
+    "osc_rmsnorm_linear_grouped_gather": (_i, [_vp, _vp, _i, _i64, _vp, C.c_float, _vp, _vp, _i, _vp, _i64, _vp, _sz, _vp]),
+    "osc_swiglu_fp8_linear_grouped": (_i, [_vp, _vp, _vp, _i, _i64, _vp, _i64, _vp, _sz, _vp]),
     "osc_rmsnorm": (_i, [_vp, _i, _i, _i64, _vp, C.c_float, _vp, _i64, _vp]),
     "osc_swiglu": (_i, [_vp, _i, _i, _i64, _vp, _i64, _vp]),
     "osc_swiglu_fp8_quantize": (_i, [_vp, _i, _i, _i64, _vp, _vp, _vp]),
@@ -285,8 +287,19 @@ def osc_linear_grouped_gather(w: OscWeights, X: torch.Tensor, row_token: torch.T
                                           workspace.numel() * workspace.element_size(), _stream(stream)))
 
 
+def osc_rmsnorm_linear_grouped_gather(w: OscWeights, H: torch.Tensor, gamma: torch.Tensor, eps: float, row_token: torch.Tensor,
+                                      off: torch.Tensor, Y: torch.Tensor, workspace: torch.Tensor, stream=None):
+    """osc_linear_grouped_gather with the RMSNorm of the residual stream H fused into the quantizer."""
+    T, M = H.shape[0], row_token.shape[0]
+    _check(_lib.osc_rmsnorm_linear_grouped_gather(w.ptr, _ptr(H), T, H.stride(0) if T else w.K, _ptr(gamma), float(eps),
+                                                  _ptr(row_token), _ptr(off), M, _ptr(Y), Y.stride(0) if M else w.N,
+                                                  _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                                  _stream(stream)))
+
+
 def osc_rmsnorm(H: torch.Tensor, gamma: torch.Tensor, eps: float, X: torch.Tensor, stream=None):
-    """X = bf16(RMSNorm(H) * gamma), double arithmetic with one rounding: the unfused reference point."""
+    """X = bf16(RMSNorm(H) * gamma) (statistic in double, element-wise part in fp32, one rounding to bf16):
+    the unfused reference point."""
     M, K = H.shape
     _check(_lib.osc_rmsnorm(_ptr(H), M, K, H.stride(0) if M else K, _ptr(gamma), float(eps), _ptr(X),
                             X.stride(0) if M else K, _stream(stream)))
@@ -324,6 +337,15 @@ def osc_swiglu_fp8_linear(w: "Fp8Weights", GU: torch.Tensor, Y: torch.Tensor, wo
     _check(_lib.osc_swiglu_fp8_linear(w.ptr, _ptr(GU), M, GU.stride(0) if M else 2 * w.K, _ptr(Y),
                                       Y.stride(0) if M else w.N, _ptr(workspace),
                                       workspace.numel() * workspace.element_size(), _stream(stream)))
+
+
+def osc_swiglu_fp8_linear_grouped(w: "Fp8Weights", GU: torch.Tensor, off: torch.Tensor, Y: torch.Tensor,
+                                  workspace: torch.Tensor, stream=None):
+    """Grouped FP8 linear on silu(gate) * up of the experts' gate|up rows, the activation never written."""
+    M = GU.shape[0]
+    _check(_lib.osc_swiglu_fp8_linear_grouped(w.ptr, _ptr(GU), _ptr(off), M, GU.stride(0) if M else 2 * w.K, _ptr(Y),
+                                              Y.stride(0) if M else w.N, _ptr(workspace),
+                                              workspace.numel() * workspace.element_size(), _stream(stream)))
 
 
 def osc_linear_grouped(w: OscWeights, X: torch.Tensor, off: torch.Tensor, Y: torch.Tensor, workspace: torch.Tensor,

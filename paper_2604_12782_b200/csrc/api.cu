@@ -551,7 +551,6 @@ osc_status osc_rmsnorm(const void* H, int M, int K, int64_t ldh, const void* gam
 
 static osc_status rmsnorm_quantize_impl(const osc_weights* w, const void* H, int M, int64_t ldh, const void* gamma,
                                         float eps, void* xq, void* sfa, void* xo, cudaStream_t st) {
-    if (w->grouped) return fail(OSC_ERR_INVALID_ARG, "grouped weights are not supported by the fused RMSNorm");
     if (w->K > 8192) return fail(OSC_ERR_SHAPE, "K = %d: the fused RMSNorm stages a row in shared memory, K <= 8192", w->K);
     if (M == 0) return OSC_OK;
     if (!gamma || !aligned16(gamma)) return fail(OSC_ERR_ALIGN, "gamma must be non-null and 16-byte aligned");
@@ -566,13 +565,14 @@ static osc_status rmsnorm_quantize_impl(const osc_weights* w, const void* H, int
 osc_status osc_rmsnorm_quantize_extract(const osc_weights* w, const void* H, int M, int64_t ldh, const void* gamma,
                                         float eps, void* xq, void* sfa, void* xo, void* stream) {
     if (osc_status s = check_act(w, H, M, ldh)) return s;
+    if (w->grouped) return fail(OSC_ERR_INVALID_ARG, "grouped weights: use osc_rmsnorm_linear_grouped_gather");
     return rmsnorm_quantize_impl(w, H, M, ldh, gamma, eps, xq, sfa, xo, static_cast<cudaStream_t>(stream));
 }
 
 osc_status osc_rmsnorm_linear(const osc_weights* w, const void* H, int M, int64_t ldh, const void* gamma, float eps,
                               void* Y, int64_t ldy, void* workspace, size_t workspace_bytes, void* stream) {
     if (osc_status s = check_act(w, H, M, ldh)) return s;
-    if (w->grouped) return fail(OSC_ERR_INVALID_ARG, "grouped weights are not supported by the fused RMSNorm");
+    if (w->grouped) return fail(OSC_ERR_INVALID_ARG, "grouped weights: use osc_rmsnorm_linear_grouped_gather");
     if (M == 0) return OSC_OK;
     osc_act_sizes_t sz;
     osc_act_sizes(w, M, &sz);
@@ -640,9 +640,10 @@ osc_status osc_gather_workspace_bytes(const osc_weights* w, int T, int M_total, 
     return OSC_OK;
 }
 
-osc_status osc_linear_grouped_gather(const osc_weights* w, const void* X, int T, int64_t ldx, const int32_t* row_token,
-                                     const int32_t* off, int M_total, void* Y, int64_t ldy, void* workspace,
-                                     size_t workspace_bytes, void* stream) {
+// gamma == nullptr: X holds the activations; else X is the residual stream and the RMSNorm runs inside the quantizer
+static osc_status grouped_gather_impl(const osc_weights* w, const void* X, int T, int64_t ldx, const void* gamma, float eps,
+                                      const int32_t* row_token, const int32_t* off, int M_total, void* Y, int64_t ldy,
+                                      void* workspace, size_t workspace_bytes, void* stream) {
     if (osc_status s = check_act(w, X, T, ldx)) return s;
     if (!w->grouped) return fail(OSC_ERR_INVALID_ARG, "dense weights: use osc_linear");
     if (M_total < 0) return fail(OSC_ERR_INVALID_ARG, "M_total = %d is negative", M_total);
@@ -667,12 +668,29 @@ osc_status osc_linear_grouped_gather(const osc_weights* w, const void* X, int T,
     cudaError_t e = launch_build_sched(off, w->E, sched, max_tiles, sched2, max_tiles2, st);
     if (e != cudaSuccess) return cuda_fail(e, "build_sched_kernel");
     // Algorithm 2 once per token (it does not depend on the expert), as a dense problem of T rows
-    if (osc_status s = quantize_impl(w, X, T, ldx, ws + g.xq_u, ws + g.sf_u, ws + g.xo_u, nullptr, 0, st)) return s;
+    if (gamma) {
+        if (osc_status s = rmsnorm_quantize_impl(w, X, T, ldx, gamma, eps, ws + g.xq_u, ws + g.sf_u, ws + g.xo_u, st)) return s;
+    } else {
+        if (osc_status s = quantize_impl(w, X, T, ldx, ws + g.xq_u, ws + g.sf_u, ws + g.xo_u, nullptr, 0, st)) return s;
+    }
     e = launch_gather_quantized(row_token, T, w->K, w->Kop, ws + g.xq_u, ws + g.sf_u, ws + g.xo_u, ws + sz.xq_offset,
                                 ws + sz.sfa_offset, ws + sz.xo_offset, sched, max_tiles, st);
     if (e != cudaSuccess) return cuda_fail(e, "gather_quantized_kernel");
     return gemm_impl(w, ws + sz.xq_offset, ws + sz.sfa_offset, ws + sz.xo_offset, M_total, Y, ldy, sched, max_tiles,
                      sched2, max_tiles2, st);
+}
+
+osc_status osc_linear_grouped_gather(const osc_weights* w, const void* X, int T, int64_t ldx, const int32_t* row_token,
+                                     const int32_t* off, int M_total, void* Y, int64_t ldy, void* workspace,
+                                     size_t workspace_bytes, void* stream) {
+    return grouped_gather_impl(w, X, T, ldx, nullptr, 0.0f, row_token, off, M_total, Y, ldy, workspace, workspace_bytes, stream);
+}
+
+osc_status osc_rmsnorm_linear_grouped_gather(const osc_weights* w, const void* H, int T, int64_t ldh, const void* gamma,
+                                             float eps, const int32_t* row_token, const int32_t* off, int M_total, void* Y,
+                                             int64_t ldy, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!gamma) return fail(OSC_ERR_INVALID_ARG, "gamma is null");
+    return grouped_gather_impl(w, H, T, ldh, gamma, eps, row_token, off, M_total, Y, ldy, workspace, workspace_bytes, stream);
 }
 
 // ------------------------------------------------------- offline profiling
@@ -837,12 +855,24 @@ osc_status osc_fp8_gemm(const osc_fp8_weights* w, const void* x8, const void* sx
     return fp8_gemm_impl(w, x8, sx, M, Y, ldy, nullptr, 0, nullptr, 0, static_cast<cudaStream_t>(stream));
 }
 
+static osc_status check_swiglu(const void* GU, int M, int I, int64_t ldg);
+
+// swiglu: X is the gate|up matrix [M, 2K] and the quantizer computes the activation on the way in
 static osc_status fp8_linear_impl(const osc_fp8_weights* w, const void* X, const int32_t* off, int M, int64_t ldx,
-                                  void* Y, int64_t ldy, void* workspace, size_t workspace_bytes, void* stream) {
+                                  void* Y, int64_t ldy, void* workspace, size_t workspace_bytes, void* stream,
+                                  bool swiglu = false) {
     if (!w) return fail(OSC_ERR_INVALID_ARG, "weights handle is null");
+    if (swiglu) {
+        if (osc_status s = check_swiglu(X, M, w->K, ldx)) return s;
+    }
     if (M < 0) return fail(OSC_ERR_INVALID_ARG, "M = %d is negative", M);
     if (M == 0) return OSC_OK;
     if (w->grouped && !off) return fail(OSC_ERR_INVALID_ARG, "off is null");
+    if (!swiglu) {   // what osc_fp8_quantize would refuse, refused before the schedule builder is launched
+        if (!X) return fail(OSC_ERR_INVALID_ARG, "X is null");
+        if (ldx < w->K) return fail(OSC_ERR_SHAPE, "ldx = %lld < K", (long long)ldx);
+        if (ldx % 8 || !aligned16(X)) return fail(OSC_ERR_ALIGN, "X must be 16-byte aligned and ldx a multiple of 8");
+    }
     osc_fp8_act_sizes_t sz;
     osc_fp8_act_sizes(w, M, &sz);
     if (!workspace || !aligned16(workspace)) return fail(OSC_ERR_ALIGN, "workspace must be non-null and 16-byte aligned");
@@ -863,7 +893,11 @@ static osc_status fp8_linear_impl(const osc_fp8_weights* w, const void* X, const
         if (e != cudaSuccess) return cuda_fail(e, "build_sched_kernel");
         if (pair) sched2 = s + sched_ints(max_tiles); else sched = s;
     }
-    if (osc_status s = osc_fp8_quantize(X, M, w->K, ldx, ws + sz.x8_offset, ws + sz.sx_offset, stream)) return s;
+    if (swiglu) {
+        if (osc_status s = osc_swiglu_fp8_quantize(X, M, w->K, ldx, ws + sz.x8_offset, ws + sz.sx_offset, stream)) return s;
+    } else {
+        if (osc_status s = osc_fp8_quantize(X, M, w->K, ldx, ws + sz.x8_offset, ws + sz.sx_offset, stream)) return s;
+    }
     return fp8_gemm_impl(w, ws + sz.x8_offset, ws + sz.sx_offset, M, Y, ldy, sched, max_tiles, sched2, max_tiles2, st);
 }
 
@@ -913,19 +947,14 @@ osc_status osc_swiglu_fp8_quantize(const void* GU, int M, int I, int64_t ldg, vo
 
 osc_status osc_swiglu_fp8_linear(const osc_fp8_weights* w, const void* GU, int M, int64_t ldg, void* Y, int64_t ldy,
                                  void* workspace, size_t workspace_bytes, void* stream) {
-    if (!w) return fail(OSC_ERR_INVALID_ARG, "weights handle is null");
-    if (w->grouped) return fail(OSC_ERR_INVALID_ARG, "grouped weights are not supported by the fused SwiGLU");
-    if (osc_status s = check_swiglu(GU, M, w->K, ldg)) return s;
-    if (M == 0) return OSC_OK;
-    osc_fp8_act_sizes_t sz;
-    osc_fp8_act_sizes(w, M, &sz);
-    if (!workspace || !aligned16(workspace)) return fail(OSC_ERR_ALIGN, "workspace must be non-null and 16-byte aligned");
-    if (workspace_bytes < sz.workspace_bytes)
-        return fail(OSC_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", workspace_bytes, sz.workspace_bytes);
-    uint8_t* ws = static_cast<uint8_t*>(workspace);
-    if (osc_status s = osc_swiglu_fp8_quantize(GU, M, w->K, ldg, ws + sz.x8_offset, ws + sz.sx_offset, stream)) return s;
-    return fp8_gemm_impl(w, ws + sz.x8_offset, ws + sz.sx_offset, M, Y, ldy, nullptr, 0, nullptr, 0,
-                         static_cast<cudaStream_t>(stream));
+    if (w && w->grouped) return fail(OSC_ERR_INVALID_ARG, "grouped weights: use osc_swiglu_fp8_linear_grouped");
+    return fp8_linear_impl(w, GU, nullptr, M, ldg, Y, ldy, workspace, workspace_bytes, stream, true);
+}
+osc_status osc_swiglu_fp8_linear_grouped(const osc_fp8_weights* w, const void* GU_perm, const int32_t* off, int M_total,
+                                         int64_t ldg, void* Y, int64_t ldy, void* workspace, size_t workspace_bytes,
+                                         void* stream) {
+    if (w && !w->grouped) return fail(OSC_ERR_INVALID_ARG, "dense weights: use osc_swiglu_fp8_linear");
+    return fp8_linear_impl(w, GU_perm, off, M_total, ldg, Y, ldy, workspace, workspace_bytes, stream, true);
 }
 
 // ------------------------------------------------- MXFP8 form of the fallback

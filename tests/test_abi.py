@@ -109,3 +109,11 @@ def test_producer_fusions_validate_before_launching(B):
     assert sq(0x1000, 4, 128, 256, 0x2004, 0x3000, None) == -4
     assert lib.osc_rmsnorm_linear(None, None, 0, 0, None, C.c_float(0), None, 0, None, 0, None) == -1
     assert lib.osc_swiglu_fp8_linear(None, None, 0, 0, None, 0, None, 0, None) == -1
+
+
+def test_grouped_fused_calls_refuse_null_handles():
+    from paper_2604_12782_b200 import binding as B
+    lib = B._lib
+    assert lib.osc_swiglu_fp8_linear_grouped(None, None, None, 0, 0, None, 0, None, 0, None) == -1
+    assert lib.osc_rmsnorm_linear_grouped_gather(None, None, 0, 0, None, C.c_float(0), None, None, 0, None, 0, None, 0,
+                                                 None) == -1

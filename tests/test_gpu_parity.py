@@ -393,3 +393,75 @@ def test_grouped_gather_equals_grouped_on_permuted_rows(B, oracle, kind):
     with pytest.raises(B.OscError) as err:
         B.osc_linear_grouped_gather(w, dev_bf16(Xtok), torch.from_numpy(row_token).cuda(), off, Yb, ws_b[:sz.workspace_bytes])
     assert err.value.status == -5
+
+
+@pytest.mark.parametrize("kind", ["small", "mid"])
+def test_rmsnorm_grouped_gather(B, oracle, kind):
+    """The dispatch-fused grouped linear behind an RMSNorm: equals the gather call on the separately normalized tokens
+    bit for bit, and the oracle (RMSNorm, Algorithm 2, Eq. 5 per expert) within tolerance."""
+    counts = grouped_counts(kind)
+    E, K, N, T = counts.size, 512, (320 if kind == "mid" else 192), 150
+    c = synth.moe_gate_up_case(E, counts, K=K, N=N, seed=6)
+    M = c["M"]
+    rng = np.random.default_rng(12)
+    Hb, _ = synth.osc_activations_only(10, T, K, 1)
+    gb = synth.f32_to_bf16_bits(rng.uniform(0.3, 2.0, K).astype(np.float32) * rng.choice([-1.0, 1.0], K).astype(np.float32))
+    row_token = rng.integers(0, T, size=M).astype(np.int32)
+    w = B.osc_prepare_weights_grouped(dev_bf16(c["W"].reshape(E * N, K)).view(E, N, K), c["lut"])
+    off, rt = torch.from_numpy(c["off"]).cuda(), torch.from_numpy(row_token).cuda()
+    nbytes = B.osc_gather_workspace_bytes(w, T, M)
+    H, g = dev_bf16(Hb), dev_bf16(gb)
+    Xn = torch.empty((T, K), dtype=torch.bfloat16, device="cuda")
+    B.osc_rmsnorm(H, g, 1e-5, Xn)
+    Ya = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+    B.osc_linear_grouped_gather(w, Xn, rt, off, Ya, poison(nbytes))
+    Yb = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+    B.osc_rmsnorm_linear_grouped_gather(w, H, g, 1e-5, rt, off, Yb, poison(nbytes))
+    B.osc_sync_check()
+    assert torch.equal(Ya.view(torch.int16), Yb.view(torch.int16))
+    Xperm = oracle.rmsnorm(Hb, gb, 1e-5)[row_token]
+    Yh = host_f64(Yb)
+    for e in range(E):
+        r0, r1 = int(c["off"][e]), int(c["off"][e + 1])
+        if r1 > r0:
+            Yref, Tb, *_ = oracle.linear(Xperm[r0:r1], c["W"][e], c["lut"])
+            assert_within_tolerance(Yh[r0:r1], Yref, Tb, f"rmsnorm + gathered grouped, expert {e}")
+    with pytest.raises(B.OscError) as err:      # dense handle
+        wd = B.osc_prepare_weights(dev_bf16(c["W"][0]), c["lut"])
+        B.osc_rmsnorm_linear_grouped_gather(wd, H, g, 1e-5, rt, off, Yb, poison(nbytes))
+    assert err.value.status == -1
+
+
+@pytest.mark.parametrize("kind", ["small", "mid"])
+def test_swiglu_fp8_grouped(B, oracle, kind):
+    """Grouped FP8 down projection on the experts' gate|up rows: equals the grouped FP8 linear on the separately
+    computed activation bit for bit, and the oracle (SwiGLU, per-token FP8, GEMM per expert) within tolerance."""
+    counts = grouped_counts(kind)
+    E, I, N = counts.size, 384, (320 if kind == "mid" else 128)
+    d = synth.moe_down_case(E, counts, K=I, N=N, seed=7)
+    M = d["M"]
+    rng = np.random.default_rng(13)
+    GUb = synth.f32_to_bf16_bits(rng.normal(0.0, 1.5, (M, 2 * I)).astype(np.float32))
+    w = B.osc_fp8_prepare_weights_grouped(dev_bf16(d["W"].reshape(E * N, I)).view(E, N, I))
+    off = torch.from_numpy(d["off"]).cuda()
+    nbytes = B.osc_fp8_act_sizes(w, M).workspace_bytes
+    GU = dev_bf16(GUb)
+    Hh = torch.empty((M, I), dtype=torch.bfloat16, device="cuda")
+    B.osc_swiglu(GU, I, Hh)
+    Ya = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+    B.osc_fp8_linear_grouped(w, Hh, off, Ya, poison(nbytes))
+    Yb = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+    B.osc_swiglu_fp8_linear_grouped(w, GU, off, Yb, poison(nbytes))
+    B.osc_sync_check()
+    assert torch.equal(Ya.view(torch.int16), Yb.view(torch.int16))
+    hb = oracle.swiglu(GUb, I)
+    Yh = host_f64(Yb)
+    for e in range(E):
+        r0, r1 = int(d["off"][e]), int(d["off"][e + 1])
+        if r1 > r0:
+            Yref, Tb, *_ = oracle.fp8_linear(hb[r0:r1], d["W"][e])
+            assert_within_tolerance(Yh[r0:r1], Yref, Tb, f"swiglu + grouped fp8, expert {e}")
+    with pytest.raises(B.OscError) as err:      # dense handle
+        wd = B.osc_fp8_prepare_weights(dev_bf16(d["W"][0]))
+        B.osc_swiglu_fp8_linear_grouped(wd, GU, off, Yb, poison(nbytes))
+    assert err.value.status == -1
