@@ -142,14 +142,16 @@ static bool use_pair_kernel(bool grouped, int M, int E, long single_ns = 0, long
 // 14.4 us), with 32 tiles and 96 stages it is behind (24.4 vs 21.9 us); up to 256 rows (its 256-token form, one
 // CTA per SM) when the K loop is long and the tiles with their K split still fit the machine, where the tile
 // kernels leave most SMs idle.  OSC_DECODE=0 disables, OSC_DECODE=2 forces it up to 256 rows.
-static bool use_decode_kernel(bool grouped, int M, int N, int nkb, int num_sms) {
+// no_row128: the format has no 128-row-tile kernel (NVFP4), so up to 64 rows the alternative is the pair kernel with
+// three quarters of its tile empty: QKV / gate_up / o_proj at 64 rows 10.9 / 19.3 / 10.5 us against 13.8 / 22.9 / 13.6.
+static bool use_decode_kernel(bool grouped, int M, int N, int nkb, int num_sms, bool no_row128 = false) {
     const char* e = getenv("OSC_DECODE");   // read per call: tests switch it inside one process
     const int mode = e ? atoi(e) : 1;
     if (mode == 0 || grouped || M > 256) return false;
     if (mode == 2) return true;
     const int tiles = (N + 127) / 128;
     if (M <= 32) return true;
-    if (M <= 64) return tiles >= num_sms || nkb >= 64;
+    if (M <= 64) return no_row128 || tiles >= num_sms || nkb >= 64;
     return nkb >= 64 && 2 * tiles <= num_sms;
 }
 
@@ -1304,6 +1306,9 @@ osc_status osc_nvfp4_prepare_weights(const void* W, int N, int K, int64_t ldw, c
             s = make_tmap(&w->tm_bo2[v], wo, true, (uint64_t)N, (uint64_t)t.Kop * 2, (uint64_t)t.Kop * 2, half);
     }
     if (s == OSC_OK) s = make_tmap_sf(&w->tm_sfw, sfw, (uint64_t)sf16_bytes(N, K) / 512, 4);
+    // 128-row weight tiles of the few-row kernel
+    if (s == OSC_OK) s = make_tmap(&w->tm_b[1], wq, false, (uint64_t)N, K / 2, K / 2, 128);
+    if (s == OSC_OK && t.Kop > 0) s = make_tmap(&w->tm_bo[1], wo, true, (uint64_t)N, (uint64_t)t.Kop * 2, (uint64_t)t.Kop * 2, 128);
     if (s != OSC_OK) { delete w; return s; }
     *out = w;
     return OSC_OK;
@@ -1354,8 +1359,28 @@ osc_status osc_nvfp4_gemm(const osc_weights* w, const void* xq, const void* sfa,
     if (es < -120 || es > 120) return fail(OSC_ERR_INVALID_ARG, "sum of the tensor exponents %d outside -120..120", es);
     GemmArgs a;
     memset(&a, 0, sizeof a);
+    const int nkb = (w->K + 255) / 256 + w->Kop / 64;
+    if (use_decode_kernel(false, M, w->N, nkb, w->num_sms, true)) {   // few rows: weights stream once, K split over a cluster
+        const uint32_t tok_box = (uint32_t)((M + 15) / 16 * 16);
+        if (osc_status s = make_tmap(&a.tm_a, xq, false, M, w->K / 2, w->K / 2, tok_box)) return s;
+        a.tm_b = w->tm_b[1];
+        if (w->Kop > 0) {
+            if (osc_status s = make_tmap(&a.tm_ao, xo, true, M, (uint64_t)w->Kop * 2, (uint64_t)w->Kop * 2, tok_box)) return s;
+            a.tm_bo = w->tm_bo[1];
+        }
+        a.sfa = static_cast<const uint8_t*>(sfa);
+        a.sfw = w->sfw;
+        a.Y = static_cast<uint16_t*>(Y);
+        a.ldy = ldy;
+        a.M = M; a.N = w->N; a.K = w->K; a.Kop = w->Kop;
+        a.num_sms = w->num_sms;
+        a.out_scale = ldexpf(1.0f, es);
+        cudaError_t e = launch_gemm_nvf4_decode(a, gemm_decode_split(w->N, nkb, w->num_sms), static_cast<cudaStream_t>(stream));
+        if (e != cudaSuccess) return cuda_fail(e, "gemm_decode_kernel(nvfp4)");
+        return OSC_OK;
+    }
     if (osc_status s = make_tmap(&a.tm_a, xq, false, M, w->K / 2, w->K / 2, 128)) return s;
-    const int bn = gemm_pair_block_n(false, false, (M + 255) / 256, w->N, (w->K + 255) / 256 + w->Kop / 64, w->num_sms);
+    const int bn = gemm_pair_block_n(false, false, (M + 255) / 256, w->N, nkb, w->num_sms);
     a.tm_b = w->tm_b2[bn == 256];
     if (w->Kop > 0) {
         if (osc_status s = make_tmap(&a.tm_ao, xo, true, M, (uint64_t)w->Kop * 2, (uint64_t)w->Kop * 2, 128)) return s;

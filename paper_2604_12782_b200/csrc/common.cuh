@@ -125,6 +125,7 @@ int gemm_pair_block_n(bool fp8, bool allow_240, long row_tiles, int N, int stage
 cudaError_t launch_gemm_dual_decode(const GemmArgs& a, int S, cudaStream_t st);
 cudaError_t launch_gemm_fp8_decode(const GemmArgs& a, int S, cudaStream_t st);
 cudaError_t launch_gemm_mxf8_decode(const GemmArgs& a, int S, cudaStream_t st);
+cudaError_t launch_gemm_nvf4_decode(const GemmArgs& a, int S, cudaStream_t st);
 int gemm_decode_split(int N, int nkb, int num_sms);
 cudaError_t launch_retile_sf(const uint8_t* src, uint8_t* dst, int N, int K, int bn, cudaStream_t st);
 

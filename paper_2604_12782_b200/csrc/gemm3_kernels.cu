@@ -16,8 +16,9 @@
 // activation quantizer.
 //
 //   warp 0    : TMA producer          warp 1 : MMA issuer, TMEM owner        warps 2-5 : epilogue
-// Modes and K-block order are those of the other GEMM kernels (Path A block-scaled FP4 blocks, then the
-// BF16 blocks of Path B; or E4M3 blocks with per-row scales applied in the epilogue).
+// Modes and K-block order are those of the other GEMM kernels (Path A block-scaled FP4 blocks - MXFP4 or
+// NVFP4 - then the BF16 blocks of Path B; or E4M3 blocks with per-row scales applied in the epilogue, or
+// block-scaled E4M3).
 #include <cuda_bf16.h>
 
 #include "common.cuh"
@@ -29,6 +30,8 @@ namespace decode {
 constexpr int MODE_OSC = 0;
 constexpr int MODE_FP8 = 1;
 constexpr int MODE_MXF8 = 2;            // block-scaled FP8 (MXFP8): one 128-channel scale block per stage and operand
+constexpr int MODE_NVF4 = 3;            // Eq. 5 on NVFP4: E4M3 scale per 16 channels (four 64-channel scale blocks per
+                                        // stage), BF16 branch, power-of-two output scale
 constexpr int BF = 128;                 // output features per CTA = MMA rows = TMEM lanes
 constexpr int ROW_BYTES = 128;
 constexpr int W_BYTES = BF * ROW_BYTES;        // 16 KB of weights per stage
@@ -40,17 +43,23 @@ constexpr int MAX_CLUSTER = 8;
 template <int MODE, int TOK>
 struct Cfg {
     static constexpr bool SCALED = MODE != MODE_FP8;
-    static constexpr int KA = (MODE == MODE_OSC) ? 2 : 1;            // 128-channel scale blocks per stage
+    static constexpr bool DUAL = MODE == MODE_OSC || MODE == MODE_NVF4;   // has the BF16 branch (Path B)
+    static constexpr int KA = (MODE == MODE_OSC) ? 2 : (MODE == MODE_NVF4) ? 4 : 1;   // 512-byte scale blocks per stage
+    static constexpr int SF_K = (MODE == MODE_NVF4) ? 64 : 128;      // channels per scale block
     static constexpr int XATOMS = (TOK > 128) ? 2 : 1;               // 128-row scale blocks of the activations
     static constexpr int X_BYTES = TOK * ROW_BYTES;                  // activations per stage
-    static constexpr int SFW_BYTES = SCALED ? 1024 : 0;              // weight scales per stage (MXFP8 uses half of it)
-    static constexpr int SFX_BYTES = SCALED ? XATOMS * 1024 : 0;     // activation scales
+    static constexpr int SF_ROWBLOCK = (KA > 2 ? KA : 2) * 512;      // one 128-row block's scales of a stage (MXFP8 uses half)
+    static constexpr int SFW_BYTES = SCALED ? SF_ROWBLOCK : 0;       // weight scales per stage
+    static constexpr int SFX_BYTES = SCALED ? XATOMS * SF_ROWBLOCK : 0;   // activation scales
     static constexpr int STAGE_BYTES = W_BYTES + X_BYTES + SFW_BYTES + SFX_BYTES;
-    static constexpr int STAGES = 4;   // TOK = 64: ~105 KB per CTA, the CTAs of two consecutive launches share an SM,
-                                       // so the next call's weight loads overlap this call's reduction and stores
+    // TOK = 64: ~105 KB per CTA, so that two CTAs share an SM (a split tile set larger than the SM count still runs in
+    // one wave, and the next call's weight loads overlap this call's reduction and stores).  NVFP4's stage is 2 KB
+    // larger (twice the scale bytes) and four of them miss that budget by 256 bytes: three stages there.
+    static constexpr int STAGES = (MODE == MODE_NVF4 && TOK <= 64) ? 3 : 4;
     static constexpr int CTAS_PER_SM = (TOK <= 64) ? 2 : 1;
-    static constexpr int TM_SFW = TOK;            // TMEM: accumulator (TOK columns), weight scales (2 K blocks x 4
-    static constexpr int TM_SFX = TOK + 8;        // columns), activation scales (2 K blocks x XATOMS x 4 columns)
+    static constexpr int TM_SFW = TOK;            // TMEM: accumulator (TOK columns), weight scales (KA blocks x 4
+    static constexpr int TM_SFX = TOK + (KA > 2 ? KA : 2) * 4;   // columns), activation scales (KA x XATOMS x 4 columns)
+    static_assert(TM_SFX + (KA > 2 ? KA : 2) * XATOMS * 4 <= ((TOK <= 64) ? 128 : 512), "TMEM columns");
     static constexpr int TMEM_COLS = (TOK <= 64) ? 128 : 512;
     static constexpr int PARTIAL_BYTES = TOK * BF * 4;   // parked partial tile [token][feature], aliases the first stages
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
@@ -105,7 +114,7 @@ __global__ void __launch_bounds__(THREADS, Cfg<MODE, TOK>::CTAS_PER_SM) gemm_dec
         fence_barrier_init();
         prefetch_tmap(&args.tm_a);
         prefetch_tmap(&args.tm_b);
-        if (MODE == MODE_OSC && args.Kop > 0) {
+        if (C::DUAL && args.Kop > 0) {
             prefetch_tmap(&args.tm_ao);
             prefetch_tmap(&args.tm_bo);
         }
@@ -123,11 +132,11 @@ __global__ void __launch_bounds__(THREADS, Cfg<MODE, TOK>::CTAS_PER_SM) gemm_dec
     const int N = args.N, K = args.K, M = args.M;
     const int ntok = (M + 15) / 16 * 16;                       // MMA N
     const int xatoms = (ntok + 127) / 128;                     // 128-row scale blocks the activations span
-    const int elems_per_kb = (MODE == MODE_OSC) ? 256 : 128;
+    const int elems_per_kb = C::DUAL ? 256 : 128;
     const int nkb_a = (K + elems_per_kb - 1) / elems_per_kb;
-    const int nkb_b = (MODE == MODE_OSC) ? args.Kop / 64 : 0;
+    const int nkb_b = C::DUAL ? args.Kop / 64 : 0;
     const int nkb = nkb_a + nkb_b;
-    const int katoms_total = K / 128;
+    const int katoms_total = K / C::SF_K;
     // my K slice: blocks [kb0, kb1) of the tile's K loop
     const int per = (nkb + S - 1) / S;
     const int kb0 = min(nkb, rank * per);
@@ -164,7 +173,7 @@ __global__ void __launch_bounds__(THREADS, Cfg<MODE, TOK>::CTAS_PER_SM) gemm_dec
                 if (C::SCALED) {
                     const int ka = min(C::KA, katoms_total - C::KA * kb);
                     for (int j = 0; j < xatoms; ++j)   // 128-row scale blocks of the activations
-                        bulk_load(st + W_BYTES + X_BYTES + C::SFW_BYTES + j * 1024,
+                        bulk_load(st + W_BYTES + X_BYTES + C::SFW_BYTES + j * C::SF_ROWBLOCK,
                                   args.sfa + ((int64_t)j * katoms_total + C::KA * kb) * 512, (uint32_t)ka * 512u, &full_bar[s]);
                 }
             } else {
@@ -201,6 +210,7 @@ __global__ void __launch_bounds__(THREADS, Cfg<MODE, TOK>::CTAS_PER_SM) gemm_dec
         int s = 0;
         uint32_t ph = 0;
         const uint32_t idesc_a = (MODE == MODE_OSC)    ? idesc_mxf4(BF, ntok)
+                                 : (MODE == MODE_NVF4) ? idesc_nvf4(BF, ntok)
                                  : (MODE == MODE_MXF8) ? idesc_mxf8(BF, ntok)
                                                        : idesc_e4m3(BF, ntok);
         const uint32_t idesc_b = idesc_bf16(BF, ntok);
@@ -238,6 +248,27 @@ __global__ void __launch_bounds__(THREADS, Cfg<MODE, TOK>::CTAS_PER_SM) gemm_dec
                                      (first | (uint32_t)k) ? 1u : 0u);
                         }
                     }
+                } else if (MODE == MODE_NVF4 && kb < nkb_a) {
+                    // four 64-channel scale blocks per stage, one per K = 64 instruction (a whole scale column each)
+                    const int ka = min(4, katoms_total - 4 * kb);
+                    const uint64_t sfw_d = sf_hi | (uint64_t)((sbase + W_BYTES + X_BYTES) >> 4);
+                    const uint64_t sfx_d = sf_hi | (uint64_t)((sbase + W_BYTES + X_BYTES + C::SFW_BYTES) >> 4);
+#pragma unroll
+                    for (int a = 0; a < 4; ++a) {
+                        if (a < ka) {
+                            tc_copy_sf(tmem_base + TM_SFW + a * 4, sfw_d + (uint64_t)(a * 32));
+#pragma unroll
+                            for (int j = 0; j < C::XATOMS; ++j)
+                                if (j < xatoms)
+                                    tc_copy_sf(tmem_base + TM_SFX + a * (C::XATOMS * 4) + j * 4,
+                                               sfx_d + (uint64_t)(j * (C::SF_ROWBLOCK / 16) + a * 32));
+                        }
+                    }
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        if (k < ka)
+                            mma_nvf4(tmem_base, wdesc + 2 * k, xdesc + 2 * k, idesc_a, tmem_base + TM_SFW + k * 4,
+                                     tmem_base + TM_SFX + k * (C::XATOMS * 4), (first | (uint32_t)k) ? 1u : 0u);
                 } else if (MODE == MODE_MXF8) {
                     const uint64_t sfw_d = sf_hi | (uint64_t)((sbase + W_BYTES + X_BYTES) >> 4);
                     const uint64_t sfx_d = sf_hi | (uint64_t)((sbase + W_BYTES + X_BYTES + C::SFW_BYTES) >> 4);
@@ -249,7 +280,7 @@ __global__ void __launch_bounds__(THREADS, Cfg<MODE, TOK>::CTAS_PER_SM) gemm_dec
                     for (int k = 0; k < 4; ++k)
                         mma_mxf8(tmem_base, wdesc + 2 * k, xdesc + 2 * k, idesc_a | idesc_sf_ids(k, k), tmem_base + TM_SFW,
                                  tmem_base + TM_SFX, (first | (uint32_t)k) ? 1u : 0u);
-                } else if (MODE == MODE_OSC) {
+                } else if (C::DUAL) {
 #pragma unroll
                     for (int k = 0; k < 4; ++k)
                         mma_f16(tmem_base, wdesc + 2 * k, xdesc + 2 * k, idesc_b, (first | (uint32_t)k) ? 1u : 0u);
@@ -303,6 +334,7 @@ done:
                     if (t < M) {
                         float v = __uint_as_float(r[i]);
                         if (MODE == MODE_FP8) v = v * (args.sx[t] * swn);
+                        if (MODE == MODE_NVF4) v *= args.out_scale;   // back out of the scaled domain: an exact power of two
                         args.Y[(int64_t)t * args.ldy + n] = __bfloat16_as_ushort(__float2bfloat16_rn(v));
                     }
                 }
@@ -358,6 +390,7 @@ done:
                     const float sxt = args.sx[t];
                     o.x *= sxt * sw4.x; o.y *= sxt * sw4.y; o.z *= sxt * sw4.z; o.w *= sxt * sw4.w;
                 }
+                if (MODE == MODE_NVF4) { o.x *= args.out_scale; o.y *= args.out_scale; o.z *= args.out_scale; o.w *= args.out_scale; }
                 if (n4 < N) {
                     const __nv_bfloat162 lo = __floats2bfloat162_rn(o.x, o.y), hi = __floats2bfloat162_rn(o.z, o.w);
                     *reinterpret_cast<uint2*>(args.Y + (int64_t)t * args.ldy + n4) =
@@ -422,6 +455,9 @@ int gemm_decode_split(int N, int nkb, int num_sms) {
 
 cudaError_t launch_gemm_dual_decode(const GemmArgs& a, int S, cudaStream_t st) {
     return a.M <= 64 ? decode::launch_cfg<decode::MODE_OSC, 64>(a, S, st) : decode::launch_cfg<decode::MODE_OSC, 256>(a, S, st);
+}
+cudaError_t launch_gemm_nvf4_decode(const GemmArgs& a, int S, cudaStream_t st) {
+    return a.M <= 64 ? decode::launch_cfg<decode::MODE_NVF4, 64>(a, S, st) : decode::launch_cfg<decode::MODE_NVF4, 256>(a, S, st);
 }
 cudaError_t launch_gemm_mxf8_decode(const GemmArgs& a, int S, cudaStream_t st) {
     return a.M <= 64 ? decode::launch_cfg<decode::MODE_MXF8, 64>(a, S, st) : decode::launch_cfg<decode::MODE_MXF8, 256>(a, S, st);

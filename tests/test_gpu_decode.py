@@ -145,3 +145,32 @@ def test_decode_kernel_mxfp8(B, oracle, env, M, K, N, split):
         B.osc_sync_check()
         assert np.array_equal(ws[sz.x8_offset:sz.x8_offset + M * K].cpu().numpy().reshape(M, K), x8)
         assert_within_tolerance(host_f64(Y), Yref, T, f"mxfp8 decode={mode} M={M} K={K} N={N} S={split}")
+
+
+@pytest.mark.parametrize("M,K,N,kind,split", [
+    (1, 128, 64, "one", None), (16, 512, 512, "two", None), (17, 384, 320, "one", 2), (33, 640, 192, "two", 3),
+    (64, 1024, 448, "one", 4), (48, 2048, 256, "empty", 8), (64, 4096, 512, "one", None), (20, 4096, 384, "two", 3),
+    (65, 512, 192, "two", None), (129, 384, 320, "one", 3), (200, 2048, 128, "one", 4), (256, 640, 448, "two", 1),
+    (250, 4096, 64, "one", 8)])
+def test_decode_kernel_nvfp4(B, oracle, env, M, K, N, kind, split):
+    """NVFP4 / G = 16 on the few-row kernel (four 64-channel scale blocks per stage, E4M3 scales, power-of-two output
+    scale), forced for every M <= 256 and every cluster size, against the oracle and against the pair kernel."""
+    c = synth.osc16_linear_case(M + K + 3, M, K, N)
+    rng = np.random.default_rng(N + M)
+    lut16 = {"one": c["lut16"], "empty": np.full((K // 16, 1), -1, np.int8),
+             "two": np.stack([rng.permutation(16)[:2] for _ in range(K // 16)]).astype(np.int8)}[kind]
+    ex, ew = synth.nvfp4_tensor_exponent(c["X"]), synth.nvfp4_tensor_exponent(c["W"])
+    Yref, T, *_ = oracle.nvfp4_linear(c["X"], c["W"], lut16, ex, ew)
+    w = B.osc_nvfp4_prepare_weights(dev_bf16(c["W"]), lut16, ew)
+    sz = B.osc_nvfp4_act_sizes(w, M)
+    X = dev_bf16(c["X"])
+    for mode in (2, 0):
+        env(mode, split if mode else None)
+        ws = poison(sz.workspace_bytes)
+        big = torch.full((M + 2, N + 8), 7.0, dtype=torch.bfloat16, device="cuda")
+        B.osc_nvfp4_linear(w, X, ex, big[1:M + 1, :N], ws)
+        B.osc_sync_check()
+        assert_within_tolerance(host_f64(big[1:M + 1, :N]), Yref, T, f"nvfp4 decode={mode} M={M} K={K} N={N} S={split}")
+        guard = big.clone()
+        guard[1:M + 1, :N] = 7.0
+        assert (guard == 7.0).all(), "wrote outside Y"
