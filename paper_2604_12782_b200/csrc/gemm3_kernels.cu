@@ -1,11 +1,12 @@
-// Few-row ("decode") variant of the tensor-core kernels: M <= 64 activation rows, dense weights.
+// Few-row ("decode") variant of the tensor-core kernels: up to 64 activation rows (two CTAs per SM) or up to 256
+// (one CTA per SM), dense weights.
 //
 // With a handful of tokens the linear layer streams its weights once and is bound by HBM bandwidth and
 // by latency, not by the tensor cores (the memory-bound column of the paper's efficiency table,
 // M = 16-64).  The roles of the operands are swapped: a CTA owns 128 OUTPUT FEATURES (weight rows), which
-// become the 128 rows of the MMA, and the tokens become its N dimension (16..64), so no tensor-core row
-// is spent on padding and a stage moves 16 KB of weights for 2-8 KB of activations.  To put every SM on
-// the weight stream, the K loop of one 128-feature tile is split over the S CTAs of a thread-block
+// become the 128 rows of the MMA, and the tokens become its N dimension (16..256), so no tensor-core row
+// is spent on padding and a stage moves 16 KB of weights for 2-8 KB of activations (up to 32 KB in the
+// 256-row form).  To put every SM on the weight stream, the K loop of one 128-feature tile is split over the S CTAs of a thread-block
 // cluster; each CTA accumulates its K slice in its own TMEM, parks the fp32 partial tile in its shared
 // memory, and after a cluster barrier every CTA adds, in rank order, the partials of its share of the
 // tokens through distributed shared memory (deterministic, no global scratch, no atomics) and writes
