@@ -544,16 +544,36 @@ def run_sweep(args):
             B.osc_rmsnorm(p.X[j], gam, eps, Xn[j])
             B.osc_linear(p.w[j], Xn[j], p.Y[j], p.ws[j])
 
+        # with the residual update in front of the norm (h' = h + r written to a scratch stream, so nothing drifts)
+        Rr = [torch.roll(p.X[j], 7, 0).contiguous() for j in range(p.n)]
+        Hn = torch.empty(M, K, dtype=torch.bfloat16, device="cuda")
+
+        def fused_add_q(i):
+            j = i % p.n
+            B.osc_add_rmsnorm_quantize_extract(p.w[j], p.X[j], Rr[j], gam, eps, Hn, *p.views(j))
+
+        def fused_add_lin(i):
+            j = i % p.n
+            B.osc_add_rmsnorm_linear(p.w[j], p.X[j], Rr[j], gam, eps, Hn, p.Y[j], p.ws[j])
+
+        def two_step_add_lin(i):
+            j = i % p.n
+            B.osc_add_rmsnorm(p.X[j], Rr[j], gam, eps, Hn, Xn[j])
+            B.osc_linear(p.w[j], Xn[j], p.Y[j], p.ws[j])
+
         t = {k: time_loop(torch, f, steps, warm) for k, f in
              (("fused_quant_ms", fused_q), ("norm_ms", norm_only), ("two_step_quant_ms", two_step_q),
-              ("fused_linear_ms", fused_lin), ("two_step_linear_ms", two_step_lin))}
+              ("fused_linear_ms", fused_lin), ("two_step_linear_ms", two_step_lin),
+              ("add_fused_quant_ms", fused_add_q), ("add_fused_linear_ms", fused_add_lin),
+              ("add_two_step_linear_ms", two_step_add_lin))}
         B.osc_sync_check()
         byts = roofline.quantize_extract_bytes(M, K, p.K_o_pad)   # one read of the rows + the quantizer's outputs
+        t["add_fused_quant_frac_hbm"] = (byts + 4.0 * M * K) / (t["add_fused_quant_ms"] * 1e-3) / peaks["hbm"]
         rows.append({"name": name, "M": M, "K": K, "N": N, "K_o": p.K_o, **t, "ms": t["fused_linear_ms"],
                      "fused_quant_gbs": byts / t["fused_quant_ms"] / 1e6,
                      "fused_quant_frac_hbm": byts / (t["fused_quant_ms"] * 1e-3) / peaks["hbm"],
                      "speedup_linear": t["two_step_linear_ms"] / t["fused_linear_ms"]})
-        del p, Xn
+        del p, Xn, Rr, Hn
         torch.cuda.empty_cache()
 
     def profile_row(name, S, K, seed=0):
@@ -798,7 +818,32 @@ def run_sweep(args):
         B.osc_sync_check()
         rows.append({"name": "layer.fused(rmsnorm+qkv,o_proj,rmsnorm+gate_up,swiglu+down_fp8)", "M": M, "ms": ms_f,
                      "separate_kernels_ms": ms_s, "speedup": ms_s / ms_f})
-        del qkv, opj, gup, dwn, Xn, Hh
+        # the same with the two residual updates of the layer in the picture: h' = h + branch output in front of each
+        # norm, written to a scratch stream so that the values do not drift over the timed iterations
+        Hn = [torch.empty(M, 4096, dtype=torch.bfloat16, device="cuda") for _ in range(2)]
+
+        def fused_res(i):
+            j = i % 2
+            B.osc_add_rmsnorm_linear(qkv.w[j], qkv.X[j], dwn.Y[j], gam, eps, Hn[0], qkv.Y[j], qkv.ws[j])
+            B.osc_linear(opj.w[j], opj.X[j], opj.Y[j], opj.ws[j])
+            B.osc_add_rmsnorm_linear(gup.w[j], gup.X[j], opj.Y[j], gam, eps, Hn[1], gup.Y[j], gup.ws[j])
+            B.osc_swiglu_fp8_linear(dwn.w[j], gup.Y[j], dwn.Y[j], dwn.ws[j])
+
+        def separate_res(i):
+            j = i % 2
+            B.osc_add_rmsnorm(qkv.X[j], dwn.Y[j], gam, eps, Hn[0], Xn)
+            B.osc_linear(qkv.w[j], Xn, qkv.Y[j], qkv.ws[j])
+            B.osc_linear(opj.w[j], opj.X[j], opj.Y[j], opj.ws[j])
+            B.osc_add_rmsnorm(gup.X[j], opj.Y[j], gam, eps, Hn[1], Xn)
+            B.osc_linear(gup.w[j], Xn, gup.Y[j], gup.ws[j])
+            B.osc_swiglu(gup.Y[j], 12288, Hh)
+            B.osc_fp8_linear(dwn.w[j], Hh, dwn.Y[j], dwn.ws[j])
+
+        ms_f, ms_s = time_loop(torch, fused_res, steps, warm), time_loop(torch, separate_res, steps, warm)
+        B.osc_sync_check()
+        rows.append({"name": "layer.fused_with_residual(add+rmsnorm+qkv,o_proj,add+rmsnorm+gate_up,swiglu+down_fp8)", "M": M,
+                     "ms": ms_f, "separate_kernels_ms": ms_s, "speedup": ms_s / ms_f})
+        del qkv, opj, gup, dwn, Xn, Hh, Hn
         torch.cuda.empty_cache()
 
     # MoE: 128 experts, top-8 of 8192 tokens, Zipf(1.1) load

@@ -193,6 +193,24 @@ osc_status osc_rmsnorm_quantize_extract(const osc_weights* w, const void* H, int
 osc_status osc_rmsnorm_linear(const osc_weights* w, const void* H, int M, int64_t ldh, const void* gamma, float eps,
                               void* Y, int64_t ldy, void* workspace, size_t workspace_bytes, void* stream);
 
+/* The same with the residual update of a decoder layer in front of the norm (Section 3.3: the quantizer sits
+ * directly behind the operator that produces the activations; here that operator is "add, then RMSNorm"):
+ *
+ *   H'[m,k] = bf16( H[m,k] + R[m,k] )      one fp32 addition (exact, or past the bf16 rounding point), nearest even
+ *
+ * H' goes to Hout (dev bf16 [M, ldo]) and the norm and Algorithm 2 run on H'.  R: dev bf16 [M, ldr], the branch
+ * output (attention or MLP) to add.  Hout may be H or R themselves (update in place); other overlaps are not
+ * allowed.  ldr, ldo >= K, multiples of 8; R, Hout 16-byte aligned.  Everything else as in the calls above;
+ * osc_add_rmsnorm is the unfused reference point and writes X as osc_rmsnorm does. */
+osc_status osc_add_rmsnorm(const void* H, const void* R, int M, int K, int64_t ldh, int64_t ldr, const void* gamma, float eps,
+                           void* Hout, int64_t ldo, void* X, int64_t ldx, void* stream);
+osc_status osc_add_rmsnorm_quantize_extract(const osc_weights* w, const void* H, const void* R, int M, int64_t ldh,
+                                            int64_t ldr, const void* gamma, float eps, void* Hout, int64_t ldo, void* xq,
+                                            void* sfa, void* xo, void* stream);
+osc_status osc_add_rmsnorm_linear(const osc_weights* w, const void* H, const void* R, int M, int64_t ldh, int64_t ldr,
+                                  const void* gamma, float eps, void* Hout, int64_t ldo, void* Y, int64_t ldy,
+                                  void* workspace, size_t workspace_bytes, void* stream);
+
 /* Grouped (MoE) form: rows of X_perm are sorted by expert, expert e owns rows
  * [off[e], off[e+1]); off: dev int32 [E+1], off[E] == M_total.  Expert e's scale rows start
  * at scale row sum_{e'<e} roundup(m_e', 128).  The tile schedule is built on the device. */

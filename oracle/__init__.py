@@ -404,4 +404,4 @@ def swiglu(GU: np.ndarray, I: int) -> np.ndarray:
     return H
 
 
-from .rmsnorm import f64_to_bf16_bits, rmsnorm  # noqa: E402,F401
+from .rmsnorm import add_rmsnorm, f64_to_bf16_bits, residual_add, rmsnorm  # noqa: E402,F401

@@ -13,6 +13,8 @@ high precision, the element-wise part in fp32, one final rounding to bf16):
 with x, gamma bf16 values and eps an fp32 value.  The fused path is this function followed by Algorithm 2
 on its output.
 
+residual_add / add_rmsnorm: the residual update of a decoder layer in front of the norm, h' = bf16(h + r).
+
 Pins (tests/test_oracle_rmsnorm.py): torch's float64 rms_norm as the library routine (agreement to one bf16
 unit, equality almost everywhere), closed forms (constant rows, one non-zero per row, eps = 0 rows of +-1),
 power-of-two scale invariance at eps = 0, hand-worked double -> bf16 roundings (ties, subnormals, overflow,
@@ -59,3 +61,18 @@ def rmsnorm(H: np.ndarray, gamma: np.ndarray, eps: float) -> np.ndarray:
         t = x.astype(np.float32) * r32[:, None]                # fp32 product, rounded to nearest
         y = t * g32[None, :]                                   # second fp32 product
     return f64_to_bf16_bits(y.astype(np.float64))              # exact widening, then the one rounding to bf16
+
+
+def residual_add(H: np.ndarray, R: np.ndarray) -> np.ndarray:
+    """The residual update in front of the norm: bf16 bits of the exact sum h + r, rounded once, nearest even.
+    The double addition is exact while the exponents differ by fewer than 45 binades; beyond that the smaller
+    addend is more than 2^35 times smaller than half a bf16 step of the larger one, which lies on the bf16 grid, so
+    it cannot carry the sum across a rounding boundary (checked against rational arithmetic in the tests)."""
+    return f64_to_bf16_bits(_bf16_bits_to_f64(H) + _bf16_bits_to_f64(R))
+
+
+def add_rmsnorm(H: np.ndarray, R: np.ndarray, gamma: np.ndarray, eps: float):
+    """-> (H' = residual_add(H, R), rmsnorm(H', gamma, eps))."""
+    Hs = residual_add(H, R)
+    return Hs, rmsnorm(Hs, gamma, eps)
+

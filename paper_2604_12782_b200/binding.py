@@ -80,6 +80,9 @@ _SIGS = {
     "osc_linear_grouped_gather": (_i, [_vp, _vp, _i, _i64, _vp, _vp, _i, _vp, _i64, _vp, _sz, _vp]),
     "osc_rmsnorm_linear_grouped_gather": (_i, [_vp, _vp, _i, _i64, _vp, C.c_float, _vp, _vp, _i, _vp, _i64, _vp, _sz, _vp]),
     "osc_swiglu_fp8_linear_grouped": (_i, [_vp, _vp, _vp, _i, _i64, _vp, _i64, _vp, _sz, _vp]),
+    "osc_add_rmsnorm": (_i, [_vp, _vp, _i, _i, _i64, _i64, _vp, C.c_float, _vp, _i64, _vp, _i64, _vp]),
+    "osc_add_rmsnorm_quantize_extract": (_i, [_vp, _vp, _vp, _i, _i64, _i64, _vp, C.c_float, _vp, _i64, _vp, _vp, _vp, _vp]),
+    "osc_add_rmsnorm_linear": (_i, [_vp, _vp, _vp, _i, _i64, _i64, _vp, C.c_float, _vp, _i64, _vp, _i64, _vp, _sz, _vp]),
     "osc_rmsnorm": (_i, [_vp, _i, _i, _i64, _vp, C.c_float, _vp, _i64, _vp]),
     "osc_swiglu": (_i, [_vp, _i, _i, _i64, _vp, _i64, _vp]),
     "osc_swiglu_fp8_quantize": (_i, [_vp, _i, _i, _i64, _vp, _vp, _vp]),
@@ -303,6 +306,34 @@ def osc_rmsnorm(H: torch.Tensor, gamma: torch.Tensor, eps: float, X: torch.Tenso
     M, K = H.shape
     _check(_lib.osc_rmsnorm(_ptr(H), M, K, H.stride(0) if M else K, _ptr(gamma), float(eps), _ptr(X),
                             X.stride(0) if M else K, _stream(stream)))
+
+
+def osc_add_rmsnorm(H: torch.Tensor, R: torch.Tensor, gamma: torch.Tensor, eps: float, Hout: torch.Tensor, X: torch.Tensor,
+                    stream=None):
+    """Hout = bf16(H + R), X = RMSNorm(Hout) * gamma: the unfused reference point of the residual form."""
+    M, K = H.shape
+    _check(_lib.osc_add_rmsnorm(_ptr(H), _ptr(R), M, K, H.stride(0) if M else K, R.stride(0) if M else K, _ptr(gamma),
+                                float(eps), _ptr(Hout), Hout.stride(0) if M else K, _ptr(X), X.stride(0) if M else K,
+                                _stream(stream)))
+
+
+def osc_add_rmsnorm_quantize_extract(w: OscWeights, H: torch.Tensor, R: torch.Tensor, gamma: torch.Tensor, eps: float,
+                                     Hout: torch.Tensor, xq, sfa, xo, stream=None):
+    """Residual update, RMSNorm and Algorithm 2 in one pass: Hout = bf16(H + R) is the only full-width tensor written."""
+    M = H.shape[0]
+    _check(_lib.osc_add_rmsnorm_quantize_extract(w.ptr, _ptr(H), _ptr(R), M, H.stride(0) if M else w.K,
+                                                 R.stride(0) if M else w.K, _ptr(gamma), float(eps), _ptr(Hout),
+                                                 Hout.stride(0) if M else w.K, _ptr(xq), _ptr(sfa),
+                                                 _ptr(xo) if w.K_o_pad else None, _stream(stream)))
+
+
+def osc_add_rmsnorm_linear(w: OscWeights, H: torch.Tensor, R: torch.Tensor, gamma: torch.Tensor, eps: float,
+                           Hout: torch.Tensor, Y: torch.Tensor, workspace: torch.Tensor, stream=None):
+    M = H.shape[0]
+    _check(_lib.osc_add_rmsnorm_linear(w.ptr, _ptr(H), _ptr(R), M, H.stride(0) if M else w.K, R.stride(0) if M else w.K,
+                                       _ptr(gamma), float(eps), _ptr(Hout), Hout.stride(0) if M else w.K, _ptr(Y),
+                                       Y.stride(0) if M else w.N, _ptr(workspace),
+                                       workspace.numel() * workspace.element_size(), _stream(stream)))
 
 
 def osc_rmsnorm_quantize_extract(w: OscWeights, H: torch.Tensor, gamma: torch.Tensor, eps: float, xq, sfa, xo, stream=None):

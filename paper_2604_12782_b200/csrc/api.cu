@@ -535,8 +535,23 @@ osc_status osc_linear(const osc_weights* w, const void* X, int M, int64_t ldx, v
 }
 
 // ---- RMSNorm fused in front of Algorithm 2
-osc_status osc_rmsnorm(const void* H, int M, int K, int64_t ldh, const void* gamma, float eps, void* X, int64_t ldx,
-                       void* stream) {
+// Optional residual update in front of the norm: h' = bf16(h + r), written to Hout.
+struct Residual {
+    const void* R = nullptr;
+    int64_t ldr = 0;
+    void* Hout = nullptr;
+    int64_t ldo = 0;
+};
+static osc_status check_residual(const Residual& res, int K) {
+    if (!res.R || !res.Hout) return fail(OSC_ERR_INVALID_ARG, "R / Hout is null");
+    if (res.ldr < K || res.ldo < K) return fail(OSC_ERR_SHAPE, "ldr = %lld, ldo = %lld < K = %d", (long long)res.ldr, (long long)res.ldo, K);
+    if (res.ldr % 8 || res.ldo % 8 || !aligned16(res.R) || !aligned16(res.Hout))
+        return fail(OSC_ERR_ALIGN, "R and Hout must be 16-byte aligned, ldr and ldo multiples of 8");
+    return OSC_OK;
+}
+
+static osc_status rmsnorm_only_impl(const void* H, int M, int K, int64_t ldh, const void* gamma, float eps, void* X,
+                                    int64_t ldx, void* stream, const Residual* res) {
     if (M < 0) return fail(OSC_ERR_INVALID_ARG, "M = %d is negative", M);
     if (K <= 0 || K % 128) return fail(OSC_ERR_SHAPE, "K = %d must be a positive multiple of 128", K);
     if (K > 8192) return fail(OSC_ERR_SHAPE, "K = %d: the fused RMSNorm stages a row in shared memory, K <= 8192", K);
@@ -545,21 +560,43 @@ osc_status osc_rmsnorm(const void* H, int M, int K, int64_t ldh, const void* gam
     if (ldh < K || ldx < K) return fail(OSC_ERR_SHAPE, "ldh = %lld, ldx = %lld < K = %d", (long long)ldh, (long long)ldx, K);
     if (ldh % 8 || ldx % 8 || !aligned16(H) || !aligned16(X) || !aligned16(gamma))
         return fail(OSC_ERR_ALIGN, "H, X and gamma must be 16-byte aligned, ldh and ldx multiples of 8");
+    if (res) {
+        if (osc_status s = check_residual(*res, K)) return s;
+    }
+    const Residual none;
+    const Residual& rs = res ? *res : none;
     cudaError_t e = launch_rmsnorm_quant(false, H, ldh, M, K, gamma, eps, X, ldx, nullptr, nullptr, nullptr, nullptr,
-                                         0, 0, static_cast<cudaStream_t>(stream));
+                                         0, 0, static_cast<cudaStream_t>(stream), rs.R, rs.ldr, rs.Hout, rs.ldo);
     if (e != cudaSuccess) return cuda_fail(e, "rmsnorm_quant_kernel(norm only)");
     return OSC_OK;
 }
 
+osc_status osc_rmsnorm(const void* H, int M, int K, int64_t ldh, const void* gamma, float eps, void* X, int64_t ldx,
+                       void* stream) {
+    return rmsnorm_only_impl(H, M, K, ldh, gamma, eps, X, ldx, stream, nullptr);
+}
+osc_status osc_add_rmsnorm(const void* H, const void* R, int M, int K, int64_t ldh, int64_t ldr, const void* gamma, float eps,
+                           void* Hout, int64_t ldo, void* X, int64_t ldx, void* stream) {
+    Residual res;
+    res.R = R; res.ldr = ldr; res.Hout = Hout; res.ldo = ldo;
+    return rmsnorm_only_impl(H, M, K, ldh, gamma, eps, X, ldx, stream, &res);
+}
+
 static osc_status rmsnorm_quantize_impl(const osc_weights* w, const void* H, int M, int64_t ldh, const void* gamma,
-                                        float eps, void* xq, void* sfa, void* xo, cudaStream_t st) {
+                                        float eps, void* xq, void* sfa, void* xo, cudaStream_t st,
+                                        const Residual* res = nullptr) {
     if (w->K > 8192) return fail(OSC_ERR_SHAPE, "K = %d: the fused RMSNorm stages a row in shared memory, K <= 8192", w->K);
     if (M == 0) return OSC_OK;
     if (!gamma || !aligned16(gamma)) return fail(OSC_ERR_ALIGN, "gamma must be non-null and 16-byte aligned");
     if (!xq || !sfa || (w->Kop > 0 && !xo)) return fail(OSC_ERR_INVALID_ARG, "null output pointer");
     if (!aligned16(xq) || !aligned16(sfa) || !aligned16(xo)) return fail(OSC_ERR_ALIGN, "outputs must be 16-byte aligned");
+    if (res) {
+        if (osc_status s = check_residual(*res, w->K)) return s;
+    }
+    const Residual none;
+    const Residual& rs = res ? *res : none;
     cudaError_t e = launch_rmsnorm_quant(true, H, ldh, M, w->K, gamma, eps, nullptr, 0, w->idx_o, xq, sfa,
-                                         w->Kop ? xo : nullptr, w->Ko, w->Kop, st);
+                                         w->Kop ? xo : nullptr, w->Ko, w->Kop, st, rs.R, rs.ldr, rs.Hout, rs.ldo);
     if (e != cudaSuccess) return cuda_fail(e, "rmsnorm_quant_kernel");
     return OSC_OK;
 }
@@ -571,8 +608,19 @@ osc_status osc_rmsnorm_quantize_extract(const osc_weights* w, const void* H, int
     return rmsnorm_quantize_impl(w, H, M, ldh, gamma, eps, xq, sfa, xo, static_cast<cudaStream_t>(stream));
 }
 
-osc_status osc_rmsnorm_linear(const osc_weights* w, const void* H, int M, int64_t ldh, const void* gamma, float eps,
-                              void* Y, int64_t ldy, void* workspace, size_t workspace_bytes, void* stream) {
+osc_status osc_add_rmsnorm_quantize_extract(const osc_weights* w, const void* H, const void* R, int M, int64_t ldh,
+                                            int64_t ldr, const void* gamma, float eps, void* Hout, int64_t ldo, void* xq,
+                                            void* sfa, void* xo, void* stream) {
+    if (osc_status s = check_act(w, H, M, ldh)) return s;
+    if (w->grouped) return fail(OSC_ERR_INVALID_ARG, "grouped weights: use osc_rmsnorm_linear_grouped_gather");
+    Residual res;
+    res.R = R; res.ldr = ldr; res.Hout = Hout; res.ldo = ldo;
+    return rmsnorm_quantize_impl(w, H, M, ldh, gamma, eps, xq, sfa, xo, static_cast<cudaStream_t>(stream), &res);
+}
+
+static osc_status rmsnorm_linear_impl(const osc_weights* w, const void* H, int M, int64_t ldh, const void* gamma, float eps,
+                                      void* Y, int64_t ldy, void* workspace, size_t workspace_bytes, void* stream,
+                                      const Residual* res) {
     if (osc_status s = check_act(w, H, M, ldh)) return s;
     if (w->grouped) return fail(OSC_ERR_INVALID_ARG, "grouped weights: use osc_rmsnorm_linear_grouped_gather");
     if (M == 0) return OSC_OK;
@@ -586,9 +634,21 @@ osc_status osc_rmsnorm_linear(const osc_weights* w, const void* H, int M, int64_
     if (ldy % 8 || !aligned16(Y)) return fail(OSC_ERR_ALIGN, "Y must be 16-byte aligned and ldy a multiple of 8");
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (osc_status s = rmsnorm_quantize_impl(w, H, M, ldh, gamma, eps, ws + sz.xq_offset, ws + sz.sfa_offset, ws + sz.xo_offset, st))
+    if (osc_status s = rmsnorm_quantize_impl(w, H, M, ldh, gamma, eps, ws + sz.xq_offset, ws + sz.sfa_offset, ws + sz.xo_offset, st, res))
         return s;
     return gemm_impl(w, ws + sz.xq_offset, ws + sz.sfa_offset, ws + sz.xo_offset, M, Y, ldy, nullptr, 0, nullptr, 0, st);
+}
+
+osc_status osc_rmsnorm_linear(const osc_weights* w, const void* H, int M, int64_t ldh, const void* gamma, float eps,
+                              void* Y, int64_t ldy, void* workspace, size_t workspace_bytes, void* stream) {
+    return rmsnorm_linear_impl(w, H, M, ldh, gamma, eps, Y, ldy, workspace, workspace_bytes, stream, nullptr);
+}
+osc_status osc_add_rmsnorm_linear(const osc_weights* w, const void* H, const void* R, int M, int64_t ldh, int64_t ldr,
+                                  const void* gamma, float eps, void* Hout, int64_t ldo, void* Y, int64_t ldy,
+                                  void* workspace, size_t workspace_bytes, void* stream) {
+    Residual res;
+    res.R = R; res.ldr = ldr; res.Hout = Hout; res.ldo = ldo;
+    return rmsnorm_linear_impl(w, H, M, ldh, gamma, eps, Y, ldy, workspace, workspace_bytes, stream, &res);
 }
 
 osc_status osc_linear_grouped(const osc_weights* w, const void* X_perm, const int32_t* off, int M_total, int64_t ldx,

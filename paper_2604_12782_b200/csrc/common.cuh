@@ -73,7 +73,8 @@ cudaError_t launch_gather_quantized(const int32_t* row_token, int T, int K, int 
 // norm_kernels.cu
 cudaError_t launch_rmsnorm_quant(bool quant, const void* H, int64_t ldh, int M, int K, const void* gamma, float eps,
                                  void* Xn, int64_t ldx, const int32_t* idx_o, void* xq, void* sf,
-                                 void* xo, int Ko, int Kop, cudaStream_t st);
+                                 void* xo, int Ko, int Kop, cudaStream_t st, const void* R = nullptr, int64_t ldr = 0,
+                                 void* Hout = nullptr, int64_t ldo = 0);
 
 cudaError_t launch_swiglu_fp8(bool quant, const void* GU, int64_t ldg, int M, int I, void* Hout, int64_t ldh, void* x8,
                               void* sx, cudaStream_t st);

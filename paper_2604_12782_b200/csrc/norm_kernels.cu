@@ -38,12 +38,15 @@ __device__ __forceinline__ void team_sync(int slot) {
     asm volatile("bar.sync %0, %1;" ::"r"(slot + 1), "r"(RN_TEAM) : "memory");
 }
 
-template <bool QUANT>
-__global__ void __launch_bounds__(RN_THREADS)
+// Two CTAs per SM (28 rows in flight) need at most 36 registers per thread; the residual update is a template
+// parameter so that the plain form keeps its 32.
+template <bool QUANT, bool ADD>
+__global__ void __launch_bounds__(RN_THREADS, 2)
 rmsnorm_quant_kernel(const uint16_t* __restrict__ H, int64_t ldh, int M, int M_pad, int K,
                      const uint16_t* __restrict__ gamma, float eps, uint16_t* __restrict__ Xn, int64_t ldx,
                      const int32_t* __restrict__ idx_o, uint8_t* __restrict__ xq,
-                     uint8_t* __restrict__ sf, uint16_t* __restrict__ xo, int Ko, int Kop) {
+                     uint8_t* __restrict__ sf, uint16_t* __restrict__ xo, int Ko, int Kop,
+                     const uint16_t* R, int64_t ldr, uint16_t* Hout, int64_t ldo) {
     // [RN_ROWS][K / 8] rows, then per row: one mbarrier, two partial sums (double), one give-up flag
     extern __shared__ uint4 rn_rows[];
     grid_launch_dependents();
@@ -86,14 +89,30 @@ rmsnorm_quant_kernel(const uint16_t* __restrict__ H, int64_t ldh, int M, int M_p
     // buffer holds) so that its barriers below stay matched
     wait_bounded(bar, 0u, give_up, 41);
 
-    // ---- first pass: sum of squares, each warp over every second step of chunks
+    // ---- first pass: sum of squares, each warp over every second step of chunks.  With a residual update (R != null)
+    // the row becomes h' = bf16(h + r) first - one fp32 addition, exact or beyond the bf16 rounding point, then nearest
+    // even - which goes back to the residual stream (Hout; it may be H or R themselves: the row of H is already in
+    // shared memory, and a chunk of R is read by the thread that then overwrites it) and replaces the shared row.
+    const uint4* rrow = ADD ? reinterpret_cast<const uint4*>(R + (int64_t)r * ldr) : nullptr;
+    uint4* orow = ADD ? reinterpret_cast<uint4*>(Hout + (int64_t)r * ldo) : nullptr;
     const int nsteps = (nch + RN_TEAM - 1) / RN_TEAM;
     double ss0 = 0.0, ss1 = 0.0, ss2 = 0.0, ss3 = 0.0;   // four chains: the fp64 pipe's latency is long
 #pragma unroll 4
     for (int i = 0; i < nsteps; ++i) {
         const int c = i * RN_TEAM + tl;
         const uint4 v = (c < nch) ? row[c] : make_uint4(0u, 0u, 0u, 0u);
-        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+        uint32_t w[4] = {v.x, v.y, v.z, v.w};
+        if (ADD && c < nch) {
+            const uint4 d = rrow[c];
+            const uint32_t dw[4] = {d.x, d.y, d.z, d.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                w[j] = bf162_bits(__floats2bfloat162_rn(__fadd_rn(__uint_as_float(w[j] << 16), __uint_as_float(dw[j] << 16)),
+                                                        __fadd_rn(__uint_as_float(w[j] & 0xFFFF0000u), __uint_as_float(dw[j] & 0xFFFF0000u))));
+            const uint4 hs = make_uint4(w[0], w[1], w[2], w[3]);
+            row[c] = hs;
+            orow[c] = hs;
+        }
 #pragma unroll
         for (int j = 0; j < 4; j += 2) {
             const double a0 = (double)__uint_as_float(w[j] << 16), b0 = (double)__uint_as_float(w[j] & 0xFFFF0000u);
@@ -189,25 +208,35 @@ rmsnorm_quant_kernel(const uint16_t* __restrict__ H, int64_t ldh, int M, int M_p
     }
 }
 
-// QUANT: Xn unused.  !QUANT: the quantizer arguments unused.  K <= 8192.
+constexpr int kRnTail = RN_ROWS * (8 + RN_WPR * 8 + 4) + 8;   // mbarriers, partial sums, give-up flags
+
+template <bool QUANT, bool ADD>
+static cudaError_t launch_rmsnorm_cfg(dim3 grid, dim3 block, size_t smem, cudaStream_t st, const void* H, int64_t ldh, int M,
+                                      int M_pad, int K, const void* gamma, float eps, void* Xn, int64_t ldx,
+                                      const int32_t* idx_o, void* xq, void* sf, void* xo, int Ko, int Kop, const void* R,
+                                      int64_t ldr, void* Hout, int64_t ldo) {
+    static PerDevice configured;
+    if (cudaError_t e = opt_in_shared_memory(configured, rmsnorm_quant_kernel<QUANT, ADD>, RN_ROWS * 8192 * 2 + kRnTail)) return e;
+    return launch_pdl(rmsnorm_quant_kernel<QUANT, ADD>, grid, block, smem, st, static_cast<const uint16_t*>(H), ldh, M, M_pad, K,
+                      static_cast<const uint16_t*>(gamma), eps, static_cast<uint16_t*>(Xn), ldx, idx_o,
+                      static_cast<uint8_t*>(xq), static_cast<uint8_t*>(sf), static_cast<uint16_t*>(xo), Ko, Kop,
+                      static_cast<const uint16_t*>(R), ldr, static_cast<uint16_t*>(Hout), ldo);
+}
+
+// QUANT: Xn unused.  !QUANT: the quantizer arguments unused.  K <= 8192.  R != null: residual update h' = bf16(h + r)
+// written to Hout before the norm.
 cudaError_t launch_rmsnorm_quant(bool quant, const void* H, int64_t ldh, int M, int K, const void* gamma, float eps,
                                  void* Xn, int64_t ldx, const int32_t* idx_o, void* xq, void* sf,
-                                 void* xo, int Ko, int Kop, cudaStream_t st) {
+                                 void* xo, int Ko, int Kop, cudaStream_t st, const void* R, int64_t ldr, void* Hout,
+                                 int64_t ldo) {
     if (M <= 0) return cudaSuccess;
     const int M_pad = quant ? (M + 127) / 128 * 128 : M;
     const dim3 grid((M_pad + RN_ROWS - 1) / RN_ROWS), block(RN_THREADS);
-    constexpr int kTail = RN_ROWS * (8 + RN_WPR * 8 + 4) + 8;   // mbarriers, partial sums, give-up flags
-    const size_t smem = (size_t)RN_ROWS * K * 2 + kTail;
-    static PerDevice configured_q, configured_n;
-    if (cudaError_t e = opt_in_shared_memory(configured_q, rmsnorm_quant_kernel<true>, RN_ROWS * 8192 * 2 + kTail)) return e;
-    if (cudaError_t e = opt_in_shared_memory(configured_n, rmsnorm_quant_kernel<false>, RN_ROWS * 8192 * 2 + kTail)) return e;
-    if (quant)
-        return launch_pdl(rmsnorm_quant_kernel<true>, grid, block, smem, st, static_cast<const uint16_t*>(H), ldh, M, M_pad, K,
-                          static_cast<const uint16_t*>(gamma), eps, static_cast<uint16_t*>(Xn), ldx, idx_o,
-                          static_cast<uint8_t*>(xq), static_cast<uint8_t*>(sf), static_cast<uint16_t*>(xo), Ko, Kop);
-    return launch_pdl(rmsnorm_quant_kernel<false>, grid, block, smem, st, static_cast<const uint16_t*>(H), ldh, M, M_pad, K,
-                      static_cast<const uint16_t*>(gamma), eps, static_cast<uint16_t*>(Xn), ldx, idx_o,
-                      static_cast<uint8_t*>(xq), static_cast<uint8_t*>(sf), static_cast<uint16_t*>(xo), Ko, Kop);
+    const size_t smem = (size_t)RN_ROWS * K * 2 + kRnTail;
+    return quant ? (R ? launch_rmsnorm_cfg<true, true>(grid, block, smem, st, H, ldh, M, M_pad, K, gamma, eps, Xn, ldx, idx_o, xq, sf, xo, Ko, Kop, R, ldr, Hout, ldo)
+                      : launch_rmsnorm_cfg<true, false>(grid, block, smem, st, H, ldh, M, M_pad, K, gamma, eps, Xn, ldx, idx_o, xq, sf, xo, Ko, Kop, R, ldr, Hout, ldo))
+                 : (R ? launch_rmsnorm_cfg<false, true>(grid, block, smem, st, H, ldh, M, M_pad, K, gamma, eps, Xn, ldx, idx_o, xq, sf, xo, Ko, Kop, R, ldr, Hout, ldo)
+                      : launch_rmsnorm_cfg<false, false>(grid, block, smem, st, H, ldh, M, M_pad, K, gamma, eps, Xn, ldx, idx_o, xq, sf, xo, Ko, Kop, R, ldr, Hout, ldo));
 }
 
 // ------------------------------------------------------------------ SwiGLU + per-token FP8

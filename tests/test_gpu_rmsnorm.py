@@ -148,3 +148,90 @@ def test_rmsnorm_linear_within_tolerance(B, oracle, M, K, N):
                       torch.zeros(8192 + 128, dtype=torch.bfloat16, device="cuda"), 1e-6,
                       torch.zeros(2, 8192 + 128, dtype=torch.bfloat16, device="cuda"))
     assert e.value.status == -2
+
+
+# ---- the residual update in front of the norm: H' = bf16(H + R)
+
+def branch_rows(rng, Hb):
+    """A branch output to add: mostly smaller than the stream, with entries that cancel it exactly, entries many
+    binades below and above it, and half-step ties."""
+    H = synth.bf16_bits_to_f64(Hb)
+    R = rng.standard_normal(H.shape) * np.abs(H).mean(axis=1, keepdims=True) * 0.3
+    Rb = synth.f32_to_bf16_bits(R.astype(np.float32))
+    flat_h, flat_r = Hb.reshape(-1), Rb.reshape(-1)
+    idx = rng.choice(flat_h.size, size=max(8, flat_h.size // 50), replace=False)
+    q = idx.size // 4
+    flat_r[idx[:q]] = flat_h[idx[:q]] ^ 0x8000                                              # exact cancellation
+    flat_r[idx[q:2 * q]] = synth.f32_to_bf16_bits((H.reshape(-1)[idx[q:2 * q]] * 2.0 ** -8).astype(np.float32))   # ties
+    flat_r[idx[2 * q:3 * q]] = synth.f32_to_bf16_bits((H.reshape(-1)[idx[2 * q:3 * q]] * 2.0 ** -30).astype(np.float32))
+    flat_r[idx[3 * q:]] = synth.f32_to_bf16_bits((H.reshape(-1)[idx[3 * q:]] * 2.0 ** 20).astype(np.float32))
+    return Rb
+
+
+@pytest.mark.parametrize("M,K,where", [(1, 128, "new"), (37, 384, "H"), (130, 1024, "R"), (64, 4096, "new"), (9, 8192, "H"),
+                                       (300, 2048, "new")])
+def test_add_rmsnorm_bit_exact(B, oracle, M, K, where):
+    rng = np.random.default_rng(M + 2 * K)
+    Hb, gb = residual_rows(rng, M, K), gamma_bits(rng, K)
+    Rb = branch_rows(rng, Hb)
+    Hs_ref, X_ref = oracle.add_rmsnorm(Hb, Rb, gb, 1e-6)
+    ld = K + 16
+    Hbig = torch.full((M, ld), 7.0, dtype=torch.bfloat16, device="cuda")
+    Rbig = torch.full((M, ld), 7.0, dtype=torch.bfloat16, device="cuda")
+    Obig = torch.full((M, ld), 7.0, dtype=torch.bfloat16, device="cuda")
+    Hbig[:, :K], Rbig[:, :K] = dev_bf16(Hb), dev_bf16(Rb)
+    out = {"new": Obig, "H": Hbig, "R": Rbig}[where][:, :K]           # a fresh tensor, or the update in place
+    X = torch.empty((M, K), dtype=torch.bfloat16, device="cuda")
+    B.osc_add_rmsnorm(Hbig[:, :K], Rbig[:, :K], dev_bf16(gb), 1e-6, out, X)
+    B.osc_sync_check()
+    assert np.array_equal(host_bf16_bits(out), Hs_ref)
+    assert np.array_equal(host_bf16_bits(X), X_ref)
+    for big in (Hbig, Rbig, Obig):
+        assert (big[:, K:] == 7.0).all(), "wrote into the padding"
+    if where != "H":
+        assert np.array_equal(host_bf16_bits(Hbig[:, :K]), Hb)
+    if where != "R":
+        assert np.array_equal(host_bf16_bits(Rbig[:, :K]), Rb)
+
+
+@pytest.mark.parametrize("M,K,C", [(129, 384, 2), (300, 1024, 2), (70, 4096, 1), (40, 8192, 3)])
+def test_add_rmsnorm_quantize_extract_bit_exact(B, oracle, M, K, C):
+    rng = np.random.default_rng(M * 5 + K)
+    Hb, gb = residual_rows(rng, M, K), gamma_bits(rng, K)
+    Rb = branch_rows(rng, Hb)
+    lut = rand_lut(rng, K, C)
+    w = B.osc_prepare_weights(dev_bf16(synth.osc_weights_only(1, K, 64, 1)["W"]), lut)
+    sz = B.osc_act_sizes(w, M)
+    xq, sfa, xo = poison(sz.xq_bytes), poison(sz.sfa_bytes), poison(sz.xo_bytes)
+    H = dev_bf16(Hb)
+    B.osc_add_rmsnorm_quantize_extract(w, H, dev_bf16(Rb), dev_bf16(gb), 1e-6, H, xq, sfa, xo)     # stream updated in place
+    B.osc_sync_check()
+    Hs_ref, X_ref = oracle.add_rmsnorm(Hb, Rb, gb, 1e-6)
+    assert np.array_equal(host_bf16_bits(H), Hs_ref)
+    ref = oracle.quantize_extract(X_ref, lut)
+    assert np.array_equal(host_u8(xq)[:sz.xq_bytes].reshape(M, K // 2), ref["xq"])
+    valid = valid_sf_bytes(oracle, M, K)
+    assert np.array_equal(host_u8(sfa)[:sz.sfa_bytes][valid], ref["sf"][valid])
+    if ref["K_o_pad"]:
+        assert np.array_equal(host_u8(xo)[:sz.xo_bytes].view(np.uint16).reshape(M, ref["K_o_pad"]), ref["xo"])
+
+
+def test_add_rmsnorm_linear(B, oracle):
+    M, K, N = 333, 1024, 448
+    rng = np.random.default_rng(21)
+    Hb, gb = residual_rows(rng, M, K), gamma_bits(rng, K)
+    Rb = branch_rows(rng, Hb)
+    c = synth.osc_linear_case(3, M, K, N, 2)
+    w = B.osc_prepare_weights(dev_bf16(c["W"]), c["lut"])
+    ws = poison(B.osc_act_sizes(w, M).workspace_bytes)
+    Y = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+    Hout = torch.empty((M, K), dtype=torch.bfloat16, device="cuda")
+    B.osc_add_rmsnorm_linear(w, dev_bf16(Hb), dev_bf16(Rb), dev_bf16(gb), 1e-6, Hout, Y, ws)
+    B.osc_sync_check()
+    Hs_ref, X_ref = oracle.add_rmsnorm(Hb, Rb, gb, 1e-6)
+    assert np.array_equal(host_bf16_bits(Hout), Hs_ref)
+    Yref, T, *_ = oracle.linear(X_ref, c["W"], c["lut"])
+    assert_within_tolerance(host_f64(Y), Yref, T, "add + rmsnorm + linear")
+    with pytest.raises(B.OscError) as err:          # a missing branch tensor is refused before any launch
+        B.osc_add_rmsnorm_linear(w, dev_bf16(Hb), dev_bf16(Rb)[:0], dev_bf16(gb), 1e-6, Hout, Y, ws)
+    assert err.value.status == -1

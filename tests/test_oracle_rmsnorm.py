@@ -103,3 +103,86 @@ def test_eps_matters_for_small_rows(oracle):
     want = 2.0 ** -10 / np.sqrt(2.0 ** -20 + float(np.float32(eps)))
     assert abs(got - want) <= 2.0 ** -9 * want      # half a bf16 ulp, relative
     assert got < 0.5                                   # without eps it would be 1
+
+
+# ---- the residual update in front of the norm
+
+def _bf16_value(b):
+    """Exact rational value of a finite bf16 bit pattern."""
+    from fractions import Fraction
+    s = -1 if b & 0x8000 else 1
+    e, m = (b >> 7) & 0xFF, b & 0x7F
+    if e == 0:
+        return s * Fraction(m, 1 << 7) * Fraction(2) ** -126
+    return s * (1 + Fraction(m, 1 << 7)) * Fraction(2) ** (e - 127)
+
+
+def _round_to_bf16(q):
+    """Nearest bf16 (ties to even) of an exact rational, by search over the bit patterns of the right sign."""
+    from fractions import Fraction
+    if q == 0:
+        return None   # sign of zero: checked separately
+    sign = 0x8000 if q < 0 else 0
+    a = abs(q)
+    lo, hi = 0, 0x7F80          # magnitudes are ordered like their bit patterns; 0x7F80 stands for 2^128
+    top = Fraction(2) ** 128
+    val = lambda b: top if b == 0x7F80 else _bf16_value(b)
+    while hi - lo > 1:
+        mid = (lo + hi) // 2
+        if val(mid) <= a:
+            lo = mid
+        else:
+            hi = mid
+    dl, dh = a - val(lo), val(hi) - a
+    pick = lo if dl < dh else hi if dh < dl else (lo if lo % 2 == 0 else hi)
+    return sign | pick
+
+
+def test_residual_add_against_rational_arithmetic(oracle):
+    rng = np.random.default_rng(5)
+    a = rng.integers(0, 0x7F80, size=3000).astype(np.uint16) | (rng.integers(0, 2, size=3000).astype(np.uint16) << 15)
+    b = rng.integers(0, 0x7F80, size=3000).astype(np.uint16) | (rng.integers(0, 2, size=3000).astype(np.uint16) << 15)
+    # near-equal exponents (cancellation, carries, ties) are rare among random patterns: plant them
+    b[:1500] = (a[:1500] & 0x8000) ^ (rng.integers(0, 2, size=1500).astype(np.uint16) << 15) | \
+        np.clip((a[:1500] & 0x7FFF).astype(np.int32) + rng.integers(-1200, 1200, size=1500), 0, 0x7F7F).astype(np.uint16)
+    got = oracle.residual_add(a.reshape(1, -1), b.reshape(1, -1)).ravel()
+    for x, y, g in zip(a, b, got):
+        q = _bf16_value(int(x)) + _bf16_value(int(y))
+        want = _round_to_bf16(q)
+        if want is None:
+            assert int(g) & 0x7FFF == 0
+        else:
+            assert int(g) == want, (hex(int(x)), hex(int(y)), hex(int(g)), hex(want))
+
+
+def test_residual_add_special_cases(oracle):
+    one, ulp = 0x3F80, 2.0 ** -7
+    cases = [
+        (bits([1.0]), bits([0.0]), 0x3F80),
+        (bits([1.0]), bits([2.0 ** -8]), 0x3F80),            # tie -> even
+        (bits([1.0 + ulp]), bits([2.0 ** -8]), 0x3F82),      # tie from an odd pattern -> up to the even one
+        (bits([1.0]), bits([2.0 ** -8 + 2.0 ** -15]), 0x3F81),
+        (bits([1.0]), bits([-1.0]), 0x0000),                 # exact cancellation: +0
+        (bits([3.0e38]), bits([3.0e38]), 0x7F80),            # overflow -> +inf
+        (bits([1.0]), bits([1e-30]), 0x3F80),
+        (bits([2.0 ** -126]), bits([-(2.0 ** -127)]), 0x0040),   # into the subnormals, exact
+    ]
+    for h, r, want in cases:
+        got = int(oracle.residual_add(h.reshape(1, 1), r.reshape(1, 1))[0, 0])
+        assert got == want, (hex(got), hex(want))
+    rng = np.random.default_rng(6)
+    H, R = bits(rng.standard_normal((4, 64))), bits(rng.standard_normal((4, 64)) * 0.1)
+    assert np.array_equal(oracle.residual_add(H, R), oracle.residual_add(R, H))            # commutative
+    assert np.array_equal(oracle.residual_add(H, bits(np.zeros((4, 64)))), H)
+
+
+def test_add_rmsnorm_is_the_norm_of_the_updated_stream(oracle):
+    rng = np.random.default_rng(7)
+    H, R = bits(rng.standard_normal((5, 256)) * 3), bits(rng.standard_normal((5, 256)))
+    g = bits(rng.uniform(0.5, 2.0, 256))
+    Hs, Y = oracle.add_rmsnorm(H, R, g, 1e-6)
+    assert np.array_equal(Hs, oracle.residual_add(H, R))
+    assert np.array_equal(Y, oracle.rmsnorm(Hs, g, 1e-6))
+    # against torch: float64 sum rounded through torch's own bf16 conversion, then torch's rms_norm
+    hs_t = (torch.from_numpy(synth.bf16_bits_to_f64(H)) + torch.from_numpy(synth.bf16_bits_to_f64(R))).to(torch.bfloat16)
+    assert np.array_equal(hs_t.view(torch.int16).numpy().view(np.uint16), Hs)
