@@ -117,3 +117,25 @@ def test_grouped_fused_calls_refuse_null_handles():
     assert lib.osc_swiglu_fp8_linear_grouped(None, None, None, 0, 0, None, 0, None, 0, None) == -1
     assert lib.osc_rmsnorm_linear_grouped_gather(None, None, 0, 0, None, C.c_float(0), None, None, 0, None, 0, None, 0,
                                                  None) == -1
+
+
+def test_residual_forms_validate_before_launching():
+    from paper_2604_12782_b200 import binding as B
+    lib = B._lib
+    f = lib.osc_add_rmsnorm
+    f.argtypes = B._SIGS["osc_add_rmsnorm"][1]
+    f.restype = C.c_int
+    ok = dict(H=0x1000, R=0x2000, M=4, K=256, ldh=256, ldr=256, g=0x3000, eps=1e-6, Ho=0x4000, ldo=256, X=0x5000, ldx=256)
+
+    def call(**kw):
+        a = {**ok, **kw}
+        return f(a["H"], a["R"], a["M"], a["K"], a["ldh"], a["ldr"], a["g"], a["eps"], a["Ho"], a["ldo"], a["X"], a["ldx"], None)
+    assert call(M=0) == 0
+    assert call(M=-1) == -1
+    assert call(K=100) == -2 and call(K=8192 + 128, ldh=8320, ldr=8320, ldo=8320, ldx=8320) == -2
+    assert call(R=None) == -1 and call(Ho=None) == -1
+    assert call(ldr=128) == -2 and call(ldo=128) == -2
+    assert call(ldr=260) == -4 and call(R=0x2008) == -4 and call(Ho=0x4004) == -4
+    assert lib.osc_add_rmsnorm_linear(None, None, None, 0, 0, 0, None, C.c_float(0), None, 0, None, 0, None, 0, None) == -1
+    assert lib.osc_add_rmsnorm_quantize_extract(None, None, None, 0, 0, 0, None, C.c_float(0), None, 0, None, None, None,
+                                                None) == -1
