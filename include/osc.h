@@ -17,6 +17,10 @@
  *     *_prepare_* and released by *_destroy.
  *   - stream is a cudaStream_t passed as void*.  All work is enqueued on it; no call
  *     synchronizes except osc_sync_check.  A failed validation launches nothing.
+ *   - Devices: a handle belongs to the device that was current when it was prepared (its buffers live there and
+ *     it remembers that device's SM count); call with that device current and a stream of that device.  One
+ *     process per GPU is the intended arrangement: the path has no exchange step, so several GPUs run
+ *     independent replicas (or disjoint row ranges of M) with no collective.
  *   - Threads: calls on distinct handles (or on one handle with distinct activation buffers and workspaces)
  *     may be made from several host threads at once; the library keeps no mutable state of its own beyond
  *     once-only caches (driver entry point, per-device kernel attributes) that are safe to race on.  Two
