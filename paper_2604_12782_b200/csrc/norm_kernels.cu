@@ -273,6 +273,30 @@ __device__ __forceinline__ float swiglu32(float g, float u) {
     const float d = __fadd_rn(1.0f, exp32(-g));
     return __fmul_rn(__fmul_rn(g, __frcp_rn(d)), u);
 }
+// The same two elements at a time on the packed fp32 instructions of sm_100 (add / mul / fma on register pairs, each
+// half rounded to nearest like the scalar instruction): identical results, about a third fewer issue slots in a kernel
+// that is bound by them.  exp32x2 takes g and computes exp32(-g): fl(g * -log2e) = fl(-g * log2e), and t - n is
+// written as the fused n * -1 + t, whose product is exact.
+__device__ __forceinline__ float2 exp32x2_neg(float2 g) {
+    float2 t = __fmul2_rn(g, make_float2(-1.44269502f, -1.44269502f));
+    t.x = fminf(fmaxf(t.x, -64.0f), 126.0f);
+    t.y = fminf(fmaxf(t.y, -64.0f), 126.0f);
+    const float2 tn = __fadd2_rn(t, make_float2(12582912.0f, 12582912.0f));
+    const float2 n = __fadd2_rn(tn, make_float2(-12582912.0f, -12582912.0f));
+    const int nx = __float_as_int(tn.x) - 0x4B400000, ny = __float_as_int(tn.y) - 0x4B400000;
+    const float2 f = __ffma2_rn(n, make_float2(-1.0f, -1.0f), t);
+    float2 p = make_float2(0.00133335579f, 0.00133335579f);
+    p = __ffma2_rn(p, f, make_float2(0.00961812865f, 0.00961812865f));
+    p = __ffma2_rn(p, f, make_float2(0.0555041097f, 0.0555041097f));
+    p = __ffma2_rn(p, f, make_float2(0.240226507f, 0.240226507f));
+    p = __ffma2_rn(p, f, make_float2(0.693147182f, 0.693147182f));
+    p = __ffma2_rn(p, f, make_float2(1.0f, 1.0f));
+    return __fmul2_rn(p, make_float2(__int_as_float((nx + 127) << 23), __int_as_float((ny + 127) << 23)));
+}
+__device__ __forceinline__ float2 swiglu32x2(float2 g, float2 u) {
+    const float2 d = __fadd2_rn(make_float2(1.0f, 1.0f), exp32x2_neg(g));
+    return __fmul2_rn(__fmul2_rn(g, make_float2(__frcp_rn(d.x), __frcp_rn(d.y))), u);
+}
 
 constexpr int SG_THREADS = 256;
 constexpr int SG_MAXCH = 8;   // 16-byte chunks of h per thread: I <= 256 x 8 x 8
@@ -309,9 +333,9 @@ swiglu_fp8_kernel(const uint16_t* __restrict__ GU, int64_t ldg, int M, int I, ui
             uint32_t o[4];
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-                const float lo = swiglu32(__uint_as_float(gw[j] << 16), __uint_as_float(uw[j] << 16));
-                const float hi = swiglu32(__uint_as_float(gw[j] & 0xFFFF0000u), __uint_as_float(uw[j] & 0xFFFF0000u));
-                o[j] = bf162_bits(__floats2bfloat162_rn(lo, hi));
+                const float2 h2 = swiglu32x2(make_float2(__uint_as_float(gw[j] << 16), __uint_as_float(gw[j] & 0xFFFF0000u)),
+                                             make_float2(__uint_as_float(uw[j] << 16), __uint_as_float(uw[j] & 0xFFFF0000u)));
+                o[j] = bf162_bits(__floats2bfloat162_rn(h2.x, h2.y));
             }
             h[i] = make_uint4(o[0], o[1], o[2], o[3]);
             if (QUANT) {   // packed bf16 magnitudes, two at a time
@@ -346,8 +370,11 @@ swiglu_fp8_kernel(const uint16_t* __restrict__ GU, int64_t ldg, int M, int I, ui
             const uint32_t w[4] = {h[i].x, h[i].y, h[i].z, h[i].w};
             uint32_t e[4];
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
-                e[j] = e4m3x2(__fmul_rn(__uint_as_float(w[j] << 16), inv), __fmul_rn(__uint_as_float(w[j] & 0xFFFF0000u), inv)) & 0xFFFFu;
+            for (int j = 0; j < 4; ++j) {
+                const float2 sc = __fmul2_rn(make_float2(__uint_as_float(w[j] << 16), __uint_as_float(w[j] & 0xFFFF0000u)),
+                                             make_float2(inv, inv));
+                e[j] = e4m3x2(sc.x, sc.y) & 0xFFFFu;
+            }
             *reinterpret_cast<uint2*>(orow + c * 8) = make_uint2(e[0] | (e[1] << 16), e[2] | (e[3] << 16));
         }
     }
