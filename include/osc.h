@@ -54,7 +54,7 @@
  * weight-streaming kernel with the operands swapped and K split over a thread-block cluster; grouped problems
  * with large experts and dense problems with many tiles on 256-row CTA-pair tiles; the rest (up to 128 rows,
  * small experts, and dense problems whose 128-row tiles fit in one wave and beat the pair kernel's estimate) on
- * 128-row tiles.  The NVFP4 form has the few-row kernel (up to 64 rows) and the pair kernel.  Results of
+ * 128-row tiles.  The NVFP4 form runs on the same three kernels (few-row kernel up to 64 rows).  Results of
  * different kernels for the same inputs agree within the accumulation-order rounding of fp32, not bit for
  * bit; one kernel is deterministic run to run.
  * Environment variables for experiments (read by the library, not part of the contract): OSC_DECODE (0 = never,

@@ -1366,9 +1366,12 @@ osc_status osc_nvfp4_prepare_weights(const void* W, int N, int K, int64_t ldw, c
             s = make_tmap(&w->tm_bo2[v], wo, true, (uint64_t)N, (uint64_t)t.Kop * 2, (uint64_t)t.Kop * 2, half);
     }
     if (s == OSC_OK) s = make_tmap_sf(&w->tm_sfw, sfw, (uint64_t)sf16_bytes(N, K) / 512, 4);
-    // 128-row weight tiles of the few-row kernel
-    if (s == OSC_OK) s = make_tmap(&w->tm_b[1], wq, false, (uint64_t)N, K / 2, K / 2, 128);
-    if (s == OSC_OK && t.Kop > 0) s = make_tmap(&w->tm_bo[1], wo, true, (uint64_t)N, (uint64_t)t.Kop * 2, (uint64_t)t.Kop * 2, 128);
+    // weight tiles of the few-row kernel (128 rows) and of the 128-row-tile kernel (64, 128, 192 rows)
+    for (int v = 0; v < 3 && s == OSC_OK; ++v) {
+        s = make_tmap(&w->tm_b[v], wq, false, (uint64_t)N, K / 2, K / 2, 64 * (v + 1));
+        if (s == OSC_OK && t.Kop > 0)
+            s = make_tmap(&w->tm_bo[v], wo, true, (uint64_t)N, (uint64_t)t.Kop * 2, (uint64_t)t.Kop * 2, 64 * (v + 1));
+    }
     if (s != OSC_OK) { delete w; return s; }
     *out = w;
     return OSC_OK;
@@ -1440,7 +1443,26 @@ osc_status osc_nvfp4_gemm(const osc_weights* w, const void* xq, const void* sfa,
         return OSC_OK;
     }
     if (osc_status s = make_tmap(&a.tm_a, xq, false, M, w->K / 2, w->K / 2, 128)) return s;
-    const int bn = gemm_pair_block_n(false, false, (M + 255) / 256, w->N, nkb, w->num_sms);
+    long single_ns = 0, pair_ns = 0;
+    const int bn1 = gemm_block_n((M + 127) / 128, w->N, w->num_sms, &single_ns, 192);
+    const int bn = gemm_pair_block_n(false, false, (M + 255) / 256, w->N, nkb, w->num_sms, &pair_ns);
+    if (!use_pair_kernel(false, M, 1, single_ns * nkb, pair_ns, single_ns <= 390)) {   // 128-row tiles in one wave
+        a.tm_b = w->tm_b[bn1 / 64 - 1];
+        if (w->Kop > 0) {
+            if (osc_status s = make_tmap(&a.tm_ao, xo, true, M, (uint64_t)w->Kop * 2, (uint64_t)w->Kop * 2, 128)) return s;
+            a.tm_bo = w->tm_bo[bn1 / 64 - 1];
+        }
+        a.sfa = static_cast<const uint8_t*>(sfa);
+        a.sfw = w->sfw;
+        a.Y = static_cast<uint16_t*>(Y);
+        a.ldy = ldy;
+        a.M = M; a.N = w->N; a.K = w->K; a.Kop = w->Kop;
+        a.num_sms = w->num_sms;
+        a.out_scale = ldexpf(1.0f, es);
+        cudaError_t e = launch_gemm_nvf4(a, bn1, static_cast<cudaStream_t>(stream));
+        if (e != cudaSuccess) return cuda_fail(e, "gemm_kernel(nvfp4)");
+        return OSC_OK;
+    }
     a.tm_b = w->tm_b2[bn == 256];
     if (w->Kop > 0) {
         if (osc_status s = make_tmap(&a.tm_ao, xo, true, M, (uint64_t)w->Kop * 2, (uint64_t)w->Kop * 2, 128)) return s;

@@ -113,7 +113,8 @@ struct GemmArgs {
 cudaError_t launch_gemm_dual(const GemmArgs& a, int bn, cudaStream_t st);
 cudaError_t launch_gemm_fp8(const GemmArgs& a, int bn, cudaStream_t st);
 cudaError_t launch_gemm_mxf8(const GemmArgs& a, int bn, cudaStream_t st);
-int gemm_block_n(int row_tiles, int N, int num_sms, long* cost_ns = nullptr);
+cudaError_t launch_gemm_nvf4(const GemmArgs& a, int bn, cudaStream_t st);
+int gemm_block_n(int row_tiles, int N, int num_sms, long* cost_ns = nullptr, int widest = 256);
 
 // gemm2_kernels.cu (CTA pairs: 256-row tiles, dense or grouped)
 cudaError_t launch_gemm_dual_pair(const GemmArgs& a, int bn, cudaStream_t st);

@@ -18,6 +18,9 @@
 // MODE_MXF8: the same fallback in its 8-bit micro-scaling form: E4M3 elements with one E8M0 scale per 32
 //            (128 channels and one 128-channel scale block per operand row block and stage, four K=32
 //            block-scaled MMAs taking scale byte k of the TMEM column); nothing to apply in the epilogue.
+// MODE_NVF4: Eq. 5 on NVFP4 (dense only): as MODE_OSC with an E4M3 scale per 16 channels - four 64-channel scale
+//            blocks per stage, one whole TMEM scale column per K=64 MMA - and a power-of-two output scale in the
+//            epilogue; tiles up to 192 columns wide.
 //
 // A tile's first row, last valid row, first scale row and expert come either from arithmetic
 // (dense) or from the device-built schedule (grouped): rows past an expert's end are computed
@@ -31,6 +34,8 @@ namespace osc {
 constexpr int MODE_OSC = 0;
 constexpr int MODE_FP8 = 1;
 constexpr int MODE_MXF8 = 2;
+constexpr int MODE_NVF4 = 3;   // Eq. 5 on NVFP4: E4M3 scale per 16 channels (four 64-channel scale blocks per stage), BF16
+                               // branch, power-of-two output scale
 
 constexpr int BM = 128;            // rows per tile = TMEM lanes
 constexpr int ROW_BYTES = 128;     // bytes per operand row and stage (one 128-byte swizzle row)
@@ -45,21 +50,25 @@ template <int MODE, int BN>
 struct Cfg {
     static constexpr int SFB_ATOMS = (BN > 128) ? 2 : 1;  // 128-row scale blocks a tile can touch
     static constexpr bool SCALED = MODE != MODE_FP8;
-    static constexpr int KA = (MODE == MODE_OSC) ? 2 : 1;   // 128-channel scale blocks per stage
-    // TMEM columns of one stage's scales (A: 8, B: 2 x atoms x 4; MXFP8 uses half of them); the FP8 mode keeps
-    // no scales in TMEM
-    static constexpr int SF_COLS = SCALED ? 8 + 2 * SFB_ATOMS * 4 : 0;
+    static constexpr bool DUAL = MODE == MODE_OSC || MODE == MODE_NVF4;   // has the BF16 branch (Path B)
+    static constexpr int KA = (MODE == MODE_OSC) ? 2 : (MODE == MODE_NVF4) ? 4 : 1;   // 512-byte scale blocks per stage
+    static constexpr int SF_K = (MODE == MODE_NVF4) ? 64 : 128;                       // channels per scale block
+    static constexpr int KA_ROOM = KA > 2 ? KA : 2;
+    // TMEM columns of one stage's scales (A: 4 per block, B: 4 per block and 128-row atom; MXFP8 uses half of
+    // them); the FP8 mode keeps no scales in TMEM
+    static constexpr int SF_COLS = SCALED ? KA_ROOM * 4 + KA_ROOM * SFB_ATOMS * 4 : 0;
     static constexpr int ACC_STAGES = (2 * BN + SF_COLS <= TMEM_COLS) ? 2 : 1;
     static constexpr int B_BYTES = BN * ROW_BYTES;
-    static constexpr int SFA_BYTES = SCALED ? 1024 : 0;              // room for two blocks (MXFP8 fills one)
-    static constexpr int SFB_BYTES = SCALED ? SFB_ATOMS * 1024 : 0;
+    static constexpr int SF_ROWBLOCK = KA_ROOM * 512;                // one 128-row block's scales of a stage (MXFP8 fills half)
+    static constexpr int SFA_BYTES = SCALED ? SF_ROWBLOCK : 0;
+    static constexpr int SFB_BYTES = SCALED ? SFB_ATOMS * SF_ROWBLOCK : 0;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES + SFA_BYTES + SFB_BYTES;  // multiple of 1024
     static constexpr int EPI_WARP_BYTES = (BN / 64) * G_EPI_TILE_BYTES;            // one lane quarter's 32 x BN outputs
     static constexpr int EPI_BYTES = 4 * EPI_WARP_BYTES;
     static constexpr int STAGES = (224 * 1024 - EPI_BYTES) / STAGE_BYTES;
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
     static constexpr int TM_SFA = ACC_STAGES * BN;  // TMEM column of the activation scales
-    static constexpr int TM_SFB = TM_SFA + 8;       // weight scales
+    static constexpr int TM_SFB = TM_SFA + KA_ROOM * 4;   // weight scales
     static_assert(STAGE_BYTES % 1024 == 0, "stage must keep 1024-byte alignment");
     static_assert(TM_SFA + SF_COLS <= TMEM_COLS, "TMEM budget");
     static_assert(STAGES >= 3, "ring too shallow");
@@ -136,7 +145,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
         fence_barrier_init();
         prefetch_tmap(&args.tm_a);
         prefetch_tmap(&args.tm_b);
-        if (MODE == MODE_OSC && args.Kop > 0) {
+        if (C::DUAL && args.Kop > 0) {
             prefetch_tmap(&args.tm_ao);
             prefetch_tmap(&args.tm_bo);
         }
@@ -157,11 +166,11 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
     const int num_n = (N + BN - 1) / BN;
     const int total = num_m * num_n;
     // K blocks: Path A / FP8 first, then Path B
-    const int elems_per_kb = (MODE == MODE_OSC) ? 256 : 128;
+    const int elems_per_kb = C::DUAL ? 256 : 128;
     const int nkb_a = (K + elems_per_kb - 1) / elems_per_kb;
-    const int nkb_b = (MODE == MODE_OSC) ? args.Kop / 64 : 0;
+    const int nkb_b = C::DUAL ? args.Kop / 64 : 0;
     const int nkb = nkb_a + nkb_b;
-    const int katoms_total = K / 128;   // 128-channel scale blocks along K
+    const int katoms_total = K / C::SF_K;   // scale blocks along K
     const int natoms = (N + 127) / 128;  // 128-row scale blocks of one expert's weights
     constexpr int KA = C::KA;
 
@@ -190,7 +199,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
                                 const int atom = min(ti.n0 / 128 + j, natoms - 1);
                                 const uint8_t* sw = args.sfw +
                                     (((int64_t)ti.expert * natoms + atom) * katoms_total + KA * kb) * 512;
-                                bulk_load(st + A_BYTES + C::B_BYTES + C::SFA_BYTES + j * 1024, sw, sfb, &full_bar[s]);
+                                bulk_load(st + A_BYTES + C::B_BYTES + C::SFA_BYTES + j * C::SF_ROWBLOCK, sw, sfb, &full_bar[s]);
                             }
                         } else {
                             mbar_arrive_expect_tx(&full_bar[s], A_BYTES + C::B_BYTES);
@@ -215,6 +224,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
         int acc = 0;
         uint32_t acc_ph = 0;
         constexpr uint32_t IDESC_A = (MODE == MODE_OSC)    ? idesc_mxf4(BM, BN)
+                                     : (MODE == MODE_NVF4) ? idesc_nvf4(BM, BN)
                                      : (MODE == MODE_MXF8) ? idesc_mxf8(BM, BN)
                                                            : idesc_e4m3(BM, BN);
         constexpr uint32_t IDESC_B = idesc_bf16(BM, BN);
@@ -257,7 +267,27 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
                                          (kb | k) ? 1u : 0u);
                             }
                         }
-                    } else if (MODE == MODE_OSC) {
+                    } else if (MODE == MODE_NVF4 && kb < nkb_a) {
+                        // four 64-channel scale blocks per stage, one per K = 64 instruction (a whole scale column each)
+                        const int ka = min(4, katoms_total - 4 * kb);
+                        const uint64_t sfa_d = sf_hi | (uint64_t)((sbase + A_BYTES + C::B_BYTES) >> 4);
+                        const uint64_t sfb_d = sf_hi | (uint64_t)((sbase + A_BYTES + C::B_BYTES + C::SFA_BYTES) >> 4);
+#pragma unroll
+                        for (int a = 0; a < 4; ++a) {
+                            if (a < ka) {
+                                tc_copy_sf(tmem_base + C::TM_SFA + a * 4, sfa_d + (uint64_t)(a * 32));
+#pragma unroll
+                                for (int j = 0; j < C::SFB_ATOMS; ++j)
+                                    tc_copy_sf(tmem_base + C::TM_SFB + a * (C::SFB_ATOMS * 4) + j * 4,
+                                               sfb_d + (uint64_t)(j * (C::SF_ROWBLOCK / 16) + a * 32));
+                            }
+                        }
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)
+                            if (k < ka)
+                                mma_nvf4(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC_A, tmem_base + C::TM_SFA + k * 4,
+                                         sfb_tm + k * (C::SFB_ATOMS * 4), (kb | k) ? 1u : 0u);
+                    } else if (C::DUAL) {
 #pragma unroll
                         for (int k = 0; k < 4; ++k) mma_f16(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC_B, 1u);
                     } else if (MODE == MODE_MXF8) {
@@ -343,6 +373,10 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
                                 lo = lo * (sxr * wx);
                                 hi = hi * (sxr * wy);
                             }
+                            if (MODE == MODE_NVF4) {   // back out of the scaled domain: an exact power of two
+                                lo *= args.out_scale;
+                                hi *= args.out_scale;
+                            }
                             const __nv_bfloat162 b2 = __floats2bfloat162_rn(lo, hi);
                             o[i] = *reinterpret_cast<const uint32_t*>(&b2);
                         }
@@ -399,19 +433,20 @@ done:
 // measured on B200 at 96 stages: ~230 ns for 64 columns, ~265 ns for 128, ~390 ns for 192; 256 extrapolated.  With many
 // tiles the widest wins (least time per column), with few a narrower one that still fits in one wave.
 // cost_ns (optional) receives the estimate for one K stage times the waves.  OSC_BLOCK_N overrides.
-int gemm_block_n(int row_tiles, int N, int num_sms, long* cost_ns) {
+int gemm_block_n(int row_tiles, int N, int num_sms, long* cost_ns, int widest) {
     static const int forced = [] {
         const char* e = getenv("OSC_BLOCK_N");
         const int v = e ? atoi(e) : 0;
         return (v == 64 || v == 128 || v == 192 || v == 256) ? v : 0;
     }();
     if (cost_ns) *cost_ns = 0;
-    if (forced) return forced;
+    if (forced) return forced < widest ? forced : widest;
     const int cand[4] = {256, 192, 128, 64};
     const long stage_ns[4] = {470, 390, 265, 230};
     long best = -1;
     int best_bn = 64;
     for (int i = 0; i < 4; ++i) {
+        if (cand[i] > widest) continue;
         const long tiles = (long)row_tiles * ((N + cand[i] - 1) / cand[i]);
         const long waves = (tiles + num_sms - 1) / num_sms;
         const long cost = waves * stage_ns[i];
@@ -449,6 +484,14 @@ cudaError_t launch_gemm_fp8(const GemmArgs& a, int bn, cudaStream_t st) {
         case 128: return launch_cfg<MODE_FP8, 128>(a, st);
         case 192: return launch_cfg<MODE_FP8, 192>(a, st);
         default: return launch_cfg<MODE_FP8, 256>(a, st);
+    }
+}
+// NVFP4: up to 192 columns (a 256-wide tile's stage, with twice the scale bytes, leaves room for two stages only)
+cudaError_t launch_gemm_nvf4(const GemmArgs& a, int bn, cudaStream_t st) {
+    switch (bn) {
+        case 64: return launch_cfg<MODE_NVF4, 64>(a, st);
+        case 128: return launch_cfg<MODE_NVF4, 128>(a, st);
+        default: return launch_cfg<MODE_NVF4, 192>(a, st);
     }
 }
 cudaError_t launch_gemm_mxf8(const GemmArgs& a, int bn, cudaStream_t st) {

@@ -53,8 +53,11 @@ def run_case(B, oracle, Xb, Wb, lut16, what):
     return w, sz, ws, Y, ex
 
 
+# The last three rows reach the 128-row-tile kernel with 64-, 128- and 192-column tiles (65-128 rows; the width follows
+# from the number of tiles against the number of SMs), the first two the few-row kernel, the rest the pair kernel.
 @pytest.mark.parametrize("M,K,N,kind", [(1, 128, 64, "one"), (64, 512, 512, "one"), (127, 384, 192, "two"),
-                                        (129, 256, 320, "empty"), (300, 640, 448, "one"), (515, 128, 64, "two")])
+                                        (129, 256, 320, "empty"), (300, 640, 448, "one"), (515, 128, 64, "two"),
+                                        (100, 640, 320, "two"), (97, 256, 12288, "one"), (128, 128, 24576, "two")])
 def test_nvfp4_linear_small(B, oracle, M, K, N, kind):
     c = synth.osc16_linear_case(M + K, M, K, N)
     rng = np.random.default_rng(N)
