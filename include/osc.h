@@ -430,7 +430,7 @@ osc_status osc_dyn_linear(const osc_weights* w, const void* X, int M, int64_t ld
  * The table lists local channels 0..15 per 16-channel group: lut16 is host int8 [K/16][lut_c], -1 = none.
  * Scale bytes: 512-byte blocks of 128 rows x 64 channels,
  *   byte(r, b) = ((r/128)*(K/64) + b/4)*512 + (r%32)*16 + ((r%128)/32)*4 + b%4   (b = block index along K),
- * ceil(rows/128) * (K/64) * 512 bytes per tensor.  Dense problems only; same conventions as osc_linear.
+ * ceil(rows/128) * (K/64) * 512 bytes per tensor.  Same conventions as osc_linear; the grouped form follows below.
  * The handle is an osc_weights accepted only by the osc_nvfp4_* calls and osc_weights_destroy;
  * osc_nvfp4_weight_sizes and osc_nvfp4_act_sizes fill the structs of their MXFP4 counterparts. */
 osc_status osc_nvfp4_weight_sizes(int N, int K, const int8_t* lut16, int lut_c, osc_weight_sizes_t* out);
@@ -443,6 +443,18 @@ osc_status osc_nvfp4_gemm(const osc_weights* w, const void* xq, const void* sfa,
                           int64_t ldy, void* stream);
 osc_status osc_nvfp4_linear(const osc_weights* w, const void* X, int M, int64_t ldx, int ex, void* Y, int64_t ldy,
                             void* workspace, size_t workspace_bytes, void* stream);
+
+/* Grouped (MoE) form of the NVFP4 path: E experts stacked as W[E][N][K] (ldw = K), one table and one weight
+ * tensor exponent ew for the layer, every expert quantized on its own (its scale blocks start on a 128-row
+ * block); buffers are E times the dense sizes (osc_nvfp4_weight_sizes_grouped).  Rows of X_perm sorted by
+ * expert and off as in osc_linear_grouped; expert e's activation scale rows start at scale row
+ * sum_{e'<e} roundup(m_e', 128); workspace from osc_nvfp4_act_sizes(w, M_total).  A grouped handle is accepted
+ * by osc_nvfp4_act_sizes, osc_nvfp4_linear_grouped and osc_weights_destroy only. */
+osc_status osc_nvfp4_weight_sizes_grouped(int E, int N, int K, const int8_t* lut16, int lut_c, osc_weight_sizes_t* out);
+osc_status osc_nvfp4_prepare_weights_grouped(const void* W, int E, int N, int K, const int8_t* lut16, int lut_c, int ew,
+                                             void* wq, void* sfw, void* wo, void* meta, void* stream, osc_weights** out);
+osc_status osc_nvfp4_linear_grouped(const osc_weights* w, const void* X_perm, const int32_t* off, int M_total, int64_t ldx,
+                                    int ex, void* Y, int64_t ldy, void* workspace, size_t workspace_bytes, void* stream);
 
 #ifdef __cplusplus
 }

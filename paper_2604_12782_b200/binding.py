@@ -106,6 +106,9 @@ _SIGS = {
     "osc_dyn_linear": (_i, [_vp, _vp, _i, _i64, _vp, _i64, _vp, _sz, _vp]),
     "osc_nvfp4_weight_sizes": (_i, [_i, _i, _vp, _i, C.POINTER(WeightSizes)]),
     "osc_nvfp4_prepare_weights": (_i, [_vp, _i, _i, _i64, _vp, _i, _i, _vp, _vp, _vp, _vp, _vp, C.POINTER(_vp)]),
+    "osc_nvfp4_weight_sizes_grouped": (_i, [_i, _i, _i, _vp, _i, C.POINTER(WeightSizes)]),
+    "osc_nvfp4_prepare_weights_grouped": (_i, [_vp, _i, _i, _i, _vp, _i, _i, _vp, _vp, _vp, _vp, _vp, C.POINTER(_vp)]),
+    "osc_nvfp4_linear_grouped": (_i, [_vp, _vp, _vp, _i, _i64, _i, _vp, _i64, _vp, _sz, _vp]),
     "osc_nvfp4_act_sizes": (_i, [_vp, _i, C.POINTER(ActSizes)]),
     "osc_nvfp4_quantize_extract": (_i, [_vp, _vp, _i, _i64, _i, _vp, _vp, _vp, _vp]),
     "osc_nvfp4_gemm": (_i, [_vp, _vp, _vp, _vp, _i, _i, _vp, _i64, _vp]),
@@ -589,6 +592,32 @@ def osc_nvfp4_prepare_weights(W: torch.Tensor, lut16, ew: int, stream=None) -> O
     w = OscWeights(h.value, bufs)
     w.E, w.N, w.K, w.K_o, w.K_o_pad, w.sizes, w.ew = 1, N, K, sz.K_o, sz.K_o_pad, sz, int(ew)
     return w
+
+
+def osc_nvfp4_prepare_weights_grouped(W: torch.Tensor, lut16, ew: int, stream=None) -> OscWeights:
+    """W: cuda bf16 [E, N, K] contiguous; one table and one tensor exponent for all experts."""
+    E, N, K = W.shape
+    assert W.is_contiguous()
+    lut16 = _lut16(lut16, K)
+    sz = WeightSizes()
+    _check(_lib.osc_nvfp4_weight_sizes_grouped(E, N, K, lut16.ctypes.data, lut16.shape[1], C.byref(sz)))
+    bufs = {k: _alloc(getattr(sz, k + "_bytes"), W.device) for k in ("wq", "sfw", "wo", "meta")}
+    h = _vp()
+    _check(_lib.osc_nvfp4_prepare_weights_grouped(_ptr(W), E, N, K, lut16.ctypes.data, lut16.shape[1], int(ew),
+                                                  _ptr(bufs["wq"]), _ptr(bufs["sfw"]),
+                                                  _ptr(bufs["wo"]) if sz.wo_bytes else None, _ptr(bufs["meta"]),
+                                                  _stream(stream), C.byref(h)))
+    w = OscWeights(h.value, bufs)
+    w.E, w.N, w.K, w.K_o, w.K_o_pad, w.sizes, w.ew = E, N, K, sz.K_o, sz.K_o_pad, sz, int(ew)
+    return w
+
+
+def osc_nvfp4_linear_grouped(w: OscWeights, X: torch.Tensor, off: torch.Tensor, ex: int, Y: torch.Tensor,
+                             workspace: torch.Tensor, stream=None):
+    M = X.shape[0]
+    _check(_lib.osc_nvfp4_linear_grouped(w.ptr, _ptr(X), _ptr(off), M, X.stride(0) if M else w.K, int(ex), _ptr(Y),
+                                         Y.stride(0) if M else w.N, _ptr(workspace),
+                                         workspace.numel() * workspace.element_size(), _stream(stream)))
 
 
 def osc_nvfp4_act_sizes(w: OscWeights, M: int) -> ActSizes:

@@ -1302,26 +1302,30 @@ static osc_status widen_lut16(const int8_t* lut16, int K, int C, std::vector<int
 }
 
 osc_status osc_nvfp4_weight_sizes(int N, int K, const int8_t* lut16, int lut_c, osc_weight_sizes_t* out) {
+    return osc_nvfp4_weight_sizes_grouped(1, N, K, lut16, lut_c, out);
+}
+osc_status osc_nvfp4_weight_sizes_grouped(int E, int N, int K, const int8_t* lut16, int lut_c, osc_weight_sizes_t* out) {
     if (!out) return fail(OSC_ERR_INVALID_ARG, "out is null");
-    if (osc_status s = check_nk(1, N, K)) return s;
+    if (osc_status s = check_nk(E, N, K)) return s;
     std::vector<int8_t> lut;
     if (osc_status s = widen_lut16(lut16, K, lut_c, &lut)) return s;
     Table t;
     if (osc_status s = parse_lut(lut.data(), K, 2 * (lut_c > 0 ? lut_c : 1), &t)) return s;
     out->K_o = t.Ko;
     out->K_o_pad = t.Kop;
-    out->wq_bytes = (size_t)N * (K / 2);
-    out->sfw_bytes = sf16_bytes(N, K);
-    out->wo_bytes = (size_t)N * t.Kop * 2;
+    out->wq_bytes = (size_t)E * N * (K / 2);
+    out->sfw_bytes = (size_t)E * sf16_bytes(N, K);
+    out->wo_bytes = (size_t)E * N * t.Kop * 2;
     out->meta_bytes = meta_table_bytes(K, t.Ko);
     return OSC_OK;
 }
 
-osc_status osc_nvfp4_prepare_weights(const void* W, int N, int K, int64_t ldw, const int8_t* lut16, int lut_c, int ew,
-                                     void* wq, void* sfw, void* wo, void* meta, void* stream, osc_weights** out) {
+static osc_status nvfp4_prepare_impl(const void* W, int E, int N, int K, int64_t ldw, const int8_t* lut16, int lut_c, int ew,
+                                     void* wq, void* sfw, void* wo, void* meta, void* stream, osc_weights** out,
+                                     bool grouped) {
     if (!out) return fail(OSC_ERR_INVALID_ARG, "out is null");
     *out = nullptr;
-    if (osc_status s = check_nk(1, N, K)) return s;
+    if (osc_status s = check_nk(E, N, K)) return s;
     if (ew < -100 || ew > 100) return fail(OSC_ERR_INVALID_ARG, "tensor exponent %d outside -100..100", ew);
     std::vector<int8_t> lut;
     if (osc_status s = widen_lut16(lut16, K, lut_c, &lut)) return s;
@@ -1343,7 +1347,7 @@ osc_status osc_nvfp4_prepare_weights(const void* W, int N, int K, int64_t ldw, c
     if (e != cudaSuccess) return cuda_fail(e, "cudaMemcpyAsync(meta)");
     osc_weights* w = new (std::nothrow) osc_weights();
     if (!w) return fail(OSC_ERR_INVALID_ARG, "out of host memory");
-    w->E = 1; w->N = N; w->K = K; w->Ko = t.Ko; w->Kop = t.Kop; w->grouped = false; w->dynamic = false;
+    w->E = E; w->N = N; w->K = K; w->Ko = t.Ko; w->Kop = t.Kop; w->grouped = grouped; w->dynamic = false;
     w->nvfp4 = true; w->ew = ew;
     w->wq = static_cast<const uint8_t*>(wq);
     w->sfw = static_cast<const uint8_t*>(sfw);
@@ -1352,49 +1356,64 @@ osc_status osc_nvfp4_prepare_weights(const void* W, int N, int K, int64_t ldw, c
     w->prefix = reinterpret_cast<const int32_t*>(m8 + (size_t)Kg * 4);
     w->idx_o = reinterpret_cast<const int32_t*>(m8 + (size_t)Kg * 8);
     w->num_sms = di.num_sms;
-    CUtensorMap tm_w;
-    osc_status s = make_tmap_x(&tm_w, W, N, K, ldw);
-    if (s == OSC_OK) {
-        e = launch_quant_extract_nvfp4(tm_w, N, K, w->mask, w->prefix, w->idx_o, wq, sfw, t.Kop ? wo : nullptr, t.Ko, t.Kop,
+    osc_status s = OSC_OK;
+    const size_t sfw_e = sf16_bytes(N, K);
+    for (int x = 0; x < E && s == OSC_OK; ++x) {   // every expert on its own: its scale blocks start on a 128-row block
+        CUtensorMap tm_w;
+        s = make_tmap_x(&tm_w, static_cast<const uint16_t*>(W) + (size_t)x * N * ldw, N, K, ldw);
+        if (s != OSC_OK) break;
+        e = launch_quant_extract_nvfp4(tm_w, N, K, w->mask, w->prefix, w->idx_o, static_cast<uint8_t*>(wq) + (size_t)x * N * (K / 2),
+                                       static_cast<uint8_t*>(sfw) + (size_t)x * sfw_e,
+                                       t.Kop ? static_cast<uint16_t*>(wo) + (size_t)x * N * t.Kop : nullptr, t.Ko, t.Kop,
                                        di.num_sms, ew, st);
         if (e != cudaSuccess) s = cuda_fail(e, "quant_extract_kernel(nvfp4 weights)");
     }
     for (int v = 0; v < 2 && s == OSC_OK; ++v) {
         const int half = (v == 0 ? 192 : 256) / 2;
-        s = make_tmap(&w->tm_b2[v], wq, false, (uint64_t)N, K / 2, K / 2, half);
+        s = make_tmap(&w->tm_b2[v], wq, false, (uint64_t)E * N, K / 2, K / 2, half);
         if (s == OSC_OK && t.Kop > 0)
-            s = make_tmap(&w->tm_bo2[v], wo, true, (uint64_t)N, (uint64_t)t.Kop * 2, (uint64_t)t.Kop * 2, half);
+            s = make_tmap(&w->tm_bo2[v], wo, true, (uint64_t)E * N, (uint64_t)t.Kop * 2, (uint64_t)t.Kop * 2, half);
     }
-    if (s == OSC_OK) s = make_tmap_sf(&w->tm_sfw, sfw, (uint64_t)sf16_bytes(N, K) / 512, 4);
+    if (s == OSC_OK) s = make_tmap_sf(&w->tm_sfw, sfw, (uint64_t)E * sfw_e / 512, 4);
     // weight tiles of the few-row kernel (128 rows) and of the 128-row-tile kernel (64, 128, 192 rows)
     for (int v = 0; v < 3 && s == OSC_OK; ++v) {
-        s = make_tmap(&w->tm_b[v], wq, false, (uint64_t)N, K / 2, K / 2, 64 * (v + 1));
+        s = make_tmap(&w->tm_b[v], wq, false, (uint64_t)E * N, K / 2, K / 2, 64 * (v + 1));
         if (s == OSC_OK && t.Kop > 0)
-            s = make_tmap(&w->tm_bo[v], wo, true, (uint64_t)N, (uint64_t)t.Kop * 2, (uint64_t)t.Kop * 2, 64 * (v + 1));
+            s = make_tmap(&w->tm_bo[v], wo, true, (uint64_t)E * N, (uint64_t)t.Kop * 2, (uint64_t)t.Kop * 2, 64 * (v + 1));
     }
     if (s != OSC_OK) { delete w; return s; }
     *out = w;
     return OSC_OK;
 }
 
+osc_status osc_nvfp4_prepare_weights(const void* W, int N, int K, int64_t ldw, const int8_t* lut16, int lut_c, int ew,
+                                     void* wq, void* sfw, void* wo, void* meta, void* stream, osc_weights** out) {
+    return nvfp4_prepare_impl(W, 1, N, K, ldw, lut16, lut_c, ew, wq, sfw, wo, meta, stream, out, false);
+}
+osc_status osc_nvfp4_prepare_weights_grouped(const void* W, int E, int N, int K, const int8_t* lut16, int lut_c, int ew,
+                                             void* wq, void* sfw, void* wo, void* meta, void* stream, osc_weights** out) {
+    return nvfp4_prepare_impl(W, E, N, K, K, lut16, lut_c, ew, wq, sfw, wo, meta, stream, out, true);
+}
+
 osc_status osc_nvfp4_act_sizes(const osc_weights* w, int M, osc_act_sizes_t* out) {
     if (!w || !out) return fail(OSC_ERR_INVALID_ARG, "null argument");
     if (!w->nvfp4) return fail(OSC_ERR_INVALID_ARG, "MXFP4 weights: use osc_act_sizes");
     if (M < 0) return fail(OSC_ERR_INVALID_ARG, "M = %d is negative", M);
+    const int64_t max_tiles = w->grouped ? (int64_t)M / 128 + w->E : ((int64_t)M + 127) / 128;
     out->xq_bytes = (size_t)M * (w->K / 2);
-    out->sfa_bytes = sf16_bytes(M, w->K);
+    out->sfa_bytes = (size_t)max_tiles * (w->K / 64) * 512;
     out->xo_bytes = (size_t)M * w->Kop * 2;
-    out->sched_bytes = 0;
+    out->sched_bytes = w->grouped ? sched_ints(max_tiles) * 4 + sched_ints(max_tiles256(M, w->E)) * 4 : 0;
     out->xq_offset = 0;
     out->sfa_offset = out->xq_offset + align256(out->xq_bytes);
     out->xo_offset = out->sfa_offset + align256(out->sfa_bytes);
     out->sched_offset = out->xo_offset + align256(out->xo_bytes);
-    out->workspace_bytes = out->sched_offset;
+    out->workspace_bytes = out->sched_offset + align256(out->sched_bytes);
     return OSC_OK;
 }
 
-osc_status osc_nvfp4_quantize_extract(const osc_weights* w, const void* X, int M, int64_t ldx, int ex, void* xq,
-                                      void* sfa, void* xo, void* stream) {
+static osc_status nvfp4_quantize_impl(const osc_weights* w, const void* X, int M, int64_t ldx, int ex, void* xq, void* sfa,
+                                      void* xo, void* stream, const int32_t* sched, int max_tiles) {
     if (osc_status s = check_act(w, X, M, ldx, false, true)) return s;
     if (ex < -100 || ex > 100) return fail(OSC_ERR_INVALID_ARG, "tensor exponent %d outside -100..100", ex);
     if (M == 0) return OSC_OK;
@@ -1403,13 +1422,19 @@ osc_status osc_nvfp4_quantize_extract(const osc_weights* w, const void* X, int M
     CUtensorMap tm_x;
     if (osc_status s = make_tmap_x(&tm_x, X, M, w->K, ldx)) return s;
     cudaError_t e = launch_quant_extract_nvfp4(tm_x, M, w->K, w->mask, w->prefix, w->idx_o, xq, sfa, w->Kop ? xo : nullptr,
-                                               w->Ko, w->Kop, w->num_sms, ex, static_cast<cudaStream_t>(stream));
+                                               w->Ko, w->Kop, w->num_sms, ex, static_cast<cudaStream_t>(stream), sched, max_tiles);
     if (e != cudaSuccess) return cuda_fail(e, "quant_extract_kernel(nvfp4)");
     return OSC_OK;
 }
+osc_status osc_nvfp4_quantize_extract(const osc_weights* w, const void* X, int M, int64_t ldx, int ex, void* xq,
+                                      void* sfa, void* xo, void* stream) {
+    if (w && w->grouped) return fail(OSC_ERR_INVALID_ARG, "grouped weights: use osc_nvfp4_linear_grouped");
+    return nvfp4_quantize_impl(w, X, M, ldx, ex, xq, sfa, xo, stream, nullptr, 0);
+}
 
-osc_status osc_nvfp4_gemm(const osc_weights* w, const void* xq, const void* sfa, const void* xo, int M, int ex, void* Y,
-                          int64_t ldy, void* stream) {
+static osc_status nvfp4_gemm_impl(const osc_weights* w, const void* xq, const void* sfa, const void* xo, int M, int ex, void* Y,
+                                  int64_t ldy, void* stream, const int32_t* sched, int max_tiles, const int32_t* sched2,
+                                  int max_tiles2) {
     if (!w) return fail(OSC_ERR_INVALID_ARG, "weights handle is null");
     if (!w->nvfp4) return fail(OSC_ERR_INVALID_ARG, "MXFP4 weights: use osc_gemm_dual");
     if (M < 0) return fail(OSC_ERR_INVALID_ARG, "M = %d is negative", M);
@@ -1423,7 +1448,7 @@ osc_status osc_nvfp4_gemm(const osc_weights* w, const void* xq, const void* sfa,
     GemmArgs a;
     memset(&a, 0, sizeof a);
     const int nkb = (w->K + 255) / 256 + w->Kop / 64;
-    if (use_decode_kernel(false, M, w->N, nkb, w->num_sms, true)) {   // few rows: weights stream once, K split over a cluster
+    if (use_decode_kernel(w->grouped, M, w->N, nkb, w->num_sms, true)) {   // few rows: weights stream once, K split over a cluster
         const uint32_t tok_box = (uint32_t)((M + 15) / 16 * 16);
         if (osc_status s = make_tmap(&a.tm_a, xq, false, M, w->K / 2, w->K / 2, tok_box)) return s;
         a.tm_b = w->tm_b[1];
@@ -1444,9 +1469,12 @@ osc_status osc_nvfp4_gemm(const osc_weights* w, const void* xq, const void* sfa,
     }
     if (osc_status s = make_tmap(&a.tm_a, xq, false, M, w->K / 2, w->K / 2, 128)) return s;
     long single_ns = 0, pair_ns = 0;
-    const int bn1 = gemm_block_n((M + 127) / 128, w->N, w->num_sms, &single_ns, 192);
-    const int bn = gemm_pair_block_n(false, false, (M + 255) / 256, w->N, nkb, w->num_sms, &pair_ns);
-    if (!use_pair_kernel(false, M, 1, single_ns * nkb, pair_ns, single_ns <= 390)) {   // 128-row tiles in one wave
+    const int bn1 = gemm_block_n(sched ? max_tiles : (M + 127) / 128, w->N, w->num_sms, &single_ns, 192);
+    const long row_tiles2 = w->grouped ? (max_tiles2 > w->E / 2 ? max_tiles2 - w->E / 2 : 1) : (M + 255) / 256;
+    const int bn = gemm_pair_block_n(false, false, row_tiles2, w->N, nkb, w->num_sms, &pair_ns);
+    a.sched = sched; a.max_tiles = max_tiles;
+    a.sched2 = sched2; a.max_tiles2 = max_tiles2;
+    if (!use_pair_kernel(w->grouped, M, w->E, single_ns * nkb, pair_ns, single_ns <= 390)) {   // 128-row tiles
         a.tm_b = w->tm_b[bn1 / 64 - 1];
         if (w->Kop > 0) {
             if (osc_status s = make_tmap(&a.tm_ao, xo, true, M, (uint64_t)w->Kop * 2, (uint64_t)w->Kop * 2, 128)) return s;
@@ -1469,7 +1497,8 @@ osc_status osc_nvfp4_gemm(const osc_weights* w, const void* xq, const void* sfa,
         a.tm_bo = w->tm_bo2[bn == 256];
     }
     a.tm_sfw = w->tm_sfw;
-    if (osc_status s = make_tmap_sf(&a.tm_sfa, sfa, (uint64_t)sf16_bytes(M, w->K) / 512, 4)) return s;
+    const uint64_t sf_row_blocks = w->grouped ? (uint64_t)max_tiles : (uint64_t)((M + 127) / 128);
+    if (osc_status s = make_tmap_sf(&a.tm_sfa, sfa, sf_row_blocks * (w->K / 64), 4)) return s;
     if (osc_status s = make_tmap(&a.tm_y, Y, true, M, (uint64_t)w->N * 2, (uint64_t)ldy * 2, 32)) return s;
     if (osc_status s = make_tmap(&a.tm_y16, Y, true, M, (uint64_t)w->N * 2, (uint64_t)ldy * 2, 16)) return s;
     a.sfa = static_cast<const uint8_t*>(sfa);
@@ -1484,9 +1513,47 @@ osc_status osc_nvfp4_gemm(const osc_weights* w, const void* xq, const void* sfa,
     return OSC_OK;
 }
 
+osc_status osc_nvfp4_gemm(const osc_weights* w, const void* xq, const void* sfa, const void* xo, int M, int ex, void* Y,
+                          int64_t ldy, void* stream) {
+    if (w && w->grouped) return fail(OSC_ERR_INVALID_ARG, "grouped weights: use osc_nvfp4_linear_grouped");
+    return nvfp4_gemm_impl(w, xq, sfa, xo, M, ex, Y, ldy, stream, nullptr, 0, nullptr, 0);
+}
+
+osc_status osc_nvfp4_linear_grouped(const osc_weights* w, const void* X_perm, const int32_t* off, int M_total, int64_t ldx,
+                                    int ex, void* Y, int64_t ldy, void* workspace, size_t workspace_bytes, void* stream) {
+    if (osc_status s = check_act(w, X_perm, M_total, ldx, false, true)) return s;
+    if (!w->grouped) return fail(OSC_ERR_INVALID_ARG, "dense weights: use osc_nvfp4_linear");
+    if (ex < -100 || ex > 100) return fail(OSC_ERR_INVALID_ARG, "tensor exponent %d outside -100..100", ex);
+    if (M_total == 0) return OSC_OK;
+    if (!off) return fail(OSC_ERR_INVALID_ARG, "off is null");
+    osc_act_sizes_t sz;
+    osc_nvfp4_act_sizes(w, M_total, &sz);
+    if (!workspace || !aligned16(workspace)) return fail(OSC_ERR_ALIGN, "workspace must be non-null and 16-byte aligned");
+    if (workspace_bytes < sz.workspace_bytes)
+        return fail(OSC_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", workspace_bytes, sz.workspace_bytes);
+    if (!Y) return fail(OSC_ERR_INVALID_ARG, "Y is null");
+    if (ldy < w->N) return fail(OSC_ERR_SHAPE, "ldy = %lld < N = %d", (long long)ldy, w->N);
+    if (ldy % 8 || !aligned16(Y)) return fail(OSC_ERR_ALIGN, "Y must be 16-byte aligned and ldy a multiple of 8");
+    const int es = ex + w->ew;
+    if (es < -120 || es > 120) return fail(OSC_ERR_INVALID_ARG, "sum of the tensor exponents %d outside -120..120", es);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int max_tiles = M_total / 128 + w->E;
+    const int max_tiles2 = max_tiles256(M_total, w->E);
+    int32_t* sched = reinterpret_cast<int32_t*>(ws + sz.sched_offset);
+    int32_t* sched2 = use_pair_kernel(true, M_total, w->E) ? sched + sched_ints(max_tiles) : nullptr;
+    cudaError_t e = launch_build_sched(off, w->E, sched, max_tiles, sched2, max_tiles2, st);
+    if (e != cudaSuccess) return cuda_fail(e, "build_sched_kernel");
+    if (osc_status s = nvfp4_quantize_impl(w, X_perm, M_total, ldx, ex, ws + sz.xq_offset, ws + sz.sfa_offset, ws + sz.xo_offset,
+                                           stream, sched, max_tiles)) return s;
+    return nvfp4_gemm_impl(w, ws + sz.xq_offset, ws + sz.sfa_offset, ws + sz.xo_offset, M_total, ex, Y, ldy, stream, sched,
+                           max_tiles, sched2, max_tiles2);
+}
+
 osc_status osc_nvfp4_linear(const osc_weights* w, const void* X, int M, int64_t ldx, int ex, void* Y, int64_t ldy,
                             void* workspace, size_t workspace_bytes, void* stream) {
     if (osc_status s = check_act(w, X, M, ldx, false, true)) return s;
+    if (w->grouped) return fail(OSC_ERR_INVALID_ARG, "grouped weights: use osc_nvfp4_linear_grouped");
     if (M == 0) return OSC_OK;
     osc_act_sizes_t sz;
     osc_nvfp4_act_sizes(w, M, &sz);

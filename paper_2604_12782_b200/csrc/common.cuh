@@ -57,7 +57,8 @@ cudaError_t launch_quant_extract(const CUtensorMap& tm_x, int M, int K, const ui
                                  const int32_t* sched, int max_tiles, int num_sms, cudaStream_t st);
 cudaError_t launch_quant_extract_nvfp4(const CUtensorMap& tm_x, int M, int K, const uint32_t* mask,
                                        const int32_t* prefix, const int32_t* idx_o, void* xq, void* sf, void* xo, int Ko,
-                                       int Kop, int num_sms, int tensor_e, cudaStream_t st);
+                                       int Kop, int num_sms, int tensor_e, cudaStream_t st,
+                                       const int32_t* sched = nullptr, int max_tiles = 0);
 cudaError_t launch_fp8_quant(const void* X, int64_t ldx, int M, int K, void* x8, void* sx, cudaStream_t st);
 cudaError_t launch_mxfp8_quant(const void* X, int64_t ldx, int M, int K, void* x8, void* sf, const int32_t* sched,
                                int max_tiles, cudaStream_t st);

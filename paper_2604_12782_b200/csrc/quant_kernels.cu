@@ -821,8 +821,9 @@ cudaError_t launch_quant_extract(const CUtensorMap& tm_x, int M, int K, const ui
 // NVFP4 / G = 16 form (dense only): tensor-level scale 2^tensor_e
 cudaError_t launch_quant_extract_nvfp4(const CUtensorMap& tm_x, int M, int K, const uint32_t* mask,
                                        const int32_t* prefix, const int32_t* idx_o, void* xq, void* sf, void* xo, int Ko,
-                                       int Kop, int num_sms, int tensor_e, cudaStream_t st) {
-    return launch_quant_extract_fmt<FMT_NVFP4>(tm_x, M, K, mask, prefix, idx_o, xq, sf, xo, Ko, Kop, nullptr, 0, num_sms,
+                                       int Kop, int num_sms, int tensor_e, cudaStream_t st, const int32_t* sched,
+                                       int max_tiles) {
+    return launch_quant_extract_fmt<FMT_NVFP4>(tm_x, M, K, mask, prefix, idx_o, xq, sf, xo, Ko, Kop, sched, max_tiles, num_sms,
                                                tensor_e, st);
 }
 

@@ -111,7 +111,7 @@ def test_random_dense_shape(B, oracle, seed):
     B.osc_sync_check()
 
 
-@pytest.mark.parametrize("seed", range(12))
+@pytest.mark.parametrize("seed", range(16))
 def test_random_grouped_shape(B, oracle, seed):
     """Expert row counts drawn from {0, 1, under one tile, several tiles}: both tile schedules, experts that end
     anywhere inside a tile, runs of empty experts."""
@@ -122,7 +122,7 @@ def test_random_grouped_shape(B, oracle, seed):
     if counts.sum() == 0:
         counts[0] = 5
     K, N = 128 * int(rng.integers(1, 7)), 64 * int(rng.integers(1, 9))
-    which = ["osc", "fp8", "mxfp8"][seed % 3]
+    which = ["osc", "fp8", "mxfp8", "nvfp4"][seed % 4]
     what = f"grouped {which} counts={counts.tolist()} K={K} N={N}"
     if which == "osc":
         c = synth.moe_gate_up_case(E, counts, K=K, N=N, seed=seed)
@@ -140,6 +140,18 @@ def test_random_grouped_shape(B, oracle, seed):
 
         def ref(x, wt):
             return oracle.fp8_linear(x, wt)[:2]
+    elif which == "nvfp4":
+        c = synth.moe_gate_up_case(E, counts, K=K, N=N, seed=seed)
+        lut16 = np.stack([rng.permutation(16)[:1] for _ in range(K // 16)]).astype(np.int8)
+        ex, ew = synth.nvfp4_tensor_exponent(c["X"]), synth.nvfp4_tensor_exponent(c["W"])
+        w = B.osc_nvfp4_prepare_weights_grouped(dev_bf16(c["W"].reshape(E * N, K)).view(E, N, K), lut16, ew)
+        ws = poison(B.osc_nvfp4_act_sizes(w, c["M"]).workspace_bytes)
+
+        def run(w_, X_, off_, Y_, ws_):
+            B.osc_nvfp4_linear_grouped(w_, X_, off_, ex, Y_, ws_)
+
+        def ref(x, wt):
+            return oracle.nvfp4_linear(x, wt, lut16, ex, ew)[:2]
     else:
         c = synth.moe_down_case(E, counts, K=K, N=N, seed=seed)
         w = B.osc_mxfp8_prepare_weights_grouped(dev_bf16(c["W"].reshape(E * N, K)).view(E, N, K))

@@ -107,3 +107,42 @@ def test_nvfp4_qkv_shape(B, oracle):
     Yref, T = oracle.nvfp4_gemm(act, wts, rows)
     assert_within_tolerance(host_f64(Y[torch.from_numpy(rows.astype(np.int64)).cuda()]), Yref, T, "nvfp4 qkv")
     assert not torch.isnan(Y.float()).any()
+
+
+@pytest.mark.parametrize("counts", [[3, 0, 130, 1, 257, 128], [300, 0, 5, 256, 129, 511, 1, 385], [700, 64, 0, 900]])
+def test_nvfp4_grouped(B, oracle, counts):
+    """Grouped (MoE) NVFP4: per expert equal to the dense call on that expert's rows and weights (same kernels, same
+    operands, scale rows shifted to the expert's 128-row block), and within tolerance of the oracle; small experts
+    take 128-row tiles, large ones the pair kernel; experts that end inside a tile, empty and one-row experts."""
+    counts = np.array(counts)
+    E, K, N = counts.size, 384, 320
+    M = int(counts.sum())
+    off_h = synth.offsets_from_counts(counts)
+    c = synth.osc16_linear_case(50 + E, M, K, N)
+    rng = np.random.default_rng(E)
+    Wb = synth.f32_to_bf16_bits((0.02 * rng.standard_normal((E, N, K))).astype(np.float32))
+    ex, ew = synth.nvfp4_tensor_exponent(c["X"]), synth.nvfp4_tensor_exponent(Wb)
+    w = B.osc_nvfp4_prepare_weights_grouped(dev_bf16(Wb.reshape(E * N, K)).view(E, N, K), c["lut16"], ew)
+    sz = B.osc_nvfp4_act_sizes(w, M)
+    ws = poison(sz.workspace_bytes)
+    big = torch.full((M + 2, N + 8), 7.0, dtype=torch.bfloat16, device="cuda")
+    Y = big[1:M + 1, :N]
+    B.osc_nvfp4_linear_grouped(w, dev_bf16(c["X"]), torch.from_numpy(off_h).cuda(), ex, Y, ws)
+    B.osc_sync_check()
+    guard = big.clone()
+    guard[1:M + 1, :N] = 7.0
+    assert (guard == 7.0).all(), "wrote outside Y"
+    Yh = host_f64(Y)
+    for e in range(E):
+        r0, r1 = int(off_h[e]), int(off_h[e + 1])
+        if r1 > r0:
+            Yref, T, act, _ = oracle.nvfp4_linear(c["X"][r0:r1], Wb[e], c["lut16"], ex, ew)
+            assert_within_tolerance(Yh[r0:r1], Yref, T, f"grouped nvfp4, expert {e} ({r1 - r0} rows)")
+            # the quantizer's codes of the expert's rows: bit for bit
+            got = host_u8(ws)[sz.xq_offset:sz.xq_offset + sz.xq_bytes].reshape(M, K // 2)[r0:r1]
+            assert np.array_equal(got, act["xq"])
+    wd = B.osc_nvfp4_prepare_weights(dev_bf16(Wb[0]), c["lut16"], ew)
+    with pytest.raises(B.OscError):
+        B.osc_nvfp4_linear_grouped(wd, dev_bf16(c["X"]), torch.from_numpy(off_h).cuda(), ex, Y, ws)
+    with pytest.raises(B.OscError):
+        B.osc_nvfp4_linear(w, dev_bf16(c["X"]), ex, Y, ws)
