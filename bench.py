@@ -884,6 +884,22 @@ def run_sweep(args):
     rows.append({"name": "moe.gate_up(grouped, gathered from 8192 tokens)", "M": Mt, "K": K, "N": N, "K_o": w.K_o, "ms": msg,
                  "tflops": (f4 + f16) / msg / 1e9, "pct_roofline": 100 * troofg / (msg * 1e-3), "roof_us": troofg * 1e6,
                  "speedup_vs_permuted_input": ms / msg})
+    # the same grouped problem on NVFP4 / G = 16 (the same protected channels, written as a table per 16-group)
+    lut32 = np.asarray(c["lut"]).reshape(K // 32, -1)
+    lut16 = np.full((K // 16, lut32.shape[1]), -1, np.int8)
+    for g in range(K // 32):
+        for j, ch in enumerate(lut32[g]):
+            if ch >= 0:
+                lut16[2 * g + (ch >= 16), j] = ch % 16
+    ex4, ew4 = synth.nvfp4_tensor_exponent(c["X"]), synth.nvfp4_tensor_exponent(c["W"])
+    w4 = B.osc_nvfp4_prepare_weights_grouped(Wd, lut16, ew4)
+    ws4 = torch.empty(B.osc_nvfp4_act_sizes(w4, Mt).workspace_bytes, dtype=torch.uint8, device="cuda")
+    torch.cuda.synchronize()
+    ms4 = time_loop(torch, lambda i: B.osc_nvfp4_linear_grouped(w4, Xd, off, ex4, Y, ws4), steps, warm)
+    B.osc_sync_check()
+    rows.append({"name": "moe.gate_up_nvfp4_g16(grouped)", "M": Mt, "K": K, "N": N, "K_o": w4.K_o, "ms": ms4,
+                 "tflops": (f4 + f16) / ms4 / 1e9, "vs_mxfp4": ms4 / ms})
+    del w4, ws4
     wg, Yg = w, Y
     del Xd, Wd, ws
     c = synth.moe_down_case(E, counts, weight_pool=8)
