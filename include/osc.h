@@ -17,6 +17,11 @@
  *     *_prepare_* and released by *_destroy.
  *   - stream is a cudaStream_t passed as void*.  All work is enqueued on it; no call
  *     synchronizes except osc_sync_check.  A failed validation launches nothing.
+ *     Kernels are launched with programmatic stream serialization (a kernel's prologue may overlap its
+ *     predecessor's tail, and the few-row GEMM streams weights ahead of its dependency wait); every
+ *     *_prepare_* call ends with a plain launch, so a handle may be used on the same stream directly behind
+ *     its preparation without a synchronisation.  On another stream, order the use behind the preparation
+ *     with an event as for any other stream work.
  *   - Devices: a handle belongs to the device that was current when it was prepared (its buffers live there and
  *     it remembers that device's SM count); call with that device current and a stream of that device.  One
  *     process per GPU is the intended arrangement: the path has no exchange step, so several GPUs run

@@ -64,6 +64,20 @@ static EncodeTiledFn encode_fn() {
     return fn;
 }
 
+// The encoder is a driver call and wants a current context.  A host thread that has made no CUDA call of its own
+// yet has none (runtime calls bind the primary context lazily, a bare driver call does not): on
+// CUDA_ERROR_INVALID_CONTEXT the primary context of the thread's current device is made current and the call is
+// repeated once.
+template <typename... A>
+static CUresult encode_tiled(EncodeTiledFn fn, A... a) {
+    CUresult r = fn(a...);
+    if (r == CUDA_ERROR_INVALID_CONTEXT) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess && cudaSetDevice(dev) == cudaSuccess) r = fn(a...);
+    }
+    return r;
+}
+
 // Row-major [rows, row_bytes] operand, tiles of box_rows x 128 bytes, 128-byte swizzle, zero fill.
 static osc_status make_tmap(CUtensorMap* tm, const void* base, bool bf16, uint64_t rows, uint64_t row_bytes,
                             uint64_t pitch_bytes, uint32_t box_rows) {
@@ -75,9 +89,9 @@ static osc_status make_tmap(CUtensorMap* tm, const void* base, bool bf16, uint64
     cuuint64_t gstr[1] = {pitch_bytes};
     cuuint32_t box[2] = {static_cast<cuuint32_t>(128 / esz), box_rows};
     cuuint32_t estr[2] = {1, 1};
-    CUresult r = fn(tm, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 2,
-                    const_cast<void*>(base), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    CUresult r = encode_tiled(fn, tm, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 2u,
+                              const_cast<void*>(base), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return fail(OSC_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
     return OSC_OK;
 }
@@ -91,9 +105,9 @@ static osc_status make_tmap_x(CUtensorMap* tm, const void* base, uint64_t rows, 
     cuuint64_t gstr[1] = {ld * 2};
     cuuint32_t box[2] = {64, 128};
     cuuint32_t estr[2] = {1, 1};
-    CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstr, box, estr,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    CUresult r = encode_tiled(fn, tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2u, const_cast<void*>(base), gdim, gstr, box, estr,
+                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return fail(OSC_ERR_CUDA, "cuTensorMapEncodeTiled(X) failed with code %d", (int)r);
     return OSC_OK;
 }
@@ -108,9 +122,9 @@ static osc_status make_tmap_sf(CUtensorMap* tm, const void* base, uint64_t block
     cuuint64_t gstr[1] = {512};
     cuuint32_t box[2] = {128, box_blocks};
     cuuint32_t estr[2] = {1, 1};
-    CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void*>(base), gdim, gstr, box, estr,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    CUresult r = encode_tiled(fn, tm, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2u, const_cast<void*>(base), gdim, gstr, box, estr,
+                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return fail(OSC_ERR_CUDA, "cuTensorMapEncodeTiled(scales) failed with code %d", (int)r);
     return OSC_OK;
 }
@@ -366,6 +380,7 @@ static osc_status prepare_impl(const void* W, int E, int N, int K, int64_t ldw, 
         if (e != cudaSuccess) { delete w; return cuda_fail(e, "retile_sf_kernel"); }
         s = make_tmap_sf(&w->tm_sfw_tiled, tiled, (uint64_t)tiled_sf_bytes(N, K) / 512);
     }
+    if (s == OSC_OK && (e = launch_prepare_fence(st)) != cudaSuccess) s = cuda_fail(e, "prepare_fence_kernel");
     if (s != OSC_OK) { delete w; return s; }
     *out = w;
     return OSC_OK;
@@ -802,6 +817,8 @@ static osc_status fp8_prepare_impl(const void* W, int E, int N, int K, int64_t l
     if (osc_status s = device_info(&di)) return s;
     cudaError_t e = launch_fp8_quant(W, ldw, E * N, K, w8, sw, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return cuda_fail(e, "fp8_quant_kernel(weights)");
+    e = launch_prepare_fence(static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(e, "prepare_fence_kernel");
     osc_fp8_weights* w = new (std::nothrow) osc_fp8_weights();
     if (!w) return fail(OSC_ERR_INVALID_ARG, "out of host memory");
     w->E = E; w->N = N; w->K = K; w->grouped = grouped;
@@ -1061,6 +1078,7 @@ static osc_status mxfp8_prepare_impl(const void* W, int E, int N, int K, int64_t
                                                static_cast<uint8_t*>(sfw) + (size_t)ex * sf_bytes(N, K), nullptr, 0, stream))
             return s;
     }
+    if (cudaError_t e = launch_prepare_fence(static_cast<cudaStream_t>(stream))) return cuda_fail(e, "prepare_fence_kernel");
     osc_mxfp8_weights* w = new (std::nothrow) osc_mxfp8_weights();
     if (!w) return fail(OSC_ERR_INVALID_ARG, "out of host memory");
     w->E = E; w->N = N; w->K = K; w->grouped = grouped;
@@ -1368,6 +1386,7 @@ static osc_status nvfp4_prepare_impl(const void* W, int E, int N, int K, int64_t
                                        di.num_sms, ew, st);
         if (e != cudaSuccess) s = cuda_fail(e, "quant_extract_kernel(nvfp4 weights)");
     }
+    if (s == OSC_OK && (e = launch_prepare_fence(st)) != cudaSuccess) s = cuda_fail(e, "prepare_fence_kernel");
     for (int v = 0; v < 2 && s == OSC_OK; ++v) {
         const int half = (v == 0 ? 192 : 256) / 2;
         s = make_tmap(&w->tm_b2[v], wq, false, (uint64_t)E * N, K / 2, K / 2, half);

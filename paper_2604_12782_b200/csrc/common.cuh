@@ -67,6 +67,8 @@ cudaError_t launch_dyn_quant_extract(const void* X, int64_t ldx, int M, int K, v
 cudaError_t launch_build_sched(const int32_t* off, int E, int32_t* sched128, int max_tiles128, int32_t* sched256,
                                int max_tiles256, cudaStream_t st);
 
+cudaError_t launch_prepare_fence(cudaStream_t st);   // last launch of every weight preparation
+
 cudaError_t launch_gather_quantized(const int32_t* row_token, int T, int K, int Kop, const void* xq_u, const void* sf_u,
                                     const void* xo_u, void* xq, void* sf, void* xo, const int32_t* sched, int max_tiles,
                                     cudaStream_t st);

@@ -711,6 +711,21 @@ cudaError_t launch_retile_sf(const uint8_t* src, uint8_t* dst, int N, int K, int
     return cudaGetLastError();
 }
 
+// ------------------------------------------------------------ end of a weight preparation
+// The quantizers signal their dependents at their first instruction, so with programmatic launches a
+// kernel two launches further down the stream can begin (up to its own grid_dependency_wait) while a
+// weight quantizer is still writing; the few-row GEMM uses exactly that freedom to stream weights ahead
+// of its wait.  Weights therefore must be complete before any later launch can begin: every
+// *_prepare_* call ends with this kernel, launched without the programmatic attribute (it starts after
+// everything before it on the stream has finished and its writes are visible) and without an early
+// trigger (whatever follows starts after it has finished).
+__global__ void prepare_fence_kernel() {}
+
+cudaError_t launch_prepare_fence(cudaStream_t st) {
+    prepare_fence_kernel<<<1, 32, 0, st>>>();
+    return cudaGetLastError();
+}
+
 // ------------------------------------------------- gather of quantized rows (MoE dispatch)
 // In a mixture-of-experts layer every token goes to several experts, and Algorithm 2 does not depend on the expert
 // (one table per layer): the tokens are quantized once, and this kernel copies each token's packed codes, scale bytes

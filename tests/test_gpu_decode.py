@@ -174,3 +174,52 @@ def test_decode_kernel_nvfp4(B, oracle, env, M, K, N, kind, split):
         guard = big.clone()
         guard[1:M + 1, :N] = 7.0
         assert (guard == 7.0).all(), "wrote outside Y"
+
+
+@pytest.mark.parametrize("kind", ["osc", "fp8", "mxfp8", "nvfp4"])
+def test_linear_right_after_prepare(B, oracle, kind):
+    """A few-row linear issued on the same stream directly behind its weight preparation, with nothing in between:
+    the few-row kernel streams weights ahead of its dependency wait, so the preparation has to be complete before
+    any later launch may begin.  The buffers the preparation allocates are made to reuse memory full of 0xFF, so
+    weights read too early would show.  Checked against the oracle and against the same call after a sync."""
+    M, K, N = 16, 4096, 2048
+    if kind in ("osc", "nvfp4"):
+        c = synth.osc_linear_case(5, M, K, N, 2) if kind == "osc" else synth.osc16_linear_case(5, M, K, N)
+    else:
+        c = synth.fp8_linear_case(5, M, K, N)
+    X, W = dev_bf16(c["X"]), dev_bf16(c["W"])
+    Y1 = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+    Y2 = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+    ws = poison(64 << 20)
+    # blocks of the sizes the preparation will ask for, filled with 0xFF and handed back to the caching allocator
+    for nbytes in (N * K, N * K // 2, N * 4, N * 512 * 2, N * K // 32, N * K // 16, 1 << 20):
+        poison(nbytes)
+    torch.cuda.synchronize()
+    if kind == "osc":
+        w = B.osc_prepare_weights(W, c["lut"])
+        B.osc_linear(w, X, Y1, ws)
+        torch.cuda.synchronize()
+        B.osc_linear(w, X, Y2, ws)
+        Yref, T, *_ = oracle.linear(c["X"], c["W"], c["lut"])
+    elif kind == "fp8":
+        w = B.osc_fp8_prepare_weights(W)
+        B.osc_fp8_linear(w, X, Y1, ws)
+        torch.cuda.synchronize()
+        B.osc_fp8_linear(w, X, Y2, ws)
+        Yref, T, *_ = oracle.fp8_linear(c["X"], c["W"])
+    elif kind == "mxfp8":
+        w = B.osc_mxfp8_prepare_weights(W)
+        B.osc_mxfp8_linear(w, X, Y1, ws)
+        torch.cuda.synchronize()
+        B.osc_mxfp8_linear(w, X, Y2, ws)
+        Yref, T, *_ = oracle.mxfp8_linear(c["X"], c["W"])
+    else:
+        ex, ew = synth.nvfp4_tensor_exponent(c["X"]), synth.nvfp4_tensor_exponent(c["W"])
+        w = B.osc_nvfp4_prepare_weights(W, c["lut16"], ew)
+        B.osc_nvfp4_linear(w, X, ex, Y1, ws)
+        torch.cuda.synchronize()
+        B.osc_nvfp4_linear(w, X, ex, Y2, ws)
+        Yref, T, *_ = oracle.nvfp4_linear(c["X"], c["W"], c["lut16"], ex, ew)
+    B.osc_sync_check()
+    assert_within_tolerance(host_f64(Y1), Yref, T, f"{kind}: linear directly behind prepare")
+    assert torch.equal(Y1.view(torch.int16), Y2.view(torch.int16)), "the call behind the preparation differs from the call after a sync"
