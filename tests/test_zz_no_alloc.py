@@ -57,3 +57,43 @@ def test_static_scratch_rejects_oversized_problems(B):
         B.osc_linear_static(w, X, Y)
     assert e.value.status == -5 and "osc_linear_static" in str(e.value)
     B.osc_linear_static(w, X[:0], Y[:0])              # M == 0 stays a no-op
+
+
+def test_static_scratch_from_host_threads(B):
+    """Several host threads call the entry point at once (ctypes drops the interpreter lock during the call), all on
+    one stream as the shared scratch requires, all on the same problem so that the order in which their launches
+    interleave on the stream does not matter: every result equals the one a single call gives."""
+    import threading
+    c = synth.osc_linear_case(21, 200, 512, 256, 2)
+    w = B.osc_prepare_weights(dev_bf16(c["W"]), c["lut"])
+    X = dev_bf16(c["X"])
+    Y0 = torch.full((200, 256), float("nan"), dtype=torch.bfloat16, device="cuda")
+    B.osc_linear_static(w, X, Y0)
+    B.osc_sync_check()
+    st = torch.cuda.Stream()
+    nthreads, rounds = 4, 10
+    Ys = [[torch.full((200, 256), float("nan"), dtype=torch.bfloat16, device="cuda") for _ in range(rounds)]
+          for _ in range(nthreads)]
+    torch.cuda.synchronize()
+    errors = []
+    start = threading.Barrier(nthreads)
+
+    def worker(i):
+        try:
+            start.wait()
+            for Y in Ys[i]:
+                B.osc_linear_static(w, X, Y, stream=st)
+        except Exception as e:
+            errors.append((i, repr(e)))
+
+    ts = [threading.Thread(target=worker, args=(i,)) for i in range(nthreads)]
+    for t in ts:
+        t.start()
+    for t in ts:
+        t.join()
+    st.synchronize()
+    B.osc_sync_check()
+    assert not errors, errors
+    for i in range(nthreads):
+        for Y in Ys[i]:
+            assert torch.equal(Y.view(torch.int16), Y0.view(torch.int16))
