@@ -9,12 +9,10 @@
 // 16 KB + BN x 128 B, which is what bounds the single-CTA kernel (L2 -> shared-memory feed).
 // No cluster-multicast loads are used: every CTA fetches its own operands.
 //
-// Roles per CTA: per issue lane one TMA producer warp and one MMA issuer warp (the latter active only
-// in the leader CTA, rank 0; warp 1 also owns TMEM), then eight epilogue warps.  With two accumulators
-// (BN = 192) there are TWO issue lanes: lane L owns half of the shared-memory ring, accumulator L and
-// scale buffer L, and works on every other tile of the pair.  One elected thread issues all tcgen05
-// instructions of a tile, and its per-stage bookkeeping (barrier wait, commit, loop) leaves the tensor
-// pipe idle ~60 ns per stage; with two lanes the other lane's MMAs fill those gaps.  Barriers:
+// Roles per CTA: warp 0 is the TMA producer, warp 1 the MMA issuer (active only in the leader CTA, rank 0;
+// it also owns TMEM), then eight epilogue warps.  One elected lane of the converged issuer warp issues all
+// tcgen05 instructions of a tile.  (A second producer / issuer pair working on every other tile, each on half
+// of the ring, was measured and brought nothing: the tensor pipe is the limit, not the issue rate.)  Barriers:
 //   full[s]   leader's only: one arrive.expect_tx by the leader's producer for the bytes of BOTH
 //             CTAs; the peer's loads credit the leader's barrier (cta_group::2 loads).
 //   empty[s]  one per CTA, released for both CTAs by one multicast tcgen05.commit of the leader.
@@ -64,9 +62,8 @@ struct Cfg {
     static constexpr int SFA_BYTES = SCALED ? KA * 512 : 0;
     static constexpr int SFB_BYTES = SCALED ? SFB_ATOMS * KA * 512 : 0;
     static constexpr int STAGE_BYTES = (A_BYTES + B_BYTES + SFA_BYTES + SFB_BYTES + 1023) / 1024 * 1024;
-    static constexpr int LANES = 1;                      // issue lanes (a second one brought nothing, see above)
-    static constexpr int THREADS = 32 * (2 * LANES + EPI_WARPS);
-    static constexpr int EPI_FIRST_WARP = 2 * LANES;
+    static constexpr int THREADS = 32 * (2 + EPI_WARPS);   // producer, issuer, epilogue warps
+    static constexpr int EPI_FIRST_WARP = 2;
     static constexpr int SLICES = (BN + 63) / 64;        // 64-column output slices of a tile
     static constexpr int LAST_W = BN - 64 * (SLICES - 1);  // width of the last one (64 or 48)
     // The ring's depth decides how well the operand feed rides out latency (240-wide tiles: 4 / 5 / 6 stages =
@@ -76,8 +73,7 @@ struct Cfg {
     static constexpr int EPI_FULL = EPI_WARPS * EPI_TILE_BYTES;   // one 32 x 64 staging tile per epilogue warp
     static constexpr int EPI_HALVES = ((SMEM_BUDGET - EPI_FULL / 2) / STAGE_BYTES > (SMEM_BUDGET - EPI_FULL) / STAGE_BYTES) ? 2 : 1;
     static constexpr int EPI_BYTES = EPI_FULL / EPI_HALVES;
-    static constexpr int STAGES = ((SMEM_BUDGET - EPI_BYTES) / STAGE_BYTES) / LANES * LANES;
-    static constexpr int SPL = STAGES / LANES;          // ring stages per lane
+    static constexpr int STAGES = (SMEM_BUDGET - EPI_BYTES) / STAGE_BYTES;
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/ + EPI_BYTES;
     // TMEM columns.  Accumulators start at multiples of ACC_STRIDE; a 240-wide tile keeps its second
     // accumulator at column 256 and tucks the scales into the gaps (activation scales at 240..247,
@@ -93,7 +89,7 @@ struct Cfg {
     static_assert(TILED_SF ? (TM_SFA + 4 * KA <= 256 && TM_SFB + KA * SFB_ATOMS * 4 <= TMEM_COLS && SF_BUFS == 1)
                            : (TM_SFA + SF_BUFS * SF_COLS <= TMEM_COLS), "TMEM budget");
     static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
-    static_assert(SPL >= 3, "ring too shallow");
+    static_assert(STAGES >= 3, "ring too shallow");
     static_assert((SLICES + 1) / 2 <= 2, "an epilogue warp drains at most two slices of a tile");
     static_assert(BN % 16 == 0 && BN <= 256 && (LAST_W == 64 || LAST_W == 48), "tile width");
 };
@@ -196,30 +192,25 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
         return ti;
     };
 
-    constexpr int LANES = C::LANES;
-    constexpr int SPL = C::SPL;
-    if (warp < 2 * LANES && (warp & 1) == 0) {
-        // ------------------------------------------- TMA producer of issue lane L (both CTAs)
-        const int L = warp >> 1;
+    if (warp == 0) {
+        // ------------------------------------------------------- TMA producer (both CTAs)
         int s = 0;
         uint32_t ph = 0;
-        uint64_t* fullL = full_bar + L * SPL;
-        uint64_t* emptyL = empty_bar + L * SPL;
-        uint8_t* ring = smem + L * SPL * C::STAGE_BYTES;
-        const uint32_t full0 = map_to_cta(smem_u32(fullL), 0);  // the leader's full barriers of this lane
-        for (int t = pair_id + L * num_pairs; t < total; t += LANES * num_pairs) {
+        uint8_t* ring = smem;
+        const uint32_t full0 = map_to_cta(smem_u32(full_bar), 0);  // the leader's full barriers
+        for (int t = pair_id; t < total; t += num_pairs) {
             const Tile ti = tile_of(t);
             const int n0 = ti.n0;
             const int arow = ti.row0 + (int)rank * BM;                        // my 128 activation rows
             const int brow = ti.expert * N + n0 + (int)rank * (BN / 2);       // my half of the weight rows
             const int sfa_blk = (ti.sf_row0 / 128 + (int)rank) * katoms_total;  // my 128-row scale blocks
             for (int kb = 0; kb < nkb; ++kb) {
-                if (!wait_bounded(&emptyL[s], ph ^ 1u, abort_flag, 11)) goto done;
+                if (!wait_bounded(&empty_bar[s], ph ^ 1u, abort_flag, 11)) goto done;
                 const uint32_t st = smem_u32(ring + s * C::STAGE_BYTES);
                 const uint32_t fb = full0 + (uint32_t)s * 8u;
                 if (elect_one()) {
                     if (kb < nkb_a) {
-                        if (rank == 0) mbar_arrive_expect_tx(&fullL[s], C::SCALED ? C::TX_A : C::TX_B);
+                        if (rank == 0) mbar_arrive_expect_tx(&full_bar[s], C::SCALED ? C::TX_A : C::TX_B);
                         tma_load_2d_pair(st, &args.tm_a, fb, kb * ROW_BYTES, arow);
                         tma_load_2d_pair(st + A_BYTES, &args.tm_b, fb, kb * ROW_BYTES, brow);
                         if (C::SCALED) {
@@ -235,25 +226,22 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
                         }
                     } else {
                         const int kk = kb - nkb_a;
-                        if (rank == 0) mbar_arrive_expect_tx(&fullL[s], C::TX_B);
+                        if (rank == 0) mbar_arrive_expect_tx(&full_bar[s], C::TX_B);
                         tma_load_2d_pair(st, &args.tm_ao, fb, kk * 64, arow);
                         tma_load_2d_pair(st + A_BYTES, &args.tm_bo, fb, kk * 64, brow);
                     }
                 }
                 __syncwarp();
-                if (++s == SPL) { s = 0; ph ^= 1u; }
+                if (++s == STAGES) { s = 0; ph ^= 1u; }
             }
         }
-    } else if (warp < 2 * LANES) {
-        // ---------------------- MMA issuer of issue lane L (leader CTA only, one elected lane)
+    } else if (warp == 1) {
+        // ------------------------------------ MMA issuer (leader CTA only, one elected lane)
         if (rank == 0) {
-            const int L = warp >> 1;
             int s = 0;
             uint32_t ph = 0;
             uint32_t acc_ph = 0;
-            int acc = (LANES == 2) ? L : 0;
-            uint64_t* fullL = full_bar + L * SPL;
-            uint64_t* emptyL = empty_bar + L * SPL;
+            int acc = 0;
             constexpr uint32_t IDESC_A = (MODE == MODE_OSC)    ? idesc_mxf4(2 * BM, BN)
                                          : (MODE == MODE_NVF4) ? idesc_nvf4(2 * BM, BN)
                                          : (MODE == MODE_MXF8) ? idesc_mxf8(2 * BM, BN)
@@ -261,15 +249,15 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
             constexpr uint32_t IDESC_B = idesc_bf16(2 * BM, BN);
             const uint64_t desc_hi = smem_desc_sw128(0);  // everything but the start address
             const uint64_t sf_hi = smem_desc_sf(0);
-            const uint32_t ring0 = smem_u32(smem + L * SPL * C::STAGE_BYTES);
-            for (int t = pair_id + L * num_pairs; t < total; t += LANES * num_pairs) {
+            const uint32_t ring0 = smem_u32(smem);
+            for (int t = pair_id; t < total; t += num_pairs) {
                 const int n0 = tile_of(t).n0;
                 if (!wait_bounded(&tempty_bar[acc], acc_ph ^ 1u, abort_flag, 12)) goto done;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * C::ACC_STRIDE);
                 const uint32_t sfb_tm = tmem_base + C::TM_SFB + (C::TILED_SF ? 0u : (uint32_t)((n0 % 128) / 32));
                 for (int kb = 0; kb < nkb; ++kb) {
-                    if (!wait_bounded(&fullL[s], ph, abort_flag, 13)) goto done;
+                    if (!wait_bounded(&full_bar[s], ph, abort_flag, 13)) goto done;
                     const uint32_t sbase = ring0 + s * C::STAGE_BYTES;
                     const uint64_t adesc = desc_hi | (uint64_t)(sbase >> 4);
                     const uint64_t bdesc = desc_hi | (uint64_t)((sbase + A_BYTES) >> 4);
@@ -278,9 +266,9 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
                             const int ka = min(2, katoms_total - 2 * kb);
                             const uint64_t sfa_d = sf_hi | (uint64_t)((sbase + A_BYTES + C::B_BYTES) >> 4);
                             const uint64_t sfb_d = sf_hi | (uint64_t)((sbase + A_BYTES + C::B_BYTES + C::SFA_BYTES) >> 4);
-                            // two scale buffers in TMEM: one per issue lane, or alternating by stage with a single
-                            // lane (so a stage's copies never wait for another stage's MMAs still reading theirs)
-                            const uint32_t sfo = (uint32_t)((LANES == 2) ? L : (C::SF_BUFS == 2 ? (kb & 1) : 0)) * C::TM_SF_STRIDE;
+                            // two scale buffers in TMEM where they fit, alternating by stage (so a stage's copies
+                            // never wait for another stage's MMAs still reading theirs)
+                            const uint32_t sfo = (uint32_t)(C::SF_BUFS == 2 ? (kb & 1) : 0) * C::TM_SF_STRIDE;
 #pragma unroll
                             for (int a = 0; a < 2; ++a) {
                                 if (a < ka) {
@@ -344,16 +332,14 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
                             for (int k = 0; k < 4; ++k)
                                 mma_f8_pair(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC_A, (kb | k) ? 1u : 0u);
                         }
-                        tc_commit_pair(&emptyL[s], 3);  // frees the stage in both CTAs
+                        tc_commit_pair(&empty_bar[s], 3);  // frees the stage in both CTAs
                     }
                     __syncwarp();
-                    if (++s == SPL) { s = 0; ph ^= 1u; }
+                    if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
                 if (elect_one()) tc_commit_pair(&tfull_bar[acc], 3);    // accumulator ready in both CTAs
                 __syncwarp();
-                if (LANES == 2) {
-                    acc_ph ^= 1u;                                  // the lane keeps its own accumulator
-                } else if (++acc == ACC) {
+                if (++acc == ACC) {
                     acc = 0;
                     acc_ph ^= 1u;
                 }
