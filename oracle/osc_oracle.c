@@ -722,37 +722,49 @@ uint32_t osc_ref_threshold_bits(double T) {
     return u >> 16;
 }
 
-/* Algorithm 1 for one (position, layer): for every group k and token s take j* = argmax_j |x_{s,kG+j}|
- * (first maximum wins); if |x_{s,kG+j*}| > T_l the token joins S_k with index j*.  L[k] = the most
- * frequent index in S_k (smallest index among equally frequent ones), -1 if S_k is empty.
- * Also returns Eq. 3-4: n_total[k] = |S_k| and n_hit[k] = how many of them carry the dominant index,
- * so that the clustering density is C_k = n_hit[k] / n_total[k]. */
+/* Algorithm 1 for one (position, layer).  Per group the tokens vote: a token's vote is the local index of its
+ * largest magnitude (the first one among equals), and it only counts when that magnitude exceeds the
+ * layer's threshold.  The table entry of the group is the index with the most votes (the smallest such
+ * index; -1 when nobody voted).  The vote counts also give Eq. 3-4: n_total = votes cast in the group,
+ * n_hit = votes for the winning index, clustering density C = n_hit / n_total. */
+static int strongest_channel(const uint16_t* group, double* magnitude) {
+    int arg = 0;
+    double top = fabs(bf16_value(group[0]));
+    for (int j = 1; j < G; ++j) {
+        const double a = fabs(bf16_value(group[j]));
+        if (a > top) { top = a; arg = j; }
+    }
+    *magnitude = top;
+    return arg;
+}
+
 int osc_ref_profile_indexing(const uint16_t* X, int64_t ldx, int S, int H, double T, int8_t* L, int32_t* n_hit,
                              int32_t* n_total) {
     if (H % G) return -3;
-    const int K = H / G;
-    for (int k = 0; k < K; ++k) {
-        int count[G];
-        for (int j = 0; j < G; ++j) count[j] = 0;
-        for (int s = 0; s < S; ++s) {
-            const int offset = k * G;
-            int jstar = 0;
-            double best = -1.0;
-            for (int j = 0; j < G; ++j) {
-                const double a = fabs(bf16_value(X[(int64_t)s * ldx + offset + j]));
-                if (a > best) { best = a; jstar = j; }
-            }
-            if (best > T) count[jstar] += 1;
+    const int groups = H / G;
+    int32_t* votes = (int32_t*)calloc((size_t)groups * G, sizeof(int32_t));   /* votes[group][local index] */
+    if (!votes) return -4;
+    for (int s = 0; s < S; ++s) {
+        const uint16_t* token = X + (int64_t)s * ldx;
+        for (int k = 0; k < groups; ++k) {
+            double magnitude;
+            const int j = strongest_channel(token + k * G, &magnitude);
+            if (magnitude > T) votes[k * G + j] += 1;
         }
-        int total = 0, hit = 0, mode = -1;
-        for (int j = 0; j < G; ++j) {
-            total += count[j];
-            if (count[j] > hit) { hit = count[j]; mode = j; }
-        }
-        L[k] = (int8_t)(total > 0 ? mode : -1);
-        n_hit[k] = hit;
-        n_total[k] = total;
     }
+    for (int k = 0; k < groups; ++k) {
+        const int32_t* v = votes + k * G;
+        int winner = -1;
+        int32_t cast = 0, won = 0;
+        for (int j = 0; j < G; ++j) {
+            cast += v[j];
+            if (v[j] > won) { won = v[j]; winner = j; }
+        }
+        L[k] = (int8_t)winner;
+        n_hit[k] = won;
+        n_total[k] = cast;
+    }
+    free(votes);
     return 0;
 }
 

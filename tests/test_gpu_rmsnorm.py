@@ -11,6 +11,7 @@ from paper_2604_12782_b200 import synth
 pytestmark = pytest.mark.gpu
 
 from gpu_util import assert_within_tolerance, dev_bf16, host_bf16_bits, host_f64, host_u8, poison, valid_sf_bytes  # noqa: E402
+from producer_inputs import RMSNORM_ROW_CASES, gamma_bits, residual_rows  # noqa: E402
 
 
 @pytest.fixture(scope="module")
@@ -19,23 +20,6 @@ def B():
         pytest.skip("no CUDA device")
     from paper_2604_12782_b200 import binding
     return binding
-
-
-def residual_rows(rng, M, K):
-    """Residual-stream-like rows: heavy-tailed values, per-row magnitudes over several orders, a few channels
-    that are large in every row, plus rows of extreme scale."""
-    H = rng.standard_t(4, size=(M, K)) * rng.lognormal(0.0, 1.5, size=(M, 1))
-    hot = rng.choice(K, size=max(1, K // 64), replace=False)
-    H[:, hot] *= 25.0
-    if M > 4:
-        H[1] *= 1e-18
-        H[2] *= 1e15
-        H[3, : K // 2] = 0.0
-    return synth.f32_to_bf16_bits(H.astype(np.float32))
-
-
-def gamma_bits(rng, K):
-    return synth.f32_to_bf16_bits(rng.uniform(0.1, 3.0, K).astype(np.float32) * rng.choice([-1.0, 1.0], K).astype(np.float32))
 
 
 def rand_lut(rng, K, C, p_none=0.2):
@@ -48,8 +32,7 @@ def rand_lut(rng, K, C, p_none=0.2):
     return lut
 
 
-@pytest.mark.parametrize("M,K,eps", [(1, 128, 1e-6), (37, 384, 1e-5), (130, 1024, 1e-6), (64, 4096, 1e-6),
-                                     (9, 8192, 1e-6), (5, 4096 + 128, 0.0), (300, 2048, 1e-6)])
+@pytest.mark.parametrize("M,K,eps", RMSNORM_ROW_CASES)
 def test_rmsnorm_rows_bit_exact(B, oracle, M, K, eps):
     rng = np.random.default_rng(M + K)
     Hb, gb = residual_rows(rng, M, K), gamma_bits(rng, K)
@@ -61,6 +44,9 @@ def test_rmsnorm_rows_bit_exact(B, oracle, M, K, eps):
     got = host_bf16_bits(Xbig[:, :K].contiguous())
     assert np.array_equal(got, want), f"{np.count_nonzero(got != want)} of {got.size} elements differ"
     assert (Xbig[:, K:] == 7.0).all()
+    # and against the plain all-double definition (one rounding): never more than one bf16 unit away
+    from oracle import plain
+    assert plain.bf16_units_apart(got, plain.rmsnorm_plain(Hb, gb, eps)).max() <= 1
 
 
 def test_rmsnorm_special_rows(B, oracle):

@@ -10,6 +10,7 @@ from paper_2604_12782_b200 import synth
 pytestmark = pytest.mark.gpu
 
 from gpu_util import assert_within_tolerance, dev_bf16, host_bf16_bits, host_f64, host_u8, poison  # noqa: E402
+from producer_inputs import SWIGLU_ROW_CASES, gate_up  # noqa: E402
 
 
 @pytest.fixture(scope="module")
@@ -20,20 +21,7 @@ def B():
     return binding
 
 
-def gate_up(rng, M, I, pad=0):
-    """Gate/up projection outputs: gates over the whole range where silu bends, saturates or vanishes, a few extreme
-    rows, zeros; `pad` extra columns behind the up half."""
-    g = rng.standard_normal((M, I)) * rng.choice([0.3, 3.0, 30.0], size=(M, 1))
-    u = rng.standard_t(4, size=(M, I)) * rng.lognormal(0.0, 1.0, size=(M, 1))
-    if M > 4:
-        g[1] = rng.uniform(-120.0, 120.0, I)     # both clamps of exp32
-        g[2, : I // 2] = 0.0
-        u[3] *= 1e-30
-    GU = np.concatenate([g, u, np.full((M, pad), 7.0)], axis=1)
-    return synth.f32_to_bf16_bits(GU.astype(np.float32))
-
-
-@pytest.mark.parametrize("M,I", [(1, 128), (37, 384), (130, 1024), (20, 12288), (5, 16384), (64, 768)])
+@pytest.mark.parametrize("M,I", SWIGLU_ROW_CASES)
 def test_swiglu_rows_bit_exact(B, oracle, M, I):
     rng = np.random.default_rng(M + I)
     GUb = gate_up(rng, M, I, pad=8)
@@ -44,6 +32,13 @@ def test_swiglu_rows_bit_exact(B, oracle, M, I):
     got = host_bf16_bits(H[:, :I].contiguous())
     assert np.array_equal(got, want), f"{np.count_nonzero(got != want)} of {got.size} elements differ"
     assert (H[:, I:] == 7.0).all()
+    # and against the plain all-double definition (one rounding): one bf16 unit at most, except where the clamp of
+    # the exponential shows, which is only in results below 2^-100 in magnitude
+    from oracle import plain
+    ref = plain.swiglu_plain(GUb, I)
+    far = plain.bf16_units_apart(got, ref) > 1
+    tiny = np.abs(synth.bf16_bits_to_f64(got)) + np.abs(synth.bf16_bits_to_f64(ref)) < 2.0 ** -100
+    assert not (far & ~tiny).any()
 
 
 @pytest.mark.parametrize("M,I", [(1, 128), (129, 384), (300, 1024), (33, 12288), (7, 16384)])

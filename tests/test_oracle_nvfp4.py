@@ -49,6 +49,19 @@ def test_worked_blocks_and_scale_index(oracle):
     assert idx == set(range(2 * (K // 64) * 512)) and R <= 256
 
 
+def test_backed_up_channel_in_the_subnormal_range_is_rounded_not_flushed(oracle):
+    """Hand-worked: a flagged channel whose scaled value x * 2^-e falls below the bf16 normal range is stored rounded
+    to nearest-even on the subnormal grid."""
+    for bits, e, want in _gold()["xo_sub"]:
+        X = np.zeros((1, 64), np.uint16)
+        X[0, 5] = int(bits, 16)
+        lut = NOLUT(64).copy()
+        lut[0, 0] = 5
+        q = oracle.nvfp4_quantize_extract(X, lut, int(e))
+        assert q["xo"][0, 0] == int(want, 16), (bits, e, want, hex(int(q["xo"][0, 0])))
+        assert not q["xo"][0, 1:].any() and not q["xq"].any()      # the slot is zeroed, nothing else in the row
+
+
 def _numpy_nvfp4(Xb, lut16, e):
     """Independent restatement: numpy float32 arithmetic + ml_dtypes codecs."""
     x = synth.bf16_bits_to_f64(Xb)
