@@ -13,8 +13,11 @@ timing, as in the paper.
   roofline    the dual-path GEMM kernel against the tensor peak of its own FLOP mix
               (FP4 peak = 4 x, measured BF16 peak from MEASURED_PEAKS.json)
   cpu_baseline the CPU oracle timed on a bounded sample of the same workload (rank 0, N=1 only)
-  extra       the step against the dual-path roofline of the whole linear, the quantizer's
-              HBM fraction, and the same build's FP8 W8A8 linear on the same shape
+  extra       the step against the dual-path roofline of the whole linear (measured-peak and data-sheet
+              basis), the quantizer's HBM fraction, the same build's FP8 W8A8 linear on the same shape, and
+              extra.configs: one row per shape the benchmark configurations name (median and minimum of 30
+              timed iterations, L2 cold and warm, % of the roofline on both bases, speed-up over the own FP8
+              linear on the same shape; shapes of up to 128 rows are replayed from a CUDA graph and say so)
 
 Between timed steps the buffers rotate over 4 independent sets (inputs, workspace,
 outputs and prepared weights: ~0.9 GB, 7x the L2), so no step finds its data in L2.
@@ -27,6 +30,7 @@ from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
 import sys
 import threading
@@ -43,10 +47,19 @@ WORKLOAD = {"name": "qwen3-8b-qkv", "M": 8192, "K": 4096, "N": 6144, "ch_per_gro
 NSETS = 4
 METRIC = "OSC linear TFLOP/s"
 
-# DRAM traffic of one dual-path GEMM launch on the bench workload: dram__bytes_read.sum (38.8 MB) +
-# dram__bytes_write.sum (56.4 MB) from the ncu capture summarised in
-# profiles/gemm_pair_and_quant_extract_qkv_M8192.md (same workload, one launch).
-GEMM_TRAFFIC_BYTES = 95.2e6
+DATASHEET = {"bf16_tflops": 2250.0, "hbm_gbs": 8000.0}   # dense peaks and HBM3e bandwidth of the data sheet
+
+
+def load_traffic():
+    """DRAM bytes (read + written) of one launch of the dominant kernel on the bench workload, from the one ncu
+    capture whose numbers are kept under profiles/ together with the commit and the command they came from."""
+    path = os.path.join(ROOT, "profiles", "dominant_kernel_traffic.json")
+    try:
+        with open(path) as f:
+            t = json.load(f)
+        return float(t["dram_bytes_read"]) + float(t["dram_bytes_write"]), t
+    except (OSError, KeyError, ValueError):
+        return None, None
 
 
 def load_peaks():
@@ -64,7 +77,8 @@ class ClockSampler:
     """Samples SM clock and throttle reasons through NVML while the GPU is busy."""
 
     def __init__(self, index: int):
-        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self.samples, self.stamps, self.reasons, self.max_mhz = [], [], set(), None
+        self.marks = {}
         self._stop = threading.Event()
         self._thread = None
         try:
@@ -84,6 +98,7 @@ class ClockSampler:
         while not self._stop.is_set():
             try:
                 self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                self.stamps.append(time.perf_counter())
                 try:
                     r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
                 except Exception:
@@ -93,7 +108,11 @@ class ClockSampler:
                         self.reasons.add(k)
             except Exception:
                 pass
-            time.sleep(0.002)
+            time.sleep(0.0004)
+
+    def mark(self, name):
+        """Remembers the host time of a boundary of the timed region."""
+        self.marks[name] = time.perf_counter()
 
     def start(self):
         if self.nv:
@@ -105,8 +124,12 @@ class ClockSampler:
         if self._thread:
             self._thread.join()
         med = float(np.median(self.samples)) if self.samples else None
+        t0, t1 = self.marks.get("t0"), self.marks.get("t1")
+        inside = [c for c, t in zip(self.samples, self.stamps) if t0 is not None and t1 is not None and t0 <= t <= t1]
         return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
-                "samples": len(self.samples)}
+                "samples": len(self.samples), "samples_in_timed_region": len(inside),
+                "sm_mhz_in_timed_region": float(np.median(inside)) if inside else None,
+                "span": "sampled from the start of the timed region to the end of all device-timed loops of this run"}
 
 
 # ------------------------------------------------------------------- multi-process glue
@@ -166,6 +189,8 @@ def run_reference(args):
 
 # ------------------------------------------------------------------------------ GPU arm
 def dev_bf16(torch, bits):
+    if isinstance(bits, torch.Tensor):
+        return bits
     return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).view(torch.bfloat16).cuda()
 
 
@@ -311,6 +336,178 @@ def time_split(torch, prob, steps):
     return tq, tg
 
 
+# ------------------------------------------------------------------ rows per benchmark shape
+CALLS_PER_ITERATION = 4   # plain mode: consecutive calls between two events (an event in front of every call would
+                          # add its own gap and cut the programmatic overlap between one call's GEMM and the next
+                          # call's quantizer, which is how the linears of a layer follow each other)
+
+
+def per_call_times(torch, fn, iters, warm, graph_calls=0):
+    """Milliseconds per call of fn(i), one sample per timed iteration.  Plain mode: a timed iteration is
+    CALLS_PER_ITERATION consecutive calls between two events (iters + 1 events on the current stream).  Graph mode
+    (graph_calls > 0): `graph_calls` calls are captured once in a CUDA graph and every timed iteration is one replay,
+    so the host does not pace few-row launches."""
+    if graph_calls:
+        st = torch.cuda.Stream()
+        out = []
+        with torch.cuda.stream(st):
+            for i in range(3):
+                fn(i)
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=st):
+                for i in range(graph_calls):
+                    fn(i)
+            for _ in range(max(1, warm // 2)):
+                g.replay()
+            torch.cuda.synchronize()
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(iters + 1)]
+            ev[0].record(st)
+            for i in range(iters):
+                g.replay()
+                ev[i + 1].record(st)
+            torch.cuda.synchronize()
+            out = [ev[i].elapsed_time(ev[i + 1]) / graph_calls for i in range(iters)]
+        return out
+    for i in range(warm):
+        fn(i)
+    torch.cuda.synchronize()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(iters + 1)]
+    c = CALLS_PER_ITERATION
+    ev[0].record()
+    for i in range(iters):
+        for j in range(c):
+            fn(i * c + j)
+        ev[i + 1].record()
+    torch.cuda.synchronize()
+    return [ev[i].elapsed_time(ev[i + 1]) / c for i in range(iters)]
+
+
+def sets_for_cold_l2(torch, bytes_per_set):
+    """Buffer sets to rotate over so that the data touched between two uses of a set exceeds twice the L2."""
+    l2 = torch.cuda.get_device_properties(torch.cuda.current_device()).L2_cache_size
+    return int(min(24, max(2, math.ceil(2.0 * l2 / max(bytes_per_set, 1)) + 1)))
+
+
+def config_rows(torch, B, pk, iters=30, warm=5):
+    """One row per (M, K, N) the benchmark configurations name: the Qwen3-8B QKV projection at four M, gate_up and
+    the FP8 down projection at three M, the four linears of a decoder layer at M = 4096, the two grouped MoE calls.
+    Every row: median and minimum of `iters` timed iterations with L2 cold (rotating buffer sets) and warm (one
+    set), % of its roofline on the measured-peak and on the data-sheet basis (from the cold median), and the
+    speed-up over this build's FP8 W8A8 linear on the same shape.  Inputs are drawn on the device."""
+    meas = roofline.peaks(pk["bf16_tflops"], pk["hbm_gbs"])
+    sheet = roofline.peaks(DATASHEET["bf16_tflops"], DATASHEET["hbm_gbs"])
+    rows = []
+
+    def stats(ms_list):
+        a = np.asarray(ms_list) * 1e3
+        return float(np.median(a)), float(a.min())
+
+    def measure(prob, few_rows):
+        gc = 2 * prob.n if few_rows else 0
+        cold = stats(per_call_times(torch, prob.step, iters, warm, gc))
+        warm_ = stats(per_call_times(torch, lambda i: prob.step(0), iters, warm, gc))
+        return cold, warm_, ("cuda graph replay of %d calls per timed iteration" % gc) if few_rows else "%d consecutive calls per timed iteration" % CALLS_PER_ITERATION
+
+    def osc_row(name, M, K, N, cpg, seed):
+        case = synth.osc_linear_case_torch(torch, seed, M, K, N, cpg)
+        kop = (K // 32 * cpg + 63) // 64 * 64
+        per_set = N * K / 2 + N * K / 32 + 2.0 * N * kop + 2.0 * M * K + roofline.osc_intermediate_bytes(M, K, kop) + 2.0 * M * N
+        n = sets_for_cold_l2(torch, per_set)
+        p = OscProblem(torch, B, case, n)
+        few = M <= 128
+        cold, warm_, how = measure(p, few)
+        f8 = Fp8Problem(torch, B, case, sets_for_cold_l2(torch, N * K + 3.0 * M * K + 2.0 * M * N))
+        f8cold = stats(per_call_times(torch, f8.step, iters, warm, 2 * f8.n if few else 0))
+        B.osc_sync_check()
+        f4, f16 = roofline.osc_flops(M, N, K, p.K_o)
+        r_m, r_s = (roofline.osc_roofline_seconds(M, N, K, p.K_o, pkx) * 1e6 for pkx in (meas, sheet))
+        rows.append({"name": name, "path": "osc", "M": M, "K": K, "N": N, "K_o": p.K_o, "timing": how, "sets": n,
+                     "cold_us_median": cold[0], "cold_us_min": cold[1], "warm_us_median": warm_[0], "warm_us_min": warm_[1],
+                     "tflops": (f4 + f16) / cold[0] / 1e6, "roof_us": r_m, "roof_us_datasheet": r_s,
+                     "pct_roofline": 100.0 * r_m / cold[0], "pct_roofline_datasheet": 100.0 * r_s / cold[0],
+                     "fp8_cold_us_median": f8cold[0], "speedup_vs_fp8": f8cold[0] / cold[0]})
+        del p, f8, case
+        torch.cuda.empty_cache()
+
+    def fp8_row(name, M, K, N, seed):
+        case = synth.fp8_linear_case_torch(torch, seed, M, K, N)
+        n = sets_for_cold_l2(torch, N * K + 3.0 * M * K + 2.0 * M * N)
+        p = Fp8Problem(torch, B, case, n)
+        few = M <= 128
+        cold, warm_, how = measure(p, few)
+        B.osc_sync_check()
+        r_m, r_s = (roofline.fp8_roofline_seconds(M, N, K, pkx) * 1e6 for pkx in (meas, sheet))
+        rows.append({"name": name, "path": "fp8 fallback (is the own FP8 W8A8 linear)", "M": M, "K": K, "N": N, "timing": how,
+                     "sets": n, "cold_us_median": cold[0], "cold_us_min": cold[1], "warm_us_median": warm_[0],
+                     "warm_us_min": warm_[1], "tflops": roofline.fp8_flops(M, N, K) / cold[0] / 1e6, "roof_us": r_m,
+                     "roof_us_datasheet": r_s, "pct_roofline": 100.0 * r_m / cold[0],
+                     "pct_roofline_datasheet": 100.0 * r_s / cold[0], "fp8_cold_us_median": cold[0], "speedup_vs_fp8": 1.0})
+        del p, case
+        torch.cuda.empty_cache()
+
+    for M in (16, 128, 2048, 8192):
+        osc_row("qkv", M, 4096, 6144, 2, 0)
+    for M in (128, 2048, 8192):
+        osc_row("gate_up", M, 4096, 24576, 1, 0)
+    for M in (128, 2048, 8192):
+        fp8_row("down", M, 12288, 4096, 0)
+    osc_row("layer.qkv", 4096, 4096, 6144, 2, 1)
+    osc_row("layer.o_proj", 4096, 4096, 4096, 1, 2)
+    osc_row("layer.gate_up", 4096, 4096, 24576, 1, 3)
+    fp8_row("layer.down", 4096, 12288, 4096, 4)
+
+    # grouped (MoE): 128 experts, top-8 of 8192 tokens, Zipf(1.1) load; one set of buffers is 0.7 GB, several times
+    # the L2, so the cold and the warm regime coincide and are reported as one
+    counts = synth.zipf_expert_rows()
+    E, Mt = counts.size, int(counts.sum())
+    off = torch.from_numpy(synth.offsets_from_counts(counts)).cuda()
+    K, N = 2048, 1536
+    c = synth.osc_linear_case_torch(torch, 5, Mt, K, N, 1)
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(6)
+    Wg = (0.02 * torch.randn(E, N, K, generator=gen, device="cuda", dtype=torch.float32)).to(torch.bfloat16)
+    w = B.osc_prepare_weights_grouped(Wg, c["lut"])
+    ws = torch.empty(B.osc_act_sizes(w, Mt).workspace_bytes, dtype=torch.uint8, device="cuda")
+    Y = torch.empty(Mt, N, dtype=torch.bfloat16, device="cuda")
+    t = stats(per_call_times(torch, lambda i: B.osc_linear_grouped(w, c["X"], off, Y, ws), iters, warm))
+    w8 = B.osc_fp8_prepare_weights_grouped(Wg)
+    ws8 = torch.empty(B.osc_fp8_act_sizes(w8, Mt).workspace_bytes, dtype=torch.uint8, device="cuda")
+    t8 = stats(per_call_times(torch, lambda i: B.osc_fp8_linear_grouped(w8, c["X"], off, Y, ws8), iters, warm))
+    B.osc_sync_check()
+    f4, f16 = roofline.osc_flops(Mt, N, K, w.K_o)
+    byts = 2.0 * Mt * K + E * (N * K / 2 + N * K / 32 + 2.0 * N * w.K_o) + 2.0 * Mt * N
+    r_m, r_s = (max(f4 / pkx["fp4"] + f16 / pkx["bf16"], byts / pkx["hbm"]) * 1e6 for pkx in (meas, sheet))
+    rows.append({"name": "moe.gate_up(grouped)", "path": "osc", "M": Mt, "K": K, "N": N, "K_o": w.K_o, "E": E,
+                 "timing": "%d consecutive calls per timed iteration; one buffer set larger than the L2 (cold = warm)" % CALLS_PER_ITERATION, "sets": 1,
+                 "cold_us_median": t[0], "cold_us_min": t[1], "warm_us_median": t[0], "warm_us_min": t[1],
+                 "tflops": (f4 + f16) / t[0] / 1e6, "roof_us": r_m, "roof_us_datasheet": r_s,
+                 "pct_roofline": 100.0 * r_m / t[0], "pct_roofline_datasheet": 100.0 * r_s / t[0],
+                 "fp8_cold_us_median": t8[0], "speedup_vs_fp8": t8[0] / t[0]})
+    del w, ws, Y, w8, ws8, Wg, c
+    torch.cuda.empty_cache()
+    K, N = 768, 2048
+    Xd = synth.student_t3_torch(torch, gen, (Mt, K))
+    Wg = (0.02 * torch.randn(E, N, K, generator=gen, device="cuda", dtype=torch.float32)).to(torch.bfloat16)
+    w8 = B.osc_fp8_prepare_weights_grouped(Wg)
+    ws8 = torch.empty(B.osc_fp8_act_sizes(w8, Mt).workspace_bytes, dtype=torch.uint8, device="cuda")
+    Y = torch.empty(Mt, N, dtype=torch.bfloat16, device="cuda")
+    t = stats(per_call_times(torch, lambda i: B.osc_fp8_linear_grouped(w8, Xd, off, Y, ws8), iters, warm))
+    B.osc_sync_check()
+    byts = 2.0 * Mt * K + E * (N * K + 4.0 * N) + 2.0 * Mt * N
+    r_m, r_s = (max(roofline.fp8_flops(Mt, N, K) / pkx["fp8"], byts / pkx["hbm"]) * 1e6 for pkx in (meas, sheet))
+    rows.append({"name": "moe.down(grouped)", "path": "fp8 fallback (is the own FP8 W8A8 linear)", "M": Mt, "K": K, "N": N, "E": E,
+                 "timing": "%d consecutive calls per timed iteration; one buffer set larger than the L2 (cold = warm)" % CALLS_PER_ITERATION, "sets": 1,
+                 "cold_us_median": t[0], "cold_us_min": t[1], "warm_us_median": t[0], "warm_us_min": t[1],
+                 "tflops": roofline.fp8_flops(Mt, N, K) / t[0] / 1e6, "roof_us": r_m, "roof_us_datasheet": r_s,
+                 "pct_roofline": 100.0 * r_m / t[0], "pct_roofline_datasheet": 100.0 * r_s / t[0],
+                 "fp8_cold_us_median": t[0], "speedup_vs_fp8": 1.0})
+    del w8, ws8, Y, Wg, Xd
+    torch.cuda.empty_cache()
+    return rows
+
+
+
 def run_gpu(args):
     import torch
     import torch.distributed as dist
@@ -338,29 +535,34 @@ def run_gpu(args):
         torch.cuda.synchronize()
 
     sampler = ClockSampler(local)
+    sampler.start()      # already sampling when the timed region begins (the first NVML query takes milliseconds)
     # ---- timed region: K steps of osc_linear, inputs resident in HBM
     for i in range(args.warmup):
         prob.step(i)
     barrier()
-    sampler.start()
+    sampler.mark("t0")
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for i in range(args.steps):
         prob.step(i)
     e1.record()
     barrier()
+    sampler.mark("t1")
     ms = e0.elapsed_time(e1) / args.steps
     # ---- same steps again with events between the two kernels (roofline of each kernel)
     tq, tg = time_split(torch, prob, args.steps)
     # ---- and the dominant kernel alone, launched back to back over the rotating buffer sets (operands cold in L2):
     # its average launch duration without the launch gap and the lost overlap that an event in front of it costs
     tg_loop = time_loop(torch, prob.gemm, args.steps, 3)
-    clocks = sampler.stop()
+    # the quantizer the same way (its outputs land in the rotating workspaces; nothing reads them here)
+    tq_loop = time_loop(torch, prob.quant, args.steps, 3)
     B.osc_sync_check()
 
     ms = max_over_ranks(ms, torch.device("cuda", local))
     if args.only_osc:
-        print(f"osc_linear {ms:.4f} ms/step (quantizer {tq:.4f}, gemm {tg:.4f})", file=sys.stderr)
+        sampler.stop()
+        print(f"osc_linear {ms:.4f} ms/step (quantizer {tq:.4f} / {tq_loop:.4f} back to back, gemm {tg:.4f} / {tg_loop:.4f})",
+              file=sys.stderr)
         return
 
     flops4, flops16 = roofline.osc_flops(M, N, K, Ko)
@@ -417,6 +619,14 @@ def run_gpu(args):
     ms_f8 = time_loop(torch, f8.step, args.steps, args.warmup)
     f8q, f8g = time_split(torch, f8, args.steps)
     B.osc_sync_check()
+    del f8
+    torch.cuda.empty_cache()
+    configs = None
+    if world == 1 and not args.no_configs:
+        configs = config_rows(torch, B, pk)
+    clocks = sampler.stop()
+    if clocks.get("sm_mhz_in_timed_region"):
+        clocks["ms_per_step_x_sm_mhz"] = ms * clocks["sm_mhz_in_timed_region"]
 
     if rank != 0:
         if world > 1:
@@ -426,26 +636,41 @@ def run_gpu(args):
     # roofline of the dominant kernel (dual-path GEMM): tensor peak of its own FLOP mix
     p_mix = flops / (flops4 / peaks["fp4"] + flops16 / peaks["bf16"]) / 1e12
     gemm_tflops = flops / (tg_loop * 1e-3) / 1e12
+    sheet = roofline.peaks(DATASHEET["bf16_tflops"], DATASHEET["hbm_gbs"])
+    p_mix_sheet = flops / (flops4 / sheet["fp4"] + flops16 / sheet["bf16"]) / 1e12
+    traffic, traffic_src = load_traffic()
     roof = {"bound": "tensor", "kernel": "gemm_pair_kernel<MODE_OSC> (dual-path GEMM, Eq. 5)", "achieved": gemm_tflops, "peak": p_mix,
-            "unit": "TFLOP/s", "frac": gemm_tflops / p_mix, "traffic": GEMM_TRAFFIC_BYTES,
+            "unit": "TFLOP/s", "frac": gemm_tflops / p_mix, "traffic": traffic,
+            "traffic_source": ({k: traffic_src.get(k) for k in ("commit", "captured", "command")} if traffic_src else None),
             "peak_basis": f"{pk['source']} bf16 {pk['bf16_tflops']} TFLOP/s x4 for FP4 (burst), FLOP-mix weighted",
+            "frac_of_datasheet_peak": gemm_tflops / p_mix_sheet, "datasheet_peak": p_mix_sheet,
             "ms": tg_loop, "timing": "average over back-to-back launches between two events, rotating buffer sets",
             "frac_of_sustained_peak": (gemm_tflops / (p_mix * pk["bf16_tflops_sustained"] / pk["bf16_tflops"])
                                        if pk.get("bf16_tflops_sustained") else None),
             "ms_between_events_inside_the_step": tg}
     qbytes = roofline.quantize_extract_bytes(M, K, Kop)
     t_roof = roofline.osc_roofline_seconds(M, N, K, Ko, peaks)
+    t_roof_sheet = roofline.osc_roofline_seconds(M, N, K, Ko, sheet)
     extra = {
         "pct_dual_path_roofline": 100.0 * t_roof / (ms * 1e-3),
         "roofline_us": t_roof * 1e6,
-        "quant_extract": {"ms": tq, "bytes": qbytes, "gbs": qbytes / (tq * 1e-3) / 1e9,
-                          "frac_hbm": qbytes / (tq * 1e-3) / peaks["hbm"]},
+        "pct_dual_path_roofline_datasheet": 100.0 * t_roof_sheet / (ms * 1e-3),
+        "roofline_us_datasheet": t_roof_sheet * 1e6,
+        "peaks": {"measured": {"bf16_tflops": pk["bf16_tflops"], "fp8_tflops": 2 * pk["bf16_tflops"],
+                               "fp4_tflops": 4 * pk["bf16_tflops"], "hbm_gbs": pk["hbm_gbs"], "source": pk["source"]},
+                  "datasheet": {"bf16_tflops": 2250.0, "fp8_tflops": 4500.0, "fp4_tflops": 9000.0, "hbm_gbs": 8000.0}},
+        "quant_extract": {"ms": tq_loop, "bytes": qbytes, "gbs": qbytes / (tq_loop * 1e-3) / 1e9,
+                          "frac_hbm": qbytes / (tq_loop * 1e-3) / peaks["hbm"],
+                          "frac_hbm_datasheet": qbytes / (tq_loop * 1e-3) / sheet["hbm"],
+                          "timing": "average over back-to-back launches between two events, rotating buffer sets",
+                          "ms_between_events_inside_the_step": tq},
         "fp8_linear": {"ms": ms_f8, "quant_ms": f8q, "gemm_ms": f8g,
                        "tflops": roofline.fp8_flops(M, N, K) / (ms_f8 * 1e-3) / 1e12,
                        "gemm_frac_fp8_peak": roofline.fp8_flops(M, N, K) / (f8g * 1e-3) / peaks["fp8"]},
         "speedup_vs_own_fp8_linear": ms_f8 / ms,
         "speedup_vs_own_fp8_gemm_only": f8g / tg,
         "paper_analytic_speedup_vs_w8a8": roofline.analytic_speedup_vs_w8a8(32, WORKLOAD["ch_per_group"]),
+        "configs": configs,
     }
 
     cpu = None
@@ -964,6 +1189,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="osc", choices=["osc", "reference"])
     ap.add_argument("--no-cpu", action="store_true", help="skip the cpu_baseline leg")
+    ap.add_argument("--no-configs", action="store_true", help="skip extra.configs (the rows per benchmark shape)")
     ap.add_argument("--cpu-rows", type=int, default=8192, help="activation rows of the cpu_baseline sample")
     ap.add_argument("--ref-rows", type=int, default=128, help="activation rows per step of --impl reference")
     ap.add_argument("--sweep", action="store_true")

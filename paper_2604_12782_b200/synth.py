@@ -200,3 +200,50 @@ def osc16_linear_case(seed: int, M: int, K: int, N: int):
     W = (0.02 * rng.standard_normal((N, K))).astype(np.float32)
     return {"X": f32_to_bf16_bits(X), "W": f32_to_bf16_bits(W), "lut16": ch.astype(np.int8).reshape(-1, 1),
             "M": M, "K": K, "N": N}
+
+
+# ----------------------------------------------------------------------------------------------------------------
+# The same recipes drawn on the device (torch generator): for timing-only benchmark rows, where drawing 10^8 values
+# with numpy on the host would take longer than everything that is measured.  Values are not bit-identical to the
+# numpy recipes above (another generator); shapes, distributions and the planted structure are the same.  Parity
+# tests never use these.
+
+def osc_linear_case_torch(torch, seed: int, M: int, K: int, N: int, ch_per_group: int, device="cuda"):
+    """osc_linear_case on the device -> {"X": bf16 [M,K], "W": bf16 [N,K], "lut": int8 [Kg,C] (host)}."""
+    rng = np.random.default_rng(seed)
+    Kg = K // G
+    ch = np.stack([rng.permutation(G)[:ch_per_group] for _ in range(Kg)])
+    cols = (np.arange(Kg)[:, None] * G + ch).reshape(-1)
+    factor = rng.uniform(20.0, 100.0, size=cols.size).astype(np.float32)
+    gen = torch.Generator(device=device)
+    gen.manual_seed(seed)
+    X = torch.randn(M, K, generator=gen, device=device, dtype=torch.float32)
+    cols_d = torch.from_numpy(cols.astype(np.int64)).to(device)
+    hit = torch.rand(M, cols.size, generator=gen, device=device) < 0.9
+    f = torch.where(hit, torch.from_numpy(factor).to(device)[None, :], torch.ones((), device=device))
+    X[:, cols_d] *= f
+    spikes = torch.rand(M, K, generator=gen, device=device) < 0.001
+    X = torch.where(spikes, X * 30.0, X).to(torch.bfloat16)
+    W = (0.02 * torch.randn(N, K, generator=gen, device=device, dtype=torch.float32)).to(torch.bfloat16)
+    return {"X": X, "W": W, "lut": lut_from_channels(ch), "M": M, "K": K, "N": N}
+
+
+def student_t3_torch(torch, gen, shape, device="cuda"):
+    """Student-t with 3 degrees of freedom: z / sqrt(chi2_3 / 3), in chunks of rows to bound the scratch."""
+    out = torch.empty(shape, dtype=torch.bfloat16, device=device)
+    rows = shape[0]
+    step = max(1, (1 << 24) // max(1, shape[1]))
+    for r0 in range(0, rows, step):
+        r1 = min(rows, r0 + step)
+        z = torch.randn(r1 - r0, shape[1], generator=gen, device=device)
+        c = torch.randn(3, r1 - r0, shape[1], generator=gen, device=device).square_().sum(0)
+        out[r0:r1] = (z / torch.sqrt(c / 3.0)).to(torch.bfloat16)
+    return out
+
+
+def fp8_linear_case_torch(torch, seed: int, M: int, K: int, N: int, device="cuda"):
+    gen = torch.Generator(device=device)
+    gen.manual_seed(seed)
+    X = student_t3_torch(torch, gen, (M, K), device)
+    W = (0.02 * torch.randn(N, K, generator=gen, device=device, dtype=torch.float32)).to(torch.bfloat16)
+    return {"X": X, "W": W, "M": M, "K": K, "N": N}
