@@ -64,7 +64,7 @@
  * bit; one kernel is deterministic run to run.
  * Environment variables for experiments (read by the library, not part of the contract): OSC_DECODE (0 = never,
  * 2 = always up to 256 rows), OSC_DECODE_SPLIT, OSC_PAIR (0 = 128-row tiles only, 2 = pair tiles whenever
- * eligible), OSC_PAIR_BLOCK_N, OSC_BLOCK_N, OSC_BAND, OSC_PAIRS, OSC_LOG.
+ * eligible), OSC_PAIR_BLOCK_N, OSC_BLOCK_N, OSC_BAND, OSC_PAIRS, OSC_MAP_CACHE (0 = encode every TMA descriptor anew), OSC_LOG.
  * Sizes: M, N, K and E are ints; every row offset is computed in 64 bits, so M * K (and M * N) may exceed
  * 2^31 elements.
  */

@@ -152,9 +152,18 @@ def _ptr(t):
     return int(t)
 
 
+_raw_stream = getattr(torch._C, "_cuda_getCurrentRawStream", None)
+_raw_device = getattr(torch._C, "_cuda_getDevice", None)
+
+
 def _stream(stream=None):
-    s = torch.cuda.current_stream() if stream is None else stream
-    return s.cuda_stream
+    """cudaStream_t of `stream`, or of torch's current stream.  Building a torch.cuda.Stream object for the current
+    stream costs ~3 us per call, a third of a few-row linear; torch's raw accessor gives the handle directly."""
+    if stream is not None:
+        return stream.cuda_stream
+    if _raw_stream is not None and _raw_device is not None:
+        return _raw_stream(_raw_device())
+    return torch.cuda.current_stream().cuda_stream
 
 
 def _lut(lut):

@@ -64,69 +64,86 @@ static EncodeTiledFn encode_fn() {
     return fn;
 }
 
-// The encoder is a driver call and wants a current context.  A host thread that has made no CUDA call of its own
-// yet has none (runtime calls bind the primary context lazily, a bare driver call does not): on
-// CUDA_ERROR_INVALID_CONTEXT the primary context of the thread's current device is made current and the call is
-// repeated once.
-template <typename... A>
-static CUresult encode_tiled(EncodeTiledFn fn, A... a) {
-    CUresult r = fn(a...);
-    if (r == CUDA_ERROR_INVALID_CONTEXT) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) == cudaSuccess && cudaSetDevice(dev) == cudaSuccess) r = fn(a...);
+// Every 2-D descriptor of the library goes through encode_2d.  The descriptors of a call's activation, scratch and
+// output buffers depend on caller pointers and on M, so they are built per call - and a call needs up to six of
+// them, at one to two microseconds of driver time each, which paces few-row launches from the host.  A descriptor
+// is a pure function of the arguments below (an address and a geometry, no driver object behind it), so each host
+// thread remembers the last ones it built: a serving loop that reuses its buffers encodes them once.  The cache is
+// thread-local (no lock, nothing shared between threads) and replaces its entries round-robin.
+struct MapKey {
+    const void* base;
+    uint64_t dim0, dim1, stride;
+    uint32_t box0, box1;
+    int dtype, swizzle, device;
+    bool operator==(const MapKey& o) const {
+        return base == o.base && dim0 == o.dim0 && dim1 == o.dim1 && stride == o.stride && box0 == o.box0 &&
+               box1 == o.box1 && dtype == o.dtype && swizzle == o.swizzle && device == o.device;
     }
-    return r;
+};
+constexpr int kMapCacheEntries = 64;
+struct MapCache {
+    MapKey key[kMapCacheEntries];
+    CUtensorMap map[kMapCacheEntries];
+    int used = 0, next = 0;
+};
+
+static osc_status encode_2d(CUtensorMap* tm, CUtensorMapDataType dtype, const void* base, uint64_t dim0, uint64_t dim1,
+                            uint64_t stride_bytes, uint32_t box0, uint32_t box1, CUtensorMapSwizzle swizzle,
+                            const char* what) {
+    static thread_local MapCache cache;
+    static const bool use_cache = [] { const char* e = getenv("OSC_MAP_CACHE"); return !e || atoi(e) != 0; }();
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) dev = -1;
+    const MapKey k = {base, dim0, dim1, stride_bytes, box0, box1, (int)dtype, (int)swizzle, dev};
+    if (use_cache) {
+        for (int i = 0; i < cache.used; ++i)
+            if (cache.key[i] == k) { *tm = cache.map[i]; return OSC_OK; }
+    }
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return fail(OSC_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+    cuuint64_t gdim[2] = {dim0, dim1};
+    cuuint64_t gstr[1] = {stride_bytes};
+    cuuint32_t box[2] = {box0, box1};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(tm, dtype, 2, const_cast<void*>(base), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r == CUDA_ERROR_INVALID_CONTEXT && dev >= 0 && cudaSetDevice(dev) == cudaSuccess) {
+        // The encoder is a driver call and wants a current context.  A host thread that has made no CUDA call of its
+        // own yet has none (runtime calls bind the primary context lazily, a bare driver call does not): the primary
+        // context of the thread's current device is made current and the call is repeated once.
+        r = fn(tm, dtype, 2, const_cast<void*>(base), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle,
+               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    }
+    if (r != CUDA_SUCCESS) return fail(OSC_ERR_CUDA, "cuTensorMapEncodeTiled(%s) failed with code %d", what, (int)r);
+    if (use_cache) {
+        const int slot = cache.used < kMapCacheEntries ? cache.used++ : (cache.next = (cache.next + 1) % kMapCacheEntries);
+        cache.key[slot] = k;
+        cache.map[slot] = *tm;
+    }
+    return OSC_OK;
 }
 
 // Row-major [rows, row_bytes] operand, tiles of box_rows x 128 bytes, 128-byte swizzle, zero fill.
 static osc_status make_tmap(CUtensorMap* tm, const void* base, bool bf16, uint64_t rows, uint64_t row_bytes,
                             uint64_t pitch_bytes, uint32_t box_rows) {
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return fail(OSC_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
     if (rows == 0) rows = 1;  // never dereferenced: no tile is scheduled for an empty operand
     const uint64_t esz = bf16 ? 2 : 1;
-    cuuint64_t gdim[2] = {row_bytes / esz, rows};
-    cuuint64_t gstr[1] = {pitch_bytes};
-    cuuint32_t box[2] = {static_cast<cuuint32_t>(128 / esz), box_rows};
-    cuuint32_t estr[2] = {1, 1};
-    CUresult r = encode_tiled(fn, tm, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 2u,
-                              const_cast<void*>(base), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) return fail(OSC_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
-    return OSC_OK;
+    return encode_2d(tm, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, base, row_bytes / esz, rows,
+                     pitch_bytes, static_cast<uint32_t>(128 / esz), box_rows, CU_TENSOR_MAP_SWIZZLE_128B, "operand");
 }
 
 // bf16 [rows, cols] input of the quantizer: tiles of 128 rows x 64 channels (128 bytes), 128-byte swizzle, zero fill.
 static osc_status make_tmap_x(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint64_t ld) {
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return fail(OSC_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
     if (rows == 0) rows = 1;
-    cuuint64_t gdim[2] = {cols, rows};
-    cuuint64_t gstr[1] = {ld * 2};
-    cuuint32_t box[2] = {64, 128};
-    cuuint32_t estr[2] = {1, 1};
-    CUresult r = encode_tiled(fn, tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2u, const_cast<void*>(base), gdim, gstr, box, estr,
-                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) return fail(OSC_ERR_CUDA, "cuTensorMapEncodeTiled(X) failed with code %d", (int)r);
-    return OSC_OK;
+    return encode_2d(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, base, cols, rows, ld * 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B, "X");
 }
 
 // Scale-factor buffer as [blocks, 128] uint32 (512-byte blocks), tiles of `box_blocks` consecutive blocks
 // (2 = the 256 FP4 channels of a GEMM stage, 1 = the 128 FP8 channels).
 static osc_status make_tmap_sf(CUtensorMap* tm, const void* base, uint64_t blocks, uint32_t box_blocks = 2) {
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return fail(OSC_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
     if (blocks == 0) blocks = 1;
-    cuuint64_t gdim[2] = {128, blocks};
-    cuuint64_t gstr[1] = {512};
-    cuuint32_t box[2] = {128, box_blocks};
-    cuuint32_t estr[2] = {1, 1};
-    CUresult r = encode_tiled(fn, tm, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2u, const_cast<void*>(base), gdim, gstr, box, estr,
-                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) return fail(OSC_ERR_CUDA, "cuTensorMapEncodeTiled(scales) failed with code %d", (int)r);
-    return OSC_OK;
+    return encode_2d(tm, CU_TENSOR_MAP_DATA_TYPE_UINT32, base, 128, blocks, 512, 128, box_blocks, CU_TENSOR_MAP_SWIZZLE_NONE,
+                     "scales");
 }
 
 // Grouped problems whose experts average at least 96 rows run on the CTA-pair kernel (256-row tiles), the rest on
