@@ -153,19 +153,79 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
     tc_fence_after();
     const uint32_t tmem_base = __shfl_sync(0xFFFFFFFFu, *tmem_slot, 0);
     grid_launch_dependents();
-    grid_dependency_wait();   // operands come from the kernel before this one
 
     const int N = args.N, K = args.K;
     const int32_t* __restrict__ sched = args.sched2;
-    const int num_m = sched ? sched[0] : (args.M + 2 * BM - 1) / (2 * BM);
-    const int num_n = (N + BN - 1) / BN;
-    const int total = num_m * num_n;
     const int elems_per_kb = C::DUAL ? 256 : 128;  // channels in 128 bytes of an operand row
     const int nkb_a = (K + elems_per_kb - 1) / elems_per_kb;
     const int nkb_b = C::DUAL ? args.Kop / 64 : 0;
     const int nkb = nkb_a + nkb_b;
     const int katoms_total = K / C::SF_K;   // scale blocks along K
     const int natoms = (N + 127) / 128;
+    const int num_n = (N + BN - 1) / BN;
+
+    // One stage of the operand ring, in two parts: the weight side (weight tile and weight scales: prepared
+    // once, never written by a kernel of the calling sequence) and the activation side (this call's quantizer
+    // output).  `expect` arms the leader's full barrier with the bytes of both parts and both CTAs.
+    auto load_weights = [&](int s, int kb, int n0, int expert, bool expect) {
+        const uint32_t st = smem_u32(smem + s * C::STAGE_BYTES);
+        const uint32_t fb = map_to_cta(smem_u32(full_bar), 0) + (uint32_t)s * 8u;
+        const int brow = expert * N + n0 + (int)rank * (BN / 2);       // my half of the weight rows
+        if (kb < nkb_a) {
+            if (expect && rank == 0) mbar_arrive_expect_tx(&full_bar[s], C::SCALED ? C::TX_A : C::TX_B);
+            tma_load_2d_pair(st + A_BYTES, &args.tm_b, fb, kb * ROW_BYTES, brow);
+            if (C::SCALED) {
+#pragma unroll
+                for (int j = 0; j < C::SFB_ATOMS; ++j) {
+                    const int atom = C::TILED_SF ? (expert * num_n + n0 / BN) * C::SFB_ATOMS + j
+                                                 : expert * natoms + min(n0 / 128 + j, natoms - 1);
+                    tma_load_2d_pair(st + A_BYTES + C::B_BYTES + C::SFA_BYTES + j * (C::KA * 512), &args.tm_sfw,
+                                     fb, 0, atom * katoms_total + C::KA * kb);
+                }
+            }
+        } else {
+            if (expect && rank == 0) mbar_arrive_expect_tx(&full_bar[s], C::TX_B);
+            tma_load_2d_pair(st + A_BYTES, &args.tm_bo, fb, (kb - nkb_a) * 64, brow);
+        }
+    };
+    auto load_activations = [&](int s, int kb, int row0, int sf_row0) {
+        const uint32_t st = smem_u32(smem + s * C::STAGE_BYTES);
+        const uint32_t fb = map_to_cta(smem_u32(full_bar), 0) + (uint32_t)s * 8u;
+        const int arow = row0 + (int)rank * BM;                              // my 128 activation rows
+        if (kb < nkb_a) {
+            tma_load_2d_pair(st, &args.tm_a, fb, kb * ROW_BYTES, arow);
+            if (C::SCALED)   // scale blocks: KA consecutive 512-byte blocks (128 channels each) per 128 rows
+                tma_load_2d_pair(st + A_BYTES + C::B_BYTES, &args.tm_sfa, fb, 0,
+                                 (sf_row0 / 128 + (int)rank) * katoms_total + C::KA * kb);
+        } else {
+            tma_load_2d_pair(st, &args.tm_ao, fb, (kb - nkb_a) * 64, arow);
+        }
+    };
+
+    // Dense problems: the producer fills the ring with the weight side of its first tile BEFORE the dependency
+    // wait - the CTAs of this kernel become resident while the last CTAs of the quantizer in front of it are
+    // still running, and the weights do not depend on it - and adds the activation side behind the wait.
+    // (Grouped problems read their tile list from a schedule that the kernel in front builds: nothing is
+    // known before the wait.)
+    const int num_m_dense = (args.M + 2 * BM - 1) / (2 * BM);
+    const int pre = (sched == nullptr && warp == 0 && (int)blockIdx.x / 2 < num_m_dense * num_n) ? min(STAGES, nkb) : 0;
+    int pre_n0 = 0, pre_row0 = 0;
+    if (pre > 0) {
+        const int t = blockIdx.x >> 1;
+        const int per_band = args.band * num_n;
+        const int band = t / per_band, rem = t - band * per_band;
+        const int m0 = band * args.band, h = min(args.band, num_m_dense - m0);
+        pre_n0 = (rem / h) * BN;
+        pre_row0 = (m0 + rem % h) * (2 * BM);
+        if (elect_one()) {
+            for (int kb = 0; kb < pre; ++kb) load_weights(kb, kb, pre_n0, 0, true);
+        }
+        __syncwarp();
+    }
+    grid_dependency_wait();   // activations (and a grouped schedule) come from the kernel before this one
+
+    const int num_m = sched ? sched[0] : num_m_dense;
+    const int total = num_m * num_n;
 
     // tile t -> first row, column, and (grouped) last valid row, first scale row, expert
     struct Tile { int row0, n0, row_end, sf_row0, expert; };
@@ -196,40 +256,20 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
         // ------------------------------------------------------- TMA producer (both CTAs)
         int s = 0;
         uint32_t ph = 0;
-        uint8_t* ring = smem;
-        const uint32_t full0 = map_to_cta(smem_u32(full_bar), 0);  // the leader's full barriers
+        if (pre > 0) {   // the activation side of the stages whose weight side is already under way
+            if (elect_one()) {
+                for (int kb = 0; kb < pre; ++kb) load_activations(kb, kb, pre_row0, pre_row0);
+            }
+            __syncwarp();
+            if (pre == STAGES) ph = 1u; else s = pre;
+        }
         for (int t = pair_id; t < total; t += num_pairs) {
             const Tile ti = tile_of(t);
-            const int n0 = ti.n0;
-            const int arow = ti.row0 + (int)rank * BM;                        // my 128 activation rows
-            const int brow = ti.expert * N + n0 + (int)rank * (BN / 2);       // my half of the weight rows
-            const int sfa_blk = (ti.sf_row0 / 128 + (int)rank) * katoms_total;  // my 128-row scale blocks
-            for (int kb = 0; kb < nkb; ++kb) {
+            for (int kb = (t == pair_id ? pre : 0); kb < nkb; ++kb) {
                 if (!wait_bounded(&empty_bar[s], ph ^ 1u, abort_flag, 11)) goto done;
-                const uint32_t st = smem_u32(ring + s * C::STAGE_BYTES);
-                const uint32_t fb = full0 + (uint32_t)s * 8u;
                 if (elect_one()) {
-                    if (kb < nkb_a) {
-                        if (rank == 0) mbar_arrive_expect_tx(&full_bar[s], C::SCALED ? C::TX_A : C::TX_B);
-                        tma_load_2d_pair(st, &args.tm_a, fb, kb * ROW_BYTES, arow);
-                        tma_load_2d_pair(st + A_BYTES, &args.tm_b, fb, kb * ROW_BYTES, brow);
-                        if (C::SCALED) {
-                            // scale blocks: KA consecutive 512-byte blocks (128 channels each) per 128 rows
-                            tma_load_2d_pair(st + A_BYTES + C::B_BYTES, &args.tm_sfa, fb, 0, sfa_blk + C::KA * kb);
-#pragma unroll
-                            for (int j = 0; j < C::SFB_ATOMS; ++j) {
-                                const int atom = C::TILED_SF ? (ti.expert * num_n + n0 / BN) * C::SFB_ATOMS + j
-                                                             : ti.expert * natoms + min(n0 / 128 + j, natoms - 1);
-                                tma_load_2d_pair(st + A_BYTES + C::B_BYTES + C::SFA_BYTES + j * (C::KA * 512), &args.tm_sfw,
-                                                 fb, 0, atom * katoms_total + C::KA * kb);
-                            }
-                        }
-                    } else {
-                        const int kk = kb - nkb_a;
-                        if (rank == 0) mbar_arrive_expect_tx(&full_bar[s], C::TX_B);
-                        tma_load_2d_pair(st, &args.tm_ao, fb, kk * 64, arow);
-                        tma_load_2d_pair(st + A_BYTES, &args.tm_bo, fb, kk * 64, brow);
-                    }
+                    load_weights(s, kb, ti.n0, ti.expert, true);
+                    load_activations(s, kb, ti.row0, ti.sf_row0);
                 }
                 __syncwarp();
                 if (++s == STAGES) { s = 0; ph ^= 1u; }
