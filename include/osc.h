@@ -454,12 +454,35 @@ osc_status osc_nvfp4_linear(const osc_weights* w, const void* X, int M, int64_t 
  * block); buffers are E times the dense sizes (osc_nvfp4_weight_sizes_grouped).  Rows of X_perm sorted by
  * expert and off as in osc_linear_grouped; expert e's activation scale rows start at scale row
  * sum_{e'<e} roundup(m_e', 128); workspace from osc_nvfp4_act_sizes(w, M_total).  A grouped handle is accepted
- * by osc_nvfp4_act_sizes, osc_nvfp4_linear_grouped and osc_weights_destroy only. */
+ * by osc_nvfp4_act_sizes, osc_nvfp4_linear_grouped, the two gathered forms below and osc_weights_destroy only. */
 osc_status osc_nvfp4_weight_sizes_grouped(int E, int N, int K, const int8_t* lut16, int lut_c, osc_weight_sizes_t* out);
 osc_status osc_nvfp4_prepare_weights_grouped(const void* W, int E, int N, int K, const int8_t* lut16, int lut_c, int ew,
                                              void* wq, void* sfw, void* wo, void* meta, void* stream, osc_weights** out);
 osc_status osc_nvfp4_linear_grouped(const osc_weights* w, const void* X_perm, const int32_t* off, int M_total, int64_t ldx,
                                     int ex, void* Y, int64_t ldy, void* workspace, size_t workspace_bytes, void* stream);
+
+/* The producer fusion and the dispatch gather in the NVFP4 / G = 16 form (Section 3.3 places the quantizer behind
+ * the operator that produces the activations; the efficiency table's G = 16 row is this format).
+ * osc_nvfp4_rmsnorm_quantize_extract: RMSNorm (arithmetic as osc_rmsnorm) and the NVFP4 form of Algorithm 2 in one
+ *   pass over H (dev bf16 [M, ldh], K <= 8192); ex is the tensor exponent of the NORMALIZED activations; outputs as
+ *   osc_nvfp4_quantize_extract writes them, bit for bit what that call gives on osc_rmsnorm's output.
+ * osc_nvfp4_rmsnorm_linear = that + osc_nvfp4_gemm, workspace from osc_nvfp4_act_sizes.
+ * osc_nvfp4_linear_grouped_gather / osc_nvfp4_rmsnorm_linear_grouped_gather: as osc_linear_grouped_gather /
+ *   osc_rmsnorm_linear_grouped_gather with a grouped NVFP4 handle: the T tokens are quantized once (scale blocks of
+ *   64 channels) and their quantized rows copied to the rows their experts own; equals osc_nvfp4_linear_grouped on
+ *   X_perm[r] = X[row_token[r]] bit for bit.  Workspace: osc_nvfp4_gather_workspace_bytes.
+ * Errors as for their MXFP4 counterparts. */
+osc_status osc_nvfp4_rmsnorm_quantize_extract(const osc_weights* w, const void* H, int M, int64_t ldh, const void* gamma,
+                                              float eps, int ex, void* xq, void* sfa, void* xo, void* stream);
+osc_status osc_nvfp4_rmsnorm_linear(const osc_weights* w, const void* H, int M, int64_t ldh, const void* gamma, float eps,
+                                    int ex, void* Y, int64_t ldy, void* workspace, size_t workspace_bytes, void* stream);
+osc_status osc_nvfp4_gather_workspace_bytes(const osc_weights* w, int T, int M_total, size_t* bytes);
+osc_status osc_nvfp4_linear_grouped_gather(const osc_weights* w, const void* X, int T, int64_t ldx, const int32_t* row_token,
+                                           const int32_t* off, int M_total, int ex, void* Y, int64_t ldy, void* workspace,
+                                           size_t workspace_bytes, void* stream);
+osc_status osc_nvfp4_rmsnorm_linear_grouped_gather(const osc_weights* w, const void* H, int T, int64_t ldh, const void* gamma,
+                                                   float eps, const int32_t* row_token, const int32_t* off, int M_total, int ex,
+                                                   void* Y, int64_t ldy, void* workspace, size_t workspace_bytes, void* stream);
 
 #ifdef __cplusplus
 }

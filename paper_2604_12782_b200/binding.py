@@ -113,6 +113,12 @@ _SIGS = {
     "osc_nvfp4_quantize_extract": (_i, [_vp, _vp, _i, _i64, _i, _vp, _vp, _vp, _vp]),
     "osc_nvfp4_gemm": (_i, [_vp, _vp, _vp, _vp, _i, _i, _vp, _i64, _vp]),
     "osc_nvfp4_linear": (_i, [_vp, _vp, _i, _i64, _i, _vp, _i64, _vp, _sz, _vp]),
+    "osc_nvfp4_rmsnorm_quantize_extract": (_i, [_vp, _vp, _i, _i64, _vp, C.c_float, _i, _vp, _vp, _vp, _vp]),
+    "osc_nvfp4_rmsnorm_linear": (_i, [_vp, _vp, _i, _i64, _vp, C.c_float, _i, _vp, _i64, _vp, _sz, _vp]),
+    "osc_nvfp4_gather_workspace_bytes": (_i, [_vp, _i, _i, C.POINTER(_sz)]),
+    "osc_nvfp4_linear_grouped_gather": (_i, [_vp, _vp, _i, _i64, _vp, _vp, _i, _i, _vp, _i64, _vp, _sz, _vp]),
+    "osc_nvfp4_rmsnorm_linear_grouped_gather": (_i, [_vp, _vp, _i, _i64, _vp, C.c_float, _vp, _vp, _i, _i, _vp, _i64, _vp, _sz,
+                                                     _vp]),
     "osc_mxfp8_weight_sizes": (_i, [_i, _i, _i, C.POINTER(Mxfp8WeightSizes)]),
     "osc_mxfp8_prepare_weights_grouped": (_i, [_vp, _i, _i, _i, _vp, _vp, _vp, C.POINTER(_vp)]),
     "osc_mxfp8_linear_grouped": (_i, [_vp, _vp, _vp, _i, _i64, _vp, _i64, _vp, _sz, _vp]),
@@ -651,3 +657,43 @@ def osc_nvfp4_linear(w: OscWeights, X: torch.Tensor, ex: int, Y: torch.Tensor, w
     _check(_lib.osc_nvfp4_linear(w.ptr, _ptr(X), M, X.stride(0) if M else w.K, int(ex), _ptr(Y),
                                  Y.stride(0) if M else w.N, _ptr(workspace),
                                  workspace.numel() * workspace.element_size(), _stream(stream)))
+
+
+def osc_nvfp4_rmsnorm_quantize_extract(w: OscWeights, H: torch.Tensor, gamma: torch.Tensor, eps: float, ex: int, xq, sfa, xo,
+                                       stream=None):
+    M = H.shape[0]
+    _check(_lib.osc_nvfp4_rmsnorm_quantize_extract(w.ptr, _ptr(H), M, H.stride(0) if M else w.K, _ptr(gamma), float(eps),
+                                                   int(ex), _ptr(xq), _ptr(sfa), _ptr(xo) if w.K_o_pad else None,
+                                                   _stream(stream)))
+
+
+def osc_nvfp4_rmsnorm_linear(w: OscWeights, H: torch.Tensor, gamma: torch.Tensor, eps: float, ex: int, Y: torch.Tensor,
+                             workspace: torch.Tensor, stream=None):
+    M = H.shape[0]
+    _check(_lib.osc_nvfp4_rmsnorm_linear(w.ptr, _ptr(H), M, H.stride(0) if M else w.K, _ptr(gamma), float(eps), int(ex),
+                                         _ptr(Y), Y.stride(0) if M else w.N, _ptr(workspace),
+                                         workspace.numel() * workspace.element_size(), _stream(stream)))
+
+
+def osc_nvfp4_gather_workspace_bytes(w: OscWeights, T: int, M_total: int) -> int:
+    out = _sz()
+    _check(_lib.osc_nvfp4_gather_workspace_bytes(w.ptr, T, M_total, C.byref(out)))
+    return int(out.value)
+
+
+def osc_nvfp4_linear_grouped_gather(w: OscWeights, X: torch.Tensor, row_token: torch.Tensor, off: torch.Tensor, ex: int,
+                                    Y: torch.Tensor, workspace: torch.Tensor, stream=None):
+    T, M = X.shape[0], row_token.shape[0]
+    _check(_lib.osc_nvfp4_linear_grouped_gather(w.ptr, _ptr(X), T, X.stride(0) if T else w.K, _ptr(row_token), _ptr(off), M,
+                                                int(ex), _ptr(Y), Y.stride(0) if M else w.N, _ptr(workspace),
+                                                workspace.numel() * workspace.element_size(), _stream(stream)))
+
+
+def osc_nvfp4_rmsnorm_linear_grouped_gather(w: OscWeights, H: torch.Tensor, gamma: torch.Tensor, eps: float,
+                                            row_token: torch.Tensor, off: torch.Tensor, ex: int, Y: torch.Tensor,
+                                            workspace: torch.Tensor, stream=None):
+    T, M = H.shape[0], row_token.shape[0]
+    _check(_lib.osc_nvfp4_rmsnorm_linear_grouped_gather(w.ptr, _ptr(H), T, H.stride(0) if T else w.K, _ptr(gamma), float(eps),
+                                                        _ptr(row_token), _ptr(off), M, int(ex), _ptr(Y),
+                                                        Y.stride(0) if M else w.N, _ptr(workspace),
+                                                        workspace.numel() * workspace.element_size(), _stream(stream)))

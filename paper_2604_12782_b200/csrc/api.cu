@@ -1586,6 +1586,123 @@ osc_status osc_nvfp4_linear_grouped(const osc_weights* w, const void* X_perm, co
                            max_tiles, sched2, max_tiles2);
 }
 
+// ---- NVFP4 forms of the producer fusion and of the dispatch gather
+static osc_status nvfp4_rmsnorm_quantize_impl(const osc_weights* w, const void* H, int M, int64_t ldh, const void* gamma,
+                                              float eps, int ex, void* xq, void* sfa, void* xo, void* stream) {
+    if (osc_status s = check_act(w, H, M, ldh, false, true)) return s;
+    if (ex < -100 || ex > 100) return fail(OSC_ERR_INVALID_ARG, "tensor exponent %d outside -100..100", ex);
+    if (w->K > 8192) return fail(OSC_ERR_SHAPE, "K = %d: the fused RMSNorm stages a row in shared memory, K <= 8192", w->K);
+    if (M == 0) return OSC_OK;
+    if (!gamma || !aligned16(gamma)) return fail(OSC_ERR_ALIGN, "gamma must be non-null and 16-byte aligned");
+    if (!xq || !sfa || (w->Kop > 0 && !xo)) return fail(OSC_ERR_INVALID_ARG, "null output pointer");
+    if (!aligned16(xq) || !aligned16(sfa) || !aligned16(xo)) return fail(OSC_ERR_ALIGN, "outputs must be 16-byte aligned");
+    cudaError_t e = launch_rmsnorm_quant_nvfp4(H, ldh, M, w->K, gamma, eps, w->idx_o, xq, sfa, w->Kop ? xo : nullptr, w->Ko,
+                                               w->Kop, ex, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(e, "rmsnorm_quant_kernel(nvfp4)");
+    return OSC_OK;
+}
+
+osc_status osc_nvfp4_rmsnorm_quantize_extract(const osc_weights* w, const void* H, int M, int64_t ldh, const void* gamma,
+                                              float eps, int ex, void* xq, void* sfa, void* xo, void* stream) {
+    if (w && w->grouped) return fail(OSC_ERR_INVALID_ARG, "grouped weights: use osc_nvfp4_rmsnorm_linear_grouped_gather");
+    return nvfp4_rmsnorm_quantize_impl(w, H, M, ldh, gamma, eps, ex, xq, sfa, xo, stream);
+}
+
+osc_status osc_nvfp4_rmsnorm_linear(const osc_weights* w, const void* H, int M, int64_t ldh, const void* gamma, float eps,
+                                    int ex, void* Y, int64_t ldy, void* workspace, size_t workspace_bytes, void* stream) {
+    if (osc_status s = check_act(w, H, M, ldh, false, true)) return s;
+    if (w->grouped) return fail(OSC_ERR_INVALID_ARG, "grouped weights: use osc_nvfp4_rmsnorm_linear_grouped_gather");
+    if (M == 0) return OSC_OK;
+    osc_act_sizes_t sz;
+    osc_nvfp4_act_sizes(w, M, &sz);
+    if (!workspace || !aligned16(workspace)) return fail(OSC_ERR_ALIGN, "workspace must be non-null and 16-byte aligned");
+    if (workspace_bytes < sz.workspace_bytes)
+        return fail(OSC_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", workspace_bytes, sz.workspace_bytes);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    if (osc_status s = nvfp4_rmsnorm_quantize_impl(w, H, M, ldh, gamma, eps, ex, ws + sz.xq_offset, ws + sz.sfa_offset,
+                                                   ws + sz.xo_offset, stream)) return s;
+    return osc_nvfp4_gemm(w, ws + sz.xq_offset, ws + sz.sfa_offset, ws + sz.xo_offset, M, ex, Y, ldy, stream);
+}
+
+// buffers of the T unique tokens behind the grouped workspace (NVFP4: scale blocks of 64 channels)
+static GatherLayout nvfp4_gather_layout(const osc_weights* w, int T, const osc_act_sizes_t& sz) {
+    GatherLayout g;
+    g.xq_u = sz.workspace_bytes;
+    g.sf_u = g.xq_u + align256((size_t)T * (w->K / 2));
+    g.xo_u = g.sf_u + align256((size_t)((T + 127) / 128) * (w->K / 64) * 512);
+    g.total = g.xo_u + align256((size_t)T * w->Kop * 2);
+    return g;
+}
+
+osc_status osc_nvfp4_gather_workspace_bytes(const osc_weights* w, int T, int M_total, size_t* bytes) {
+    if (!w || !bytes) return fail(OSC_ERR_INVALID_ARG, "null argument");
+    if (!w->nvfp4) return fail(OSC_ERR_INVALID_ARG, "MXFP4 weights: use osc_gather_workspace_bytes");
+    if (!w->grouped) return fail(OSC_ERR_INVALID_ARG, "dense weights have no dispatch");
+    if (T < 0 || M_total < 0) return fail(OSC_ERR_INVALID_ARG, "negative size");
+    osc_act_sizes_t sz;
+    if (osc_status s = osc_nvfp4_act_sizes(w, M_total, &sz)) return s;
+    *bytes = nvfp4_gather_layout(w, T, sz).total;
+    return OSC_OK;
+}
+
+static osc_status nvfp4_grouped_gather_impl(const osc_weights* w, const void* X, int T, int64_t ldx, const void* gamma, float eps,
+                                            const int32_t* row_token, const int32_t* off, int M_total, int ex, void* Y,
+                                            int64_t ldy, void* workspace, size_t workspace_bytes, void* stream) {
+    if (osc_status s = check_act(w, X, T, ldx, false, true)) return s;
+    if (!w->grouped) return fail(OSC_ERR_INVALID_ARG, "dense weights have no dispatch");
+    if (M_total < 0) return fail(OSC_ERR_INVALID_ARG, "M_total = %d is negative", M_total);
+    if (ex < -100 || ex > 100) return fail(OSC_ERR_INVALID_ARG, "tensor exponent %d outside -100..100", ex);
+    if (M_total == 0) return OSC_OK;
+    if (T == 0) return fail(OSC_ERR_INVALID_ARG, "rows to dispatch but no tokens");
+    if (!off || !row_token) return fail(OSC_ERR_INVALID_ARG, "off / row_token is null");
+    osc_act_sizes_t sz;
+    osc_nvfp4_act_sizes(w, M_total, &sz);
+    const GatherLayout g = nvfp4_gather_layout(w, T, sz);
+    if (!workspace || !aligned16(workspace)) return fail(OSC_ERR_ALIGN, "workspace must be non-null and 16-byte aligned");
+    if (workspace_bytes < g.total)
+        return fail(OSC_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", workspace_bytes, g.total);
+    if (!Y) return fail(OSC_ERR_INVALID_ARG, "Y is null");
+    if (ldy < w->N) return fail(OSC_ERR_SHAPE, "ldy = %lld < N = %d", (long long)ldy, w->N);
+    if (ldy % 8 || !aligned16(Y)) return fail(OSC_ERR_ALIGN, "Y must be 16-byte aligned and ldy a multiple of 8");
+    const int es = ex + w->ew;
+    if (es < -120 || es > 120) return fail(OSC_ERR_INVALID_ARG, "sum of the tensor exponents %d outside -120..120", es);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int max_tiles = M_total / 128 + w->E;
+    const int max_tiles2 = max_tiles256(M_total, w->E);
+    int32_t* sched = reinterpret_cast<int32_t*>(ws + sz.sched_offset);
+    int32_t* sched2 = use_pair_kernel(true, M_total, w->E) ? sched + sched_ints(max_tiles) : nullptr;
+    cudaError_t e = launch_build_sched(off, w->E, sched, max_tiles, sched2, max_tiles2, st);
+    if (e != cudaSuccess) return cuda_fail(e, "build_sched_kernel");
+    // the NVFP4 form of Algorithm 2 once per token, as a dense problem of T rows
+    if (gamma) {
+        if (osc_status s = nvfp4_rmsnorm_quantize_impl(w, X, T, ldx, gamma, eps, ex, ws + g.xq_u, ws + g.sf_u, ws + g.xo_u, stream))
+            return s;
+    } else {
+        if (osc_status s = nvfp4_quantize_impl(w, X, T, ldx, ex, ws + g.xq_u, ws + g.sf_u, ws + g.xo_u, stream, nullptr, 0)) return s;
+    }
+    e = launch_gather_quantized(row_token, T, w->K, w->Kop, ws + g.xq_u, ws + g.sf_u, ws + g.xo_u, ws + sz.xq_offset,
+                                ws + sz.sfa_offset, ws + sz.xo_offset, sched, max_tiles, st, 64);
+    if (e != cudaSuccess) return cuda_fail(e, "gather_quantized_kernel(nvfp4)");
+    return nvfp4_gemm_impl(w, ws + sz.xq_offset, ws + sz.sfa_offset, ws + sz.xo_offset, M_total, ex, Y, ldy, stream, sched,
+                           max_tiles, sched2, max_tiles2);
+}
+
+osc_status osc_nvfp4_linear_grouped_gather(const osc_weights* w, const void* X, int T, int64_t ldx, const int32_t* row_token,
+                                           const int32_t* off, int M_total, int ex, void* Y, int64_t ldy, void* workspace,
+                                           size_t workspace_bytes, void* stream) {
+    return nvfp4_grouped_gather_impl(w, X, T, ldx, nullptr, 0.0f, row_token, off, M_total, ex, Y, ldy, workspace, workspace_bytes,
+                                     stream);
+}
+
+osc_status osc_nvfp4_rmsnorm_linear_grouped_gather(const osc_weights* w, const void* H, int T, int64_t ldh, const void* gamma,
+                                                   float eps, const int32_t* row_token, const int32_t* off, int M_total, int ex,
+                                                   void* Y, int64_t ldy, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!gamma) return fail(OSC_ERR_INVALID_ARG, "gamma is null");
+    return nvfp4_grouped_gather_impl(w, H, T, ldh, gamma, eps, row_token, off, M_total, ex, Y, ldy, workspace, workspace_bytes,
+                                     stream);
+}
+
 osc_status osc_nvfp4_linear(const osc_weights* w, const void* X, int M, int64_t ldx, int ex, void* Y, int64_t ldy,
                             void* workspace, size_t workspace_bytes, void* stream) {
     if (osc_status s = check_act(w, X, M, ldx, false, true)) return s;

@@ -69,15 +69,20 @@ cudaError_t launch_build_sched(const int32_t* off, int E, int32_t* sched128, int
 
 cudaError_t launch_prepare_fence(cudaStream_t st);   // last launch of every weight preparation
 
+// sf_channels: channels per scale block (128 for MXFP4, 64 for NVFP4)
 cudaError_t launch_gather_quantized(const int32_t* row_token, int T, int K, int Kop, const void* xq_u, const void* sf_u,
                                     const void* xo_u, void* xq, void* sf, void* xo, const int32_t* sched, int max_tiles,
-                                    cudaStream_t st);
+                                    cudaStream_t st, int sf_channels = 128);
 
 // norm_kernels.cu
 cudaError_t launch_rmsnorm_quant(bool quant, const void* H, int64_t ldh, int M, int K, const void* gamma, float eps,
                                  void* Xn, int64_t ldx, const int32_t* idx_o, void* xq, void* sf,
                                  void* xo, int Ko, int Kop, cudaStream_t st, const void* R = nullptr, int64_t ldr = 0,
                                  void* Hout = nullptr, int64_t ldo = 0);
+
+cudaError_t launch_rmsnorm_quant_nvfp4(const void* H, int64_t ldh, int M, int K, const void* gamma, float eps,
+                                       const int32_t* idx_o, void* xq, void* sf, void* xo, int Ko, int Kop, int tensor_e,
+                                       cudaStream_t st);
 
 cudaError_t launch_swiglu_fp8(bool quant, const void* GU, int64_t ldg, int M, int I, void* Hout, int64_t ldh, void* x8,
                               void* sx, cudaStream_t st);

@@ -40,13 +40,15 @@ __device__ __forceinline__ void team_sync(int slot) {
 
 // Two CTAs per SM (28 rows in flight) need at most 36 registers per thread; the residual update is a template
 // parameter so that the plain form keeps its 32.
-template <bool QUANT, bool ADD>
-__global__ void __launch_bounds__(RN_THREADS, 2)
+// FMT: FMT_MXFP4 (Algorithm 2 as stated) or FMT_NVFP4 (blocks of 16 with E4M3 scales, tensor scale 2^tensor_e,
+// scale blocks of 64 channels; fp32 scale arithmetic, so one CTA per SM).
+template <bool QUANT, bool ADD, int FMT = FMT_MXFP4>
+__global__ void __launch_bounds__(RN_THREADS, FMT == FMT_MXFP4 ? 2 : 1)
 rmsnorm_quant_kernel(const uint16_t* __restrict__ H, int64_t ldh, int M, int M_pad, int K,
                      const uint16_t* __restrict__ gamma, float eps, uint16_t* __restrict__ Xn, int64_t ldx,
                      const int32_t* __restrict__ idx_o, uint8_t* __restrict__ xq,
                      uint8_t* __restrict__ sf, uint16_t* __restrict__ xo, int Ko, int Kop,
-                     const uint16_t* R, int64_t ldr, uint16_t* Hout, int64_t ldo) {
+                     const uint16_t* R, int64_t ldr, uint16_t* Hout, int64_t ldo, int tensor_e) {
     // [RN_ROWS][K / 8] rows, then per row: one mbarrier, two partial sums (double), one give-up flag
     extern __shared__ uint4 rn_rows[];
     grid_launch_dependents();
@@ -55,8 +57,8 @@ rmsnorm_quant_kernel(const uint16_t* __restrict__ H, int64_t ldh, int M, int M_p
     const int lane = threadIdx.x & 31;
     const int r = blockIdx.x * RN_ROWS + slot;
     if (r >= M_pad) return;                          // both warps of a team take every exit together
-    const int katoms = K / 128;
-    // scale word of (row r, 128-channel block a): block (r/128)*katoms + a, word (r%32)*4 + (r%128)/32
+    const int katoms = K / (FMT == FMT_NVFP4 ? 64 : 128);   // scale blocks along K
+    // scale word of (row r, scale block a): block (r/128)*katoms + a, word (r%32)*4 + (r%128)/32
     uint32_t* sf_row = QUANT ? reinterpret_cast<uint32_t*>(sf + (size_t)(r / 128) * katoms * 512) + (r & 31) * 4 + ((r & 127) >> 5)
                              : nullptr;
     if (r >= M) {   // rows that only pad the last 128-row scale block
@@ -160,6 +162,7 @@ rmsnorm_quant_kernel(const uint16_t* __restrict__ H, int64_t ldh, int M, int M_p
             const int ch = idx_o[t];
             e = row16[ch];
             row16[ch] = 0;
+            if (FMT == FMT_NVFP4) e = nvfp4_backup(e, tensor_e);
         }
         xo[(int64_t)r * Kop + t] = e;
     }
@@ -175,6 +178,16 @@ rmsnorm_quant_kernel(const uint16_t* __restrict__ H, int64_t ldh, int M, int M_p
         for (int j = 0; j < 4; ++j) {
             const uint4 v = in ? row[4 * g + j] : make_uint4(0u, 0u, 0u, 0u);
             w[4 * j] = v.x; w[4 * j + 1] = v.y; w[4 * j + 2] = v.z; w[4 * j + 3] = v.w;
+        }
+        if (FMT == FMT_NVFP4) {
+            uint32_t q[4];
+            const uint32_t codes = nvfp4_group(w, __uint_as_float((uint32_t)(127 - tensor_e) << 23), q);
+            if (in) *reinterpret_cast<uint4*>(xq + (int64_t)r * (K / 2) + g * 16) = make_uint4(q[0], q[1], q[2], q[3]);
+            // a 64-channel scale block is two 32-channel groups: two bytes from each of two neighbouring lanes
+            uint32_t word = codes << (16 * (g & 1));
+            word |= __shfl_xor_sync(0xFFFFFFFFu, word, 1);
+            if ((g & 1) == 0 && in) sf_row[(size_t)(g >> 1) * 128] = word;
+            continue;
         }
         __nv_bfloat162 m2 = __habs2(as_bf162(w[0]));
 #pragma unroll
@@ -210,17 +223,29 @@ rmsnorm_quant_kernel(const uint16_t* __restrict__ H, int64_t ldh, int M, int M_p
 
 constexpr int kRnTail = RN_ROWS * (8 + RN_WPR * 8 + 4) + 8;   // mbarriers, partial sums, give-up flags
 
-template <bool QUANT, bool ADD>
+template <bool QUANT, bool ADD, int FMT = FMT_MXFP4>
 static cudaError_t launch_rmsnorm_cfg(dim3 grid, dim3 block, size_t smem, cudaStream_t st, const void* H, int64_t ldh, int M,
                                       int M_pad, int K, const void* gamma, float eps, void* Xn, int64_t ldx,
                                       const int32_t* idx_o, void* xq, void* sf, void* xo, int Ko, int Kop, const void* R,
-                                      int64_t ldr, void* Hout, int64_t ldo) {
+                                      int64_t ldr, void* Hout, int64_t ldo, int tensor_e = 0) {
     static PerDevice configured;
-    if (cudaError_t e = opt_in_shared_memory(configured, rmsnorm_quant_kernel<QUANT, ADD>, RN_ROWS * 8192 * 2 + kRnTail)) return e;
-    return launch_pdl(rmsnorm_quant_kernel<QUANT, ADD>, grid, block, smem, st, static_cast<const uint16_t*>(H), ldh, M, M_pad, K,
+    if (cudaError_t e = opt_in_shared_memory(configured, rmsnorm_quant_kernel<QUANT, ADD, FMT>, RN_ROWS * 8192 * 2 + kRnTail)) return e;
+    return launch_pdl(rmsnorm_quant_kernel<QUANT, ADD, FMT>, grid, block, smem, st, static_cast<const uint16_t*>(H), ldh, M, M_pad, K,
                       static_cast<const uint16_t*>(gamma), eps, static_cast<uint16_t*>(Xn), ldx, idx_o,
                       static_cast<uint8_t*>(xq), static_cast<uint8_t*>(sf), static_cast<uint16_t*>(xo), Ko, Kop,
-                      static_cast<const uint16_t*>(R), ldr, static_cast<uint16_t*>(Hout), ldo);
+                      static_cast<const uint16_t*>(R), ldr, static_cast<uint16_t*>(Hout), ldo, tensor_e);
+}
+
+// RMSNorm + the NVFP4 form of Algorithm 2 (no residual update in this form)
+cudaError_t launch_rmsnorm_quant_nvfp4(const void* H, int64_t ldh, int M, int K, const void* gamma, float eps,
+                                       const int32_t* idx_o, void* xq, void* sf, void* xo, int Ko, int Kop, int tensor_e,
+                                       cudaStream_t st) {
+    if (M <= 0) return cudaSuccess;
+    const int M_pad = (M + 127) / 128 * 128;
+    const dim3 grid((M_pad + RN_ROWS - 1) / RN_ROWS), block(RN_THREADS);
+    return launch_rmsnorm_cfg<true, false, FMT_NVFP4>(grid, block, (size_t)RN_ROWS * K * 2 + kRnTail, st, H, ldh, M, M_pad, K,
+                                                      gamma, eps, nullptr, 0, idx_o, xq, sf, xo, Ko, Kop, nullptr, 0, nullptr, 0,
+                                                      tensor_e);
 }
 
 // QUANT: Xn unused.  !QUANT: the quantizer arguments unused.  K <= 8192.  R != null: residual update h' = bf16(h + r)

@@ -80,6 +80,49 @@ __device__ __forceinline__ uint32_t e2m1x8(float f0, float f1, float f2, float f
 constexpr int FMT_MXFP4 = 0;
 constexpr int FMT_NVFP4 = 1;
 
+// NVFP4 arithmetic of one 32-channel group held as 16 packed bf16 pairs: two blocks of 16, per block
+// t = fl32(amax' * fl32(1/6)) with amax' the block maximum in the scaled domain (x * p2, p2 = 2^-tensor_e, exact),
+// scale byte = E4M3(t) nearest-even saturating, codes = E2M1(fl32(x * fac)) with fac = fl32(1/scale) * p2.
+// Returns the two scale bytes (block 0 in bits 7:0) and the 32 packed codes in q.
+__device__ __forceinline__ uint32_t nvfp4_group(const uint32_t (&w)[16], float p2, uint32_t (&q)[4]) {
+    uint32_t codes = 0;
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        __nv_bfloat162 m2 = __habs2(as_bf162(w[8 * h]));
+#pragma unroll
+        for (int i = 1; i < 8; ++i) m2 = __hmax2(m2, __habs2(as_bf162(w[8 * h + i])));
+        const uint32_t am2 = bf162_bits(m2);
+        const float amax = __uint_as_float(max(am2 & 0xFFFFu, am2 >> 16) << 16) * p2;   // exact
+        const float t = __fmul_rn(amax, __fdiv_rn(1.0f, 6.0f));
+        const uint32_t sb = e4m3x2(t, 0.0f) & 0xFFu;          // nearest-even, saturating at 448
+        codes |= sb << (8 * h);
+        // value of the scale byte: exponent field e, mantissa m -> (8 + m) * 2^(e - 10), or m * 2^-9
+        const int se = (int)(sb >> 3), sm = (int)(sb & 7u);
+        const float sbv = se ? __uint_as_float((uint32_t)(se + 120) << 23) * (1.0f + 0.125f * (float)sm)
+                             : 0.001953125f * (float)sm;
+        // one factor per block: fl32(1/scale) times the (exact) power of two of the tensor scale
+        const float fac = sbv > 0.0f ? __fdiv_rn(1.0f, sbv) * p2 : 0.0f;
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            float f[8];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const uint32_t u = w[8 * h + 4 * i + j];
+                f[2 * j] = __fmul_rn(__uint_as_float(u << 16), fac);
+                f[2 * j + 1] = __fmul_rn(__uint_as_float(u & 0xFFFF0000u), fac);
+            }
+            q[2 * h + i] = e2m1x8(f[0], f[1], f[2], f[3], f[4], f[5], f[6], f[7]);
+        }
+    }
+    return codes;
+}
+
+// bf16 bits of x * 2^-tensor_e rounded to bf16 (nearest even): the backed-up channel in the scaled domain of NVFP4
+__device__ __forceinline__ uint16_t nvfp4_backup(uint16_t b, int tensor_e) {
+    return __bfloat16_as_ushort(__float2bfloat16_rn(
+        __uint_as_float((uint32_t)b << 16) * __uint_as_float((uint32_t)(127 - tensor_e) << 23)));
+}
+
 template <int FMT>
 __global__ void __launch_bounds__(QE_THREADS, QE_CTAS_PER_SM)
 quant_extract_kernel(const __grid_constant__ CUtensorMap tm_x, int M, int K,
@@ -184,9 +227,7 @@ quant_extract_kernel(const __grid_constant__ CUtensorMap tm_x, int M, int K,
                                                           ((((within >> 4) ^ (grow & 7))) << 4) + (within & 15));
                 if (r < row_end) {
                     uint16_t b = *e;
-                    if (FMT == FMT_NVFP4)   // into the scaled domain of the block-scaled path (exact for normal results)
-                        b = __bfloat16_as_ushort(__float2bfloat16_rn(
-                            __uint_as_float((uint32_t)b << 16) * __uint_as_float((uint32_t)(127 - tensor_e) << 23)));
+                    if (FMT == FMT_NVFP4) b = nvfp4_backup(b, tensor_e);   // into the scaled domain of the block-scaled path
                     xo[(int64_t)r * Kop + slot] = b;
                 }
                 ++slot;
@@ -254,36 +295,8 @@ quant_extract_kernel(const __grid_constant__ CUtensorMap tm_x, int M, int K,
             // NVFP4: my 32 channels are two blocks of 16
             uint32_t codes = 0;
             if (r < row_end) {
-                const float p2 = __uint_as_float((uint32_t)(127 - tensor_e) << 23);   // 2^-tensor_e
                 uint32_t q[4];
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    __nv_bfloat162 m2 = __habs2(as_bf162(w[8 * h]));
-#pragma unroll
-                    for (int i = 1; i < 8; ++i) m2 = __hmax2(m2, __habs2(as_bf162(w[8 * h + i])));
-                    const uint32_t am2 = bf162_bits(m2);
-                    const float amax = __uint_as_float(max(am2 & 0xFFFFu, am2 >> 16) << 16) * p2;   // exact
-                    const float t = __fmul_rn(amax, __fdiv_rn(1.0f, 6.0f));
-                    const uint32_t sb = e4m3x2(t, 0.0f) & 0xFFu;          // nearest-even, saturating at 448
-                    codes |= sb << (8 * h);
-                    // value of the scale byte: exponent field e, mantissa m -> (8 + m) * 2^(e - 10), or m * 2^-9
-                    const int se = (int)(sb >> 3), sm = (int)(sb & 7u);
-                    const float sbv = se ? __uint_as_float((uint32_t)(se + 120) << 23) * (1.0f + 0.125f * (float)sm)
-                                         : 0.001953125f * (float)sm;
-                    // one factor per block: fl32(1/scale) times the (exact) power of two of the tensor scale
-                    const float fac = sbv > 0.0f ? __fdiv_rn(1.0f, sbv) * p2 : 0.0f;
-#pragma unroll
-                    for (int i = 0; i < 2; ++i) {
-                        float f[8];
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const uint32_t u = w[8 * h + 4 * i + j];
-                            f[2 * j] = __fmul_rn(__uint_as_float(u << 16), fac);
-                            f[2 * j + 1] = __fmul_rn(__uint_as_float(u & 0xFFFF0000u), fac);
-                        }
-                        q[2 * h + i] = e2m1x8(f[0], f[1], f[2], f[3], f[4], f[5], f[6], f[7]);
-                    }
-                }
+                codes = nvfp4_group(w, __uint_as_float((uint32_t)(127 - tensor_e) << 23), q);
                 *reinterpret_cast<uint4*>(xq + (int64_t)r * (K / 2) + cb * (QE_COLS / 2) + gi * 16) =
                     make_uint4(q[0], q[1], q[2], q[3]);
             }
@@ -736,7 +749,7 @@ constexpr int GQ_WARPS = 16;              // warps per block; each takes 128 / G
 constexpr int GQ_RPW = 128 / GQ_WARPS;
 
 __global__ void __launch_bounds__(32 * GQ_WARPS)
-gather_quantized_kernel(const int32_t* __restrict__ row_token, int T, int K, int Kop,
+gather_quantized_kernel(const int32_t* __restrict__ row_token, int T, int K, int Kop, int katoms,
                         const uint8_t* __restrict__ xq_u, const uint8_t* __restrict__ sf_u, const uint16_t* __restrict__ xo_u,
                         uint8_t* __restrict__ xq, uint8_t* __restrict__ sf, uint16_t* __restrict__ xo,
                         const int32_t* __restrict__ sched, int max_tiles) {
@@ -747,7 +760,7 @@ gather_quantized_kernel(const int32_t* __restrict__ row_token, int T, int K, int
     if (tile >= sched[0]) return;
     const int row0 = sched[1 + tile], row_end = sched[1 + max_tiles + tile], sf_row0 = sched[1 + 2 * max_tiles + tile];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int katoms = K / 128;
+    // katoms: scale blocks along K (K / 128 for MXFP4, K / 64 for NVFP4)
     const int nq = K / 32;          // 16-byte chunks of a row of packed codes
     const int no = Kop / 8;         // 16-byte chunks of a row of backed-up channels
     const uint32_t* sfu32 = reinterpret_cast<const uint32_t*>(sf_u);
@@ -804,9 +817,13 @@ gather_quantized_kernel(const int32_t* __restrict__ row_token, int T, int K, int
 
 cudaError_t launch_gather_quantized(const int32_t* row_token, int T, int K, int Kop, const void* xq_u, const void* sf_u,
                                     const void* xo_u, void* xq, void* sf, void* xo, const int32_t* sched, int max_tiles,
-                                    cudaStream_t st) {
+                                    cudaStream_t st, int sf_channels) {
     if (max_tiles <= 0) return cudaSuccess;
-    return launch_pdl(gather_quantized_kernel, dim3(max_tiles), dim3(32 * GQ_WARPS), (size_t)(K / 128) * 512, st, row_token, T, K, Kop,
+    const int katoms = K / sf_channels;
+    static PerDevice configured;   // the tile's scale block row is staged in shared memory: beyond 48 KB it must be asked for
+    if ((size_t)katoms * 512 > 48 * 1024)
+        if (cudaError_t e = opt_in_shared_memory(configured, gather_quantized_kernel, 160 * 1024)) return e;
+    return launch_pdl(gather_quantized_kernel, dim3(max_tiles), dim3(32 * GQ_WARPS), (size_t)katoms * 512, st, row_token, T, K, Kop, katoms,
                       static_cast<const uint8_t*>(xq_u), static_cast<const uint8_t*>(sf_u), static_cast<const uint16_t*>(xo_u),
                       static_cast<uint8_t*>(xq), static_cast<uint8_t*>(sf), static_cast<uint16_t*>(xo), sched, max_tiles);
 }

@@ -139,3 +139,15 @@ def test_residual_forms_validate_before_launching():
     assert lib.osc_add_rmsnorm_linear(None, None, None, 0, 0, 0, None, C.c_float(0), None, 0, None, 0, None, 0, None) == -1
     assert lib.osc_add_rmsnorm_quantize_extract(None, None, None, 0, 0, 0, None, C.c_float(0), None, 0, None, None, None,
                                                 None) == -1
+
+
+def test_nvfp4_fused_calls_refuse_null_handles():
+    from paper_2604_12782_b200 import binding as B
+    lib = B._lib
+    sz = C.c_size_t()
+    assert lib.osc_nvfp4_rmsnorm_quantize_extract(None, None, 0, 0, None, C.c_float(0), 0, None, None, None, None) == -1
+    assert lib.osc_nvfp4_rmsnorm_linear(None, None, 0, 0, None, C.c_float(0), 0, None, 0, None, 0, None) == -1
+    assert lib.osc_nvfp4_gather_workspace_bytes(None, 0, 0, C.byref(sz)) == -1
+    assert lib.osc_nvfp4_linear_grouped_gather(None, None, 0, 0, None, None, 0, 0, None, 0, None, 0, None) == -1
+    assert lib.osc_nvfp4_rmsnorm_linear_grouped_gather(None, None, 0, 0, None, C.c_float(0), None, None, 0, 0, None, 0, None, 0,
+                                                       None) == -1

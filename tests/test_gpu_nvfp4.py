@@ -146,3 +146,101 @@ def test_nvfp4_grouped(B, oracle, counts):
         B.osc_nvfp4_linear_grouped(wd, dev_bf16(c["X"]), torch.from_numpy(off_h).cuda(), ex, Y, ws)
     with pytest.raises(B.OscError):
         B.osc_nvfp4_linear(w, dev_bf16(c["X"]), ex, Y, ws)
+
+
+# ---- the producer fusion and the dispatch gather in the NVFP4 form ---------------------------------------------
+
+@pytest.mark.parametrize("M,K,N,kind", [(1, 128, 64, "one"), (37, 384, 192, "two"), (130, 1024, 320, "one"),
+                                        (300, 4096, 256, "one"), (64, 8192, 64, "empty"), (700, 512, 448, "two")])
+def test_nvfp4_rmsnorm_fused(B, oracle, M, K, N, kind):
+    """RMSNorm + the NVFP4 form of Algorithm 2 in one kernel: codes, E4M3 scale bytes and backed-up channels bit for
+    bit what the oracle's RMSNorm followed by its NVFP4 quantizer gives, and byte for byte the library's own two-step
+    path; the linear within the tolerance."""
+    from producer_inputs import gamma_bits, residual_rows
+    rng = np.random.default_rng(M + K)
+    Hb, gb = residual_rows(rng, M, K), gamma_bits(rng, K)
+    lut16 = {"one": rng.integers(0, 16, size=(K // 16, 1)).astype(np.int8), "empty": np.full((K // 16, 1), -1, np.int8),
+             "two": np.stack([rng.permutation(16)[:2] for _ in range(K // 16)]).astype(np.int8)}[kind]
+    Wb = synth.f32_to_bf16_bits((0.02 * rng.standard_normal((N, K))).astype(np.float32))
+    eps = 1e-6
+    Xn = oracle.rmsnorm(Hb, gb, eps)
+    ex, ew = synth.nvfp4_tensor_exponent(Xn), synth.nvfp4_tensor_exponent(Wb)
+    w = B.osc_nvfp4_prepare_weights(dev_bf16(Wb), lut16, ew)
+    sz = B.osc_nvfp4_act_sizes(w, M)
+    ws = poison(sz.workspace_bytes)
+    Y = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+    B.osc_nvfp4_rmsnorm_linear(w, dev_bf16(Hb), dev_bf16(gb), eps, ex, Y, ws)
+    B.osc_sync_check()
+    Yref, T, act, _ = oracle.nvfp4_linear(Xn, Wb, lut16, ex, ew)
+    h = host_u8(ws)
+    check_quantized(act, h[sz.xq_offset:sz.xq_offset + sz.xq_bytes], h[sz.sfa_offset:sz.sfa_offset + sz.sfa_bytes],
+                    h[sz.xo_offset:sz.xo_offset + sz.xo_bytes], M, K)
+    assert_within_tolerance(host_f64(Y), Yref, T, f"nvfp4 rmsnorm linear M={M} K={K}")
+    # two-step path of the library: own RMSNorm kernel, then the stand-alone NVFP4 quantizer
+    Xd = torch.empty(M, K, dtype=torch.bfloat16, device="cuda")
+    B.osc_rmsnorm(dev_bf16(Hb), dev_bf16(gb), eps, Xd)
+    ws2 = poison(sz.workspace_bytes)
+    B.osc_nvfp4_quantize_extract(w, Xd, ex, ws2[sz.xq_offset:], ws2[sz.sfa_offset:], ws2[sz.xo_offset:])
+    ws3 = poison(sz.workspace_bytes)
+    B.osc_nvfp4_rmsnorm_quantize_extract(w, dev_bf16(Hb), dev_bf16(gb), eps, ex, ws3[sz.xq_offset:], ws3[sz.sfa_offset:],
+                                         ws3[sz.xo_offset:])
+    B.osc_sync_check()
+    h2, h3 = host_u8(ws2), host_u8(ws3)
+    for o, n in ((sz.xq_offset, sz.xq_bytes), (sz.xo_offset, sz.xo_bytes)):
+        assert np.array_equal(h2[o:o + n], h3[o:o + n])
+    v = sf16_valid(M, K)
+    assert np.array_equal(h2[sz.sfa_offset:sz.sfa_offset + sz.sfa_bytes][v], h3[sz.sfa_offset:sz.sfa_offset + sz.sfa_bytes][v])
+    B.osc_nvfp4_rmsnorm_linear(w, dev_bf16(Hb)[:0], dev_bf16(gb), eps, ex, Y[:0], ws)     # M == 0: a no-op
+    wm = B.osc_prepare_weights(dev_bf16(Wb), np.full((K // 32, 1), -1, np.int8))
+    with pytest.raises(B.OscError):                                                        # an MXFP4 handle is refused
+        B.osc_nvfp4_rmsnorm_linear(wm, dev_bf16(Hb), dev_bf16(gb), eps, ex, Y, ws)
+
+
+@pytest.mark.parametrize("counts,with_norm", [([3, 0, 130, 1, 257, 128], False), ([300, 0, 5, 256, 129, 511, 1, 385], True),
+                                              ([700, 64, 0, 900], False)])
+def test_nvfp4_grouped_gather(B, oracle, counts, with_norm):
+    """The dispatch fused behind the NVFP4 quantizer: T tokens quantized once and their quantized rows gathered; bit
+    for bit what osc_nvfp4_linear_grouped gives on the permuted matrix X[row_token] (and, behind an RMSNorm, on the
+    permuted normalized rows)."""
+    from producer_inputs import gamma_bits
+    counts = np.array(counts)
+    E, K, N = counts.size, 512, 320
+    M = int(counts.sum())
+    T = max(1, M // 3)
+    off_h = synth.offsets_from_counts(counts)
+    off = torch.from_numpy(off_h).cuda()
+    rng = np.random.default_rng(E + M)
+    c = synth.osc16_linear_case(60 + E, T, K, N)
+    row_token_h = rng.integers(0, T, size=M).astype(np.int32)
+    row_token = torch.from_numpy(row_token_h).cuda()
+    Wb = synth.f32_to_bf16_bits((0.02 * rng.standard_normal((E, N, K))).astype(np.float32))
+    gb = gamma_bits(rng, K)
+    src = oracle.rmsnorm(c["X"], gb, 1e-6) if with_norm else c["X"]
+    ex, ew = synth.nvfp4_tensor_exponent(src), synth.nvfp4_tensor_exponent(Wb)
+    w = B.osc_nvfp4_prepare_weights_grouped(dev_bf16(Wb.reshape(E * N, K)).view(E, N, K), c["lut16"], ew)
+    wsg = poison(B.osc_nvfp4_gather_workspace_bytes(w, T, M))
+    Y = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+    if with_norm:
+        B.osc_nvfp4_rmsnorm_linear_grouped_gather(w, dev_bf16(c["X"]), dev_bf16(gb), 1e-6, row_token, off, ex, Y, wsg)
+    else:
+        B.osc_nvfp4_linear_grouped_gather(w, dev_bf16(c["X"]), row_token, off, ex, Y, wsg)
+    B.osc_sync_check()
+    # the grouped call on the permuted matrix
+    Xp = np.ascontiguousarray(src[row_token_h])
+    sz = B.osc_nvfp4_act_sizes(w, M)
+    ws = poison(sz.workspace_bytes)
+    Y2 = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+    B.osc_nvfp4_linear_grouped(w, dev_bf16(Xp), off, ex, Y2, ws)
+    B.osc_sync_check()
+    assert torch.equal(Y.view(torch.int16), Y2.view(torch.int16))
+    hg, hp = host_u8(wsg), host_u8(ws)
+    for o, n in ((sz.xq_offset, sz.xq_bytes), (sz.xo_offset, sz.xo_bytes)):
+        assert np.array_equal(hg[o:o + n], hp[o:o + n])
+    # and against the oracle, expert by expert
+    Yh = host_f64(Y)
+    for e in range(E):
+        r0, r1 = int(off_h[e]), int(off_h[e + 1])
+        if r1 > r0:
+            Yref, Tt, *_ = oracle.nvfp4_linear(Xp[r0:r1], Wb[e], c["lut16"], ex, ew)
+            assert_within_tolerance(Yh[r0:r1], Yref, Tt, f"gathered grouped nvfp4, expert {e}")
+    assert not torch.isnan(Y.float()).any()
