@@ -1049,6 +1049,25 @@ def run_sweep(args):
         B.osc_sync_check()
         rows.append({"name": "layer.fused(rmsnorm+qkv,o_proj,rmsnorm+gate_up,swiglu+down_fp8)", "M": M, "ms": ms_f,
                      "separate_kernels_ms": ms_s, "speedup": ms_s / ms_f})
+        # the same with the activation in the epilogue of the gate|up projection: the [M, 2I] matrix is never written,
+        # the down projection's quantizer reads H [M, I]
+        gu_w = [B.osc_prepare_weights_gate_up(torch.roll(dev_bf16(torch, synth.osc_linear_case(2, 1, 4096, 24576, 1)["W"]), 61 * j, 0).contiguous(),
+                                              synth.osc_linear_case(2, 1, 4096, 24576, 1)["lut"]) for j in range(1)]
+        gu_ws = torch.empty(B.osc_linear_swiglu_workspace_bytes(gu_w[0], M), dtype=torch.uint8, device="cuda")
+        Hd = torch.empty(M, 12288, dtype=torch.bfloat16, device="cuda")
+
+        def fused_epilogue(i):
+            j = i % 2
+            B.osc_rmsnorm_linear(qkv.w[j], qkv.X[j], gam, eps, qkv.Y[j], qkv.ws[j])
+            B.osc_linear(opj.w[j], opj.X[j], opj.Y[j], opj.ws[j])
+            B.osc_rmsnorm_linear_swiglu(gu_w[0], gup.X[j], gam, eps, Hd, gu_ws)
+            B.osc_fp8_linear(dwn.w[j], Hd, dwn.Y[j], dwn.ws[j])
+
+        ms_e = time_loop(torch, fused_epilogue, steps, warm)
+        B.osc_sync_check()
+        rows.append({"name": "layer.fused_epilogue(rmsnorm+qkv,o_proj,rmsnorm+gate_up+swiglu,down_fp8)", "M": M, "ms": ms_e,
+                     "fused_quantizers_ms": ms_f, "separate_kernels_ms": ms_s, "speedup_vs_separate": ms_s / ms_e})
+        del gu_w, gu_ws, Hd
         # the same with the two residual updates of the layer in the picture: h' = h + branch output in front of each
         # norm, written to a scratch stream so that the values do not drift over the timed iterations
         Hn = [torch.empty(M, 4096, dtype=torch.bfloat16, device="cuda") for _ in range(2)]

@@ -329,6 +329,30 @@ osc_status osc_swiglu_fp8_linear_grouped(const osc_fp8_weights* w, const void* G
                                          int64_t ldg, void* Y, int64_t ldy, void* workspace, size_t workspace_bytes,
                                          void* stream);
 
+/* ---- SwiGLU in the epilogue of the gate|up projection ------------------------------------------------------
+ * The next step of the same placement (Section 3.3): the activation is applied where the gate|up projection's
+ * accumulators are, so the [M, 2I] output of that projection is never written or read; H [M, I] goes to the down
+ * projection's FP8 quantizer (Section 3.4) at half the bytes.
+ *   W    dev bf16 [2I, ldw]: gate rows [0, I) above up rows [I, 2I) (the nn.Linear layout of a fused gate_up weight).
+ *   osc_gate_up_weight_sizes / osc_prepare_weights_gate_up: as osc_weight_sizes / osc_prepare_weights with N = 2I;
+ *        meta is larger (a second per-tile copy of the weight scales, rows of a tile in gate|up order).  The handle
+ *        is a full dense OSC handle: osc_linear, osc_gemm_dual, ... give the plain [M, 2I] projection with it.
+ *   osc_linear_swiglu: H = bf16( silu(bf16(Yg)) * bf16(Yu) ) with Y = the OSC linear of Algorithm 2 + Eq. 5 and the
+ *        activation arithmetic of osc_swiglu: bit for bit what osc_swiglu gives on osc_gemm_dual's output for the same
+ *        quantized operands.  H dev bf16 [M, ldh], ldh >= I, multiple of 8.  I a multiple of 64.
+ *        Workspace: osc_linear_swiglu_workspace_bytes(w, M) (the buffers of osc_act_sizes; problems of up to 256 rows
+ *        run the plain projection into a scratch [M, 2I] behind them and the stand-alone activation).
+ *   osc_rmsnorm_linear_swiglu: the same behind an RMSNorm fused into the quantizer (as osc_rmsnorm_linear).
+ * Errors: OSC_ERR_INVALID_ARG for a handle not prepared by osc_prepare_weights_gate_up, otherwise as osc_linear. */
+osc_status osc_gate_up_weight_sizes(int I, int K, const int8_t* lut, int lut_c, osc_weight_sizes_t* out);
+osc_status osc_prepare_weights_gate_up(const void* W, int I, int K, int64_t ldw, const int8_t* lut, int lut_c, void* wq,
+                                       void* sfw, void* wo, void* meta, void* stream, osc_weights** out);
+osc_status osc_linear_swiglu_workspace_bytes(const osc_weights* w, int M, size_t* bytes);
+osc_status osc_linear_swiglu(const osc_weights* w, const void* X, int M, int64_t ldx, void* H, int64_t ldh, void* workspace,
+                             size_t workspace_bytes, void* stream);
+osc_status osc_rmsnorm_linear_swiglu(const osc_weights* w, const void* Hin, int M, int64_t ldh_in, const void* gamma, float eps,
+                                     void* H, int64_t ldh, void* workspace, size_t workspace_bytes, void* stream);
+
 /* ------------------------------------- MXFP8 form of the fallback (Section 3.4) */
 
 /* Section 3.4 allows "FP8 (or equivalent 8-bit micro-scaling formats)" for the W2 inputs and Section 4

@@ -113,6 +113,11 @@ _SIGS = {
     "osc_nvfp4_quantize_extract": (_i, [_vp, _vp, _i, _i64, _i, _vp, _vp, _vp, _vp]),
     "osc_nvfp4_gemm": (_i, [_vp, _vp, _vp, _vp, _i, _i, _vp, _i64, _vp]),
     "osc_nvfp4_linear": (_i, [_vp, _vp, _i, _i64, _i, _vp, _i64, _vp, _sz, _vp]),
+    "osc_gate_up_weight_sizes": (_i, [_i, _i, _vp, _i, C.POINTER(WeightSizes)]),
+    "osc_prepare_weights_gate_up": (_i, [_vp, _i, _i, _i64, _vp, _i, _vp, _vp, _vp, _vp, _vp, C.POINTER(_vp)]),
+    "osc_linear_swiglu_workspace_bytes": (_i, [_vp, _i, C.POINTER(_sz)]),
+    "osc_linear_swiglu": (_i, [_vp, _vp, _i, _i64, _vp, _i64, _vp, _sz, _vp]),
+    "osc_rmsnorm_linear_swiglu": (_i, [_vp, _vp, _i, _i64, _vp, C.c_float, _vp, _i64, _vp, _sz, _vp]),
     "osc_nvfp4_rmsnorm_quantize_extract": (_i, [_vp, _vp, _i, _i64, _vp, C.c_float, _i, _vp, _vp, _vp, _vp]),
     "osc_nvfp4_rmsnorm_linear": (_i, [_vp, _vp, _i, _i64, _vp, C.c_float, _i, _vp, _i64, _vp, _sz, _vp]),
     "osc_nvfp4_gather_workspace_bytes": (_i, [_vp, _i, _i, C.POINTER(_sz)]),
@@ -697,3 +702,41 @@ def osc_nvfp4_rmsnorm_linear_grouped_gather(w: OscWeights, H: torch.Tensor, gamm
                                                         _ptr(row_token), _ptr(off), M, int(ex), _ptr(Y),
                                                         Y.stride(0) if M else w.N, _ptr(workspace),
                                                         workspace.numel() * workspace.element_size(), _stream(stream)))
+
+
+def osc_prepare_weights_gate_up(W: torch.Tensor, lut, stream=None) -> OscWeights:
+    """W: cuda bf16 [2I, K], gate rows above up rows.  A dense OSC handle that also serves osc_linear_swiglu."""
+    N, K = W.shape
+    I = N // 2
+    lut = _lut(lut)
+    sz = WeightSizes()
+    _check(_lib.osc_gate_up_weight_sizes(I, K, lut.ctypes.data, lut.shape[1], C.byref(sz)))
+    bufs = {k: _alloc(getattr(sz, k + "_bytes"), W.device) for k in ("wq", "sfw", "wo", "meta")}
+    h = _vp()
+    _check(_lib.osc_prepare_weights_gate_up(_ptr(W), I, K, W.stride(0), lut.ctypes.data, lut.shape[1], _ptr(bufs["wq"]),
+                                            _ptr(bufs["sfw"]), _ptr(bufs["wo"]) if sz.wo_bytes else None, _ptr(bufs["meta"]),
+                                            _stream(stream), C.byref(h)))
+    w = OscWeights(h.value, bufs)
+    w.E, w.N, w.K, w.K_o, w.K_o_pad, w.sizes = 1, N, K, sz.K_o, sz.K_o_pad, sz
+    return w
+
+
+def osc_linear_swiglu_workspace_bytes(w: OscWeights, M: int) -> int:
+    out = _sz()
+    _check(_lib.osc_linear_swiglu_workspace_bytes(w.ptr, M, C.byref(out)))
+    return int(out.value)
+
+
+def osc_linear_swiglu(w: OscWeights, X: torch.Tensor, H: torch.Tensor, workspace: torch.Tensor, stream=None):
+    """H [M, I] = silu(gate) * up of the gate|up projection of X, the activation applied in the GEMM epilogue."""
+    M = X.shape[0]
+    _check(_lib.osc_linear_swiglu(w.ptr, _ptr(X), M, X.stride(0) if M else w.K, _ptr(H), H.stride(0) if M else w.N // 2,
+                                  _ptr(workspace), workspace.numel() * workspace.element_size(), _stream(stream)))
+
+
+def osc_rmsnorm_linear_swiglu(w: OscWeights, Hin: torch.Tensor, gamma: torch.Tensor, eps: float, H: torch.Tensor,
+                              workspace: torch.Tensor, stream=None):
+    M = Hin.shape[0]
+    _check(_lib.osc_rmsnorm_linear_swiglu(w.ptr, _ptr(Hin), M, Hin.stride(0) if M else w.K, _ptr(gamma), float(eps), _ptr(H),
+                                          H.stride(0) if M else w.N // 2, _ptr(workspace),
+                                          workspace.numel() * workspace.element_size(), _stream(stream)))

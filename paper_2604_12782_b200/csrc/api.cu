@@ -253,6 +253,8 @@ struct osc_weights {
     CUtensorMap tm_b[4], tm_bo[4];    // single-CTA kernel: weight tiles of 64 / 128 / 192 / 256 rows
     CUtensorMap tm_b2[3], tm_bo2[3];  // CTA-pair kernel: half tiles for 192-, 256- and 240-wide tiles
     CUtensorMap tm_sfw, tm_sfw_tiled;  // scale blocks: standard layout / per-tile copy for 240-wide tiles
+    bool gate_up;                      // prepared by osc_prepare_weights_gate_up: rows [0, N/2) gate, [N/2, N) up
+    CUtensorMap tm_sfw_gu;             // per-tile copy of the scales in the gate|up arrangement of a tile
 };
 struct osc_fp8_weights {
     int E, N, K;
@@ -324,7 +326,7 @@ osc_status osc_weight_sizes(int E, int N, int K, const int8_t* lut, int lut_c, o
 
 static osc_status prepare_impl(const void* W, int E, int N, int K, int64_t ldw, const int8_t* lut, int lut_c,
                                void* wq, void* sfw, void* wo, void* meta, void* stream, bool grouped,
-                               osc_weights** out, bool dynamic = false) {
+                               osc_weights** out, bool dynamic = false, bool gate_up = false) {
     if (!out) return fail(OSC_ERR_INVALID_ARG, "out is null");
     *out = nullptr;
     if (osc_status s = check_nk(E, N, K)) return s;
@@ -396,6 +398,13 @@ static osc_status prepare_impl(const void* W, int E, int N, int K, int64_t ldw, 
         e = launch_retile_sf(static_cast<const uint8_t*>(sfw), tiled, N, K, kTiledBN, st);
         if (e != cudaSuccess) { delete w; return cuda_fail(e, "retile_sf_kernel"); }
         s = make_tmap_sf(&w->tm_sfw_tiled, tiled, (uint64_t)tiled_sf_bytes(N, K) / 512);
+        if (s == OSC_OK && gate_up) {   // a second copy behind the first, rows of a tile in gate|up order
+            uint8_t* tiled_gu = tiled + tiled_sf_bytes(N, K);
+            e = launch_retile_sf(static_cast<const uint8_t*>(sfw), tiled_gu, N, K, kTiledBN, st, true);
+            if (e != cudaSuccess) { delete w; return cuda_fail(e, "retile_sf_kernel(gate|up)"); }
+            s = make_tmap_sf(&w->tm_sfw_gu, tiled_gu, (uint64_t)tiled_sf_bytes(N, K) / 512);
+            w->gate_up = true;
+        }
     }
     if (s == OSC_OK && (e = launch_prepare_fence(st)) != cudaSuccess) s = cuda_fail(e, "prepare_fence_kernel");
     if (s != OSC_OK) { delete w; return s; }
@@ -411,6 +420,19 @@ osc_status osc_prepare_weights_grouped(const void* W, int E, int N, int K, const
                                        void* sfw, void* wo, void* meta, void* stream, osc_weights** out) {
     return prepare_impl(W, E, N, K, K, lut, lut_c, wq, sfw, wo, meta, stream, true, out);
 }
+// ---- gate|up projection with the SwiGLU in the GEMM epilogue
+osc_status osc_gate_up_weight_sizes(int I, int K, const int8_t* lut, int lut_c, osc_weight_sizes_t* out) {
+    if (I <= 0 || I % 64 || I > (1 << 29)) return fail(OSC_ERR_SHAPE, "I = %d must be a positive multiple of 64", I);
+    if (osc_status s = osc_weight_sizes(1, 2 * I, K, lut, lut_c, out)) return s;
+    out->meta_bytes += tiled_sf_bytes(2 * I, K);
+    return OSC_OK;
+}
+osc_status osc_prepare_weights_gate_up(const void* W, int I, int K, int64_t ldw, const int8_t* lut, int lut_c, void* wq,
+                                       void* sfw, void* wo, void* meta, void* stream, osc_weights** out) {
+    if (I <= 0 || I % 64 || I > (1 << 29)) return fail(OSC_ERR_SHAPE, "I = %d must be a positive multiple of 64", I);
+    return prepare_impl(W, 1, 2 * I, K, ldw, lut, lut_c, wq, sfw, wo, meta, stream, false, out, false, true);
+}
+
 osc_status osc_weights_destroy(osc_weights* w) {
     delete w;
     return OSC_OK;
@@ -681,6 +703,89 @@ osc_status osc_add_rmsnorm_linear(const osc_weights* w, const void* H, const voi
     Residual res;
     res.R = R; res.ldr = ldr; res.Hout = Hout; res.ldo = ldo;
     return rmsnorm_linear_impl(w, H, M, ldh, gamma, eps, Y, ldy, workspace, workspace_bytes, stream, &res);
+}
+
+// ---- osc_linear on a gate|up handle with the activation in the epilogue: H = silu(gate) * up, [M, N/2]
+// Problems of more than kSwigluFusedMinRows rows run on the pair kernel's gate|up form; smaller ones take the plain
+// GEMM of the library's routing into a scratch Y behind the quantizer's buffers, then the stand-alone activation.
+constexpr int kSwigluFusedMinRows = 256;
+static bool swiglu_fused(const osc_weights* w, int M) {
+    static const int mode = [] { const char* e = getenv("OSC_SWIGLU_FUSED"); return e ? atoi(e) : 1; }();
+    return mode != 0 && M > kSwigluFusedMinRows && (w->N / 2) % 8 == 0;
+}
+
+osc_status osc_linear_swiglu_workspace_bytes(const osc_weights* w, int M, size_t* bytes) {
+    if (!w || !bytes) return fail(OSC_ERR_INVALID_ARG, "null argument");
+    if (!w->gate_up) return fail(OSC_ERR_INVALID_ARG, "not a gate|up handle: use osc_prepare_weights_gate_up");
+    osc_act_sizes_t sz;
+    if (osc_status s = osc_act_sizes(w, M, &sz)) return s;
+    *bytes = sz.workspace_bytes + (swiglu_fused(w, M) ? 0 : align256((size_t)M * w->N * 2));
+    return OSC_OK;
+}
+
+static osc_status linear_swiglu_impl(const osc_weights* w, const void* X, int M, int64_t ldx, const void* gamma, float eps,
+                                     void* H, int64_t ldh, void* workspace, size_t workspace_bytes, void* stream) {
+    if (osc_status s = check_act(w, X, M, ldx)) return s;
+    if (!w->gate_up) return fail(OSC_ERR_INVALID_ARG, "not a gate|up handle: use osc_prepare_weights_gate_up");
+    if (M == 0) return OSC_OK;
+    const int I = w->N / 2;
+    osc_act_sizes_t sz;
+    osc_act_sizes(w, M, &sz);
+    size_t need = 0;
+    osc_linear_swiglu_workspace_bytes(w, M, &need);
+    if (!workspace || !aligned16(workspace)) return fail(OSC_ERR_ALIGN, "workspace must be non-null and 16-byte aligned");
+    if (workspace_bytes < need) return fail(OSC_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", workspace_bytes, need);
+    if (!H) return fail(OSC_ERR_INVALID_ARG, "H is null");
+    if (ldh < I) return fail(OSC_ERR_SHAPE, "ldh = %lld < I = %d", (long long)ldh, I);
+    if (ldh % 8 || !aligned16(H)) return fail(OSC_ERR_ALIGN, "H must be 16-byte aligned and ldh a multiple of 8");
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint8_t *xq = ws + sz.xq_offset, *sfa = ws + sz.sfa_offset, *xo = ws + sz.xo_offset;
+    if (gamma) {
+        if (osc_status s = rmsnorm_quantize_impl(w, X, M, ldx, gamma, eps, xq, sfa, xo, st)) return s;
+    } else {
+        if (osc_status s = quantize_impl(w, X, M, ldx, xq, sfa, xo, nullptr, 0, st)) return s;
+    }
+    if (!swiglu_fused(w, M)) {
+        uint8_t* Y = ws + sz.workspace_bytes;
+        if (osc_status s = gemm_impl(w, xq, sfa, xo, M, Y, w->N, nullptr, 0, nullptr, 0, st)) return s;
+        cudaError_t e = launch_swiglu_fp8(false, Y, w->N, M, I, H, ldh, nullptr, nullptr, st);
+        if (e != cudaSuccess) return cuda_fail(e, "swiglu_fp8_kernel(activation only)");
+        return OSC_OK;
+    }
+    GemmArgs a;
+    memset(&a, 0, sizeof a);
+    if (osc_status s = make_tmap(&a.tm_a, xq, false, M, w->K / 2, w->K / 2, 128)) return s;
+    if (w->Kop > 0) {
+        if (osc_status s = make_tmap(&a.tm_ao, xo, true, M, (uint64_t)w->Kop * 2, (uint64_t)w->Kop * 2, 128)) return s;
+    }
+    a.tm_b = w->tm_b2[2];
+    a.tm_bo = w->tm_bo2[2];
+    a.tm_sfw = w->tm_sfw_gu;
+    if (osc_status s = make_tmap_sf(&a.tm_sfa, sfa, (uint64_t)((M + 127) / 128) * (w->K / 128))) return s;
+    // H as the store target: boxes of 32 columns x 16 rows, 64-byte swizzle (a staged row is 64 bytes)
+    if (osc_status s = encode_2d(&a.tm_y16, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, H, (uint64_t)I, (uint64_t)M, (uint64_t)ldh * 2, 32, 16,
+                                 CU_TENSOR_MAP_SWIZZLE_64B, "H")) return s;
+    a.tm_y = a.tm_y16;
+    a.sfa = sfa;
+    a.sfw = w->sfw;
+    a.Y = static_cast<uint16_t*>(H);
+    a.ldy = ldh;
+    a.M = M; a.N = w->N; a.K = w->K; a.Kop = w->Kop;
+    a.num_sms = w->num_sms;
+    cudaError_t e = launch_gemm_dual_pair_swiglu(a, st);
+    if (e != cudaSuccess) return cuda_fail(e, "gemm_pair_kernel(gate|up, swiglu)");
+    return OSC_OK;
+}
+
+osc_status osc_linear_swiglu(const osc_weights* w, const void* X, int M, int64_t ldx, void* H, int64_t ldh, void* workspace,
+                             size_t workspace_bytes, void* stream) {
+    return linear_swiglu_impl(w, X, M, ldx, nullptr, 0.0f, H, ldh, workspace, workspace_bytes, stream);
+}
+osc_status osc_rmsnorm_linear_swiglu(const osc_weights* w, const void* Hin, int M, int64_t ldh_in, const void* gamma, float eps,
+                                     void* H, int64_t ldh, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!gamma) return fail(OSC_ERR_INVALID_ARG, "gamma is null");
+    return linear_swiglu_impl(w, Hin, M, ldh_in, gamma, eps, H, ldh, workspace, workspace_bytes, stream);
 }
 
 osc_status osc_linear_grouped(const osc_weights* w, const void* X_perm, const int32_t* off, int M_total, int64_t ldx,

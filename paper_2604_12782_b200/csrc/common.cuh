@@ -127,6 +127,7 @@ int gemm_block_n(int row_tiles, int N, int num_sms, long* cost_ns = nullptr, int
 // gemm2_kernels.cu (CTA pairs: 256-row tiles, dense or grouped)
 cudaError_t launch_gemm_dual_pair(const GemmArgs& a, int bn, cudaStream_t st);
 cudaError_t launch_gemm_fp8_pair(const GemmArgs& a, int bn, cudaStream_t st);
+cudaError_t launch_gemm_dual_pair_swiglu(const GemmArgs& a, cudaStream_t st);
 cudaError_t launch_gemm_mxf8_pair(const GemmArgs& a, int bn, cudaStream_t st);
 cudaError_t launch_gemm_nvf4_pair(const GemmArgs& a, int bn, cudaStream_t st);
 int gemm_pair_block_n(bool fp8, bool allow_240, long row_tiles, int N, int stages, int num_sms, long* cost_ns = nullptr);
@@ -137,6 +138,6 @@ cudaError_t launch_gemm_fp8_decode(const GemmArgs& a, int S, cudaStream_t st);
 cudaError_t launch_gemm_mxf8_decode(const GemmArgs& a, int S, cudaStream_t st);
 cudaError_t launch_gemm_nvf4_decode(const GemmArgs& a, int S, cudaStream_t st);
 int gemm_decode_split(int N, int nkb, int num_sms);
-cudaError_t launch_retile_sf(const uint8_t* src, uint8_t* dst, int N, int K, int bn, cudaStream_t st);
+cudaError_t launch_retile_sf(const uint8_t* src, uint8_t* dst, int N, int K, int bn, cudaStream_t st, bool gate_up = false);
 
 }  // namespace osc

@@ -94,9 +94,25 @@ struct Cfg {
     static_assert(BN % 16 == 0 && BN <= 256 && (LAST_W == 64 || LAST_W == 48), "tile width");
 };
 
-template <int MODE, int BN>
-__global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(const __grid_constant__ GemmArgs args) {
+// GU (gate|up projection with the SwiGLU in the epilogue, dense MODE_OSC with per-tile weight scales only): the
+// weight matrix holds the gate rows [0, N/2) above the up rows [N/2, N).  A tile takes BN/2 gate features and the
+// same BN/2 up features - the leader CTA loads the gate half of the weight tile, its peer the up half, and the
+// per-tile copy of the weight scales is arranged the same way - so accumulator columns [0, BN/2) and [BN/2, BN)
+// hold gate and up of the same features, and the epilogue writes h = silu(gate) * up, BN/2 columns of
+// H [M, N/2], instead of BN columns of Y.  Both are rounded to bf16 first and combined by the arithmetic of
+// osc_swiglu, so H equals that call on this kernel's own Y bit for bit.
+// The activation costs ~37 instructions per element, and an epilogue of eight warps (two per scheduler) runs them
+// latency-bound, slower than the tile's K loop: the gate|up form has sixteen epilogue warps, one per 32-feature chunk
+// and TMEM lane quarter, each with a staging tile of 16 rows x 64 bytes (two store passes per chunk).
+__host__ __device__ constexpr int epi_warps(bool gu) { return gu ? 16 : EPI_WARPS; }
+__host__ __device__ constexpr int pair_threads(bool gu) { return 32 * (2 + epi_warps(gu)); }
+
+template <int MODE, int BN, bool GU = false>
+__global__ void __launch_bounds__(pair_threads(GU), 1) gemm_pair_kernel(const __grid_constant__ GemmArgs args) {
     using C = Cfg<MODE, BN>;
+    constexpr int EW = epi_warps(GU);
+    static_assert(!GU || (MODE == MODE_OSC && C::TILED_SF && (BN / 2) % 8 == 0 && BN / 2 <= 128 &&
+                          C::EPI_BYTES >= EW * 16 * 64), "gate|up epilogue: tile geometry");
     constexpr int STAGES = C::STAGES;
     constexpr int ACC = C::ACC_STAGES;
 
@@ -127,7 +143,7 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
         }
         for (int i = 0; i < ACC; ++i) {
             mbar_init(&tfull_bar[i], 1);
-            mbar_init(&tempty_bar[i], 2 * EPI_WARPS);
+            mbar_init(&tempty_bar[i], 2 * EW);
         }
         *abort_flag = 0;
         fence_barrier_init();
@@ -170,7 +186,8 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
     auto load_weights = [&](int s, int kb, int n0, int expert, bool expect) {
         const uint32_t st = smem_u32(smem + s * C::STAGE_BYTES);
         const uint32_t fb = map_to_cta(smem_u32(full_bar), 0) + (uint32_t)s * 8u;
-        const int brow = expert * N + n0 + (int)rank * (BN / 2);       // my half of the weight rows
+        // my half of the weight rows (gate|up: the leader's half are gate rows, the peer's the up rows of the same features)
+        const int brow = GU ? (int)rank * (N / 2) + (n0 / BN) * (BN / 2) : expert * N + n0 + (int)rank * (BN / 2);
         if (kb < nkb_a) {
             if (expect && rank == 0) mbar_arrive_expect_tx(&full_bar[s], C::SCALED ? C::TX_A : C::TX_B);
             tma_load_2d_pair(st + A_BYTES, &args.tm_b, fb, kb * ROW_BYTES, brow);
@@ -398,7 +415,8 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
         int acc = 0;
         uint32_t acc_ph = 0;
         const uint32_t tempty0 = map_to_cta(smem_u32(&tempty_bar[0]), 0);
-        uint8_t* stage_buf = smem + STAGES * C::STAGE_BYTES + (half * 4 + q) * (EPI_TILE_BYTES / C::EPI_HALVES);
+        uint8_t* stage_buf = smem + STAGES * C::STAGE_BYTES +
+                             (half * 4 + q) * (GU ? 16 * 64 : EPI_TILE_BYTES / C::EPI_HALVES);
         for (int t = pair_id; t < total; t += num_pairs) {
             const Tile ti = tile_of(t);
             const int n0 = ti.n0;
@@ -421,6 +439,80 @@ __global__ void __launch_bounds__(Cfg<MODE, BN>::THREADS, 1) gemm_pair_kernel(co
             }
             if (!wait_bounded(&tfull_bar[acc], acc_ph, abort_flag, 14)) goto done;
             tc_fence_after();
+            if (GU) {
+                // h = silu(gate) * up for the tile's BN/2 features in chunks of 32 (the last one narrower): this warp
+                // takes chunk `half` of its lane quarter.  Staging tile: 16 rows x 64 bytes with the 64-byte swizzle of
+                // the store's descriptor, two passes.
+                const int I = N >> 1;
+                const int f0 = (n0 / BN) * (BN / 2);
+                uint8_t* buf = stage_buf;
+                const int c0 = half * 32;                            // first feature of the chunk inside the tile
+                const int col = f0 + c0;                             // first column of the chunk in H
+                if (c0 < BN / 2) {
+                    const int wd = min(32, BN / 2 - c0);
+                    uint32_t rg[32], ru[32];
+                    const uint32_t tbase = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * C::ACC_STRIDE);
+                    tmem_ld_32x32(tbase + c0, rg);                   // (a narrow chunk reads past its columns: ignored below)
+                    tmem_ld_32x32(tbase + BN / 2 + c0, ru);
+                    tmem_ld_wait();
+                    if (col < I) {
+                        uint4 pk[4];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            uint32_t o[4];
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                const int x = j * 8 + 2 * i;
+                                // the projection's outputs as the unfused path stores them: bf16, nearest even
+                                const uint32_t g2 = bf162_bits(__floats2bfloat162_rn(__uint_as_float(rg[x]), __uint_as_float(rg[x + 1])));
+                                const uint32_t u2 = bf162_bits(__floats2bfloat162_rn(__uint_as_float(ru[x]), __uint_as_float(ru[x + 1])));
+                                const float2 h2 = swiglu32x2(make_float2(__uint_as_float(g2 << 16), __uint_as_float(g2 & 0xFFFF0000u)),
+                                                             make_float2(__uint_as_float(u2 << 16), __uint_as_float(u2 & 0xFFFF0000u)));
+                                o[i] = bf162_bits(__floats2bfloat162_rn(h2.x, h2.y));
+                            }
+                            pk[j] = make_uint4(o[0], o[1], o[2], o[3]);
+                        }
+#pragma unroll
+                        for (int hh = 0; hh < 2; ++hh) {
+                            if (lane == 0) tma_store_wait_read<0>();     // the staging tile must be free again
+                            __syncwarp();
+                            if ((lane >> 4) == hh) {
+                                const int rl = lane & 15;
+#pragma unroll
+                                for (int j = 0; j < 4; ++j)
+                                    *reinterpret_cast<uint4*>(buf + rl * 64 + ((j ^ ((rl >> 1) & 3)) << 4)) = pk[j];
+                            }
+                            fence_proxy_async_smem();
+                            __syncwarp();
+                            const int prow0 = wrow0 + hh * 16;
+                            if (wd == 32) {
+                                if (lane == 0) {
+                                    tma_store_2d_hint(&args.tm_y16, buf, col, prow0, y_policy);   // clipped at M rows, I columns
+                                    tma_store_commit();
+                                }
+                            } else {
+                                // the narrow last chunk is no store box (its neighbours belong to the next tile):
+                                // row-masked 16-byte stores from the staged tile
+                                const int j4 = lane & 3;
+#pragma unroll
+                                for (int rr = 0; rr < 2; ++rr) {
+                                    const int rl = rr * 8 + (lane >> 2);
+                                    if (prow0 + rl < args.M && j4 * 8 < wd && col + j4 * 8 < I)
+                                        *reinterpret_cast<uint4*>(args.Y + (int64_t)(prow0 + rl) * args.ldy + col + j4 * 8) =
+                                            *reinterpret_cast<const uint4*>(buf + rl * 64 + ((j4 ^ ((rl >> 1) & 3)) << 4));
+                                }
+                                __syncwarp();
+                            }
+                        }
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(tempty0 + (uint32_t)acc * 8u);
+                __syncwarp();
+                if (++acc == ACC) { acc = 0; acc_ph ^= 1u; }
+                continue;
+            }
             // grouped problems: rows past the expert's end belong to the next expert and must not be written,
             // so a warp whose 32 rows straddle the end writes its staged tiles with row-masked stores
             const bool clip = sched != nullptr && wrow0 + 32 > ti.row_end;
@@ -539,15 +631,15 @@ static int band_height(const GemmArgs& a) {
     return fit < 4 ? 4 : fit > 32 ? 32 : (int)fit;
 }
 
-template <int MODE, int BN>
+template <int MODE, int BN, bool GU = false>
 static cudaError_t launch_cfg(const GemmArgs& a, cudaStream_t st) {
     using C = Cfg<MODE, BN>;
     static PerDevice configured, resident;
-    if (cudaError_t e = opt_in_shared_memory(configured, gemm_pair_kernel<MODE, BN>, C::SMEM_BYTES)) return e;
+    if (cudaError_t e = opt_in_shared_memory(configured, gemm_pair_kernel<MODE, BN, GU>, C::SMEM_BYTES)) return e;
     const int total = a.sched2 ? a.num_sms : ((a.M + 2 * BM - 1) / (2 * BM)) * ((a.N + BN - 1) / BN);
     if (total <= 0) return cudaSuccess;
     cudaLaunchConfig_t cfg = {};
-    cfg.blockDim = dim3(C::THREADS);
+    cfg.blockDim = dim3(pair_threads(GU));
     cfg.dynamicSmemBytes = C::SMEM_BYTES;
     cfg.stream = st;
     cudaLaunchAttribute attr[2];
@@ -566,7 +658,7 @@ static cudaError_t launch_cfg(const GemmArgs& a, cudaStream_t st) {
     if (max_pairs == 0) {
         cfg.gridDim = dim3(a.num_sms);
         int n = 0;
-        cudaError_t e = cudaOccupancyMaxActiveClusters(&n, gemm_pair_kernel<MODE, BN>, &cfg);
+        cudaError_t e = cudaOccupancyMaxActiveClusters(&n, gemm_pair_kernel<MODE, BN, GU>, &cfg);
         if (e != cudaSuccess) return e;
         max_pairs = n > 0 ? n : 1;
         if (slot >= 0) { resident.value[slot] = max_pairs; resident.done[slot] = true; }
@@ -579,7 +671,7 @@ static cudaError_t launch_cfg(const GemmArgs& a, cudaStream_t st) {
     cfg.gridDim = dim3(2 * pairs);
     GemmArgs b = a;
     b.band = band_height<MODE>(a);
-    return cudaLaunchKernelEx(&cfg, gemm_pair_kernel<MODE, BN>, b);
+    return cudaLaunchKernelEx(&cfg, gemm_pair_kernel<MODE, BN, GU>, b);
 }
 
 }  // namespace pair
@@ -622,6 +714,11 @@ cudaError_t launch_gemm_dual_pair(const GemmArgs& a, int bn, cudaStream_t st) {
     if (bn == 192) return pair::launch_cfg<pair::MODE_OSC, 192>(a, st);
     if (bn == 240) return pair::launch_cfg<pair::MODE_OSC, 240>(a, st);
     return pair::launch_cfg<pair::MODE_OSC, 256>(a, st);
+}
+// gate|up projection with the SwiGLU in the epilogue: a.Y / a.ldy / a.tm_y describe H [M, N/2], a.tm_sfw the
+// gate|up arrangement of the per-tile weight scales
+cudaError_t launch_gemm_dual_pair_swiglu(const GemmArgs& a, cudaStream_t st) {
+    return pair::launch_cfg<pair::MODE_OSC, 240, true>(a, st);
 }
 cudaError_t launch_gemm_mxf8_pair(const GemmArgs& a, int bn, cudaStream_t st) {
     if (bn == 192) return pair::launch_cfg<pair::MODE_MXF8, 192>(a, st);

@@ -695,7 +695,9 @@ build_sched_kernel(const int32_t* __restrict__ off, int E, int32_t* __restrict__
 // dst holds, for every bn-row tile of the weight matrix, ceil(bn/128) 128-row scale blocks per
 // 128-channel block in which the tile's first row is row 0 (rows past the tile or past N: code 0).
 // Block order: [tile][block of the tile][K block]; inside a block the usual 512-byte arrangement.
-__global__ void retile_sf_kernel(const uint8_t* __restrict__ src, uint8_t* __restrict__ dst, int N, int K, int bn) {
+// gate_up: the matrix holds gate rows [0, N/2) above up rows [N/2, N) and tile t covers bn/2 gate features followed
+// by the same bn/2 up features: row j of the tile is matrix row t*bn/2 + j (j < bn/2) or N/2 + t*bn/2 + j - bn/2.
+__global__ void retile_sf_kernel(const uint8_t* __restrict__ src, uint8_t* __restrict__ dst, int N, int K, int bn, int gate_up) {
     const int katoms = K / 128;
     const int atoms_per_tile = (bn + 127) / 128;
     const int ntiles = (N + bn - 1) / bn;
@@ -708,19 +710,25 @@ __global__ void retile_sf_kernel(const uint8_t* __restrict__ src, uint8_t* __res
         const int tile = (int)(blk / ((int64_t)katoms * atoms_per_tile));
         const int r32 = byte >> 4, q = (byte >> 2) & 3, g4 = byte & 3;
         const int j = at * 128 + q * 32 + r32;  // row inside the tile
-        const int n = tile * bn + j;
+        int n = tile * bn + j;
+        bool valid = j < bn && n < N;
+        if (gate_up) {
+            const int hb = bn / 2, f = tile * hb + (j < hb ? j : j - hb);   // feature
+            n = (j < hb ? 0 : N / 2) + f;
+            valid = j < bn && f < N / 2;
+        }
         uint8_t v = 0;
-        if (j < bn && n < N)
+        if (valid)
             v = src[((int64_t)(n / 128) * katoms + ka) * 512 + (n % 32) * 16 + ((n % 128) / 32) * 4 + g4];
         dst[i] = v;
     }
 }
 
-cudaError_t launch_retile_sf(const uint8_t* src, uint8_t* dst, int N, int K, int bn, cudaStream_t st) {
+cudaError_t launch_retile_sf(const uint8_t* src, uint8_t* dst, int N, int K, int bn, cudaStream_t st, bool gate_up) {
     const int64_t total = (int64_t)((N + bn - 1) / bn) * ((bn + 127) / 128) * (K / 128) * 512;
     if (total <= 0) return cudaSuccess;
     const int blocks = (int)((total + 255) / 256 < 2048 ? (total + 255) / 256 : 2048);
-    retile_sf_kernel<<<blocks, 256, 0, st>>>(src, dst, N, K, bn);
+    retile_sf_kernel<<<blocks, 256, 0, st>>>(src, dst, N, K, bn, gate_up ? 1 : 0);
     return cudaGetLastError();
 }
 
