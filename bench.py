@@ -17,7 +17,8 @@ timing, as in the paper.
               basis), the quantizer's HBM fraction, the same build's FP8 W8A8 linear on the same shape, and
               extra.configs: one row per shape the benchmark configurations name (median and minimum of 30
               timed iterations, L2 cold and warm, % of the roofline on both bases, speed-up over the own FP8
-              linear on the same shape; shapes of up to 128 rows are replayed from a CUDA graph and say so)
+              linear on the same shape; every row is replayed from a CUDA graph and says so, with the median
+              of plain stream launches beside it)
 
 Between timed steps the buffers rotate over 4 independent sets (inputs, workspace,
 outputs and prepared weights: ~0.9 GB, 7x the L2), so no step finds its data in L2.
@@ -95,20 +96,25 @@ class ClockSampler:
         names = {"hw_slowdown": nv.nvmlClocksEventReasonHwSlowdown if hasattr(nv, "nvmlClocksEventReasonHwSlowdown") else 0x8,
                  "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20, "sw_power_cap": 0x4,
                  "hw_power_brake": 0x80}
+        n = 0
         while not self._stop.is_set():
             try:
+                # an NVML query takes about a millisecond: the clock every round, the reasons every fourth, no sleep in
+                # between, so that even a timed region of a few milliseconds gets more than one clock sample
                 self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
                 self.stamps.append(time.perf_counter())
-                try:
-                    r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
-                except Exception:
-                    r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
-                for k, bit in names.items():
-                    if r & bit:
-                        self.reasons.add(k)
+                n += 1
+                if n % 4 == 1:
+                    try:
+                        r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                    except Exception:
+                        r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                    for k, bit in names.items():
+                        if r & bit:
+                            self.reasons.add(k)
             except Exception:
-                pass
-            time.sleep(0.0004)
+                time.sleep(0.001)
+            time.sleep(0.00005)   # yields the interpreter lock to the launching thread
 
     def mark(self, name):
         """Remembers the host time of a boundary of the timed region."""
@@ -118,6 +124,9 @@ class ClockSampler:
         if self.nv:
             self._thread = threading.Thread(target=self._run, daemon=True)
             self._thread.start()
+            t_end = time.perf_counter() + 2.0      # the first query can take tens of milliseconds: wait for it, so
+            while not self.samples and time.perf_counter() < t_end:   # that the sampler is running when timing starts
+                time.sleep(0.001)
 
     def stop(self):
         self._stop.set()
@@ -403,11 +412,25 @@ def config_rows(torch, B, pk, iters=30, warm=5):
         a = np.asarray(ms_list) * 1e3
         return float(np.median(a)), float(a.min())
 
-    def measure(prob, few_rows):
-        gc = 2 * prob.n if few_rows else 0
+    def settle():
+        """A short idle gap in front of every measurement: rows that follow a long tensor-bound row otherwise inherit
+        its power-capped clock, and the same row read 60 us in one run and 80 us in the next."""
+        torch.cuda.synchronize()
+        time.sleep(0.2)
+
+    def measure(prob):
+        """Every row the same way: the calls captured once in a CUDA graph (2 x sets calls, rotating over the sets for
+        the cold regime, one set for the warm one) and one replay per timed iteration - device time without the
+        host's launch path, which paces few-row calls and adds 1-2 us per kernel boundary to the others.  The
+        median of the same calls launched one by one on the stream is reported beside it."""
+        gc = max(4, 2 * prob.n)
+        settle()
         cold = stats(per_call_times(torch, prob.step, iters, warm, gc))
+        settle()
         warm_ = stats(per_call_times(torch, lambda i: prob.step(0), iters, warm, gc))
-        return cold, warm_, ("cuda graph replay of %d calls per timed iteration" % gc) if few_rows else "%d consecutive calls per timed iteration" % CALLS_PER_ITERATION
+        settle()
+        plain = stats(per_call_times(torch, prob.step, iters, warm))
+        return cold, warm_, plain, "cuda graph replay of %d calls per timed iteration" % gc
 
     def osc_row(name, M, K, N, cpg, seed):
         case = synth.osc_linear_case_torch(torch, seed, M, K, N, cpg)
@@ -415,17 +438,19 @@ def config_rows(torch, B, pk, iters=30, warm=5):
         per_set = N * K / 2 + N * K / 32 + 2.0 * N * kop + 2.0 * M * K + roofline.osc_intermediate_bytes(M, K, kop) + 2.0 * M * N
         n = sets_for_cold_l2(torch, per_set)
         p = OscProblem(torch, B, case, n)
-        few = M <= 128
-        cold, warm_, how = measure(p, few)
+        cold, warm_, plain, how = measure(p)
         f8 = Fp8Problem(torch, B, case, sets_for_cold_l2(torch, N * K + 3.0 * M * K + 2.0 * M * N))
-        f8cold = stats(per_call_times(torch, f8.step, iters, warm, 2 * f8.n if few else 0))
+        settle()
+        f8cold = stats(per_call_times(torch, f8.step, iters, warm, max(4, 2 * f8.n)))
         B.osc_sync_check()
         f4, f16 = roofline.osc_flops(M, N, K, p.K_o)
         r_m, r_s = (roofline.osc_roofline_seconds(M, N, K, p.K_o, pkx) * 1e6 for pkx in (meas, sheet))
         rows.append({"name": name, "path": "osc", "M": M, "K": K, "N": N, "K_o": p.K_o, "timing": how, "sets": n,
                      "cold_us_median": cold[0], "cold_us_min": cold[1], "warm_us_median": warm_[0], "warm_us_min": warm_[1],
+                     "plain_launches_cold_us_median": plain[0], "plain_launches_cold_us_min": plain[1],
                      "tflops": (f4 + f16) / cold[0] / 1e6, "roof_us": r_m, "roof_us_datasheet": r_s,
                      "pct_roofline": 100.0 * r_m / cold[0], "pct_roofline_datasheet": 100.0 * r_s / cold[0],
+                     "pct_roofline_plain_launches": 100.0 * r_m / plain[0],
                      "fp8_cold_us_median": f8cold[0], "speedup_vs_fp8": f8cold[0] / cold[0]})
         del p, f8, case
         torch.cuda.empty_cache()
@@ -434,15 +459,16 @@ def config_rows(torch, B, pk, iters=30, warm=5):
         case = synth.fp8_linear_case_torch(torch, seed, M, K, N)
         n = sets_for_cold_l2(torch, N * K + 3.0 * M * K + 2.0 * M * N)
         p = Fp8Problem(torch, B, case, n)
-        few = M <= 128
-        cold, warm_, how = measure(p, few)
+        cold, warm_, plain, how = measure(p)
         B.osc_sync_check()
         r_m, r_s = (roofline.fp8_roofline_seconds(M, N, K, pkx) * 1e6 for pkx in (meas, sheet))
         rows.append({"name": name, "path": "fp8 fallback (is the own FP8 W8A8 linear)", "M": M, "K": K, "N": N, "timing": how,
                      "sets": n, "cold_us_median": cold[0], "cold_us_min": cold[1], "warm_us_median": warm_[0],
-                     "warm_us_min": warm_[1], "tflops": roofline.fp8_flops(M, N, K) / cold[0] / 1e6, "roof_us": r_m,
+                     "warm_us_min": warm_[1], "plain_launches_cold_us_median": plain[0], "plain_launches_cold_us_min": plain[1],
+                     "tflops": roofline.fp8_flops(M, N, K) / cold[0] / 1e6, "roof_us": r_m,
                      "roof_us_datasheet": r_s, "pct_roofline": 100.0 * r_m / cold[0],
-                     "pct_roofline_datasheet": 100.0 * r_s / cold[0], "fp8_cold_us_median": cold[0], "speedup_vs_fp8": 1.0})
+                     "pct_roofline_datasheet": 100.0 * r_s / cold[0], "pct_roofline_plain_launches": 100.0 * r_m / plain[0],
+                     "fp8_cold_us_median": cold[0], "speedup_vs_fp8": 1.0})
         del p, case
         torch.cuda.empty_cache()
 
@@ -470,17 +496,23 @@ def config_rows(torch, B, pk, iters=30, warm=5):
     w = B.osc_prepare_weights_grouped(Wg, c["lut"])
     ws = torch.empty(B.osc_act_sizes(w, Mt).workspace_bytes, dtype=torch.uint8, device="cuda")
     Y = torch.empty(Mt, N, dtype=torch.bfloat16, device="cuda")
-    t = stats(per_call_times(torch, lambda i: B.osc_linear_grouped(w, c["X"], off, Y, ws), iters, warm))
+    settle()
+    t = stats(per_call_times(torch, lambda i: B.osc_linear_grouped(w, c["X"], off, Y, ws), iters, warm, 4))
+    settle()
+    tp = stats(per_call_times(torch, lambda i: B.osc_linear_grouped(w, c["X"], off, Y, ws), iters, warm))
     w8 = B.osc_fp8_prepare_weights_grouped(Wg)
     ws8 = torch.empty(B.osc_fp8_act_sizes(w8, Mt).workspace_bytes, dtype=torch.uint8, device="cuda")
-    t8 = stats(per_call_times(torch, lambda i: B.osc_fp8_linear_grouped(w8, c["X"], off, Y, ws8), iters, warm))
+    settle()
+    t8 = stats(per_call_times(torch, lambda i: B.osc_fp8_linear_grouped(w8, c["X"], off, Y, ws8), iters, warm, 4))
     B.osc_sync_check()
     f4, f16 = roofline.osc_flops(Mt, N, K, w.K_o)
     byts = 2.0 * Mt * K + E * (N * K / 2 + N * K / 32 + 2.0 * N * w.K_o) + 2.0 * Mt * N
     r_m, r_s = (max(f4 / pkx["fp4"] + f16 / pkx["bf16"], byts / pkx["hbm"]) * 1e6 for pkx in (meas, sheet))
     rows.append({"name": "moe.gate_up(grouped)", "path": "osc", "M": Mt, "K": K, "N": N, "K_o": w.K_o, "E": E,
-                 "timing": "%d consecutive calls per timed iteration; one buffer set larger than the L2 (cold = warm)" % CALLS_PER_ITERATION, "sets": 1,
+                 "timing": "cuda graph replay of 4 calls per timed iteration; one buffer set larger than the L2 (cold = warm)", "sets": 1,
                  "cold_us_median": t[0], "cold_us_min": t[1], "warm_us_median": t[0], "warm_us_min": t[1],
+                 "plain_launches_cold_us_median": tp[0], "plain_launches_cold_us_min": tp[1],
+                 "pct_roofline_plain_launches": 100.0 * r_m / tp[0],
                  "tflops": (f4 + f16) / t[0] / 1e6, "roof_us": r_m, "roof_us_datasheet": r_s,
                  "pct_roofline": 100.0 * r_m / t[0], "pct_roofline_datasheet": 100.0 * r_s / t[0],
                  "fp8_cold_us_median": t8[0], "speedup_vs_fp8": t8[0] / t[0]})
@@ -492,13 +524,18 @@ def config_rows(torch, B, pk, iters=30, warm=5):
     w8 = B.osc_fp8_prepare_weights_grouped(Wg)
     ws8 = torch.empty(B.osc_fp8_act_sizes(w8, Mt).workspace_bytes, dtype=torch.uint8, device="cuda")
     Y = torch.empty(Mt, N, dtype=torch.bfloat16, device="cuda")
-    t = stats(per_call_times(torch, lambda i: B.osc_fp8_linear_grouped(w8, Xd, off, Y, ws8), iters, warm))
+    settle()
+    t = stats(per_call_times(torch, lambda i: B.osc_fp8_linear_grouped(w8, Xd, off, Y, ws8), iters, warm, 4))
+    settle()
+    tp = stats(per_call_times(torch, lambda i: B.osc_fp8_linear_grouped(w8, Xd, off, Y, ws8), iters, warm))
     B.osc_sync_check()
     byts = 2.0 * Mt * K + E * (N * K + 4.0 * N) + 2.0 * Mt * N
     r_m, r_s = (max(roofline.fp8_flops(Mt, N, K) / pkx["fp8"], byts / pkx["hbm"]) * 1e6 for pkx in (meas, sheet))
     rows.append({"name": "moe.down(grouped)", "path": "fp8 fallback (is the own FP8 W8A8 linear)", "M": Mt, "K": K, "N": N, "E": E,
-                 "timing": "%d consecutive calls per timed iteration; one buffer set larger than the L2 (cold = warm)" % CALLS_PER_ITERATION, "sets": 1,
+                 "timing": "cuda graph replay of 4 calls per timed iteration; one buffer set larger than the L2 (cold = warm)", "sets": 1,
                  "cold_us_median": t[0], "cold_us_min": t[1], "warm_us_median": t[0], "warm_us_min": t[1],
+                 "plain_launches_cold_us_median": tp[0], "plain_launches_cold_us_min": tp[1],
+                 "pct_roofline_plain_launches": 100.0 * r_m / tp[0],
                  "tflops": roofline.fp8_flops(Mt, N, K) / t[0] / 1e6, "roof_us": r_m, "roof_us_datasheet": r_s,
                  "pct_roofline": 100.0 * r_m / t[0], "pct_roofline_datasheet": 100.0 * r_s / t[0],
                  "fp8_cold_us_median": t[0], "speedup_vs_fp8": 1.0})

@@ -104,6 +104,8 @@ struct Cfg {
 // The activation costs ~37 instructions per element, and an epilogue of eight warps (two per scheduler) runs them
 // latency-bound, slower than the tile's K loop: the gate|up form has sixteen epilogue warps, one per 32-feature chunk
 // and TMEM lane quarter, each with a staging tile of 16 rows x 64 bytes (two store passes per chunk).
+// (Sixteen epilogue warps for the plain forms too were measured: 2-4 us slower per call on every shape - the epilogue
+// there is short, and the extra warps cost registers (96 instead of 150 per thread, spills) and staging passes.)
 __host__ __device__ constexpr int epi_warps(bool gu) { return gu ? 16 : EPI_WARPS; }
 __host__ __device__ constexpr int pair_threads(bool gu) { return 32 * (2 + epi_warps(gu)); }
 
@@ -415,8 +417,9 @@ __global__ void __launch_bounds__(pair_threads(GU), 1) gemm_pair_kernel(const __
         int acc = 0;
         uint32_t acc_ph = 0;
         const uint32_t tempty0 = map_to_cta(smem_u32(&tempty_bar[0]), 0);
-        uint8_t* stage_buf = smem + STAGES * C::STAGE_BYTES +
-                             (half * 4 + q) * (GU ? 16 * 64 : EPI_TILE_BYTES / C::EPI_HALVES);
+        // the staging area is shared out evenly: 32, 16 or 8 rows of 128 bytes per warp and pass
+        constexpr int WARP_STAGE_BYTES = GU ? 16 * 64 : C::EPI_BYTES / EW;
+        uint8_t* stage_buf = smem + STAGES * C::STAGE_BYTES + (half * 4 + q) * WARP_STAGE_BYTES;
         for (int t = pair_id; t < total; t += num_pairs) {
             const Tile ti = tile_of(t);
             const int n0 = ti.n0;
@@ -432,8 +435,8 @@ __global__ void __launch_bounds__(pair_threads(GU), 1) gemm_pair_kernel(const __
                 const float* swp = args.sw + (int64_t)ti.expert * N;
 #pragma unroll
                 for (int u = 0; u < 2; ++u) {
-                    const int col = n0 + (half + u * (EPI_WARPS / 4)) * 64 + 2 * lane;
-                    if (half + u * (EPI_WARPS / 4) < C::SLICES && col + 1 < N)
+                    const int col = n0 + (half + u * (EW / 4)) * 64 + 2 * lane;
+                    if (half + u * (EW / 4) < C::SLICES && col + 1 < N)
                         wsc[u] = *reinterpret_cast<const float2*>(swp + col);
                 }
             }
@@ -518,7 +521,7 @@ __global__ void __launch_bounds__(pair_threads(GU), 1) gemm_pair_kernel(const __
             const bool clip = sched != nullptr && wrow0 + 32 > ti.row_end;
             int ord = 0;
 #pragma unroll 1
-            for (int c = half; c < C::SLICES; c += EPI_WARPS / 4, ++ord) {
+            for (int c = half; c < C::SLICES; c += EW / 4, ++ord) {
                 uint32_t r0[32], r1[32];
                 const float2 wv = ord == 0 ? wsc[0] : wsc[1];
                 const uint32_t tcol = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * C::ACC_STRIDE + c * 64);
@@ -555,7 +558,8 @@ __global__ void __launch_bounds__(pair_threads(GU), 1) gemm_pair_kernel(const __
                         }
                         pk[j] = make_uint4(o[0], o[1], o[2], o[3]);
                     }
-                    constexpr int HV = C::EPI_HALVES, RPH = 32 / HV;   // staging passes per slice, rows per pass
+                    constexpr int RPH = WARP_STAGE_BYTES / 128, HV = 32 / RPH;   // rows per pass, staging passes per slice
+                    static_assert(GU || HV == 1 || HV == 2, "store boxes of 32 or 16 rows");
 #pragma unroll
                     for (int hh = 0; hh < HV; ++hh) {
                         if (lane == 0) tma_store_wait_read<0>();  // the one staging tile must be free again
