@@ -54,7 +54,7 @@ DATASHEET = {"bf16_tflops": 2250.0, "hbm_gbs": 8000.0}   # dense peaks and HBM3e
 def load_traffic():
     """DRAM bytes (read + written) of one launch of the dominant kernel on the bench workload, from the one ncu
     capture whose numbers are kept under profiles/ together with the commit and the command they came from."""
-    path = os.path.join(ROOT, "profiles", "dominant_kernel_traffic.json")
+    path = os.path.join(ROOT, "profiles", "dominant_kernel_traffic.txt")
     try:
         with open(path) as f:
             t = json.load(f)
