@@ -159,12 +159,9 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
     tc_fence_after();
     const uint32_t tmem_base = __shfl_sync(0xFFFFFFFFu, *tmem_slot, 0);
     grid_launch_dependents();
-    grid_dependency_wait();   // operands (and the grouped schedule) come from the kernels before this one
 
     const int N = args.N, K = args.K;
-    const int num_m = num_row_tiles(args);
     const int num_n = (N + BN - 1) / BN;
-    const int total = num_m * num_n;
     // K blocks: Path A / FP8 first, then Path B
     const int elems_per_kb = C::DUAL ? 256 : 128;
     const int nkb_a = (K + elems_per_kb - 1) / elems_per_kb;
@@ -174,44 +171,78 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
     const int natoms = (N + 127) / 128;  // 128-row scale blocks of one expert's weights
     constexpr int KA = C::KA;
 
+    // One stage of the ring in two parts: the weight side (prepared once, never written by a kernel of the calling
+    // sequence) and the activation side (the quantizer's output).  `expect` arms the stage's barrier with the bytes of both.
+    auto load_weights = [&](int s, int kb, const TileInfo& ti, bool expect) {
+        uint8_t* st = smem + s * C::STAGE_BYTES;
+        const int brow = ti.expert * N + ti.n0;
+        if (kb < nkb_a) {
+            const uint32_t sfb = C::SCALED ? (uint32_t)min(KA, katoms_total - KA * kb) * 512u : 0u;   // scale bytes per row block
+            if (expect) mbar_arrive_expect_tx(&full_bar[s], A_BYTES + C::B_BYTES + sfb * (1 + C::SFB_ATOMS));
+            tma_load_2d(st + A_BYTES, &args.tm_b, &full_bar[s], kb * ROW_BYTES, brow);
+            if (C::SCALED) {
+#pragma unroll
+                for (int j = 0; j < C::SFB_ATOMS; ++j) {
+                    const int atom = min(ti.n0 / 128 + j, natoms - 1);
+                    const uint8_t* sw = args.sfw + (((int64_t)ti.expert * natoms + atom) * katoms_total + KA * kb) * 512;
+                    bulk_load(st + A_BYTES + C::B_BYTES + C::SFA_BYTES + j * C::SF_ROWBLOCK, sw, sfb, &full_bar[s]);
+                }
+            }
+        } else {
+            if (expect) mbar_arrive_expect_tx(&full_bar[s], A_BYTES + C::B_BYTES);
+            tma_load_2d(st + A_BYTES, &args.tm_bo, &full_bar[s], (kb - nkb_a) * 64, brow);
+        }
+    };
+    auto load_activations = [&](int s, int kb, const TileInfo& ti) {
+        uint8_t* st = smem + s * C::STAGE_BYTES;
+        if (kb < nkb_a) {
+            tma_load_2d(st, &args.tm_a, &full_bar[s], kb * ROW_BYTES, ti.row0);
+            if (C::SCALED) {
+                const uint32_t sfb = (uint32_t)min(KA, katoms_total - KA * kb) * 512u;
+                const uint8_t* sa = args.sfa + ((int64_t)(ti.sf_row0 / 128) * katoms_total + KA * kb) * 512;
+                bulk_load(st + A_BYTES + C::B_BYTES, sa, sfb, &full_bar[s]);
+            }
+        } else {
+            tma_load_2d(st, &args.tm_ao, &full_bar[s], (kb - nkb_a) * 64, ti.row0);
+        }
+    };
+
+    // Dense problems: the weight side of the first tile's first ring of stages goes out BEFORE the dependency wait (the
+    // CTA is resident while the quantizer in front still runs, and the weights do not depend on it); a grouped problem
+    // reads its tiles from the schedule that the kernel in front builds, so nothing is known before the wait.
+    const int num_m_dense = (args.M + BM - 1) / BM;
+    const int pre = (args.sched == nullptr && warp == 0 && (int)blockIdx.x < num_m_dense * num_n) ? min(STAGES, nkb) : 0;
+    if (pre > 0) {
+        const TileInfo ti = tile_info<BN>(args, blockIdx.x, num_m_dense, num_n);
+        if (elect_one()) {
+            for (int kb = 0; kb < pre; ++kb) load_weights(kb, kb, ti, true);
+        }
+        __syncwarp();
+    }
+    grid_dependency_wait();   // activations (and the grouped schedule) come from the kernels before this one
+
+    const int num_m = num_row_tiles(args);
+    const int total = num_m * num_n;
+
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
         int s = 0;
         uint32_t ph = 0;
+        if (pre > 0) {   // the activation side of the stages whose weight side is already under way
+            const TileInfo ti = tile_info<BN>(args, blockIdx.x, num_m, num_n);
+            if (elect_one()) {
+                for (int kb = 0; kb < pre; ++kb) load_activations(kb, kb, ti);
+            }
+            __syncwarp();
+            if (pre == STAGES) ph = 1u; else s = pre;
+        }
         for (int t = blockIdx.x; t < total; t += gridDim.x) {
             const TileInfo ti = tile_info<BN>(args, t, num_m, num_n);
-            const int brow = ti.expert * N + ti.n0;
-            for (int kb = 0; kb < nkb; ++kb) {
+            for (int kb = (t == (int)blockIdx.x ? pre : 0); kb < nkb; ++kb) {
                 if (!wait_bounded(&empty_bar[s], ph ^ 1u, abort_flag, 1)) goto done;
-                uint8_t* st = smem + s * C::STAGE_BYTES;
                 if (elect_one()) {
-                    if (kb < nkb_a) {
-                        if (C::SCALED) {
-                            const int ka = min(KA, katoms_total - KA * kb);  // 128-channel scale blocks in this stage
-                            const uint32_t sfb = (uint32_t)ka * 512u;
-                            mbar_arrive_expect_tx(&full_bar[s], A_BYTES + C::B_BYTES + sfb * (1 + C::SFB_ATOMS));
-                            tma_load_2d(st, &args.tm_a, &full_bar[s], kb * ROW_BYTES, ti.row0);
-                            tma_load_2d(st + A_BYTES, &args.tm_b, &full_bar[s], kb * ROW_BYTES, brow);
-                            const uint8_t* sa = args.sfa + ((int64_t)(ti.sf_row0 / 128) * katoms_total + KA * kb) * 512;
-                            bulk_load(st + A_BYTES + C::B_BYTES, sa, sfb, &full_bar[s]);
-#pragma unroll
-                            for (int j = 0; j < C::SFB_ATOMS; ++j) {
-                                const int atom = min(ti.n0 / 128 + j, natoms - 1);
-                                const uint8_t* sw = args.sfw +
-                                    (((int64_t)ti.expert * natoms + atom) * katoms_total + KA * kb) * 512;
-                                bulk_load(st + A_BYTES + C::B_BYTES + C::SFA_BYTES + j * C::SF_ROWBLOCK, sw, sfb, &full_bar[s]);
-                            }
-                        } else {
-                            mbar_arrive_expect_tx(&full_bar[s], A_BYTES + C::B_BYTES);
-                            tma_load_2d(st, &args.tm_a, &full_bar[s], kb * ROW_BYTES, ti.row0);
-                            tma_load_2d(st + A_BYTES, &args.tm_b, &full_bar[s], kb * ROW_BYTES, brow);
-                        }
-                    } else {
-                        const int kk = kb - nkb_a;
-                        mbar_arrive_expect_tx(&full_bar[s], A_BYTES + C::B_BYTES);
-                        tma_load_2d(st, &args.tm_ao, &full_bar[s], kk * 64, ti.row0);
-                        tma_load_2d(st + A_BYTES, &args.tm_bo, &full_bar[s], kk * 64, brow);
-                    }
+                    load_weights(s, kb, ti, true);
+                    load_activations(s, kb, ti);
                 }
                 __syncwarp();
                 if (++s == STAGES) { s = 0; ph ^= 1u; }
