@@ -1182,6 +1182,8 @@ def run_sweep(args):
                  "tflops": (f4 + f16) / ms4 / 1e9, "vs_mxfp4": ms4 / ms})
     del w4, ws4
     wg, Yg = w, Y
+    wgu = B.osc_prepare_weights_gate_up_grouped(Wd, c["lut"])     # the same experts with the SwiGLU in the epilogue
+    wsgu = torch.empty(B.osc_swiglu_gather_workspace_bytes(wgu, T_tok, Mt), dtype=torch.uint8, device="cuda")
     del Xd, Wd, ws
     c = synth.moe_down_case(E, counts, weight_pool=8)
     Xd = dev_bf16(torch, c["X"])
@@ -1214,11 +1216,18 @@ def run_sweep(args):
         B.osc_swiglu(Yg, K, Hh)
         B.osc_fp8_linear_grouped(w, Hh, off, Y, ws)
 
+    def moe_fused_epilogue(i):
+        B.osc_rmsnorm_linear_swiglu_grouped_gather(wgu, Xtok, gamma, 1e-6, row_token, off, Hh, wsgu)
+        B.osc_fp8_linear_grouped(w, Hh, off, Y, ws)
+
     ms_f, ms_s = time_loop(torch, moe_fused, steps, warm), time_loop(torch, moe_separate, steps, warm)
+    ms_e = time_loop(torch, moe_fused_epilogue, steps, warm)
     B.osc_sync_check()
     rows.append({"name": "moe.layer.fused(rmsnorm+gather+gate_up, swiglu+down_fp8)", "M": Mt, "ms": ms_f,
                  "separate_kernels_ms": ms_s, "speedup": ms_s / ms_f})
-    del w, ws, wg, Yg, wsg, Xtok, Xn, Hh
+    rows.append({"name": "moe.layer.fused_epilogue(rmsnorm+gather+gate_up+swiglu, down_fp8)", "M": Mt, "ms": ms_e,
+                 "separate_kernels_ms": ms_s, "speedup": ms_s / ms_e})
+    del w, ws, wg, wgu, wsgu, Yg, wsg, Xtok, Xn, Hh
     w = B.osc_mxfp8_prepare_weights_grouped(Wd)
     sz = B.osc_mxfp8_act_sizes(w, c["M"])
     ws = torch.empty(sz.workspace_bytes, dtype=torch.uint8, device="cuda")

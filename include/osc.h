@@ -352,6 +352,28 @@ osc_status osc_linear_swiglu(const osc_weights* w, const void* X, int M, int64_t
                              size_t workspace_bytes, void* stream);
 osc_status osc_rmsnorm_linear_swiglu(const osc_weights* w, const void* Hin, int M, int64_t ldh_in, const void* gamma, float eps,
                                      void* H, int64_t ldh, void* workspace, size_t workspace_bytes, void* stream);
+/* Grouped (MoE) forms: E experts' gate|up matrices stacked as W[E][2I][K]; one table for the layer.
+ *   osc_gate_up_weight_sizes_grouped / osc_prepare_weights_gate_up_grouped: as osc_prepare_weights_grouped with N = 2I, meta
+ *        additionally holding every expert's per-tile scale copy in gate|up order.  The handle also serves
+ *        osc_linear_grouped and osc_linear_grouped_gather (the plain [M_total, 2I] projection).
+ *   osc_linear_swiglu_grouped: rows of X_perm sorted by expert, off as in osc_linear_grouped; H dev bf16 [M_total, ldh].
+ *        Workspace: osc_linear_swiglu_workspace_bytes(w, M_total).  Experts of fewer than 96 rows on average run the plain
+ *        grouped projection into a scratch behind the workspace and the stand-alone activation.
+ *   osc_linear_swiglu_grouped_gather / osc_rmsnorm_linear_swiglu_grouped_gather: the dispatch fused behind the quantizer
+ *        (as osc_linear_grouped_gather / osc_rmsnorm_linear_grouped_gather); workspace: osc_swiglu_gather_workspace_bytes.
+ *   Per expert the result equals the dense call on that expert's rows and weights bit for bit. */
+osc_status osc_gate_up_weight_sizes_grouped(int E, int I, int K, const int8_t* lut, int lut_c, osc_weight_sizes_t* out);
+osc_status osc_prepare_weights_gate_up_grouped(const void* W, int E, int I, int K, const int8_t* lut, int lut_c, void* wq,
+                                               void* sfw, void* wo, void* meta, void* stream, osc_weights** out);
+osc_status osc_linear_swiglu_grouped(const osc_weights* w, const void* X_perm, const int32_t* off, int M_total, int64_t ldx,
+                                     void* H, int64_t ldh, void* workspace, size_t workspace_bytes, void* stream);
+osc_status osc_swiglu_gather_workspace_bytes(const osc_weights* w, int T, int M_total, size_t* bytes);
+osc_status osc_linear_swiglu_grouped_gather(const osc_weights* w, const void* X, int T, int64_t ldx, const int32_t* row_token,
+                                            const int32_t* off, int M_total, void* H, int64_t ldh, void* workspace,
+                                            size_t workspace_bytes, void* stream);
+osc_status osc_rmsnorm_linear_swiglu_grouped_gather(const osc_weights* w, const void* Hin, int T, int64_t ldh_in, const void* gamma,
+                                                    float eps, const int32_t* row_token, const int32_t* off, int M_total, void* H,
+                                                    int64_t ldh, void* workspace, size_t workspace_bytes, void* stream);
 
 /* ------------------------------------- MXFP8 form of the fallback (Section 3.4) */
 

@@ -118,6 +118,12 @@ _SIGS = {
     "osc_linear_swiglu_workspace_bytes": (_i, [_vp, _i, C.POINTER(_sz)]),
     "osc_linear_swiglu": (_i, [_vp, _vp, _i, _i64, _vp, _i64, _vp, _sz, _vp]),
     "osc_rmsnorm_linear_swiglu": (_i, [_vp, _vp, _i, _i64, _vp, C.c_float, _vp, _i64, _vp, _sz, _vp]),
+    "osc_gate_up_weight_sizes_grouped": (_i, [_i, _i, _i, _vp, _i, C.POINTER(WeightSizes)]),
+    "osc_prepare_weights_gate_up_grouped": (_i, [_vp, _i, _i, _i, _vp, _i, _vp, _vp, _vp, _vp, _vp, C.POINTER(_vp)]),
+    "osc_linear_swiglu_grouped": (_i, [_vp, _vp, _vp, _i, _i64, _vp, _i64, _vp, _sz, _vp]),
+    "osc_swiglu_gather_workspace_bytes": (_i, [_vp, _i, _i, C.POINTER(_sz)]),
+    "osc_linear_swiglu_grouped_gather": (_i, [_vp, _vp, _i, _i64, _vp, _vp, _i, _vp, _i64, _vp, _sz, _vp]),
+    "osc_rmsnorm_linear_swiglu_grouped_gather": (_i, [_vp, _vp, _i, _i64, _vp, C.c_float, _vp, _vp, _i, _vp, _i64, _vp, _sz, _vp]),
     "osc_nvfp4_rmsnorm_quantize_extract": (_i, [_vp, _vp, _i, _i64, _vp, C.c_float, _i, _vp, _vp, _vp, _vp]),
     "osc_nvfp4_rmsnorm_linear": (_i, [_vp, _vp, _i, _i64, _vp, C.c_float, _i, _vp, _i64, _vp, _sz, _vp]),
     "osc_nvfp4_gather_workspace_bytes": (_i, [_vp, _i, _i, C.POINTER(_sz)]),
@@ -740,3 +746,52 @@ def osc_rmsnorm_linear_swiglu(w: OscWeights, Hin: torch.Tensor, gamma: torch.Ten
     _check(_lib.osc_rmsnorm_linear_swiglu(w.ptr, _ptr(Hin), M, Hin.stride(0) if M else w.K, _ptr(gamma), float(eps), _ptr(H),
                                           H.stride(0) if M else w.N // 2, _ptr(workspace),
                                           workspace.numel() * workspace.element_size(), _stream(stream)))
+
+
+def osc_prepare_weights_gate_up_grouped(W: torch.Tensor, lut, stream=None) -> OscWeights:
+    """W: cuda bf16 [E, 2I, K] contiguous, every expert's gate rows above its up rows."""
+    E, N, K = W.shape
+    assert W.is_contiguous()
+    lut = _lut(lut)
+    sz = WeightSizes()
+    _check(_lib.osc_gate_up_weight_sizes_grouped(E, N // 2, K, lut.ctypes.data, lut.shape[1], C.byref(sz)))
+    bufs = {k: _alloc(getattr(sz, k + "_bytes"), W.device) for k in ("wq", "sfw", "wo", "meta")}
+    h = _vp()
+    _check(_lib.osc_prepare_weights_gate_up_grouped(_ptr(W), E, N // 2, K, lut.ctypes.data, lut.shape[1], _ptr(bufs["wq"]),
+                                                    _ptr(bufs["sfw"]), _ptr(bufs["wo"]) if sz.wo_bytes else None,
+                                                    _ptr(bufs["meta"]), _stream(stream), C.byref(h)))
+    w = OscWeights(h.value, bufs)
+    w.E, w.N, w.K, w.K_o, w.K_o_pad, w.sizes = E, N, K, sz.K_o, sz.K_o_pad, sz
+    return w
+
+
+def osc_linear_swiglu_grouped(w: OscWeights, X: torch.Tensor, off: torch.Tensor, H: torch.Tensor, workspace: torch.Tensor,
+                              stream=None):
+    M = X.shape[0]
+    _check(_lib.osc_linear_swiglu_grouped(w.ptr, _ptr(X), _ptr(off), M, X.stride(0) if M else w.K, _ptr(H),
+                                          H.stride(0) if M else w.N // 2, _ptr(workspace),
+                                          workspace.numel() * workspace.element_size(), _stream(stream)))
+
+
+def osc_swiglu_gather_workspace_bytes(w: OscWeights, T: int, M_total: int) -> int:
+    out = _sz()
+    _check(_lib.osc_swiglu_gather_workspace_bytes(w.ptr, T, M_total, C.byref(out)))
+    return int(out.value)
+
+
+def osc_linear_swiglu_grouped_gather(w: OscWeights, X: torch.Tensor, row_token: torch.Tensor, off: torch.Tensor, H: torch.Tensor,
+                                     workspace: torch.Tensor, stream=None):
+    T, M = X.shape[0], row_token.shape[0]
+    _check(_lib.osc_linear_swiglu_grouped_gather(w.ptr, _ptr(X), T, X.stride(0) if T else w.K, _ptr(row_token), _ptr(off), M,
+                                                 _ptr(H), H.stride(0) if M else w.N // 2, _ptr(workspace),
+                                                 workspace.numel() * workspace.element_size(), _stream(stream)))
+
+
+def osc_rmsnorm_linear_swiglu_grouped_gather(w: OscWeights, Hin: torch.Tensor, gamma: torch.Tensor, eps: float,
+                                             row_token: torch.Tensor, off: torch.Tensor, H: torch.Tensor, workspace: torch.Tensor,
+                                             stream=None):
+    T, M = Hin.shape[0], row_token.shape[0]
+    _check(_lib.osc_rmsnorm_linear_swiglu_grouped_gather(w.ptr, _ptr(Hin), T, Hin.stride(0) if T else w.K, _ptr(gamma),
+                                                         float(eps), _ptr(row_token), _ptr(off), M, _ptr(H),
+                                                         H.stride(0) if M else w.N // 2, _ptr(workspace),
+                                                         workspace.numel() * workspace.element_size(), _stream(stream)))

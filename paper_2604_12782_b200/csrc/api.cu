@@ -386,7 +386,7 @@ static osc_status prepare_impl(const void* W, int E, int N, int K, int64_t ldw, 
             s = make_tmap(&w->tm_bo[v], wo, true, (uint64_t)E * N, (uint64_t)t.Kop * 2, (uint64_t)t.Kop * 2, 64 * (v + 1));
     }
     for (int v = 0; v < 3 && s == OSC_OK; ++v) {
-        if (grouped && v == 2) break;  // the per-tile scale copy exists for dense weights only
+        if (grouped && v == 2 && !gate_up) break;  // 240-wide tiles need a per-tile scale copy: dense weights, or gate|up
         const int half = (v == 0 ? 192 : v == 1 ? 256 : kTiledBN) / 2;
         s = make_tmap(&w->tm_b2[v], wq, false, (uint64_t)E * N, K / 2, K / 2, half);
         if (s == OSC_OK && t.Kop > 0)
@@ -405,6 +405,15 @@ static osc_status prepare_impl(const void* W, int E, int N, int K, int64_t ldw, 
             s = make_tmap_sf(&w->tm_sfw_gu, tiled_gu, (uint64_t)tiled_sf_bytes(N, K) / 512);
             w->gate_up = true;
         }
+    } else if (s == OSC_OK && gate_up) {   // grouped gate|up: one gate|up-ordered per-tile copy per expert, behind the table
+        uint8_t* tiled_gu = m8 + tiled_off;
+        const size_t per = tiled_sf_bytes(N, K);
+        for (int x = 0; x < E; ++x) {
+            e = launch_retile_sf(static_cast<const uint8_t*>(sfw) + (size_t)x * sfw_e, tiled_gu + (size_t)x * per, N, K, kTiledBN, st, true);
+            if (e != cudaSuccess) { delete w; return cuda_fail(e, "retile_sf_kernel(gate|up, grouped)"); }
+        }
+        s = make_tmap_sf(&w->tm_sfw_gu, tiled_gu, (uint64_t)E * per / 512);
+        w->gate_up = true;
     }
     if (s == OSC_OK && (e = launch_prepare_fence(st)) != cudaSuccess) s = cuda_fail(e, "prepare_fence_kernel");
     if (s != OSC_OK) { delete w; return s; }
@@ -431,6 +440,17 @@ osc_status osc_prepare_weights_gate_up(const void* W, int I, int K, int64_t ldw,
                                        void* sfw, void* wo, void* meta, void* stream, osc_weights** out) {
     if (I <= 0 || I % 64 || I > (1 << 29)) return fail(OSC_ERR_SHAPE, "I = %d must be a positive multiple of 64", I);
     return prepare_impl(W, 1, 2 * I, K, ldw, lut, lut_c, wq, sfw, wo, meta, stream, false, out, false, true);
+}
+osc_status osc_gate_up_weight_sizes_grouped(int E, int I, int K, const int8_t* lut, int lut_c, osc_weight_sizes_t* out) {
+    if (I <= 0 || I % 64 || I > (1 << 29)) return fail(OSC_ERR_SHAPE, "I = %d must be a positive multiple of 64", I);
+    if (osc_status s = osc_weight_sizes(E, 2 * I, K, lut, lut_c, out)) return s;
+    out->meta_bytes = meta_table_bytes(K, out->K_o) + (size_t)E * tiled_sf_bytes(2 * I, K);
+    return OSC_OK;
+}
+osc_status osc_prepare_weights_gate_up_grouped(const void* W, int E, int I, int K, const int8_t* lut, int lut_c, void* wq,
+                                               void* sfw, void* wo, void* meta, void* stream, osc_weights** out) {
+    if (I <= 0 || I % 64 || I > (1 << 29)) return fail(OSC_ERR_SHAPE, "I = %d must be a positive multiple of 64", I);
+    return prepare_impl(W, E, 2 * I, K, K, lut, lut_c, wq, sfw, wo, meta, stream, true, out, false, true);
 }
 
 osc_status osc_weights_destroy(osc_weights* w) {
@@ -711,7 +731,8 @@ osc_status osc_add_rmsnorm_linear(const osc_weights* w, const void* H, const voi
 constexpr int kSwigluFusedMinRows = 256;
 static bool swiglu_fused(const osc_weights* w, int M) {
     static const int mode = [] { const char* e = getenv("OSC_SWIGLU_FUSED"); return e ? atoi(e) : 1; }();
-    return mode != 0 && M > kSwigluFusedMinRows && (w->N / 2) % 8 == 0;
+    if (mode == 0 || (w->N / 2) % 8) return false;
+    return w->grouped ? use_pair_kernel(true, M, w->E) : M > kSwigluFusedMinRows;   // grouped: experts of 96 rows and more on average
 }
 
 osc_status osc_linear_swiglu_workspace_bytes(const osc_weights* w, int M, size_t* bytes) {
@@ -723,33 +744,15 @@ osc_status osc_linear_swiglu_workspace_bytes(const osc_weights* w, int M, size_t
     return OSC_OK;
 }
 
-static osc_status linear_swiglu_impl(const osc_weights* w, const void* X, int M, int64_t ldx, const void* gamma, float eps,
-                                     void* H, int64_t ldh, void* workspace, size_t workspace_bytes, void* stream) {
-    if (osc_status s = check_act(w, X, M, ldx)) return s;
-    if (!w->gate_up) return fail(OSC_ERR_INVALID_ARG, "not a gate|up handle: use osc_prepare_weights_gate_up");
-    if (M == 0) return OSC_OK;
+// The dual-path GEMM of a gate|up handle with the activation applied to its output: in the epilogue of the pair kernel's
+// gate|up form where that runs, else the plain GEMM into `scratch_y` [M, N] and the stand-alone activation.
+static osc_status gemm_swiglu_impl(const osc_weights* w, uint8_t* xq, uint8_t* sfa, uint8_t* xo, int M, void* H, int64_t ldh,
+                                   const int32_t* sched, int max_tiles, const int32_t* sched2, int max_tiles2, uint8_t* scratch_y,
+                                   cudaStream_t st) {
     const int I = w->N / 2;
-    osc_act_sizes_t sz;
-    osc_act_sizes(w, M, &sz);
-    size_t need = 0;
-    osc_linear_swiglu_workspace_bytes(w, M, &need);
-    if (!workspace || !aligned16(workspace)) return fail(OSC_ERR_ALIGN, "workspace must be non-null and 16-byte aligned");
-    if (workspace_bytes < need) return fail(OSC_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", workspace_bytes, need);
-    if (!H) return fail(OSC_ERR_INVALID_ARG, "H is null");
-    if (ldh < I) return fail(OSC_ERR_SHAPE, "ldh = %lld < I = %d", (long long)ldh, I);
-    if (ldh % 8 || !aligned16(H)) return fail(OSC_ERR_ALIGN, "H must be 16-byte aligned and ldh a multiple of 8");
-    uint8_t* ws = static_cast<uint8_t*>(workspace);
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    uint8_t *xq = ws + sz.xq_offset, *sfa = ws + sz.sfa_offset, *xo = ws + sz.xo_offset;
-    if (gamma) {
-        if (osc_status s = rmsnorm_quantize_impl(w, X, M, ldx, gamma, eps, xq, sfa, xo, st)) return s;
-    } else {
-        if (osc_status s = quantize_impl(w, X, M, ldx, xq, sfa, xo, nullptr, 0, st)) return s;
-    }
     if (!swiglu_fused(w, M)) {
-        uint8_t* Y = ws + sz.workspace_bytes;
-        if (osc_status s = gemm_impl(w, xq, sfa, xo, M, Y, w->N, nullptr, 0, nullptr, 0, st)) return s;
-        cudaError_t e = launch_swiglu_fp8(false, Y, w->N, M, I, H, ldh, nullptr, nullptr, st);
+        if (osc_status s = gemm_impl(w, xq, sfa, xo, M, scratch_y, w->N, sched, max_tiles, sched2, max_tiles2, st)) return s;
+        cudaError_t e = launch_swiglu_fp8(false, scratch_y, w->N, M, I, H, ldh, nullptr, nullptr, st);
         if (e != cudaSuccess) return cuda_fail(e, "swiglu_fp8_kernel(activation only)");
         return OSC_OK;
     }
@@ -762,7 +765,8 @@ static osc_status linear_swiglu_impl(const osc_weights* w, const void* X, int M,
     a.tm_b = w->tm_b2[2];
     a.tm_bo = w->tm_bo2[2];
     a.tm_sfw = w->tm_sfw_gu;
-    if (osc_status s = make_tmap_sf(&a.tm_sfa, sfa, (uint64_t)((M + 127) / 128) * (w->K / 128))) return s;
+    const uint64_t sf_row_blocks = w->grouped ? (uint64_t)max_tiles : (uint64_t)((M + 127) / 128);
+    if (osc_status s = make_tmap_sf(&a.tm_sfa, sfa, sf_row_blocks * (w->K / 128))) return s;
     // H as the store target: boxes of 32 columns x 16 rows, 64-byte swizzle (a staged row is 64 bytes)
     if (osc_status s = encode_2d(&a.tm_y16, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, H, (uint64_t)I, (uint64_t)M, (uint64_t)ldh * 2, 32, 16,
                                  CU_TENSOR_MAP_SWIZZLE_64B, "H")) return s;
@@ -773,9 +777,43 @@ static osc_status linear_swiglu_impl(const osc_weights* w, const void* X, int M,
     a.ldy = ldh;
     a.M = M; a.N = w->N; a.K = w->K; a.Kop = w->Kop;
     a.num_sms = w->num_sms;
+    a.sched = sched; a.max_tiles = max_tiles;
+    a.sched2 = sched2; a.max_tiles2 = max_tiles2;
     cudaError_t e = launch_gemm_dual_pair_swiglu(a, st);
     if (e != cudaSuccess) return cuda_fail(e, "gemm_pair_kernel(gate|up, swiglu)");
     return OSC_OK;
+}
+
+static osc_status check_h(const osc_weights* w, const void* H, int64_t ldh) {
+    const int I = w->N / 2;
+    if (!H) return fail(OSC_ERR_INVALID_ARG, "H is null");
+    if (ldh < I) return fail(OSC_ERR_SHAPE, "ldh = %lld < I = %d", (long long)ldh, I);
+    if (ldh % 8 || !aligned16(H)) return fail(OSC_ERR_ALIGN, "H must be 16-byte aligned and ldh a multiple of 8");
+    return OSC_OK;
+}
+
+static osc_status linear_swiglu_impl(const osc_weights* w, const void* X, int M, int64_t ldx, const void* gamma, float eps,
+                                     void* H, int64_t ldh, void* workspace, size_t workspace_bytes, void* stream) {
+    if (osc_status s = check_act(w, X, M, ldx)) return s;
+    if (!w->gate_up) return fail(OSC_ERR_INVALID_ARG, "not a gate|up handle: use osc_prepare_weights_gate_up");
+    if (w->grouped) return fail(OSC_ERR_INVALID_ARG, "grouped weights: use osc_linear_swiglu_grouped");
+    if (M == 0) return OSC_OK;
+    osc_act_sizes_t sz;
+    osc_act_sizes(w, M, &sz);
+    size_t need = 0;
+    osc_linear_swiglu_workspace_bytes(w, M, &need);
+    if (!workspace || !aligned16(workspace)) return fail(OSC_ERR_ALIGN, "workspace must be non-null and 16-byte aligned");
+    if (workspace_bytes < need) return fail(OSC_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", workspace_bytes, need);
+    if (osc_status s = check_h(w, H, ldh)) return s;
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint8_t *xq = ws + sz.xq_offset, *sfa = ws + sz.sfa_offset, *xo = ws + sz.xo_offset;
+    if (gamma) {
+        if (osc_status s = rmsnorm_quantize_impl(w, X, M, ldx, gamma, eps, xq, sfa, xo, st)) return s;
+    } else {
+        if (osc_status s = quantize_impl(w, X, M, ldx, xq, sfa, xo, nullptr, 0, st)) return s;
+    }
+    return gemm_swiglu_impl(w, xq, sfa, xo, M, H, ldh, nullptr, 0, nullptr, 0, ws + sz.workspace_bytes, st);
 }
 
 osc_status osc_linear_swiglu(const osc_weights* w, const void* X, int M, int64_t ldx, void* H, int64_t ldh, void* workspace,
@@ -890,6 +928,97 @@ osc_status osc_rmsnorm_linear_grouped_gather(const osc_weights* w, const void* H
                                              int64_t ldy, void* workspace, size_t workspace_bytes, void* stream) {
     if (!gamma) return fail(OSC_ERR_INVALID_ARG, "gamma is null");
     return grouped_gather_impl(w, H, T, ldh, gamma, eps, row_token, off, M_total, Y, ldy, workspace, workspace_bytes, stream);
+}
+
+// ---- grouped (MoE) gate|up projection with the SwiGLU in the epilogue
+osc_status osc_linear_swiglu_grouped(const osc_weights* w, const void* X_perm, const int32_t* off, int M_total, int64_t ldx,
+                                     void* H, int64_t ldh, void* workspace, size_t workspace_bytes, void* stream) {
+    if (osc_status s = check_act(w, X_perm, M_total, ldx)) return s;
+    if (!w->gate_up) return fail(OSC_ERR_INVALID_ARG, "not a gate|up handle: use osc_prepare_weights_gate_up_grouped");
+    if (!w->grouped) return fail(OSC_ERR_INVALID_ARG, "dense weights: use osc_linear_swiglu");
+    if (M_total == 0) return OSC_OK;
+    if (!off) return fail(OSC_ERR_INVALID_ARG, "off is null");
+    osc_act_sizes_t sz;
+    osc_act_sizes(w, M_total, &sz);
+    size_t need = 0;
+    osc_linear_swiglu_workspace_bytes(w, M_total, &need);
+    if (!workspace || !aligned16(workspace)) return fail(OSC_ERR_ALIGN, "workspace must be non-null and 16-byte aligned");
+    if (workspace_bytes < need) return fail(OSC_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", workspace_bytes, need);
+    if (osc_status s = check_h(w, H, ldh)) return s;
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int max_tiles = M_total / 128 + w->E;
+    const int max_tiles2 = max_tiles256(M_total, w->E);
+    int32_t* sched = reinterpret_cast<int32_t*>(ws + sz.sched_offset);
+    int32_t* sched2 = use_pair_kernel(true, M_total, w->E) ? sched + sched_ints(max_tiles) : nullptr;
+    cudaError_t e = launch_build_sched(off, w->E, sched, max_tiles, sched2, max_tiles2, st);
+    if (e != cudaSuccess) return cuda_fail(e, "build_sched_kernel");
+    uint8_t *xq = ws + sz.xq_offset, *sfa = ws + sz.sfa_offset, *xo = ws + sz.xo_offset;
+    if (osc_status s = quantize_impl(w, X_perm, M_total, ldx, xq, sfa, xo, sched, max_tiles, st)) return s;
+    return gemm_swiglu_impl(w, xq, sfa, xo, M_total, H, ldh, sched, max_tiles, sched2, max_tiles2, ws + sz.workspace_bytes, st);
+}
+
+// The same with the dispatch fused behind the quantizer (tokens quantized once, optionally behind an RMSNorm, their
+// quantized rows gathered): workspace = the gathered call's buffers, then the scratch [M_total, 2I] if the fused form
+// does not run.
+osc_status osc_swiglu_gather_workspace_bytes(const osc_weights* w, int T, int M_total, size_t* bytes) {
+    if (!w || !bytes) return fail(OSC_ERR_INVALID_ARG, "null argument");
+    if (!w->gate_up) return fail(OSC_ERR_INVALID_ARG, "not a gate|up handle: use osc_prepare_weights_gate_up_grouped");
+    size_t g = 0;
+    if (osc_status s = osc_gather_workspace_bytes(w, T, M_total, &g)) return s;
+    *bytes = align256(g) + (swiglu_fused(w, M_total) ? 0 : align256((size_t)M_total * w->N * 2));
+    return OSC_OK;
+}
+
+static osc_status swiglu_grouped_gather_impl(const osc_weights* w, const void* X, int T, int64_t ldx, const void* gamma, float eps,
+                                             const int32_t* row_token, const int32_t* off, int M_total, void* H, int64_t ldh,
+                                             void* workspace, size_t workspace_bytes, void* stream) {
+    if (osc_status s = check_act(w, X, T, ldx)) return s;
+    if (!w->gate_up) return fail(OSC_ERR_INVALID_ARG, "not a gate|up handle: use osc_prepare_weights_gate_up_grouped");
+    if (!w->grouped) return fail(OSC_ERR_INVALID_ARG, "dense weights have no dispatch");
+    if (M_total < 0) return fail(OSC_ERR_INVALID_ARG, "M_total = %d is negative", M_total);
+    if (M_total == 0) return OSC_OK;
+    if (T == 0) return fail(OSC_ERR_INVALID_ARG, "rows to dispatch but no tokens");
+    if (!off || !row_token) return fail(OSC_ERR_INVALID_ARG, "off / row_token is null");
+    osc_act_sizes_t sz;
+    osc_act_sizes(w, M_total, &sz);
+    const GatherLayout g = gather_layout(w, T, sz);
+    size_t need = 0;
+    osc_swiglu_gather_workspace_bytes(w, T, M_total, &need);
+    if (!workspace || !aligned16(workspace)) return fail(OSC_ERR_ALIGN, "workspace must be non-null and 16-byte aligned");
+    if (workspace_bytes < need) return fail(OSC_ERR_WORKSPACE, "workspace has %zu bytes, %zu needed", workspace_bytes, need);
+    if (osc_status s = check_h(w, H, ldh)) return s;
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int max_tiles = M_total / 128 + w->E;
+    const int max_tiles2 = max_tiles256(M_total, w->E);
+    int32_t* sched = reinterpret_cast<int32_t*>(ws + sz.sched_offset);
+    int32_t* sched2 = use_pair_kernel(true, M_total, w->E) ? sched + sched_ints(max_tiles) : nullptr;
+    cudaError_t e = launch_build_sched(off, w->E, sched, max_tiles, sched2, max_tiles2, st);
+    if (e != cudaSuccess) return cuda_fail(e, "build_sched_kernel");
+    if (gamma) {
+        if (osc_status s = rmsnorm_quantize_impl(w, X, T, ldx, gamma, eps, ws + g.xq_u, ws + g.sf_u, ws + g.xo_u, st)) return s;
+    } else {
+        if (osc_status s = quantize_impl(w, X, T, ldx, ws + g.xq_u, ws + g.sf_u, ws + g.xo_u, nullptr, 0, st)) return s;
+    }
+    e = launch_gather_quantized(row_token, T, w->K, w->Kop, ws + g.xq_u, ws + g.sf_u, ws + g.xo_u, ws + sz.xq_offset,
+                                ws + sz.sfa_offset, ws + sz.xo_offset, sched, max_tiles, st);
+    if (e != cudaSuccess) return cuda_fail(e, "gather_quantized_kernel");
+    return gemm_swiglu_impl(w, ws + sz.xq_offset, ws + sz.sfa_offset, ws + sz.xo_offset, M_total, H, ldh, sched, max_tiles, sched2,
+                            max_tiles2, ws + align256(g.total), st);
+}
+
+osc_status osc_linear_swiglu_grouped_gather(const osc_weights* w, const void* X, int T, int64_t ldx, const int32_t* row_token,
+                                            const int32_t* off, int M_total, void* H, int64_t ldh, void* workspace,
+                                            size_t workspace_bytes, void* stream) {
+    return swiglu_grouped_gather_impl(w, X, T, ldx, nullptr, 0.0f, row_token, off, M_total, H, ldh, workspace, workspace_bytes, stream);
+}
+osc_status osc_rmsnorm_linear_swiglu_grouped_gather(const osc_weights* w, const void* Hin, int T, int64_t ldh_in, const void* gamma,
+                                                    float eps, const int32_t* row_token, const int32_t* off, int M_total, void* H,
+                                                    int64_t ldh, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!gamma) return fail(OSC_ERR_INVALID_ARG, "gamma is null");
+    return swiglu_grouped_gather_impl(w, Hin, T, ldh_in, gamma, eps, row_token, off, M_total, H, ldh, workspace, workspace_bytes,
+                                      stream);
 }
 
 // ------------------------------------------------------- offline profiling

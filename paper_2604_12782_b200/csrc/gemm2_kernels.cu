@@ -94,7 +94,7 @@ struct Cfg {
     static_assert(BN % 16 == 0 && BN <= 256 && (LAST_W == 64 || LAST_W == 48), "tile width");
 };
 
-// GU (gate|up projection with the SwiGLU in the epilogue, dense MODE_OSC with per-tile weight scales only): the
+// GU (gate|up projection with the SwiGLU in the epilogue, MODE_OSC with per-tile weight scales, dense or grouped): the
 // weight matrix holds the gate rows [0, N/2) above the up rows [N/2, N).  A tile takes BN/2 gate features and the
 // same BN/2 up features - the leader CTA loads the gate half of the weight tile, its peer the up half, and the
 // per-tile copy of the weight scales is arranged the same way - so accumulator columns [0, BN/2) and [BN/2, BN)
@@ -189,7 +189,7 @@ __global__ void __launch_bounds__(pair_threads(GU), 1) gemm_pair_kernel(const __
         const uint32_t st = smem_u32(smem + s * C::STAGE_BYTES);
         const uint32_t fb = map_to_cta(smem_u32(full_bar), 0) + (uint32_t)s * 8u;
         // my half of the weight rows (gate|up: the leader's half are gate rows, the peer's the up rows of the same features)
-        const int brow = GU ? (int)rank * (N / 2) + (n0 / BN) * (BN / 2) : expert * N + n0 + (int)rank * (BN / 2);
+        const int brow = GU ? expert * N + (int)rank * (N / 2) + (n0 / BN) * (BN / 2) : expert * N + n0 + (int)rank * (BN / 2);
         if (kb < nkb_a) {
             if (expect && rank == 0) mbar_arrive_expect_tx(&full_bar[s], C::SCALED ? C::TX_A : C::TX_B);
             tma_load_2d_pair(st + A_BYTES, &args.tm_b, fb, kb * ROW_BYTES, brow);
@@ -488,19 +488,20 @@ __global__ void __launch_bounds__(pair_threads(GU), 1) gemm_pair_kernel(const __
                             fence_proxy_async_smem();
                             __syncwarp();
                             const int prow0 = wrow0 + hh * 16;
-                            if (wd == 32) {
+                            // grouped problems: rows past the expert's end belong to the next expert
+                            if (wd == 32 && !(sched != nullptr && prow0 + 16 > ti.row_end)) {
                                 if (lane == 0) {
                                     tma_store_2d_hint(&args.tm_y16, buf, col, prow0, y_policy);   // clipped at M rows, I columns
                                     tma_store_commit();
                                 }
                             } else {
-                                // the narrow last chunk is no store box (its neighbours belong to the next tile):
-                                // row-masked 16-byte stores from the staged tile
+                                // the narrow last chunk is no store box (its neighbours belong to the next tile), nor is a
+                                // pass that straddles an expert's end: row-masked 16-byte stores from the staged tile
                                 const int j4 = lane & 3;
 #pragma unroll
                                 for (int rr = 0; rr < 2; ++rr) {
                                     const int rl = rr * 8 + (lane >> 2);
-                                    if (prow0 + rl < args.M && j4 * 8 < wd && col + j4 * 8 < I)
+                                    if (prow0 + rl < ti.row_end && j4 * 8 < wd && col + j4 * 8 < I)
                                         *reinterpret_cast<uint4*>(args.Y + (int64_t)(prow0 + rl) * args.ldy + col + j4 * 8) =
                                             *reinterpret_cast<const uint4*>(buf + rl * 64 + ((j4 ^ ((rl >> 1) & 3)) << 4));
                                 }

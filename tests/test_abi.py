@@ -151,3 +151,21 @@ def test_nvfp4_fused_calls_refuse_null_handles():
     assert lib.osc_nvfp4_linear_grouped_gather(None, None, 0, 0, None, None, 0, 0, None, 0, None, 0, None) == -1
     assert lib.osc_nvfp4_rmsnorm_linear_grouped_gather(None, None, 0, 0, None, C.c_float(0), None, None, 0, 0, None, 0, None, 0,
                                                        None) == -1
+
+
+def test_gate_up_calls_refuse_null_handles_and_odd_shapes():
+    from paper_2604_12782_b200 import binding as B
+    lib = B._lib
+    sz = C.c_size_t()
+    assert lib.osc_linear_swiglu(None, None, 0, 0, None, 0, None, 0, None) == -1
+    assert lib.osc_linear_swiglu_grouped(None, None, None, 0, 0, None, 0, None, 0, None) == -1
+    assert lib.osc_swiglu_gather_workspace_bytes(None, 0, 0, C.byref(sz)) == -1
+    assert lib.osc_linear_swiglu_grouped_gather(None, None, 0, 0, None, None, 0, None, 0, None, 0, None) == -1
+    assert lib.osc_rmsnorm_linear_swiglu_grouped_gather(None, None, 0, 0, None, C.c_float(0), None, None, 0, None, 0, None, 0,
+                                                        None) == -1
+    lut = np.full((16, 1), -1, np.int8)
+    ws = B.WeightSizes()
+    assert lib.osc_gate_up_weight_sizes_grouped(0, 64, 512, lut.ctypes.data, 1, C.byref(ws)) == -1     # no experts
+    assert lib.osc_gate_up_weight_sizes_grouped(2, 60, 512, lut.ctypes.data, 1, C.byref(ws)) == -2     # I not a multiple of 8
+    assert lib.osc_gate_up_weight_sizes_grouped(2, 64, 512, lut.ctypes.data, 1, C.byref(ws)) == 0
+    assert ws.wq_bytes == 2 * 128 * 256

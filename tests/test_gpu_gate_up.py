@@ -97,3 +97,62 @@ def test_rmsnorm_linear_swiglu_and_errors(B, oracle):
     with pytest.raises(B.OscError) as e:
         B.osc_linear_swiglu(w, dev_bf16(Hb), H, ws[:64])
     assert e.value.status == -5
+
+
+# experts: large ones (the pair kernel's gate|up form: experts that end inside a 256-row tile, inside a 16-row store pass,
+# empty and one-row experts) and small ones (the route through a scratch Y)
+@pytest.mark.parametrize("counts,mode", [([300, 0, 5, 256, 129, 511, 1, 385], "perm"), ([700, 64, 0, 900], "perm"),
+                                         ([3, 0, 130, 1, 257, 128], "gather"), ([17, 40, 3, 0, 25], "perm"),
+                                         ([300, 0, 5, 256, 129, 511, 1, 385], "norm_gather")])
+def test_linear_swiglu_grouped(B, oracle, counts, mode):
+    """Grouped (MoE) gate|up projection with the SwiGLU in the epilogue: per expert bit for bit the dense call on that
+    expert's rows and weights, nothing written outside H, and within the pushed-through tolerance of the oracle."""
+    from producer_inputs import gamma_bits
+    counts = np.array(counts)
+    E, K, I = counts.size, 384, 256
+    M = int(counts.sum())
+    off_h = synth.offsets_from_counts(counts)
+    off = torch.from_numpy(off_h).cuda()
+    rng = np.random.default_rng(E + M)
+    T = max(1, M // 3)
+    c = synth.osc_linear_case(70 + E, T if mode != "perm" else M, K, 64, 1)
+    Wb = synth.f32_to_bf16_bits((0.08 * rng.standard_normal((E, 2 * I, K))).astype(np.float32))
+    gb = gamma_bits(rng, K)
+    w = B.osc_prepare_weights_gate_up_grouped(dev_bf16(Wb.reshape(E * 2 * I, K)).view(E, 2 * I, K), c["lut"])
+    big = torch.full((M + 2, I + 8), 7.0, dtype=torch.bfloat16, device="cuda")
+    H = big[1:M + 1, :I]
+    if mode == "perm":
+        Xp = c["X"]
+        ws = poison(B.osc_linear_swiglu_workspace_bytes(w, M))
+        B.osc_linear_swiglu_grouped(w, dev_bf16(Xp), off, H, ws)
+    else:
+        row_token_h = rng.integers(0, T, size=M).astype(np.int32)
+        src = oracle.rmsnorm(c["X"], gb, 1e-6) if mode == "norm_gather" else c["X"]
+        Xp = np.ascontiguousarray(src[row_token_h])
+        ws = poison(B.osc_swiglu_gather_workspace_bytes(w, T, M))
+        row_token = torch.from_numpy(row_token_h).cuda()
+        if mode == "norm_gather":
+            B.osc_rmsnorm_linear_swiglu_grouped_gather(w, dev_bf16(c["X"]), dev_bf16(gb), 1e-6, row_token, off, H, ws)
+        else:
+            B.osc_linear_swiglu_grouped_gather(w, dev_bf16(c["X"]), row_token, off, H, ws)
+    B.osc_sync_check()
+    guard = big.clone()
+    guard[1:M + 1, :I] = 7.0
+    assert (guard == 7.0).all(), "wrote outside H"
+    got = host_bf16_bits(H.contiguous())
+    Hf = host_f64(H)
+    for e in range(E):
+        r0, r1 = int(off_h[e]), int(off_h[e + 1])
+        if r1 == r0:
+            continue
+        Yref, T_, *_ = oracle.linear(Xp[r0:r1], Wb[e], c["lut"])
+        href, bound = h_bound(Yref, T_, I)
+        err = np.abs(Hf[r0:r1] - href)
+        assert (err <= bound).all(), f"expert {e}: worst err/bound {np.max(err / bound):.3f}"
+        # the dense fused call on the expert's own rows and weights
+        wd = B.osc_prepare_weights_gate_up(dev_bf16(Wb[e]), c["lut"])
+        Hd = torch.full((r1 - r0, I), float("nan"), dtype=torch.bfloat16, device="cuda")
+        B.osc_linear_swiglu(wd, dev_bf16(Xp[r0:r1]), Hd, poison(B.osc_linear_swiglu_workspace_bytes(wd, r1 - r0)))
+        B.osc_sync_check()
+        assert np.array_equal(got[r0:r1], host_bf16_bits(Hd)), f"expert {e} differs from the dense call"
+    assert not torch.isnan(H.float()).any()
