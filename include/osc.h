@@ -63,7 +63,7 @@
  * different kernels for the same inputs agree within the accumulation-order rounding of fp32, not bit for
  * bit; one kernel is deterministic run to run.
  * Environment variables for experiments (read by the library, not part of the contract): OSC_DECODE (0 = never,
- * 2 = always up to 256 rows), OSC_DECODE_SPLIT, OSC_PAIR (0 = 128-row tiles only, 2 = pair tiles whenever
+ * 2 = always up to 256 rows), OSC_DECODE_SPLIT, OSC_DECODE_FUSED_ROWS (0 = the quantizer always its own kernel), OSC_PAIR (0 = 128-row tiles only, 2 = pair tiles whenever
  * eligible), OSC_PAIR_BLOCK_N, OSC_BLOCK_N, OSC_BAND, OSC_PAIRS, OSC_MAP_CACHE (0 = encode every TMA descriptor anew), OSC_LOG.
  * Sizes: M, N, K and E are ints; every row offset is computed in 64 bits, so M * K (and M * N) may exceed
  * 2^31 elements.
@@ -157,7 +157,10 @@ osc_status osc_quantize_extract(const osc_weights* w, const void* X, int M, int6
 osc_status osc_gemm_dual(const osc_weights* w, const void* xq, const void* sfa, const void* xo, int M,
                          void* Y, int64_t ldy, void* stream);
 
-/* osc_quantize_extract followed by osc_gemm_dual; workspace (dev) holds xq/sfa/xo. */
+/* osc_quantize_extract followed by osc_gemm_dual; workspace (dev) holds xq/sfa/xo between the two and is scratch: its
+ * content after the call is unspecified.  With sixteen rows or fewer and a short K loop the few-row kernel quantizes
+ * the activations of each CTA's K slice itself (the scales of Algorithm 2 are local to a group) and no quantizer
+ * kernel runs; Y equals the two-step result bit for bit. */
 osc_status osc_linear(const osc_weights* w, const void* X, int M, int64_t ldx, void* Y, int64_t ldy,
                       void* workspace, size_t workspace_bytes, void* stream);
 

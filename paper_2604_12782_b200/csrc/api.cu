@@ -589,6 +589,46 @@ osc_status osc_gemm_dual(const osc_weights* w, const void* xq, const void* sfa, 
     return gemm_impl(w, xq, sfa, xo, M, Y, ldy, nullptr, 0, nullptr, 0, static_cast<cudaStream_t>(stream));
 }
 
+// With very few rows the quantizer kernel in front of the few-row GEMM costs more than its work: the GEMM kernel's
+// CTAs quantize the activations of their own K slice themselves (same arithmetic, same result).  Every feature
+// tile repeats that work, one warp per stage, so it pays while (row quarters) x (stages per CTA) stays small -
+// measured on B200, graph replay, two kernels -> one: QKV 4096 -> 6144 8.3 / 8.8 / 9.3 -> 6.5 / 7.3 / 8.9 us at 1 / 8 / 16
+// rows, o_proj 8.3 / 8.5 -> 5.8 / 7.8 us at 4 / 16 rows, gate_up (18 stages per CTA) 14.4 / 14.6 -> 12.8 / 13.2 us at 1 / 4
+// rows but 14.9 -> 16.9 us at 16 rows, K = 12288 with 768 flagged channels 12.6 -> 9.8 us at 4 rows but 13.1 -> 20.5 us
+// at 16 (the Path-B blocks are gathered two bytes at a time).  Tables of more than 1024 flagged channels take
+// the two kernels.  OSC_DECODE_FUSED_ROWS = 0: always two kernels; = n: the fused form whenever M <= min(n, 16).
+static bool decode_quantizes_itself(const osc_weights* w, int M) {
+    if (M > 16 || w->Kop > 1024) return false;
+    const int nkb = (w->K + 255) / 256 + w->Kop / 64;
+    if (!use_decode_kernel(w->grouped, M, w->N, nkb, w->num_sms)) return false;
+    if (const char* e = getenv("OSC_DECODE_FUSED_ROWS")) return M <= atoi(e);   // read per call: tests switch it inside one process
+    const int S = gemm_decode_split(w->N, nkb, w->num_sms);
+    const int quarters = (M + 3) / 4;
+    return quarters * ((nkb + S - 1) / S) <= 24 && quarters * (w->Kop / 64) <= 24;
+}
+static osc_status gemm_decode_quant_impl(const osc_weights* w, const void* X, int M, int64_t ldx, void* Y, int64_t ldy,
+                                         cudaStream_t st) {
+    GemmArgs a;
+    memset(&a, 0, sizeof a);
+    a.tm_b = w->tm_b[1];
+    if (w->Kop > 0) a.tm_bo = w->tm_bo[1];
+    a.sfw = w->sfw;
+    a.Y = static_cast<uint16_t*>(Y);
+    a.ldy = ldy;
+    a.M = M; a.N = w->N; a.K = w->K; a.Kop = w->Kop;
+    a.num_sms = w->num_sms;
+    DecodeX xa;
+    xa.X = static_cast<const uint16_t*>(X);
+    xa.ldx = ldx;
+    xa.mask = w->mask;
+    xa.idx_o = w->idx_o;
+    xa.Ko = w->Ko;
+    const int S = gemm_decode_split(w->N, (w->K + 255) / 256 + w->Kop / 64, w->num_sms);
+    cudaError_t e = launch_gemm_dual_decode_quant(a, xa, S, st);
+    if (e != cudaSuccess) return cuda_fail(e, "gemm_decode_kernel(dual, quantizing)");
+    return OSC_OK;
+}
+
 osc_status osc_linear(const osc_weights* w, const void* X, int M, int64_t ldx, void* Y, int64_t ldy,
                       void* workspace, size_t workspace_bytes, void* stream) {
     if (osc_status s = check_act(w, X, M, ldx)) return s;
@@ -604,6 +644,7 @@ osc_status osc_linear(const osc_weights* w, const void* X, int M, int64_t ldx, v
     if (ldy % 8 || !aligned16(Y)) return fail(OSC_ERR_ALIGN, "Y must be 16-byte aligned and ldy a multiple of 8");
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (decode_quantizes_itself(w, M)) return gemm_decode_quant_impl(w, X, M, ldx, Y, ldy, st);
     if (osc_status s = quantize_impl(w, X, M, ldx, ws + sz.xq_offset, ws + sz.sfa_offset, ws + sz.xo_offset, nullptr, 0, st)) return s;
     return gemm_impl(w, ws + sz.xq_offset, ws + sz.sfa_offset, ws + sz.xo_offset, M, Y, ldy, nullptr, 0, nullptr, 0, st);
 }

@@ -133,7 +133,16 @@ cudaError_t launch_gemm_nvf4_pair(const GemmArgs& a, int bn, cudaStream_t st);
 int gemm_pair_block_n(bool fp8, bool allow_240, long row_tiles, int N, int stages, int num_sms, long* cost_ns = nullptr);
 
 // gemm3_kernels.cu (few rows: operands swapped, K split over a cluster)
+// activations of the few-row kernel's in-kernel quantizer (Algorithm 2 on the CTA's own K slice)
+struct DecodeX {
+    const uint16_t* X;     // bf16 [M, ldx]
+    int64_t ldx;
+    const uint32_t* mask;  // flagged channels per 32-channel group
+    const int32_t* idx_o;  // channel of every column of the buffer B
+    int Ko;
+};
 cudaError_t launch_gemm_dual_decode(const GemmArgs& a, int S, cudaStream_t st);
+cudaError_t launch_gemm_dual_decode_quant(const GemmArgs& a, const DecodeX& xa, int S, cudaStream_t st);
 cudaError_t launch_gemm_fp8_decode(const GemmArgs& a, int S, cudaStream_t st);
 cudaError_t launch_gemm_mxf8_decode(const GemmArgs& a, int S, cudaStream_t st);
 cudaError_t launch_gemm_nvf4_decode(const GemmArgs& a, int S, cudaStream_t st);

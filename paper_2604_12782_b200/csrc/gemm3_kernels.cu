@@ -17,6 +17,12 @@
 // activation quantizer.
 //
 //   warp 0    : TMA producer          warp 1 : MMA issuer, TMEM owner        warps 2-5 : epilogue
+// QX form (MXFP4, up to 16 rows): no quantizer kernel runs in front.  The scales of Algorithm 2 are local to a
+// 32-channel group, so a CTA can quantize exactly the activations of its own K slice: while the weight stream is in
+// flight, warps 2-5 read the bf16 rows of X, zero the flagged channels, compute scale and codes with the
+// quantizer's own arithmetic and write the stage's activation tile (128-byte swizzle), its scale blocks, and for
+// the blocks of Path B the gathered flagged channels, straight into the ring.  Every cluster of a feature tile
+// repeats this for the same few rows (they come from L2), which costs less than a kernel boundary.
 // Modes and K-block order are those of the other GEMM kernels (Path A block-scaled FP4 blocks - MXFP4 or
 // NVFP4 - then the BF16 blocks of Path B; or E4M3 blocks with per-row scales applied in the epilogue, or
 // block-scaled E4M3).
@@ -38,6 +44,7 @@ constexpr int ROW_BYTES = 128;
 constexpr int W_BYTES = BF * ROW_BYTES;        // 16 KB of weights per stage
 constexpr int THREADS = 192;
 constexpr int MAX_CLUSTER = 8;
+constexpr int QX_IDX_BYTES = 4096;      // QX form: the channels of up to 1024 columns of the buffer B, in shared memory
 
 // TOK = most activation rows per call: 64 (two CTAs per SM) or 256 (one CTA per SM; for long K loops, where a
 // 128-row-tile kernel would leave most SMs without a tile)
@@ -83,9 +90,49 @@ __device__ __forceinline__ float4 ld_cluster_f32x4(uint32_t cluster_addr) {
     return v;
 }
 
-template <int MODE, int TOK>
-__global__ void __launch_bounds__(THREADS, Cfg<MODE, TOK>::CTAS_PER_SM) gemm_decode_kernel(const __grid_constant__ GemmArgs args) {
+// QX form: NQ live row quarters of a stage (lane -> row 4j + lane/8 of quarter j, 32-channel group lane%8), quantized
+// with the quantizer's arithmetic and written into the stage's activation tile (128-byte swizzle) and scale blocks.
+// One straight-line body per count, so that the chains of the quarters overlap; the other quarters get zero codes
+// and scales.
+template <int NQ>
+__device__ __forceinline__ void qx_quantize_quarters(uint32_t (&w)[4][16], uint32_t flagged, int lane, uint8_t* xt, uint8_t* sfx) {
+    const int g = lane & 7;
+    uint32_t q[4][4];
+    int code[4];
+    if (flagged) {      // zero-out: the flagged channels go through Path B
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const uint32_t keep = ~(((flagged >> (2 * i)) & 1u ? 0x0000FFFFu : 0u) | ((flagged >> (2 * i + 1)) & 1u ? 0xFFFF0000u : 0u));
+#pragma unroll
+            for (int j = 0; j < NQ; ++j) w[j][i] &= keep;
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        if (j < NQ) {
+            code[j] = mxfp4_group(w[j], q[j]);   // an all-zero group (row past M, channels past K): code 0, codes 0
+        } else {
+            code[j] = 0;
+            q[j][0] = q[j][1] = q[j][2] = q[j][3] = 0u;
+        }
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const int row = 4 * j + (lane >> 3);
+        uint32_t word = (uint32_t)code[j] << (8 * (g & 3));
+        word |= __shfl_xor_sync(0xFFFFFFFFu, word, 1);
+        word |= __shfl_xor_sync(0xFFFFFFFFu, word, 2);
+        if ((g & 3) == 0) *reinterpret_cast<uint32_t*>(sfx + (g >> 2) * 512 + (row & 31) * 16 + (row >> 5) * 4) = word;
+        *reinterpret_cast<uint4*>(xt + row * ROW_BYTES + ((g ^ (row & 7)) << 4)) = make_uint4(q[j][0], q[j][1], q[j][2], q[j][3]);
+    }
+}
+
+template <int MODE, int TOK, bool QX>
+__global__ void __launch_bounds__(THREADS, Cfg<MODE, TOK>::CTAS_PER_SM)
+gemm_decode_kernel(const __grid_constant__ GemmArgs args, const DecodeX xa) {
     using C = Cfg<MODE, TOK>;
+    static_assert(!QX || (MODE == MODE_OSC && TOK <= 64), "in-kernel activation quantizer: MXFP4, few rows");
+    constexpr int QWARPS = THREADS / 32 - 2;   // warps 2.. quantize in the QX form
     constexpr int STAGES = C::STAGES;
     constexpr int X_BYTES = C::X_BYTES, TM_SFW = C::TM_SFW, TM_SFX = C::TM_SFX, TMEM_COLS = C::TMEM_COLS;
 
@@ -107,16 +154,16 @@ __global__ void __launch_bounds__(THREADS, Cfg<MODE, TOK>::CTAS_PER_SM) gemm_dec
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < STAGES; ++i) {
-            mbar_init(&full_bar[i], 1);
+            mbar_init(&full_bar[i], QX ? 2 : 1);   // the weight loads, and in the QX form the slot's quantizing warp
             mbar_init(&empty_bar[i], 1);
         }
         mbar_init(tfull_bar, 1);
         *abort_flag = 0;
         fence_barrier_init();
-        prefetch_tmap(&args.tm_a);
+        if (!QX) prefetch_tmap(&args.tm_a);
         prefetch_tmap(&args.tm_b);
         if (C::DUAL && args.Kop > 0) {
-            prefetch_tmap(&args.tm_ao);
+            if (!QX) prefetch_tmap(&args.tm_ao);
             prefetch_tmap(&args.tm_bo);
         }
     }
@@ -150,8 +197,9 @@ __global__ void __launch_bounds__(THREADS, Cfg<MODE, TOK>::CTAS_PER_SM) gemm_dec
         // ------------------------------------------------------------ TMA producer
         // weights (and their scales) of the first ring before the dependency wait, activations after it
         auto expect = [&](int kb, int s) {
-            uint32_t bytes = W_BYTES + (uint32_t)(ntok * ROW_BYTES);   // the activation tile holds ntok rows
-            if (C::SCALED && kb < nkb_a) bytes += (uint32_t)(1 + xatoms) * 512u * (uint32_t)min(C::KA, katoms_total - C::KA * kb);
+            uint32_t bytes = W_BYTES + (QX ? 0u : (uint32_t)(ntok * ROW_BYTES));   // the activation tile holds ntok rows
+            if (C::SCALED && kb < nkb_a)
+                bytes += (uint32_t)(QX ? 1 : 1 + xatoms) * 512u * (uint32_t)min(C::KA, katoms_total - C::KA * kb);
             mbar_arrive_expect_tx(&full_bar[s], bytes);
         };
         auto load_w = [&](int kb, int s) {
@@ -189,11 +237,13 @@ __global__ void __launch_bounds__(THREADS, Cfg<MODE, TOK>::CTAS_PER_SM) gemm_dec
             }
         }
         __syncwarp();
-        grid_dependency_wait();   // the quantized activations come from the kernel before this one
-        if (elect_one()) {
-            for (int i = 0; i < first; ++i) load_x(kb0 + i, i);
+        if (!QX) {
+            grid_dependency_wait();   // the quantized activations come from the kernel before this one
+            if (elect_one()) {
+                for (int i = 0; i < first; ++i) load_x(kb0 + i, i);
+            }
+            __syncwarp();
         }
-        __syncwarp();
         int s = 0;
         uint32_t ph = 1;          // the ring has been filled once
         for (int kb = kb0 + first; kb < kb1; ++kb) {
@@ -201,7 +251,7 @@ __global__ void __launch_bounds__(THREADS, Cfg<MODE, TOK>::CTAS_PER_SM) gemm_dec
             if (elect_one()) {
                 expect(kb, s);
                 load_w(kb, s);
-                load_x(kb, s);
+                if (!QX) load_x(kb, s);
             }
             __syncwarp();
             if (++s == STAGES) { s = 0; ph ^= 1u; }
@@ -297,6 +347,75 @@ __global__ void __launch_bounds__(THREADS, Cfg<MODE, TOK>::CTAS_PER_SM) gemm_dec
         }
         if (elect_one()) tc_commit(tfull_bar);
         __syncwarp();
+    } else if (QX) {
+        // ------------------------------------------------ activations of my K slice, quantized in place (QX form)
+        // Sixteen token rows at most.  Quantizing one group is a long dependent chain, so the stages are dealt to
+        // the warps in turn (warp j fills ring slot j: the slots are as many as the warps) and several stages are
+        // in the making at once; a lane holds (row, 32-channel group) of four row quarters for a block of Path A,
+        // (row, eight flagged channels) for a block of Path B, all loads of a stage in flight before the first use.
+        static_assert(!QX || STAGES == QWARPS, "one ring slot per quantizing warp");
+        const int wq = warp - 2;
+        const int g = lane & 7;
+        int32_t* idx_s = reinterpret_cast<int32_t*>(smem + STAGES * C::STAGE_BYTES + 256);   // behind the barriers
+        for (int o = (int)threadIdx.x - 64; o < args.Kop; o += QWARPS * 32) idx_s[o] = o < xa.Ko ? __ldg(xa.idx_o + o) : -1;
+        asm volatile("bar.sync 1, %0;" ::"n"(QWARPS * 32) : "memory");
+        grid_dependency_wait();             // X comes from the kernel before this one
+        uint8_t* xt = smem + wq * C::STAGE_BYTES + W_BYTES;
+        uint64_t* my_full = &full_bar[wq];
+        uint32_t ph = 0;
+        for (int kb = kb0 + wq; kb < kb1; kb += QWARPS) {
+            uint32_t w[4][16];
+            uint32_t flagged = 0u;
+            const bool path_a = kb < nkb_a;
+            const bool in_k = path_a && kb * 256 + g * 32 < K;
+            if (in_k) flagged = __ldg(xa.mask + kb * 8 + g);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int row = 4 * j + (lane >> 3);
+#pragma unroll
+                for (int i = 0; i < 16; ++i) w[j][i] = 0u;
+                if (row < M) {
+                    const uint16_t* xrow = xa.X + (int64_t)row * xa.ldx;
+                    if (in_k) {
+                        const uint4* src = reinterpret_cast<const uint4*>(xrow + kb * 256 + g * 32);
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const uint4 v = src[i];
+                            w[j][4 * i] = v.x; w[j][4 * i + 1] = v.y; w[j][4 * i + 2] = v.z; w[j][4 * i + 3] = v.w;
+                        }
+                    } else if (!path_a) {
+                        const int o0 = (kb - nkb_a) * 64 + 8 * g;
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) {
+                            const int ch = idx_s[o0 + e];
+                            if (ch >= 0) w[j][e] = xrow[ch];
+                        }
+                    }
+                }
+            }
+            if (kb - kb0 >= STAGES) {       // my slot's previous stage has been multiplied
+                if (!wait_bounded(&empty_bar[wq], ph, abort_flag, 34)) break;
+                ph ^= 1u;
+            }
+            uint8_t* sfx = xt + X_BYTES + C::SFW_BYTES;
+            switch (path_a ? (min(M, 16) + 3) >> 2 : 0) {   // live row quarters: straight-line code for each count
+                case 1: qx_quantize_quarters<1>(w, flagged, lane, xt, sfx); break;
+                case 2: qx_quantize_quarters<2>(w, flagged, lane, xt, sfx); break;
+                case 3: qx_quantize_quarters<3>(w, flagged, lane, xt, sfx); break;
+                case 4: qx_quantize_quarters<4>(w, flagged, lane, xt, sfx); break;
+                default:                                    // a block of Path B: the gathered channels as they are
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const int row = 4 * j + (lane >> 3);
+                        *reinterpret_cast<uint4*>(xt + row * ROW_BYTES + ((g ^ (row & 7)) << 4)) =
+                            make_uint4(w[j][0] | (w[j][1] << 16), w[j][2] | (w[j][3] << 16), w[j][4] | (w[j][5] << 16),
+                                       w[j][6] | (w[j][7] << 16));
+                    }
+            }
+            fence_proxy_async_smem();       // written through the generic proxy, read by the tensor core
+            __syncwarp();
+            if (lane == 0) mbar_arrive(my_full);
+        }
     }
 
 done:
@@ -410,16 +529,17 @@ done:
     }
 }
 
-template <int MODE, int TOK>
-static cudaError_t launch_cfg(const GemmArgs& a, int S, cudaStream_t st) {
+template <int MODE, int TOK, bool QX = false>
+static cudaError_t launch_cfg(const GemmArgs& a, int S, cudaStream_t st, const DecodeX& xa = DecodeX{}) {
     using C = Cfg<MODE, TOK>;
     static PerDevice configured;
-    if (cudaError_t e = opt_in_shared_memory(configured, gemm_decode_kernel<MODE, TOK>, C::SMEM_BYTES)) return e;
+    constexpr int SMEM = C::SMEM_BYTES + (QX ? QX_IDX_BYTES : 0);
+    if (cudaError_t e = opt_in_shared_memory(configured, gemm_decode_kernel<MODE, TOK, QX>, SMEM)) return e;
     const int tiles = (a.N + BF - 1) / BF;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(tiles * S);
     cfg.blockDim = dim3(THREADS);
-    cfg.dynamicSmemBytes = C::SMEM_BYTES;
+    cfg.dynamicSmemBytes = SMEM;
     cfg.stream = st;
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -430,7 +550,7 @@ static cudaError_t launch_cfg(const GemmArgs& a, int S, cudaStream_t st) {
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, gemm_decode_kernel<MODE, TOK>, a);
+    return cudaLaunchKernelEx(&cfg, gemm_decode_kernel<MODE, TOK, QX>, a, xa);
 }
 
 }  // namespace decode
@@ -456,6 +576,9 @@ int gemm_decode_split(int N, int nkb, int num_sms) {
 
 cudaError_t launch_gemm_dual_decode(const GemmArgs& a, int S, cudaStream_t st) {
     return a.M <= 64 ? decode::launch_cfg<decode::MODE_OSC, 64>(a, S, st) : decode::launch_cfg<decode::MODE_OSC, 256>(a, S, st);
+}
+cudaError_t launch_gemm_dual_decode_quant(const GemmArgs& a, const DecodeX& xa, int S, cudaStream_t st) {
+    return decode::launch_cfg<decode::MODE_OSC, 64, true>(a, S, st, xa);
 }
 cudaError_t launch_gemm_nvf4_decode(const GemmArgs& a, int S, cudaStream_t st) {
     return a.M <= 64 ? decode::launch_cfg<decode::MODE_NVF4, 64>(a, S, st) : decode::launch_cfg<decode::MODE_NVF4, 256>(a, S, st);

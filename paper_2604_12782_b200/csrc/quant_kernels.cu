@@ -117,6 +117,39 @@ __device__ __forceinline__ uint32_t nvfp4_group(const uint32_t (&w)[16], float p
     return codes;
 }
 
+// MXFP4 arithmetic of one 32-channel group held as 16 packed bf16 pairs (Algorithm 2, CalculateScale + Quantize).
+// Returns the E8M0 code and the 32 packed E2M1 codes in q.
+__device__ __forceinline__ int mxfp4_group(const uint32_t (&w)[16], uint32_t (&q)[4]) {
+    // amax on the bf16 magnitudes, two at a time
+    __nv_bfloat162 m8[8];   // a tree, not a chain of sixteen: the thread has little else to overlap it with
+#pragma unroll
+    for (int i = 0; i < 8; ++i) m8[i] = __hmax2(__habs2(as_bf162(w[2 * i])), __habs2(as_bf162(w[2 * i + 1])));
+    const __nv_bfloat162 m2 = __hmax2(__hmax2(__hmax2(m8[0], m8[1]), __hmax2(m8[2], m8[3])),
+                                      __hmax2(__hmax2(m8[4], m8[5]), __hmax2(m8[6], m8[7])));
+    const uint32_t am2 = bf162_bits(m2);
+    const uint32_t am = max(am2 & 0xFFFFu, am2 >> 16);
+    // CalculateScale: E8M0 code = biased exponent of amax - 2, floored at 0 (2^(floor(log2 amax) - 2))
+    const int ex = (int)(am >> 7);
+    int code = max(ex - 2, 0);
+    if (ex == 255) code = 255;
+    // Quantize: x * 2^(127 - code) is exact (a power of two, two bf16 values per multiply; results below
+    // the bf16 normal range are far under the 0.25 tie point and keep their sign), then hardware E2M1
+    // rounding (nearest-even, saturating) of the fp32 extensions
+    const __nv_bfloat162 inv2 = as_bf162(((uint32_t)(254 - min(code, 253)) << 7) * 0x10001u);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        float f[8];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const uint32_t p = bf162_bits(__hmul2(as_bf162(w[4 * i + j]), inv2));
+            f[2 * j] = __uint_as_float(p << 16);
+            f[2 * j + 1] = __uint_as_float(p & 0xFFFF0000u);
+        }
+        q[i] = e2m1x8(f[0], f[1], f[2], f[3], f[4], f[5], f[6], f[7]);
+    }
+    return code;
+}
+
 // bf16 bits of x * 2^-tensor_e rounded to bf16 (nearest even): the backed-up channel in the scaled domain of NVFP4
 __device__ __forceinline__ uint16_t nvfp4_backup(uint16_t b, int tensor_e) {
     return __bfloat16_as_ushort(__float2bfloat16_rn(
@@ -251,34 +284,8 @@ quant_extract_kernel(const __grid_constant__ CUtensorMap tm_x, int M, int K,
             if (FMT == FMT_MXFP4) {
             int code = 0;
             if (r < row_end) {  // rows past the end (next expert / padding) count as zeros: code 0, nothing stored
-                // amax on the bf16 magnitudes, two at a time
-                __nv_bfloat162 m8[8];   // a tree, not a chain of sixteen: the thread has little else to overlap it with
-#pragma unroll
-                for (int i = 0; i < 8; ++i) m8[i] = __hmax2(__habs2(as_bf162(w[2 * i])), __habs2(as_bf162(w[2 * i + 1])));
-                const __nv_bfloat162 m2 = __hmax2(__hmax2(__hmax2(m8[0], m8[1]), __hmax2(m8[2], m8[3])),
-                                                  __hmax2(__hmax2(m8[4], m8[5]), __hmax2(m8[6], m8[7])));
-                const uint32_t am2 = bf162_bits(m2);
-                const uint32_t am = max(am2 & 0xFFFFu, am2 >> 16);
-                // CalculateScale: E8M0 code = biased exponent of amax - 2, floored at 0 (2^(floor(log2 amax) - 2))
-                const int ex = (int)(am >> 7);
-                code = max(ex - 2, 0);
-                if (ex == 255) code = 255;
-                // Quantize: x * 2^(127 - code) is exact (a power of two, two bf16 values per multiply; results below
-                // the bf16 normal range are far under the 0.25 tie point and keep their sign), then hardware E2M1
-                // rounding (nearest-even, saturating) of the fp32 extensions
-                const __nv_bfloat162 inv2 = as_bf162(((uint32_t)(254 - min(code, 253)) << 7) * 0x10001u);
                 uint32_t q[4];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    float f[8];
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const uint32_t p = bf162_bits(__hmul2(as_bf162(w[4 * i + j]), inv2));
-                        f[2 * j] = __uint_as_float(p << 16);
-                        f[2 * j + 1] = __uint_as_float(p & 0xFFFF0000u);
-                    }
-                    q[i] = e2m1x8(f[0], f[1], f[2], f[3], f[4], f[5], f[6], f[7]);
-                }
+                code = mxfp4_group(w, q);
                 *reinterpret_cast<uint4*>(xq + (int64_t)r * (K / 2) + cb * (QE_COLS / 2) + gi * 16) =
                     make_uint4(q[0], q[1], q[2], q[3]);
             }

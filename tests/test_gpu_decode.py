@@ -29,10 +29,11 @@ def B():
 
 @pytest.fixture
 def env():
-    saved = {k: os.environ.get(k) for k in ("OSC_DECODE", "OSC_DECODE_SPLIT")}
+    saved = {k: os.environ.get(k) for k in ("OSC_DECODE", "OSC_DECODE_SPLIT", "OSC_DECODE_FUSED_ROWS")}
 
-    def set_(decode, split=None):
+    def set_(decode, split=None, fused_rows=0):
         os.environ["OSC_DECODE"] = str(decode)
+        os.environ["OSC_DECODE_FUSED_ROWS"] = str(fused_rows)   # 0: the quantizer kernel runs in front
         if split is None:
             os.environ.pop("OSC_DECODE_SPLIT", None)
         else:
@@ -60,6 +61,9 @@ CASES = [  # M, K, N, table, split (None = the library's choice)
     (64, 1024, 448, "one", 4), (48, 2048, 256, "two", 8), (5, 256, 128, "empty", 1), (64, 128, 64, "full", 2),
     (31, 1536, 1024, "one", 5), (64, 4096, 512, "two", None), (20, 4096, 384, "two", 3), (64, 3072, 256, "one", 5),
     (32, 4096, 128, "two", 7),
+    # sixteen rows or fewer also run with the quantizer inside the kernel
+    (16, 4096, 384, "two", 3), (9, 640, 192, "two", 3), (16, 1536, 1024, "one", 5), (13, 128, 64, "full", 2),
+    (2, 3072, 256, "one", 8), (16, 2048, 128, "two", 1), (11, 1024, 64, "full", 4),
     # the 256-row form: one and two 128-row scale blocks of activations, token counts off the multiples of 16
     (65, 512, 192, "two", None), (128, 1024, 256, "one", 2), (129, 384, 320, "two", 3), (200, 2048, 128, "one", 4),
     (256, 640, 448, "two", 1), (250, 4096, 64, "two", 8), (144, 256, 128, "empty", 2), (256, 128, 64, "full", 2),
@@ -91,6 +95,21 @@ def test_decode_kernel_osc(B, oracle, env, M, K, N, kind, split):
     # the two kernels add the same exact products in different orders: equal up to fp32 rounding of the sums
     d = (outs[2].float() - outs[0].float()).abs().cpu().numpy().astype(np.float64)
     assert (d <= 2.0 ** -7 * np.abs(Yref) + 1e-3 * T).all()
+    if M <= 16:
+        # the form that quantizes the activations of its K slice inside the few-row kernel: no workspace traffic,
+        # the same codes, scales and accumulation order, hence the same bits
+        env(2, split, fused_rows=16)
+        ws = poison(sz.workspace_bytes)
+        before = ws.clone()
+        Ybig = torch.full((M + 2, N + 64), 7.0, dtype=torch.bfloat16, device="cuda")
+        Y = Ybig[1:M + 1, :N]
+        B.osc_linear(w, dev_bf16(c["X"]), Y, ws)
+        B.osc_sync_check()
+        assert torch.equal(ws, before), "the quantizing form does not use the workspace"
+        assert torch.equal(Y.view(torch.int16), outs[2].view(torch.int16))
+        guard = Ybig.clone()
+        guard[1:M + 1, :N] = 7.0
+        assert (guard == 7.0).all(), "wrote outside Y"
 
 
 @pytest.mark.parametrize("M,K,N,split", [(1, 128, 64, None), (16, 768, 320, 3), (40, 1536, 1024, 4), (64, 12288, 256, 8),
