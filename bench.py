@@ -311,6 +311,7 @@ def time_graph(torch, fn, n):
     """Milliseconds of GPU time per call when `n` calls are captured once in a CUDA graph and replayed: what a
     few-row (decode) step costs when the host does not pace the launches."""
     st = torch.cuda.Stream()
+    st.wait_stream(torch.cuda.current_stream())   # the problem's buffers and weights were prepared there
     with torch.cuda.stream(st):
         for i in range(3):
             fn(i)
