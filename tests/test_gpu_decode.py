@@ -195,8 +195,9 @@ def test_decode_kernel_nvfp4(B, oracle, env, M, K, N, kind, split):
         assert (guard == 7.0).all(), "wrote outside Y"
 
 
+@pytest.mark.parametrize("side_stream", [False, True], ids=["default_stream", "side_stream"])
 @pytest.mark.parametrize("kind", ["osc", "fp8", "mxfp8", "nvfp4"])
-def test_linear_right_after_prepare(B, oracle, kind):
+def test_linear_right_after_prepare(B, oracle, kind, side_stream):
     """A few-row linear issued on the same stream directly behind its weight preparation, with nothing in between:
     the few-row kernel streams weights ahead of its dependency wait, so the preparation has to be complete before
     any later launch may begin.  The buffers the preparation allocates are made to reuse memory full of 0xFF, so
@@ -214,6 +215,14 @@ def test_linear_right_after_prepare(B, oracle, kind):
     for nbytes in (N * K, N * K // 2, N * 4, N * 512 * 2, N * K // 32, N * K // 16, 1 << 20):
         poison(nbytes)
     torch.cuda.synchronize()
+    if side_stream:   # a stream of its own (non-blocking): programmatic launches overlap for certain
+        with torch.cuda.stream(torch.cuda.Stream()):
+            _right_after_prepare(B, oracle, kind, c, X, W, Y1, Y2, ws, M)
+    else:
+        _right_after_prepare(B, oracle, kind, c, X, W, Y1, Y2, ws, M)
+
+
+def _right_after_prepare(B, oracle, kind, c, X, W, Y1, Y2, ws, M):
     if kind == "osc":
         w = B.osc_prepare_weights(W, c["lut"])
         B.osc_linear(w, X, Y1, ws)

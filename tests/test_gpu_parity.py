@@ -348,6 +348,41 @@ def test_calls_can_be_captured_in_a_cuda_graph(B, oracle):
     assert outs[24].shape[0] == 24
 
 
+@pytest.mark.parametrize("M", [16, 64, 300, 1500])
+def test_back_to_back_calls_on_a_stream_of_their_own(B, M):
+    """Every kernel is launched as a programmatic dependent of the one in front; on a non-blocking stream of its own
+    the launches really overlap.  A chain of calls that reuse one workspace and feed each other (the output of a
+    linear is the input of the next) must give the bytes of the same calls with a synchronisation between them."""
+    K = N = 512
+    X_bits, W_bits, lut = make_case("rand2", M, N, K, 3)
+    X = dev_bf16(X_bits)
+    w = B.osc_prepare_weights(dev_bf16(W_bits), lut)
+    w8 = B.osc_fp8_prepare_weights(dev_bf16(W_bits))
+    ws = poison(max(B.osc_act_sizes(w, M).workspace_bytes, B.osc_fp8_act_sizes(w8, M).workspace_bytes))
+    torch.cuda.synchronize()
+
+    def chain(sync):
+        a, b = (torch.zeros((M, N), dtype=torch.bfloat16, device="cuda") for _ in range(2))
+        src = X
+        for i in range(6):
+            dst = a if i % 2 == 0 else b
+            if i % 3 == 2:
+                B.osc_fp8_linear(w8, src, dst, ws)
+            else:
+                B.osc_linear(w, src, dst, ws)
+            if sync:
+                torch.cuda.synchronize()
+            src = dst
+        torch.cuda.synchronize()
+        return src.clone()
+    want = chain(True)
+    with torch.cuda.stream(torch.cuda.Stream()):
+        got = chain(False)
+    B.osc_sync_check()
+    assert torch.isfinite(want.float()).all()
+    assert torch.equal(got.view(torch.int16), want.view(torch.int16))
+
+
 @pytest.mark.parametrize("kind", ["small", "mid"])
 def test_grouped_gather_equals_grouped_on_permuted_rows(B, oracle, kind):
     """Dispatch fused behind the quantizer: tokens quantized once, quantized rows gathered per expert.  Must equal the
