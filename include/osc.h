@@ -364,7 +364,8 @@ osc_status osc_rmsnorm_linear_swiglu(const osc_weights* w, const void* Hin, int 
  *        grouped projection into a scratch behind the workspace and the stand-alone activation.
  *   osc_linear_swiglu_grouped_gather / osc_rmsnorm_linear_swiglu_grouped_gather: the dispatch fused behind the quantizer
  *        (as osc_linear_grouped_gather / osc_rmsnorm_linear_grouped_gather); workspace: osc_swiglu_gather_workspace_bytes.
- *   Per expert the result equals the dense call on that expert's rows and weights bit for bit. */
+ *   Per expert the result equals the dense call on that expert's rows and weights: bit for bit where both run the CTA-pair
+ *   kernel (experts of more than 256 rows in a layer of large experts), within the fp32 accumulation-order rounding otherwise. */
 osc_status osc_gate_up_weight_sizes_grouped(int E, int I, int K, const int8_t* lut, int lut_c, osc_weight_sizes_t* out);
 osc_status osc_prepare_weights_gate_up_grouped(const void* W, int E, int I, int K, const int8_t* lut, int lut_c, void* wq,
                                                void* sfw, void* wo, void* meta, void* stream, osc_weights** out);

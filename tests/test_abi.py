@@ -166,6 +166,6 @@ def test_gate_up_calls_refuse_null_handles_and_odd_shapes():
     lut = np.full((16, 1), -1, np.int8)
     ws = B.WeightSizes()
     assert lib.osc_gate_up_weight_sizes_grouped(0, 64, 512, lut.ctypes.data, 1, C.byref(ws)) == -1     # no experts
-    assert lib.osc_gate_up_weight_sizes_grouped(2, 60, 512, lut.ctypes.data, 1, C.byref(ws)) == -2     # I not a multiple of 8
+    assert lib.osc_gate_up_weight_sizes_grouped(2, 60, 512, lut.ctypes.data, 1, C.byref(ws)) == -2     # I not a multiple of 64
     assert lib.osc_gate_up_weight_sizes_grouped(2, 64, 512, lut.ctypes.data, 1, C.byref(ws)) == 0
     assert ws.wq_bytes == 2 * 128 * 256

@@ -105,8 +105,9 @@ def test_rmsnorm_linear_swiglu_and_errors(B, oracle):
                                          ([3, 0, 130, 1, 257, 128], "gather"), ([17, 40, 3, 0, 25], "perm"),
                                          ([300, 0, 5, 256, 129, 511, 1, 385], "norm_gather")])
 def test_linear_swiglu_grouped(B, oracle, counts, mode):
-    """Grouped (MoE) gate|up projection with the SwiGLU in the epilogue: per expert bit for bit the dense call on that
-    expert's rows and weights, nothing written outside H, and within the pushed-through tolerance of the oracle."""
+    """Grouped (MoE) gate|up projection with the SwiGLU in the epilogue: per expert the dense call on that expert's rows
+    and weights (bit for bit where both take the CTA-pair kernel), nothing written outside H, and within the
+    pushed-through tolerance of the oracle."""
     from producer_inputs import gamma_bits
     counts = np.array(counts)
     E, K, I = counts.size, 384, 256
@@ -154,5 +155,8 @@ def test_linear_swiglu_grouped(B, oracle, counts, mode):
         Hd = torch.full((r1 - r0, I), float("nan"), dtype=torch.bfloat16, device="cuda")
         B.osc_linear_swiglu(wd, dev_bf16(Xp[r0:r1]), Hd, poison(B.osc_linear_swiglu_workspace_bytes(wd, r1 - r0)))
         B.osc_sync_check()
-        assert np.array_equal(got[r0:r1], host_bf16_bits(Hd)), f"expert {e} differs from the dense call"
+        if r1 - r0 > 256 and M >= 96 * E:   # both on the CTA-pair kernel's gate|up form: the same accumulation order
+            assert np.array_equal(got[r0:r1], host_bf16_bits(Hd)), f"expert {e} differs from the dense call"
+        else:                               # another kernel for the dense call: equal up to the rounding of the fp32 sums
+            assert (np.abs(Hf[r0:r1] - host_f64(Hd)) <= 2.0 * bound).all()
     assert not torch.isnan(H.float()).any()
