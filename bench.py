@@ -359,6 +359,7 @@ def per_call_times(torch, fn, iters, warm, graph_calls=0):
     so the host does not pace few-row launches."""
     if graph_calls:
         st = torch.cuda.Stream()
+        st.wait_stream(torch.cuda.current_stream())   # the problem's buffers and weights were prepared there
         out = []
         with torch.cuda.stream(st):
             for i in range(3):
