@@ -15,24 +15,14 @@ static __device__ __align__(256) unsigned char g_osc_static_scratch[OSC_STATIC_S
 
 namespace osc {
 
-constexpr int kMaxDevices = 64;
-// One slot per device ordinal.  Host threads may make their first call on a device at the same time: both then look
-// the address up and store the same value, so the slots are atomics like the library's other once-only caches.
-static std::atomic<void*> g_scratch_ptr[kMaxDevices] = {};
-
-// Device address of the scratch array on the current device; looked up once per device.
+// Device address of the scratch array on the current device.  Asked for on every call (a host-side table lookup in
+// the runtime): nothing is cached here, so host threads need no coordination and a context that was torn down and
+// created again is served with its own copy of the array.
 static osc_status static_scratch_address(void** out) {
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
-    if (dev < 0 || dev >= kMaxDevices) return fail(OSC_ERR_INVALID_ARG, "device index %d not supported", dev);
-    void* p = g_scratch_ptr[dev].load();
-    if (!p) {
-        e = cudaGetSymbolAddress(&p, g_osc_static_scratch);
-        if (e != cudaSuccess) return cuda_fail(e, "cudaGetSymbolAddress(static scratch)");
-        if (!p) return fail(OSC_ERR_CUDA, "cudaGetSymbolAddress returned a null address");
-        g_scratch_ptr[dev].store(p);
-    }
+    void* p = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&p, g_osc_static_scratch);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaGetSymbolAddress(static scratch)");
+    if (!p) return fail(OSC_ERR_CUDA, "cudaGetSymbolAddress returned a null address");
     *out = p;
     return OSC_OK;
 }
