@@ -26,6 +26,8 @@
  *     it remembers that device's SM count); call with that device current and a stream of that device.  One
  *     process per GPU is the intended arrangement: the path has no exchange step, so several GPUs run
  *     independent replicas (or disjoint row ranges of M) with no collective.
+ *     cudaDeviceReset (or any other loss of the device's context) invalidates every handle made on that device
+ *     and the kernel attributes the library set there: destroy the handles first and use a fresh process, or do not reset.
  *   - Threads: calls on distinct handles (or on one handle with distinct activation buffers and workspaces)
  *     may be made from several host threads at once; the library keeps no mutable state of its own beyond
  *     once-only caches (driver entry point, per-device kernel attributes) that are safe to race on.  Two
