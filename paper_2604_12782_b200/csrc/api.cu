@@ -1626,7 +1626,8 @@ osc_status osc_nvfp4_weight_sizes_grouped(int E, int N, int K, const int8_t* lut
     out->wq_bytes = (size_t)E * N * (K / 2);
     out->sfw_bytes = (size_t)E * sf16_bytes(N, K);
     out->wo_bytes = (size_t)E * N * t.Kop * 2;
-    out->meta_bytes = meta_table_bytes(K, t.Ko);
+    // dense: the per-tile copy of the weight scales for 240-wide tiles (scale blocks of 64 channels: twice the MXFP4 copy)
+    out->meta_bytes = meta_table_bytes(K, t.Ko) + (E == 1 ? 2 * tiled_sf_bytes(N, K) : 0);
     return OSC_OK;
 }
 
@@ -1678,9 +1679,15 @@ static osc_status nvfp4_prepare_impl(const void* W, int E, int N, int K, int64_t
                                        di.num_sms, ew, st);
         if (e != cudaSuccess) s = cuda_fail(e, "quant_extract_kernel(nvfp4 weights)");
     }
+    if (s == OSC_OK && !grouped) {   // 240-wide tiles read a per-tile copy of the weight scales (behind the table in meta)
+        uint8_t* tiled = m8 + meta_table_bytes(K, t.Ko);
+        e = launch_retile_sf(static_cast<const uint8_t*>(sfw), tiled, N, K, kTiledBN, st, false, 64);
+        if (e != cudaSuccess) s = cuda_fail(e, "retile_sf_kernel(nvfp4)");
+        if (s == OSC_OK) s = make_tmap_sf(&w->tm_sfw_tiled, tiled, (uint64_t)(2 * tiled_sf_bytes(N, K)) / 512, 4);
+    }
     if (s == OSC_OK && (e = launch_prepare_fence(st)) != cudaSuccess) s = cuda_fail(e, "prepare_fence_kernel");
-    for (int v = 0; v < 2 && s == OSC_OK; ++v) {
-        const int half = (v == 0 ? 192 : 256) / 2;
+    for (int v = 0; v < (grouped ? 2 : 3) && s == OSC_OK; ++v) {
+        const int half = (v == 0 ? 192 : v == 1 ? 256 : kTiledBN) / 2;
         s = make_tmap(&w->tm_b2[v], wq, false, (uint64_t)E * N, K / 2, K / 2, half);
         if (s == OSC_OK && t.Kop > 0)
             s = make_tmap(&w->tm_bo2[v], wo, true, (uint64_t)E * N, (uint64_t)t.Kop * 2, (uint64_t)t.Kop * 2, half);
@@ -1782,7 +1789,7 @@ static osc_status nvfp4_gemm_impl(const osc_weights* w, const void* xq, const vo
     long single_ns = 0, pair_ns = 0;
     const int bn1 = gemm_block_n(sched ? max_tiles : (M + 127) / 128, w->N, w->num_sms, &single_ns, 192);
     const long row_tiles2 = w->grouped ? (max_tiles2 > w->E / 2 ? max_tiles2 - w->E / 2 : 1) : (M + 255) / 256;
-    const int bn = gemm_pair_block_n(false, false, row_tiles2, w->N, nkb, w->num_sms, &pair_ns);
+    const int bn = gemm_pair_block_n(false, !w->grouped, row_tiles2, w->N, nkb, w->num_sms, &pair_ns);
     a.sched = sched; a.max_tiles = max_tiles;
     a.sched2 = sched2; a.max_tiles2 = max_tiles2;
     if (!use_pair_kernel(w->grouped, M, w->E, single_ns * nkb, pair_ns, single_ns <= 390)) {   // 128-row tiles
@@ -1802,12 +1809,13 @@ static osc_status nvfp4_gemm_impl(const osc_weights* w, const void* xq, const vo
         if (e != cudaSuccess) return cuda_fail(e, "gemm_kernel(nvfp4)");
         return OSC_OK;
     }
-    a.tm_b = w->tm_b2[bn == 256];
+    const int v2 = bn == 192 ? 0 : bn == 256 ? 1 : 2;
+    a.tm_b = w->tm_b2[v2];
     if (w->Kop > 0) {
         if (osc_status s = make_tmap(&a.tm_ao, xo, true, M, (uint64_t)w->Kop * 2, (uint64_t)w->Kop * 2, 128)) return s;
-        a.tm_bo = w->tm_bo2[bn == 256];
+        a.tm_bo = w->tm_bo2[v2];
     }
-    a.tm_sfw = w->tm_sfw;
+    a.tm_sfw = (bn == kTiledBN) ? w->tm_sfw_tiled : w->tm_sfw;
     const uint64_t sf_row_blocks = w->grouped ? (uint64_t)max_tiles : (uint64_t)((M + 127) / 128);
     if (osc_status s = make_tmap_sf(&a.tm_sfa, sfa, sf_row_blocks * (w->K / 64), 4)) return s;
     if (osc_status s = make_tmap(&a.tm_y, Y, true, M, (uint64_t)w->N * 2, (uint64_t)ldy * 2, 32)) return s;

@@ -147,6 +147,7 @@ cudaError_t launch_gemm_fp8_decode(const GemmArgs& a, int S, cudaStream_t st);
 cudaError_t launch_gemm_mxf8_decode(const GemmArgs& a, int S, cudaStream_t st);
 cudaError_t launch_gemm_nvf4_decode(const GemmArgs& a, int S, cudaStream_t st);
 int gemm_decode_split(int N, int nkb, int num_sms);
-cudaError_t launch_retile_sf(const uint8_t* src, uint8_t* dst, int N, int K, int bn, cudaStream_t st, bool gate_up = false);
+cudaError_t launch_retile_sf(const uint8_t* src, uint8_t* dst, int N, int K, int bn, cudaStream_t st, bool gate_up = false,
+                             int sf_channels = 128);
 
 }  // namespace osc

@@ -55,7 +55,11 @@ struct Cfg {
     static constexpr int KA = (MODE == MODE_OSC) ? 2 : (MODE == MODE_NVF4) ? 4 : 1;
     static constexpr bool DUAL = MODE == MODE_OSC || MODE == MODE_NVF4;   // has the BF16 branch (Path B)
     static constexpr int SF_K = (MODE == MODE_NVF4) ? 64 : 128;           // channels per scale block
-    static constexpr int SF_COLS = SCALED ? KA * (4 + SFB_ATOMS * 4) : 0;  // TMEM columns of one stage's scales
+    // Scale blocks of a stage that sit in TMEM at a time.  NVFP4 on 240-wide tiles has room for two of its four: the
+    // issuer copies two, issues their two instructions, copies the other two into the same columns and issues theirs
+    // (copies and multiplications of one thread run in the order they were issued).
+    static constexpr int KA_T = (MODE == MODE_NVF4 && TILED_SF) ? 2 : KA;
+    static constexpr int SF_COLS = SCALED ? KA_T * (4 + SFB_ATOMS * 4) : 0;  // TMEM columns of the scales in TMEM at a time
     static constexpr int ACC_STAGES = (2 * BN + SF_COLS <= TMEM_COLS) ? 2 : 1;
     static constexpr int SF_BUFS = (ACC_STAGES * BN + 2 * SF_COLS <= TMEM_COLS) ? 2 : 1;
     static constexpr int B_BYTES = (BN / 2) * ROW_BYTES;
@@ -80,13 +84,13 @@ struct Cfg {
     // weight scales at 496..511).
     static constexpr int ACC_STRIDE = TILED_SF ? 256 : BN;
     static constexpr int TM_SFA = TILED_SF ? BN : ACC_STAGES * BN;
-    static constexpr int TM_SFB = TILED_SF ? 256 + BN : TM_SFA + 4 * KA;
+    static constexpr int TM_SFB = TILED_SF ? 256 + BN : TM_SFA + 4 * KA_T;
     static constexpr int TM_SF_STRIDE = SF_COLS;         // columns of one scale buffer (when there are two)
     static constexpr uint32_t TX_A = 2u * (A_BYTES + B_BYTES + SFA_BYTES + SFB_BYTES);  // both CTAs, Path A
     static constexpr uint32_t TX_B = 2u * (A_BYTES + B_BYTES);                          // both CTAs, Path B / FP8
     static_assert(STAGE_BYTES % 1024 == 0, "stage must keep 1024-byte alignment");
     static_assert(B_BYTES % 1024 == 0, "weight half-tile must keep 1024-byte alignment");
-    static_assert(TILED_SF ? (TM_SFA + 4 * KA <= 256 && TM_SFB + KA * SFB_ATOMS * 4 <= TMEM_COLS && SF_BUFS == 1)
+    static_assert(TILED_SF ? (TM_SFA + 4 * KA_T <= 256 && TM_SFB + KA_T * SFB_ATOMS * 4 <= TMEM_COLS && SF_BUFS == 1)
                            : (TM_SFA + SF_BUFS * SF_COLS <= TMEM_COLS), "TMEM budget");
     static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
     static_assert(STAGES >= 3, "ring too shallow");
@@ -354,21 +358,26 @@ __global__ void __launch_bounds__(pair_threads(GU), 1) gemm_pair_kernel(const __
                             const uint64_t sfb_d = sf_hi | (uint64_t)((sbase + A_BYTES + C::B_BYTES + C::SFA_BYTES) >> 4);
                             const uint32_t sfo = (uint32_t)(C::SF_BUFS == 2 ? (kb & 1) : 0) * C::TM_SF_STRIDE;
 #pragma unroll
-                            for (int a = 0; a < 4; ++a) {
-                                if (a < ka) {
-                                    tc_copy_sf_pair(tmem_base + sfo + C::TM_SFA + a * 4, sfa_d + (uint64_t)(a * 32));
+                            for (int h = 0; h < 4 / C::KA_T; ++h) {   // KA_T blocks in TMEM at a time (all four, or two by two)
 #pragma unroll
-                                    for (int j = 0; j < C::SFB_ATOMS; ++j)
-                                        tc_copy_sf_pair(tmem_base + sfo + C::TM_SFB + a * (C::SFB_ATOMS * 4) + j * 4,
-                                                        sfb_d + (uint64_t)(j * (C::KA * 32) + a * 32));
+                                for (int t = 0; t < C::KA_T; ++t) {
+                                    const int a = h * C::KA_T + t;
+                                    if (a < ka) {
+                                        tc_copy_sf_pair(tmem_base + sfo + C::TM_SFA + t * 4, sfa_d + (uint64_t)(a * 32));
+#pragma unroll
+                                        for (int j = 0; j < C::SFB_ATOMS; ++j)
+                                            tc_copy_sf_pair(tmem_base + sfo + C::TM_SFB + t * (C::SFB_ATOMS * 4) + j * 4,
+                                                            sfb_d + (uint64_t)(j * (C::KA * 32) + a * 32));
+                                    }
                                 }
-                            }
 #pragma unroll
-                            for (int k = 0; k < 4; ++k) {
-                                if (k < ka)
-                                    mma_nvf4_pair(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC_A,
-                                                  tmem_base + sfo + C::TM_SFA + k * 4,
-                                                  sfb_tm + sfo + k * (C::SFB_ATOMS * 4), (kb | k) ? 1u : 0u);
+                                for (int t = 0; t < C::KA_T; ++t) {
+                                    const int k = h * C::KA_T + t;
+                                    if (k < ka)
+                                        mma_nvf4_pair(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC_A,
+                                                      tmem_base + sfo + C::TM_SFA + t * 4,
+                                                      sfb_tm + sfo + t * (C::SFB_ATOMS * 4), (kb | k) ? 1u : 0u);
+                                }
                             }
                         } else if (C::DUAL) {
 #pragma unroll
@@ -731,6 +740,7 @@ cudaError_t launch_gemm_mxf8_pair(const GemmArgs& a, int bn, cudaStream_t st) {
 }
 cudaError_t launch_gemm_nvf4_pair(const GemmArgs& a, int bn, cudaStream_t st) {
     if (bn == 192) return pair::launch_cfg<pair::MODE_NVF4, 192>(a, st);
+    if (bn == 240) return pair::launch_cfg<pair::MODE_NVF4, 240>(a, st);
     return pair::launch_cfg<pair::MODE_NVF4, 256>(a, st);
 }
 cudaError_t launch_gemm_fp8_pair(const GemmArgs& a, int bn, cudaStream_t st) {

@@ -704,8 +704,10 @@ build_sched_kernel(const int32_t* __restrict__ off, int E, int32_t* __restrict__
 // Block order: [tile][block of the tile][K block]; inside a block the usual 512-byte arrangement.
 // gate_up: the matrix holds gate rows [0, N/2) above up rows [N/2, N) and tile t covers bn/2 gate features followed
 // by the same bn/2 up features: row j of the tile is matrix row t*bn/2 + j (j < bn/2) or N/2 + t*bn/2 + j - bn/2.
-__global__ void retile_sf_kernel(const uint8_t* __restrict__ src, uint8_t* __restrict__ dst, int N, int K, int bn, int gate_up) {
-    const int katoms = K / 128;
+// sf_channels: channels per scale block (128: MXFP4 / MXFP8, 64: NVFP4).
+__global__ void retile_sf_kernel(const uint8_t* __restrict__ src, uint8_t* __restrict__ dst, int N, int K, int bn, int gate_up,
+                                 int sf_channels) {
+    const int katoms = K / sf_channels;
     const int atoms_per_tile = (bn + 127) / 128;
     const int ntiles = (N + bn - 1) / bn;
     const int64_t total = (int64_t)ntiles * atoms_per_tile * katoms * 512;
@@ -731,11 +733,12 @@ __global__ void retile_sf_kernel(const uint8_t* __restrict__ src, uint8_t* __res
     }
 }
 
-cudaError_t launch_retile_sf(const uint8_t* src, uint8_t* dst, int N, int K, int bn, cudaStream_t st, bool gate_up) {
-    const int64_t total = (int64_t)((N + bn - 1) / bn) * ((bn + 127) / 128) * (K / 128) * 512;
+cudaError_t launch_retile_sf(const uint8_t* src, uint8_t* dst, int N, int K, int bn, cudaStream_t st, bool gate_up,
+                             int sf_channels) {
+    const int64_t total = (int64_t)((N + bn - 1) / bn) * ((bn + 127) / 128) * (K / sf_channels) * 512;
     if (total <= 0) return cudaSuccess;
     const int blocks = (int)((total + 255) / 256 < 2048 ? (total + 255) / 256 : 2048);
-    retile_sf_kernel<<<blocks, 256, 0, st>>>(src, dst, N, K, bn, gate_up ? 1 : 0);
+    retile_sf_kernel<<<blocks, 256, 0, st>>>(src, dst, N, K, bn, gate_up ? 1 : 0, sf_channels);
     return cudaGetLastError();
 }
 
