@@ -64,6 +64,7 @@ CASES = [  # M, K, N, table, split (None = the library's choice)
     # sixteen rows or fewer also run with the quantizer inside the kernel
     (16, 4096, 384, "two", 3), (9, 640, 192, "two", 3), (16, 1536, 1024, "one", 5), (13, 128, 64, "full", 2),
     (2, 3072, 256, "one", 8), (16, 2048, 128, "two", 1), (11, 1024, 64, "full", 4),
+    (8, 2048, 128, "full", 2),      # more than 1024 flagged channels: the quantizer stays a kernel of its own
     # the 256-row form: one and two 128-row scale blocks of activations, token counts off the multiples of 16
     (65, 512, 192, "two", None), (128, 1024, 256, "one", 2), (129, 384, 320, "two", 3), (200, 2048, 128, "one", 4),
     (256, 640, 448, "two", 1), (250, 4096, 64, "two", 8), (144, 256, 128, "empty", 2), (256, 128, 64, "full", 2),
@@ -105,7 +106,7 @@ def test_decode_kernel_osc(B, oracle, env, M, K, N, kind, split):
         Y = Ybig[1:M + 1, :N]
         B.osc_linear(w, dev_bf16(c["X"]), Y, ws)
         B.osc_sync_check()
-        assert torch.equal(ws, before), "the quantizing form does not use the workspace"
+        assert torch.equal(ws, before) == (w.K_o_pad <= 1024), "the quantizing form does not use the workspace"
         assert torch.equal(Y.view(torch.int16), outs[2].view(torch.int16))
         guard = Ybig.clone()
         guard[1:M + 1, :N] = 7.0
