@@ -352,9 +352,10 @@ CALLS_PER_ITERATION = 4   # plain mode: consecutive calls between two events (an
                           # call's quantizer, which is how the linears of a layer follow each other)
 
 
-def per_call_times(torch, fn, iters, warm, graph_calls=0):
+def per_call_times(torch, fn, iters, warm, graph_calls=0, calls=0):
     """Milliseconds per call of fn(i), one sample per timed iteration.  Plain mode: a timed iteration is
-    CALLS_PER_ITERATION consecutive calls between two events (iters + 1 events on the current stream).  Graph mode
+    `calls` (default CALLS_PER_ITERATION) consecutive calls between two events (iters + 1 events on the current
+    stream).  Graph mode
     (graph_calls > 0): `graph_calls` calls are captured once in a CUDA graph and every timed iteration is one replay,
     so the host does not pace few-row launches."""
     if graph_calls:
@@ -384,7 +385,7 @@ def per_call_times(torch, fn, iters, warm, graph_calls=0):
         fn(i)
     torch.cuda.synchronize()
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(iters + 1)]
-    c = CALLS_PER_ITERATION
+    c = calls or CALLS_PER_ITERATION
     ev[0].record()
     for i in range(iters):
         for j in range(c):
@@ -431,7 +432,8 @@ def config_rows(torch, B, pk, iters=30, warm=5):
         settle()
         warm_ = stats(per_call_times(torch, lambda i: prob.step(0), iters, warm, gc))
         settle()
-        plain = stats(per_call_times(torch, prob.step, iters, warm))
+        # few-row calls last ~10 us: sixteen of them between two events, so that the events' own gap stays a few per cent
+        plain = stats(per_call_times(torch, prob.step, iters, warm, calls=16 if prob.M <= 128 else 0))
         return cold, warm_, plain, "cuda graph replay of %d calls per timed iteration" % gc
 
     def osc_row(name, M, K, N, cpg, seed):
